@@ -1,0 +1,256 @@
+/*
+ * fp64 CPU oracle for the Mixture-of-Depths Attention (MoDA) operator.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of the
+ * operator's definition that the CUDA path is checked against.  It shares no
+ * code with the CUDA path and must never be called from the product path.
+ *
+ * What it computes (paper Sec. 2.2 "Mixture-of-Depths Attention": every query
+ * attends to the causal sequence keys of its own layer and to its own depth
+ * keys from the preceding layers, all scores normalised by ONE softmax; scores
+ * and causal mask as in Eq. 2, M_ij = 0 iff j <= i; depth keys of a query are
+ * those stored at the SAME position, as in the Depth Attention paragraph):
+ *
+ *   for every batch b, head h, position t:
+ *     s_j = scale * <q_t, k_j>          j = 0..t        (sequence, causal inclusive)
+ *     u_i = scale * <q_t, kd_i[t]>      i = 0..l-1      (depth, always visible)
+ *     m   = max over all s_j, u_i
+ *     Z   = sum_j exp(s_j - m) + sum_i exp(u_i - m)
+ *     LSE_t = m + ln Z                                  (natural log)
+ *     O_t = ( sum_j exp(s_j-LSE) v_j + sum_i exp(u_i-LSE) vd_i[t] )
+ *
+ * Alg. 1 of the paper reaches the same values blockwise with an online softmax;
+ * because the result is exactly defined, the oracle is the definition itself:
+ * two passes per row (max, then sums), no tiling, no online rescaling.
+ *
+ * The backward pass is not printed in the paper; it is the derivative of the
+ * definition above with respect to every input, for a given dO:
+ *     D_t   = <dO_t, O_t>
+ *     dp_j  = <dO_t, v_j>          dr_i = <dO_t, vd_i[t]>
+ *     ds_j  = p_j (dp_j - D_t)     du_i = r_i (dr_i - D_t)
+ *     dQ_t  = scale ( sum_j ds_j k_j + sum_i du_i kd_i[t] )
+ *     dK_j  = scale sum_{t>=j} ds_tj q_t        dV_j = sum_{t>=j} p_tj dO_t
+ *     dKd_i[t] = scale du_i q_t                 dVd_i[t] = r_i dO_t
+ *
+ * Layouts (all row-major, double):
+ *     Q, K, V, O, dO, dQ, dK, dV : [B][T][H][d]
+ *     Kd, Vd, dKd, dVd           : [l][B][T][H][d]
+ *     LSE                        : [B][H][T]
+ *
+ * Pins (see tests/test_oracle_pins.py): masked library attention over the
+ * flattened key set, l = 0 against library causal attention, the two-softmax
+ * decomposition identity, closed forms, invariances, finite differences and
+ * library autograd, gradient sum identities.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdlib.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static inline size_t idx4(int b, int t, int h, int T, int H, int d)
+{
+    return (((size_t)b * T + t) * H + h) * (size_t)d;
+}
+
+static inline double dot(const double *a, const double *b, int d)
+{
+    double acc = 0.0;
+    for (int c = 0; c < d; ++c) acc += a[c] * b[c];
+    return acc;
+}
+
+int moda_oracle_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* One row of the forward definition.  s (length t+1) and u (length l) are
+ * scratch; on return they hold the probabilities p_j and r_i. */
+static void fwd_row(const double *Q, const double *K, const double *V,
+                    const double *Kd, const double *Vd,
+                    int B, int T, int H, int d, int l, double scale,
+                    int b, int h, int t,
+                    double *s, double *u, double *o_row, double *lse_out)
+{
+    const double *q = Q + idx4(b, t, h, T, H, d);
+    const size_t slot = (size_t)B * T * H * d;
+    double m = -INFINITY;
+    for (int j = 0; j <= t; ++j) {
+        s[j] = scale * dot(q, K + idx4(b, j, h, T, H, d), d);
+        if (s[j] > m) m = s[j];
+    }
+    for (int i = 0; i < l; ++i) {
+        u[i] = scale * dot(q, Kd + i * slot + idx4(b, t, h, T, H, d), d);
+        if (u[i] > m) m = u[i];
+    }
+    double Z = 0.0;
+    for (int j = 0; j <= t; ++j) Z += exp(s[j] - m);
+    for (int i = 0; i < l; ++i) Z += exp(u[i] - m);
+    const double lse = m + log(Z);
+    for (int c = 0; c < d; ++c) o_row[c] = 0.0;
+    for (int j = 0; j <= t; ++j) {
+        s[j] = exp(s[j] - lse);
+        const double *v = V + idx4(b, j, h, T, H, d);
+        for (int c = 0; c < d; ++c) o_row[c] += s[j] * v[c];
+    }
+    for (int i = 0; i < l; ++i) {
+        u[i] = exp(u[i] - lse);
+        const double *v = Vd + i * slot + idx4(b, t, h, T, H, d);
+        for (int c = 0; c < d; ++c) o_row[c] += u[i] * v[c];
+    }
+    *lse_out = lse;
+}
+
+/* Forward for every (b, h, t).  Returns 0, or -1 if scratch allocation fails. */
+int moda_oracle_fwd(const double *Q, const double *K, const double *V,
+                    const double *Kd, const double *Vd,
+                    int B, int T, int H, int d, int l, double scale,
+                    double *O, double *LSE)
+{
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(T + 1));
+        double *u = (double *)malloc(sizeof(double) * (size_t)(l + 1));
+        if (!s || !u) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+#pragma omp for collapse(3) schedule(dynamic, 8)
+            for (int b = 0; b < B; ++b)
+                for (int h = 0; h < H; ++h)
+                    for (int t = 0; t < T; ++t)
+                        fwd_row(Q, K, V, Kd, Vd, B, T, H, d, l, scale, b, h, t, s, u,
+                                O + idx4(b, t, h, T, H, d),
+                                LSE + ((size_t)b * H + h) * T + t);
+        }
+        free(s);
+        free(u);
+    }
+    return failed ? -1 : 0;
+}
+
+/* Forward for a list of sampled rows: rows[3*r + {0,1,2}] = (b, h, t).
+ * O_rows is [n_rows][d], LSE_rows is [n_rows]. */
+int moda_oracle_fwd_rows(const double *Q, const double *K, const double *V,
+                         const double *Kd, const double *Vd,
+                         int B, int T, int H, int d, int l, double scale,
+                         const int *rows, int n_rows,
+                         double *O_rows, double *LSE_rows)
+{
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(T + 1));
+        double *u = (double *)malloc(sizeof(double) * (size_t)(l + 1));
+        if (!s || !u) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+#pragma omp for schedule(dynamic, 1)
+            for (int r = 0; r < n_rows; ++r)
+                fwd_row(Q, K, V, Kd, Vd, B, T, H, d, l, scale,
+                        rows[3 * r], rows[3 * r + 1], rows[3 * r + 2], s, u,
+                        O_rows + (size_t)r * d, LSE_rows + r);
+        }
+        free(s);
+        free(u);
+    }
+    return failed ? -1 : 0;
+}
+
+/*
+ * Backward.  O and LSE are recomputed here in fp64 (the oracle never consumes
+ * a forward result from elsewhere).  Two sweeps so that no two threads ever
+ * add into the same output element:
+ *   sweep over query rows t  : dQ_t, dKd_i[t], dVd_i[t]   (row-local)
+ *   sweep over key rows j    : dK_j, dV_j = sums over t >= j
+ * Both sweeps evaluate p_tj = exp(s_tj - LSE_t) from the definition.
+ */
+int moda_oracle_bwd(const double *Q, const double *K, const double *V,
+                    const double *Kd, const double *Vd, const double *dO,
+                    int B, int T, int H, int d, int l, double scale,
+                    double *dQ, double *dK, double *dV, double *dKd, double *dVd)
+{
+    const size_t E = (size_t)B * T * H * d;
+    double *O = (double *)malloc(sizeof(double) * E);
+    double *LSE = (double *)malloc(sizeof(double) * (size_t)B * H * T);
+    double *Dl = (double *)malloc(sizeof(double) * (size_t)B * H * T);
+    if (!O || !LSE || !Dl) {
+        free(O); free(LSE); free(Dl);
+        return -1;
+    }
+    int rc = moda_oracle_fwd(Q, K, V, Kd, Vd, B, T, H, d, l, scale, O, LSE);
+    if (rc != 0) {
+        free(O); free(LSE); free(Dl);
+        return rc;
+    }
+
+    /* D_t = <dO_t, O_t> and the row-local gradients. */
+#pragma omp parallel for collapse(3) schedule(dynamic, 8)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h)
+            for (int t = 0; t < T; ++t) {
+                const size_t r = idx4(b, t, h, T, H, d);
+                const double *q = Q + r, *go = dO + r;
+                const double lse = LSE[((size_t)b * H + h) * T + t];
+                const double D = dot(go, O + r, d);
+                Dl[((size_t)b * H + h) * T + t] = D;
+                double *gq = dQ + r;
+                for (int c = 0; c < d; ++c) gq[c] = 0.0;
+                for (int j = 0; j <= t; ++j) {
+                    const double *k = K + idx4(b, j, h, T, H, d);
+                    const double p = exp(scale * dot(q, k, d) - lse);
+                    const double dp = dot(go, V + idx4(b, j, h, T, H, d), d);
+                    const double ds = p * (dp - D);
+                    for (int c = 0; c < d; ++c) gq[c] += scale * ds * k[c];
+                }
+                for (int i = 0; i < l; ++i) {
+                    const double *kd = Kd + i * E + r;
+                    const double rr = exp(scale * dot(q, kd, d) - lse);
+                    const double dr = dot(go, Vd + i * E + r, d);
+                    const double du = rr * (dr - D);
+                    double *gkd = dKd + i * E + r, *gvd = dVd + i * E + r;
+                    for (int c = 0; c < d; ++c) {
+                        gq[c] += scale * du * kd[c];
+                        gkd[c] = scale * du * q[c];
+                        gvd[c] = rr * go[c];
+                    }
+                }
+            }
+
+    /* dK_j, dV_j: sums over the queries t >= j that see key j. */
+#pragma omp parallel for collapse(3) schedule(dynamic, 8)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h)
+            for (int j = 0; j < T; ++j) {
+                const size_t rj = idx4(b, j, h, T, H, d);
+                const double *k = K + rj, *v = V + rj;
+                double *gk = dK + rj, *gv = dV + rj;
+                for (int c = 0; c < d; ++c) { gk[c] = 0.0; gv[c] = 0.0; }
+                for (int t = j; t < T; ++t) {
+                    const size_t rt = idx4(b, t, h, T, H, d);
+                    const double *q = Q + rt, *go = dO + rt;
+                    const size_t bt = ((size_t)b * H + h) * T + t;
+                    const double p = exp(scale * dot(q, k, d) - LSE[bt]);
+                    const double ds = p * (dot(go, v, d) - Dl[bt]);
+                    for (int c = 0; c < d; ++c) {
+                        gk[c] += scale * ds * q[c];
+                        gv[c] += p * go[c];
+                    }
+                }
+            }
+
+    free(O); free(LSE); free(Dl);
+    return 0;
+}

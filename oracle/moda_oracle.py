@@ -1,0 +1,140 @@
+"""ctypes front end of the fp64 CPU oracle (``moda_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by ``__graft_entry__.smoke()`` and by
+the CPU-baseline / ``--impl reference`` legs of ``bench.py``.  Nothing in the product
+package imports this module, and this module imports nothing from the product package.
+
+All arrays are numpy float64, C-contiguous, in the logical layouts of the paper's
+statement of the operator (Sec. 2.2, Alg. 1 input/output lines):
+
+    Q, K, V, O, dO, dQ, dK, dV : [B, T, H, d]
+    Kd, Vd, dKd, dVd           : [l, B, T, H, d]   (depth slot i = layer i's K, V)
+    LSE                        : [B, H, T]         (natural log, over sequence+depth keys)
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "moda_oracle.c")
+_LIB = os.path.join(_HERE, "libmoda_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+_dp = ctypes.POINTER(ctypes.c_double)
+_ip = ctypes.POINTER(ctypes.c_int)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain -O2, OpenMP; no fast-math). Returns the .so path."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + f".tmp{os.getpid()}"
+            cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.moda_oracle_threads.restype = ctypes.c_int
+        lib.moda_oracle_fwd.restype = ctypes.c_int
+        lib.moda_oracle_fwd.argtypes = [_dp] * 5 + [ctypes.c_int] * 5 + [ctypes.c_double, _dp, _dp]
+        lib.moda_oracle_fwd_rows.restype = ctypes.c_int
+        lib.moda_oracle_fwd_rows.argtypes = (
+            [_dp] * 5 + [ctypes.c_int] * 5 + [ctypes.c_double, _ip, ctypes.c_int, _dp, _dp]
+        )
+        lib.moda_oracle_bwd.restype = ctypes.c_int
+        lib.moda_oracle_bwd.argtypes = [_dp] * 6 + [ctypes.c_int] * 5 + [ctypes.c_double] + [_dp] * 5
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    """Number of OpenMP threads the oracle will use."""
+    return int(_load().moda_oracle_threads())
+
+
+def _f64(a, shape):
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    if a.shape != tuple(shape):
+        raise ValueError(f"expected shape {tuple(shape)}, got {a.shape}")
+    return a
+
+
+def _ptr(a):
+    return a.ctypes.data_as(_dp)
+
+
+def _prep(Q, K, V, Kd, Vd):
+    Q = np.ascontiguousarray(Q, dtype=np.float64)
+    if Q.ndim != 4:
+        raise ValueError("Q must be [B, T, H, d]")
+    B, T, H, d = Q.shape
+    K = _f64(K, (B, T, H, d))
+    V = _f64(V, (B, T, H, d))
+    l = 0 if Kd is None else int(np.shape(Kd)[0])
+    if l == 0:
+        Kd = np.zeros((0, B, T, H, d))
+        Vd = np.zeros((0, B, T, H, d))
+    Kd = _f64(Kd, (l, B, T, H, d))
+    Vd = _f64(Vd, (l, B, T, H, d))
+    return Q, K, V, Kd, Vd, (B, T, H, d, l)
+
+
+def forward(Q, K, V, Kd, Vd, scale):
+    """O [B,T,H,d] and LSE [B,H,T] of the MoDA operator (definition, fp64)."""
+    Q, K, V, Kd, Vd, (B, T, H, d, l) = _prep(Q, K, V, Kd, Vd)
+    O = np.empty((B, T, H, d))
+    LSE = np.empty((B, H, T))
+    rc = _load().moda_oracle_fwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(Kd), _ptr(Vd),
+                                 B, T, H, d, l, float(scale), _ptr(O), _ptr(LSE))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return O, LSE
+
+
+def forward_rows(Q, K, V, Kd, Vd, scale, rows):
+    """Forward for sampled rows only. ``rows`` is an int array [n, 3] of (b, h, t).
+
+    Returns O_rows [n, d] and LSE_rows [n]."""
+    Q, K, V, Kd, Vd, (B, T, H, d, l) = _prep(Q, K, V, Kd, Vd)
+    rows = np.ascontiguousarray(rows, dtype=np.int32).reshape(-1, 3)
+    if rows.size and not ((rows >= 0).all() and (rows[:, 0] < B).all()
+                          and (rows[:, 1] < H).all() and (rows[:, 2] < T).all()):
+        raise ValueError("row index out of range")
+    n = rows.shape[0]
+    O = np.empty((n, d))
+    LSE = np.empty((n,))
+    rc = _load().moda_oracle_fwd_rows(_ptr(Q), _ptr(K), _ptr(V), _ptr(Kd), _ptr(Vd),
+                                      B, T, H, d, l, float(scale),
+                                      rows.ctypes.data_as(_ip), n, _ptr(O), _ptr(LSE))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return O, LSE
+
+
+def backward(Q, K, V, Kd, Vd, dO, scale):
+    """dQ, dK, dV [B,T,H,d] and dKd, dVd [l,B,T,H,d] for upstream gradient dO."""
+    Q, K, V, Kd, Vd, (B, T, H, d, l) = _prep(Q, K, V, Kd, Vd)
+    dO = _f64(dO, (B, T, H, d))
+    dQ = np.empty((B, T, H, d))
+    dK = np.empty((B, T, H, d))
+    dV = np.empty((B, T, H, d))
+    dKd = np.empty((l, B, T, H, d))
+    dVd = np.empty((l, B, T, H, d))
+    rc = _load().moda_oracle_bwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(Kd), _ptr(Vd), _ptr(dO),
+                                 B, T, H, d, l, float(scale),
+                                 _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dKd), _ptr(dVd))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return dQ, dK, dV, dKd, dVd

@@ -1,0 +1,125 @@
+/*
+ * moda.h -- C ABI of the B200 (sm_100a) Mixture-of-Depths Attention (MoDA) operator.
+ *
+ * The operator (paper Sec. 2.2, "Mixture-of-Depths Attention"; forward schedule in
+ * Alg. 1): for every batch b, head h and position t, the query q_t attends, under ONE
+ * softmax, to
+ *     - the sequence keys/values of its own layer at positions 0..t (causal mask of
+ *       Eq. 2, inclusive of t), and
+ *     - the l depth keys/values stored for the SAME position t by the preceding layers
+ *       (slots i = 0..l-1; always visible).
+ *   s_j = scale <q_t,k_j>, u_i = scale <q_t,kd_i[t]>,
+ *   LSE_t = ln( sum_j e^{s_j} + sum_i e^{u_i} ),
+ *   O_t = sum_j e^{s_j-LSE_t} v_j + sum_i e^{u_i-LSE_t} vd_i[t].
+ * With l = 0 the operator is plain causal attention.
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers, 16-byte aligned, owned by the caller; the
+ *     library allocates no device memory and keeps no per-call state.
+ *   - bf16 = IEEE bfloat16 bits.  Q, K, V, O, dO, dQ, dK, dV are contiguous [B][T][H][d].
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work and return; they
+ *     never synchronise.  The current CUDA device must be the one that owns the buffers
+ *     and must be an sm_100 part.
+ *   - Return value: MODA_OK or a negative MODA_ERR_* code.  When an error is returned
+ *     nothing has been launched.  No C++ exception crosses the boundary, nothing prints.
+ *   - Supported shapes: B, T, H >= 1; d in {64, 128}; 0 <= l <= MODA_MAX_DEPTH.
+ *     T need not be a multiple of the 128-row tile.
+ *
+ * Depth-KV cache layout (chosen so that a warp whose lanes own consecutive query rows
+ * reads 512 contiguous bytes per load, and one (slot, b, h, tile, K|V) block is one
+ * contiguous 128*d*2-byte run that a bulk copy can move):
+ *
+ *     cache[slot][b][h][tile][kv][chunk][row][8]      (bf16)
+ *       slot  : depth slot 0..l_max-1 (layer index of the K, V that were appended)
+ *       tile  : position / 128, 0..ceil(T/128)-1        row : position % 128
+ *       kv    : 0 = key, 1 = value                      chunk : feature / 8, 0..d/8-1
+ *     rows of the last tile beyond T are zero.  One slot spans
+ *     moda_depth_cache_bytes(B,T,H,d,1) bytes, so the layer-l call simply reads the first
+ *     l slots of a buffer that grows by one slot per layer ("write" step of Sec. 2.2).
+ */
+#ifndef MODA_H
+#define MODA_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MODA_MAX_DEPTH 32
+
+#define MODA_OK 0
+#define MODA_ERR_NULL_POINTER (-1)    /* a required pointer is null */
+#define MODA_ERR_MISALIGNED (-2)      /* a tensor pointer is not 16-byte aligned */
+#define MODA_ERR_BAD_SHAPE (-3)       /* B, T or H < 1, or a size product overflows */
+#define MODA_ERR_BAD_HEAD_DIM (-4)    /* d not in {64, 128} */
+#define MODA_ERR_BAD_DEPTH (-5)       /* l outside [0, MODA_MAX_DEPTH] */
+#define MODA_ERR_BAD_SLOT (-6)        /* slot outside [0, MODA_MAX_DEPTH) */
+#define MODA_ERR_WORKSPACE (-7)       /* workspace null or smaller than required */
+#define MODA_ERR_DEVICE (-8)          /* current device is not sm_100 */
+#define MODA_ERR_CUDA (-9)            /* a CUDA runtime/driver call failed (see moda_last_cuda_error) */
+#define MODA_ERR_DEVICE_TIMEOUT (-10) /* an earlier kernel gave up a bounded wait (see moda_last_status) */
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int moda_version(void);
+
+/* Static, human-readable text for a MODA_* code. */
+const char* moda_strerror(int code);
+
+/* cudaError_t value of the last failing CUDA call seen by this thread (0 if none). */
+int moda_last_cuda_error(void);
+
+/*
+ * Reads (and optionally clears) the device status word.  Every wait inside the kernels
+ * is bounded; a wait that runs out stores (site << 8) | 1 here and the kernel tears
+ * down normally, leaving its outputs undefined.  0 means no kernel has reported a
+ * problem.  This call synchronises the device.  Returns the status word (>= 0) or a
+ * negative MODA_ERR_CUDA.
+ */
+int moda_last_status(int clear);
+
+/* Bytes of a depth-KV cache (or depth-gradient buffer) holding l_max slots. 0 on bad arguments. */
+size_t moda_depth_cache_bytes(int B, int T, int H, int d, int l_max);
+
+/*
+ * "Write" step of Sec. 2.2: store one layer's keys and values, K_i and V_i (bf16
+ * [B][T][H][d]), into slot `slot` of `cache` in the layout above (tail rows zeroed).
+ */
+int moda_depth_cache_append(void* cache, int B, int T, int H, int d, int slot,
+                            const void* K_i, const void* V_i, void* stream);
+
+/* Inverse of append: copy slot `slot` of `cache` back to [B][T][H][d] tensors (either output may be null). */
+int moda_depth_cache_unpack(const void* cache, int B, int T, int H, int d, int slot,
+                            void* K_i, void* V_i, void* stream);
+
+/*
+ * Forward (Sec. 2.2 definition; Alg. 1 computes the same values with an online
+ * softmax).  depth_kv holds at least l slots in the cache layout (may be null when
+ * l == 0).  Writes O (bf16 [B][T][H][d]) and LSE (fp32 [B][H][T], natural log, taken over
+ * the union of sequence and depth keys).  bf16 inputs, fp32 accumulation and softmax.
+ */
+int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth_kv,
+                  int B, int T, int H, int d, int l, float scale,
+                  void* O, float* LSE, void* stream);
+
+/* Bytes of scratch moda_attn_bwd needs (fp32 row terms D_t = <dO_t, O_t>). */
+size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l);
+
+/*
+ * Backward of the definition above (the paper prints no backward pass; it is the
+ * derivative of Sec. 2.2's operator).  Inputs as for the forward call plus O, LSE as
+ * written by it and the upstream gradient dO.  Writes dQ, dK, dV (bf16 [B][T][H][d]) and,
+ * when l > 0, slots 0..l-1 of d_depth_kv (bf16, cache layout: kv = 0 holds dKd, kv = 1
+ * holds dVd; tail rows zero).  `workspace` is caller-owned scratch of at least
+ * moda_bwd_workspace_bytes() bytes; its contents need not be preserved between calls.
+ */
+int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth_kv,
+                  const void* O, const void* dO, const float* LSE,
+                  int B, int T, int H, int d, int l, float scale,
+                  void* dQ, void* dK, void* dV, void* d_depth_kv,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MODA_H */

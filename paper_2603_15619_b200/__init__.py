@@ -1,0 +1,18 @@
+"""B200 (sm_100a) implementation of the Mixture-of-Depths Attention operator.
+
+``binding`` exposes the C ABI of ``include/moda.h`` (hand-written CUDA kernels behind it);
+``synthetic`` holds the seeded input recipes; ``flops`` the FLOP / byte accounting of the
+reported metric.  The CUDA library is loaded on first use and there is no fallback path.
+"""
+from .binding import (  # noqa: F401
+    ModaError,
+    alloc_depth_cache,
+    moda_attn_bwd,
+    moda_attn_fwd,
+    moda_bwd_workspace_bytes,
+    moda_depth_cache_append,
+    moda_depth_cache_bytes,
+    moda_depth_cache_unpack,
+    moda_last_status,
+    moda_version,
+)

@@ -1,0 +1,174 @@
+"""ctypes binding of libmoda_b200.so: same names as the C ABI in include/moda.h.
+
+Argument marshalling only -- every step of the operator runs in the CUDA kernels behind
+the C entry points.  Tensors are torch CUDA tensors (PyTorch supplies device memory and
+streams, nothing else).  There is no CPU fallback: if the library cannot be loaded, or a
+call returns an error code, a ``ModaError`` is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmoda_b200.so")
+
+MODA_MAX_DEPTH = 32
+SYMBOLS = (
+    "moda_version", "moda_strerror", "moda_last_cuda_error", "moda_last_status",
+    "moda_depth_cache_bytes", "moda_depth_cache_append", "moda_depth_cache_unpack",
+    "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd",
+)
+
+
+class ModaError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what} failed: [{code}] {strerror(code)}"
+                         + (f" (cudaError {last_cuda_error()})" if code == -9 else ""))
+        self.code = code
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load the CUDA library (raises if it has not been built: there is no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2603_15619_b200.build` "
+            "(or __graft_entry__.build()). The MoDA operator has no CPU or PyTorch fallback.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.moda_version.restype = ci
+    lib.moda_strerror.restype = ctypes.c_char_p
+    lib.moda_strerror.argtypes = [ci]
+    lib.moda_last_cuda_error.restype = ci
+    lib.moda_last_status.restype = ci
+    lib.moda_last_status.argtypes = [ci]
+    lib.moda_depth_cache_bytes.restype = sz
+    lib.moda_depth_cache_bytes.argtypes = [ci] * 5
+    lib.moda_depth_cache_append.restype = ci
+    lib.moda_depth_cache_append.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp]
+    lib.moda_depth_cache_unpack.restype = ci
+    lib.moda_depth_cache_unpack.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp]
+    lib.moda_attn_fwd.restype = ci
+    lib.moda_attn_fwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp]
+    lib.moda_bwd_workspace_bytes.restype = sz
+    lib.moda_bwd_workspace_bytes.argtypes = [ci] * 5
+    lib.moda_attn_bwd.restype = ci
+    lib.moda_attn_bwd.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 5 + [sz, vp]
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("device (CUDA) tensors required")
+    if not t.is_contiguous():
+        raise ValueError("contiguous tensors required")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise ModaError(rc, what)
+
+
+def _bthd(t, name):
+    if t.dtype != torch.bfloat16 or t.dim() != 4:
+        raise ValueError(f"{name} must be a bf16 [B, T, H, d] tensor")
+    return tuple(t.shape)
+
+
+def moda_version() -> int:
+    return int(load().moda_version())
+
+
+def strerror(code: int) -> str:
+    return load().moda_strerror(int(code)).decode()
+
+
+def last_cuda_error() -> int:
+    return int(load().moda_last_cuda_error())
+
+
+def moda_last_status(clear: bool = False) -> int:
+    """Device status word (0 = no kernel gave up a wait). Synchronises the device."""
+    return int(load().moda_last_status(int(clear)))
+
+
+def moda_depth_cache_bytes(B, T, H, d, l_max) -> int:
+    return int(load().moda_depth_cache_bytes(B, T, H, d, l_max))
+
+
+def alloc_depth_cache(B, T, H, d, l_max, device="cuda") -> torch.Tensor:
+    """Caller-side helper: a bf16 buffer of moda_depth_cache_bytes() bytes (uninitialised)."""
+    n = moda_depth_cache_bytes(B, T, H, d, l_max)
+    if n == 0 and l_max != 0:
+        raise ValueError("bad depth-cache shape")
+    return torch.empty(max(n // 2, 8), dtype=torch.bfloat16, device=device)
+
+
+def moda_depth_cache_append(cache, slot, K_i, V_i, stream=None):
+    B, T, H, d = _bthd(K_i, "K_i")
+    assert _bthd(V_i, "V_i") == (B, T, H, d)
+    _check(load().moda_depth_cache_append(_ptr(cache), B, T, H, d, int(slot), _ptr(K_i), _ptr(V_i), _stream(stream)),
+           "moda_depth_cache_append")
+
+
+def moda_depth_cache_unpack(cache, slot, K_i, V_i, stream=None):
+    ref = K_i if K_i is not None else V_i
+    B, T, H, d = _bthd(ref, "K_i/V_i")
+    _check(load().moda_depth_cache_unpack(_ptr(cache), B, T, H, d, int(slot), _ptr(K_i), _ptr(V_i), _stream(stream)),
+           "moda_depth_cache_unpack")
+
+
+def moda_attn_fwd(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):
+    """O [B,T,H,d] bf16 and LSE [B,H,T] fp32 of the MoDA operator (outputs allocated if not given)."""
+    B, T, H, d = _bthd(Q, "Q")
+    assert _bthd(K, "K") == (B, T, H, d) and _bthd(V, "V") == (B, T, H, d)
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None:
+        LSE = torch.empty((B, H, T), dtype=torch.float32, device=Q.device)
+    _check(load().moda_attn_fwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
+                                B, T, H, d, int(l), float(scale), _ptr(O), _ptr(LSE), _stream(stream)),
+           "moda_attn_fwd")
+    return O, LSE
+
+
+def moda_bwd_workspace_bytes(B, T, H, d, l) -> int:
+    return int(load().moda_bwd_workspace_bytes(B, T, H, d, l))
+
+
+def moda_attn_bwd(Q, K, V, depth_kv, O, dO, LSE, l, scale,
+                  dQ=None, dK=None, dV=None, d_depth_kv=None, workspace=None, stream=None):
+    """dQ, dK, dV [B,T,H,d] bf16 and the depth gradients (cache layout, slots < l)."""
+    B, T, H, d = _bthd(Q, "Q")
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(Q) if dK is None else dK
+    dV = torch.empty_like(Q) if dV is None else dV
+    if l > 0 and d_depth_kv is None:
+        d_depth_kv = alloc_depth_cache(B, T, H, d, l, Q.device)
+    need = moda_bwd_workspace_bytes(B, T, H, d, l)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
+    _check(load().moda_attn_bwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
+                                _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, d, int(l), float(scale),
+                                _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
+                                _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "moda_attn_bwd")
+    return dQ, dK, dV, d_depth_kv

@@ -1,0 +1,232 @@
+// C ABI of the MoDA operator (see include/moda.h): argument validation, tensor-map
+// construction and kernel launches.  Everything that computes lives in the kernels.
+#include "../../include/moda.h"
+
+#include <cstdint>
+#include <cstring>
+#include <mutex>
+
+#include "moda_bwd.cuh"
+#include "moda_cache.cuh"
+#include "moda_fwd.cuh"
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace moda;
+
+thread_local int tl_last_cuda_error = 0;
+
+inline bool cuda_ok(cudaError_t e) {
+    if (e == cudaSuccess) return true;
+    tl_last_cuda_error = static_cast<int>(e);
+    (void)cudaGetLastError();   // clear the sticky-free error so that later calls start clean
+    return false;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// Tensor map over a contiguous bf16 [B][T][H][d] tensor; one box = 128 positions x 64
+// features of one (b, h), written to shared memory with the 128-byte swizzle.
+// Out-of-range rows (ragged last tile) read as zero and are dropped on store.
+bool make_bthd_map(CUtensorMap* map, const void* base, int B, int T, int H, int d) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) { tl_last_cuda_error = static_cast<int>(cudaErrorNotSupported); return false; }
+    const cuuint64_t dims[4] = {cuuint64_t(d), cuuint64_t(H), cuuint64_t(T), cuuint64_t(B)};
+    const cuuint64_t strides[3] = {cuuint64_t(d) * 2, cuuint64_t(H) * d * 2, cuuint64_t(T) * H * d * 2};
+    const cuuint32_t box[4] = {64, 1, cuuint32_t(kTileRows), 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { tl_last_cuda_error = static_cast<int>(cudaErrorInvalidValue); return false; }
+    return true;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(int B, int T, int H, int d) {
+    if (B < 1 || T < 1 || H < 1) return MODA_ERR_BAD_SHAPE;
+    if (d != 64 && d != 128) return MODA_ERR_BAD_HEAD_DIM;
+    // keep every element count and grid size inside 31 / 63 bits
+    const long long rows = (long long)B * H * num_tiles(T);
+    if (rows > 0x3fffffffLL) return MODA_ERR_BAD_SHAPE;
+    if ((long long)B * T > 0x7fffffffLL / H) return MODA_ERR_BAD_SHAPE;
+    return MODA_OK;
+}
+
+int check_device() {
+    static thread_local int cached_dev = -1;
+    static thread_local int cached_rc = MODA_ERR_DEVICE;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (dev == cached_dev) return cached_rc;
+    int major = 0;
+    if (!cuda_ok(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev))) return MODA_ERR_CUDA;
+    cached_dev = dev;
+    cached_rc = (major == 10) ? MODA_OK : MODA_ERR_DEVICE;
+    return cached_rc;
+}
+
+template <typename Kernel>
+bool set_smem_limit(Kernel k, int bytes) {
+    return cuda_ok(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+}
+
+template <int D>
+int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int H, int l,
+               float scale, void* O, float* LSE, cudaStream_t stream) {
+    CUtensorMap mQ, mK, mV, mO;
+    if (!make_bthd_map(&mQ, Q, B, T, H, D) || !make_bthd_map(&mK, K, B, T, H, D) ||
+        !make_bthd_map(&mV, V, B, T, H, D) || !make_bthd_map(&mO, O, B, T, H, D))
+        return MODA_ERR_CUDA;
+    static thread_local int configured_dev = -1;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (configured_dev != dev) {
+        if (!set_smem_limit(moda_fwd_kernel<D>, FwdSmem<D>::kDynamic)) return MODA_ERR_CUDA;
+        configured_dev = dev;
+    }
+    FwdParams p;
+    p.depth_kv = static_cast<const __nv_bfloat16*>(depth_kv);
+    p.O = static_cast<__nv_bfloat16*>(O);
+    p.LSE = LSE;
+    p.B = B; p.T = T; p.H = H; p.l = l;
+    p.scale_log2 = scale * kLog2e;
+    const unsigned grid = unsigned(B) * H * num_tiles(T);
+    moda_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kDynamic, stream>>>(mQ, mK, mV, mO, p);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+
+template <int D, bool kToCache>
+int launch_cache_copy(void* cache, int B, int T, int H, int slot, void* Xk, void* Xv, cudaStream_t stream) {
+    uint4* slot_base = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(cache) + size_t(slot) * cache_slot_elems(B, T, H, D));
+    const unsigned grid = unsigned(B) * H * num_tiles(T) * 2;
+    depth_cache_copy_kernel<D, kToCache><<<grid, 256, 0, stream>>>(slot_base, static_cast<uint4*>(Xk), static_cast<uint4*>(Xv), T, H);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int moda_version(void) { return 100; }
+
+const char* moda_strerror(int code) {
+    switch (code) {
+        case MODA_OK: return "ok";
+        case MODA_ERR_NULL_POINTER: return "a required pointer is null";
+        case MODA_ERR_MISALIGNED: return "a tensor pointer is not 16-byte aligned";
+        case MODA_ERR_BAD_SHAPE: return "B, T and H must be >= 1 and the tensor must fit 31-bit row counts";
+        case MODA_ERR_BAD_HEAD_DIM: return "head width d must be 64 or 128";
+        case MODA_ERR_BAD_DEPTH: return "depth l must be in [0, 32]";
+        case MODA_ERR_BAD_SLOT: return "depth slot must be in [0, 32)";
+        case MODA_ERR_WORKSPACE: return "workspace is null or too small";
+        case MODA_ERR_DEVICE: return "the current CUDA device is not an sm_100 part";
+        case MODA_ERR_CUDA: return "a CUDA call failed (see moda_last_cuda_error)";
+        case MODA_ERR_DEVICE_TIMEOUT: return "a kernel gave up a bounded wait (see moda_last_status)";
+        default: return "unknown error code";
+    }
+}
+
+int moda_last_cuda_error(void) { return tl_last_cuda_error; }
+
+int moda_last_status(int clear) {
+    int st = 0;
+    if (!cuda_ok(cudaDeviceSynchronize())) return MODA_ERR_CUDA;
+    if (!cuda_ok(cudaMemcpyFromSymbol(&st, g_moda_status, sizeof(int)))) return MODA_ERR_CUDA;
+    if (clear && st != 0) {
+        const int zero = 0;
+        if (!cuda_ok(cudaMemcpyToSymbol(g_moda_status, &zero, sizeof(int)))) return MODA_ERR_CUDA;
+    }
+    return st;
+}
+
+size_t moda_depth_cache_bytes(int B, int T, int H, int d, int l_max) {
+    if (check_shape(B, T, H, d) != MODA_OK || l_max < 0 || l_max > MODA_MAX_DEPTH) return 0;
+    return size_t(l_max) * cache_slot_elems(B, T, H, d) * 2;
+}
+
+int moda_depth_cache_append(void* cache, int B, int T, int H, int d, int slot,
+                            const void* K_i, const void* V_i, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (slot < 0 || slot >= MODA_MAX_DEPTH) return MODA_ERR_BAD_SLOT;
+    if (!cache || !K_i || !V_i) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(cache) || !aligned16(K_i) || !aligned16(V_i)) return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_cache_copy<128, true>(cache, B, T, H, slot, const_cast<void*>(K_i), const_cast<void*>(V_i), st)
+                    : launch_cache_copy<64, true>(cache, B, T, H, slot, const_cast<void*>(K_i), const_cast<void*>(V_i), st);
+}
+
+int moda_depth_cache_unpack(const void* cache, int B, int T, int H, int d, int slot,
+                            void* K_i, void* V_i, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (slot < 0 || slot >= MODA_MAX_DEPTH) return MODA_ERR_BAD_SLOT;
+    if (!cache || (!K_i && !V_i)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(cache) || !aligned16(K_i) || !aligned16(V_i)) return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_cache_copy<128, false>(const_cast<void*>(cache), B, T, H, slot, K_i, V_i, st)
+                    : launch_cache_copy<64, false>(const_cast<void*>(cache), B, T, H, slot, K_i, V_i, st);
+}
+
+int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth_kv,
+                  int B, int T, int H, int d, int l, float scale,
+                  void* O, float* LSE, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (!Q || !K || !V || !O || !LSE || (l > 0 && !depth_kv)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
+        (l > 0 && !aligned16(depth_kv)))
+        return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv, B, T, H, l, scale, O, LSE, st)
+                    : launch_fwd<64>(Q, K, V, depth_kv, B, T, H, l, scale, O, LSE, st);
+}
+
+size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l) {
+    if (check_shape(B, T, H, d) != MODA_OK || l < 0 || l > MODA_MAX_DEPTH) return 0;
+    return bwd_workspace_bytes(B, T, H);
+}
+
+int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth_kv,
+                  const void* O, const void* dO, const float* LSE,
+                  int B, int T, int H, int d, int l, float scale,
+                  void* dQ, void* dK, void* dV, void* d_depth_kv,
+                  void* workspace, size_t workspace_bytes, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv || !d_depth_kv)))
+        return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(LSE) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) ||
+        (l > 0 && (!aligned16(depth_kv) || !aligned16(d_depth_kv))))
+        return MODA_ERR_MISALIGNED;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < bwd_workspace_bytes(B, T, H)) return MODA_ERR_WORKSPACE;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    BwdArgs a;
+    a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv; a.O = O; a.dO = dO; a.LSE = LSE;
+    a.B = B; a.T = T; a.H = H; a.l = l; a.scale = scale;
+    a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
+    return d == 128 ? launch_bwd<128>(a, st) : launch_bwd<64>(a, st);
+}
+
+}  // extern "C"

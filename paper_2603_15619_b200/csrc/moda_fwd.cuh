@@ -1,0 +1,481 @@
+// MoDA forward kernel for sm_100a (Sec. 2.2 definition; Alg. 1 gives the blockwise
+// online-softmax schedule this kernel re-designs for tcgen05 / TMEM / TMA).
+//
+// One CTA owns one (b, h, 128-query-row tile).  320 threads, five roles:
+//
+//   warps 0-3  softmax   one thread per query row.  Reads the score tile S_j from TMEM,
+//                        keeps the running (m, l) of the online softmax in registers, writes
+//                        P_j = exp2(S_j c - m) as packed bf16 back into the TMEM columns of
+//                        S_j, rescales the O accumulator only when the running maximum grew
+//                        by more than 2^8, and runs the epilogue.
+//   warps 4-7  depth     one thread per query row.  Reads the row's l depth keys/values
+//                        straight from the depth cache (16-byte loads, a warp reads 512
+//                        contiguous bytes), builds an independent partial softmax state
+//                        (m_d, l_d, o_d) on the CUDA cores and parks o_d in TMEM.  Merging
+//                        two partial softmax states is exact, so the epilogue obtains the
+//                        single softmax over sequence and depth keys that the paper defines.
+//   warp 8     TMA       one lane streams the Q tile and the K_j / V_j tiles (128B swizzle)
+//                        through two-stage rings.
+//   warp 9     MMA       (warps 10, 11 idle: they complete the third warpgroup so that
+//                        registers can be re-balanced between warpgroups)
+//                        one lane issues S_j = Q K_j^T (operands in shared memory) and
+//                        O += P_j V_j (P_j from TMEM, V_j MN-major in shared memory); also
+//                        owns the TMEM allocation.
+//
+// TMEM columns (fp32): [0,128) S_0/P_0   [128,256) S_1/P_1   [256,256+D) O   [384,384+D) o_d.
+// The depth scores never touch the tensor cores and no score matrix is ever materialised.
+#pragma once
+
+#include "moda_cache.cuh"
+#include "sm100_ptx.cuh"
+
+namespace moda {
+
+constexpr int kFwdThreads = 384;   // three warpgroups: softmax, depth, {TMA, MMA, 2 idle warps}
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;   // log2 units
+
+template <int D>
+struct FwdSmem {
+    static constexpr int kTileBytes = kTileRows * D * 2;          // one 128 x D bf16 tile
+    static constexpr int kSubBytes = kTileRows * 128;             // one 128 x 64 sub-tile
+    static constexpr int kQ = 0;
+    static constexpr int kK = kQ + kTileBytes;                    // 2 stages
+    static constexpr int kV = kK + 2 * kTileBytes;                // 2 stages
+    static constexpr int kU = kV + 2 * kTileBytes;                // depth scores [32][128] fp32
+    static constexpr int kMd = kU + 32 * kTileRows * 4;           // m_d [128], l_d [128]
+    static constexpr int kBars = kMd + 2 * kTileRows * 4;
+    static constexpr int kNumBars = 18;
+    static constexpr int kMisc = kBars + kNumBars * 8;            // tmem base, abort flag
+    static constexpr int kTotal = kMisc + 16;
+    static constexpr int kDynamic = kTotal + 1024;                // slack for 1024-byte alignment
+};
+
+enum FwdBar : int {
+    kBarQ = 0,
+    kBarKFull = 1,    // +stage
+    kBarKEmpty = 3,   // +stage
+    kBarVFull = 5,    // +stage
+    kBarVEmpty = 7,   // +stage
+    kBarSFull = 9,    // +buffer
+    kBarPFull = 11,   // +buffer
+    kBarOReady = 13,  // one phase per PV_j (used by the lazy rescale, which knows PV_{j-2} is complete)
+    kBarDepth = 14,
+    kBarOFinal = 15,  // single phase: every MMA of the CTA has completed
+    kBarDrain = 16,
+};
+
+struct FwdParams {
+    const __nv_bfloat16* depth_kv;   // cache layout, >= l slots (unused when l == 0)
+    __nv_bfloat16* O;
+    float* LSE;
+    int B, T, H, l;
+    float scale_log2;                // scale * log2(e)
+};
+
+// Shared-memory address of 16-byte chunk `c` (0..D/8-1) of row `r` inside a 128 x D tile that
+// TMA wrote as D/64 sub-tiles of [128][64] with the 128-byte swizzle.
+__device__ __forceinline__ uint32_t swz_chunk_offset(int r, int c) {
+    return uint32_t(c >> 3) * uint32_t(kTileRows * 128) + uint32_t(r) * 128u + (uint32_t((c & 7) ^ (r & 7)) << 4);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kFwdThreads, 1)
+moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
+                const FwdParams p) {
+    using L = FwdSmem<D>;
+    constexpr int NSUB = D / 64;
+    constexpr int CH = D / 8;
+    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t kColO = 256, kColOd = 384;
+
+    if (g_moda_status != 0) return;   // an earlier kernel gave up a wait: do not pile up more timeouts
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    float* sU = reinterpret_cast<float*>(smem + L::kU);
+    float* sMd = reinterpret_cast<float*>(smem + L::kMd);
+    float* sLd = sMd + kTileRows;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 4);
+    auto bar = [&](int i) { return sbase + L::kBars + 8u * uint32_t(i); };
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+
+    const int nq = num_tiles(p.T);
+    const int bh = blockIdx.x / nq;
+    const int qt = nq - 1 - (blockIdx.x % nq);      // heaviest query tiles of a head first
+    const int b = bh / p.H, h = bh % p.H;
+    const int q0 = qt * kTileRows;
+    const int n_kv = qt + 1;                         // causal: key tiles 0..qt
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(kBarQ), 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(kBarKFull + s), 1);
+            mbar_init(bar(kBarKEmpty + s), 1);
+            mbar_init(bar(kBarVFull + s), 1);
+            mbar_init(bar(kBarVEmpty + s), 1);
+            mbar_init(bar(kBarSFull + s), 1);
+            mbar_init(bar(kBarPFull + s), 128);
+        }
+        mbar_init(bar(kBarOReady), 1);
+        mbar_init(bar(kBarDepth), 128);
+        mbar_init(bar(kBarOFinal), 1);
+        mbar_init(bar(kBarDrain), 1);
+        fence_mbar_init();
+    }
+    if (warp == 9) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    // Register budget: the launch gives every warp 168 registers (3 warps per scheduler);
+    // the producer warpgroup hands most of its share to the two compute warpgroups.
+    if (warp < 4) {
+        // =========================== softmax + epilogue ===========================
+        setmaxnreg_inc<216>();
+        const int r = tid;                               // query row inside the tile = TMEM lane
+        const uint32_t lane_addr = uint32_t(warp * 32) << 16;
+        float m_ref = -INFINITY;                         // reference maximum (log2 domain) the stored P, O use
+        float l_sum = 0.f;
+        for (int j = 0; j < n_kv; ++j) {
+            const int buf = j & 1;
+            const uint32_t tS = tmem + lane_addr + uint32_t(buf) * 128u;
+            mbar_wait(bar(kBarSFull + buf), (j >> 1) & 1, abort_flag, 10);
+            tc_fence_after_sync();
+            uint32_t s0[32], s1[32], s2[32], s3[32];
+            tmem_ld32(tS + 0, s0);
+            tmem_ld32(tS + 32, s1);
+            tmem_ld32(tS + 64, s2);
+            tmem_ld32(tS + 96, s3);
+            tmem_wait_ld();
+            if (j == n_kv - 1) {                         // diagonal tile: causal mask, key <= query
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    if (i > r) s0[i] = 0xff800000u;
+                    if (i + 32 > r) s1[i] = 0xff800000u;
+                    if (i + 64 > r) s2[i] = 0xff800000u;
+                    if (i + 96 > r) s3[i] = 0xff800000u;
+                }
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                mx0 = fmaxf(mx0, __uint_as_float(s0[i]));
+                mx1 = fmaxf(mx1, __uint_as_float(s1[i]));
+                mx2 = fmaxf(mx2, __uint_as_float(s2[i]));
+                mx3 = fmaxf(mx3, __uint_as_float(s3[i]));
+            }
+            const float m_new = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+            if (j == 0) {
+                m_ref = m_new;                           // nothing accumulated yet
+            } else if (__any_sync(0xffffffffu, m_new - m_ref > kRescaleThreshold)) {
+                // The maximum grew a lot: bring O and l to the new reference.  O may only be
+                // touched between PV_{j-1} completing and PV_j being issued; PV_j waits for
+                // this thread's arrival on kBarPFull below.
+                mbar_wait(bar(kBarOReady), (j - 1) & 1, abort_flag, 11);
+                tc_fence_after_sync();
+                const float f = fast_exp2(m_ref - m_new);
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tmem + lane_addr + kColO + c * 32, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                    tmem_st32(tmem + lane_addr + kColO + c * 32, o);
+                }
+                l_sum *= f;
+                m_ref = m_new;
+            }
+            const float neg_m = -m_ref;
+            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+            uint32_t pk0[16], pk1[16], pk2[16], pk3[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float a0 = fast_exp2(fmaf(__uint_as_float(s0[2 * i]), p.scale_log2, neg_m));
+                const float a1 = fast_exp2(fmaf(__uint_as_float(s0[2 * i + 1]), p.scale_log2, neg_m));
+                const float b0 = fast_exp2(fmaf(__uint_as_float(s1[2 * i]), p.scale_log2, neg_m));
+                const float b1 = fast_exp2(fmaf(__uint_as_float(s1[2 * i + 1]), p.scale_log2, neg_m));
+                const float c0 = fast_exp2(fmaf(__uint_as_float(s2[2 * i]), p.scale_log2, neg_m));
+                const float c1 = fast_exp2(fmaf(__uint_as_float(s2[2 * i + 1]), p.scale_log2, neg_m));
+                const float d0 = fast_exp2(fmaf(__uint_as_float(s3[2 * i]), p.scale_log2, neg_m));
+                const float d1 = fast_exp2(fmaf(__uint_as_float(s3[2 * i + 1]), p.scale_log2, neg_m));
+                sum0 += a0 + a1; sum1 += b0 + b1; sum2 += c0 + c1; sum3 += d0 + d1;
+                pk0[i] = pack_bf16x2(a0, a1);
+                pk1[i] = pack_bf16x2(b0, b1);
+                pk2[i] = pack_bf16x2(c0, c1);
+                pk3[i] = pack_bf16x2(d0, d1);
+            }
+            l_sum += (sum0 + sum1) + (sum2 + sum3);
+            // P_j (bf16, two per column) overlays the first 64 columns of S_j.
+            tmem_st16(tS + 0, pk0);
+            tmem_st16(tS + 16, pk1);
+            tmem_st16(tS + 32, pk2);
+            tmem_st16(tS + 48, pk3);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(bar(kBarPFull + buf));
+        }
+
+        // ------------------------------ epilogue ------------------------------
+        mbar_wait(bar(kBarOFinal), 0, abort_flag, 12);
+        tc_fence_after_sync();
+        float a_s = 1.f, a_d = 0.f, m_fin = m_ref, l_fin = l_sum;
+        if (p.l > 0) {
+            mbar_wait(bar(kBarDepth), 0, abort_flag, 13);
+            tc_fence_after_sync();
+            const float m_d = sMd[r], l_d = sLd[r];
+            m_fin = fmaxf(m_ref, m_d);
+            a_s = fast_exp2(m_ref - m_fin);
+            a_d = fast_exp2(m_d - m_fin);
+            l_fin = a_s * l_sum + a_d * l_d;
+        }
+        const float inv = 1.f / l_fin;
+        a_s *= inv;
+        a_d *= inv;
+        // O tile -> shared memory (the Q buffer, in the same swizzled layout) -> TMA store.
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem + lane_addr + kColO + c * 32, o);
+            tmem_wait_ld();
+            float of[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) of[i] = __uint_as_float(o[i]) * a_s;
+            if (p.l > 0) {
+                uint32_t od[32];
+                tmem_ld32(tmem + lane_addr + kColOd + c * 32, od);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) of[i] = fmaf(__uint_as_float(od[i]), a_d, of[i]);
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                uint4 v;
+                v.x = pack_bf16x2(of[8 * g + 0], of[8 * g + 1]);
+                v.y = pack_bf16x2(of[8 * g + 2], of[8 * g + 3]);
+                v.z = pack_bf16x2(of[8 * g + 4], of[8 * g + 5]);
+                v.w = pack_bf16x2(of[8 * g + 6], of[8 * g + 7]);
+                *reinterpret_cast<uint4*>(smem + L::kQ + swz_chunk_offset(r, c * 4 + g)) = v;
+            }
+        }
+        if (q0 + r < p.T) p.LSE[(size_t(b) * p.H + h) * p.T + q0 + r] = (m_fin + log2f(l_fin)) * kLn2;
+        fence_proxy_async_smem();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (tid == 0) {
+#pragma unroll
+            for (int s = 0; s < NSUB; ++s)
+                tma_store_4d(&mapO, sbase + L::kQ + s * L::kSubBytes, s * 64, h, q0, b);
+            tma_store_commit();
+            tma_store_wait_all();
+        }
+    } else if (warp < 8) {
+        // =========================== depth partial state ===========================
+        setmaxnreg_inc<216>();
+        if (p.l > 0) {
+            const int r = tid - 128;
+            const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+            const int ntile = nq;
+            const size_t slot_stride = cache_slot_elems(p.B, p.T, p.H, D) / 8;           // in uint4
+            const uint4* blkK = reinterpret_cast<const uint4*>(p.depth_kv) +
+                                (((size_t(b) * p.H + h) * ntile + qt) * 2 + 0) * (kTileRows * CH) + r;
+            const uint4* blkV = blkK + kTileRows * CH;
+            mbar_wait(bar(kBarQ), 0, abort_flag, 20);
+            // ---- depth scores u_i = <q, kd_i>, 64 features per sweep ----
+#pragma unroll 1
+            for (int half = 0; half < NSUB; ++half) {
+                float q[64];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, half * 8 + c));
+                    q[8 * c + 0] = bf16_lo_to_f32(v.x); q[8 * c + 1] = bf16_hi_to_f32(v.x);
+                    q[8 * c + 2] = bf16_lo_to_f32(v.y); q[8 * c + 3] = bf16_hi_to_f32(v.y);
+                    q[8 * c + 4] = bf16_lo_to_f32(v.z); q[8 * c + 5] = bf16_hi_to_f32(v.z);
+                    q[8 * c + 6] = bf16_lo_to_f32(v.w); q[8 * c + 7] = bf16_hi_to_f32(v.w);
+                }
+                uint4 kb[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) kb[c] = __ldg(blkK + (half * 8 + c) * kTileRows);
+#pragma unroll 1
+                for (int i = 0; i < p.l; ++i) {
+                    uint4 cur[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) cur[c] = kb[c];
+                    if (i + 1 < p.l) {
+                        const uint4* nxt = blkK + size_t(i + 1) * slot_stride + (half * 8) * kTileRows;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) kb[c] = __ldg(nxt + c * kTileRows);
+                    }
+                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        a0 = fmaf(q[8 * c + 0], bf16_lo_to_f32(cur[c].x), a0);
+                        a1 = fmaf(q[8 * c + 1], bf16_hi_to_f32(cur[c].x), a1);
+                        a2 = fmaf(q[8 * c + 2], bf16_lo_to_f32(cur[c].y), a2);
+                        a3 = fmaf(q[8 * c + 3], bf16_hi_to_f32(cur[c].y), a3);
+                        a0 = fmaf(q[8 * c + 4], bf16_lo_to_f32(cur[c].z), a0);
+                        a1 = fmaf(q[8 * c + 5], bf16_hi_to_f32(cur[c].z), a1);
+                        a2 = fmaf(q[8 * c + 6], bf16_lo_to_f32(cur[c].w), a2);
+                        a3 = fmaf(q[8 * c + 7], bf16_hi_to_f32(cur[c].w), a3);
+                    }
+                    const float part = (a0 + a1) + (a2 + a3);
+                    if (half == 0) sU[i * kTileRows + r] = part;
+                    else sU[i * kTileRows + r] += part;
+                }
+            }
+            // ---- partial softmax over the l depth scores ----
+            float m_d = -INFINITY;
+            for (int i = 0; i < p.l; ++i) m_d = fmaxf(m_d, sU[i * kTileRows + r] * p.scale_log2);
+            float l_d = 0.f;
+            for (int i = 0; i < p.l; ++i) {
+                const float w = fast_exp2(fmaf(sU[i * kTileRows + r], p.scale_log2, -m_d));
+                sU[i * kTileRows + r] = w;
+                l_d += w;
+            }
+            sMd[r] = m_d;
+            sLd[r] = l_d;
+            // ---- o_d = sum_i w_i vd_i, 64 features per sweep, parked in TMEM ----
+#pragma unroll 1
+            for (int half = 0; half < NSUB; ++half) {
+                float acc[64];
+#pragma unroll
+                for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+                uint4 vb[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) vb[c] = __ldg(blkV + (half * 8 + c) * kTileRows);
+#pragma unroll 1
+                for (int i = 0; i < p.l; ++i) {
+                    uint4 cur[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) cur[c] = vb[c];
+                    if (i + 1 < p.l) {
+                        const uint4* nxt = blkV + size_t(i + 1) * slot_stride + (half * 8) * kTileRows;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) vb[c] = __ldg(nxt + c * kTileRows);
+                    }
+                    const float w = sU[i * kTileRows + r];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        acc[8 * c + 0] = fmaf(w, bf16_lo_to_f32(cur[c].x), acc[8 * c + 0]);
+                        acc[8 * c + 1] = fmaf(w, bf16_hi_to_f32(cur[c].x), acc[8 * c + 1]);
+                        acc[8 * c + 2] = fmaf(w, bf16_lo_to_f32(cur[c].y), acc[8 * c + 2]);
+                        acc[8 * c + 3] = fmaf(w, bf16_hi_to_f32(cur[c].y), acc[8 * c + 3]);
+                        acc[8 * c + 4] = fmaf(w, bf16_lo_to_f32(cur[c].z), acc[8 * c + 4]);
+                        acc[8 * c + 5] = fmaf(w, bf16_hi_to_f32(cur[c].z), acc[8 * c + 5]);
+                        acc[8 * c + 6] = fmaf(w, bf16_lo_to_f32(cur[c].w), acc[8 * c + 6]);
+                        acc[8 * c + 7] = fmaf(w, bf16_hi_to_f32(cur[c].w), acc[8 * c + 7]);
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t o[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(acc[32 * c + i]);
+                    tmem_st32(tmem + lane_addr + kColOd + half * 64 + c * 32, o);
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(bar(kBarDepth));
+        }
+    } else {
+      setmaxnreg_dec<72>();   // one instruction for the whole producer warpgroup (warps 8-11)
+      if (warp == 8) {
+        // =========================== TMA producer ===========================
+        if (lane == 0) {
+            tma_prefetch_desc(&mapQ);
+            tma_prefetch_desc(&mapK);
+            tma_prefetch_desc(&mapV);
+            mbar_arrive_expect_tx(bar(kBarQ), L::kTileBytes);
+#pragma unroll
+            for (int s = 0; s < NSUB; ++s)
+                tma_load_4d(sbase + L::kQ + s * L::kSubBytes, &mapQ, bar(kBarQ), s * 64, h, q0, b);
+            for (int j = 0; j < n_kv; ++j) {
+                const int st = j & 1;
+                if (j >= 2) mbar_wait(bar(kBarKEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 30);
+                mbar_arrive_expect_tx(bar(kBarKFull + st), L::kTileBytes);
+#pragma unroll
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_4d(sbase + L::kK + st * L::kTileBytes + s * L::kSubBytes, &mapK, bar(kBarKFull + st),
+                                s * 64, h, j * kTileRows, b);
+                if (j >= 2) mbar_wait(bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 31);
+                mbar_arrive_expect_tx(bar(kBarVFull + st), L::kTileBytes);
+#pragma unroll
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_4d(sbase + L::kV + st * L::kTileBytes + s * L::kSubBytes, &mapV, bar(kBarVFull + st),
+                                s * 64, h, j * kTileRows, b);
+            }
+        }
+      } else if (warp == 9) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
+            constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
+            auto issue_s = [&](int j) {
+                const int st = j & 1;
+                mbar_wait(bar(kBarKFull + st), (j >> 1) & 1, abort_flag, 40);
+                tc_fence_after_sync();
+                const uint32_t aQ = sbase + L::kQ, aK = sbase + L::kK + st * L::kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t ad = desc_kmajor_sw128(aQ + (kk >> 2) * L::kSubBytes, kk & 3);
+                    const uint64_t bd = desc_kmajor_sw128(aK + (kk >> 2) * L::kSubBytes, kk & 3);
+                    umma_ss(tmem + uint32_t(st) * 128u, ad, bd, idesc_s, kk > 0);
+                }
+                umma_commit(bar(kBarSFull + st));
+                umma_commit(bar(kBarKEmpty + st));
+            };
+            mbar_wait(bar(kBarQ), 0, abort_flag, 41);
+            issue_s(0);
+            if (n_kv > 1) issue_s(1);
+            for (int j = 0; j < n_kv; ++j) {
+                const int st = j & 1;
+                mbar_wait(bar(kBarVFull + st), (j >> 1) & 1, abort_flag, 42);
+                mbar_wait(bar(kBarPFull + st), (j >> 1) & 1, abort_flag, 43);
+                tc_fence_after_sync();
+                const uint32_t aV = sbase + L::kV + st * L::kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < kTileRows / 16; ++kk) {
+                    const uint64_t bd = desc_mnmajor_sw128(aV, kk, L::kSubBytes);
+                    umma_ts(tmem + kColO, tmem + uint32_t(st) * 128u + kk * 8, bd, idesc_o, (j > 0) || (kk > 0));
+                }
+                umma_commit(bar(kBarVEmpty + st));
+                umma_commit(bar(kBarOReady));
+                if (j + 2 < n_kv) issue_s(j + 2);
+            }
+            umma_commit(bar(kBarOFinal));
+            if (*abort_flag != 0) {
+                // A wait gave up somewhere: make sure no MMA is still in flight before TMEM is released.
+                umma_commit(bar(kBarDrain));
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar(kBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+            }
+        }
+      }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag != 0 && tid == 256) {
+        // Abort path only: give bulk copies still in flight a bounded time to land before the CTA's
+        // shared memory is handed to another CTA.
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) {}
+    }
+    __syncthreads();
+    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+}
+
+}  // namespace moda

@@ -119,6 +119,26 @@ int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth
                   void* dQ, void* dK, void* dV, void* d_depth_kv,
                   void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * moda_attn_bwd is three launches; this entry point runs a subset of them so that each can
+ * be timed or profiled on its own.  `stages` is a bit mask:
+ *     MODA_BWD_STAGE_ROWTERMS  D_t = <dO_t, O_t> for every row, into `workspace`
+ *     MODA_BWD_STAGE_DQ        dQ and the depth gradients (reads D_t from `workspace`)
+ *     MODA_BWD_STAGE_DKDV      dK and dV                  (reads D_t from `workspace`)
+ * moda_attn_bwd(...) is moda_attn_bwd_stages(..., MODA_BWD_ALL_STAGES, stream).  All arguments
+ * are validated as for moda_attn_bwd whatever the mask; a mask outside [1, 7] is
+ * MODA_ERR_BAD_SHAPE.
+ */
+#define MODA_BWD_STAGE_ROWTERMS 1
+#define MODA_BWD_STAGE_DQ 2
+#define MODA_BWD_STAGE_DKDV 4
+#define MODA_BWD_ALL_STAGES 7
+int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void* depth_kv,
+                         const void* O, const void* dO, const float* LSE,
+                         int B, int T, int H, int d, int l, float scale,
+                         void* dQ, void* dK, void* dV, void* d_depth_kv,
+                         void* workspace, size_t workspace_bytes, int stages, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -19,8 +19,9 @@ MODA_MAX_DEPTH = 32
 SYMBOLS = (
     "moda_version", "moda_strerror", "moda_last_cuda_error", "moda_last_status",
     "moda_depth_cache_bytes", "moda_depth_cache_append", "moda_depth_cache_unpack",
-    "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd",
+    "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd", "moda_attn_bwd_stages",
 )
+MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
 
 
 class ModaError(RuntimeError):
@@ -62,6 +63,8 @@ def load() -> ctypes.CDLL:
     lib.moda_bwd_workspace_bytes.argtypes = [ci] * 5
     lib.moda_attn_bwd.restype = ci
     lib.moda_attn_bwd.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 5 + [sz, vp]
+    lib.moda_attn_bwd_stages.restype = ci
+    lib.moda_attn_bwd_stages.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 5 + [sz, ci, vp]
     _lib = lib
     return lib
 
@@ -155,8 +158,10 @@ def moda_bwd_workspace_bytes(B, T, H, d, l) -> int:
 
 
 def moda_attn_bwd(Q, K, V, depth_kv, O, dO, LSE, l, scale,
-                  dQ=None, dK=None, dV=None, d_depth_kv=None, workspace=None, stream=None):
-    """dQ, dK, dV [B,T,H,d] bf16 and the depth gradients (cache layout, slots < l)."""
+                  dQ=None, dK=None, dV=None, d_depth_kv=None, workspace=None, stream=None, stages=None):
+    """dQ, dK, dV [B,T,H,d] bf16 and the depth gradients (cache layout, slots < l).
+
+    With ``stages`` (a MODA_BWD_STAGE_* mask) the call goes through moda_attn_bwd_stages."""
     B, T, H, d = _bthd(Q, "Q")
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(Q) if dK is None else dK
@@ -166,9 +171,17 @@ def moda_attn_bwd(Q, K, V, depth_kv, O, dO, LSE, l, scale,
     need = moda_bwd_workspace_bytes(B, T, H, d, l)
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
-    _check(load().moda_attn_bwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
-                                _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, d, int(l), float(scale),
-                                _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
-                                _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
-           "moda_attn_bwd")
+    args = [_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
+            _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, d, int(l), float(scale),
+            _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
+            _ptr(workspace), workspace.numel() * workspace.element_size()]
+    if stages is None:
+        _check(load().moda_attn_bwd(*args, _stream(stream)), "moda_attn_bwd")
+    else:
+        _check(load().moda_attn_bwd_stages(*args, int(stages), _stream(stream)), "moda_attn_bwd_stages")
     return dQ, dK, dV, d_depth_kv
+
+
+def moda_attn_bwd_stages(*args, stages, **kwargs):
+    """moda_attn_bwd restricted to the launches selected by the ``stages`` bit mask."""
+    return moda_attn_bwd(*args, stages=stages, **kwargs)

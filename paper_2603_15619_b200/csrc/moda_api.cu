@@ -44,12 +44,12 @@ EncodeTiledFn get_encode_fn() {
 // Tensor map over a contiguous bf16 [B][T][H][d] tensor; one box = 128 positions x 64
 // features of one (b, h), written to shared memory with the 128-byte swizzle.
 // Out-of-range rows (ragged last tile) read as zero and are dropped on store.
-bool make_bthd_map(CUtensorMap* map, const void* base, int B, int T, int H, int d) {
+bool make_bthd_map(CUtensorMap* map, const void* base, int B, int T, int H, int d, int box_rows = kTileRows) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) { tl_last_cuda_error = static_cast<int>(cudaErrorNotSupported); return false; }
     const cuuint64_t dims[4] = {cuuint64_t(d), cuuint64_t(H), cuuint64_t(T), cuuint64_t(B)};
     const cuuint64_t strides[3] = {cuuint64_t(d) * 2, cuuint64_t(H) * d * 2, cuuint64_t(T) * H * d * 2};
-    const cuuint32_t box[4] = {64, 1, cuuint32_t(kTileRows), 1};
+    const cuuint32_t box[4] = {64, 1, cuuint32_t(box_rows), 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -111,6 +111,56 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     const unsigned grid = unsigned(B) * H * num_tiles(T);
     moda_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kDynamic, stream>>>(mQ, mK, mV, mO, p);
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+
+template <int D>
+int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
+    const int B = a.B, T = a.T, H = a.H;
+    CUtensorMap mQ, mdO, mK64, mV64, mdQ, mK, mV, mQ64, mdO64, mdK, mdV;
+    if (!make_bthd_map(&mQ, a.Q, B, T, H, D) || !make_bthd_map(&mdO, a.dO, B, T, H, D) ||
+        !make_bthd_map(&mK64, a.K, B, T, H, D, kKeyTile) || !make_bthd_map(&mV64, a.V, B, T, H, D, kKeyTile) ||
+        !make_bthd_map(&mdQ, a.dQ, B, T, H, D) || !make_bthd_map(&mK, a.K, B, T, H, D) ||
+        !make_bthd_map(&mV, a.V, B, T, H, D) || !make_bthd_map(&mQ64, a.Q, B, T, H, D, kKeyTile) ||
+        !make_bthd_map(&mdO64, a.dO, B, T, H, D, kKeyTile) || !make_bthd_map(&mdK, a.dK, B, T, H, D) ||
+        !make_bthd_map(&mdV, a.dV, B, T, H, D))
+        return MODA_ERR_CUDA;
+    static thread_local int configured_dev = -1;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (configured_dev != dev) {
+        if (!set_smem_limit(moda_bwd_dq_kernel<D>, DqSmem<D>::kDynamic) ||
+            !set_smem_limit(moda_bwd_dkdv_kernel<D>, DkvSmem<D>::kDynamic))
+            return MODA_ERR_CUDA;
+        configured_dev = dev;
+    }
+    float* delta = static_cast<float*>(a.workspace);
+    if (stages & 1) {
+        constexpr int rows_per_block = 256 / (D / 8);
+        const long long nrows = (long long)B * T * H;
+        const unsigned grid = unsigned((nrows + rows_per_block - 1) / rows_per_block);
+        bwd_delta_kernel<D><<<grid, 256, 0, stream>>>(static_cast<const uint4*>(a.O), static_cast<const uint4*>(a.dO), delta, B, T, H);
+        if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    }
+    const unsigned grid = unsigned(B) * H * num_tiles(T);
+    if (stages & 2) {
+        DqParams p;
+        p.depth_kv = static_cast<const __nv_bfloat16*>(a.depth_kv);
+        p.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
+        p.LSE = a.LSE; p.delta = delta;
+        p.B = B; p.T = T; p.H = H; p.l = a.l;
+        p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
+        moda_bwd_dq_kernel<D><<<grid, kBwdDqThreads, DqSmem<D>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
+        if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    }
+    if (stages & 4) {
+        DkvParams p;
+        p.LSE = a.LSE; p.delta = delta;
+        p.B = B; p.T = T; p.H = H;
+        p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
+        moda_bwd_dkdv_kernel<D><<<grid, kBwdDkvThreads, DkvSmem<D>::kDynamic, stream>>>(mK, mV, mQ64, mdO64, mdK, mdV, p);
+        if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    }
+    return MODA_OK;
 }
 
 template <int D, bool kToCache>
@@ -211,7 +261,17 @@ int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth
                   int B, int T, int H, int d, int l, float scale,
                   void* dQ, void* dK, void* dV, void* d_depth_kv,
                   void* workspace, size_t workspace_bytes, void* stream) {
+    return moda_attn_bwd_stages(Q, K, V, depth_kv, O, dO, LSE, B, T, H, d, l, scale, dQ, dK, dV, d_depth_kv,
+                                workspace, workspace_bytes, MODA_BWD_ALL_STAGES, stream);
+}
+
+int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void* depth_kv,
+                         const void* O, const void* dO, const float* LSE,
+                         int B, int T, int H, int d, int l, float scale,
+                         void* dQ, void* dK, void* dV, void* d_depth_kv,
+                         void* workspace, size_t workspace_bytes, int stages, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (stages <= 0 || stages > MODA_BWD_ALL_STAGES) return MODA_ERR_BAD_SHAPE;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv || !d_depth_kv)))
         return MODA_ERR_NULL_POINTER;
@@ -226,7 +286,7 @@ int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth
     a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv; a.O = O; a.dO = dO; a.LSE = LSE;
     a.B = B; a.T = T; a.H = H; a.l = l; a.scale = scale;
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
-    return d == 128 ? launch_bwd<128>(a, st) : launch_bwd<64>(a, st);
+    return d == 128 ? launch_bwd<128>(a, stages, st) : launch_bwd<64>(a, stages, st);
 }
 
 }  // extern "C"

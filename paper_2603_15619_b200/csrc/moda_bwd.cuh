@@ -1,13 +1,780 @@
-// placeholder while the forward path is brought up
+// MoDA backward kernels for sm_100a.  The paper prints no backward pass; these kernels
+// evaluate the derivative of the Sec. 2.2 operator.  With P = exp(S - LSE) (sequence),
+// R = exp(U - LSE) (depth), D_t = <dO_t, O_t>:
+//
+//   dS = P o (dO V^T - D),   dU_i = R_i (<dO, Vd_i> - D)
+//   dQ = scale (dS K + sum_i dU_i Kd_i)     dK = scale dS^T Q     dV = P^T dO
+//   dKd_i = scale dU_i Q                    dVd_i = R_i dO        (row-local)
+//
+// Three launches on the caller's stream, all deterministic (no atomics):
+//   1. bwd_delta_kernel      D_t for every row (fp32 workspace).
+//   2. moda_bwd_dq_kernel    one CTA per 128-query tile, loops over 64-key tiles: S and
+//                            dP = dO V^T on tcgen05, dS written back to TMEM as bf16, dQ += dS K
+//                            accumulated in TMEM.  A second warpgroup does the whole depth
+//                            backward for the tile's rows on the CUDA cores (reads the depth
+//                            cache, writes dKd / dVd in cache layout) and parks its dQ share in
+//                            TMEM; the epilogue adds the two.
+//   3. moda_bwd_dkdv_kernel  one CTA per 128-key tile, loops over 64-query tiles in the
+//                            transposed formulation (S^T = K Q^T, dP^T = V dO^T) so that
+//                            P^T and dS^T are TMEM A-operands of dV += P^T dO, dK += dS^T Q.
 #pragma once
+
 #include "moda_cache.cuh"
+#include "moda_fwd.cuh"
 #include "sm100_ptx.cuh"
+
 namespace moda {
+
 struct BwdArgs {
-    const void *Q, *K, *V, *depth_kv, *O, *dO; const float* LSE;
-    int B, T, H, l; float scale;
+    const void *Q, *K, *V, *depth_kv, *O, *dO;
+    const float* LSE;
+    int B, T, H, l;
+    float scale;
     void *dQ, *dK, *dV, *d_depth_kv, *workspace;
 };
-inline size_t bwd_workspace_bytes(int B, int T, int H) { return size_t(B) * H * T * 4; }
-template <int D> int launch_bwd(const BwdArgs&, cudaStream_t) { return -9; }
+
+inline size_t bwd_workspace_bytes(int B, int T, int H) {
+    return (size_t(B) * H * T * 4 + 15) & ~size_t(15);
 }
+
+__device__ __forceinline__ float dot8_bf16(const uint4& a, const uint4& b) {
+    float acc = bf16_lo_to_f32(a.x) * bf16_lo_to_f32(b.x);
+    acc = fmaf(bf16_hi_to_f32(a.x), bf16_hi_to_f32(b.x), acc);
+    acc = fmaf(bf16_lo_to_f32(a.y), bf16_lo_to_f32(b.y), acc);
+    acc = fmaf(bf16_hi_to_f32(a.y), bf16_hi_to_f32(b.y), acc);
+    acc = fmaf(bf16_lo_to_f32(a.z), bf16_lo_to_f32(b.z), acc);
+    acc = fmaf(bf16_hi_to_f32(a.z), bf16_hi_to_f32(b.z), acc);
+    acc = fmaf(bf16_lo_to_f32(a.w), bf16_lo_to_f32(b.w), acc);
+    acc = fmaf(bf16_hi_to_f32(a.w), bf16_hi_to_f32(b.w), acc);
+    return acc;
+}
+
+// D_t = <dO_t, O_t>, one group of d/8 lanes per row of the [B][T][H] row space; written as [B][H][T].
+template <int D>
+__global__ void __launch_bounds__(256)
+bwd_delta_kernel(const uint4* __restrict__ O, const uint4* __restrict__ dO, float* __restrict__ delta,
+                 int B, int T, int H) {
+    constexpr int CH = D / 8;
+    constexpr int ROWS = 256 / CH;
+    const long long nrows = (long long)B * T * H;
+    const long long row = (long long)blockIdx.x * ROWS + threadIdx.x / CH;
+    const int c = threadIdx.x % CH;
+    float acc = 0.f;
+    if (row < nrows) acc = dot8_bf16(O[row * CH + c], dO[row * CH + c]);
+#pragma unroll
+    for (int off = CH / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (row < nrows && c == 0) {
+        const int h = int(row % H);
+        const long long bt = row / H;
+        const int t = int(bt % T);
+        const int b = int(bt / T);
+        delta[(size_t(b) * H + h) * T + t] = acc;
+    }
+}
+
+// =====================================================================================
+// dQ + depth gradients
+// =====================================================================================
+constexpr int kBwdDqThreads = 384;
+constexpr int kKeyTile = 64;     // keys per inner tile of the dQ kernel / queries per inner tile of the dK,dV kernel
+
+template <int D>
+struct DqSmem {
+    static constexpr int kTileBytes = kTileRows * D * 2;             // 128 x D
+    static constexpr int kSubBytes = kTileRows * 128;                // 128 x 64 sub-tile
+    static constexpr int kHalfTileBytes = kKeyTile * D * 2;          // 64 x D
+    static constexpr int kHalfSubBytes = kKeyTile * 128;             // 64 x 64 sub-tile
+    static constexpr int kStages = 3;
+    static constexpr int kQ = 0;
+    static constexpr int kdO = kQ + kTileBytes;
+    static constexpr int kKV = kdO + kTileBytes;                     // stages of [K_j | V_j]
+    static constexpr int kU = kKV + kStages * 2 * kHalfTileBytes;    // [32][128] fp32: u_i, then R_i
+    static constexpr int kDr = kU + 32 * kTileRows * 4;              // [32][128] fp32: <dO,Vd_i>, then dU_i
+    static constexpr int kBars = kDr + 32 * kTileRows * 4;
+    static constexpr int kNumBars = 16;
+    static constexpr int kMisc = kBars + kNumBars * 8;
+    static constexpr int kTotal = kMisc + 16;
+    static constexpr int kDynamic = kTotal + 1024;
+};
+
+enum DqBar : int {
+    kDqBarQ = 0,
+    kDqBarKVFull = 1,    // +stage (3)
+    kDqBarKVEmpty = 4,   // +stage (3)
+    kDqBarSFull = 7,     // +buffer (2)
+    kDqBarPFull = 9,     // +buffer (2)
+    kDqBarFinal = 11,
+    kDqBarDepth = 12,
+    kDqBarDrain = 13,
+};
+
+struct DqParams {
+    const __nv_bfloat16* depth_kv;
+    __nv_bfloat16* d_depth_kv;
+    const float* LSE;
+    const float* delta;
+    int B, T, H, l;
+    float scale, scale_log2;
+};
+
+// bf16x2 product with both factors already packed.
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kBwdDqThreads, 1)
+moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
+                   const __grid_constant__ CUtensorMap mapK64, const __grid_constant__ CUtensorMap mapV64,
+                   const __grid_constant__ CUtensorMap mapdQ, const DqParams p) {
+    using L = DqSmem<D>;
+    constexpr int NSUB = D / 64;
+    constexpr int CH = D / 8;
+    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t kColS = 0, kColdP = 128, kColdQ = 256, kColdQd = 384;
+
+    if (g_moda_status != 0) return;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    float* sU = reinterpret_cast<float*>(smem + L::kU);
+    float* sDr = reinterpret_cast<float*>(smem + L::kDr);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 4);
+    auto bar = [&](int i) { return sbase + L::kBars + 8u * uint32_t(i); };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nq = num_tiles(p.T);
+    const int bh = blockIdx.x / nq;
+    const int qt = nq - 1 - (blockIdx.x % nq);
+    const int b = bh / p.H, h = bh % p.H;
+    const int q0 = qt * kTileRows;
+    const int n_kv = min(2 * (qt + 1), (p.T + kKeyTile - 1) / kKeyTile);   // 64-key tiles at or below the diagonal
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(kDqBarQ), 1);
+        for (int s = 0; s < L::kStages; ++s) {
+            mbar_init(bar(kDqBarKVFull + s), 1);
+            mbar_init(bar(kDqBarKVEmpty + s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(kDqBarSFull + s), 1);
+            mbar_init(bar(kDqBarPFull + s), 128);
+        }
+        mbar_init(bar(kDqBarFinal), 1);
+        mbar_init(bar(kDqBarDepth), 128);
+        mbar_init(bar(kDqBarDrain), 1);
+        fence_mbar_init();
+    }
+    if (warp == 9) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp < 4) {
+        // =========================== P, dS and the dQ epilogue ===========================
+        setmaxnreg_inc<216>();
+        const int r = tid;
+        const uint32_t lane_addr = uint32_t(warp * 32) << 16;
+        const bool valid = q0 + r < p.T;
+        const size_t row_idx = (size_t(b) * p.H + h) * p.T + q0 + r;
+        const float neg_lse2 = valid ? -p.LSE[row_idx] * kLog2e : -INFINITY;   // invalid rows get P = 0
+        const float delta = valid ? p.delta[row_idx] : 0.f;
+        for (int j = 0; j < n_kv; ++j) {
+            const int buf = j & 1;
+            mbar_wait(bar(kDqBarSFull + buf), (j >> 1) & 1, abort_flag, 50);
+            tc_fence_after_sync();
+            uint32_t s0[32], s1[32], g0[32], g1[32];
+            tmem_ld32(tmem + lane_addr + kColS + buf * 64, s0);
+            tmem_ld32(tmem + lane_addr + kColS + buf * 64 + 32, s1);
+            tmem_ld32(tmem + lane_addr + kColdP + buf * 64, g0);
+            tmem_ld32(tmem + lane_addr + kColdP + buf * 64 + 32, g1);
+            tmem_wait_ld();
+            const int koff = j * kKeyTile - q0;      // key of column c is visible to row r iff koff + c <= r
+            const bool masked = koff + kKeyTile - 1 > 0;
+            uint32_t pk0[16], pk1[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                float pa = fast_exp2(fmaf(__uint_as_float(s0[2 * i]), p.scale_log2, neg_lse2));
+                float pb = fast_exp2(fmaf(__uint_as_float(s0[2 * i + 1]), p.scale_log2, neg_lse2));
+                float pc = fast_exp2(fmaf(__uint_as_float(s1[2 * i]), p.scale_log2, neg_lse2));
+                float pd = fast_exp2(fmaf(__uint_as_float(s1[2 * i + 1]), p.scale_log2, neg_lse2));
+                if (masked) {
+                    if (koff + 2 * i > r) pa = 0.f;
+                    if (koff + 2 * i + 1 > r) pb = 0.f;
+                    if (koff + 32 + 2 * i > r) pc = 0.f;
+                    if (koff + 32 + 2 * i + 1 > r) pd = 0.f;
+                }
+                pk0[i] = pack_bf16x2(pa * (__uint_as_float(g0[2 * i]) - delta), pb * (__uint_as_float(g0[2 * i + 1]) - delta));
+                pk1[i] = pack_bf16x2(pc * (__uint_as_float(g1[2 * i]) - delta), pd * (__uint_as_float(g1[2 * i + 1]) - delta));
+            }
+            // dS_j (bf16, two per column) overlays the first 32 columns of S_j.
+            tmem_st16(tmem + lane_addr + kColS + buf * 64, pk0);
+            tmem_st16(tmem + lane_addr + kColS + buf * 64 + 16, pk1);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(bar(kDqBarPFull + buf));
+        }
+        mbar_wait(bar(kDqBarFinal), 0, abort_flag, 51);
+        tc_fence_after_sync();
+        if (p.l > 0) {
+            mbar_wait(bar(kDqBarDepth), 0, abort_flag, 52);
+            tc_fence_after_sync();
+        }
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem + lane_addr + kColdQ + c * 32, o);
+            tmem_wait_ld();
+            float of[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) of[i] = __uint_as_float(o[i]);
+            if (p.l > 0) {
+                uint32_t od[32];
+                tmem_ld32(tmem + lane_addr + kColdQd + c * 32, od);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) of[i] += __uint_as_float(od[i]);
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                uint4 v;
+                v.x = pack_bf16x2(of[8 * g + 0] * p.scale, of[8 * g + 1] * p.scale);
+                v.y = pack_bf16x2(of[8 * g + 2] * p.scale, of[8 * g + 3] * p.scale);
+                v.z = pack_bf16x2(of[8 * g + 4] * p.scale, of[8 * g + 5] * p.scale);
+                v.w = pack_bf16x2(of[8 * g + 6] * p.scale, of[8 * g + 7] * p.scale);
+                *reinterpret_cast<uint4*>(smem + L::kQ + swz_chunk_offset(r, c * 4 + g)) = v;
+            }
+        }
+        fence_proxy_async_smem();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (tid == 0) {
+#pragma unroll
+            for (int s = 0; s < NSUB; ++s) tma_store_4d(&mapdQ, sbase + L::kQ + s * L::kSubBytes, s * 64, h, q0, b);
+            tma_store_commit();
+            tma_store_wait_all();
+        }
+    } else if (warp < 8) {
+        // =========================== depth backward (row-local) ===========================
+        setmaxnreg_inc<216>();
+        if (p.l > 0) {
+            const int r = tid - 128;
+            const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+            const bool valid = q0 + r < p.T;
+            const size_t row_idx = (size_t(b) * p.H + h) * p.T + q0 + r;
+            const float neg_lse2 = valid ? -p.LSE[row_idx] * kLog2e : -INFINITY;
+            const float delta = valid ? p.delta[row_idx] : 0.f;
+            const size_t slot_stride = cache_slot_elems(p.B, p.T, p.H, D) / 8;          // in uint4
+            const size_t blk = (((size_t(b) * p.H + h) * nq + qt) * 2) * (kTileRows * CH) + r;
+            const uint4* blkK = reinterpret_cast<const uint4*>(p.depth_kv) + blk;
+            const uint4* blkV = blkK + kTileRows * CH;
+            uint4* gK = reinterpret_cast<uint4*>(p.d_depth_kv) + blk;
+            uint4* gV = gK + kTileRows * CH;
+            mbar_wait(bar(kDqBarQ), 0, abort_flag, 60);
+
+            auto load8 = [&](uint4 (&dst)[8], const uint4* base, int i, int half) {
+                const uint4* src = base + size_t(i) * slot_stride + (half * 8) * kTileRows;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) dst[c] = __ldg(src + c * kTileRows);
+            };
+            auto load_row_f32 = [&](float (&dst)[64], int smem_off, int half) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(smem + smem_off + swz_chunk_offset(r, half * 8 + c));
+                    dst[8 * c + 0] = bf16_lo_to_f32(v.x); dst[8 * c + 1] = bf16_hi_to_f32(v.x);
+                    dst[8 * c + 2] = bf16_lo_to_f32(v.y); dst[8 * c + 3] = bf16_hi_to_f32(v.y);
+                    dst[8 * c + 4] = bf16_lo_to_f32(v.z); dst[8 * c + 5] = bf16_hi_to_f32(v.z);
+                    dst[8 * c + 6] = bf16_lo_to_f32(v.w); dst[8 * c + 7] = bf16_hi_to_f32(v.w);
+                }
+            };
+            auto dot64 = [&](const float (&x)[64], const uint4 (&y)[8]) {
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    a0 = fmaf(x[8 * c + 0], bf16_lo_to_f32(y[c].x), a0);
+                    a1 = fmaf(x[8 * c + 1], bf16_hi_to_f32(y[c].x), a1);
+                    a2 = fmaf(x[8 * c + 2], bf16_lo_to_f32(y[c].y), a2);
+                    a3 = fmaf(x[8 * c + 3], bf16_hi_to_f32(y[c].y), a3);
+                    a0 = fmaf(x[8 * c + 4], bf16_lo_to_f32(y[c].z), a0);
+                    a1 = fmaf(x[8 * c + 5], bf16_hi_to_f32(y[c].z), a1);
+                    a2 = fmaf(x[8 * c + 6], bf16_lo_to_f32(y[c].w), a2);
+                    a3 = fmaf(x[8 * c + 7], bf16_hi_to_f32(y[c].w), a3);
+                }
+                return (a0 + a1) + (a2 + a3);
+            };
+
+            // ---- pass A: u_i = <q, kd_i> ----
+#pragma unroll 1
+            for (int half = 0; half < NSUB; ++half) {
+                float q[64];
+                load_row_f32(q, L::kQ, half);
+                uint4 nxt[8];
+                load8(nxt, blkK, 0, half);
+#pragma unroll 1
+                for (int i = 0; i < p.l; ++i) {
+                    uint4 cur[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) cur[c] = nxt[c];
+                    if (i + 1 < p.l) load8(nxt, blkK, i + 1, half);
+                    const float part = dot64(q, cur);
+                    if (half == 0) sU[i * kTileRows + r] = part;
+                    else sU[i * kTileRows + r] += part;
+                }
+            }
+            // R_i = exp(u_i - LSE): the forward's LSE already covers sequence and depth keys.
+            for (int i = 0; i < p.l; ++i)
+                sU[i * kTileRows + r] = fast_exp2(fmaf(sU[i * kTileRows + r], p.scale_log2, neg_lse2));
+
+            // ---- pass B: <dO, vd_i>, and dVd_i = R_i dO ----
+#pragma unroll 1
+            for (int half = 0; half < NSUB; ++half) {
+                float g[64];
+                load_row_f32(g, L::kdO, half);
+                uint4 nxt[8];
+                load8(nxt, blkV, 0, half);
+#pragma unroll 1
+                for (int i = 0; i < p.l; ++i) {
+                    uint4 cur[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) cur[c] = nxt[c];
+                    if (i + 1 < p.l) load8(nxt, blkV, i + 1, half);
+                    const float part = dot64(g, cur);
+                    if (half == 0) sDr[i * kTileRows + r] = part;
+                    else sDr[i * kTileRows + r] += part;
+                    const float w = sU[i * kTileRows + r];
+                    uint4* dst = gV + size_t(i) * slot_stride + (half * 8) * kTileRows;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        uint4 o;
+                        o.x = pack_bf16x2(w * g[8 * c + 0], w * g[8 * c + 1]);
+                        o.y = pack_bf16x2(w * g[8 * c + 2], w * g[8 * c + 3]);
+                        o.z = pack_bf16x2(w * g[8 * c + 4], w * g[8 * c + 5]);
+                        o.w = pack_bf16x2(w * g[8 * c + 6], w * g[8 * c + 7]);
+                        dst[c * kTileRows] = o;
+                    }
+                }
+            }
+            // dU_i = R_i (<dO, vd_i> - D)
+            for (int i = 0; i < p.l; ++i)
+                sDr[i * kTileRows + r] = sU[i * kTileRows + r] * (sDr[i * kTileRows + r] - delta);
+
+            // ---- pass C: dQ share sum_i dU_i kd_i (parked in TMEM), dKd_i = scale dU_i q ----
+#pragma unroll 1
+            for (int half = 0; half < NSUB; ++half) {
+                uint4 qp[8];                               // q kept packed: only multiplied, never summed
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    qp[c] = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, half * 8 + c));
+                float acc[64];
+#pragma unroll
+                for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+                uint4 nxt[8];
+                load8(nxt, blkK, 0, half);
+#pragma unroll 1
+                for (int i = 0; i < p.l; ++i) {
+                    uint4 cur[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) cur[c] = nxt[c];
+                    if (i + 1 < p.l) load8(nxt, blkK, i + 1, half);
+                    const float du = sDr[i * kTileRows + r];
+                    const float sdu = du * p.scale;
+                    const uint32_t sdu2 = pack_bf16x2(sdu, sdu);
+                    uint4* dst = gK + size_t(i) * slot_stride + (half * 8) * kTileRows;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        acc[8 * c + 0] = fmaf(du, bf16_lo_to_f32(cur[c].x), acc[8 * c + 0]);
+                        acc[8 * c + 1] = fmaf(du, bf16_hi_to_f32(cur[c].x), acc[8 * c + 1]);
+                        acc[8 * c + 2] = fmaf(du, bf16_lo_to_f32(cur[c].y), acc[8 * c + 2]);
+                        acc[8 * c + 3] = fmaf(du, bf16_hi_to_f32(cur[c].y), acc[8 * c + 3]);
+                        acc[8 * c + 4] = fmaf(du, bf16_lo_to_f32(cur[c].z), acc[8 * c + 4]);
+                        acc[8 * c + 5] = fmaf(du, bf16_hi_to_f32(cur[c].z), acc[8 * c + 5]);
+                        acc[8 * c + 6] = fmaf(du, bf16_lo_to_f32(cur[c].w), acc[8 * c + 6]);
+                        acc[8 * c + 7] = fmaf(du, bf16_hi_to_f32(cur[c].w), acc[8 * c + 7]);
+                        uint4 o;
+                        o.x = mul_bf16x2(qp[c].x, sdu2);
+                        o.y = mul_bf16x2(qp[c].y, sdu2);
+                        o.z = mul_bf16x2(qp[c].z, sdu2);
+                        o.w = mul_bf16x2(qp[c].w, sdu2);
+                        dst[c * kTileRows] = o;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t o[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(acc[32 * c + i]);
+                    tmem_st32(tmem + lane_addr + kColdQd + half * 64 + c * 32, o);
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(bar(kDqBarDepth));
+        }
+    } else {
+        setmaxnreg_dec<72>();
+        if (warp == 8) {
+            // =========================== TMA producer ===========================
+            if (lane == 0) {
+                tma_prefetch_desc(&mapQ);
+                tma_prefetch_desc(&mapdO);
+                tma_prefetch_desc(&mapK64);
+                tma_prefetch_desc(&mapV64);
+                mbar_arrive_expect_tx(bar(kDqBarQ), 2 * L::kTileBytes);
+#pragma unroll
+                for (int s = 0; s < NSUB; ++s) {
+                    tma_load_4d(sbase + L::kQ + s * L::kSubBytes, &mapQ, bar(kDqBarQ), s * 64, h, q0, b);
+                    tma_load_4d(sbase + L::kdO + s * L::kSubBytes, &mapdO, bar(kDqBarQ), s * 64, h, q0, b);
+                }
+                for (int j = 0; j < n_kv; ++j) {
+                    const int st = j % L::kStages;
+                    if (j >= L::kStages)
+                        mbar_wait(bar(kDqBarKVEmpty + st), ((j - L::kStages) / L::kStages) & 1, abort_flag, 70);
+                    mbar_arrive_expect_tx(bar(kDqBarKVFull + st), 2 * L::kHalfTileBytes);
+                    const uint32_t dstK = sbase + L::kKV + st * 2 * L::kHalfTileBytes;
+                    const uint32_t dstV = dstK + L::kHalfTileBytes;
+#pragma unroll
+                    for (int s = 0; s < NSUB; ++s) {
+                        tma_load_4d(dstK + s * L::kHalfSubBytes, &mapK64, bar(kDqBarKVFull + st), s * 64, h, j * kKeyTile, b);
+                        tma_load_4d(dstV + s * L::kHalfSubBytes, &mapV64, bar(kDqBarKVFull + st), s * 64, h, j * kKeyTile, b);
+                    }
+                }
+            }
+        } else if (warp == 9) {
+            // =========================== MMA issuer ===========================
+            if (lane == 0) {
+                constexpr uint32_t idesc_s = make_idesc_bf16(128, kKeyTile, false, false);
+                constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, false, true);
+                const uint32_t aQ = sbase + L::kQ, adO = sbase + L::kdO;
+                auto issue_sdp = [&](int j) {
+                    const int st = j % L::kStages, buf = j & 1;
+                    mbar_wait(bar(kDqBarKVFull + st), (j / L::kStages) & 1, abort_flag, 80);
+                    tc_fence_after_sync();
+                    const uint32_t aK = sbase + L::kKV + st * 2 * L::kHalfTileBytes;
+                    const uint32_t aV = aK + L::kHalfTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma_ss(tmem + kColS + buf * 64, desc_kmajor_sw128(aQ + (kk >> 2) * L::kSubBytes, kk & 3),
+                                desc_kmajor_sw128(aK + (kk >> 2) * L::kHalfSubBytes, kk & 3), idesc_s, kk > 0);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma_ss(tmem + kColdP + buf * 64, desc_kmajor_sw128(adO + (kk >> 2) * L::kSubBytes, kk & 3),
+                                desc_kmajor_sw128(aV + (kk >> 2) * L::kHalfSubBytes, kk & 3), idesc_s, kk > 0);
+                    umma_commit(bar(kDqBarSFull + buf));
+                };
+                mbar_wait(bar(kDqBarQ), 0, abort_flag, 81);
+                issue_sdp(0);
+                if (n_kv > 1) issue_sdp(1);
+                for (int j = 0; j < n_kv; ++j) {
+                    const int st = j % L::kStages, buf = j & 1;
+                    mbar_wait(bar(kDqBarPFull + buf), (j >> 1) & 1, abort_flag, 82);
+                    tc_fence_after_sync();
+                    const uint32_t aK = sbase + L::kKV + st * 2 * L::kHalfTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < kKeyTile / 16; ++kk)
+                        umma_ts(tmem + kColdQ, tmem + kColS + buf * 64 + kk * 8,
+                                desc_mnmajor_sw128(aK, kk, L::kHalfSubBytes), idesc_dq, (j > 0) || (kk > 0));
+                    umma_commit(bar(kDqBarKVEmpty + st));
+                    if (j + 2 < n_kv) issue_sdp(j + 2);
+                }
+                umma_commit(bar(kDqBarFinal));
+                if (*abort_flag != 0) {
+                    umma_commit(bar(kDqBarDrain));
+                    const uint64_t t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar(kDqBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag != 0 && tid == 256) {
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) {}
+    }
+    __syncthreads();
+    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+}
+
+// =====================================================================================
+// dK, dV
+// =====================================================================================
+constexpr int kBwdDkvThreads = 192;
+
+template <int D>
+struct DkvSmem {
+    static constexpr int kTileBytes = kTileRows * D * 2;
+    static constexpr int kSubBytes = kTileRows * 128;
+    static constexpr int kHalfTileBytes = kKeyTile * D * 2;
+    static constexpr int kHalfSubBytes = kKeyTile * 128;
+    static constexpr int kStages = 3;
+    static constexpr int kK = 0;
+    static constexpr int kV = kK + kTileBytes;
+    static constexpr int kQdO = kV + kTileBytes;                       // stages of [Q_i | dO_i]
+    static constexpr int kLse = kQdO + kStages * 2 * kHalfTileBytes;   // [stage][64] -LSE*log2(e)
+    static constexpr int kDelta = kLse + kStages * kKeyTile * 4;       // [stage][64]
+    static constexpr int kBars = kDelta + kStages * kKeyTile * 4;
+    static constexpr int kNumBars = 16;
+    static constexpr int kMisc = kBars + kNumBars * 8;
+    static constexpr int kTotal = kMisc + 16;
+    static constexpr int kDynamic = kTotal + 1024;
+};
+
+enum DkvBar : int {
+    kDkvBarKV = 0,
+    kDkvBarQFull = 1,    // +stage (3)
+    kDkvBarQEmpty = 4,   // +stage (3)
+    kDkvBarSFull = 7,    // +buffer (2)
+    kDkvBarPFull = 9,    // +buffer (2)
+    kDkvBarFinal = 11,
+    kDkvBarDrain = 12,
+};
+
+struct DkvParams {
+    const float* LSE;
+    const float* delta;
+    int B, T, H;
+    float scale, scale_log2;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kBwdDkvThreads, 1)
+moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+                     const __grid_constant__ CUtensorMap mapQ64, const __grid_constant__ CUtensorMap mapdO64,
+                     const __grid_constant__ CUtensorMap mapdK, const __grid_constant__ CUtensorMap mapdV,
+                     const DkvParams p) {
+    using L = DkvSmem<D>;
+    constexpr int NSUB = D / 64;
+    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t kColST = 0, kColdPT = 128, kColdK = 256, kColdV = 384;
+
+    if (g_moda_status != 0) return;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    float* sLse = reinterpret_cast<float*>(smem + L::kLse);
+    float* sDelta = reinterpret_cast<float*>(smem + L::kDelta);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 4);
+    auto bar = [&](int i) { return sbase + L::kBars + 8u * uint32_t(i); };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nk = num_tiles(p.T);
+    const int bh = blockIdx.x / nk;
+    const int kt = blockIdx.x % nk;                       // key tiles in ascending order: most work first
+    const int b = bh / p.H, h = bh % p.H;
+    const int k0 = kt * kTileRows;
+    const int nq64 = (p.T + kKeyTile - 1) / kKeyTile;
+    const int i_first = 2 * kt;                           // first 64-query tile that can see this key tile
+    const int n_it = nq64 - i_first;
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(kDkvBarKV), 1);
+        for (int s = 0; s < L::kStages; ++s) {
+            mbar_init(bar(kDkvBarQFull + s), 32);
+            mbar_init(bar(kDkvBarQEmpty + s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(kDkvBarSFull + s), 1);
+            mbar_init(bar(kDkvBarPFull + s), 128);
+        }
+        mbar_init(bar(kDkvBarFinal), 1);
+        mbar_init(bar(kDkvBarDrain), 1);
+        fence_mbar_init();
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp < 4) {
+        // =========================== P^T, dS^T and the dK / dV epilogue ===========================
+        const int r = tid;                                   // key row inside the tile = TMEM lane
+        const uint32_t lane_addr = uint32_t(warp * 32) << 16;
+        for (int it = 0; it < n_it; ++it) {
+            const int st = it % L::kStages, buf = it & 1;
+            const int qoff = (i_first + it) * kKeyTile - k0;  // query of column c sees key row r iff qoff + c >= r
+            mbar_wait(bar(kDkvBarQFull + st), (it / L::kStages) & 1, abort_flag, 90);   // LSE / D_t of this stage
+            mbar_wait(bar(kDkvBarSFull + buf), (it >> 1) & 1, abort_flag, 91);
+            tc_fence_after_sync();
+            const float* lse = sLse + st * kKeyTile;
+            const float* dl = sDelta + st * kKeyTile;
+            const bool masked = qoff < kTileRows - 1;
+#pragma unroll
+            for (int hc = 0; hc < 2; ++hc) {                 // 32 query columns at a time
+                uint32_t s[32], g[32];
+                tmem_ld32(tmem + lane_addr + kColST + buf * 64 + hc * 32, s);
+                tmem_ld32(tmem + lane_addr + kColdPT + buf * 64 + hc * 32, g);
+                tmem_wait_ld();
+                uint32_t pp[16], pd[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int c0 = hc * 32 + 2 * i;
+                    float pa = fast_exp2(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, lse[c0]));
+                    float pb = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, lse[c0 + 1]));
+                    if (masked) {
+                        if (qoff + c0 < r) pa = 0.f;
+                        if (qoff + c0 + 1 < r) pb = 0.f;
+                    }
+                    pp[i] = pack_bf16x2(pa, pb);
+                    pd[i] = pack_bf16x2(pa * (__uint_as_float(g[2 * i]) - dl[c0]), pb * (__uint_as_float(g[2 * i + 1]) - dl[c0 + 1]));
+                }
+                // P^T overlays S^T, dS^T overlays dP^T (bf16, two per column)
+                tmem_st16(tmem + lane_addr + kColST + buf * 64 + hc * 16, pp);
+                tmem_st16(tmem + lane_addr + kColdPT + buf * 64 + hc * 16, pd);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(bar(kDkvBarPFull + buf));
+        }
+        mbar_wait(bar(kDkvBarFinal), 0, abort_flag, 92);
+        tc_fence_after_sync();
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {            // 0: dK (scaled), 1: dV
+            const float mul = which == 0 ? p.scale : 1.f;
+            const uint32_t col = which == 0 ? kColdK : kColdV;
+            const int dst_off = which == 0 ? L::kK : L::kV;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tmem + lane_addr + col + c * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(o[8 * g + 0]) * mul, __uint_as_float(o[8 * g + 1]) * mul);
+                    v.y = pack_bf16x2(__uint_as_float(o[8 * g + 2]) * mul, __uint_as_float(o[8 * g + 3]) * mul);
+                    v.z = pack_bf16x2(__uint_as_float(o[8 * g + 4]) * mul, __uint_as_float(o[8 * g + 5]) * mul);
+                    v.w = pack_bf16x2(__uint_as_float(o[8 * g + 6]) * mul, __uint_as_float(o[8 * g + 7]) * mul);
+                    *reinterpret_cast<uint4*>(smem + dst_off + swz_chunk_offset(r, c * 4 + g)) = v;
+                }
+            }
+        }
+        fence_proxy_async_smem();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (tid == 0) {
+#pragma unroll
+            for (int s = 0; s < NSUB; ++s) {
+                tma_store_4d(&mapdK, sbase + L::kK + s * L::kSubBytes, s * 64, h, k0, b);
+                tma_store_4d(&mapdV, sbase + L::kV + s * L::kSubBytes, s * 64, h, k0, b);
+            }
+            tma_store_commit();
+            tma_store_wait_all();
+        }
+    } else if (warp == 4) {
+        // =========================== loader: TMA tiles + per-query LSE, D_t ===========================
+        if (lane == 0) {
+            tma_prefetch_desc(&mapK);
+            tma_prefetch_desc(&mapV);
+            tma_prefetch_desc(&mapQ64);
+            tma_prefetch_desc(&mapdO64);
+            mbar_arrive_expect_tx(bar(kDkvBarKV), 2 * L::kTileBytes);
+#pragma unroll
+            for (int s = 0; s < NSUB; ++s) {
+                tma_load_4d(sbase + L::kK + s * L::kSubBytes, &mapK, bar(kDkvBarKV), s * 64, h, k0, b);
+                tma_load_4d(sbase + L::kV + s * L::kSubBytes, &mapV, bar(kDkvBarKV), s * 64, h, k0, b);
+            }
+        }
+        const size_t row_base = (size_t(b) * p.H + h) * p.T;
+        for (int it = 0; it < n_it; ++it) {
+            const int st = it % L::kStages;
+            const int qrow0 = (i_first + it) * kKeyTile;
+            if (it >= L::kStages)
+                mbar_wait(bar(kDkvBarQEmpty + st), ((it - L::kStages) / L::kStages) & 1, abort_flag, 100);
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int c = lane + 32 * k;
+                const bool valid = qrow0 + c < p.T;
+                // invalid (padding) queries get -LSE = -inf so that their P is exactly 0
+                sLse[st * kKeyTile + c] = valid ? -p.LSE[row_base + qrow0 + c] * kLog2e : -INFINITY;
+                sDelta[st * kKeyTile + c] = valid ? p.delta[row_base + qrow0 + c] : 0.f;
+            }
+            if (lane == 0) {
+                mbar_arrive_expect_tx(bar(kDkvBarQFull + st), 2 * L::kHalfTileBytes);
+                const uint32_t dstQ = sbase + L::kQdO + st * 2 * L::kHalfTileBytes;
+                const uint32_t dstdO = dstQ + L::kHalfTileBytes;
+#pragma unroll
+                for (int s = 0; s < NSUB; ++s) {
+                    tma_load_4d(dstQ + s * L::kHalfSubBytes, &mapQ64, bar(kDkvBarQFull + st), s * 64, h, qrow0, b);
+                    tma_load_4d(dstdO + s * L::kHalfSubBytes, &mapdO64, bar(kDkvBarQFull + st), s * 64, h, qrow0, b);
+                }
+            } else {
+                mbar_arrive(bar(kDkvBarQFull + st));
+            }
+        }
+    } else {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, kKeyTile, false, false);
+            constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
+            const uint32_t aK = sbase + L::kK, aV = sbase + L::kV;
+            auto issue_s = [&](int it) {
+                const int st = it % L::kStages, buf = it & 1;
+                mbar_wait(bar(kDkvBarQFull + st), (it / L::kStages) & 1, abort_flag, 110);
+                tc_fence_after_sync();
+                const uint32_t aQ = sbase + L::kQdO + st * 2 * L::kHalfTileBytes;
+                const uint32_t adO = aQ + L::kHalfTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma_ss(tmem + kColST + buf * 64, desc_kmajor_sw128(aK + (kk >> 2) * L::kSubBytes, kk & 3),
+                            desc_kmajor_sw128(aQ + (kk >> 2) * L::kHalfSubBytes, kk & 3), idesc_s, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma_ss(tmem + kColdPT + buf * 64, desc_kmajor_sw128(aV + (kk >> 2) * L::kSubBytes, kk & 3),
+                            desc_kmajor_sw128(adO + (kk >> 2) * L::kHalfSubBytes, kk & 3), idesc_s, kk > 0);
+                umma_commit(bar(kDkvBarSFull + buf));
+            };
+            mbar_wait(bar(kDkvBarKV), 0, abort_flag, 111);
+            issue_s(0);
+            if (n_it > 1) issue_s(1);
+            for (int it = 0; it < n_it; ++it) {
+                const int st = it % L::kStages, buf = it & 1;
+                mbar_wait(bar(kDkvBarPFull + buf), (it >> 1) & 1, abort_flag, 112);
+                tc_fence_after_sync();
+                const uint32_t aQ = sbase + L::kQdO + st * 2 * L::kHalfTileBytes;
+                const uint32_t adO = aQ + L::kHalfTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < kKeyTile / 16; ++kk)
+                    umma_ts(tmem + kColdV, tmem + kColST + buf * 64 + kk * 8,
+                            desc_mnmajor_sw128(adO, kk, L::kHalfSubBytes), idesc_acc, (it > 0) || (kk > 0));
+#pragma unroll
+                for (int kk = 0; kk < kKeyTile / 16; ++kk)
+                    umma_ts(tmem + kColdK, tmem + kColdPT + buf * 64 + kk * 8,
+                            desc_mnmajor_sw128(aQ, kk, L::kHalfSubBytes), idesc_acc, (it > 0) || (kk > 0));
+                umma_commit(bar(kDkvBarQEmpty + st));
+                if (it + 2 < n_it) issue_s(it + 2);
+            }
+            umma_commit(bar(kDkvBarFinal));
+            if (*abort_flag != 0) {
+                umma_commit(bar(kDkvBarDrain));
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar(kDkvBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag != 0 && tid == 128) {
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) {}
+    }
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+}
+
+}  // namespace moda

@@ -1,0 +1,80 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, and rejects bad arguments before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2603_15619_b200 as moda
+from paper_2603_15619_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "moda.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(moda_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_loads_and_exports_every_declared_symbol():
+    lib = binding.load()
+    names = declared_symbols()
+    assert set(names) == set(binding.SYMBOLS), (names, binding.SYMBOLS)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert moda.moda_version() >= 100
+
+
+def test_strerror_covers_all_codes():
+    for code in range(0, -11, -1):
+        assert binding.strerror(code) != "unknown error code"
+    assert binding.strerror(-99) == "unknown error code"
+
+
+def test_size_queries_are_host_arithmetic():
+    # cache[slot][b][h][tile][kv][chunk][row][8] with 128-row tiles, bf16
+    assert moda.moda_depth_cache_bytes(1, 256, 2, 64, 4) == 4 * 1 * 2 * 2 * 2 * 128 * 64 * 2
+    assert moda.moda_depth_cache_bytes(2, 129, 3, 128, 1) == 2 * 3 * 2 * 2 * 128 * 128 * 2
+    assert moda.moda_depth_cache_bytes(1, 256, 2, 96, 4) == 0      # unsupported head width
+    assert moda.moda_depth_cache_bytes(1, 256, 2, 64, 33) == 0     # more than 32 slots
+    assert moda.moda_depth_cache_bytes(1, 0, 2, 64, 1) == 0
+    assert moda.moda_bwd_workspace_bytes(2, 100, 3, 64, 0) >= 2 * 3 * 100 * 4
+    assert moda.moda_bwd_workspace_bytes(2, 100, 3, 64, 0) % 16 == 0
+
+
+def test_argument_validation_rejects_before_any_launch():
+    lib = binding.load()
+    vp = ctypes.c_void_p
+    p = vp(4096)                        # aligned, non-null, never dereferenced: validation fails first
+    odd = vp(4100)
+    fwd = lambda *a: lib.moda_attn_fwd(*a)
+    base = dict(B=1, T=128, H=1, d=64, l=0)
+
+    def call(Q=p, K=p, V=p, dkv=None, O=p, LSE=p, scale=0.125, **kw):
+        a = dict(base, **kw)
+        return fwd(Q, K, V, dkv, a["B"], a["T"], a["H"], a["d"], a["l"], ctypes.c_float(scale), O, LSE, None)
+
+    assert call(B=0) == -3 and call(T=0) == -3 and call(H=-1) == -3
+    assert call(d=96) == -4
+    assert call(l=-1) == -5 and call(l=33) == -5
+    assert call(Q=None) == -1 and call(O=None) == -1 and call(LSE=None) == -1
+    assert call(l=2, dkv=None) == -1
+    assert call(K=odd) == -2
+    assert lib.moda_depth_cache_append(p, 1, 128, 1, 64, 32, p, p, None) == -6
+    assert lib.moda_depth_cache_append(p, 1, 128, 1, 64, -1, p, p, None) == -6
+    assert lib.moda_depth_cache_append(None, 1, 128, 1, 64, 0, p, p, None) == -1
+    # backward: workspace too small / missing, bad stage mask
+    args = [p] * 7 + [1, 128, 1, 64, 0, ctypes.c_float(0.125)] + [p, p, p, None]
+    assert lib.moda_attn_bwd(*args, p, ctypes.c_size_t(8), None) == -7
+    assert lib.moda_attn_bwd(*args, None, ctypes.c_size_t(1 << 20), None) == -7
+    assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 0, None) == -3
+    assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 8, None) == -3
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(ImportError):
+        binding.load()

@@ -1,0 +1,489 @@
+#!/usr/bin/env python
+"""Benchmark of the MoDA attention operator on B200: one JSON line on stdout.
+
+A "step" is one pass of the whole hot path for one attention layer over one batch of
+synthetic inputs that are already resident in HBM: the depth-cache "write" of the layer's
+own K, V (one slot), the forward kernel, and the three backward launches (row terms,
+dQ + depth gradients, dK/dV).  `value` is forward+backward TFLOP/s with the FLOP convention
+of paper_2603_15619_b200/flops.py (causal-halved sequence part + depth part, backward =
+2.5 x forward).  Default workload: c2 (B=4, T=4096, H=16, d=128, l=23).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl moda|reference]
+
+For N > 1 launch with torch.distributed.run; every rank runs the same workload on its own
+GPU (independent batch shards, no collective on the data path: weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2603_15619_b200 import flops, synthetic  # noqa: E402
+
+METRIC = "MoDA fwd+bwd TFLOP/s (fwd and % of B200 BF16 peak in `detail`; ratio to own l=0 kernel in `sweep`)"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (bytes); keyed by (workload, kernel).  None where no capture exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        ident = str(device_index)
+        try:
+            ident = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid).replace("GPU-", "")
+        except Exception:
+            pass
+        self.cmd = ["nvidia-smi", "-i", ident, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t_begin: float, t_end: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        rows = [l for (t, l) in self.lines if t_begin - 0.05 <= t <= t_end + 0.15] or [l for (_, l) in self.lines]
+        for l in rows:
+            parts = [x.strip() for x in l.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def ev():
+    return torch.cuda.Event(enable_timing=True)
+
+
+class Layer:
+    """Device buffers of one workload plus the calls of one step."""
+
+    KERNELS = ("cache_append", "fwd", "bwd_rowterms", "bwd_dq_depth", "bwd_dkdv")
+
+    def __init__(self, w: synthetic.Workload, seed: int, device):
+        import paper_2603_15619_b200 as moda
+        self.moda, self.w = moda, w
+        self.q = synthetic.tensor(w, "Q", seed, 0, device)
+        self.k = synthetic.tensor(w, "K", seed, 0, device)
+        self.v = synthetic.tensor(w, "V", seed, 0, device)
+        self.dO = synthetic.tensor(w, "dO", seed, 0, device)
+        self.cache = self.dcache = None
+        if w.l > 0:
+            self.cache = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, w.l, device)
+            self.dcache = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, w.l, device)
+            for i in range(w.l):
+                moda.moda_depth_cache_append(self.cache, i, synthetic.tensor(w, "Kd", seed, i, device),
+                                             synthetic.tensor(w, "Vd", seed, i, device))
+        self.next_slot = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, 1, device)   # slot this layer writes for later layers
+        self.O = torch.empty_like(self.q)
+        self.LSE = torch.empty((w.B, w.H, w.T), dtype=torch.float32, device=device)
+        self.dQ, self.dK, self.dV = (torch.empty_like(self.q) for _ in range(3))
+        self.ws = torch.empty(moda.moda_bwd_workspace_bytes(w.B, w.T, w.H, w.d, w.l), dtype=torch.uint8, device=device)
+
+    def append(self):
+        self.moda.moda_depth_cache_append(self.next_slot, 0, self.k, self.v)
+
+    def fwd(self):
+        self.moda.moda_attn_fwd(self.q, self.k, self.v, self.cache, self.w.l, self.w.scale, O=self.O, LSE=self.LSE)
+
+    def bwd(self, stages=None):
+        self.moda.moda_attn_bwd(self.q, self.k, self.v, self.cache, self.O, self.dO, self.LSE, self.w.l, self.w.scale,
+                                dQ=self.dQ, dK=self.dK, dV=self.dV, d_depth_kv=self.dcache, workspace=self.ws, stages=stages)
+
+    def step(self, events=None):
+        """One pass of the hot path; with `events` (6 CUDA events) records one between launches."""
+        calls = (self.append, self.fwd, lambda: self.bwd(1), lambda: self.bwd(2), lambda: self.bwd(4))
+        if events is None:
+            self.append(); self.fwd(); self.bwd()
+            return
+        events[0].record()
+        for i, c in enumerate(calls):
+            c()
+            events[i + 1].record()
+
+    # algorithmic HBM bytes / FLOPs per launch (every tensor moved once)
+    def kernel_model(self):
+        w = self.w
+        E = w.B * w.T * w.H * w.d
+        rows = w.B * w.H * w.T
+        f_fwd = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l)
+        seq = flops.fwd_flops(w.B, w.T, w.H, w.d, 0)
+        dep = flops.depth_fwd_flops(w.B, w.T, w.H, w.d, w.l)
+        return {
+            "cache_append": {"bytes": 2.0 * 4 * E, "flops": 0.0},
+            "fwd": {"bytes": flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l), "flops": f_fwd},
+            "bwd_rowterms": {"bytes": 2.0 * 2 * E + 4.0 * rows, "flops": 2.0 * E},
+            # reads Q dO K V + depth cache + LSE, D; writes dQ + depth gradients; 3 of the 5 backward contractions
+            "bwd_dq_depth": {"bytes": 2.0 * (5 * E + 4 * w.l * E) + 8.0 * rows, "flops": 1.5 * seq + 2.5 * dep},
+            # reads Q K V dO + LSE, D; writes dK dV; 4 contractions in the split formulation (2 recomputed)
+            "bwd_dkdv": {"bytes": 2.0 * 6 * E + 8.0 * rows, "flops": 2.0 * seq},
+        }
+
+
+def pick_workload(args):
+    import dataclasses
+    w = synthetic.WORKLOADS[args.workload.split("_")[0]]
+    if "_l" in args.workload:
+        w = w.with_l(int(args.workload.split("_l")[1]))
+    if args.batch > 0:
+        w = dataclasses.replace(w, B=args.batch, name=f"{w.name}_B{args.batch}")
+    return w
+
+
+def run_moda(args, rank, world, device):
+    import paper_2603_15619_b200 as moda
+    peaks = load_peaks()
+    w = pick_workload(args)
+    layer = Layer(w, seed=rank, device=device)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+
+    for _ in range(max(args.warmup, 3)):
+        layer.step()
+    torch.cuda.synchronize()
+    if moda.moda_last_status() != 0:
+        raise RuntimeError(f"device status {moda.moda_last_status()} after warm-up")
+
+    K = args.steps
+    evs = [[ev() for _ in range(6)] for _ in range(K)]
+    sampler = ClockSampler(device.index)
+    sampler.start()
+    time.sleep(0.3)
+    barrier()
+    torch.cuda.synchronize()
+    t_begin = time.time()
+    for s in range(K):
+        layer.step(evs[s])
+    torch.cuda.synchronize()
+    t_end = time.time()
+    barrier()
+    clocks = sampler.stop(t_begin, t_end)
+    total_ms = evs[0][0].elapsed_time(evs[-1][5])
+    ms_per_step = total_ms / K
+    if world > 1:
+        t = torch.tensor([ms_per_step], device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms_per_step = float(t.item())
+    status = moda.moda_last_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} after the timed region")
+
+    per_kernel = {}
+    for i, name in enumerate(Layer.KERNELS):
+        per_kernel[name] = sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K
+    step_flops = flops.fwd_bwd_flops(w.B, w.T, w.H, w.d, w.l)
+    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel ----
+    model = layer.kernel_model()
+    dom = max(per_kernel, key=per_kernel.get)
+    dur = per_kernel[dom] * 1e-3
+    long_region = (t_end - t_begin) > 1.0
+    tensor_peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
+    t_hbm = model[dom]["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_tensor = model[dom]["flops"] / (tensor_peak * 1e12)
+    if t_hbm >= t_tensor:
+        roof = {"bound": "hbm", "achieved": model[dom]["bytes"] / dur / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "tensor", "achieved": model[dom]["flops"] / dur / 1e12, "peak": tensor_peak, "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((w.name, dom))
+    roof.update({"kernel": dom, "kernel_ms": per_kernel[dom], "peak_source": peaks["source"],
+                 "peak_kind": ("sustained" if long_region else "burst") if roof["bound"] == "tensor" else "copy",
+                 "algorithmic_bytes": model[dom]["bytes"], "algorithmic_flops": model[dom]["flops"]})
+
+    fwd_tflops = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l) / (per_kernel["fwd"] * 1e-3) / 1e12
+    bwd_ms = per_kernel["bwd_rowterms"] + per_kernel["bwd_dq_depth"] + per_kernel["bwd_dkdv"]
+    detail = {
+        "kernel_ms": {k: round(v, 4) for k, v in per_kernel.items()},
+        "fwd_tflops": round(fwd_tflops, 1),
+        "bwd_tflops": round(flops.bwd_flops(w.B, w.T, w.H, w.d, w.l) / (bwd_ms * 1e-3) / 1e12, 1),
+        "fwd_frac_of_measured_burst_bf16": round(fwd_tflops / peaks["bf16_tflops"], 4),
+        "fwd_frac_of_measured_sustained_bf16": round(fwd_tflops / peaks["bf16_tflops_sustained"], 4),
+        "fwd_frac_of_nominal_bf16": round(fwd_tflops / NOMINAL_BF16_TFLOPS, 4),
+        "fwd_depth_read_gbs": round(flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / (per_kernel["fwd"] * 1e-3) / 1e9, 1),
+        "flop_convention": "fwd = 4BHd T^2/2 + 4BHTld; bwd = 2.5 x fwd; step = 3.5 x fwd",
+    }
+
+    out = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{w.name}: B={w.B} T={w.T} H={w.H} d={w.d} l={w.l} (per GPU), bf16 N(0,1) inputs, fp32 accumulate",
+                   "step": "depth-cache append of one slot + forward + backward (row terms, dQ+depth grads, dK/dV)",
+                   "l2_policy": "inputs larger than L2 (depth cache %.2f GiB + 4 x %.0f MiB activations per step)"
+                                % (flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / 2 ** 30, w.B * w.T * w.H * w.d * 2 / 2 ** 20),
+                   "parallelism": f"independent batch shards x{world}, no collective"},
+        "roofline": roof, "clocks": clocks, "gpu_launches": 5 * K, "detail": detail,
+    }
+
+    if rank == 0 and world == 1 and not args.no_sweep:
+        out["sweep"] = run_sweep(peaks, device, layer)
+    if not args.no_e2e:
+        out["e2e"] = run_e2e(layer, min(K, 3), world, step_flops, device)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w, budget_s=20.0)
+    return out
+
+
+def time_calls(fn, iters, warm=2):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    a, b = ev(), ev()
+    a.record()
+    for _ in range(iters):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / iters
+
+
+def run_sweep(peaks, device, first_layer):
+    """fwd / bwd time of every configured workload and of its l = 0 twin (same kernels, no depth slots)."""
+    rows = []
+    W = synthetic.WORKLOADS
+    plan = [("c2", W["c2"], 5)] + [(f"c3_l{l}", W["c3"].with_l(l), 5) for l in synthetic.C3_DEPTHS] + \
+           [("c4", W["c4"], 2), ("c5", W["c5"], 2)]
+    base_cache = {}
+    del first_layer
+    for name, w, iters in plan:
+        res = {}
+        for tag, ww in (("l0", w.with_l(0)), ("moda", w)):
+            key = (ww.B, ww.T, ww.H, ww.d, ww.l)
+            if key in base_cache:
+                res[tag] = base_cache[key]
+                continue
+            torch.cuda.empty_cache()
+            layer = Layer(ww, seed=0, device=device)
+            f_ms = time_calls(layer.fwd, iters)
+            b_ms = time_calls(layer.bwd, iters)
+            res[tag] = (f_ms, b_ms)
+            base_cache[key] = res[tag]
+            del layer
+        f_ms, b_ms = res["moda"]
+        f0, b0 = res["l0"]
+        ff = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l)
+        rows.append({
+            "workload": name, "B": w.B, "T": w.T, "H": w.H, "d": w.d, "l": w.l,
+            "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
+            "fwd_tflops": round(ff / f_ms / 1e9, 1), "fwd_bwd_tflops": round(3.5 * ff / (f_ms + b_ms) / 1e9, 1),
+            "fwd_frac_measured_burst": round(ff / f_ms / 1e9 / peaks["bf16_tflops"], 4),
+            "fwd_frac_nominal": round(ff / f_ms / 1e9 / NOMINAL_BF16_TFLOPS, 4),
+            "fwd_depth_read_gbs": round(flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / f_ms / 1e6, 1),
+            "l0_fwd_ms": round(f0, 4), "l0_bwd_ms": round(b0, 4),
+            "fwd_ratio_to_l0": round(f0 / f_ms, 4), "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f_ms + b_ms), 4),
+        })
+        log("sweep", rows[-1])
+    torch.cuda.empty_cache()
+    return rows
+
+
+def run_e2e(layer, steps, world, step_flops, device):
+    """The same step driven from pinned HOST buffers: every step copies its inputs host->device and
+    its results device->host inside the timed region."""
+    ins = [layer.q, layer.k, layer.v, layer.dO] + ([layer.cache] if layer.cache is not None else [])
+    outs = [layer.O, layer.LSE, layer.dQ, layer.dK, layer.dV] + ([layer.dcache] if layer.dcache is not None else [])
+    h_in = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in ins]
+    h_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+
+    def one():
+        for d, h in zip(ins, h_in):
+            d.copy_(h, non_blocking=True)
+        layer.step()
+        for h, d in zip(h_out, outs):
+            h.copy_(d, non_blocking=True)
+
+    one()
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    a, b = ev(), ev()
+    a.record()
+    for _ in range(steps):
+        one()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    if world > 1:
+        t = torch.tensor([ms], device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t.item())
+    nbytes = lambda ts: int(sum(t.numel() * t.element_size() for t in ts))
+    return {"value": round(world * step_flops / (ms * 1e-3) / 1e12, 3), "unit": UNIT, "ms_per_step": round(ms, 3),
+            "steps": steps, "h2d_bytes_per_step": nbytes(ins), "d2h_bytes_per_step": nbytes(outs)}
+
+
+def cpu_sample(w, n_slices, seed=0):
+    """Complete (b, h) slices of workload `w` as float64 numpy arrays (heads are independent)."""
+    pick = [(i % w.B, (i * 7) % w.H) for i in range(n_slices)]
+    x = {n: synthetic.tensor(w, n, seed, 0, "cpu") for n in ("Q", "K", "V", "dO")}
+    sl = lambda t: torch.stack([t[b, :, h] for b, h in pick], dim=0).unsqueeze(2).double().numpy()   # [n,T,1,d]
+    out = {n: sl(t) for n, t in x.items()}
+    kd = [synthetic.tensor(w, "Kd", seed, i, "cpu") for i in range(w.l)]
+    vd = [synthetic.tensor(w, "Vd", seed, i, "cpu") for i in range(w.l)]
+    import numpy as np
+    out["Kd"] = np.stack([sl(t) for t in kd]) if w.l else np.zeros((0,) + out["Q"].shape)
+    out["Vd"] = np.stack([sl(t) for t in vd]) if w.l else np.zeros((0,) + out["Q"].shape)
+    return out, pick
+
+
+def time_oracle(w, n_slices):
+    from oracle import moda_oracle as orc
+    x, pick = cpu_sample(w, n_slices)
+    t0 = time.time()
+    orc.forward(x["Q"], x["K"], x["V"], x["Kd"], x["Vd"], w.scale)
+    orc.backward(x["Q"], x["K"], x["V"], x["Kd"], x["Vd"], x["dO"], w.scale)
+    dt = time.time() - t0
+    fl = flops.fwd_bwd_flops(n_slices, w.T, 1, w.d, w.l)
+    return dt, fl, orc.threads(), pick
+
+
+def cpu_baseline(w, budget_s=20.0):
+    """The fp64 oracle, as it stands, on complete (b, h) slices of the benchmarked workload."""
+    dt, fl, cores, pick = time_oracle(w, 1)
+    n = 1
+    if dt < budget_s / 3:
+        n = int(min(w.B * w.H, max(1, budget_s / max(dt, 1e-3))))
+        dt, fl, cores, pick = time_oracle(w, n)
+    return {"value": round(fl / dt / 1e12, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} complete (b,h) slice(s) of {w.name} (T={w.T}, d={w.d}, l={w.l}), forward + backward, fp64, "
+                      f"{dt:.1f} s; FLOPs counted with the same convention as the GPU arm",
+            "seconds": round(dt, 2)}
+
+
+def run_reference(args, rank, world):
+    """--impl reference: the oracle timed on the host cores, same metric / config keys."""
+    w = pick_workload(args)
+    if rank != 0:
+        return None
+    K, W = args.steps, max(args.warmup, 0)
+    # bounded: each step is one complete (b, h) slice; cap the whole run near three minutes
+    t_probe, fl, cores, _ = time_oracle(w, 1)
+    budget = 180.0
+    K_eff = int(max(1, min(K, (budget - t_probe) // max(t_probe, 1e-3))))
+    W_eff = 0 if t_probe * (K_eff + W) > budget else W
+    for _ in range(W_eff):
+        time_oracle(w, 1)
+    t0 = time.time()
+    for _ in range(K_eff):
+        time_oracle(w, 1)
+    dt = (time.time() - t0) / K_eff
+    val = fl / dt / 1e12
+    return {
+        "impl": "reference", "metric": METRIC, "value": round(val, 6), "unit": UNIT, "n_gpus": world, "steps": K_eff,
+        "warmup": W_eff, "ms_per_step": round(dt * 1e3, 2), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name}: B={w.B} T={w.T} H={w.H} d={w.d} l={w.l}; each step = one complete (b,h) slice "
+                               f"(forward + backward) of that workload on the host cores"},
+        "cpu_baseline": {"value": round(val, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"one (b,h) slice of {w.name} per step, {K_eff} step(s) (requested {K})"},
+        "e2e": {"value": round(val, 6), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="moda", choices=["moda", "reference"])
+    ap.add_argument("--workload", default="c2", help="c1..c5, optionally with _l<depth> (e.g. c3_l8)")
+    ap.add_argument("--batch", type=int, default=0, help="override B of the workload (smaller profiling cases)")
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        out = run_reference(args, rank, world)
+        if out is not None:
+            print(json.dumps(out), flush=True)
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the MoDA operator has no CPU path)")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=device)
+    try:
+        out = run_moda(args, rank, world, device)
+        if rank == 0:
+            print(json.dumps(out), flush=True)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

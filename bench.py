@@ -37,7 +37,12 @@ NOMINAL_BF16_TFLOPS = 2250.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes); keyed by (workload, kernel).  None where no capture exists.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # c2 captured at B=1 and scaled x4 (traffic is proportional to B): profiles/ncu_full_c2_B1_fwd_bwd_kernels.md
+    ("c2", "fwd"): 4 * (0.824826e9 + 18.052e6),
+    ("c2", "bwd_dq_depth"): 4 * (1.227389e9 + 744.710e6),
+    ("c2", "bwd_dkdv"): 4 * (0.067713e9 + 9.716e6),
+}
 
 
 def log(*a):

@@ -59,6 +59,7 @@ extern "C" {
 #define MODA_ERR_DEVICE (-8)          /* current device is not sm_100 */
 #define MODA_ERR_CUDA (-9)            /* a CUDA runtime/driver call failed (see moda_last_cuda_error) */
 #define MODA_ERR_DEVICE_TIMEOUT (-10) /* an earlier kernel gave up a bounded wait (see moda_last_status) */
+#define MODA_ERR_SCRATCH_LIMIT (-11)  /* problem needs more built-in scratch than moda_attn_bwd_static_scratch holds */
 
 /* Library version: major * 10000 + minor * 100 + patch. */
 int moda_version(void);
@@ -138,6 +139,36 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
                          int B, int T, int H, int d, int l, float scale,
                          void* dQ, void* dK, void* dV, void* d_depth_kv,
                          void* workspace, size_t workspace_bytes, int stages, void* stream);
+
+/*
+ * Backward pass for callers that have no scratch buffer to give.  (The paper has no
+ * counterpart: this is a deployment convenience of this library, not part of the method.)
+ *
+ * moda_attn_bwd needs a caller-owned workspace for the per-row terms D_t.  Some callers cannot
+ * provide one: a plug-in that is only handed its input and output tensors by a host framework,
+ * or a serving process that sized all of its device memory at start-up and is not allowed to call
+ * cudaMalloc afterwards (the call synchronises the whole device and can fail once memory is
+ * fully committed).  This variant computes exactly what moda_attn_bwd computes, with the same
+ * kernels, but keeps D_t in an array that is compiled into the library image
+ * (MODA_STATIC_SCRATCH_ROWS fp32 values = 4 MiB, resident on every GPU that loads the library
+ * until the process exits).  It calls no cudaMalloc, cudaFree or any other allocating routine.
+ *
+ *   - Limit: B * H * T <= MODA_STATIC_SCRATCH_ROWS, otherwise MODA_ERR_SCRATCH_LIMIT is
+ *     returned and nothing is launched.  Other arguments and errors as for moda_attn_bwd.
+ *   - The first call on each device looks up the device address of the built-in array (with
+ *     that device current) and remembers it; make that first call before starting any stream
+ *     capture.  Later calls on the device only launch kernels.
+ *   - Every call on a device uses the same array, and it keeps whatever the previous call left
+ *     there.  Nothing in it has to start at zero: the first launch of each call overwrites every
+ *     row term the later launches read.  Two calls whose kernels may overlap on the GPU (different
+ *     streams, no ordering between them) race on the array and give undefined gradients; order
+ *     them, or use moda_attn_bwd with separate workspaces.
+ */
+#define MODA_STATIC_SCRATCH_ROWS (1 << 20)
+int moda_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, const void* depth_kv,
+                                 const void* O, const void* dO, const float* LSE,
+                                 int B, int T, int H, int d, int l, float scale,
+                                 void* dQ, void* dK, void* dV, void* d_depth_kv, void* stream);
 
 #ifdef __cplusplus
 }

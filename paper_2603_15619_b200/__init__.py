@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     alloc_depth_cache,
     moda_attn_bwd,
     moda_attn_bwd_stages,
+    moda_attn_bwd_static_scratch,
     moda_attn_fwd,
     moda_bwd_workspace_bytes,
     moda_depth_cache_append,

@@ -20,7 +20,9 @@ SYMBOLS = (
     "moda_version", "moda_strerror", "moda_last_cuda_error", "moda_last_status",
     "moda_depth_cache_bytes", "moda_depth_cache_append", "moda_depth_cache_unpack",
     "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd", "moda_attn_bwd_stages",
+    "moda_attn_bwd_static_scratch",
 )
+MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
 
 
@@ -65,6 +67,8 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 5 + [sz, vp]
     lib.moda_attn_bwd_stages.restype = ci
     lib.moda_attn_bwd_stages.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 5 + [sz, ci, vp]
+    lib.moda_attn_bwd_static_scratch.restype = ci
+    lib.moda_attn_bwd_static_scratch.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 4 + [vp]
     _lib = lib
     return lib
 
@@ -185,3 +189,21 @@ def moda_attn_bwd(Q, K, V, depth_kv, O, dO, LSE, l, scale,
 def moda_attn_bwd_stages(*args, stages, **kwargs):
     """moda_attn_bwd restricted to the launches selected by the ``stages`` bit mask."""
     return moda_attn_bwd(*args, stages=stages, **kwargs)
+
+
+def moda_attn_bwd_static_scratch(Q, K, V, depth_kv, O, dO, LSE, l, scale, dQ, dK, dV, d_depth_kv=None, stream=None):
+    """Backward for callers that cannot hand over a scratch buffer (a plug-in that only receives its
+    tensors, a server that may not call cudaMalloc once it is running).  Same results as
+    moda_attn_bwd; the per-row terms live in a 4 MiB array built into the library, so this call
+    takes no workspace and allocates nothing -- which is why every output must be passed in.
+
+    Limit: B*H*T <= MODA_STATIC_SCRATCH_ROWS (error -11 beyond it).  Calls on one device share that
+    array: do not let two of them overlap on the GPU."""
+    B, T, H, d = _bthd(Q, "Q")
+    if l > 0 and d_depth_kv is None:
+        raise ValueError("d_depth_kv must be provided: this entry point allocates nothing")
+    _check(load().moda_attn_bwd_static_scratch(
+        _ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None, _ptr(O), _ptr(dO), _ptr(LSE),
+        B, T, H, d, int(l), float(scale), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
+        _stream(stream)), "moda_attn_bwd_static_scratch")
+    return dQ, dK, dV, d_depth_kv

@@ -190,6 +190,7 @@ const char* moda_strerror(int code) {
         case MODA_ERR_DEVICE: return "the current CUDA device is not an sm_100 part";
         case MODA_ERR_CUDA: return "a CUDA call failed (see moda_last_cuda_error)";
         case MODA_ERR_DEVICE_TIMEOUT: return "a kernel gave up a bounded wait (see moda_last_status)";
+        case MODA_ERR_SCRATCH_LIMIT: return "B*H*T exceeds the built-in scratch of moda_attn_bwd_static_scratch (2^20 rows)";
         default: return "unknown error code";
     }
 }
@@ -290,3 +291,57 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Backward without a caller workspace: the row terms live in an array inside the library image.
+// ------------------------------------------------------------------------------------------
+namespace {
+
+// In host code this name is only a handle for the runtime, not a device address: the address
+// each GPU gave the array is looked up once per device with cudaGetSymbolAddress below.
+static __device__ __align__(256) float g_static_rowterms[MODA_STATIC_SCRATCH_ROWS];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+float* g_static_rowterms_addr[kMaxDevices] = {};
+
+// Device address of the built-in scratch on the current device (looked up on first use).
+int static_scratch_for_current_device(float** out) {
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return MODA_ERR_DEVICE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_rowterms_addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (!cuda_ok(cudaGetSymbolAddress(&ptr, g_static_rowterms)) || ptr == nullptr) return MODA_ERR_CUDA;
+        g_static_rowterms_addr[dev] = static_cast<float*>(ptr);
+    }
+    *out = g_static_rowterms_addr[dev];
+    return MODA_OK;
+}
+
+}  // namespace
+
+extern "C" int moda_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, const void* depth_kv,
+                                            const void* O, const void* dO, const float* LSE,
+                                            int B, int T, int H, int d, int l, float scale,
+                                            void* dQ, void* dK, void* dV, void* d_depth_kv, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if ((long long)B * H * T > (long long)MODA_STATIC_SCRATCH_ROWS) return MODA_ERR_SCRATCH_LIMIT;
+    if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv || !d_depth_kv)))
+        return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(LSE) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) ||
+        (l > 0 && (!aligned16(depth_kv) || !aligned16(d_depth_kv))))
+        return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    float* scratch = nullptr;
+    if (int rc = static_scratch_for_current_device(&scratch)) return rc;
+    BwdArgs a;
+    a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv; a.O = O; a.dO = dO; a.LSE = LSE;
+    a.B = B; a.T = T; a.H = H; a.l = l; a.scale = scale;
+    a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = scratch;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_bwd<128>(a, MODA_BWD_ALL_STAGES, st) : launch_bwd<64>(a, MODA_BWD_ALL_STAGES, st);
+}

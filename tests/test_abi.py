@@ -28,7 +28,7 @@ def test_library_loads_and_exports_every_declared_symbol():
 
 
 def test_strerror_covers_all_codes():
-    for code in range(0, -11, -1):
+    for code in range(0, -12, -1):
         assert binding.strerror(code) != "unknown error code"
     assert binding.strerror(-99) == "unknown error code"
 

@@ -254,3 +254,123 @@ int moda_oracle_bwd(const double *Q, const double *K, const double *V,
     free(O); free(LSE); free(Dl);
     return 0;
 }
+
+/*
+ * Backward for sampled rows (same formulas as moda_oracle_bwd, evaluated only where asked, so
+ * that single rows of very long sequences can be checked):
+ *   qrows[3*r + {0,1,2}] = (b, h, t): row-local outputs dQ_t [d], dKd_i[t] and dVd_i[t] ([l][d] each)
+ *   krows[3*r + {0,1,2}] = (b, h, j) with j >= t_start: dK_j [d] and dV_j [d], sums over t >= j.
+ * LSE_t and D_t are evaluated by the forward definition for every t in [t_start, T) of every
+ * (b, h) named in krows, which is what bounds the cost to (T - t_start) forward rows per head.
+ */
+int moda_oracle_bwd_rows(const double *Q, const double *K, const double *V,
+                         const double *Kd, const double *Vd, const double *dO,
+                         int B, int T, int H, int d, int l, double scale,
+                         const int *qrows, int n_q, const int *krows, int n_k, int t_start,
+                         double *dQ_rows, double *dKd_rows, double *dVd_rows,
+                         double *dK_rows, double *dV_rows)
+{
+    const size_t E = (size_t)B * T * H * d;
+    int failed = 0;
+    if (t_start < 0) t_start = 0;
+    const int W = T - t_start;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(T + 1));
+        double *u = (double *)malloc(sizeof(double) * (size_t)(l + 1));
+        double *o = (double *)malloc(sizeof(double) * (size_t)d);
+        if (!s || !u || !o) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+#pragma omp for schedule(dynamic, 1)
+            for (int r = 0; r < n_q; ++r) {
+                const int b = qrows[3 * r], h = qrows[3 * r + 1], t = qrows[3 * r + 2];
+                double lse;
+                fwd_row(Q, K, V, Kd, Vd, B, T, H, d, l, scale, b, h, t, s, u, o, &lse);  /* s = p_j, u = r_i */
+                const size_t rt = idx4(b, t, h, T, H, d);
+                const double *q = Q + rt, *go = dO + rt;
+                const double D = dot(go, o, d);
+                double *gq = dQ_rows + (size_t)r * d;
+                for (int c = 0; c < d; ++c) gq[c] = 0.0;
+                for (int j = 0; j <= t; ++j) {
+                    const double *k = K + idx4(b, j, h, T, H, d);
+                    const double ds = s[j] * (dot(go, V + idx4(b, j, h, T, H, d), d) - D);
+                    for (int c = 0; c < d; ++c) gq[c] += scale * ds * k[c];
+                }
+                for (int i = 0; i < l; ++i) {
+                    const double *kd = Kd + i * E + rt;
+                    const double du = u[i] * (dot(go, Vd + i * E + rt, d) - D);
+                    double *gkd = dKd_rows + ((size_t)r * l + i) * d, *gvd = dVd_rows + ((size_t)r * l + i) * d;
+                    for (int c = 0; c < d; ++c) {
+                        gq[c] += scale * du * kd[c];
+                        gkd[c] = scale * du * q[c];
+                        gvd[c] = u[i] * go[c];
+                    }
+                }
+            }
+        }
+        free(s); free(u); free(o);
+    }
+    if (failed) return -1;
+    if (n_k == 0) return 0;
+
+    /* LSE_t, D_t for t in [t_start, T) of every (b, h) that krows names (table indexed by b*H + h). */
+    char *need = (char *)calloc((size_t)B * H, 1);
+    double *lse_tab = (double *)malloc(sizeof(double) * (size_t)B * H * (W > 0 ? W : 1));
+    double *del_tab = (double *)malloc(sizeof(double) * (size_t)B * H * (W > 0 ? W : 1));
+    if (!need || !lse_tab || !del_tab) { free(need); free(lse_tab); free(del_tab); return -1; }
+    for (int r = 0; r < n_k; ++r) {
+        if (krows[3 * r + 2] < t_start) { free(need); free(lse_tab); free(del_tab); return -2; }
+        need[(size_t)krows[3 * r] * H + krows[3 * r + 1]] = 1;
+    }
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(T + 1));
+        double *u = (double *)malloc(sizeof(double) * (size_t)(l + 1));
+        double *o = (double *)malloc(sizeof(double) * (size_t)d);
+        if (!s || !u || !o) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+#pragma omp for collapse(2) schedule(dynamic, 1)
+            for (int bh = 0; bh < B * H; ++bh)
+                for (int t = t_start; t < T; ++t) {
+                    if (!need[bh]) continue;
+                    const int b = bh / H, h = bh % H;
+                    double lse;
+                    fwd_row(Q, K, V, Kd, Vd, B, T, H, d, l, scale, b, h, t, s, u, o, &lse);
+                    lse_tab[(size_t)bh * W + (t - t_start)] = lse;
+                    del_tab[(size_t)bh * W + (t - t_start)] = dot(dO + idx4(b, t, h, T, H, d), o, d);
+                }
+        }
+        free(s); free(u); free(o);
+    }
+    if (!failed) {
+#pragma omp parallel for schedule(dynamic, 1)
+        for (int r = 0; r < n_k; ++r) {
+            const int b = krows[3 * r], h = krows[3 * r + 1], j = krows[3 * r + 2];
+            const size_t rj = idx4(b, j, h, T, H, d);
+            const double *k = K + rj, *v = V + rj;
+            double *gk = dK_rows + (size_t)r * d, *gv = dV_rows + (size_t)r * d;
+            for (int c = 0; c < d; ++c) { gk[c] = 0.0; gv[c] = 0.0; }
+            for (int t = j; t < T; ++t) {
+                const size_t rt = idx4(b, t, h, T, H, d);
+                const double *q = Q + rt, *go = dO + rt;
+                const size_t e = ((size_t)b * H + h) * W + (t - t_start);
+                const double p = exp(scale * dot(q, k, d) - lse_tab[e]);
+                const double ds = p * (dot(go, v, d) - del_tab[e]);
+                for (int c = 0; c < d; ++c) {
+                    gk[c] += scale * ds * q[c];
+                    gv[c] += p * go[c];
+                }
+            }
+        }
+    }
+    free(need); free(lse_tab); free(del_tab);
+    return failed ? -1 : 0;
+}

@@ -55,6 +55,11 @@ def _load():
         )
         lib.moda_oracle_bwd.restype = ctypes.c_int
         lib.moda_oracle_bwd.argtypes = [_dp] * 6 + [ctypes.c_int] * 5 + [ctypes.c_double] + [_dp] * 5
+        lib.moda_oracle_bwd_rows.restype = ctypes.c_int
+        lib.moda_oracle_bwd_rows.argtypes = (
+            [_dp] * 6 + [ctypes.c_int] * 5 + [ctypes.c_double, _ip, ctypes.c_int, _ip, ctypes.c_int, ctypes.c_int]
+            + [_dp] * 5
+        )
         _lib = lib
     return _lib
 
@@ -138,3 +143,33 @@ def backward(Q, K, V, Kd, Vd, dO, scale):
     if rc != 0:
         raise MemoryError("oracle scratch allocation failed")
     return dQ, dK, dV, dKd, dVd
+
+
+def backward_rows(Q, K, V, Kd, Vd, dO, scale, qrows, krows=None, t_start=None):
+    """Backward for sampled rows.
+
+    ``qrows`` [n_q, 3] of (b, h, t): returns dQ_rows [n_q, d], dKd_rows, dVd_rows [n_q, l, d].
+    ``krows`` [n_k, 3] of (b, h, j), all j >= ``t_start`` (default: the smallest j): returns
+    dK_rows, dV_rows [n_k, d].  The cost of the key rows is (T - t_start) forward rows per head."""
+    Q, K, V, Kd, Vd, (B, T, H, d, l) = _prep(Q, K, V, Kd, Vd)
+    dO = _f64(dO, (B, T, H, d))
+    qrows = np.ascontiguousarray(qrows if qrows is not None else np.zeros((0, 3)), dtype=np.int32).reshape(-1, 3)
+    krows = np.ascontiguousarray(krows if krows is not None else np.zeros((0, 3)), dtype=np.int32).reshape(-1, 3)
+    for rows in (qrows, krows):
+        if rows.size and not ((rows >= 0).all() and (rows[:, 0] < B).all()
+                              and (rows[:, 1] < H).all() and (rows[:, 2] < T).all()):
+            raise ValueError("row index out of range")
+    if t_start is None:
+        t_start = int(krows[:, 2].min()) if krows.size else T
+    n_q, n_k = qrows.shape[0], krows.shape[0]
+    dQ = np.empty((n_q, d)); dKd = np.empty((n_q, l, d)); dVd = np.empty((n_q, l, d))
+    dK = np.empty((n_k, d)); dV = np.empty((n_k, d))
+    rc = _load().moda_oracle_bwd_rows(_ptr(Q), _ptr(K), _ptr(V), _ptr(Kd), _ptr(Vd), _ptr(dO),
+                                      B, T, H, d, l, float(scale),
+                                      qrows.ctypes.data_as(_ip), n_q, krows.ctypes.data_as(_ip), n_k, int(t_start),
+                                      _ptr(dQ), _ptr(dKd), _ptr(dVd), _ptr(dK), _ptr(dV))
+    if rc == -2:
+        raise ValueError("every key row must be >= t_start")
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return dQ, dKd, dVd, dK, dV

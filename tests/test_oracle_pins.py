@@ -273,3 +273,28 @@ def test_p7_gradient_sum_identities():
     Qc = np.broadcast_to(Q[:, :1], Q.shape).copy()
     _, dK2, _, dKd2, _ = orc.backward(Qc, K, V, Kd, Vd, dO, 0.3)
     np.testing.assert_allclose(dK2.sum(axis=1) + dKd2.sum(axis=(0, 2)), 0.0, atol=1e-11)
+
+
+def test_p6_sampled_row_backward_matches_library_autograd_and_full_backward():
+    rng = np.random.default_rng(13)
+    B, T, H, d, l = 2, 19, 2, 4, 3
+    Q, K, V, Kd, Vd, dO = rand_inputs(rng, B, T, H, d, l)
+    scale = 0.55
+    ts = [torch.from_numpy(x).clone().requires_grad_(True) for x in (Q, K, V, Kd, Vd)]
+    o, _ = flattened_masked_attention(*ts, scale)
+    o.backward(torch.from_numpy(dO))
+    gQ, gK, gV, gKd, gVd = (t.grad.numpy() for t in ts)
+    qrows = np.array([[0, 0, 0], [1, 1, 18], [0, 1, 7], [1, 0, 12]], dtype=np.int32)
+    krows = np.array([[0, 0, 11], [1, 1, 18], [0, 1, 15], [0, 0, 13]], dtype=np.int32)
+    dQ, dKd, dVd, dK, dV = orc.backward_rows(Q, K, V, Kd, Vd, dO, scale, qrows, krows, t_start=11)
+    for n, (b, h, t) in enumerate(qrows):
+        np.testing.assert_allclose(dQ[n], gQ[b, t, h], rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(dKd[n], gKd[:, b, t, h], rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(dVd[n], gVd[:, b, t, h], rtol=1e-10, atol=1e-12)
+    for n, (b, h, j) in enumerate(krows):
+        np.testing.assert_allclose(dK[n], gK[b, j, h], rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(dV[n], gV[b, j, h], rtol=1e-10, atol=1e-12)
+    full = orc.backward(Q, K, V, Kd, Vd, dO, scale)
+    np.testing.assert_allclose(dQ[1], full[0][1, 18, 1], rtol=1e-12, atol=1e-14)
+    with pytest.raises(ValueError):
+        orc.backward_rows(Q, K, V, Kd, Vd, dO, scale, qrows, krows, t_start=12)

@@ -8,17 +8,17 @@
 //                        P_j = exp2(S_j c - m) as packed bf16 back into the TMEM columns of
 //                        S_j, rescales the O accumulator only when the running maximum grew
 //                        by more than 2^8, and runs the epilogue.
-//   warps 4-7  depth     one thread per query row.  Reads the row's l depth keys/values
-//                        straight from the depth cache (16-byte loads, a warp reads 512
-//                        contiguous bytes), builds an independent partial softmax state
+//   warps 4-7  depth     one thread per query row.  Reads the row's l depth keys/values from
+//                        a shared-memory ring that warp 10 fills with 16 KiB bulk copies of
+//                        the depth cache, builds an independent partial softmax state
 //                        (m_d, l_d, o_d) on the CUDA cores and parks o_d in TMEM.  Merging
 //                        two partial softmax states is exact, so the epilogue obtains the
 //                        single softmax over sequence and depth keys that the paper defines.
 //   warp 8     TMA       one lane streams the Q tile and the K_j / V_j tiles (128B swizzle)
 //                        through two-stage rings.
-//   warp 9     MMA       (warps 10, 11 idle: they complete the third warpgroup so that
-//                        registers can be re-balanced between warpgroups)
-//                        one lane issues S_j = Q K_j^T (operands in shared memory) and
+//   warp 10    depth producer (one lane); warp 11 idle (completes the third warpgroup so
+//                        that registers can be re-balanced between warpgroups)
+//   warp 9     MMA       one lane issues S_j = Q K_j^T (operands in shared memory) and
 //                        O += P_j V_j (P_j from TMEM, V_j MN-major in shared memory); also
 //                        owns the TMEM allocation.
 //
@@ -45,8 +45,11 @@ struct FwdSmem {
     static constexpr int kV = kK + 2 * kTileBytes;                // 2 stages
     static constexpr int kU = kV + 2 * kTileBytes;                // depth scores [32][128] fp32
     static constexpr int kMd = kU + 32 * kTileRows * 4;           // m_d [128], l_d [128]
-    static constexpr int kBars = kMd + 2 * kTileRows * 4;
-    static constexpr int kNumBars = 18;
+    static constexpr int kRing = kMd + 2 * kTileRows * 4;         // depth units: 8 chunks x 128 rows x 16 B
+    static constexpr int kUnitBytes = 8 * kTileRows * 16;         // 16 KiB, contiguous in the depth cache
+    static constexpr int kRingStages = (D == 128) ? 3 : 6;
+    static constexpr int kBars = kRing + kRingStages * kUnitBytes;
+    static constexpr int kNumBars = 32;
     static constexpr int kMisc = kBars + kNumBars * 8;            // tmem base, abort flag
     static constexpr int kTotal = kMisc + 16;
     static constexpr int kDynamic = kTotal + 1024;                // slack for 1024-byte alignment
@@ -64,6 +67,8 @@ enum FwdBar : int {
     kBarDepth = 14,
     kBarOFinal = 15,  // single phase: every MMA of the CTA has completed
     kBarDrain = 16,
+    kBarDFull = 17,   // +ring stage (<= 6): depth unit landed
+    kBarDEmpty = 23,  // +ring stage (<= 6): all 128 depth threads have read the unit
 };
 
 struct FwdParams {
@@ -87,7 +92,6 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 const FwdParams p) {
     using L = FwdSmem<D>;
     constexpr int NSUB = D / 64;
-    constexpr int CH = D / 8;
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColO = 256, kColOd = 384;
 
@@ -129,6 +133,10 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         mbar_init(bar(kBarDepth), 128);
         mbar_init(bar(kBarOFinal), 1);
         mbar_init(bar(kBarDrain), 1);
+        for (int s = 0; s < L::kRingStages; ++s) {
+            mbar_init(bar(kBarDFull + s), 1);
+            mbar_init(bar(kBarDEmpty + s), 128);
+        }
         fence_mbar_init();
     }
     if (warp == 9) {
@@ -287,12 +295,18 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         if (p.l > 0) {
             const int r = tid - 128;
             const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
-            const int ntile = nq;
-            const size_t slot_stride = cache_slot_elems(p.B, p.T, p.H, D) / 8;           // in uint4
-            const uint4* blkK = reinterpret_cast<const uint4*>(p.depth_kv) +
-                                (((size_t(b) * p.H + h) * ntile + qt) * 2 + 0) * (kTileRows * CH) + r;
-            const uint4* blkV = blkK + kTileRows * CH;
             mbar_wait(bar(kBarQ), 0, abort_flag, 20);
+            int unit = 0;                                 // running index into the producer's unit sequence
+            // Reads this thread's 8 x 16 bytes of the next depth unit from the ring and frees the stage.
+            auto take_unit = [&](uint4 (&dst)[8]) {
+                const int st = unit % L::kRingStages;
+                mbar_wait(bar(kBarDFull + st), (unit / L::kRingStages) & 1, abort_flag, 21);
+                const uint8_t* src = smem + L::kRing + st * L::kUnitBytes + r * 16;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) dst[c] = *reinterpret_cast<const uint4*>(src + c * (kTileRows * 16));
+                mbar_arrive(bar(kBarDEmpty + st));
+                ++unit;
+            };
             // ---- depth scores u_i = <q, kd_i>, 64 features per sweep ----
 #pragma unroll 1
             for (int half = 0; half < NSUB; ++half) {
@@ -305,19 +319,10 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                     q[8 * c + 4] = bf16_lo_to_f32(v.z); q[8 * c + 5] = bf16_hi_to_f32(v.z);
                     q[8 * c + 6] = bf16_lo_to_f32(v.w); q[8 * c + 7] = bf16_hi_to_f32(v.w);
                 }
-                uint4 kb[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) kb[c] = __ldg(blkK + (half * 8 + c) * kTileRows);
 #pragma unroll 1
                 for (int i = 0; i < p.l; ++i) {
                     uint4 cur[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) cur[c] = kb[c];
-                    if (i + 1 < p.l) {
-                        const uint4* nxt = blkK + size_t(i + 1) * slot_stride + (half * 8) * kTileRows;
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) kb[c] = __ldg(nxt + c * kTileRows);
-                    }
+                    take_unit(cur);
                     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
@@ -352,19 +357,10 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 float acc[64];
 #pragma unroll
                 for (int c = 0; c < 64; ++c) acc[c] = 0.f;
-                uint4 vb[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) vb[c] = __ldg(blkV + (half * 8 + c) * kTileRows);
 #pragma unroll 1
                 for (int i = 0; i < p.l; ++i) {
                     uint4 cur[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) cur[c] = vb[c];
-                    if (i + 1 < p.l) {
-                        const uint4* nxt = blkV + size_t(i + 1) * slot_stride + (half * 8) * kTileRows;
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) vb[c] = __ldg(nxt + c * kTileRows);
-                    }
+                    take_unit(cur);
                     const float w = sU[i * kTileRows + r];
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
@@ -462,6 +458,29 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 const uint64_t t0 = globaltimer_ns();
                 while (!mbar_try_wait(bar(kBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
             }
+        }
+      } else if (warp == 10) {
+        // =========================== depth-cache producer ===========================
+        // Streams the tile's depth keys, then values, as 16 KiB units (8 feature chunks of one slot:
+        // one contiguous run of the cache) through the ring, in the order the depth warps consume
+        // them.  The ring keeps up to kRingStages x 16 KiB of HBM reads in flight per SM.
+        if (lane == 0 && p.l > 0) {
+            const uint64_t policy = l2_policy_evict_first();          // the depth cache is read exactly once
+            const size_t slot_bytes = cache_slot_elems(p.B, p.T, p.H, D) * 2;
+            const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
+                                 (((size_t(b) * p.H + h) * nq + qt) * 2) * (size_t(kTileRows) * D * 2);
+            int unit = 0;
+            for (int kv = 0; kv < 2; ++kv)
+                for (int half = 0; half < NSUB; ++half)
+                    for (int i = 0; i < p.l; ++i, ++unit) {
+                        const int st = unit % L::kRingStages;
+                        if (unit >= L::kRingStages)
+                            mbar_wait(bar(kBarDEmpty + st), ((unit / L::kRingStages) - 1) & 1, abort_flag, 32);
+                        mbar_arrive_expect_tx(bar(kBarDFull + st), L::kUnitBytes);
+                        bulk_load(sbase + L::kRing + st * L::kUnitBytes,
+                                  blk + size_t(i) * slot_bytes + size_t(kv) * (size_t(kTileRows) * D * 2) + size_t(half) * L::kUnitBytes,
+                                  L::kUnitBytes, bar(kBarDFull + st), policy);
+                    }
         }
       }
     }

@@ -90,8 +90,11 @@ struct DqSmem {
     static constexpr int kKV = kdO + kTileBytes;                     // stages of [K_j | V_j]
     static constexpr int kU = kKV + kStages * 2 * kHalfTileBytes;    // [32][128] fp32: u_i, then R_i
     static constexpr int kDr = kU + 32 * kTileRows * 4;              // [32][128] fp32: <dO,Vd_i>, then dU_i
-    static constexpr int kBars = kDr + 32 * kTileRows * 4;
-    static constexpr int kNumBars = 16;
+    static constexpr int kRing = kDr + 32 * kTileRows * 4;           // depth units: 8 chunks x 128 rows x 16 B
+    static constexpr int kUnitBytes = 8 * kTileRows * 16;
+    static constexpr int kRingStages = (D == 128) ? 2 : 6;
+    static constexpr int kBars = kRing + kRingStages * kUnitBytes;
+    static constexpr int kNumBars = 32;
     static constexpr int kMisc = kBars + kNumBars * 8;
     static constexpr int kTotal = kMisc + 16;
     static constexpr int kDynamic = kTotal + 1024;
@@ -106,6 +109,8 @@ enum DqBar : int {
     kDqBarFinal = 11,
     kDqBarDepth = 12,
     kDqBarDrain = 13,
+    kDqBarDFull = 14,    // +ring stage (<= 6)
+    kDqBarDEmpty = 20,   // +ring stage (<= 6)
 };
 
 struct DqParams {
@@ -168,6 +173,10 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         mbar_init(bar(kDqBarFinal), 1);
         mbar_init(bar(kDqBarDepth), 128);
         mbar_init(bar(kDqBarDrain), 1);
+        for (int s = 0; s < L::kRingStages; ++s) {
+            mbar_init(bar(kDqBarDFull + s), 1);
+            mbar_init(bar(kDqBarDEmpty + s), 128);
+        }
         fence_mbar_init();
     }
     if (warp == 9) {
@@ -274,16 +283,20 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             const float delta = valid ? p.delta[row_idx] : 0.f;
             const size_t slot_stride = cache_slot_elems(p.B, p.T, p.H, D) / 8;          // in uint4
             const size_t blk = (((size_t(b) * p.H + h) * nq + qt) * 2) * (kTileRows * CH) + r;
-            const uint4* blkK = reinterpret_cast<const uint4*>(p.depth_kv) + blk;
-            const uint4* blkV = blkK + kTileRows * CH;
             uint4* gK = reinterpret_cast<uint4*>(p.d_depth_kv) + blk;
             uint4* gV = gK + kTileRows * CH;
             mbar_wait(bar(kDqBarQ), 0, abort_flag, 60);
 
-            auto load8 = [&](uint4 (&dst)[8], const uint4* base, int i, int half) {
-                const uint4* src = base + size_t(i) * slot_stride + (half * 8) * kTileRows;
+            int unit = 0;                                 // running index into the producer's unit sequence
+            // Reads this thread's 8 x 16 bytes of the next depth unit from the ring and frees the stage.
+            auto take_unit = [&](uint4 (&dst)[8]) {
+                const int st = unit % L::kRingStages;
+                mbar_wait(bar(kDqBarDFull + st), (unit / L::kRingStages) & 1, abort_flag, 61);
+                const uint8_t* src = smem + L::kRing + st * L::kUnitBytes + r * 16;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) dst[c] = __ldg(src + c * kTileRows);
+                for (int c = 0; c < 8; ++c) dst[c] = *reinterpret_cast<const uint4*>(src + c * (kTileRows * 16));
+                mbar_arrive(bar(kDqBarDEmpty + st));
+                ++unit;
             };
             auto load_row_f32 = [&](float (&dst)[64], int smem_off, int half) {
 #pragma unroll
@@ -316,14 +329,10 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             for (int half = 0; half < NSUB; ++half) {
                 float q[64];
                 load_row_f32(q, L::kQ, half);
-                uint4 nxt[8];
-                load8(nxt, blkK, 0, half);
 #pragma unroll 1
                 for (int i = 0; i < p.l; ++i) {
                     uint4 cur[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) cur[c] = nxt[c];
-                    if (i + 1 < p.l) load8(nxt, blkK, i + 1, half);
+                    take_unit(cur);
                     const float part = dot64(q, cur);
                     if (half == 0) sU[i * kTileRows + r] = part;
                     else sU[i * kTileRows + r] += part;
@@ -338,14 +347,10 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             for (int half = 0; half < NSUB; ++half) {
                 float g[64];
                 load_row_f32(g, L::kdO, half);
-                uint4 nxt[8];
-                load8(nxt, blkV, 0, half);
 #pragma unroll 1
                 for (int i = 0; i < p.l; ++i) {
                     uint4 cur[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) cur[c] = nxt[c];
-                    if (i + 1 < p.l) load8(nxt, blkV, i + 1, half);
+                    take_unit(cur);
                     const float part = dot64(g, cur);
                     if (half == 0) sDr[i * kTileRows + r] = part;
                     else sDr[i * kTileRows + r] += part;
@@ -376,14 +381,10 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 float acc[64];
 #pragma unroll
                 for (int c = 0; c < 64; ++c) acc[c] = 0.f;
-                uint4 nxt[8];
-                load8(nxt, blkK, 0, half);
 #pragma unroll 1
                 for (int i = 0; i < p.l; ++i) {
                     uint4 cur[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) cur[c] = nxt[c];
-                    if (i + 1 < p.l) load8(nxt, blkK, i + 1, half);
+                    take_unit(cur);
                     const float du = sDr[i * kTileRows + r];
                     const float sdu = du * p.scale;
                     const uint32_t sdu2 = pack_bf16x2(sdu, sdu);
@@ -489,6 +490,31 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     umma_commit(bar(kDqBarDrain));
                     const uint64_t t0 = globaltimer_ns();
                     while (!mbar_try_wait(bar(kDqBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+                }
+            }
+        } else if (warp == 10) {
+            // =========================== depth-cache producer ===========================
+            // 16 KiB units in the order the depth warps consume them: keys (pass A), values (pass B),
+            // keys again (pass C).
+            if (lane == 0 && p.l > 0) {
+                const uint64_t policy = l2_policy_evict_first();
+                const size_t slot_bytes = cache_slot_elems(p.B, p.T, p.H, D) * 2;
+                const size_t kv_bytes = size_t(kTileRows) * D * 2;
+                const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
+                                     (((size_t(b) * p.H + h) * nq + qt) * 2) * kv_bytes;
+                int unit = 0;
+                for (int pass = 0; pass < 3; ++pass) {
+                    const int kv = (pass == 1) ? 1 : 0;
+                    for (int half = 0; half < NSUB; ++half)
+                        for (int i = 0; i < p.l; ++i, ++unit) {
+                            const int st = unit % L::kRingStages;
+                            if (unit >= L::kRingStages)
+                                mbar_wait(bar(kDqBarDEmpty + st), ((unit / L::kRingStages) - 1) & 1, abort_flag, 71);
+                            mbar_arrive_expect_tx(bar(kDqBarDFull + st), L::kUnitBytes);
+                            bulk_load(sbase + L::kRing + st * L::kUnitBytes,
+                                      blk + size_t(i) * slot_bytes + size_t(kv) * kv_bytes + size_t(half) * L::kUnitBytes,
+                                      L::kUnitBytes, bar(kDqBarDFull + st), policy);
+                        }
                 }
             }
         }

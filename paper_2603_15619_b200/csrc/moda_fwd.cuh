@@ -16,11 +16,13 @@
 //                        single softmax over sequence and depth keys that the paper defines.
 //   warp 8     TMA       one lane streams the Q tile and the K_j / V_j tiles (128B swizzle)
 //                        through two-stage rings.
-//   warp 10    depth producer (one lane); warp 11 idle (completes the third warpgroup so
-//                        that registers can be re-balanced between warpgroups)
-//   warp 9     MMA       one lane issues S_j = Q K_j^T (operands in shared memory) and
-//                        O += P_j V_j (P_j from TMEM, V_j MN-major in shared memory); also
-//                        owns the TMEM allocation.
+//   warp 10    depth producer (one lane)
+//   warp 9     MMA (S)   one lane issues S_j = Q K_j^T (operands in shared memory); owns the
+//                        TMEM allocation.
+//   warp 11    MMA (PV)  one lane issues O += P_j V_j (P_j from TMEM, V_j MN-major in shared
+//                        memory).  One tcgen05.mma costs its issuing thread about 60 cycles, as much
+//                        as a 128x128x16 MMA executes, so the two contractions are issued by two
+//                        threads on different schedulers and ordered by mbarriers.
 //
 // TMEM columns (fp32): [0,128) S_0/P_0   [128,256) S_1/P_1   [256,256+D) O   [384,384+D) o_d.
 // The depth scores never touch the tensor cores and no score matrix is ever materialised.
@@ -58,12 +60,10 @@ struct FwdSmem {
 enum FwdBar : int {
     kBarQ = 0,
     kBarKFull = 1,    // +stage
-    kBarKEmpty = 3,   // +stage
     kBarVFull = 5,    // +stage
-    kBarVEmpty = 7,   // +stage
-    kBarSFull = 9,    // +buffer
+    kBarVEmpty = 7,   // +stage: PV_j complete (V stage and score buffer free; O may be rescaled)
+    kBarSFull = 9,    // +buffer: S_j complete (also frees the K stage)
     kBarPFull = 11,   // +buffer
-    kBarOReady = 13,  // one phase per PV_j (used by the lazy rescale, which knows PV_{j-2} is complete)
     kBarDepth = 14,
     kBarOFinal = 15,  // single phase: every MMA of the CTA has completed
     kBarDrain = 16,
@@ -123,13 +123,11 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         mbar_init(bar(kBarQ), 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(kBarKFull + s), 1);
-            mbar_init(bar(kBarKEmpty + s), 1);
             mbar_init(bar(kBarVFull + s), 1);
             mbar_init(bar(kBarVEmpty + s), 1);
             mbar_init(bar(kBarSFull + s), 1);
             mbar_init(bar(kBarPFull + s), 128);
         }
-        mbar_init(bar(kBarOReady), 1);
         mbar_init(bar(kBarDepth), 128);
         mbar_init(bar(kBarOFinal), 1);
         mbar_init(bar(kBarDrain), 1);
@@ -192,7 +190,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 // The maximum grew a lot: bring O and l to the new reference.  O may only be
                 // touched between PV_{j-1} completing and PV_j being issued; PV_j waits for
                 // this thread's arrival on kBarPFull below.
-                mbar_wait(bar(kBarOReady), (j - 1) & 1, abort_flag, 11);
+                mbar_wait(bar(kBarVEmpty + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag, 11);
                 tc_fence_after_sync();
                 const float f = fast_exp2(m_ref - m_new);
 #pragma unroll
@@ -400,7 +398,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 tma_load_4d(sbase + L::kQ + s * L::kSubBytes, &mapQ, bar(kBarQ), s * 64, h, q0, b);
             for (int j = 0; j < n_kv; ++j) {
                 const int st = j & 1;
-                if (j >= 2) mbar_wait(bar(kBarKEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 30);
+                if (j >= 2) mbar_wait(bar(kBarSFull + st), ((j - 2) >> 1) & 1, abort_flag, 30);   // S_{j-2} complete
                 mbar_arrive_expect_tx(bar(kBarKFull + st), L::kTileBytes);
 #pragma unroll
                 for (int s = 0; s < NSUB; ++s)
@@ -415,48 +413,60 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             }
         }
       } else if (warp == 9) {
-        // =========================== MMA issuer ===========================
+        // =========================== MMA issuer: S_j = Q K_j^T ===========================
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
-            constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
-            auto issue_s = [&](int j) {
+            // every descriptor is built once; inside the loop a descriptor is one 64-bit add (the
+            // start-address field counts 16-byte units and stays inside its 14 bits below 256 KiB)
+            uint64_t dq[D / 16];
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) dq[kk] = desc_kmajor_sw128(sbase + L::kQ + (kk >> 2) * L::kSubBytes, kk & 3);
+            const uint64_t dk0 = desc_kmajor_sw128(sbase + L::kK, 0);
+            mbar_wait(bar(kBarQ), 0, abort_flag, 41);
+            for (int j = 0; j < n_kv; ++j) {
                 const int st = j & 1;
                 mbar_wait(bar(kBarKFull + st), (j >> 1) & 1, abort_flag, 40);
+                // score buffer st still holds P_{j-2} until PV_{j-2} has completed
+                if (j >= 2) mbar_wait(bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 44);
                 tc_fence_after_sync();
-                const uint32_t aQ = sbase + L::kQ, aK = sbase + L::kK + st * L::kTileBytes;
+                const uint64_t dk = dk0 + uint64_t((st * L::kTileBytes) >> 4);
+                const uint32_t ts = tmem + uint32_t(st) * 128u;
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint64_t ad = desc_kmajor_sw128(aQ + (kk >> 2) * L::kSubBytes, kk & 3);
-                    const uint64_t bd = desc_kmajor_sw128(aK + (kk >> 2) * L::kSubBytes, kk & 3);
-                    umma_ss(tmem + uint32_t(st) * 128u, ad, bd, idesc_s, kk > 0);
-                }
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma_ss(ts, dq[kk], dk + uint64_t(((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4), idesc_s, kk > 0);
                 umma_commit(bar(kBarSFull + st));
-                umma_commit(bar(kBarKEmpty + st));
-            };
-            mbar_wait(bar(kBarQ), 0, abort_flag, 41);
-            issue_s(0);
-            if (n_kv > 1) issue_s(1);
+            }
+            if (*abort_flag != 0) {
+                // A wait gave up somewhere: make sure no MMA of this thread is still in flight before TMEM is released.
+                umma_commit(bar(kBarDrain));
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar(kBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+            }
+        }
+      } else if (warp == 11) {
+        // =========================== MMA issuer: O += P_j V_j ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
+            const uint64_t dv0 = desc_mnmajor_sw128(sbase + L::kV, 0, L::kSubBytes);
             for (int j = 0; j < n_kv; ++j) {
                 const int st = j & 1;
                 mbar_wait(bar(kBarVFull + st), (j >> 1) & 1, abort_flag, 42);
                 mbar_wait(bar(kBarPFull + st), (j >> 1) & 1, abort_flag, 43);
                 tc_fence_after_sync();
-                const uint32_t aV = sbase + L::kV + st * L::kTileBytes;
+                const uint64_t dv = dv0 + uint64_t((st * L::kTileBytes) >> 4);
+                const uint32_t tp = tmem + uint32_t(st) * 128u;
+                umma_ts(tmem + kColO, tp, dv, idesc_o, j > 0);
 #pragma unroll
-                for (int kk = 0; kk < kTileRows / 16; ++kk) {
-                    const uint64_t bd = desc_mnmajor_sw128(aV, kk, L::kSubBytes);
-                    umma_ts(tmem + kColO, tmem + uint32_t(st) * 128u + kk * 8, bd, idesc_o, (j > 0) || (kk > 0));
-                }
+                for (int kk = 1; kk < kTileRows / 16; ++kk)
+                    umma_ts(tmem + kColO, tp + kk * 8, dv + uint64_t(kk * 128), idesc_o, 1);
                 umma_commit(bar(kBarVEmpty + st));
-                umma_commit(bar(kBarOReady));
-                if (j + 2 < n_kv) issue_s(j + 2);
             }
+            // All S MMAs completed before the P they fed was written, so the last PV is the last MMA.
             umma_commit(bar(kBarOFinal));
             if (*abort_flag != 0) {
                 // A wait gave up somewhere: make sure no MMA is still in flight before TMEM is released.
-                umma_commit(bar(kBarDrain));
                 const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(bar(kBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+                while (!mbar_try_wait(bar(kBarOFinal), 0) && globaltimer_ns() - t0 < 20000000ull) {}
             }
         }
       } else if (warp == 10) {

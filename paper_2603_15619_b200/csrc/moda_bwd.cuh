@@ -75,7 +75,11 @@ bwd_delta_kernel(const uint4* __restrict__ O, const uint4* __restrict__ dO, floa
 // =====================================================================================
 // dQ + depth gradients
 // =====================================================================================
-constexpr int kBwdDqThreads = 384;
+// 512 threads: warps 0-3 form dS and run the epilogue, warps 4-7 do the depth backward, warp 8 is the
+// TMA producer, warp 9 the depth-cache producer, and the three contractions of a tile are issued by
+// three threads on three schedulers (warp 12: S = Q K^T, warp 13: dP = dO V^T, warp 14: dQ += dS K),
+// ordered by mbarriers only.
+constexpr int kBwdDqThreads = 512;
 constexpr int kKeyTile = 64;     // keys per inner tile of the dQ kernel / queries per inner tile of the dK,dV kernel
 
 template <int D>
@@ -103,14 +107,14 @@ struct DqSmem {
 enum DqBar : int {
     kDqBarQ = 0,
     kDqBarKVFull = 1,    // +stage (3)
-    kDqBarKVEmpty = 4,   // +stage (3)
-    kDqBarSFull = 7,     // +buffer (2)
-    kDqBarPFull = 9,     // +buffer (2)
+    kDqBarKVEmpty = 4,   // +stage (3): dQ_j complete (K_j, V_j and the score buffer are free)
+    kDqBarSFull = 7,     // +buffer (2), count 2: S_j and dP_j complete
+    kDqBarPFull = 9,     // +buffer (2), count 128: dS_j written (and dP_j consumed)
     kDqBarFinal = 11,
     kDqBarDepth = 12,
-    kDqBarDrain = 13,
-    kDqBarDFull = 14,    // +ring stage (<= 6)
-    kDqBarDEmpty = 20,   // +ring stage (<= 6)
+    kDqBarDrain = 13,    // +issuer (3): abort path only
+    kDqBarDFull = 16,    // +ring stage (<= 6)
+    kDqBarDEmpty = 22,   // +ring stage (<= 6)
 };
 
 struct DqParams {
@@ -167,19 +171,19 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             mbar_init(bar(kDqBarKVEmpty + s), 1);
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(kDqBarSFull + s), 1);
+            mbar_init(bar(kDqBarSFull + s), 2);
             mbar_init(bar(kDqBarPFull + s), 128);
         }
         mbar_init(bar(kDqBarFinal), 1);
         mbar_init(bar(kDqBarDepth), 128);
-        mbar_init(bar(kDqBarDrain), 1);
+        for (int s = 0; s < 3; ++s) mbar_init(bar(kDqBarDrain + s), 1);
         for (int s = 0; s < L::kRingStages; ++s) {
             mbar_init(bar(kDqBarDFull + s), 1);
             mbar_init(bar(kDqBarDEmpty + s), 128);
         }
         fence_mbar_init();
     }
-    if (warp == 9) {
+    if (warp == 12) {
         tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -188,9 +192,18 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
+    // Abort path of an issuing thread: wait (bounded) until its own MMAs have drained.
+    auto drain_on_abort = [&](int which) {
+        if (*abort_flag != 0) {
+            umma_commit(bar(kDqBarDrain + which));
+            const uint64_t t0 = globaltimer_ns();
+            while (!mbar_try_wait(bar(kDqBarDrain + which), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+        }
+    };
+
     if (warp < 4) {
         // =========================== P, dS and the dQ epilogue ===========================
-        setmaxnreg_inc<216>();
+        setmaxnreg_inc<168>();
         const int r = tid;
         const uint32_t lane_addr = uint32_t(warp * 32) << 16;
         const bool valid = q0 + r < p.T;
@@ -201,33 +214,29 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             const int buf = j & 1;
             mbar_wait(bar(kDqBarSFull + buf), (j >> 1) & 1, abort_flag, 50);
             tc_fence_after_sync();
-            uint32_t s0[32], s1[32], g0[32], g1[32];
-            tmem_ld32(tmem + lane_addr + kColS + buf * 64, s0);
-            tmem_ld32(tmem + lane_addr + kColS + buf * 64 + 32, s1);
-            tmem_ld32(tmem + lane_addr + kColdP + buf * 64, g0);
-            tmem_ld32(tmem + lane_addr + kColdP + buf * 64 + 32, g1);
-            tmem_wait_ld();
             const int koff = j * kKeyTile - q0;      // key of column c is visible to row r iff koff + c <= r
             const bool masked = koff + kKeyTile - 1 > 0;
-            uint32_t pk0[16], pk1[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                float pa = fast_exp2(fmaf(__uint_as_float(s0[2 * i]), p.scale_log2, neg_lse2));
-                float pb = fast_exp2(fmaf(__uint_as_float(s0[2 * i + 1]), p.scale_log2, neg_lse2));
-                float pc = fast_exp2(fmaf(__uint_as_float(s1[2 * i]), p.scale_log2, neg_lse2));
-                float pd = fast_exp2(fmaf(__uint_as_float(s1[2 * i + 1]), p.scale_log2, neg_lse2));
-                if (masked) {
-                    if (koff + 2 * i > r) pa = 0.f;
-                    if (koff + 2 * i + 1 > r) pb = 0.f;
-                    if (koff + 32 + 2 * i > r) pc = 0.f;
-                    if (koff + 32 + 2 * i + 1 > r) pd = 0.f;
+            for (int hc = 0; hc < 2; ++hc) {         // 32 key columns at a time
+                uint32_t sv[32], gv[32];
+                tmem_ld32(tmem + lane_addr + kColS + buf * 64 + hc * 32, sv);
+                tmem_ld32(tmem + lane_addr + kColdP + buf * 64 + hc * 32, gv);
+                tmem_wait_ld();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float pa = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), p.scale_log2, neg_lse2));
+                    float pb = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), p.scale_log2, neg_lse2));
+                    if (masked) {
+                        if (koff + hc * 32 + 2 * i > r) pa = 0.f;
+                        if (koff + hc * 32 + 2 * i + 1 > r) pb = 0.f;
+                    }
+                    pk[i] = pack_bf16x2(pa * (__uint_as_float(gv[2 * i]) - delta), pb * (__uint_as_float(gv[2 * i + 1]) - delta));
                 }
-                pk0[i] = pack_bf16x2(pa * (__uint_as_float(g0[2 * i]) - delta), pb * (__uint_as_float(g0[2 * i + 1]) - delta));
-                pk1[i] = pack_bf16x2(pc * (__uint_as_float(g1[2 * i]) - delta), pd * (__uint_as_float(g1[2 * i + 1]) - delta));
+                // dS_j (bf16, two per column) overlays the first 32 columns of S_j; the block just
+                // written (columns 16 hc .. 16 hc + 15) was read in this or the previous half.
+                tmem_st16(tmem + lane_addr + kColS + buf * 64 + hc * 16, pk);
             }
-            // dS_j (bf16, two per column) overlays the first 32 columns of S_j.
-            tmem_st16(tmem + lane_addr + kColS + buf * 64, pk0);
-            tmem_st16(tmem + lane_addr + kColS + buf * 64 + 16, pk1);
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(kDqBarPFull + buf));
@@ -419,8 +428,8 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             tc_fence_before_sync();
             mbar_arrive(bar(kDqBarDepth));
         }
-    } else {
-        setmaxnreg_dec<72>();
+    } else if (warp < 12) {
+        setmaxnreg_dec<64>();
         if (warp == 8) {
             // =========================== TMA producer ===========================
             if (lane == 0) {
@@ -449,50 +458,6 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 }
             }
         } else if (warp == 9) {
-            // =========================== MMA issuer ===========================
-            if (lane == 0) {
-                constexpr uint32_t idesc_s = make_idesc_bf16(128, kKeyTile, false, false);
-                constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, false, true);
-                const uint32_t aQ = sbase + L::kQ, adO = sbase + L::kdO;
-                auto issue_sdp = [&](int j) {
-                    const int st = j % L::kStages, buf = j & 1;
-                    mbar_wait(bar(kDqBarKVFull + st), (j / L::kStages) & 1, abort_flag, 80);
-                    tc_fence_after_sync();
-                    const uint32_t aK = sbase + L::kKV + st * 2 * L::kHalfTileBytes;
-                    const uint32_t aV = aK + L::kHalfTileBytes;
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        umma_ss(tmem + kColS + buf * 64, desc_kmajor_sw128(aQ + (kk >> 2) * L::kSubBytes, kk & 3),
-                                desc_kmajor_sw128(aK + (kk >> 2) * L::kHalfSubBytes, kk & 3), idesc_s, kk > 0);
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        umma_ss(tmem + kColdP + buf * 64, desc_kmajor_sw128(adO + (kk >> 2) * L::kSubBytes, kk & 3),
-                                desc_kmajor_sw128(aV + (kk >> 2) * L::kHalfSubBytes, kk & 3), idesc_s, kk > 0);
-                    umma_commit(bar(kDqBarSFull + buf));
-                };
-                mbar_wait(bar(kDqBarQ), 0, abort_flag, 81);
-                issue_sdp(0);
-                if (n_kv > 1) issue_sdp(1);
-                for (int j = 0; j < n_kv; ++j) {
-                    const int st = j % L::kStages, buf = j & 1;
-                    mbar_wait(bar(kDqBarPFull + buf), (j >> 1) & 1, abort_flag, 82);
-                    tc_fence_after_sync();
-                    const uint32_t aK = sbase + L::kKV + st * 2 * L::kHalfTileBytes;
-#pragma unroll
-                    for (int kk = 0; kk < kKeyTile / 16; ++kk)
-                        umma_ts(tmem + kColdQ, tmem + kColS + buf * 64 + kk * 8,
-                                desc_mnmajor_sw128(aK, kk, L::kHalfSubBytes), idesc_dq, (j > 0) || (kk > 0));
-                    umma_commit(bar(kDqBarKVEmpty + st));
-                    if (j + 2 < n_kv) issue_sdp(j + 2);
-                }
-                umma_commit(bar(kDqBarFinal));
-                if (*abort_flag != 0) {
-                    umma_commit(bar(kDqBarDrain));
-                    const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(bar(kDqBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
-                }
-            }
-        } else if (warp == 10) {
             // =========================== depth-cache producer ===========================
             // 16 KiB units in the order the depth warps consume them: keys (pass A), values (pass B),
             // keys again (pass C).
@@ -518,6 +483,58 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 }
             }
         }
+    } else {
+        setmaxnreg_dec<64>();
+        if (warp == 12 || warp == 13) {
+            // ============ MMA issuers: S = Q K^T (warp 12), dP = dO V^T (warp 13) ============
+            if (lane == 0) {
+                const bool is_s = (warp == 12);
+                constexpr uint32_t idesc_s = make_idesc_bf16(128, kKeyTile, false, false);
+                const uint32_t a_tile = sbase + (is_s ? L::kQ : L::kdO);
+                const uint32_t col = is_s ? kColS : kColdP;
+                uint64_t da[D / 16];
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) da[kk] = desc_kmajor_sw128(a_tile + (kk >> 2) * L::kSubBytes, kk & 3);
+                const uint64_t db0 = desc_kmajor_sw128(sbase + L::kKV + (is_s ? 0 : L::kHalfTileBytes), 0);
+                mbar_wait(bar(kDqBarQ), 0, abort_flag, 81);
+                for (int j = 0; j < n_kv; ++j) {
+                    const int st = j % L::kStages, buf = j & 1;
+                    mbar_wait(bar(kDqBarKVFull + st), (j / L::kStages) & 1, abort_flag, 80);
+                    if (j >= 2) {
+                        // S buffer: dS_{j-2} overlays it until dQ_{j-2} has completed;
+                        // dP buffer: free once the row warps have read dP_{j-2} (their arrival for tile j-2)
+                        if (is_s) mbar_wait(bar(kDqBarKVEmpty + (j - 2) % L::kStages), ((j - 2) / L::kStages) & 1, abort_flag, 83);
+                        else mbar_wait(bar(kDqBarPFull + buf), ((j - 2) >> 1) & 1, abort_flag, 84);
+                    }
+                    tc_fence_after_sync();
+                    const uint64_t db = db0 + uint64_t((st * 2 * L::kHalfTileBytes) >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma_ss(tmem + col + buf * 64, da[kk], db + uint64_t(((kk >> 2) * L::kHalfSubBytes + (kk & 3) * 32) >> 4), idesc_s, kk > 0);
+                    umma_commit(bar(kDqBarSFull + buf));
+                }
+                drain_on_abort(is_s ? 0 : 1);
+            }
+        } else if (warp == 14) {
+            // ============ MMA issuer: dQ += dS K (warp 14) ============
+            if (lane == 0) {
+                constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, false, true);
+                const uint64_t db0 = desc_mnmajor_sw128(sbase + L::kKV, 0, L::kHalfSubBytes);
+                for (int j = 0; j < n_kv; ++j) {
+                    const int st = j % L::kStages, buf = j & 1;
+                    mbar_wait(bar(kDqBarPFull + buf), (j >> 1) & 1, abort_flag, 82);
+                    tc_fence_after_sync();
+                    const uint64_t db = db0 + uint64_t((st * 2 * L::kHalfTileBytes) >> 4);
+                    umma_ts(tmem + kColdQ, tmem + kColS + buf * 64, db, idesc_dq, j > 0);
+#pragma unroll
+                    for (int kk = 1; kk < kKeyTile / 16; ++kk)
+                        umma_ts(tmem + kColdQ, tmem + kColS + buf * 64 + kk * 8, db + uint64_t(kk * 128), idesc_dq, 1);
+                    umma_commit(bar(kDqBarKVEmpty + st));
+                }
+                umma_commit(bar(kDqBarFinal));
+                drain_on_abort(2);
+            }
+        }
     }
 
     tc_fence_before_sync();
@@ -527,13 +544,18 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         while (globaltimer_ns() - t0 < 2000000ull) {}
     }
     __syncthreads();
-    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 12) tmem_dealloc(tmem, kTmemCols);
 }
 
 // =====================================================================================
 // dK, dV
 // =====================================================================================
-constexpr int kBwdDkvThreads = 192;
+// 384 threads: warps 0-3 form P^T / dS^T and run the epilogue, warp 4 loads, and the four
+// contractions of an iteration are issued by four threads on four schedulers (one tcgen05.mma
+// costs its issuing thread about as long as a 128x64x16 MMA runs twice over, so a single issuer
+// would be the bottleneck): warp 5 S^T = K Q^T, warp 6 dP^T = V dO^T, warp 7 dV += P^T dO,
+// warp 8 dK += dS^T Q.  MMAs of different threads are ordered by mbarriers only.
+constexpr int kBwdDkvThreads = 384;
 
 template <int D>
 struct DkvSmem {
@@ -556,12 +578,12 @@ struct DkvSmem {
 
 enum DkvBar : int {
     kDkvBarKV = 0,
-    kDkvBarQFull = 1,    // +stage (3)
-    kDkvBarQEmpty = 4,   // +stage (3)
-    kDkvBarSFull = 7,    // +buffer (2)
-    kDkvBarPFull = 9,    // +buffer (2)
-    kDkvBarFinal = 11,
-    kDkvBarDrain = 12,
+    kDkvBarQFull = 1,    // +stage (3): Q_i, dO_i, LSE, D_t of the stage have landed
+    kDkvBarQEmpty = 4,   // +stage (3), count 2: dV and dK of the stage's iteration are complete
+    kDkvBarSFull = 7,    // +buffer (2), count 2: S^T and dP^T of the iteration are complete
+    kDkvBarPFull = 9,    // +buffer (2), count 128: P^T and dS^T are written
+    kDkvBarFinal = 11,   // count 2: the last dV and dK are complete
+    kDkvBarDrain = 12,   // +issuer (4): abort path only
 };
 
 struct DkvParams {
@@ -608,14 +630,14 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         mbar_init(bar(kDkvBarKV), 1);
         for (int s = 0; s < L::kStages; ++s) {
             mbar_init(bar(kDkvBarQFull + s), 32);
-            mbar_init(bar(kDkvBarQEmpty + s), 1);
+            mbar_init(bar(kDkvBarQEmpty + s), 2);
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(kDkvBarSFull + s), 1);
+            mbar_init(bar(kDkvBarSFull + s), 2);
             mbar_init(bar(kDkvBarPFull + s), 128);
         }
-        mbar_init(bar(kDkvBarFinal), 1);
-        mbar_init(bar(kDkvBarDrain), 1);
+        mbar_init(bar(kDkvBarFinal), 2);
+        for (int s = 0; s < 4; ++s) mbar_init(bar(kDkvBarDrain + s), 1);
         fence_mbar_init();
     }
     if (warp == 5) {
@@ -627,8 +649,18 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
+    // Abort path of an issuing thread: wait (bounded) until its own MMAs have drained.
+    auto drain_on_abort = [&](int which) {
+        if (*abort_flag != 0) {
+            umma_commit(bar(kDkvBarDrain + which));
+            const uint64_t t0 = globaltimer_ns();
+            while (!mbar_try_wait(bar(kDkvBarDrain + which), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+        }
+    };
+
     if (warp < 4) {
         // =========================== P^T, dS^T and the dK / dV epilogue ===========================
+        setmaxnreg_inc<232>();
         const int r = tid;                                   // key row inside the tile = TMEM lane
         const uint32_t lane_addr = uint32_t(warp * 32) << 16;
         for (int it = 0; it < n_it; ++it) {
@@ -701,7 +733,9 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tma_store_commit();
             tma_store_wait_all();
         }
-    } else if (warp == 4) {
+    } else if (warp < 8) {
+      setmaxnreg_dec<64>();
+      if (warp == 4) {
         // =========================== loader: TMA tiles + per-query LSE, D_t ===========================
         if (lane == 0) {
             tma_prefetch_desc(&mapK);
@@ -742,55 +776,74 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 mbar_arrive(bar(kDkvBarQFull + st));
             }
         }
-    } else {
-        // =========================== MMA issuer ===========================
+      } else if (warp == 5 || warp == 6) {
+        // ============ MMA issuers: S^T = K Q^T (warp 5), dP^T = V dO^T (warp 6) ============
         if (lane == 0) {
+            const bool is_s = (warp == 5);
             constexpr uint32_t idesc_s = make_idesc_bf16(128, kKeyTile, false, false);
-            constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
-            const uint32_t aK = sbase + L::kK, aV = sbase + L::kV;
-            auto issue_s = [&](int it) {
+            const uint32_t a_tile = sbase + (is_s ? L::kK : L::kV);
+            const uint32_t col = is_s ? kColST : kColdPT;
+            uint64_t da[D / 16];
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) da[kk] = desc_kmajor_sw128(a_tile + (kk >> 2) * L::kSubBytes, kk & 3);
+            const uint64_t db0 = desc_kmajor_sw128(sbase + L::kQdO + (is_s ? 0 : L::kHalfTileBytes), 0);
+            mbar_wait(bar(kDkvBarKV), 0, abort_flag, 111);
+            for (int it = 0; it < n_it; ++it) {
                 const int st = it % L::kStages, buf = it & 1;
                 mbar_wait(bar(kDkvBarQFull + st), (it / L::kStages) & 1, abort_flag, 110);
+                // buffer `buf` still feeds dV / dK of iteration it-2 (P^T, dS^T overlay it)
+                if (it >= 2) mbar_wait(bar(kDkvBarQEmpty + (it - 2) % L::kStages), ((it - 2) / L::kStages) & 1, abort_flag, 113);
                 tc_fence_after_sync();
-                const uint32_t aQ = sbase + L::kQdO + st * 2 * L::kHalfTileBytes;
-                const uint32_t adO = aQ + L::kHalfTileBytes;
+                const uint64_t db = db0 + uint64_t((st * 2 * L::kHalfTileBytes) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
-                    umma_ss(tmem + kColST + buf * 64, desc_kmajor_sw128(aK + (kk >> 2) * L::kSubBytes, kk & 3),
-                            desc_kmajor_sw128(aQ + (kk >> 2) * L::kHalfSubBytes, kk & 3), idesc_s, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    umma_ss(tmem + kColdPT + buf * 64, desc_kmajor_sw128(aV + (kk >> 2) * L::kSubBytes, kk & 3),
-                            desc_kmajor_sw128(adO + (kk >> 2) * L::kHalfSubBytes, kk & 3), idesc_s, kk > 0);
+                    umma_ss(tmem + col + buf * 64, da[kk], db + uint64_t(((kk >> 2) * L::kHalfSubBytes + (kk & 3) * 32) >> 4), idesc_s, kk > 0);
                 umma_commit(bar(kDkvBarSFull + buf));
-            };
-            mbar_wait(bar(kDkvBarKV), 0, abort_flag, 111);
-            issue_s(0);
-            if (n_it > 1) issue_s(1);
+            }
+            drain_on_abort(is_s ? 0 : 1);
+        }
+      } else {
+        // ============ MMA issuer: dV += P^T dO (warp 7) ============
+        if (lane == 0) {
+            constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
+            const uint64_t db0 = desc_mnmajor_sw128(sbase + L::kQdO + L::kHalfTileBytes, 0, L::kHalfSubBytes);
             for (int it = 0; it < n_it; ++it) {
                 const int st = it % L::kStages, buf = it & 1;
                 mbar_wait(bar(kDkvBarPFull + buf), (it >> 1) & 1, abort_flag, 112);
                 tc_fence_after_sync();
-                const uint32_t aQ = sbase + L::kQdO + st * 2 * L::kHalfTileBytes;
-                const uint32_t adO = aQ + L::kHalfTileBytes;
+                const uint64_t db = db0 + uint64_t((st * 2 * L::kHalfTileBytes) >> 4);
+                umma_ts(tmem + kColdV, tmem + kColST + buf * 64, db, idesc_acc, it > 0);
 #pragma unroll
-                for (int kk = 0; kk < kKeyTile / 16; ++kk)
-                    umma_ts(tmem + kColdV, tmem + kColST + buf * 64 + kk * 8,
-                            desc_mnmajor_sw128(adO, kk, L::kHalfSubBytes), idesc_acc, (it > 0) || (kk > 0));
-#pragma unroll
-                for (int kk = 0; kk < kKeyTile / 16; ++kk)
-                    umma_ts(tmem + kColdK, tmem + kColdPT + buf * 64 + kk * 8,
-                            desc_mnmajor_sw128(aQ, kk, L::kHalfSubBytes), idesc_acc, (it > 0) || (kk > 0));
+                for (int kk = 1; kk < kKeyTile / 16; ++kk)
+                    umma_ts(tmem + kColdV, tmem + kColST + buf * 64 + kk * 8, db + uint64_t(kk * 128), idesc_acc, 1);
                 umma_commit(bar(kDkvBarQEmpty + st));
-                if (it + 2 < n_it) issue_s(it + 2);
             }
             umma_commit(bar(kDkvBarFinal));
-            if (*abort_flag != 0) {
-                umma_commit(bar(kDkvBarDrain));
-                const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(bar(kDkvBarDrain), 0) && globaltimer_ns() - t0 < 20000000ull) {}
-            }
+            drain_on_abort(2);
         }
+      }
+    } else {
+      setmaxnreg_dec<64>();
+      if (warp == 8) {
+        // ============ MMA issuer: dK += dS^T Q (warp 8) ============
+        if (lane == 0) {
+            constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
+            const uint64_t db0 = desc_mnmajor_sw128(sbase + L::kQdO, 0, L::kHalfSubBytes);
+            for (int it = 0; it < n_it; ++it) {
+                const int st = it % L::kStages, buf = it & 1;
+                mbar_wait(bar(kDkvBarPFull + buf), (it >> 1) & 1, abort_flag, 114);
+                tc_fence_after_sync();
+                const uint64_t db = db0 + uint64_t((st * 2 * L::kHalfTileBytes) >> 4);
+                umma_ts(tmem + kColdK, tmem + kColdPT + buf * 64, db, idesc_acc, it > 0);
+#pragma unroll
+                for (int kk = 1; kk < kKeyTile / 16; ++kk)
+                    umma_ts(tmem + kColdK, tmem + kColdPT + buf * 64 + kk * 8, db + uint64_t(kk * 128), idesc_acc, 1);
+                umma_commit(bar(kDkvBarQEmpty + st));
+            }
+            umma_commit(bar(kDkvBarFinal));
+            drain_on_abort(3);
+        }
+      }
     }
 
     tc_fence_before_sync();

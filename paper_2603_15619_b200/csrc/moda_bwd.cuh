@@ -550,12 +550,13 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
 // =====================================================================================
 // dK, dV
 // =====================================================================================
-// 384 threads: warps 0-3 form P^T / dS^T and run the epilogue, warp 4 loads, and the four
-// contractions of an iteration are issued by four threads on four schedulers (one tcgen05.mma
-// costs its issuing thread about as long as a 128x64x16 MMA runs twice over, so a single issuer
-// would be the bottleneck): warp 5 S^T = K Q^T, warp 6 dP^T = V dO^T, warp 7 dV += P^T dO,
-// warp 8 dK += dS^T Q.  MMAs of different threads are ordered by mbarriers only.
-constexpr int kBwdDkvThreads = 384;
+// 512 threads.  Warps 0-3 and 4-7 form P^T / dS^T (each warpgroup takes 32 of the 64 query columns
+// of an iteration; a thread owns one key row) and run the epilogue (dK by the first, dV by the
+// second).  Warp 8 loads.  The four contractions of an iteration are issued by four threads on four
+// schedulers, because one tcgen05.mma costs its issuing thread about 60 cycles: warp 9 S^T = K Q^T,
+// warp 10 dP^T = V dO^T, warp 11 dV += P^T dO, warp 12 dK += dS^T Q.  MMAs of different threads are
+// ordered by mbarriers only.
+constexpr int kBwdDkvThreads = 512;
 
 template <int D>
 struct DkvSmem {
@@ -567,9 +568,9 @@ struct DkvSmem {
     static constexpr int kK = 0;
     static constexpr int kV = kK + kTileBytes;
     static constexpr int kQdO = kV + kTileBytes;                       // stages of [Q_i | dO_i]
-    static constexpr int kLse = kQdO + kStages * 2 * kHalfTileBytes;   // [stage][64] -LSE*log2(e)
-    static constexpr int kDelta = kLse + kStages * kKeyTile * 4;       // [stage][64]
-    static constexpr int kBars = kDelta + kStages * kKeyTile * 4;
+    // per stage, per pair of query columns: {-LSE c, -LSE c+1, D c, D c+1} (one 16-byte load per pair)
+    static constexpr int kRowTerms = kQdO + kStages * 2 * kHalfTileBytes;
+    static constexpr int kBars = kRowTerms + kStages * kKeyTile * 8;
     static constexpr int kNumBars = 16;
     static constexpr int kMisc = kBars + kNumBars * 8;
     static constexpr int kTotal = kMisc + 16;
@@ -581,7 +582,7 @@ enum DkvBar : int {
     kDkvBarQFull = 1,    // +stage (3): Q_i, dO_i, LSE, D_t of the stage have landed
     kDkvBarQEmpty = 4,   // +stage (3), count 2: dV and dK of the stage's iteration are complete
     kDkvBarSFull = 7,    // +buffer (2), count 2: S^T and dP^T of the iteration are complete
-    kDkvBarPFull = 9,    // +buffer (2), count 128: P^T and dS^T are written
+    kDkvBarPFull = 9,    // +buffer (2), count 256: P^T and dS^T are written
     kDkvBarFinal = 11,   // count 2: the last dV and dK are complete
     kDkvBarDrain = 12,   // +issuer (4): abort path only
 };
@@ -609,8 +610,7 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
-    float* sLse = reinterpret_cast<float*>(smem + L::kLse);
-    float* sDelta = reinterpret_cast<float*>(smem + L::kDelta);
+    float4* sRow = reinterpret_cast<float4*>(smem + L::kRowTerms);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 4);
     auto bar = [&](int i) { return sbase + L::kBars + 8u * uint32_t(i); };
@@ -634,13 +634,13 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(kDkvBarSFull + s), 2);
-            mbar_init(bar(kDkvBarPFull + s), 128);
+            mbar_init(bar(kDkvBarPFull + s), 256);
         }
         mbar_init(bar(kDkvBarFinal), 2);
         for (int s = 0; s < 4; ++s) mbar_init(bar(kDkvBarDrain + s), 1);
         fence_mbar_init();
     }
-    if (warp == 5) {
+    if (warp == 9) {
         tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -658,72 +658,71 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         }
     };
 
-    if (warp < 4) {
+    if (warp < 8) {
         // =========================== P^T, dS^T and the dK / dV epilogue ===========================
-        setmaxnreg_inc<232>();
-        const int r = tid;                                   // key row inside the tile = TMEM lane
-        const uint32_t lane_addr = uint32_t(warp * 32) << 16;
+        setmaxnreg_inc<152>();
+        const int hc = warp >> 2;                            // which 32 query columns of every iteration
+        const int r = tid & 127;                             // key row inside the tile = TMEM lane
+        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
         for (int it = 0; it < n_it; ++it) {
             const int st = it % L::kStages, buf = it & 1;
             const int qoff = (i_first + it) * kKeyTile - k0;  // query of column c sees key row r iff qoff + c >= r
             mbar_wait(bar(kDkvBarQFull + st), (it / L::kStages) & 1, abort_flag, 90);   // LSE / D_t of this stage
             mbar_wait(bar(kDkvBarSFull + buf), (it >> 1) & 1, abort_flag, 91);
             tc_fence_after_sync();
-            const float* lse = sLse + st * kKeyTile;
-            const float* dl = sDelta + st * kKeyTile;
+            const float4* rt = sRow + st * (kKeyTile / 2) + hc * 16;
             const bool masked = qoff < kTileRows - 1;
+            uint32_t s[32], g[32];
+            tmem_ld32(tmem + lane_addr + kColST + buf * 64 + hc * 32, s);
+            tmem_ld32(tmem + lane_addr + kColdPT + buf * 64 + hc * 32, g);
+            tmem_wait_ld();
+            uint32_t pp[16], pd[16];
 #pragma unroll
-            for (int hc = 0; hc < 2; ++hc) {                 // 32 query columns at a time
-                uint32_t s[32], g[32];
-                tmem_ld32(tmem + lane_addr + kColST + buf * 64 + hc * 32, s);
-                tmem_ld32(tmem + lane_addr + kColdPT + buf * 64 + hc * 32, g);
-                tmem_wait_ld();
-                uint32_t pp[16], pd[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int c0 = hc * 32 + 2 * i;
-                    float pa = fast_exp2(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, lse[c0]));
-                    float pb = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, lse[c0 + 1]));
-                    if (masked) {
-                        if (qoff + c0 < r) pa = 0.f;
-                        if (qoff + c0 + 1 < r) pb = 0.f;
-                    }
-                    pp[i] = pack_bf16x2(pa, pb);
-                    pd[i] = pack_bf16x2(pa * (__uint_as_float(g[2 * i]) - dl[c0]), pb * (__uint_as_float(g[2 * i + 1]) - dl[c0 + 1]));
+            for (int i = 0; i < 16; ++i) {
+                const int c0 = hc * 32 + 2 * i;
+                const float4 t = rt[i];                      // {-LSE c0, -LSE c0+1, D c0, D c0+1}, same for all rows
+                float pa = fast_exp2(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, t.x));
+                float pb = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, t.y));
+                if (masked) {
+                    if (qoff + c0 < r) pa = 0.f;
+                    if (qoff + c0 + 1 < r) pb = 0.f;
                 }
-                // P^T overlays S^T, dS^T overlays dP^T (bf16, two per column)
-                tmem_st16(tmem + lane_addr + kColST + buf * 64 + hc * 16, pp);
-                tmem_st16(tmem + lane_addr + kColdPT + buf * 64 + hc * 16, pd);
+                pp[i] = pack_bf16x2(pa, pb);
+                pd[i] = pack_bf16x2(pa * (__uint_as_float(g[2 * i]) - t.z), pb * (__uint_as_float(g[2 * i + 1]) - t.w));
             }
+            // P^T overlays S^T, dS^T overlays dP^T (bf16, two per column).  Each warpgroup writes over
+            // the first 16 of the 32 columns it has just read itself (columns 32 hc .. 32 hc + 15), so
+            // the two never touch each other's scores; the MMA issuers address the two blocks per k-step.
+            tmem_st16(tmem + lane_addr + kColST + buf * 64 + hc * 32, pp);
+            tmem_st16(tmem + lane_addr + kColdPT + buf * 64 + hc * 32, pd);
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(kDkvBarPFull + buf));
         }
         mbar_wait(bar(kDkvBarFinal), 0, abort_flag, 92);
         tc_fence_after_sync();
-#pragma unroll
-        for (int which = 0; which < 2; ++which) {            // 0: dK (scaled), 1: dV
-            const float mul = which == 0 ? p.scale : 1.f;
-            const uint32_t col = which == 0 ? kColdK : kColdV;
-            const int dst_off = which == 0 ? L::kK : L::kV;
+        {                                                    // first warpgroup: dK (scaled); second: dV
+            const float mul = hc == 0 ? p.scale : 1.f;
+            const uint32_t col = hc == 0 ? kColdK : kColdV;
+            const int dst_off = hc == 0 ? L::kK : L::kV;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tmem + lane_addr + col + c * 32, o);
                 tmem_wait_ld();
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
+                for (int g4 = 0; g4 < 4; ++g4) {
                     uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(o[8 * g + 0]) * mul, __uint_as_float(o[8 * g + 1]) * mul);
-                    v.y = pack_bf16x2(__uint_as_float(o[8 * g + 2]) * mul, __uint_as_float(o[8 * g + 3]) * mul);
-                    v.z = pack_bf16x2(__uint_as_float(o[8 * g + 4]) * mul, __uint_as_float(o[8 * g + 5]) * mul);
-                    v.w = pack_bf16x2(__uint_as_float(o[8 * g + 6]) * mul, __uint_as_float(o[8 * g + 7]) * mul);
-                    *reinterpret_cast<uint4*>(smem + dst_off + swz_chunk_offset(r, c * 4 + g)) = v;
+                    v.x = pack_bf16x2(__uint_as_float(o[8 * g4 + 0]) * mul, __uint_as_float(o[8 * g4 + 1]) * mul);
+                    v.y = pack_bf16x2(__uint_as_float(o[8 * g4 + 2]) * mul, __uint_as_float(o[8 * g4 + 3]) * mul);
+                    v.z = pack_bf16x2(__uint_as_float(o[8 * g4 + 4]) * mul, __uint_as_float(o[8 * g4 + 5]) * mul);
+                    v.w = pack_bf16x2(__uint_as_float(o[8 * g4 + 6]) * mul, __uint_as_float(o[8 * g4 + 7]) * mul);
+                    *reinterpret_cast<uint4*>(smem + dst_off + swz_chunk_offset(r, c * 4 + g4)) = v;
                 }
             }
         }
         fence_proxy_async_smem();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (tid == 0) {
 #pragma unroll
             for (int s = 0; s < NSUB; ++s) {
@@ -733,9 +732,9 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tma_store_commit();
             tma_store_wait_all();
         }
-    } else if (warp < 8) {
+    } else if (warp < 12) {
       setmaxnreg_dec<64>();
-      if (warp == 4) {
+      if (warp == 8) {
         // =========================== loader: TMA tiles + per-query LSE, D_t ===========================
         if (lane == 0) {
             tma_prefetch_desc(&mapK);
@@ -755,13 +754,16 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             const int qrow0 = (i_first + it) * kKeyTile;
             if (it >= L::kStages)
                 mbar_wait(bar(kDkvBarQEmpty + st), ((it - L::kStages) / L::kStages) & 1, abort_flag, 100);
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                const int c = lane + 32 * k;
-                const bool valid = qrow0 + c < p.T;
-                // invalid (padding) queries get -LSE = -inf so that their P is exactly 0
-                sLse[st * kKeyTile + c] = valid ? -p.LSE[row_base + qrow0 + c] * kLog2e : -INFINITY;
-                sDelta[st * kKeyTile + c] = valid ? p.delta[row_base + qrow0 + c] : 0.f;
+            {
+                // lane handles the column pair (2 lane, 2 lane + 1); invalid (padding) queries get
+                // -LSE = -inf so that their P is exactly 0
+                const int c = 2 * lane;
+                float4 t;
+                t.x = (qrow0 + c < p.T) ? -p.LSE[row_base + qrow0 + c] * kLog2e : -INFINITY;
+                t.y = (qrow0 + c + 1 < p.T) ? -p.LSE[row_base + qrow0 + c + 1] * kLog2e : -INFINITY;
+                t.z = (qrow0 + c < p.T) ? p.delta[row_base + qrow0 + c] : 0.f;
+                t.w = (qrow0 + c + 1 < p.T) ? p.delta[row_base + qrow0 + c + 1] : 0.f;
+                sRow[st * (kKeyTile / 2) + lane] = t;
             }
             if (lane == 0) {
                 mbar_arrive_expect_tx(bar(kDkvBarQFull + st), 2 * L::kHalfTileBytes);
@@ -776,10 +778,10 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 mbar_arrive(bar(kDkvBarQFull + st));
             }
         }
-      } else if (warp == 5 || warp == 6) {
-        // ============ MMA issuers: S^T = K Q^T (warp 5), dP^T = V dO^T (warp 6) ============
+      } else if (warp == 9 || warp == 10) {
+        // ============ MMA issuers: S^T = K Q^T (warp 9), dP^T = V dO^T (warp 10) ============
         if (lane == 0) {
-            const bool is_s = (warp == 5);
+            const bool is_s = (warp == 9);
             constexpr uint32_t idesc_s = make_idesc_bf16(128, kKeyTile, false, false);
             const uint32_t a_tile = sbase + (is_s ? L::kK : L::kV);
             const uint32_t col = is_s ? kColST : kColdPT;
@@ -803,7 +805,7 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             drain_on_abort(is_s ? 0 : 1);
         }
       } else {
-        // ============ MMA issuer: dV += P^T dO (warp 7) ============
+        // ============ MMA issuer: dV += P^T dO (warp 11) ============
         if (lane == 0) {
             constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
             const uint64_t db0 = desc_mnmajor_sw128(sbase + L::kQdO + L::kHalfTileBytes, 0, L::kHalfSubBytes);
@@ -814,8 +816,8 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 const uint64_t db = db0 + uint64_t((st * 2 * L::kHalfTileBytes) >> 4);
                 umma_ts(tmem + kColdV, tmem + kColST + buf * 64, db, idesc_acc, it > 0);
 #pragma unroll
-                for (int kk = 1; kk < kKeyTile / 16; ++kk)
-                    umma_ts(tmem + kColdV, tmem + kColST + buf * 64 + kk * 8, db + uint64_t(kk * 128), idesc_acc, 1);
+                for (int kk = 1; kk < kKeyTile / 16; ++kk)   // 16 queries per k-step: 8 columns, in block kk / 2
+                    umma_ts(tmem + kColdV, tmem + kColST + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, db + uint64_t(kk * 128), idesc_acc, 1);
                 umma_commit(bar(kDkvBarQEmpty + st));
             }
             umma_commit(bar(kDkvBarFinal));
@@ -824,8 +826,8 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
       }
     } else {
       setmaxnreg_dec<64>();
-      if (warp == 8) {
-        // ============ MMA issuer: dK += dS^T Q (warp 8) ============
+      if (warp == 12) {
+        // ============ MMA issuer: dK += dS^T Q (warp 12) ============
         if (lane == 0) {
             constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
             const uint64_t db0 = desc_mnmajor_sw128(sbase + L::kQdO, 0, L::kHalfSubBytes);
@@ -837,7 +839,7 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 umma_ts(tmem + kColdK, tmem + kColdPT + buf * 64, db, idesc_acc, it > 0);
 #pragma unroll
                 for (int kk = 1; kk < kKeyTile / 16; ++kk)
-                    umma_ts(tmem + kColdK, tmem + kColdPT + buf * 64 + kk * 8, db + uint64_t(kk * 128), idesc_acc, 1);
+                    umma_ts(tmem + kColdK, tmem + kColdPT + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, db + uint64_t(kk * 128), idesc_acc, 1);
                 umma_commit(bar(kDkvBarQEmpty + st));
             }
             umma_commit(bar(kDkvBarFinal));
@@ -853,7 +855,7 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         while (globaltimer_ns() - t0 < 2000000ull) {}
     }
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
 }  // namespace moda

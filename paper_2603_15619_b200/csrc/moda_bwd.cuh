@@ -75,11 +75,11 @@ bwd_delta_kernel(const uint4* __restrict__ O, const uint4* __restrict__ dO, floa
 // =====================================================================================
 // dQ + depth gradients
 // =====================================================================================
-// 512 threads: warps 0-3 form dS and run the epilogue, warps 4-7 do the depth backward, warp 8 is the
-// TMA producer, warp 9 the depth-cache producer, and the three contractions of a tile are issued by
-// three threads on three schedulers (warp 12: S = Q K^T, warp 13: dP = dO V^T, warp 14: dQ += dS K),
-// ordered by mbarriers only.
-constexpr int kBwdDqThreads = 512;
+// 640 threads: warps 0-3 and 4-7 form dS (each warpgroup takes 32 of a tile's 64 key columns) and
+// run the epilogue, warps 8-11 do the depth backward, warp 12 is the TMA producer, warp 13 the
+// depth-cache producer, and the three contractions of a tile are issued by three threads on three
+// schedulers (warp 16: S = Q K^T, warp 17: dP = dO V^T, warp 18: dQ += dS K), ordered by mbarriers only.
+constexpr int kBwdDqThreads = 640;
 constexpr int kKeyTile = 64;     // keys per inner tile of the dQ kernel / queries per inner tile of the dK,dV kernel
 
 template <int D>
@@ -109,7 +109,7 @@ enum DqBar : int {
     kDqBarKVFull = 1,    // +stage (3)
     kDqBarKVEmpty = 4,   // +stage (3): dQ_j complete (K_j, V_j and the score buffer are free)
     kDqBarSFull = 7,     // +buffer (2), count 2: S_j and dP_j complete
-    kDqBarPFull = 9,     // +buffer (2), count 128: dS_j written (and dP_j consumed)
+    kDqBarPFull = 9,     // +buffer (2), count 256: dS_j written (and dP_j consumed)
     kDqBarFinal = 11,
     kDqBarDepth = 12,
     kDqBarDrain = 13,    // +issuer (3): abort path only
@@ -172,7 +172,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(kDqBarSFull + s), 2);
-            mbar_init(bar(kDqBarPFull + s), 128);
+            mbar_init(bar(kDqBarPFull + s), 256);
         }
         mbar_init(bar(kDqBarFinal), 1);
         mbar_init(bar(kDqBarDepth), 128);
@@ -183,7 +183,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         }
         fence_mbar_init();
     }
-    if (warp == 12) {
+    if (warp == 16) {
         tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -201,11 +201,12 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         }
     };
 
-    if (warp < 4) {
+    if (warp < 8) {
         // =========================== P, dS and the dQ epilogue ===========================
-        setmaxnreg_inc<168>();
-        const int r = tid;
-        const uint32_t lane_addr = uint32_t(warp * 32) << 16;
+        setmaxnreg_inc<104>();
+        const int hc = warp >> 2;                    // which 32 key columns of every tile
+        const int r = tid & 127;
+        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
         const bool valid = q0 + r < p.T;
         const size_t row_idx = (size_t(b) * p.H + h) * p.T + q0 + r;
         const float neg_lse2 = valid ? -p.LSE[row_idx] * kLog2e : -INFINITY;   // invalid rows get P = 0
@@ -214,29 +215,26 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             const int buf = j & 1;
             mbar_wait(bar(kDqBarSFull + buf), (j >> 1) & 1, abort_flag, 50);
             tc_fence_after_sync();
-            const int koff = j * kKeyTile - q0;      // key of column c is visible to row r iff koff + c <= r
-            const bool masked = koff + kKeyTile - 1 > 0;
+            const int koff = j * kKeyTile + hc * 32 - q0;    // key of column c is visible to row r iff koff + c <= r
+            const bool masked = koff + 31 > 0;
+            uint32_t sv[32], gv[32];
+            tmem_ld32(tmem + lane_addr + kColS + buf * 64 + hc * 32, sv);
+            tmem_ld32(tmem + lane_addr + kColdP + buf * 64 + hc * 32, gv);
+            tmem_wait_ld();
+            uint32_t pk[16];
 #pragma unroll
-            for (int hc = 0; hc < 2; ++hc) {         // 32 key columns at a time
-                uint32_t sv[32], gv[32];
-                tmem_ld32(tmem + lane_addr + kColS + buf * 64 + hc * 32, sv);
-                tmem_ld32(tmem + lane_addr + kColdP + buf * 64 + hc * 32, gv);
-                tmem_wait_ld();
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float pa = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), p.scale_log2, neg_lse2));
-                    float pb = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), p.scale_log2, neg_lse2));
-                    if (masked) {
-                        if (koff + hc * 32 + 2 * i > r) pa = 0.f;
-                        if (koff + hc * 32 + 2 * i + 1 > r) pb = 0.f;
-                    }
-                    pk[i] = pack_bf16x2(pa * (__uint_as_float(gv[2 * i]) - delta), pb * (__uint_as_float(gv[2 * i + 1]) - delta));
+            for (int i = 0; i < 16; ++i) {
+                float pa = fast_exp2(fmaf(__uint_as_float(sv[2 * i]), p.scale_log2, neg_lse2));
+                float pb = fast_exp2(fmaf(__uint_as_float(sv[2 * i + 1]), p.scale_log2, neg_lse2));
+                if (masked) {
+                    if (koff + 2 * i > r) pa = 0.f;
+                    if (koff + 2 * i + 1 > r) pb = 0.f;
                 }
-                // dS_j (bf16, two per column) overlays the first 32 columns of S_j; the block just
-                // written (columns 16 hc .. 16 hc + 15) was read in this or the previous half.
-                tmem_st16(tmem + lane_addr + kColS + buf * 64 + hc * 16, pk);
+                pk[i] = pack_bf16x2(pa * (__uint_as_float(gv[2 * i]) - delta), pb * (__uint_as_float(gv[2 * i + 1]) - delta));
             }
+            // dS_j (bf16, two per column) overlays S_j: each warpgroup writes over the first 16 of the
+            // 32 columns it has just read itself, so the two never touch each other's scores.
+            tmem_st16(tmem + lane_addr + kColS + buf * 64 + hc * 32, pk);
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(kDqBarPFull + buf));
@@ -247,8 +245,10 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             mbar_wait(bar(kDqBarDepth), 0, abort_flag, 52);
             tc_fence_after_sync();
         }
+        // first warpgroup converts the first half of the feature columns, the second the rest
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
+        for (int cc = 0; cc < D / 64; ++cc) {
+            const int c = hc * (D / 64) + cc;
             uint32_t o[32];
             tmem_ld32(tmem + lane_addr + kColdQ + c * 32, o);
             tmem_wait_ld();
@@ -273,18 +273,18 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             }
         }
         fence_proxy_async_smem();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (tid == 0) {
 #pragma unroll
             for (int s = 0; s < NSUB; ++s) tma_store_4d(&mapdQ, sbase + L::kQ + s * L::kSubBytes, s * 64, h, q0, b);
             tma_store_commit();
             tma_store_wait_all();
         }
-    } else if (warp < 8) {
+    } else if (warp < 12) {
         // =========================== depth backward (row-local) ===========================
-        setmaxnreg_inc<216>();
+        setmaxnreg_inc<176>();
         if (p.l > 0) {
-            const int r = tid - 128;
+            const int r = tid - 256;
             const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
             const bool valid = q0 + r < p.T;
             const size_t row_idx = (size_t(b) * p.H + h) * p.T + q0 + r;
@@ -428,9 +428,9 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             tc_fence_before_sync();
             mbar_arrive(bar(kDqBarDepth));
         }
-    } else if (warp < 12) {
-        setmaxnreg_dec<64>();
-        if (warp == 8) {
+    } else if (warp < 16) {
+        setmaxnreg_dec<48>();
+        if (warp == 12) {
             // =========================== TMA producer ===========================
             if (lane == 0) {
                 tma_prefetch_desc(&mapQ);
@@ -457,7 +457,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     }
                 }
             }
-        } else if (warp == 9) {
+        } else if (warp == 13) {
             // =========================== depth-cache producer ===========================
             // 16 KiB units in the order the depth warps consume them: keys (pass A), values (pass B),
             // keys again (pass C).
@@ -484,11 +484,11 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             }
         }
     } else {
-        setmaxnreg_dec<64>();
-        if (warp == 12 || warp == 13) {
-            // ============ MMA issuers: S = Q K^T (warp 12), dP = dO V^T (warp 13) ============
-            if (lane == 0) {
-                const bool is_s = (warp == 12);
+        setmaxnreg_dec<48>();
+        if (warp == 16 || warp == 17) {
+            // ============ MMA issuers: S = Q K^T (warp 16), dP = dO V^T (warp 17) ============
+            {   // whole warp: operands are warp-uniform, one elected lane issues
+                const bool is_s = (warp == 16);
                 constexpr uint32_t idesc_s = make_idesc_bf16(128, kKeyTile, false, false);
                 const uint32_t a_tile = sbase + (is_s ? L::kQ : L::kdO);
                 const uint32_t col = is_s ? kColS : kColdP;
@@ -515,9 +515,9 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 }
                 drain_on_abort(is_s ? 0 : 1);
             }
-        } else if (warp == 14) {
-            // ============ MMA issuer: dQ += dS K (warp 14) ============
-            if (lane == 0) {
+        } else if (warp == 18) {
+            // ============ MMA issuer: dQ += dS K (warp 18) ============
+            {   // whole warp: operands are warp-uniform, one elected lane issues
                 constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, false, true);
                 const uint64_t db0 = desc_mnmajor_sw128(sbase + L::kKV, 0, L::kHalfSubBytes);
                 for (int j = 0; j < n_kv; ++j) {
@@ -527,8 +527,8 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     const uint64_t db = db0 + uint64_t((st * 2 * L::kHalfTileBytes) >> 4);
                     umma_ts(tmem + kColdQ, tmem + kColS + buf * 64, db, idesc_dq, j > 0);
 #pragma unroll
-                    for (int kk = 1; kk < kKeyTile / 16; ++kk)
-                        umma_ts(tmem + kColdQ, tmem + kColS + buf * 64 + kk * 8, db + uint64_t(kk * 128), idesc_dq, 1);
+                    for (int kk = 1; kk < kKeyTile / 16; ++kk)   // 16 keys per k-step: 8 columns, in block kk / 2
+                        umma_ts(tmem + kColdQ, tmem + kColS + buf * 64 + (kk >> 1) * 32 + (kk & 1) * 8, db + uint64_t(kk * 128), idesc_dq, 1);
                     umma_commit(bar(kDqBarKVEmpty + st));
                 }
                 umma_commit(bar(kDqBarFinal));
@@ -544,7 +544,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         while (globaltimer_ns() - t0 < 2000000ull) {}
     }
     __syncthreads();
-    if (warp == 12) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 16) tmem_dealloc(tmem, kTmemCols);
 }
 
 // =====================================================================================
@@ -780,7 +780,7 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         }
       } else if (warp == 9 || warp == 10) {
         // ============ MMA issuers: S^T = K Q^T (warp 9), dP^T = V dO^T (warp 10) ============
-        if (lane == 0) {
+        {   // whole warp: operands are warp-uniform, one elected lane issues
             const bool is_s = (warp == 9);
             constexpr uint32_t idesc_s = make_idesc_bf16(128, kKeyTile, false, false);
             const uint32_t a_tile = sbase + (is_s ? L::kK : L::kV);
@@ -806,7 +806,7 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         }
       } else {
         // ============ MMA issuer: dV += P^T dO (warp 11) ============
-        if (lane == 0) {
+        {   // whole warp: operands are warp-uniform, one elected lane issues
             constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
             const uint64_t db0 = desc_mnmajor_sw128(sbase + L::kQdO + L::kHalfTileBytes, 0, L::kHalfSubBytes);
             for (int it = 0; it < n_it; ++it) {
@@ -828,7 +828,7 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
       setmaxnreg_dec<64>();
       if (warp == 12) {
         // ============ MMA issuer: dK += dS^T Q (warp 12) ============
-        if (lane == 0) {
+        {   // whole warp: operands are warp-uniform, one elected lane issues
             constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
             const uint64_t db0 = desc_mnmajor_sw128(sbase + L::kQdO, 0, L::kHalfSubBytes);
             for (int it = 0; it < n_it; ++it) {

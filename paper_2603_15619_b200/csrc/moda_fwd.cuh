@@ -177,11 +177,11 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             }
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                mx0 = fmaxf(mx0, __uint_as_float(s0[i]));
-                mx1 = fmaxf(mx1, __uint_as_float(s1[i]));
-                mx2 = fmaxf(mx2, __uint_as_float(s2[i]));
-                mx3 = fmaxf(mx3, __uint_as_float(s3[i]));
+            for (int i = 0; i < 32; i += 2) {            // 3-input max: one instruction per two scores
+                mx0 = max3(mx0, __uint_as_float(s0[i]), __uint_as_float(s0[i + 1]));
+                mx1 = max3(mx1, __uint_as_float(s1[i]), __uint_as_float(s1[i + 1]));
+                mx2 = max3(mx2, __uint_as_float(s2[i]), __uint_as_float(s2[i + 1]));
+                mx3 = max3(mx3, __uint_as_float(s3[i]), __uint_as_float(s3[i + 1]));
             }
             const float m_new = fmaxf(m_ref, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
             if (j == 0) {
@@ -414,7 +414,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         }
       } else if (warp == 9) {
         // =========================== MMA issuer: S_j = Q K_j^T ===========================
-        if (lane == 0) {
+        {   // whole warp: operands are warp-uniform, one elected lane issues
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
             // every descriptor is built once; inside the loop a descriptor is one 64-bit add (the
             // start-address field counts 16-byte units and stays inside its 14 bits below 256 KiB)
@@ -445,7 +445,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         }
       } else if (warp == 11) {
         // =========================== MMA issuer: O += P_j V_j ===========================
-        if (lane == 0) {
+        {   // whole warp: operands are warp-uniform, one elected lane issues
             constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
             const uint64_t dv0 = desc_mnmajor_sw128(sbase + L::kV, 0, L::kSubBytes);
             for (int j = 0; j < n_kv; ++j) {

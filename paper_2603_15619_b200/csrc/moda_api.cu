@@ -9,6 +9,7 @@
 #include "moda_bwd.cuh"
 #include "moda_cache.cuh"
 #include "moda_fwd.cuh"
+#include "moda_fwd_wide.cuh"
 #include "sm100_ptx.cuh"
 
 namespace {
@@ -88,9 +89,14 @@ bool set_smem_limit(Kernel k, int bytes) {
     return cuda_ok(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
 }
 
+// d = 128 runs moda_fwd_kernel (one softmax warpgroup: the tensor pipe and the MMA issue rate set the
+// pace); d = 64 runs moda_fwd2_kernel (two softmax warpgroups, three score buffers: the exponentials do).
 template <int D>
 int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int H, int l,
                float scale, void* O, float* LSE, cudaStream_t stream) {
+    constexpr bool kWide = (D == 64);
+    constexpr int kSmem = kWide ? Fwd2Smem<D>::kDynamic : FwdSmem<D>::kDynamic;
+    constexpr int kThreads = kWide ? kFwd2Threads : kFwdThreads;
     CUtensorMap mQ, mK, mV, mO;
     if (!make_bthd_map(&mQ, Q, B, T, H, D) || !make_bthd_map(&mK, K, B, T, H, D) ||
         !make_bthd_map(&mV, V, B, T, H, D) || !make_bthd_map(&mO, O, B, T, H, D))
@@ -99,7 +105,8 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
     if (configured_dev != dev) {
-        if (!set_smem_limit(moda_fwd_kernel<D>, FwdSmem<D>::kDynamic)) return MODA_ERR_CUDA;
+        const bool ok = kWide ? set_smem_limit(moda_fwd2_kernel<D>, kSmem) : set_smem_limit(moda_fwd_kernel<D>, kSmem);
+        if (!ok) return MODA_ERR_CUDA;
         configured_dev = dev;
     }
     FwdParams p;
@@ -109,7 +116,8 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.B = B; p.T = T; p.H = H; p.l = l;
     p.scale_log2 = scale * kLog2e;
     const unsigned grid = unsigned(B) * H * num_tiles(T);
-    moda_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kDynamic, stream>>>(mQ, mK, mV, mO, p);
+    if (kWide) moda_fwd2_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
+    else moda_fwd_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 

@@ -82,6 +82,12 @@ bwd_delta_kernel(const uint4* __restrict__ O, const uint4* __restrict__ dO, floa
 constexpr int kBwdDqThreads = 640;
 constexpr int kKeyTile = 64;     // keys per inner tile of the dQ kernel / queries per inner tile of the dK,dV kernel
 
+// The depth backward walks the slots in groups of kDepthGroup: keys (scores), values, keys again
+// (dQ share, dKd).  The second visit of a group's keys comes a few hundred KiB per SM after the
+// first, so it is served by L2 and the depth cache crosses HBM once; the per-slot row terms only
+// need kDepthGroup entries of shared memory.
+constexpr int kDepthGroup = 4;
+
 template <int D>
 struct DqSmem {
     static constexpr int kTileBytes = kTileRows * D * 2;             // 128 x D
@@ -92,11 +98,11 @@ struct DqSmem {
     static constexpr int kQ = 0;
     static constexpr int kdO = kQ + kTileBytes;
     static constexpr int kKV = kdO + kTileBytes;                     // stages of [K_j | V_j]
-    static constexpr int kU = kKV + kStages * 2 * kHalfTileBytes;    // [32][128] fp32: u_i, then R_i
-    static constexpr int kDr = kU + 32 * kTileRows * 4;              // [32][128] fp32: <dO,Vd_i>, then dU_i
-    static constexpr int kRing = kDr + 32 * kTileRows * 4;           // depth units: 8 chunks x 128 rows x 16 B
+    static constexpr int kU = kKV + kStages * 2 * kHalfTileBytes;    // [kDepthGroup][128] fp32: u_i, then R_i
+    static constexpr int kDr = kU + kDepthGroup * kTileRows * 4;     // [kDepthGroup][128] fp32: <dO,Vd_i>, then dU_i
+    static constexpr int kRing = kDr + kDepthGroup * kTileRows * 4;  // depth units: 8 chunks x 128 rows x 16 B
     static constexpr int kUnitBytes = 8 * kTileRows * 16;
-    static constexpr int kRingStages = (D == 128) ? 2 : 6;
+    static constexpr int kRingStages = (D == 128) ? 3 : 6;
     static constexpr int kBars = kRing + kRingStages * kUnitBytes;
     static constexpr int kNumBars = 32;
     static constexpr int kMisc = kBars + kNumBars * 8;
@@ -333,95 +339,111 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 return (a0 + a1) + (a2 + a3);
             };
 
-            // ---- pass A: u_i = <q, kd_i> ----
 #pragma unroll 1
-            for (int half = 0; half < NSUB; ++half) {
-                float q[64];
-                load_row_f32(q, L::kQ, half);
+            for (int g0 = 0; g0 < p.l; g0 += kDepthGroup) {
+                const int gl = min(kDepthGroup, p.l - g0);
+                // ---- pass A: u_i = <q, kd_i> ----
 #pragma unroll 1
-                for (int i = 0; i < p.l; ++i) {
-                    uint4 cur[8];
-                    take_unit(cur);
-                    const float part = dot64(q, cur);
-                    if (half == 0) sU[i * kTileRows + r] = part;
-                    else sU[i * kTileRows + r] += part;
-                }
-            }
-            // R_i = exp(u_i - LSE): the forward's LSE already covers sequence and depth keys.
-            for (int i = 0; i < p.l; ++i)
-                sU[i * kTileRows + r] = fast_exp2(fmaf(sU[i * kTileRows + r], p.scale_log2, neg_lse2));
-
-            // ---- pass B: <dO, vd_i>, and dVd_i = R_i dO ----
+                for (int half = 0; half < NSUB; ++half) {
+                    float q[64];
+                    load_row_f32(q, L::kQ, half);
 #pragma unroll 1
-            for (int half = 0; half < NSUB; ++half) {
-                float g[64];
-                load_row_f32(g, L::kdO, half);
-#pragma unroll 1
-                for (int i = 0; i < p.l; ++i) {
-                    uint4 cur[8];
-                    take_unit(cur);
-                    const float part = dot64(g, cur);
-                    if (half == 0) sDr[i * kTileRows + r] = part;
-                    else sDr[i * kTileRows + r] += part;
-                    const float w = sU[i * kTileRows + r];
-                    uint4* dst = gV + size_t(i) * slot_stride + (half * 8) * kTileRows;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        uint4 o;
-                        o.x = pack_bf16x2(w * g[8 * c + 0], w * g[8 * c + 1]);
-                        o.y = pack_bf16x2(w * g[8 * c + 2], w * g[8 * c + 3]);
-                        o.z = pack_bf16x2(w * g[8 * c + 4], w * g[8 * c + 5]);
-                        o.w = pack_bf16x2(w * g[8 * c + 6], w * g[8 * c + 7]);
-                        dst[c * kTileRows] = o;
+                    for (int ii = 0; ii < gl; ++ii) {
+                        uint4 cur[8];
+                        take_unit(cur);
+                        const float part = dot64(q, cur);
+                        if (half == 0) sU[ii * kTileRows + r] = part;
+                        else sU[ii * kTileRows + r] += part;
                     }
                 }
-            }
-            // dU_i = R_i (<dO, vd_i> - D)
-            for (int i = 0; i < p.l; ++i)
-                sDr[i * kTileRows + r] = sU[i * kTileRows + r] * (sDr[i * kTileRows + r] - delta);
+                // R_i = exp(u_i - LSE): the forward's LSE already covers sequence and depth keys.
+                for (int ii = 0; ii < gl; ++ii)
+                    sU[ii * kTileRows + r] = fast_exp2(fmaf(sU[ii * kTileRows + r], p.scale_log2, neg_lse2));
 
-            // ---- pass C: dQ share sum_i dU_i kd_i (parked in TMEM), dKd_i = scale dU_i q ----
+                // ---- pass B: <dO, vd_i>, and dVd_i = R_i dO ----
 #pragma unroll 1
-            for (int half = 0; half < NSUB; ++half) {
-                uint4 qp[8];                               // q kept packed: only multiplied, never summed
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    qp[c] = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, half * 8 + c));
-                float acc[64];
-#pragma unroll
-                for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+                for (int half = 0; half < NSUB; ++half) {
+                    float g[64];
+                    load_row_f32(g, L::kdO, half);
 #pragma unroll 1
-                for (int i = 0; i < p.l; ++i) {
-                    uint4 cur[8];
-                    take_unit(cur);
-                    const float du = sDr[i * kTileRows + r];
-                    const float sdu = du * p.scale;
-                    const uint32_t sdu2 = pack_bf16x2(sdu, sdu);
-                    uint4* dst = gK + size_t(i) * slot_stride + (half * 8) * kTileRows;
+                    for (int ii = 0; ii < gl; ++ii) {
+                        uint4 cur[8];
+                        take_unit(cur);
+                        const float part = dot64(g, cur);
+                        if (half == 0) sDr[ii * kTileRows + r] = part;
+                        else sDr[ii * kTileRows + r] += part;
+                        const float w = sU[ii * kTileRows + r];
+                        uint4* dst = gV + size_t(g0 + ii) * slot_stride + (half * 8) * kTileRows;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        acc[8 * c + 0] = fmaf(du, bf16_lo_to_f32(cur[c].x), acc[8 * c + 0]);
-                        acc[8 * c + 1] = fmaf(du, bf16_hi_to_f32(cur[c].x), acc[8 * c + 1]);
-                        acc[8 * c + 2] = fmaf(du, bf16_lo_to_f32(cur[c].y), acc[8 * c + 2]);
-                        acc[8 * c + 3] = fmaf(du, bf16_hi_to_f32(cur[c].y), acc[8 * c + 3]);
-                        acc[8 * c + 4] = fmaf(du, bf16_lo_to_f32(cur[c].z), acc[8 * c + 4]);
-                        acc[8 * c + 5] = fmaf(du, bf16_hi_to_f32(cur[c].z), acc[8 * c + 5]);
-                        acc[8 * c + 6] = fmaf(du, bf16_lo_to_f32(cur[c].w), acc[8 * c + 6]);
-                        acc[8 * c + 7] = fmaf(du, bf16_hi_to_f32(cur[c].w), acc[8 * c + 7]);
-                        uint4 o;
-                        o.x = mul_bf16x2(qp[c].x, sdu2);
-                        o.y = mul_bf16x2(qp[c].y, sdu2);
-                        o.z = mul_bf16x2(qp[c].z, sdu2);
-                        o.w = mul_bf16x2(qp[c].w, sdu2);
-                        dst[c * kTileRows] = o;
+                        for (int c = 0; c < 8; ++c) {
+                            uint4 o;
+                            o.x = pack_bf16x2(w * g[8 * c + 0], w * g[8 * c + 1]);
+                            o.y = pack_bf16x2(w * g[8 * c + 2], w * g[8 * c + 3]);
+                            o.z = pack_bf16x2(w * g[8 * c + 4], w * g[8 * c + 5]);
+                            o.w = pack_bf16x2(w * g[8 * c + 6], w * g[8 * c + 7]);
+                            dst[c * kTileRows] = o;
+                        }
                     }
                 }
+                // dU_i = R_i (<dO, vd_i> - D)
+                for (int ii = 0; ii < gl; ++ii)
+                    sDr[ii * kTileRows + r] = sU[ii * kTileRows + r] * (sDr[ii * kTileRows + r] - delta);
+
+                // ---- pass C: dQ share sum_i dU_i kd_i (accumulated in TMEM across groups), dKd_i = scale dU_i q ----
+#pragma unroll 1
+                for (int half = 0; half < NSUB; ++half) {
+                    uint4 qp[8];                           // q kept packed: only multiplied, never summed
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t o[32];
+                    for (int c = 0; c < 8; ++c)
+                        qp[c] = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, half * 8 + c));
+                    float acc[64];
+                    if (g0 == 0) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(acc[32 * c + i]);
-                    tmem_st32(tmem + lane_addr + kColdQd + half * 64 + c * 32, o);
+                        for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tmem + lane_addr + kColdQd + half * 64 + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) acc[32 * c + i] = __uint_as_float(o[i]);
+                        }
+                    }
+#pragma unroll 1
+                    for (int ii = 0; ii < gl; ++ii) {
+                        uint4 cur[8];
+                        take_unit(cur);
+                        const float du = sDr[ii * kTileRows + r];
+                        const float sdu = du * p.scale;
+                        const uint32_t sdu2 = pack_bf16x2(sdu, sdu);
+                        uint4* dst = gK + size_t(g0 + ii) * slot_stride + (half * 8) * kTileRows;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            acc[8 * c + 0] = fmaf(du, bf16_lo_to_f32(cur[c].x), acc[8 * c + 0]);
+                            acc[8 * c + 1] = fmaf(du, bf16_hi_to_f32(cur[c].x), acc[8 * c + 1]);
+                            acc[8 * c + 2] = fmaf(du, bf16_lo_to_f32(cur[c].y), acc[8 * c + 2]);
+                            acc[8 * c + 3] = fmaf(du, bf16_hi_to_f32(cur[c].y), acc[8 * c + 3]);
+                            acc[8 * c + 4] = fmaf(du, bf16_lo_to_f32(cur[c].z), acc[8 * c + 4]);
+                            acc[8 * c + 5] = fmaf(du, bf16_hi_to_f32(cur[c].z), acc[8 * c + 5]);
+                            acc[8 * c + 6] = fmaf(du, bf16_lo_to_f32(cur[c].w), acc[8 * c + 6]);
+                            acc[8 * c + 7] = fmaf(du, bf16_hi_to_f32(cur[c].w), acc[8 * c + 7]);
+                            uint4 o;
+                            o.x = mul_bf16x2(qp[c].x, sdu2);
+                            o.y = mul_bf16x2(qp[c].y, sdu2);
+                            o.z = mul_bf16x2(qp[c].z, sdu2);
+                            o.w = mul_bf16x2(qp[c].w, sdu2);
+                            dst[c * kTileRows] = o;
+                        }
+                    }
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t o[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(acc[32 * c + i]);
+                        tmem_st32(tmem + lane_addr + kColdQd + half * 64 + c * 32, o);
+                    }
+                    tmem_wait_st();                        // the next group reads these columns back
                 }
             }
             tmem_wait_st();
@@ -459,27 +481,33 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             }
         } else if (warp == 13) {
             // =========================== depth-cache producer ===========================
-            // 16 KiB units in the order the depth warps consume them: keys (pass A), values (pass B),
-            // keys again (pass C).
+            // 16 KiB units in the order the depth warps consume them, group by group: keys (pass A),
+            // values (pass B), keys again (pass C).
             if (lane == 0 && p.l > 0) {
                 const uint64_t policy = l2_policy_evict_first();
                 const size_t slot_bytes = cache_slot_elems(p.B, p.T, p.H, D) * 2;
                 const size_t kv_bytes = size_t(kTileRows) * D * 2;
                 const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
                                      (((size_t(b) * p.H + h) * nq + qt) * 2) * kv_bytes;
+                // keys of a group are fetched twice; the first fetch is kept in L2 (evict_last), the second
+                // fetch and the values are not needed again (evict_first)
+                const uint64_t keep = l2_policy_evict_last();
                 int unit = 0;
-                for (int pass = 0; pass < 3; ++pass) {
-                    const int kv = (pass == 1) ? 1 : 0;
-                    for (int half = 0; half < NSUB; ++half)
-                        for (int i = 0; i < p.l; ++i, ++unit) {
-                            const int st = unit % L::kRingStages;
-                            if (unit >= L::kRingStages)
-                                mbar_wait(bar(kDqBarDEmpty + st), ((unit / L::kRingStages) - 1) & 1, abort_flag, 71);
-                            mbar_arrive_expect_tx(bar(kDqBarDFull + st), L::kUnitBytes);
-                            bulk_load(sbase + L::kRing + st * L::kUnitBytes,
-                                      blk + size_t(i) * slot_bytes + size_t(kv) * kv_bytes + size_t(half) * L::kUnitBytes,
-                                      L::kUnitBytes, bar(kDqBarDFull + st), policy);
-                        }
+                for (int g0 = 0; g0 < p.l; g0 += kDepthGroup) {
+                    const int gl = min(kDepthGroup, p.l - g0);
+                    for (int pass = 0; pass < 3; ++pass) {
+                        const int kv = (pass == 1) ? 1 : 0;
+                        for (int half = 0; half < NSUB; ++half)
+                            for (int ii = 0; ii < gl; ++ii, ++unit) {
+                                const int st = unit % L::kRingStages;
+                                if (unit >= L::kRingStages)
+                                    mbar_wait(bar(kDqBarDEmpty + st), ((unit / L::kRingStages) - 1) & 1, abort_flag, 71);
+                                mbar_arrive_expect_tx(bar(kDqBarDFull + st), L::kUnitBytes);
+                                bulk_load(sbase + L::kRing + st * L::kUnitBytes,
+                                          blk + size_t(g0 + ii) * slot_bytes + size_t(kv) * kv_bytes + size_t(half) * L::kUnitBytes,
+                                          L::kUnitBytes, bar(kDqBarDFull + st), pass == 0 ? keep : policy);
+                            }
+                    }
                 }
             }
         }

@@ -21,6 +21,7 @@ __device__ int g_moda_status = 0;
 enum : int {
     kStatusOk = 0,
     kStatusWaitTimeout = 1,   // | (site << 8)
+    kStatusSmemLayout = 2,    // the dynamic shared-memory segment is too small for the kernel's plan
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -150,6 +151,11 @@ __device__ __forceinline__ void tma_store_wait_all() {
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t pol;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
     return pol;
 }
 __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar, uint64_t policy) {

@@ -121,6 +121,13 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 
+// Which dQ kernel at d = 128: two K/V stages and a five-unit depth ring when streaming the depth cache
+// outweighs the sequence contractions (measured cross-over near l d / T = 0.6), otherwise three K/V
+// stages and a three-unit ring.  At d = 64 three K/V stages and eight units fit together.
+inline bool dq_depth_heavy(int T, int l, int d) {
+    return d == 128 && l > 0 && 3ll * l * d >= 2ll * T;
+}
+
 template <int D>
 int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
     const int B = a.B, T = a.T, H = a.H;
@@ -136,7 +143,8 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
     if (configured_dev != dev) {
-        if (!set_smem_limit(moda_bwd_dq_kernel<D>, DqSmem<D>::kDynamic) ||
+        if (!set_smem_limit(moda_bwd_dq_kernel<D, 3>, DqSmem<D, 3>::kDynamic) ||
+            (D == 128 && !set_smem_limit(moda_bwd_dq_kernel<128, 2>, DqSmem<128, 2>::kDynamic)) ||
             !set_smem_limit(moda_bwd_dkdv_kernel<D>, DkvSmem<D>::kDynamic))
             return MODA_ERR_CUDA;
         configured_dev = dev;
@@ -157,7 +165,10 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
         p.LSE = a.LSE; p.delta = delta;
         p.B = B; p.T = T; p.H = H; p.l = a.l;
         p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
-        moda_bwd_dq_kernel<D><<<grid, kBwdDqThreads, DqSmem<D>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
+        if (dq_depth_heavy(T, a.l, D))
+            moda_bwd_dq_kernel<128, 2><<<grid, kBwdDqThreads, DqSmem<128, 2>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
+        else
+            moda_bwd_dq_kernel<D, 3><<<grid, kBwdDqThreads, DqSmem<D, 3>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     }
     if (stages & 4) {

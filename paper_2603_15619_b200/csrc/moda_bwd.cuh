@@ -88,13 +88,16 @@ constexpr int kKeyTile = 64;     // keys per inner tile of the dQ kernel / queri
 // need kDepthGroup entries of shared memory.
 constexpr int kDepthGroup = 4;
 
-template <int D>
+// KVS = stages of the [K_j | V_j] ring.  Three keep the tensor pipe fed on long sequences; two leave
+// room for a deeper depth ring (more HBM reads in flight per SM), which is what bounds shapes whose
+// depth cache outweighs the sequence work (the host picks, see launch_bwd).
+template <int D, int KVS>
 struct DqSmem {
     static constexpr int kTileBytes = kTileRows * D * 2;             // 128 x D
     static constexpr int kSubBytes = kTileRows * 128;                // 128 x 64 sub-tile
     static constexpr int kHalfTileBytes = kKeyTile * D * 2;          // 64 x D
     static constexpr int kHalfSubBytes = kKeyTile * 128;             // 64 x 64 sub-tile
-    static constexpr int kStages = 3;
+    static constexpr int kStages = KVS;
     static constexpr int kQ = 0;
     static constexpr int kdO = kQ + kTileBytes;
     static constexpr int kKV = kdO + kTileBytes;                     // stages of [K_j | V_j]
@@ -102,12 +105,15 @@ struct DqSmem {
     static constexpr int kDr = kU + kDepthGroup * kTileRows * 4;     // [kDepthGroup][128] fp32: <dO,Vd_i>, then dU_i
     static constexpr int kRing = kDr + kDepthGroup * kTileRows * 4;  // depth units: 8 chunks x 128 rows x 16 B
     static constexpr int kUnitBytes = 8 * kTileRows * 16;
-    static constexpr int kRingStages = (D == 128) ? 3 : 6;
-    static constexpr int kBars = kRing + kRingStages * kUnitBytes;
     static constexpr int kNumBars = 32;
+    static constexpr int kSmemLimit = 232448;                        // 227 KiB per CTA on sm_100
+    static constexpr int kRingFit = (kSmemLimit - 1024 - kRing - kNumBars * 8 - 16) / kUnitBytes;
+    static constexpr int kRingStages = kRingFit < 8 ? kRingFit : 8;  // every unit that fits, at most 8
+    static constexpr int kBars = kRing + kRingStages * kUnitBytes;
     static constexpr int kMisc = kBars + kNumBars * 8;
     static constexpr int kTotal = kMisc + 16;
     static constexpr int kDynamic = kTotal + 1024;
+    static_assert(kRingStages >= 3, "depth ring too shallow");
 };
 
 enum DqBar : int {
@@ -119,8 +125,8 @@ enum DqBar : int {
     kDqBarFinal = 11,
     kDqBarDepth = 12,
     kDqBarDrain = 13,    // +issuer (3): abort path only
-    kDqBarDFull = 16,    // +ring stage (<= 6)
-    kDqBarDEmpty = 22,   // +ring stage (<= 6)
+    kDqBarDFull = 16,    // +ring stage (<= 8)
+    kDqBarDEmpty = 24,   // +ring stage (<= 8)
 };
 
 struct DqParams {
@@ -139,12 +145,12 @@ __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
     return r;
 }
 
-template <int D>
+template <int D, int KVS>
 __global__ void __launch_bounds__(kBwdDqThreads, 1)
 moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
                    const __grid_constant__ CUtensorMap mapK64, const __grid_constant__ CUtensorMap mapV64,
                    const __grid_constant__ CUtensorMap mapdQ, const DqParams p) {
-    using L = DqSmem<D>;
+    using L = DqSmem<D, KVS>;
     constexpr int NSUB = D / 64;
     constexpr int CH = D / 8;
     constexpr uint32_t kTmemCols = 512;
@@ -310,6 +316,9 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 const uint8_t* src = smem + L::kRing + st * L::kUnitBytes + r * 16;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) dst[c] = *reinterpret_cast<const uint4*>(src + c * (kTileRows * 16));
+                // The stage is refilled by the async proxy (bulk copy) while these loads went through the
+                // generic proxy: the proxy fence orders them before the refill that this arrival allows.
+                fence_proxy_async_smem();
                 mbar_arrive(bar(kDqBarDEmpty + st));
                 ++unit;
             };

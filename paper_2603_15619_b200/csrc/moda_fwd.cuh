@@ -302,6 +302,9 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 const uint8_t* src = smem + L::kRing + st * L::kUnitBytes + r * 16;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) dst[c] = *reinterpret_cast<const uint4*>(src + c * (kTileRows * 16));
+                // The stage is refilled by the async proxy (bulk copy) while these loads went through the
+                // generic proxy: the proxy fence orders them before the refill that this arrival allows.
+                fence_proxy_async_smem();
                 mbar_arrive(bar(kBarDEmpty + st));
                 ++unit;
             };

@@ -40,7 +40,10 @@
  * Pins (see tests/test_oracle_pins.py): masked library attention over the
  * flattened key set, l = 0 against library causal attention, the two-softmax
  * decomposition identity, closed forms, invariances, finite differences and
- * library autograd, gradient sum identities.
+ * library autograd, gradient sum identities.  The grouped-query functions at the end of
+ * the file have their own pins (tests/test_oracle_gqa_pins.py): masked library attention
+ * with the group-aware masks plus library autograd, the head-repetition identity, the
+ * paper's base-time example, finite differences.
  */
 #include <math.h>
 #include <stddef.h>
@@ -373,4 +376,136 @@ int moda_oracle_bwd_rows(const double *Q, const double *K, const double *V,
     }
     free(need); free(lse_tab); free(del_tab);
     return failed ? -1 : 0;
+}
+
+/*
+ * Grouped-query form (paper Sec. 3, "Group-aware depth KV calculation", and the Preparation
+ * paragraph of the implementation section): Hq query heads share Hk = Hq / G key/value heads.
+ * With the query rows of one KV head flattened as i_q = t * G + g, the base time of a row is
+ * floor(i_q / G) = t; it sees sequence keys i_k <= base time and the depth keys stored at its
+ * base time.  In the [B][T][H][d] layout used here that is: query head hq uses KV head
+ * hk = hq / G (the G heads of a group are adjacent), for K, V and for the depth K, V alike.
+ *
+ *   Q, O, dO, dQ : [B][T][Hq][d]      K, V, dK, dV : [B][T][Hk][d]
+ *   Kd, Vd, dKd, dVd : [l][B][T][Hk][d]      LSE : [B][Hq][T]
+ *
+ * Gradients of the shared tensors are the sums over the G query heads of a group.  Written
+ * out from the definition on its own (it does not call the G = 1 functions above, which stay
+ * as they are); the tests pin it to them through the head-repetition identity.
+ */
+int moda_oracle_base_time(int i_q, int G)
+{
+    return i_q / G;
+}
+
+int moda_oracle_fwd_gqa(const double *Q, const double *K, const double *V,
+                        const double *Kd, const double *Vd,
+                        int B, int T, int Hq, int Hk, int d, int l, double scale,
+                        double *O, double *LSE)
+{
+    if (Hk < 1 || Hq % Hk != 0) return -3;
+    const int G = Hq / Hk;
+    const size_t slot = (size_t)B * T * Hk * d;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *x = (double *)malloc(sizeof(double) * (size_t)(T + l + 1));
+        if (!x) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+#pragma omp for collapse(3) schedule(dynamic, 8)
+            for (int b = 0; b < B; ++b)
+                for (int hq = 0; hq < Hq; ++hq)
+                    for (int t = 0; t < T; ++t) {
+                        const int hk = hq / G;
+                        const double *q = Q + idx4(b, t, hq, T, Hq, d);
+                        const int n = t + 1 + l;          /* keys of this row: t+1 sequence, then l depth */
+                        double m = -INFINITY;
+                        for (int j = 0; j < n; ++j) {
+                            const double *k = (j <= t) ? K + idx4(b, j, hk, T, Hk, d)
+                                                       : Kd + (size_t)(j - t - 1) * slot + idx4(b, t, hk, T, Hk, d);
+                            x[j] = scale * dot(q, k, d);
+                            if (x[j] > m) m = x[j];
+                        }
+                        double Z = 0.0;
+                        for (int j = 0; j < n; ++j) Z += exp(x[j] - m);
+                        const double lse = m + log(Z);
+                        double *o = O + idx4(b, t, hq, T, Hq, d);
+                        for (int c = 0; c < d; ++c) o[c] = 0.0;
+                        for (int j = 0; j < n; ++j) {
+                            const double *v = (j <= t) ? V + idx4(b, j, hk, T, Hk, d)
+                                                       : Vd + (size_t)(j - t - 1) * slot + idx4(b, t, hk, T, Hk, d);
+                            const double p = exp(x[j] - lse);
+                            for (int c = 0; c < d; ++c) o[c] += p * v[c];
+                        }
+                        LSE[((size_t)b * Hq + hq) * T + t] = lse;
+                    }
+        }
+        free(x);
+    }
+    return failed ? -1 : 0;
+}
+
+int moda_oracle_bwd_gqa(const double *Q, const double *K, const double *V,
+                        const double *Kd, const double *Vd, const double *dO,
+                        int B, int T, int Hq, int Hk, int d, int l, double scale,
+                        double *dQ, double *dK, double *dV, double *dKd, double *dVd)
+{
+    if (Hk < 1 || Hq % Hk != 0) return -3;
+    const int G = Hq / Hk;
+    const size_t Eq = (size_t)B * T * Hq * d, slot = (size_t)B * T * Hk * d;
+    double *O = (double *)malloc(sizeof(double) * Eq);
+    double *LSE = (double *)malloc(sizeof(double) * (size_t)B * Hq * T);
+    if (!O || !LSE) { free(O); free(LSE); return -1; }
+    int rc = moda_oracle_fwd_gqa(Q, K, V, Kd, Vd, B, T, Hq, Hk, d, l, scale, O, LSE);
+    if (rc != 0) { free(O); free(LSE); return rc; }
+
+    /* One thread owns one (b, hk): every output element it adds into belongs to that pair. */
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b)
+        for (int hk = 0; hk < Hk; ++hk) {
+            for (int t = 0; t < T; ++t) {
+                const size_t rk = idx4(b, t, hk, T, Hk, d);
+                for (int c = 0; c < d; ++c) { dK[rk + c] = 0.0; dV[rk + c] = 0.0; }
+                for (int i = 0; i < l; ++i)
+                    for (int c = 0; c < d; ++c) { dKd[i * slot + rk + c] = 0.0; dVd[i * slot + rk + c] = 0.0; }
+            }
+            for (int g = 0; g < G; ++g) {
+                const int hq = hk * G + g;
+                for (int t = 0; t < T; ++t) {
+                    const size_t rq = idx4(b, t, hq, T, Hq, d);
+                    const double *q = Q + rq, *go = dO + rq;
+                    const double lse = LSE[((size_t)b * Hq + hq) * T + t];
+                    const double D = dot(go, O + rq, d);
+                    double *gq = dQ + rq;
+                    for (int c = 0; c < d; ++c) gq[c] = 0.0;
+                    for (int j = 0; j <= t; ++j) {
+                        const size_t rj = idx4(b, j, hk, T, Hk, d);
+                        const double p = exp(scale * dot(q, K + rj, d) - lse);
+                        const double ds = p * (dot(go, V + rj, d) - D);
+                        for (int c = 0; c < d; ++c) {
+                            gq[c] += scale * ds * K[rj + c];
+                            dK[rj + c] += scale * ds * q[c];
+                            dV[rj + c] += p * go[c];
+                        }
+                    }
+                    const size_t rt = idx4(b, t, hk, T, Hk, d);
+                    for (int i = 0; i < l; ++i) {
+                        const double *kd = Kd + i * slot + rt, *vd = Vd + i * slot + rt;
+                        const double r = exp(scale * dot(q, kd, d) - lse);
+                        const double du = r * (dot(go, vd, d) - D);
+                        for (int c = 0; c < d; ++c) {
+                            gq[c] += scale * du * kd[c];
+                            dKd[i * slot + rt + c] += scale * du * q[c];
+                            dVd[i * slot + rt + c] += r * go[c];
+                        }
+                    }
+                }
+            }
+        }
+    free(O); free(LSE);
+    return 0;
 }

@@ -60,6 +60,12 @@ def _load():
             [_dp] * 6 + [ctypes.c_int] * 5 + [ctypes.c_double, _ip, ctypes.c_int, _ip, ctypes.c_int, ctypes.c_int]
             + [_dp] * 5
         )
+        lib.moda_oracle_base_time.restype = ctypes.c_int
+        lib.moda_oracle_base_time.argtypes = [ctypes.c_int, ctypes.c_int]
+        lib.moda_oracle_fwd_gqa.restype = ctypes.c_int
+        lib.moda_oracle_fwd_gqa.argtypes = [_dp] * 5 + [ctypes.c_int] * 6 + [ctypes.c_double, _dp, _dp]
+        lib.moda_oracle_bwd_gqa.restype = ctypes.c_int
+        lib.moda_oracle_bwd_gqa.argtypes = [_dp] * 6 + [ctypes.c_int] * 6 + [ctypes.c_double] + [_dp] * 5
         _lib = lib
     return _lib
 
@@ -173,3 +179,54 @@ def backward_rows(Q, K, V, Kd, Vd, dO, scale, qrows, krows=None, t_start=None):
     if rc != 0:
         raise MemoryError("oracle scratch allocation failed")
     return dQ, dKd, dVd, dK, dV
+
+
+# ---------------------------------------------------------------------------------------
+# Grouped-query form (Sec. 3, group-aware depth KV): Q, O, dO, dQ have Hq heads; K, V and the
+# depth K, V have Hk = Hq / G heads; query head hq uses KV head hq // G.
+# ---------------------------------------------------------------------------------------
+def base_time(i_q: int, G: int) -> int:
+    """Base-time index of flattened query row i_q = t * G + g."""
+    return int(_load().moda_oracle_base_time(int(i_q), int(G)))
+
+
+def _prep_gqa(Q, K, V, Kd, Vd):
+    Q = np.ascontiguousarray(Q, dtype=np.float64)
+    K = np.ascontiguousarray(K, dtype=np.float64)
+    if Q.ndim != 4 or K.ndim != 4:
+        raise ValueError("Q must be [B, T, Hq, d] and K [B, T, Hk, d]")
+    B, T, Hq, d = Q.shape
+    Hk = K.shape[2]
+    if K.shape != (B, T, Hk, d) or Hk < 1 or Hq % Hk:
+        raise ValueError("K must be [B, T, Hk, d] with Hk dividing Hq")
+    V = _f64(V, (B, T, Hk, d))
+    l = 0 if Kd is None else int(np.shape(Kd)[0])
+    if l == 0:
+        Kd = np.zeros((0, B, T, Hk, d)); Vd = np.zeros((0, B, T, Hk, d))
+    Kd = _f64(Kd, (l, B, T, Hk, d)); Vd = _f64(Vd, (l, B, T, Hk, d))
+    return Q, K, V, Kd, Vd, (B, T, Hq, Hk, d, l)
+
+
+def forward_gqa(Q, K, V, Kd, Vd, scale):
+    """O [B,T,Hq,d] and LSE [B,Hq,T] of the grouped-query MoDA operator (definition, fp64)."""
+    Q, K, V, Kd, Vd, (B, T, Hq, Hk, d, l) = _prep_gqa(Q, K, V, Kd, Vd)
+    O = np.empty((B, T, Hq, d)); LSE = np.empty((B, Hq, T))
+    rc = _load().moda_oracle_fwd_gqa(_ptr(Q), _ptr(K), _ptr(V), _ptr(Kd), _ptr(Vd),
+                                     B, T, Hq, Hk, d, l, float(scale), _ptr(O), _ptr(LSE))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return O, LSE
+
+
+def backward_gqa(Q, K, V, Kd, Vd, dO, scale):
+    """dQ [B,T,Hq,d], dK, dV [B,T,Hk,d], dKd, dVd [l,B,T,Hk,d] (sums over the heads of a group)."""
+    Q, K, V, Kd, Vd, (B, T, Hq, Hk, d, l) = _prep_gqa(Q, K, V, Kd, Vd)
+    dO = _f64(dO, (B, T, Hq, d))
+    dQ = np.empty((B, T, Hq, d)); dK = np.empty((B, T, Hk, d)); dV = np.empty((B, T, Hk, d))
+    dKd = np.empty((l, B, T, Hk, d)); dVd = np.empty((l, B, T, Hk, d))
+    rc = _load().moda_oracle_bwd_gqa(_ptr(Q), _ptr(K), _ptr(V), _ptr(Kd), _ptr(Vd), _ptr(dO),
+                                     B, T, Hq, Hk, d, l, float(scale),
+                                     _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dKd), _ptr(dVd))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return dQ, dK, dV, dKd, dVd

@@ -60,6 +60,8 @@ extern "C" {
 #define MODA_ERR_CUDA (-9)            /* a CUDA runtime/driver call failed (see moda_last_cuda_error) */
 #define MODA_ERR_DEVICE_TIMEOUT (-10) /* an earlier kernel gave up a bounded wait (see moda_last_status) */
 #define MODA_ERR_SCRATCH_LIMIT (-11)  /* problem needs more built-in scratch than moda_attn_bwd_static_scratch holds */
+#define MODA_ERR_BAD_GROUP (-12)      /* H_kv does not divide H, or more than MODA_MAX_GROUP query heads per group */
+#define MODA_MAX_GROUP 8
 
 /* Library version: major * 10000 + minor * 100 + patch. */
 int moda_version(void);
@@ -139,6 +141,36 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
                          int B, int T, int H, int d, int l, float scale,
                          void* dQ, void* dK, void* dV, void* d_depth_kv,
                          void* workspace, size_t workspace_bytes, int stages, void* stream);
+
+/*
+ * Grouped-query form (Sec. 3, "Group-aware depth KV calculation"; the paper's models use
+ * grouped-query attention).  H query heads share H_kv = H / G key/value heads: query head h
+ * uses key/value head h / G, i.e. the G heads of a group are adjacent, which is the paper's
+ * flattened query row i_q = t G + g with base time floor(i_q / G) = t; a row sees the sequence
+ * keys up to its base time and the depth keys stored at its base time.
+ *     Q, O, dO, dQ : bf16 [B][T][H][d]          K, V, dK, dV : bf16 [B][T][H_kv][d]
+ *     depth_kv, d_depth_kv : cache layout with H_kv heads (moda_depth_cache_bytes(B, T, H_kv, d, l))
+ *     LSE : fp32 [B][H][T]                      workspace : moda_bwd_workspace_bytes(B, T, H, d, l)
+ * dK, dV and the depth gradients are the sums over the G query heads of a group; the sum is
+ * taken in a fixed order (no atomics), so results are bit-reproducible.  The depth gradients
+ * are rounded to bf16 once per head of the group (G - 1 extra roundings).  H_kv must divide H
+ * and G <= MODA_MAX_GROUP (MODA_ERR_BAD_GROUP otherwise); H_kv == H is exactly
+ * moda_attn_fwd / moda_attn_bwd.  Everything else (validation, streams, ownership, errors) is
+ * as for those calls.
+ */
+int moda_attn_fwd_gqa(const void* Q, const void* K, const void* V, const void* depth_kv,
+                      int B, int T, int H, int H_kv, int d, int l, float scale,
+                      void* O, float* LSE, void* stream);
+int moda_attn_bwd_gqa(const void* Q, const void* K, const void* V, const void* depth_kv,
+                      const void* O, const void* dO, const float* LSE,
+                      int B, int T, int H, int H_kv, int d, int l, float scale,
+                      void* dQ, void* dK, void* dV, void* d_depth_kv,
+                      void* workspace, size_t workspace_bytes, void* stream);
+int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const void* depth_kv,
+                             const void* O, const void* dO, const float* LSE,
+                             int B, int T, int H, int H_kv, int d, int l, float scale,
+                             void* dQ, void* dK, void* dV, void* d_depth_kv,
+                             void* workspace, size_t workspace_bytes, int stages, void* stream);
 
 /*
  * Backward pass for callers that have no scratch buffer to give.  (The paper has no

@@ -8,9 +8,12 @@ from .binding import (  # noqa: F401
     ModaError,
     alloc_depth_cache,
     moda_attn_bwd,
+    moda_attn_bwd_gqa,
+    moda_attn_bwd_gqa_stages,
     moda_attn_bwd_stages,
     moda_attn_bwd_static_scratch,
     moda_attn_fwd,
+    moda_attn_fwd_gqa,
     moda_bwd_workspace_bytes,
     moda_depth_cache_append,
     moda_depth_cache_bytes,

@@ -21,6 +21,7 @@ SYMBOLS = (
     "moda_depth_cache_bytes", "moda_depth_cache_append", "moda_depth_cache_unpack",
     "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd", "moda_attn_bwd_stages",
     "moda_attn_bwd_static_scratch",
+    "moda_attn_fwd_gqa", "moda_attn_bwd_gqa", "moda_attn_bwd_gqa_stages",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -69,6 +70,12 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd_stages.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 5 + [sz, ci, vp]
     lib.moda_attn_bwd_static_scratch.restype = ci
     lib.moda_attn_bwd_static_scratch.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 4 + [vp]
+    lib.moda_attn_fwd_gqa.restype = ci
+    lib.moda_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
+    lib.moda_attn_bwd_gqa.restype = ci
+    lib.moda_attn_bwd_gqa.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
+    lib.moda_attn_bwd_gqa_stages.restype = ci
+    lib.moda_attn_bwd_gqa_stages.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, ci, vp]
     _lib = lib
     return lib
 
@@ -207,3 +214,55 @@ def moda_attn_bwd_static_scratch(Q, K, V, depth_kv, O, dO, LSE, l, scale, dQ, dK
         B, T, H, d, int(l), float(scale), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
         _stream(stream)), "moda_attn_bwd_static_scratch")
     return dQ, dK, dV, d_depth_kv
+
+
+def _gqa_shapes(Q, K, V):
+    B, T, H, d = _bthd(Q, "Q")
+    Bk, Tk, Hk, dk = _bthd(K, "K")
+    if (Bk, Tk, dk) != (B, T, d) or _bthd(V, "V") != (B, T, Hk, d):
+        raise ValueError("K and V must be bf16 [B, T, H_kv, d] tensors matching Q's B, T and d")
+    return B, T, H, Hk, d
+
+
+def moda_attn_fwd_gqa(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):
+    """Grouped-query forward: Q [B,T,H,d], K, V [B,T,H_kv,d], depth cache with H_kv heads.
+
+    Returns O [B,T,H,d] bf16 and LSE [B,H,T] fp32 (allocated if not given)."""
+    B, T, H, Hk, d = _gqa_shapes(Q, K, V)
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None:
+        LSE = torch.empty((B, H, T), dtype=torch.float32, device=Q.device)
+    _check(load().moda_attn_fwd_gqa(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
+                                    B, T, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE), _stream(stream)),
+           "moda_attn_fwd_gqa")
+    return O, LSE
+
+
+def moda_attn_bwd_gqa(Q, K, V, depth_kv, O, dO, LSE, l, scale,
+                      dQ=None, dK=None, dV=None, d_depth_kv=None, workspace=None, stream=None, stages=None):
+    """Grouped-query backward: dQ [B,T,H,d], dK, dV [B,T,H_kv,d], depth gradients (cache layout, H_kv heads).
+
+    With ``stages`` (a MODA_BWD_STAGE_* mask) the call goes through moda_attn_bwd_gqa_stages."""
+    B, T, H, Hk, d = _gqa_shapes(Q, K, V)
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(K) if dK is None else dK
+    dV = torch.empty_like(V) if dV is None else dV
+    if l > 0 and d_depth_kv is None:
+        d_depth_kv = alloc_depth_cache(B, T, Hk, d, l, Q.device)
+    if workspace is None:
+        workspace = torch.empty(moda_bwd_workspace_bytes(B, T, H, d, l), dtype=torch.uint8, device=Q.device)
+    args = [_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
+            _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, Hk, d, int(l), float(scale),
+            _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
+            _ptr(workspace), workspace.numel() * workspace.element_size()]
+    if stages is None:
+        _check(load().moda_attn_bwd_gqa(*args, _stream(stream)), "moda_attn_bwd_gqa")
+    else:
+        _check(load().moda_attn_bwd_gqa_stages(*args, int(stages), _stream(stream)), "moda_attn_bwd_gqa_stages")
+    return dQ, dK, dV, d_depth_kv
+
+
+def moda_attn_bwd_gqa_stages(*args, stages, **kwargs):
+    """moda_attn_bwd_gqa restricted to the launches selected by the ``stages`` bit mask."""
+    return moda_attn_bwd_gqa(*args, stages=stages, **kwargs)

@@ -71,6 +71,12 @@ int check_shape(int B, int T, int H, int d) {
     return MODA_OK;
 }
 
+// Query heads H on H_kv key/value heads: H_kv must divide H, at most MODA_MAX_GROUP heads per group.
+int check_groups(int H, int H_kv) {
+    if (H_kv < 1 || H % H_kv != 0 || H / H_kv > MODA_MAX_GROUP) return MODA_ERR_BAD_GROUP;
+    return MODA_OK;
+}
+
 int check_device() {
     static thread_local int cached_dev = -1;
     static thread_local int cached_rc = MODA_ERR_DEVICE;
@@ -92,14 +98,14 @@ bool set_smem_limit(Kernel k, int bytes) {
 // d = 128 runs moda_fwd_kernel (one softmax warpgroup: the tensor pipe and the MMA issue rate set the
 // pace); d = 64 runs moda_fwd2_kernel (two softmax warpgroups, three score buffers: the exponentials do).
 template <int D>
-int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int H, int l,
+int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int H, int Hk, int l,
                float scale, void* O, float* LSE, cudaStream_t stream) {
     constexpr bool kWide = (D == 64);
     constexpr int kSmem = kWide ? Fwd2Smem<D>::kDynamic : FwdSmem<D>::kDynamic;
     constexpr int kThreads = kWide ? kFwd2Threads : kFwdThreads;
     CUtensorMap mQ, mK, mV, mO;
-    if (!make_bthd_map(&mQ, Q, B, T, H, D) || !make_bthd_map(&mK, K, B, T, H, D) ||
-        !make_bthd_map(&mV, V, B, T, H, D) || !make_bthd_map(&mO, O, B, T, H, D))
+    if (!make_bthd_map(&mQ, Q, B, T, H, D) || !make_bthd_map(&mK, K, B, T, Hk, D) ||
+        !make_bthd_map(&mV, V, B, T, Hk, D) || !make_bthd_map(&mO, O, B, T, H, D))
         return MODA_ERR_CUDA;
     static thread_local int configured_dev = -1;
     int dev = 0;
@@ -114,6 +120,7 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.O = static_cast<__nv_bfloat16*>(O);
     p.LSE = LSE;
     p.B = B; p.T = T; p.H = H; p.l = l;
+    p.G = H / Hk;
     p.scale_log2 = scale * kLog2e;
     const unsigned grid = unsigned(B) * H * num_tiles(T);
     if (kWide) moda_fwd2_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
@@ -130,14 +137,14 @@ inline bool dq_depth_heavy(int T, int l, int d) {
 
 template <int D>
 int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
-    const int B = a.B, T = a.T, H = a.H;
+    const int B = a.B, T = a.T, H = a.H, Hk = a.Hk, G = a.H / a.Hk;
     CUtensorMap mQ, mdO, mK64, mV64, mdQ, mK, mV, mQ64, mdO64, mdK, mdV;
     if (!make_bthd_map(&mQ, a.Q, B, T, H, D) || !make_bthd_map(&mdO, a.dO, B, T, H, D) ||
-        !make_bthd_map(&mK64, a.K, B, T, H, D, kKeyTile) || !make_bthd_map(&mV64, a.V, B, T, H, D, kKeyTile) ||
-        !make_bthd_map(&mdQ, a.dQ, B, T, H, D) || !make_bthd_map(&mK, a.K, B, T, H, D) ||
-        !make_bthd_map(&mV, a.V, B, T, H, D) || !make_bthd_map(&mQ64, a.Q, B, T, H, D, kKeyTile) ||
-        !make_bthd_map(&mdO64, a.dO, B, T, H, D, kKeyTile) || !make_bthd_map(&mdK, a.dK, B, T, H, D) ||
-        !make_bthd_map(&mdV, a.dV, B, T, H, D))
+        !make_bthd_map(&mK64, a.K, B, T, Hk, D, kKeyTile) || !make_bthd_map(&mV64, a.V, B, T, Hk, D, kKeyTile) ||
+        !make_bthd_map(&mdQ, a.dQ, B, T, H, D) || !make_bthd_map(&mK, a.K, B, T, Hk, D) ||
+        !make_bthd_map(&mV, a.V, B, T, Hk, D) || !make_bthd_map(&mQ64, a.Q, B, T, H, D, kKeyTile) ||
+        !make_bthd_map(&mdO64, a.dO, B, T, H, D, kKeyTile) || !make_bthd_map(&mdK, a.dK, B, T, Hk, D) ||
+        !make_bthd_map(&mdV, a.dV, B, T, Hk, D))
         return MODA_ERR_CUDA;
     static thread_local int configured_dev = -1;
     int dev = 0;
@@ -157,24 +164,30 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
         bwd_delta_kernel<D><<<grid, 256, 0, stream>>>(static_cast<const uint4*>(a.O), static_cast<const uint4*>(a.dO), delta, B, T, H);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     }
-    const unsigned grid = unsigned(B) * H * num_tiles(T);
+    // one CTA per (batch, key/value head, 128-row tile)
+    const unsigned grid = unsigned(B) * Hk * num_tiles(T);
     if (stages & 2) {
         DqParams p;
         p.depth_kv = static_cast<const __nv_bfloat16*>(a.depth_kv);
         p.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
         p.LSE = a.LSE; p.delta = delta;
-        p.B = B; p.T = T; p.H = H; p.l = a.l;
+        p.B = B; p.T = T; p.H = H; p.l = a.l; p.G = G;
         p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
-        if (dq_depth_heavy(T, a.l, D))
-            moda_bwd_dq_kernel<128, 2><<<grid, kBwdDqThreads, DqSmem<128, 2>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
-        else
-            moda_bwd_dq_kernel<D, 3><<<grid, kBwdDqThreads, DqSmem<D, 3>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
-        if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+        // One launch per member g of the groups: launch g handles query head hk G + g of every
+        // key/value head and adds its depth gradients to those of the launches before it.
+        for (int g = 0; g < G; ++g) {
+            p.g = g;
+            if (dq_depth_heavy(T, a.l, D))
+                moda_bwd_dq_kernel<128, 2><<<grid, kBwdDqThreads, DqSmem<128, 2>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
+            else
+                moda_bwd_dq_kernel<D, 3><<<grid, kBwdDqThreads, DqSmem<D, 3>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
+            if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+        }
     }
     if (stages & 4) {
         DkvParams p;
         p.LSE = a.LSE; p.delta = delta;
-        p.B = B; p.T = T; p.H = H;
+        p.B = B; p.T = T; p.H = H; p.G = G;
         p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
         moda_bwd_dkdv_kernel<D><<<grid, kBwdDkvThreads, DkvSmem<D>::kDynamic, stream>>>(mK, mV, mQ64, mdO64, mdK, mdV, p);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
@@ -209,6 +222,7 @@ const char* moda_strerror(int code) {
         case MODA_ERR_DEVICE: return "the current CUDA device is not an sm_100 part";
         case MODA_ERR_CUDA: return "a CUDA call failed (see moda_last_cuda_error)";
         case MODA_ERR_DEVICE_TIMEOUT: return "a kernel gave up a bounded wait (see moda_last_status)";
+        case MODA_ERR_BAD_GROUP: return "H_kv must divide H with at most 8 query heads per key/value head";
         case MODA_ERR_SCRATCH_LIMIT: return "B*H*T exceeds the built-in scratch of moda_attn_bwd_static_scratch (2^20 rows)";
         default: return "unknown error code";
     }
@@ -259,7 +273,14 @@ int moda_depth_cache_unpack(const void* cache, int B, int T, int H, int d, int s
 int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth_kv,
                   int B, int T, int H, int d, int l, float scale,
                   void* O, float* LSE, void* stream) {
+    return moda_attn_fwd_gqa(Q, K, V, depth_kv, B, T, H, H, d, l, scale, O, LSE, stream);
+}
+
+int moda_attn_fwd_gqa(const void* Q, const void* K, const void* V, const void* depth_kv,
+                      int B, int T, int H, int H_kv, int d, int l, float scale,
+                      void* O, float* LSE, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_groups(H, H_kv)) return rc;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!Q || !K || !V || !O || !LSE || (l > 0 && !depth_kv)) return MODA_ERR_NULL_POINTER;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
@@ -267,8 +288,8 @@ int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth
         return MODA_ERR_MISALIGNED;
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv, B, T, H, l, scale, O, LSE, st)
-                    : launch_fwd<64>(Q, K, V, depth_kv, B, T, H, l, scale, O, LSE, st);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv, B, T, H, H_kv, l, scale, O, LSE, st)
+                    : launch_fwd<64>(Q, K, V, depth_kv, B, T, H, H_kv, l, scale, O, LSE, st);
 }
 
 size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l) {
@@ -290,7 +311,26 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
                          int B, int T, int H, int d, int l, float scale,
                          void* dQ, void* dK, void* dV, void* d_depth_kv,
                          void* workspace, size_t workspace_bytes, int stages, void* stream) {
+    return moda_attn_bwd_gqa_stages(Q, K, V, depth_kv, O, dO, LSE, B, T, H, H, d, l, scale, dQ, dK, dV, d_depth_kv,
+                                    workspace, workspace_bytes, stages, stream);
+}
+
+int moda_attn_bwd_gqa(const void* Q, const void* K, const void* V, const void* depth_kv,
+                      const void* O, const void* dO, const float* LSE,
+                      int B, int T, int H, int H_kv, int d, int l, float scale,
+                      void* dQ, void* dK, void* dV, void* d_depth_kv,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    return moda_attn_bwd_gqa_stages(Q, K, V, depth_kv, O, dO, LSE, B, T, H, H_kv, d, l, scale, dQ, dK, dV, d_depth_kv,
+                                    workspace, workspace_bytes, MODA_BWD_ALL_STAGES, stream);
+}
+
+int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const void* depth_kv,
+                             const void* O, const void* dO, const float* LSE,
+                             int B, int T, int H, int H_kv, int d, int l, float scale,
+                             void* dQ, void* dK, void* dV, void* d_depth_kv,
+                             void* workspace, size_t workspace_bytes, int stages, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_groups(H, H_kv)) return rc;
     if (stages <= 0 || stages > MODA_BWD_ALL_STAGES) return MODA_ERR_BAD_SHAPE;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv || !d_depth_kv)))
@@ -304,7 +344,7 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     BwdArgs a;
     a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv; a.O = O; a.dO = dO; a.LSE = LSE;
-    a.B = B; a.T = T; a.H = H; a.l = l; a.scale = scale;
+    a.B = B; a.T = T; a.H = H; a.Hk = H_kv; a.l = l; a.scale = scale;
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
     return d == 128 ? launch_bwd<128>(a, stages, st) : launch_bwd<64>(a, stages, st);
 }
@@ -359,7 +399,7 @@ extern "C" int moda_attn_bwd_static_scratch(const void* Q, const void* K, const 
     if (int rc = static_scratch_for_current_device(&scratch)) return rc;
     BwdArgs a;
     a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv; a.O = O; a.dO = dO; a.LSE = LSE;
-    a.B = B; a.T = T; a.H = H; a.l = l; a.scale = scale;
+    a.B = B; a.T = T; a.H = H; a.Hk = H; a.l = l; a.scale = scale;
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = scratch;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return d == 128 ? launch_bwd<128>(a, MODA_BWD_ALL_STAGES, st) : launch_bwd<64>(a, MODA_BWD_ALL_STAGES, st);

@@ -28,7 +28,7 @@ namespace moda {
 struct BwdArgs {
     const void *Q, *K, *V, *depth_kv, *O, *dO;
     const float* LSE;
-    int B, T, H, l;
+    int B, T, H, Hk, l;          // H query heads on Hk key/value heads
     float scale;
     void *dQ, *dK, *dV, *d_depth_kv, *workspace;
 };
@@ -134,9 +134,21 @@ struct DqParams {
     __nv_bfloat16* d_depth_kv;
     const float* LSE;
     const float* delta;
-    int B, T, H, l;
+    int B, T, H, l;     // H = number of query heads
+    int G;              // query heads per key/value head
+    int g;              // this launch handles query head hk G + g of every key/value head hk
     float scale, scale_log2;
 };
+
+// Sum of two groups of 8 bf16, added in fp32 and rounded once.
+__device__ __forceinline__ uint4 add_bf16x8(const uint4& a, const uint4& b) {
+    uint4 r;
+    r.x = pack_bf16x2(bf16_lo_to_f32(a.x) + bf16_lo_to_f32(b.x), bf16_hi_to_f32(a.x) + bf16_hi_to_f32(b.x));
+    r.y = pack_bf16x2(bf16_lo_to_f32(a.y) + bf16_lo_to_f32(b.y), bf16_hi_to_f32(a.y) + bf16_hi_to_f32(b.y));
+    r.z = pack_bf16x2(bf16_lo_to_f32(a.z) + bf16_lo_to_f32(b.z), bf16_hi_to_f32(a.z) + bf16_hi_to_f32(b.z));
+    r.w = pack_bf16x2(bf16_lo_to_f32(a.w) + bf16_lo_to_f32(b.w), bf16_hi_to_f32(a.w) + bf16_hi_to_f32(b.w));
+    return r;
+}
 
 // bf16x2 product with both factors already packed.
 __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
@@ -171,7 +183,9 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     const int nq = num_tiles(p.T);
     const int bh = blockIdx.x / nq;
     const int qt = nq - 1 - (blockIdx.x % nq);
-    const int b = bh / p.H, h = bh % p.H;
+    const int Hk = p.H / p.G;
+    const int b = bh / Hk, hk = bh % Hk;             // key/value head
+    const int h = hk * p.G + p.g;                    // query head
     const int q0 = qt * kTileRows;
     const int n_kv = min(2 * (qt + 1), (p.T + kKeyTile - 1) / kKeyTile);   // 64-key tiles at or below the diagonal
 
@@ -302,8 +316,12 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             const size_t row_idx = (size_t(b) * p.H + h) * p.T + q0 + r;
             const float neg_lse2 = valid ? -p.LSE[row_idx] * kLog2e : -INFINITY;
             const float delta = valid ? p.delta[row_idx] : 0.f;
-            const size_t slot_stride = cache_slot_elems(p.B, p.T, p.H, D) / 8;          // in uint4
-            const size_t blk = (((size_t(b) * p.H + h) * nq + qt) * 2) * (kTileRows * CH) + r;
+            const size_t slot_stride = cache_slot_elems(p.B, p.T, Hk, D) / 8;           // in uint4
+            const size_t blk = (((size_t(b) * Hk + hk) * nq + qt) * 2) * (kTileRows * CH) + r;
+            // The depth gradients are sums over the G query heads of a group: the launch for g = 0
+            // writes them, every later launch of the same backward adds its share to what is there
+            // (same thread, same addresses; launches are ordered by the stream).
+            const bool add_to = p.g > 0;
             uint4* gK = reinterpret_cast<uint4*>(p.d_depth_kv) + blk;
             uint4* gV = gK + kTileRows * CH;
             mbar_wait(bar(kDqBarQ), 0, abort_flag, 60);
@@ -390,6 +408,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                             o.y = pack_bf16x2(w * g[8 * c + 2], w * g[8 * c + 3]);
                             o.z = pack_bf16x2(w * g[8 * c + 4], w * g[8 * c + 5]);
                             o.w = pack_bf16x2(w * g[8 * c + 6], w * g[8 * c + 7]);
+                            if (add_to) o = add_bf16x8(o, dst[c * kTileRows]);
                             dst[c * kTileRows] = o;
                         }
                     }
@@ -442,6 +461,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                             o.y = mul_bf16x2(qp[c].y, sdu2);
                             o.z = mul_bf16x2(qp[c].z, sdu2);
                             o.w = mul_bf16x2(qp[c].w, sdu2);
+                            if (add_to) o = add_bf16x8(o, dst[c * kTileRows]);
                             dst[c * kTileRows] = o;
                         }
                     }
@@ -483,8 +503,8 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     const uint32_t dstV = dstK + L::kHalfTileBytes;
 #pragma unroll
                     for (int s = 0; s < NSUB; ++s) {
-                        tma_load_4d(dstK + s * L::kHalfSubBytes, &mapK64, bar(kDqBarKVFull + st), s * 64, h, j * kKeyTile, b);
-                        tma_load_4d(dstV + s * L::kHalfSubBytes, &mapV64, bar(kDqBarKVFull + st), s * 64, h, j * kKeyTile, b);
+                        tma_load_4d(dstK + s * L::kHalfSubBytes, &mapK64, bar(kDqBarKVFull + st), s * 64, hk, j * kKeyTile, b);
+                        tma_load_4d(dstV + s * L::kHalfSubBytes, &mapV64, bar(kDqBarKVFull + st), s * 64, hk, j * kKeyTile, b);
                     }
                 }
             }
@@ -494,10 +514,10 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             // values (pass B), keys again (pass C).
             if (lane == 0 && p.l > 0) {
                 const uint64_t policy = l2_policy_evict_first();
-                const size_t slot_bytes = cache_slot_elems(p.B, p.T, p.H, D) * 2;
+                const size_t slot_bytes = cache_slot_elems(p.B, p.T, Hk, D) * 2;
                 const size_t kv_bytes = size_t(kTileRows) * D * 2;
                 const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
-                                     (((size_t(b) * p.H + h) * nq + qt) * 2) * kv_bytes;
+                                     (((size_t(b) * Hk + hk) * nq + qt) * 2) * kv_bytes;
                 // keys of a group are fetched twice; the first fetch is kept in L2 (evict_last), the second
                 // fetch and the values are not needed again (evict_first)
                 const uint64_t keep = l2_policy_evict_last();
@@ -627,7 +647,8 @@ enum DkvBar : int {
 struct DkvParams {
     const float* LSE;
     const float* delta;
-    int B, T, H;
+    int B, T, H;        // H = number of query heads
+    int G;              // query heads per key/value head; dK, dV sum over the G heads of a group
     float scale, scale_log2;
 };
 
@@ -656,11 +677,13 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
     const int nk = num_tiles(p.T);
     const int bh = blockIdx.x / nk;
     const int kt = blockIdx.x % nk;                       // key tiles in ascending order: most work first
-    const int b = bh / p.H, h = bh % p.H;
+    const int Hk = p.H / p.G;
+    const int b = bh / Hk, h = bh % Hk;                   // h: key/value head of this CTA
     const int k0 = kt * kTileRows;
     const int nq64 = (p.T + kKeyTile - 1) / kKeyTile;
     const int i_first = 2 * kt;                           // first 64-query tile that can see this key tile
-    const int n_it = nq64 - i_first;
+    const int n_per = nq64 - i_first;                     // query tiles per query head
+    const int n_it = n_per * p.G;                         // iteration it: query head h G + it / n_per, tile i_first + it % n_per
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -703,7 +726,7 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
         const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
         for (int it = 0; it < n_it; ++it) {
             const int st = it % L::kStages, buf = it & 1;
-            const int qoff = (i_first + it) * kKeyTile - k0;  // query of column c sees key row r iff qoff + c >= r
+            const int qoff = (i_first + it % n_per) * kKeyTile - k0;  // query of column c sees key row r iff qoff + c >= r
             mbar_wait(bar(kDkvBarQFull + st), (it / L::kStages) & 1, abort_flag, 90);   // LSE / D_t of this stage
             mbar_wait(bar(kDkvBarSFull + buf), (it >> 1) & 1, abort_flag, 91);
             tc_fence_after_sync();
@@ -785,10 +808,11 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 tma_load_4d(sbase + L::kV + s * L::kSubBytes, &mapV, bar(kDkvBarKV), s * 64, h, k0, b);
             }
         }
-        const size_t row_base = (size_t(b) * p.H + h) * p.T;
         for (int it = 0; it < n_it; ++it) {
             const int st = it % L::kStages;
-            const int qrow0 = (i_first + it) * kKeyTile;
+            const int hq = h * p.G + it / n_per;
+            const size_t row_base = (size_t(b) * p.H + hq) * p.T;
+            const int qrow0 = (i_first + it % n_per) * kKeyTile;
             if (it >= L::kStages)
                 mbar_wait(bar(kDkvBarQEmpty + st), ((it - L::kStages) / L::kStages) & 1, abort_flag, 100);
             {
@@ -808,8 +832,8 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
                 const uint32_t dstdO = dstQ + L::kHalfTileBytes;
 #pragma unroll
                 for (int s = 0; s < NSUB; ++s) {
-                    tma_load_4d(dstQ + s * L::kHalfSubBytes, &mapQ64, bar(kDkvBarQFull + st), s * 64, h, qrow0, b);
-                    tma_load_4d(dstdO + s * L::kHalfSubBytes, &mapdO64, bar(kDkvBarQFull + st), s * 64, h, qrow0, b);
+                    tma_load_4d(dstQ + s * L::kHalfSubBytes, &mapQ64, bar(kDkvBarQFull + st), s * 64, hq, qrow0, b);
+                    tma_load_4d(dstdO + s * L::kHalfSubBytes, &mapdO64, bar(kDkvBarQFull + st), s * 64, hq, qrow0, b);
                 }
             } else {
                 mbar_arrive(bar(kDkvBarQFull + st));

@@ -75,9 +75,30 @@ struct FwdParams {
     const __nv_bfloat16* depth_kv;   // cache layout, >= l slots (unused when l == 0)
     __nv_bfloat16* O;
     float* LSE;
-    int B, T, H, l;
+    int B, T, H, l;                  // H = number of query heads
+    int G;                           // query heads per key/value head (1 = plain multi-head attention)
     float scale_log2;                // scale * log2(e)
 };
+
+// Which (batch, query head, key/value head, query tile) a CTA works on.  The G query heads that
+// share a key/value head (Sec. 3, group-aware depth KV: rows with the same base time reuse the same
+// depth blocks) are adjacent CTAs, so they run together and the depth block and the K/V tiles they
+// share cross HBM once and are served by L2 to the others; inside a key/value head the heaviest
+// query tiles come first.
+struct TileCoord {
+    int b, h, hk, qt;
+};
+__device__ __forceinline__ TileCoord tile_coord(int block, int nq, int H, int G) {
+    const int per_kv = nq * G;
+    const int bhk = block / per_kv, rem = block % per_kv;
+    const int Hk = H / G;
+    TileCoord c;
+    c.b = bhk / Hk;
+    c.hk = bhk % Hk;
+    c.h = c.hk * G + rem % G;
+    c.qt = nq - 1 - rem / G;
+    return c;
+}
 
 // Shared-memory address of 16-byte chunk `c` (0..D/8-1) of row `r` inside a 128 x D tile that
 // TMA wrote as D/64 sub-tiles of [128][64] with the 128-byte swizzle.
@@ -112,9 +133,9 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     const int lane = tid & 31;
 
     const int nq = num_tiles(p.T);
-    const int bh = blockIdx.x / nq;
-    const int qt = nq - 1 - (blockIdx.x % nq);      // heaviest query tiles of a head first
-    const int b = bh / p.H, h = bh % p.H;
+    const TileCoord tc = tile_coord(blockIdx.x, nq, p.H, p.G);
+    const int b = tc.b, h = tc.h, hk = tc.hk, qt = tc.qt;
+    const int Hk = p.H / p.G;
     const int q0 = qt * kTileRows;
     const int n_kv = qt + 1;                         // causal: key tiles 0..qt
 
@@ -406,13 +427,13 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 #pragma unroll
                 for (int s = 0; s < NSUB; ++s)
                     tma_load_4d(sbase + L::kK + st * L::kTileBytes + s * L::kSubBytes, &mapK, bar(kBarKFull + st),
-                                s * 64, h, j * kTileRows, b);
+                                s * 64, hk, j * kTileRows, b);
                 if (j >= 2) mbar_wait(bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 31);
                 mbar_arrive_expect_tx(bar(kBarVFull + st), L::kTileBytes);
 #pragma unroll
                 for (int s = 0; s < NSUB; ++s)
                     tma_load_4d(sbase + L::kV + st * L::kTileBytes + s * L::kSubBytes, &mapV, bar(kBarVFull + st),
-                                s * 64, h, j * kTileRows, b);
+                                s * 64, hk, j * kTileRows, b);
             }
         }
       } else if (warp == 9) {
@@ -479,9 +500,9 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         // them.  The ring keeps up to kRingStages x 16 KiB of HBM reads in flight per SM.
         if (lane == 0 && p.l > 0) {
             const uint64_t policy = l2_policy_evict_first();          // the depth cache is read exactly once
-            const size_t slot_bytes = cache_slot_elems(p.B, p.T, p.H, D) * 2;
+            const size_t slot_bytes = cache_slot_elems(p.B, p.T, Hk, D) * 2;
             const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
-                                 (((size_t(b) * p.H + h) * nq + qt) * 2) * (size_t(kTileRows) * D * 2);
+                                 (((size_t(b) * Hk + hk) * nq + qt) * 2) * (size_t(kTileRows) * D * 2);
             int unit = 0;
             for (int kv = 0; kv < 2; ++kv)
                 for (int half = 0; half < NSUB; ++half)

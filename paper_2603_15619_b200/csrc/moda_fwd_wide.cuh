@@ -126,9 +126,9 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const int lane = tid & 31;
 
     const int nq = num_tiles(p.T);
-    const int bh = blockIdx.x / nq;
-    const int qt = nq - 1 - (blockIdx.x % nq);      // heaviest query tiles of a head first
-    const int b = bh / p.H, h = bh % p.H;
+    const TileCoord tc = tile_coord(blockIdx.x, nq, p.H, p.G);
+    const int b = tc.b, h = tc.h, hk = tc.hk, qt = tc.qt;
+    const int Hk = p.H / p.G;
     const int q0 = qt * kTileRows;
     const int n_kv = min((kTileRows / kFwdBN) * (qt + 1), (p.T + kFwdBN - 1) / kFwdBN);   // key tiles at or below the diagonal
 
@@ -458,13 +458,13 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
                 for (int s = 0; s < NSUB; ++s)
                     tma_load_4d(sbase + L::kK + st * L::kKeyTileBytes + s * L::kKeySubBytes, &mapK, bar(k2BarKFull + st),
-                                s * 64, h, j * kFwdBN, b);
+                                s * 64, hk, j * kFwdBN, b);
                 if (j >= L::kStages) mbar_wait(bar(k2BarVEmpty + st), par, abort_flag, 31);
                 mbar_arrive_expect_tx(bar(k2BarVFull + st), L::kKeyTileBytes);
 #pragma unroll
                 for (int s = 0; s < NSUB; ++s)
                     tma_load_4d(sbase + L::kV + st * L::kKeyTileBytes + s * L::kKeySubBytes, &mapV, bar(k2BarVFull + st),
-                                s * 64, h, j * kFwdBN, b);
+                                s * 64, hk, j * kFwdBN, b);
             }
         }
       } else if (warp == 13) {
@@ -531,9 +531,9 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         // them.  The ring keeps up to kRingStages x 16 KiB of HBM reads in flight per SM.
         if (lane == 0 && p.l > 0) {
             const uint64_t policy = l2_policy_evict_first();          // the depth cache is read exactly once
-            const size_t slot_bytes = cache_slot_elems(p.B, p.T, p.H, D) * 2;
+            const size_t slot_bytes = cache_slot_elems(p.B, p.T, Hk, D) * 2;
             const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
-                                 (((size_t(b) * p.H + h) * nq + qt) * 2) * (size_t(kTileRows) * D * 2);
+                                 (((size_t(b) * Hk + hk) * nq + qt) * 2) * (size_t(kTileRows) * D * 2);
             int unit = 0;
             for (int kv = 0; kv < 2; ++kv)
                 for (int half = 0; half < NSUB; ++half)

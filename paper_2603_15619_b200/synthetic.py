@@ -95,3 +95,13 @@ def make(w: Workload, seed: int = 0, device="cpu") -> dict:
         Vd[i] = tensor(w, "Vd", seed, i, device)
     out["Kd"], out["Vd"] = Kd, Vd
     return out
+
+
+def make_gqa(B: int, T: int, H: int, H_kv: int, d: int, l: int, seed: int = 0, device="cpu", **kw) -> dict:
+    """Inputs of a grouped-query problem: Q, dO [B,T,H,d]; K, V [B,T,H_kv,d]; Kd, Vd [l,B,T,H_kv,d]."""
+    wq = Workload("gqa/q", B, T, H, d, l, **kw)
+    wk = Workload("gqa/kv", B, T, H_kv, d, l, **kw)
+    out = make(wk, seed, device)
+    out["Q"] = tensor(wq, "Q", seed, 0, device)
+    out["dO"] = tensor(wq, "dO", seed, 0, device)
+    return out

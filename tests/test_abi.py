@@ -28,7 +28,7 @@ def test_library_loads_and_exports_every_declared_symbol():
 
 
 def test_strerror_covers_all_codes():
-    for code in range(0, -12, -1):
+    for code in range(0, -13, -1):
         assert binding.strerror(code) != "unknown error code"
     assert binding.strerror(-99) == "unknown error code"
 
@@ -71,6 +71,11 @@ def test_argument_validation_rejects_before_any_launch():
     assert lib.moda_attn_bwd(*args, None, ctypes.c_size_t(1 << 20), None) == -7
     assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 0, None) == -3
     assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 8, None) == -3
+    # grouped-query entry points: H_kv must divide H, at most 8 query heads per group
+    gqa = lambda H, Hk: lib.moda_attn_fwd_gqa(p, p, p, None, 1, 128, H, Hk, 64, 0, ctypes.c_float(0.125), p, p, None)
+    assert gqa(6, 4) == -12 and gqa(4, 0) == -12 and gqa(16, 1) == -12
+    gargs = [p] * 7 + [1, 128, 6, 4, 64, 0, ctypes.c_float(0.125)] + [p, p, p, None]
+    assert lib.moda_attn_bwd_gqa(*gargs, p, ctypes.c_size_t(1 << 20), None) == -12
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

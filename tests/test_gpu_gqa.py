@@ -1,0 +1,90 @@
+"""Grouped-query MoDA on the GPU against the fp64 oracle (through the C ABI).
+
+H query heads on H_kv key/value heads (paper Sec. 3, group-aware depth KV): forward, backward,
+the G = 1 entry points as the special case, bit-reproducibility of the grouped sums.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2603_15619_b200 as moda
+from paper_2603_15619_b200 import synthetic
+from oracle import moda_oracle as orc
+
+from parity import (TOL_GRAD_REL_L2, TOL_LSE_ABS, TOL_O_MAX_ABS, TOL_O_REL_L2, build_cache, f64, rel_l2,
+                    unpack_cache)
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    # B, T, H, H_kv, d, l
+    (1, 256, 4, 2, 64, 4), (2, 300, 4, 1, 64, 3), (1, 384, 8, 2, 128, 5), (2, 129, 2, 1, 128, 2),
+    (1, 640, 6, 3, 128, 8), (1, 200, 4, 2, 64, 0), (1, 1, 2, 1, 64, 2), (1, 1000, 8, 1, 64, 1),
+]
+
+
+def run(x, l, scale):
+    B, T, H, d = x["Q"].shape
+    Hk = x["K"].shape[2]
+    cache = build_cache(x["Kd"], x["Vd"]) if l > 0 else None
+    O, LSE = moda.moda_attn_fwd_gqa(x["Q"], x["K"], x["V"], cache, l, scale)
+    dcache = None
+    if l > 0:
+        dcache = moda.alloc_depth_cache(B, T, Hk, d, l)
+        dcache.fill_(5.0)
+    dQ = torch.full_like(x["Q"], 3.0)
+    dK = torch.full_like(x["K"], 3.0)
+    dV = torch.full_like(x["V"], 3.0)
+    moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale,
+                           dQ=dQ, dK=dK, dV=dV, d_depth_kv=dcache)
+    assert moda.moda_last_status() == 0
+    if l > 0:
+        dKd, dVd = unpack_cache(dcache, l, B, T, Hk, d)
+    else:
+        dKd = dVd = torch.zeros((0, B, T, Hk, d), dtype=torch.bfloat16, device="cuda")
+    return O, LSE, (dQ, dK, dV, dKd, dVd)
+
+
+def grad_err(g, r):
+    g, r = f64(g), np.asarray(r)
+    return float(np.linalg.norm(g - r) / (np.linalg.norm(r) + 1e-5 * np.sqrt(r.size))) if r.size else 0.0
+
+
+@pytest.mark.parametrize("B,T,H,Hk,d,l", SHAPES)
+def test_grouped_query_forward_and_backward_match_the_oracle(B, T, H, Hk, d, l):
+    scale = d ** -0.5
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=31, device="cuda")
+    O, LSE, grads = run(x, l, scale)
+    xs = [f64(x[n]) for n in ("Q", "K", "V", "Kd", "Vd")]
+    O_ref, LSE_ref = orc.forward_gqa(*xs, scale)
+    assert rel_l2(f64(O), O_ref) <= TOL_O_REL_L2
+    assert float(np.abs(f64(O) - O_ref).max()) <= TOL_O_MAX_ABS
+    assert float(np.abs(f64(LSE) - LSE_ref).max()) <= TOL_LSE_ABS
+    ref = orc.backward_gqa(*xs, f64(x["dO"]), scale)
+    for name, g, r in zip(("dQ", "dK", "dV", "dKd", "dVd"), grads, ref):
+        assert grad_err(g, r) <= TOL_GRAD_REL_L2, f"{name}: {grad_err(g, r):.3e}"
+
+
+def test_one_head_per_group_is_bitwise_the_plain_entry_points():
+    B, T, H, d, l = 2, 300, 3, 64, 4
+    w = synthetic.Workload("g1", B, T, H, d, l)
+    x = synthetic.make(w, seed=5, device="cuda")
+    cache = build_cache(x["Kd"], x["Vd"])
+    O, LSE = moda.moda_attn_fwd(x["Q"], x["K"], x["V"], cache, l, w.scale)
+    O2, LSE2 = moda.moda_attn_fwd_gqa(x["Q"], x["K"], x["V"], cache, l, w.scale)
+    assert torch.equal(O, O2) and torch.equal(LSE, LSE2)
+    a = moda.moda_attn_bwd(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, w.scale)
+    b = moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, w.scale)
+    for s, t in zip(a, b):
+        assert torch.equal(s, t)
+
+
+def test_grouped_sums_are_bit_reproducible():
+    B, T, H, Hk, d, l = 1, 640, 8, 2, 128, 6
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=9, device="cuda")
+    first = run(x, l, d ** -0.5)
+    for rep in range(10):
+        again = run(x, l, d ** -0.5)
+        assert torch.equal(first[0], again[0]) and torch.equal(first[1], again[1])
+        for name, s, t in zip(("dQ", "dK", "dV", "dKd", "dVd"), first[2], again[2]):
+            assert torch.equal(s, t), f"{name} changed on repeat {rep}"

@@ -150,10 +150,11 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
  * keys up to its base time and the depth keys stored at its base time.
  *     Q, O, dO, dQ : bf16 [B][T][H][d]          K, V, dK, dV : bf16 [B][T][H_kv][d]
  *     depth_kv, d_depth_kv : cache layout with H_kv heads (moda_depth_cache_bytes(B, T, H_kv, d, l))
- *     LSE : fp32 [B][H][T]                      workspace : moda_bwd_workspace_bytes(B, T, H, d, l)
- * dK, dV and the depth gradients are the sums over the G query heads of a group; the sum is
- * taken in a fixed order (no atomics), so results are bit-reproducible.  The depth gradients
- * are rounded to bf16 once per head of the group (G - 1 extra roundings).  H_kv must divide H
+ *     LSE : fp32 [B][H][T]                      workspace : moda_bwd_workspace_bytes_gqa(B, T, H, H_kv, d, l)
+ * dK, dV and the depth gradients are the sums over the G query heads of a group, taken in fp32 in
+ * a fixed order (no atomics), so results are bit-reproducible.  With G > 1 the workspace also
+ * holds two fp32 factors per (row, slot, query head), from which a second kernel forms the depth
+ * gradients without reading the depth cache again.  H_kv must divide H
  * and G <= MODA_MAX_GROUP (MODA_ERR_BAD_GROUP otherwise); H_kv == H is exactly
  * moda_attn_fwd / moda_attn_bwd.  Everything else (validation, streams, ownership, errors) is
  * as for those calls.
@@ -161,6 +162,7 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
 int moda_attn_fwd_gqa(const void* Q, const void* K, const void* V, const void* depth_kv,
                       int B, int T, int H, int H_kv, int d, int l, float scale,
                       void* O, float* LSE, void* stream);
+size_t moda_bwd_workspace_bytes_gqa(int B, int T, int H, int H_kv, int d, int l);
 int moda_attn_bwd_gqa(const void* Q, const void* K, const void* V, const void* depth_kv,
                       const void* O, const void* dO, const float* LSE,
                       int B, int T, int H, int H_kv, int d, int l, float scale,

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     moda_attn_fwd,
     moda_attn_fwd_gqa,
     moda_bwd_workspace_bytes,
+    moda_bwd_workspace_bytes_gqa,
     moda_depth_cache_append,
     moda_depth_cache_bytes,
     moda_depth_cache_unpack,

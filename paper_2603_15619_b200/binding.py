@@ -21,7 +21,7 @@ SYMBOLS = (
     "moda_depth_cache_bytes", "moda_depth_cache_append", "moda_depth_cache_unpack",
     "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd", "moda_attn_bwd_stages",
     "moda_attn_bwd_static_scratch",
-    "moda_attn_fwd_gqa", "moda_attn_bwd_gqa", "moda_attn_bwd_gqa_stages",
+    "moda_attn_fwd_gqa", "moda_bwd_workspace_bytes_gqa", "moda_attn_bwd_gqa", "moda_attn_bwd_gqa_stages",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -72,6 +72,8 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd_static_scratch.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 4 + [vp]
     lib.moda_attn_fwd_gqa.restype = ci
     lib.moda_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
+    lib.moda_bwd_workspace_bytes_gqa.restype = sz
+    lib.moda_bwd_workspace_bytes_gqa.argtypes = [ci] * 6
     lib.moda_attn_bwd_gqa.restype = ci
     lib.moda_attn_bwd_gqa.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
     lib.moda_attn_bwd_gqa_stages.restype = ci
@@ -216,6 +218,10 @@ def moda_attn_bwd_static_scratch(Q, K, V, depth_kv, O, dO, LSE, l, scale, dQ, dK
     return dQ, dK, dV, d_depth_kv
 
 
+def moda_bwd_workspace_bytes_gqa(B, T, H, H_kv, d, l) -> int:
+    return int(load().moda_bwd_workspace_bytes_gqa(B, T, H, H_kv, d, l))
+
+
 def _gqa_shapes(Q, K, V):
     B, T, H, d = _bthd(Q, "Q")
     Bk, Tk, Hk, dk = _bthd(K, "K")
@@ -251,7 +257,7 @@ def moda_attn_bwd_gqa(Q, K, V, depth_kv, O, dO, LSE, l, scale,
     if l > 0 and d_depth_kv is None:
         d_depth_kv = alloc_depth_cache(B, T, Hk, d, l, Q.device)
     if workspace is None:
-        workspace = torch.empty(moda_bwd_workspace_bytes(B, T, H, d, l), dtype=torch.uint8, device=Q.device)
+        workspace = torch.empty(moda_bwd_workspace_bytes_gqa(B, T, H, Hk, d, l), dtype=torch.uint8, device=Q.device)
     args = [_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
             _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, Hk, d, int(l), float(scale),
             _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,

@@ -164,26 +164,42 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
         bwd_delta_kernel<D><<<grid, 256, 0, stream>>>(static_cast<const uint4*>(a.O), static_cast<const uint4*>(a.dO), delta, B, T, H);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     }
-    // one CTA per (batch, key/value head, 128-row tile)
-    const unsigned grid = unsigned(B) * Hk * num_tiles(T);
     if (stages & 2) {
+        // one CTA per (batch, query head, 128-row tile)
+        const unsigned grid = unsigned(B) * H * num_tiles(T);
         DqParams p;
         p.depth_kv = static_cast<const __nv_bfloat16*>(a.depth_kv);
         p.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
         p.LSE = a.LSE; p.delta = delta;
         p.B = B; p.T = T; p.H = H; p.l = a.l; p.G = G;
         p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
-        // One launch per member g of the groups: launch g handles query head hk G + g of every
-        // key/value head and adds its depth gradients to those of the launches before it.
-        for (int g = 0; g < G; ++g) {
-            p.g = g;
-            if (dq_depth_heavy(T, a.l, D))
-                moda_bwd_dq_kernel<128, 2><<<grid, kBwdDqThreads, DqSmem<128, 2>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
-            else
-                moda_bwd_dq_kernel<D, 3><<<grid, kBwdDqThreads, DqSmem<D, 3>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
+        // Grouped-query: the dQ kernel leaves R_i, dU_i per (row, slot, head) behind the row terms D_t
+        // and a second, write-bound kernel forms the depth gradients as sums over each group.
+        float* rowterms = reinterpret_cast<float*>(static_cast<char*>(a.workspace) + bwd_workspace_bytes(B, T, H));
+        p.depth_rowterms = (G > 1 && a.l > 0) ? rowterms : nullptr;
+        if (dq_depth_heavy(T, a.l, D))
+            moda_bwd_dq_kernel<128, 2><<<grid, kBwdDqThreads, DqSmem<128, 2>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
+        else
+            moda_bwd_dq_kernel<D, 3><<<grid, kBwdDqThreads, DqSmem<D, 3>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
+        if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+        if (G > 1 && a.l > 0) {
+            const unsigned g2 = unsigned(B) * Hk * num_tiles(T) * 2;
+            const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.Q);
+            const __nv_bfloat16* go = static_cast<const __nv_bfloat16*>(a.dO);
+            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.d_depth_kv);
+#define MODA_GROUP_CASE(GG) \
+            case GG: depth_grad_group_kernel<D, GG><<<g2, 256, 0, stream>>>(q, go, rowterms, out, B, T, Hk, a.l, a.scale); break;
+            switch (G) {
+                MODA_GROUP_CASE(2) MODA_GROUP_CASE(3) MODA_GROUP_CASE(4) MODA_GROUP_CASE(5)
+                MODA_GROUP_CASE(6) MODA_GROUP_CASE(7) MODA_GROUP_CASE(8)
+                default: return MODA_ERR_BAD_GROUP;
+            }
+#undef MODA_GROUP_CASE
             if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
         }
     }
+    // dK, dV: one CTA per (batch, key/value head, 128-row tile)
+    const unsigned grid = unsigned(B) * Hk * num_tiles(T);
     if (stages & 4) {
         DkvParams p;
         p.LSE = a.LSE; p.delta = delta;
@@ -297,6 +313,11 @@ size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l) {
     return bwd_workspace_bytes(B, T, H);
 }
 
+size_t moda_bwd_workspace_bytes_gqa(int B, int T, int H, int H_kv, int d, int l) {
+    if (check_shape(B, T, H, d) != MODA_OK || check_groups(H, H_kv) != MODA_OK || l < 0 || l > MODA_MAX_DEPTH) return 0;
+    return bwd_workspace_bytes_gqa(B, T, H, H_kv, l);
+}
+
 int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth_kv,
                   const void* O, const void* dO, const float* LSE,
                   int B, int T, int H, int d, int l, float scale,
@@ -339,7 +360,7 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
         !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) ||
         (l > 0 && (!aligned16(depth_kv) || !aligned16(d_depth_kv))))
         return MODA_ERR_MISALIGNED;
-    if (!workspace || !aligned16(workspace) || workspace_bytes < bwd_workspace_bytes(B, T, H)) return MODA_ERR_WORKSPACE;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < bwd_workspace_bytes_gqa(B, T, H, H_kv, l)) return MODA_ERR_WORKSPACE;
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     BwdArgs a;

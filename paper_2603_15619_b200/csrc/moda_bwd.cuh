@@ -36,6 +36,12 @@ struct BwdArgs {
 inline size_t bwd_workspace_bytes(int B, int T, int H) {
     return (size_t(B) * H * T * 4 + 15) & ~size_t(15);
 }
+// Grouped-query backward: the row terms D_t, then R_i and dU_i of every (row, slot, head).
+inline size_t bwd_workspace_bytes_gqa(int B, int T, int H, int Hk, int l) {
+    const size_t base = bwd_workspace_bytes(B, T, H);
+    if (H == Hk) return base;
+    return base + size_t(B) * Hk * num_tiles(T) * l * 2 * kTileRows * (H / Hk) * 4;
+}
 
 __device__ __forceinline__ float dot8_bf16(const uint4& a, const uint4& b) {
     float acc = bf16_lo_to_f32(a.x) * bf16_lo_to_f32(b.x);
@@ -136,19 +142,12 @@ struct DqParams {
     const float* delta;
     int B, T, H, l;     // H = number of query heads
     int G;              // query heads per key/value head
-    int g;              // this launch handles query head hk G + g of every key/value head hk
+    // G == 1: the depth gradients are written by this kernel (null here).  G > 1: they are sums
+    // over the heads of a group, so the kernel only leaves its per-row factors here, R_i and dU_i
+    // as [b][hk][tile][slot][{R, dU}][row 128][g] fp32, and depth_grad_group_kernel forms the sums.
+    float* depth_rowterms;
     float scale, scale_log2;
 };
-
-// Sum of two groups of 8 bf16, added in fp32 and rounded once.
-__device__ __forceinline__ uint4 add_bf16x8(const uint4& a, const uint4& b) {
-    uint4 r;
-    r.x = pack_bf16x2(bf16_lo_to_f32(a.x) + bf16_lo_to_f32(b.x), bf16_hi_to_f32(a.x) + bf16_hi_to_f32(b.x));
-    r.y = pack_bf16x2(bf16_lo_to_f32(a.y) + bf16_lo_to_f32(b.y), bf16_hi_to_f32(a.y) + bf16_hi_to_f32(b.y));
-    r.z = pack_bf16x2(bf16_lo_to_f32(a.z) + bf16_lo_to_f32(b.z), bf16_hi_to_f32(a.z) + bf16_hi_to_f32(b.z));
-    r.w = pack_bf16x2(bf16_lo_to_f32(a.w) + bf16_lo_to_f32(b.w), bf16_hi_to_f32(a.w) + bf16_hi_to_f32(b.w));
-    return r;
-}
 
 // bf16x2 product with both factors already packed.
 __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
@@ -181,11 +180,9 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nq = num_tiles(p.T);
-    const int bh = blockIdx.x / nq;
-    const int qt = nq - 1 - (blockIdx.x % nq);
+    const TileCoord tc = tile_coord(blockIdx.x, nq, p.H, p.G);   // the heads of a group are adjacent CTAs
+    const int b = tc.b, h = tc.h, hk = tc.hk, qt = tc.qt;
     const int Hk = p.H / p.G;
-    const int b = bh / Hk, hk = bh % Hk;             // key/value head
-    const int h = hk * p.G + p.g;                    // query head
     const int q0 = qt * kTileRows;
     const int n_kv = min(2 * (qt + 1), (p.T + kKeyTile - 1) / kKeyTile);   // 64-key tiles at or below the diagonal
 
@@ -318,10 +315,11 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             const float delta = valid ? p.delta[row_idx] : 0.f;
             const size_t slot_stride = cache_slot_elems(p.B, p.T, Hk, D) / 8;           // in uint4
             const size_t blk = (((size_t(b) * Hk + hk) * nq + qt) * 2) * (kTileRows * CH) + r;
-            // The depth gradients are sums over the G query heads of a group: the launch for g = 0
-            // writes them, every later launch of the same backward adds its share to what is there
-            // (same thread, same addresses; launches are ordered by the stream).
-            const bool add_to = p.g > 0;
+            // Grouped-query launches leave R_i and dU_i of this row for depth_grad_group_kernel
+            // instead of writing depth gradients (which are sums over the heads of the group).
+            const bool store_grads = p.depth_rowterms == nullptr;
+            float* rt_row = store_grads ? nullptr
+                : p.depth_rowterms + (((size_t(b) * Hk + hk) * nq + qt) * p.l * 2) * (kTileRows * p.G) + r * p.G + (h - hk * p.G);
             uint4* gK = reinterpret_cast<uint4*>(p.d_depth_kv) + blk;
             uint4* gV = gK + kTileRows * CH;
             mbar_wait(bar(kDqBarQ), 0, abort_flag, 60);
@@ -399,23 +397,31 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                         const float part = dot64(g, cur);
                         if (half == 0) sDr[ii * kTileRows + r] = part;
                         else sDr[ii * kTileRows + r] += part;
-                        const float w = sU[ii * kTileRows + r];
-                        uint4* dst = gV + size_t(g0 + ii) * slot_stride + (half * 8) * kTileRows;
+                        if (store_grads) {
+                            const float w = sU[ii * kTileRows + r];
+                            uint4* dst = gV + size_t(g0 + ii) * slot_stride + (half * 8) * kTileRows;
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            uint4 o;
-                            o.x = pack_bf16x2(w * g[8 * c + 0], w * g[8 * c + 1]);
-                            o.y = pack_bf16x2(w * g[8 * c + 2], w * g[8 * c + 3]);
-                            o.z = pack_bf16x2(w * g[8 * c + 4], w * g[8 * c + 5]);
-                            o.w = pack_bf16x2(w * g[8 * c + 6], w * g[8 * c + 7]);
-                            if (add_to) o = add_bf16x8(o, dst[c * kTileRows]);
-                            dst[c * kTileRows] = o;
+                            for (int c = 0; c < 8; ++c) {
+                                uint4 o;
+                                o.x = pack_bf16x2(w * g[8 * c + 0], w * g[8 * c + 1]);
+                                o.y = pack_bf16x2(w * g[8 * c + 2], w * g[8 * c + 3]);
+                                o.z = pack_bf16x2(w * g[8 * c + 4], w * g[8 * c + 5]);
+                                o.w = pack_bf16x2(w * g[8 * c + 6], w * g[8 * c + 7]);
+                                dst[c * kTileRows] = o;
+                            }
                         }
                     }
                 }
                 // dU_i = R_i (<dO, vd_i> - D)
                 for (int ii = 0; ii < gl; ++ii)
                     sDr[ii * kTileRows + r] = sU[ii * kTileRows + r] * (sDr[ii * kTileRows + r] - delta);
+                if (!store_grads) {
+                    for (int ii = 0; ii < gl; ++ii) {
+                        float* dst = rt_row + size_t(g0 + ii) * 2 * (kTileRows * p.G);
+                        dst[0] = sU[ii * kTileRows + r];
+                        dst[kTileRows * p.G] = sDr[ii * kTileRows + r];
+                    }
+                }
 
                 // ---- pass C: dQ share sum_i dU_i kd_i (accumulated in TMEM across groups), dKd_i = scale dU_i q ----
 #pragma unroll 1
@@ -461,8 +467,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                             o.y = mul_bf16x2(qp[c].y, sdu2);
                             o.z = mul_bf16x2(qp[c].z, sdu2);
                             o.w = mul_bf16x2(qp[c].w, sdu2);
-                            if (add_to) o = add_bf16x8(o, dst[c * kTileRows]);
-                            dst[c * kTileRows] = o;
+                            if (store_grads) dst[c * kTileRows] = o;
                         }
                     }
 #pragma unroll
@@ -602,6 +607,62 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     }
     __syncthreads();
     if (warp == 16) tmem_dealloc(tmem, kTmemCols);
+}
+
+// =====================================================================================
+// Depth gradients of a grouped-query backward
+// =====================================================================================
+// dKd_i[t] = scale sum_g dU_i^g[t] q^g[t] and dVd_i[t] = sum_g R_i^g[t] dO^g[t] over the G query heads
+// of a key/value head, from the factors the dQ kernel left in the workspace.  Row-local and bound by
+// the one write of the depth gradients: no depth cache is read.  One CTA per (b, hk, 128-row tile,
+// dKd or dVd); a thread keeps one 8-feature chunk of the G rows (q^g or dO^g) in registers and walks
+// the slots, writing 16 bytes per slot in cache layout (consecutive lanes = consecutive rows).
+template <int D, int G>
+__global__ void __launch_bounds__(256)
+depth_grad_group_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ dO,
+                        const float* __restrict__ rowterms, __nv_bfloat16* __restrict__ d_depth_kv,
+                        int B, int T, int Hk, int l, float scale) {
+    constexpr int CH = D / 8;
+    const int nq = num_tiles(T);
+    const int kv = blockIdx.x & 1;                       // 0: dKd (dU, q, scaled), 1: dVd (R, dO)
+    const int tile_id = blockIdx.x >> 1;                 // (b * Hk + hk) * nq + qt
+    const int qt = tile_id % nq;
+    const int bhk = tile_id / nq;
+    const int b = bhk / Hk, hk = bhk % Hk;
+    const int r = threadIdx.x & 127;
+    const int t = qt * kTileRows + r;
+    const bool valid = t < T;
+    const int H = Hk * G;
+    const __nv_bfloat16* X = kv == 0 ? Q : dO;
+    const float mul = kv == 0 ? scale : 1.f;
+    const float* coef = rowterms + (size_t(tile_id) * l * 2 + (kv == 0 ? 1 : 0)) * (kTileRows * G) + r * G;
+    const size_t slot_stride = cache_slot_elems(B, T, Hk, D) / 8;                    // in uint4
+    uint4* out = reinterpret_cast<uint4*>(d_depth_kv) + (size_t(tile_id) * 2 + kv) * (kTileRows * CH) + r;
+    for (int c = threadIdx.x >> 7; c < CH; c += 2) {
+        float x[G][8];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (valid) v = *reinterpret_cast<const uint4*>(X + ((size_t(b) * T + t) * H + hk * G + g) * D + c * 8);
+            x[g][0] = bf16_lo_to_f32(v.x) * mul; x[g][1] = bf16_hi_to_f32(v.x) * mul;
+            x[g][2] = bf16_lo_to_f32(v.y) * mul; x[g][3] = bf16_hi_to_f32(v.y) * mul;
+            x[g][4] = bf16_lo_to_f32(v.z) * mul; x[g][5] = bf16_hi_to_f32(v.z) * mul;
+            x[g][6] = bf16_lo_to_f32(v.w) * mul; x[g][7] = bf16_hi_to_f32(v.w) * mul;
+        }
+        for (int i = 0; i < l; ++i) {
+            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const float w = coef[size_t(i) * 2 * (kTileRows * G) + g];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) a[k] = fmaf(w, x[g][k], a[k]);
+            }
+            uint4 o;
+            o.x = pack_bf16x2(a[0], a[1]); o.y = pack_bf16x2(a[2], a[3]);
+            o.z = pack_bf16x2(a[4], a[5]); o.w = pack_bf16x2(a[6], a[7]);
+            out[size_t(i) * slot_stride + c * kTileRows] = o;      // rows past T carry x = 0: the tail stays zero
+        }
+    }
 }
 
 // =====================================================================================

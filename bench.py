@@ -286,6 +286,7 @@ def run_moda(args, rank, world, device):
 
     if rank == 0 and world == 1 and not args.no_sweep:
         out["sweep"] = run_sweep(peaks, device, layer)
+        out["gqa_sweep"] = run_gqa_sweep(device)
     if not args.no_e2e:
         out["e2e"] = run_e2e(layer, min(K, 8), world, step_flops, device)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -342,6 +343,55 @@ def run_sweep(peaks, device, first_layer):
             "fwd_ratio_to_l0": round(f0 / f_ms, 4), "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f_ms + b_ms), 4),
         })
         log("sweep", rows[-1])
+    torch.cuda.empty_cache()
+    return rows
+
+
+# Shapes of the paper's kernel table (Table 2: B = 1, d = 64, 8 key/value heads, G query heads per
+# key/value head; sweeps over T at G = 8 and over G at T = 16384).  The table uses L = 64 depth slots;
+# this library holds at most 32, so the rows below are measured at l = 32.
+GQA_SHAPES = [(4096, 8), (8192, 8), (16384, 8), (32768, 8), (65536, 8), (16384, 2), (16384, 4)]
+
+
+def run_gqa_sweep(device):
+    """Grouped-query forward + backward at the paper's Table 2 shapes, with the l = 0 twin."""
+    import paper_2603_15619_b200 as moda
+    rows = []
+    B, d, Hk, l_full = 1, 64, 8, 32
+    for T, G in GQA_SHAPES:
+        H = Hk * G
+        res = {}
+        for l in (0, l_full):
+            torch.cuda.empty_cache()
+            x = synthetic.make_gqa(B, T, H, Hk, d, 0, seed=0, device=device)
+            cache = dcache = None
+            if l > 0:
+                wk = synthetic.Workload("gqa/kv", B, T, Hk, d, l)
+                cache = moda.alloc_depth_cache(B, T, Hk, d, l, device)
+                dcache = moda.alloc_depth_cache(B, T, Hk, d, l, device)
+                for i in range(l):
+                    moda.moda_depth_cache_append(cache, i, synthetic.tensor(wk, "Kd", 0, i, device),
+                                                 synthetic.tensor(wk, "Vd", 0, i, device))
+            O = torch.empty_like(x["Q"])
+            LSE = torch.empty((B, H, T), dtype=torch.float32, device=device)
+            dQ, dK, dV = torch.empty_like(x["Q"]), torch.empty_like(x["K"]), torch.empty_like(x["V"])
+            ws = torch.empty(moda.moda_bwd_workspace_bytes_gqa(B, T, H, Hk, d, l), dtype=torch.uint8, device=device)
+            scale = d ** -0.5
+            fwd = lambda: moda.moda_attn_fwd_gqa(x["Q"], x["K"], x["V"], cache, l, scale, O=O, LSE=LSE)
+            bwd = lambda: moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale,
+                                                 dQ=dQ, dK=dK, dV=dV, d_depth_kv=dcache, workspace=ws)
+            iters = 2 if T >= 32768 else 5
+            res[l] = (time_calls(fwd, iters), time_calls(bwd, iters))
+            del x, cache, dcache, O, LSE, dQ, dK, dV, ws
+        (f0, b0), (f1, b1) = res[0], res[l_full]
+        ff = 4.0 * B * H * d * (T * (T + 1) / 2) + 4.0 * B * H * T * l_full * d
+        rows.append({"B": B, "T": T, "H": H, "H_kv": Hk, "G": G, "d": d, "l": l_full,
+                     "fwd_ms": round(f1, 4), "bwd_ms": round(b1, 4), "fwd_bwd_ms": round(f1 + b1, 4),
+                     "l0_fwd_bwd_ms": round(f0 + b0, 4),
+                     "extra_time_pct": round(100.0 * ((f1 + b1) / (f0 + b0) - 1.0), 2),
+                     "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f1 + b1), 4),
+                     "fwd_tflops": round(ff / f1 / 1e9, 1), "fwd_bwd_tflops": round(3.5 * ff / (f1 + b1) / 1e9, 1)})
+        log("gqa_sweep", rows[-1])
     torch.cuda.empty_cache()
     return rows
 

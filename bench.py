@@ -120,6 +120,27 @@ def ev():
     return torch.cuda.Event(enable_timing=True)
 
 
+# ---- multi-GPU plumbing: ranks work on independent shards (no collective on the data path) ----
+def shard_seed(rank: int) -> int:
+    """Seed of the synthetic shard that rank `rank` generates and processes (weak scaling: every
+    rank holds one full per-GPU workload of its own)."""
+    return int(rank)
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Slowest rank's time: the job advances at the pace of its slowest shard."""
+    if world <= 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, flops_per_rank_step: float, ms_per_step: float) -> float:
+    """Whole-job TFLOP/s: every rank does `flops_per_rank_step` per step, in `ms_per_step`."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
 class Layer:
     """Device buffers of one workload plus the calls of one step."""
 
@@ -199,7 +220,7 @@ def run_moda(args, rank, world, device):
     import paper_2603_15619_b200 as moda
     peaks = load_peaks()
     w = pick_workload(args)
-    layer = Layer(w, seed=rank, device=device)
+    layer = Layer(w, seed=shard_seed(rank), device=device)
 
     def barrier():
         if world > 1:
@@ -227,10 +248,7 @@ def run_moda(args, rank, world, device):
     clocks = sampler.stop(t_begin, t_end)
     total_ms = evs[0][0].elapsed_time(evs[-1][5])
     ms_per_step = total_ms / K
-    if world > 1:
-        t = torch.tensor([ms_per_step], device=device)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms_per_step = float(t.item())
+    ms_per_step = max_over_ranks(ms_per_step, world, device)
     status = moda.moda_last_status()
     if status != 0:
         raise RuntimeError(f"device status {status} after the timed region")
@@ -239,7 +257,7 @@ def run_moda(args, rank, world, device):
     for i, name in enumerate(Layer.KERNELS):
         per_kernel[name] = sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K
     step_flops = flops.fwd_bwd_flops(w.B, w.T, w.H, w.d, w.l)
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = job_value(world, step_flops, ms_per_step)
 
     # ---- roofline of the dominant kernel ----
     model = layer.kernel_model()
@@ -443,12 +461,9 @@ def run_e2e(layer, steps, world, step_flops, device):
     b.record(s_out)
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / steps
-    if world > 1:
-        t = torch.tensor([ms], device=device)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, device)
     nbytes = lambda ts: int(sum(t.numel() * t.element_size() for t in ts))
-    return {"value": round(world * step_flops / (ms * 1e-3) / 1e12, 3), "unit": UNIT, "ms_per_step": round(ms, 3),
+    return {"value": round(job_value(world, step_flops, ms), 3), "unit": UNIT, "ms_per_step": round(ms, 3),
             "steps": steps, "h2d_bytes_per_step": nbytes(ins[0]), "d2h_bytes_per_step": nbytes(outs[0]),
             "overlap": "upload of step i+1 and download of step i-1 run beside the kernels of step i (2 buffer sets, 3 streams)"}
 

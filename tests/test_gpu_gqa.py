@@ -88,3 +88,26 @@ def test_grouped_sums_are_bit_reproducible():
         assert torch.equal(first[0], again[0]) and torch.equal(first[1], again[1])
         for name, s, t in zip(("dQ", "dK", "dV", "dKd", "dVd"), first[2], again[2]):
             assert torch.equal(s, t), f"{name} changed on repeat {rep}"
+
+
+def test_paper_table2_shape_one_group_against_the_oracle():
+    # The shape family of the paper's kernel table (B = 1, d = 64, 8 key/value heads, G = 8) at
+    # T = 8192, l = 32, on the GPU in full; key/value groups are independent, so the oracle checks
+    # one whole group (8 query heads on key/value head 3) as a problem of its own.
+    B, T, H, Hk, d, l = 1, 8192, 64, 8, 64, 32
+    G, hk = H // Hk, 3
+    scale = d ** -0.5
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=2, device="cuda", k_head_norm=True)
+    O, LSE, grads = run(x, l, scale)
+    qs = slice(hk * G, (hk + 1) * G)
+    xs = [f64(x["Q"][:, :, qs]), f64(x["K"][:, :, hk:hk + 1]), f64(x["V"][:, :, hk:hk + 1]),
+          f64(x["Kd"][:, :, :, hk:hk + 1]), f64(x["Vd"][:, :, :, hk:hk + 1])]
+    O_ref, LSE_ref = orc.forward_gqa(*xs, scale)
+    assert rel_l2(f64(O[:, :, qs]), O_ref) <= TOL_O_REL_L2
+    assert float(np.abs(f64(O[:, :, qs]) - O_ref).max()) <= TOL_O_MAX_ABS
+    assert float(np.abs(f64(LSE[:, qs]) - LSE_ref).max()) <= TOL_LSE_ABS
+    ref = orc.backward_gqa(*xs, f64(x["dO"][:, :, qs]), scale)
+    dQ, dK, dV, dKd, dVd = grads
+    got = (dQ[:, :, qs], dK[:, :, hk:hk + 1], dV[:, :, hk:hk + 1], dKd[:, :, :, hk:hk + 1], dVd[:, :, :, hk:hk + 1])
+    for name, g, r in zip(("dQ", "dK", "dV", "dKd", "dVd"), got, ref):
+        assert grad_err(g, r) <= TOL_GRAD_REL_L2, f"{name}: {grad_err(g, r):.3e}"

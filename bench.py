@@ -371,12 +371,12 @@ def run_sweep(peaks, device, first_layer):
 GQA_SHAPES = [(4096, 8), (8192, 8), (16384, 8), (32768, 8), (65536, 8), (16384, 2), (16384, 4)]
 
 
-def run_gqa_sweep(device):
+def run_gqa_sweep(device, shapes=None):
     """Grouped-query forward + backward at the paper's Table 2 shapes, with the l = 0 twin."""
     import paper_2603_15619_b200 as moda
     rows = []
     B, d, Hk, l_full = 1, 64, 8, 32
-    for T, G in GQA_SHAPES:
+    for T, G in (shapes or GQA_SHAPES):
         H = Hk * G
         res = {}
         for l in (0, l_full):
@@ -548,6 +548,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gqa-shape", default="", help="T,G: time only this grouped-query shape (B=1, d=64, 8 key/value "
+                                                    "heads, l=32 and l=0) and print its row; for profiling")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -568,7 +570,11 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         torch.distributed.init_process_group("nccl", device_id=device)
     try:
-        out = run_moda(args, rank, world, device)
+        if args.gqa_shape:
+            T, G = (int(v) for v in args.gqa_shape.split(","))
+            out = {"gqa_sweep": run_gqa_sweep(device, [(T, G)])}
+        else:
+            out = run_moda(args, rank, world, device)
         if rank == 0:
             print(json.dumps(out), flush=True)
     finally:

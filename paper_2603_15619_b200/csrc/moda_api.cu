@@ -183,12 +183,12 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
             moda_bwd_dq_kernel<D, 3><<<grid, kBwdDqThreads, DqSmem<D, 3>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
         if (G > 1 && a.l > 0) {
-            const unsigned g2 = unsigned(B) * Hk * num_tiles(T) * 2;
+            const unsigned g2 = unsigned(B) * Hk * num_tiles(T) * 2 * (D / 32);   // x {dKd, dVd} x groups of 4 chunks
             const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.Q);
             const __nv_bfloat16* go = static_cast<const __nv_bfloat16*>(a.dO);
             __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.d_depth_kv);
 #define MODA_GROUP_CASE(GG) \
-            case GG: depth_grad_group_kernel<D, GG><<<g2, 256, 0, stream>>>(q, go, rowterms, out, B, T, Hk, a.l, a.scale); break;
+            case GG: depth_grad_group_kernel<D, GG><<<g2, kGroupGradThreads, 0, stream>>>(q, go, rowterms, out, B, T, Hk, a.l, a.scale); break;
             switch (G) {
                 MODA_GROUP_CASE(2) MODA_GROUP_CASE(3) MODA_GROUP_CASE(4) MODA_GROUP_CASE(5)
                 MODA_GROUP_CASE(6) MODA_GROUP_CASE(7) MODA_GROUP_CASE(8)

@@ -615,52 +615,68 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
 // dKd_i[t] = scale sum_g dU_i^g[t] q^g[t] and dVd_i[t] = sum_g R_i^g[t] dO^g[t] over the G query heads
 // of a key/value head, from the factors the dQ kernel left in the workspace.  Row-local and bound by
 // the one write of the depth gradients: no depth cache is read.  One CTA per (b, hk, 128-row tile,
-// dKd or dVd); a thread keeps one 8-feature chunk of the G rows (q^g or dO^g) in registers and walks
-// the slots, writing 16 bytes per slot in cache layout (consecutive lanes = consecutive rows).
+// dKd or dVd, group of 4 feature chunks); a thread keeps one 8-feature chunk of the G rows (q^g or
+// dO^g) in registers and walks the slots, writing 16 bytes per slot in cache layout (consecutive
+// lanes = consecutive rows).  The factors of 8 slots at a time are staged in shared memory (every
+// thread of a row needs the same G factors per slot).
+constexpr int kGroupGradThreads = 512;
+constexpr int kGroupGradSlots = 8;
+
 template <int D, int G>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kGroupGradThreads)
 depth_grad_group_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ dO,
                         const float* __restrict__ rowterms, __nv_bfloat16* __restrict__ d_depth_kv,
                         int B, int T, int Hk, int l, float scale) {
     constexpr int CH = D / 8;
+    constexpr int CGROUPS = CH / 4;                      // chunk groups per tile: 2 (d = 64) or 4 (d = 128)
+    __shared__ __align__(16) float s_coef[kGroupGradSlots * kTileRows * G];
     const int nq = num_tiles(T);
-    const int kv = blockIdx.x & 1;                       // 0: dKd (dU, q, scaled), 1: dVd (R, dO)
-    const int tile_id = blockIdx.x >> 1;                 // (b * Hk + hk) * nq + qt
+    const int cgrp = blockIdx.x % CGROUPS;
+    const int kv = (blockIdx.x / CGROUPS) & 1;           // 0: dKd (dU, q, scaled), 1: dVd (R, dO)
+    const int tile_id = blockIdx.x / (2 * CGROUPS);      // (b * Hk + hk) * nq + qt
     const int qt = tile_id % nq;
     const int bhk = tile_id / nq;
     const int b = bhk / Hk, hk = bhk % Hk;
     const int r = threadIdx.x & 127;
+    const int c = cgrp * 4 + (threadIdx.x >> 7);
     const int t = qt * kTileRows + r;
-    const bool valid = t < T;
     const int H = Hk * G;
     const __nv_bfloat16* X = kv == 0 ? Q : dO;
     const float mul = kv == 0 ? scale : 1.f;
-    const float* coef = rowterms + (size_t(tile_id) * l * 2 + (kv == 0 ? 1 : 0)) * (kTileRows * G) + r * G;
-    const size_t slot_stride = cache_slot_elems(B, T, Hk, D) / 8;                    // in uint4
-    uint4* out = reinterpret_cast<uint4*>(d_depth_kv) + (size_t(tile_id) * 2 + kv) * (kTileRows * CH) + r;
-    for (int c = threadIdx.x >> 7; c < CH; c += 2) {
-        float x[G][8];
+    float x[G][8];
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (valid) v = *reinterpret_cast<const uint4*>(X + ((size_t(b) * T + t) * H + hk * G + g) * D + c * 8);
-            x[g][0] = bf16_lo_to_f32(v.x) * mul; x[g][1] = bf16_hi_to_f32(v.x) * mul;
-            x[g][2] = bf16_lo_to_f32(v.y) * mul; x[g][3] = bf16_hi_to_f32(v.y) * mul;
-            x[g][4] = bf16_lo_to_f32(v.z) * mul; x[g][5] = bf16_hi_to_f32(v.z) * mul;
-            x[g][6] = bf16_lo_to_f32(v.w) * mul; x[g][7] = bf16_hi_to_f32(v.w) * mul;
+    for (int g = 0; g < G; ++g) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);            // rows past T contribute zeros: the tail stays zero
+        if (t < T) v = *reinterpret_cast<const uint4*>(X + ((size_t(b) * T + t) * H + hk * G + g) * D + c * 8);
+        x[g][0] = bf16_lo_to_f32(v.x) * mul; x[g][1] = bf16_hi_to_f32(v.x) * mul;
+        x[g][2] = bf16_lo_to_f32(v.y) * mul; x[g][3] = bf16_hi_to_f32(v.y) * mul;
+        x[g][4] = bf16_lo_to_f32(v.z) * mul; x[g][5] = bf16_hi_to_f32(v.z) * mul;
+        x[g][6] = bf16_lo_to_f32(v.w) * mul; x[g][7] = bf16_hi_to_f32(v.w) * mul;
+    }
+    // factors of this tile: [slot][{R, dU}][row 128][g]; dKd uses dU, dVd uses R
+    const float* coef = rowterms + (size_t(tile_id) * l * 2 + (kv == 0 ? 1 : 0)) * (kTileRows * G);
+    const size_t slot_stride = cache_slot_elems(B, T, Hk, D) / 8;                    // in uint4
+    uint4* out = reinterpret_cast<uint4*>(d_depth_kv) + (size_t(tile_id) * 2 + kv) * (kTileRows * CH) + c * kTileRows + r;
+    for (int i0 = 0; i0 < l; i0 += kGroupGradSlots) {
+        const int n = min(kGroupGradSlots, l - i0);
+        __syncthreads();
+        for (int e = threadIdx.x; e < n * kTileRows * G; e += kGroupGradThreads) {
+            const int i = e / (kTileRows * G);
+            s_coef[e] = coef[size_t(i0 + i) * 2 * (kTileRows * G) + (e - i * (kTileRows * G))];
         }
-        for (int i = 0; i < l; ++i) {
+        __syncthreads();
+        for (int i = 0; i < n; ++i) {
             float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                const float w = coef[size_t(i) * 2 * (kTileRows * G) + g];
+                const float w = s_coef[(i * kTileRows + r) * G + g];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) a[k] = fmaf(w, x[g][k], a[k]);
             }
             uint4 o;
             o.x = pack_bf16x2(a[0], a[1]); o.y = pack_bf16x2(a[2], a[3]);
             o.z = pack_bf16x2(a[4], a[5]); o.w = pack_bf16x2(a[6], a[7]);
-            out[size_t(i) * slot_stride + c * kTileRows] = o;      // rows past T carry x = 0: the tail stays zero
+            out[size_t(i0 + i) * slot_stride] = o;
         }
     }
 }

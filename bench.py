@@ -350,6 +350,11 @@ def run_sweep(peaks, device, first_layer):
         f_ms, b_ms = res["moda"]
         f0, b0 = res["l0"]
         ff = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l)
+        # roofline of the call: the slower of (algorithmic HBM bytes / measured copy rate) and
+        # (credited FLOPs / measured cuBLAS bf16 rate; the burst figure, these kernels run alone)
+        roof = lambda fl, by: max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e3
+        roof_f = roof(ff, flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l))
+        roof_b = roof(2.5 * ff, flops.bwd_bytes(w.B, w.T, w.H, w.d, w.l))
         rows.append({
             "workload": name, "B": w.B, "T": w.T, "H": w.H, "d": w.d, "l": w.l,
             "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
@@ -357,6 +362,9 @@ def run_sweep(peaks, device, first_layer):
             "fwd_frac_measured_burst": round(ff / f_ms / 1e9 / peaks["bf16_tflops"], 4),
             "fwd_frac_nominal": round(ff / f_ms / 1e9 / NOMINAL_BF16_TFLOPS, 4),
             "fwd_depth_read_gbs": round(flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / f_ms / 1e6, 1),
+            "fwd_frac_of_roofline": round(roof_f / f_ms, 4), "bwd_frac_of_roofline": round(roof_b / b_ms, 4),
+            "fwd_bound": "hbm" if flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l) / (peaks["hbm_gbs"] * 1e9) >
+                         ff / (peaks["bf16_tflops"] * 1e12) else "tensor",
             "l0_fwd_ms": round(f0, 4), "l0_bwd_ms": round(b0, 4),
             "fwd_ratio_to_l0": round(f0 / f_ms, 4), "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f_ms + b_ms), 4),
         })

@@ -4,6 +4,7 @@
 ``synthetic`` holds the seeded input recipes; ``flops`` the FLOP / byte accounting of the
 reported metric.  The CUDA library is loaded on first use and there is no fallback path.
 """
+from .autograd import moda_attention  # noqa: F401
 from .binding import (  # noqa: F401
     ModaError,
     alloc_depth_cache,

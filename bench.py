@@ -373,21 +373,28 @@ def run_sweep(peaks, device, first_layer):
     return rows
 
 
-# Shapes of the paper's kernel table (Table 2: B = 1, d = 64, 8 key/value heads, G query heads per
-# key/value head; sweeps over T at G = 8 and over G at T = 16384).  The table uses L = 64 depth slots;
-# this library holds at most 32, so the rows below are measured at l = 32.
-GQA_SHAPES = [(4096, 8), (8192, 8), (16384, 8), (32768, 8), (65536, 8), (16384, 2), (16384, 4)]
+# Rows of the paper's kernel table (Table 2: B = 1, d = 64, 8 key/value heads, G query heads per
+# key/value head, L depth slots; sweeps over T, over G and over L) as (T, G, L, extra time of MoDA
+# over the depth-free kernel that the table prints for an A100 with Triton kernels, in percent --
+# context, not a target).  The table's G = 16 and G = 32 rows exceed MODA_MAX_GROUP and are left out.
+GQA_SHAPES = [(4096, 8, 64, 25.86), (8192, 8, 64, 18.99), (16384, 8, 64, 8.59), (32768, 8, 64, 4.38),
+              (65536, 8, 64, 2.73), (16384, 2, 64, 27.07), (16384, 4, 64, 15.76),
+              (16384, 8, 128, 15.57), (16384, 8, 256, 30.52)]
 
 
 def run_gqa_sweep(device, shapes=None):
     """Grouped-query forward + backward at the paper's Table 2 shapes, with the l = 0 twin."""
     import paper_2603_15619_b200 as moda
     rows = []
-    B, d, Hk, l_full = 1, 64, 8, 32
-    for T, G in (shapes or GQA_SHAPES):
+    B, d, Hk = 1, 64, 8
+    base_cache = {}
+    for T, G, l_full, paper_pct in (shapes or GQA_SHAPES):
         H = Hk * G
         res = {}
         for l in (0, l_full):
+            if l == 0 and (T, G) in base_cache:
+                res[0] = base_cache[(T, G)]
+                continue
             torch.cuda.empty_cache()
             x = synthetic.make_gqa(B, T, H, Hk, d, 0, seed=0, device=device)
             cache = dcache = None
@@ -408,6 +415,8 @@ def run_gqa_sweep(device, shapes=None):
                                                  dQ=dQ, dK=dK, dV=dV, d_depth_kv=dcache, workspace=ws)
             iters = 2 if T >= 32768 else 5
             res[l] = (time_calls(fwd, iters), time_calls(bwd, iters))
+            if l == 0:
+                base_cache[(T, G)] = res[0]
             del x, cache, dcache, O, LSE, dQ, dK, dV, ws
         (f0, b0), (f1, b1) = res[0], res[l_full]
         ff = 4.0 * B * H * d * (T * (T + 1) / 2) + 4.0 * B * H * T * l_full * d
@@ -415,6 +424,7 @@ def run_gqa_sweep(device, shapes=None):
                      "fwd_ms": round(f1, 4), "bwd_ms": round(b1, 4), "fwd_bwd_ms": round(f1 + b1, 4),
                      "l0_fwd_bwd_ms": round(f0 + b0, 4),
                      "extra_time_pct": round(100.0 * ((f1 + b1) / (f0 + b0) - 1.0), 2),
+                     "paper_extra_time_pct_a100_triton": paper_pct,
                      "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f1 + b1), 4),
                      "fwd_tflops": round(ff / f1 / 1e9, 1), "fwd_bwd_tflops": round(3.5 * ff / (f1 + b1) / 1e9, 1)})
         log("gqa_sweep", rows[-1])
@@ -556,8 +566,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--gqa-shape", default="", help="T,G: time only this grouped-query shape (B=1, d=64, 8 key/value "
-                                                    "heads, l=32 and l=0) and print its row; for profiling")
+    ap.add_argument("--gqa-shape", default="", help="T,G[,L]: time only this grouped-query shape (B=1, d=64, 8 key/value "
+                                                    "heads, L depth slots (default 32) and l=0) and print its row; for profiling")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -579,8 +589,8 @@ def main():
         torch.distributed.init_process_group("nccl", device_id=device)
     try:
         if args.gqa_shape:
-            T, G = (int(v) for v in args.gqa_shape.split(","))
-            out = {"gqa_sweep": run_gqa_sweep(device, [(T, G)])}
+            v = [int(t) for t in args.gqa_shape.split(",")]
+            out = {"gqa_sweep": run_gqa_sweep(device, [(v[0], v[1], v[2] if len(v) > 2 else 32, None)])}
         else:
             out = run_moda(args, rank, world, device)
         if rank == 0:

@@ -46,7 +46,9 @@
 extern "C" {
 #endif
 
-#define MODA_MAX_DEPTH 32
+/* Most depth slots per position.  The paper's models use up to 36 layers and its kernel table up to
+ * L = 256; the forward handles the slots in groups of 32 (an online softmax over the groups). */
+#define MODA_MAX_DEPTH 256
 
 #define MODA_OK 0
 #define MODA_ERR_NULL_POINTER (-1)    /* a required pointer is null */

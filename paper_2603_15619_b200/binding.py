@@ -15,7 +15,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmoda_b200.so")
 
-MODA_MAX_DEPTH = 32
+MODA_MAX_DEPTH = 256
 SYMBOLS = (
     "moda_version", "moda_strerror", "moda_last_cuda_error", "moda_last_status",
     "moda_depth_cache_bytes", "moda_depth_cache_append", "moda_depth_cache_unpack",

@@ -232,8 +232,8 @@ const char* moda_strerror(int code) {
         case MODA_ERR_MISALIGNED: return "a tensor pointer is not 16-byte aligned";
         case MODA_ERR_BAD_SHAPE: return "B, T and H must be >= 1 and the tensor must fit 31-bit row counts";
         case MODA_ERR_BAD_HEAD_DIM: return "head width d must be 64 or 128";
-        case MODA_ERR_BAD_DEPTH: return "depth l must be in [0, 32]";
-        case MODA_ERR_BAD_SLOT: return "depth slot must be in [0, 32)";
+        case MODA_ERR_BAD_DEPTH: return "depth l must be in [0, 256]";
+        case MODA_ERR_BAD_SLOT: return "depth slot must be in [0, 256)";
         case MODA_ERR_WORKSPACE: return "workspace is null or too small";
         case MODA_ERR_DEVICE: return "the current CUDA device is not an sm_100 part";
         case MODA_ERR_CUDA: return "a CUDA call failed (see moda_last_cuda_error)";

@@ -359,81 +359,103 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 mbar_arrive(bar(k2BarDEmpty + st));
                 ++unit;
             };
-            // ---- depth scores u_i = <q, kd_i>, 64 features per sweep ----
+            // The slots are handled in groups of kFwdDepthGroup (the score scratch holds one group): an
+            // online softmax over the groups, with the partial output o_d rescaled in TMEM when a later
+            // group raises the maximum.  Up to 32 slots are one group.
+            float m_d = -INFINITY, l_d = 0.f;
 #pragma unroll 1
-            for (int half = 0; half < NSUB; ++half) {
-                float q[64];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, half * 8 + c));
-                    q[8 * c + 0] = bf16_lo_to_f32(v.x); q[8 * c + 1] = bf16_hi_to_f32(v.x);
-                    q[8 * c + 2] = bf16_lo_to_f32(v.y); q[8 * c + 3] = bf16_hi_to_f32(v.y);
-                    q[8 * c + 4] = bf16_lo_to_f32(v.z); q[8 * c + 5] = bf16_hi_to_f32(v.z);
-                    q[8 * c + 6] = bf16_lo_to_f32(v.w); q[8 * c + 7] = bf16_hi_to_f32(v.w);
-                }
+            for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
+                const int gl = min(kFwdDepthGroup, p.l - g0);
+                // ---- depth scores u_i = <q, kd_i>, 64 features per sweep ----
 #pragma unroll 1
-                for (int i = 0; i < p.l; ++i) {
-                    uint4 cur[8];
-                    take_unit(cur);
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+                for (int half = 0; half < NSUB; ++half) {
+                    float q[64];
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        a0 = fmaf(q[8 * c + 0], bf16_lo_to_f32(cur[c].x), a0);
-                        a1 = fmaf(q[8 * c + 1], bf16_hi_to_f32(cur[c].x), a1);
-                        a2 = fmaf(q[8 * c + 2], bf16_lo_to_f32(cur[c].y), a2);
-                        a3 = fmaf(q[8 * c + 3], bf16_hi_to_f32(cur[c].y), a3);
-                        a0 = fmaf(q[8 * c + 4], bf16_lo_to_f32(cur[c].z), a0);
-                        a1 = fmaf(q[8 * c + 5], bf16_hi_to_f32(cur[c].z), a1);
-                        a2 = fmaf(q[8 * c + 6], bf16_lo_to_f32(cur[c].w), a2);
-                        a3 = fmaf(q[8 * c + 7], bf16_hi_to_f32(cur[c].w), a3);
+                        const uint4 v = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, half * 8 + c));
+                        q[8 * c + 0] = bf16_lo_to_f32(v.x); q[8 * c + 1] = bf16_hi_to_f32(v.x);
+                        q[8 * c + 2] = bf16_lo_to_f32(v.y); q[8 * c + 3] = bf16_hi_to_f32(v.y);
+                        q[8 * c + 4] = bf16_lo_to_f32(v.z); q[8 * c + 5] = bf16_hi_to_f32(v.z);
+                        q[8 * c + 6] = bf16_lo_to_f32(v.w); q[8 * c + 7] = bf16_hi_to_f32(v.w);
                     }
-                    const float part = (a0 + a1) + (a2 + a3);
-                    if (half == 0) sU[i * kTileRows + r] = part;
-                    else sU[i * kTileRows + r] += part;
+#pragma unroll 1
+                    for (int i = 0; i < gl; ++i) {
+                        uint4 cur[8];
+                        take_unit(cur);
+                        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            a0 = fmaf(q[8 * c + 0], bf16_lo_to_f32(cur[c].x), a0);
+                            a1 = fmaf(q[8 * c + 1], bf16_hi_to_f32(cur[c].x), a1);
+                            a2 = fmaf(q[8 * c + 2], bf16_lo_to_f32(cur[c].y), a2);
+                            a3 = fmaf(q[8 * c + 3], bf16_hi_to_f32(cur[c].y), a3);
+                            a0 = fmaf(q[8 * c + 4], bf16_lo_to_f32(cur[c].z), a0);
+                            a1 = fmaf(q[8 * c + 5], bf16_hi_to_f32(cur[c].z), a1);
+                            a2 = fmaf(q[8 * c + 6], bf16_lo_to_f32(cur[c].w), a2);
+                            a3 = fmaf(q[8 * c + 7], bf16_hi_to_f32(cur[c].w), a3);
+                        }
+                        const float part = (a0 + a1) + (a2 + a3);
+                        if (half == 0) sU[i * kTileRows + r] = part;
+                        else sU[i * kTileRows + r] += part;
+                    }
                 }
-            }
-            // ---- partial softmax over the l depth scores ----
-            float m_d = -INFINITY;
-            for (int i = 0; i < p.l; ++i) m_d = fmaxf(m_d, sU[i * kTileRows + r] * p.scale_log2);
-            float l_d = 0.f;
-            for (int i = 0; i < p.l; ++i) {
-                const float w = fast_exp2(fmaf(sU[i * kTileRows + r], p.scale_log2, -m_d));
-                sU[i * kTileRows + r] = w;
-                l_d += w;
+                // ---- partial softmax over the depth scores seen so far ----
+                float m_new = m_d;
+                for (int i = 0; i < gl; ++i) m_new = fmaxf(m_new, sU[i * kTileRows + r] * p.scale_log2);
+                const float f = fast_exp2(m_d - m_new);       // first group: exp2(-inf) = 0
+                l_d *= f;
+                for (int i = 0; i < gl; ++i) {
+                    const float w = fast_exp2(fmaf(sU[i * kTileRows + r], p.scale_log2, -m_new));
+                    sU[i * kTileRows + r] = w;
+                    l_d += w;
+                }
+                m_d = m_new;
+                // ---- o_d = sum_i w_i vd_i, 64 features per sweep, parked in TMEM ----
+#pragma unroll 1
+                for (int half = 0; half < NSUB; ++half) {
+                    float acc[64];
+                    if (g0 == 0) {
+#pragma unroll
+                        for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tmem + lane_addr + kColOd + half * 64 + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) acc[32 * c + i] = __uint_as_float(o[i]) * f;
+                        }
+                    }
+#pragma unroll 1
+                    for (int i = 0; i < gl; ++i) {
+                        uint4 cur[8];
+                        take_unit(cur);
+                        const float w = sU[i * kTileRows + r];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            acc[8 * c + 0] = fmaf(w, bf16_lo_to_f32(cur[c].x), acc[8 * c + 0]);
+                            acc[8 * c + 1] = fmaf(w, bf16_hi_to_f32(cur[c].x), acc[8 * c + 1]);
+                            acc[8 * c + 2] = fmaf(w, bf16_lo_to_f32(cur[c].y), acc[8 * c + 2]);
+                            acc[8 * c + 3] = fmaf(w, bf16_hi_to_f32(cur[c].y), acc[8 * c + 3]);
+                            acc[8 * c + 4] = fmaf(w, bf16_lo_to_f32(cur[c].z), acc[8 * c + 4]);
+                            acc[8 * c + 5] = fmaf(w, bf16_hi_to_f32(cur[c].z), acc[8 * c + 5]);
+                            acc[8 * c + 6] = fmaf(w, bf16_lo_to_f32(cur[c].w), acc[8 * c + 6]);
+                            acc[8 * c + 7] = fmaf(w, bf16_hi_to_f32(cur[c].w), acc[8 * c + 7]);
+                        }
+                    }
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t o[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(acc[32 * c + i]);
+                        tmem_st32(tmem + lane_addr + kColOd + half * 64 + c * 32, o);
+                    }
+                    tmem_wait_st();                          // a later group reads these columns back
+                }
             }
             sMd[r] = m_d;
             sLd[r] = l_d;
-            // ---- o_d = sum_i w_i vd_i, 64 features per sweep, parked in TMEM ----
-#pragma unroll 1
-            for (int half = 0; half < NSUB; ++half) {
-                float acc[64];
-#pragma unroll
-                for (int c = 0; c < 64; ++c) acc[c] = 0.f;
-#pragma unroll 1
-                for (int i = 0; i < p.l; ++i) {
-                    uint4 cur[8];
-                    take_unit(cur);
-                    const float w = sU[i * kTileRows + r];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        acc[8 * c + 0] = fmaf(w, bf16_lo_to_f32(cur[c].x), acc[8 * c + 0]);
-                        acc[8 * c + 1] = fmaf(w, bf16_hi_to_f32(cur[c].x), acc[8 * c + 1]);
-                        acc[8 * c + 2] = fmaf(w, bf16_lo_to_f32(cur[c].y), acc[8 * c + 2]);
-                        acc[8 * c + 3] = fmaf(w, bf16_hi_to_f32(cur[c].y), acc[8 * c + 3]);
-                        acc[8 * c + 4] = fmaf(w, bf16_lo_to_f32(cur[c].z), acc[8 * c + 4]);
-                        acc[8 * c + 5] = fmaf(w, bf16_hi_to_f32(cur[c].z), acc[8 * c + 5]);
-                        acc[8 * c + 6] = fmaf(w, bf16_lo_to_f32(cur[c].w), acc[8 * c + 6]);
-                        acc[8 * c + 7] = fmaf(w, bf16_hi_to_f32(cur[c].w), acc[8 * c + 7]);
-                    }
-                }
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t o[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(acc[32 * c + i]);
-                    tmem_st32(tmem + lane_addr + kColOd + half * 64 + c * 32, o);
-                }
-            }
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(k2BarDepth));
@@ -535,17 +557,20 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
                                  (((size_t(b) * Hk + hk) * nq + qt) * 2) * (size_t(kTileRows) * D * 2);
             int unit = 0;
-            for (int kv = 0; kv < 2; ++kv)
-                for (int half = 0; half < NSUB; ++half)
-                    for (int i = 0; i < p.l; ++i, ++unit) {
-                        const int st = unit % L::kRingStages;
-                        if (unit >= L::kRingStages)
-                            mbar_wait(bar(k2BarDEmpty + st), ((unit / L::kRingStages) - 1) & 1, abort_flag, 32);
-                        mbar_arrive_expect_tx(bar(k2BarDFull + st), L::kUnitBytes);
-                        bulk_load(sbase + L::kRing + st * L::kUnitBytes,
-                                  blk + size_t(i) * slot_bytes + size_t(kv) * (size_t(kTileRows) * D * 2) + size_t(half) * L::kUnitBytes,
-                                  L::kUnitBytes, bar(k2BarDFull + st), policy);
-                    }
+            for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
+                const int gl = min(kFwdDepthGroup, p.l - g0);
+                for (int kv = 0; kv < 2; ++kv)
+                    for (int half = 0; half < NSUB; ++half)
+                        for (int i = 0; i < gl; ++i, ++unit) {
+                            const int st = unit % L::kRingStages;
+                            if (unit >= L::kRingStages)
+                                mbar_wait(bar(k2BarDEmpty + st), ((unit / L::kRingStages) - 1) & 1, abort_flag, 32);
+                            mbar_arrive_expect_tx(bar(k2BarDFull + st), L::kUnitBytes);
+                            bulk_load(sbase + L::kRing + st * L::kUnitBytes,
+                                      blk + size_t(g0 + i) * slot_bytes + size_t(kv) * (size_t(kTileRows) * D * 2) + size_t(half) * L::kUnitBytes,
+                                      L::kUnitBytes, bar(k2BarDFull + st), policy);
+                        }
+            }
         }
       }
     }

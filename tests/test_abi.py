@@ -38,7 +38,7 @@ def test_size_queries_are_host_arithmetic():
     assert moda.moda_depth_cache_bytes(1, 256, 2, 64, 4) == 4 * 1 * 2 * 2 * 2 * 128 * 64 * 2
     assert moda.moda_depth_cache_bytes(2, 129, 3, 128, 1) == 2 * 3 * 2 * 2 * 128 * 128 * 2
     assert moda.moda_depth_cache_bytes(1, 256, 2, 96, 4) == 0      # unsupported head width
-    assert moda.moda_depth_cache_bytes(1, 256, 2, 64, 33) == 0     # more than 32 slots
+    assert moda.moda_depth_cache_bytes(1, 256, 2, 64, 257) == 0    # more than 256 slots
     assert moda.moda_depth_cache_bytes(1, 0, 2, 64, 1) == 0
     assert moda.moda_bwd_workspace_bytes(2, 100, 3, 64, 0) >= 2 * 3 * 100 * 4
     assert moda.moda_bwd_workspace_bytes(2, 100, 3, 64, 0) % 16 == 0
@@ -58,11 +58,11 @@ def test_argument_validation_rejects_before_any_launch():
 
     assert call(B=0) == -3 and call(T=0) == -3 and call(H=-1) == -3
     assert call(d=96) == -4
-    assert call(l=-1) == -5 and call(l=33) == -5
+    assert call(l=-1) == -5 and call(l=257) == -5
     assert call(Q=None) == -1 and call(O=None) == -1 and call(LSE=None) == -1
     assert call(l=2, dkv=None) == -1
     assert call(K=odd) == -2
-    assert lib.moda_depth_cache_append(p, 1, 128, 1, 64, 32, p, p, None) == -6
+    assert lib.moda_depth_cache_append(p, 1, 128, 1, 64, 256, p, p, None) == -6
     assert lib.moda_depth_cache_append(p, 1, 128, 1, 64, -1, p, p, None) == -6
     assert lib.moda_depth_cache_append(None, 1, 128, 1, 64, 0, p, p, None) == -1
     # backward: workspace too small / missing, bad stage mask

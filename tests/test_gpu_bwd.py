@@ -68,6 +68,8 @@ SMALL = [
     (1, 1, 1, 64, 0), (1, 1, 1, 64, 3), (1, 2, 1, 128, 1), (2, 127, 2, 64, 1), (1, 128, 1, 128, 0),
     (1, 129, 2, 128, 3), (2, 255, 1, 64, 32), (2, 257, 3, 128, 32), (1, 300, 2, 64, 8), (1, 640, 2, 128, 5),
     (1, 64, 1, 64, 2), (1, 65, 1, 128, 2), (1, 192, 2, 64, 0), (1, 1000, 1, 64, 2),
+    # more than 32 depth slots: the forward's online softmax over groups of 32 slots
+    (1, 200, 2, 64, 33), (1, 257, 1, 128, 64), (1, 130, 1, 64, 100), (1, 128, 1, 128, 256),
 ]
 
 

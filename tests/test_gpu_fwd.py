@@ -43,6 +43,8 @@ SMALL = [
     (1, 1, 1, 64, 0), (1, 1, 1, 64, 3), (1, 2, 1, 128, 1), (2, 127, 2, 64, 1), (1, 128, 1, 128, 0),
     (1, 129, 2, 128, 3), (2, 255, 1, 64, 32), (2, 257, 3, 128, 32), (1, 300, 2, 64, 8), (1, 640, 2, 128, 5),
     (1, 1024, 1, 128, 0), (1, 1000, 1, 64, 2),
+    # more than 32 depth slots: several groups of the online softmax over the depth keys
+    (1, 200, 2, 64, 33), (1, 257, 1, 128, 64), (1, 130, 1, 64, 100), (1, 128, 1, 128, 256), (2, 300, 2, 64, 65),
 ]
 
 
@@ -65,6 +67,22 @@ def test_large_scores_exercise_rescaling():
     O, LSE = run_forward(x, w)
     O_ref, LSE_ref = oracle_forward(x, w.scale)
     assert_forward_close(O, LSE, O_ref, LSE_ref, "ramp")
+
+
+@pytest.mark.parametrize("d,direction", [(64, 1), (128, 1), (64, -1)])
+def test_depth_slot_groups_rescale_each_other(d, direction):
+    # 80 depth slots = three groups of the online softmax over the depth keys; key norms grow (or
+    # shrink) with the slot index, so that later groups raise the running maximum and the partial
+    # output of earlier groups must be rescaled (or later groups arrive far below the maximum)
+    w = synthetic.Workload("g", 1, 200, 2, d, 80)
+    x = synthetic.make(w, seed=8, device="cuda")
+    ramp = torch.linspace(0.2, 3.0, w.l, device="cuda")
+    if direction < 0:
+        ramp = ramp.flip(0)
+    x["Kd"] = (x["Kd"].float() * ramp.view(w.l, 1, 1, 1, 1)).to(torch.bfloat16)
+    O, LSE = run_forward(x, w)
+    O_ref, LSE_ref = oracle_forward(x, w.scale)
+    assert_forward_close(O, LSE, O_ref, LSE_ref, "depth ramp")
 
 
 def test_l0_matches_l_gt0_with_far_away_depth_keys():

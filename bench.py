@@ -39,9 +39,9 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # profiles/ (bytes); keyed by (workload, kernel).  None where no capture exists.
 NCU_TRAFFIC_BYTES = {
     # c2 captured at B=1 and scaled x4 (traffic is proportional to B): profiles/ncu_full_c2_B1_fwd_bwd_kernels.md
-    ("c2", "fwd"): 4 * (822.428e6 + 5.828e6),
-    ("c2", "bwd_dq_depth"): 4 * (845.104e6 + 735.264e6),
-    ("c2", "bwd_dkdv"): 4 * (67.748e6 + 7.575e6),
+    ("c2", "fwd"): 4 * (822.179e6 + 6.956e6),
+    ("c2", "bwd_dq_depth"): 4 * (845.105e6 + 735.033e6),
+    ("c2", "bwd_dkdv"): 4 * (67.678e6 + 8.945e6),
 }
 
 

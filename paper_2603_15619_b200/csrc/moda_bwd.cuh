@@ -17,6 +17,11 @@
 //   3. moda_bwd_dkdv_kernel  one CTA per 128-key tile, loops over 64-query tiles in the
 //                            transposed formulation (S^T = K Q^T, dP^T = V dO^T) so that
 //                            P^T and dS^T are TMEM A-operands of dV += P^T dO, dK += dS^T Q.
+//
+// Grouped-query attention (H query heads on H / G key/value heads): dK, dV sum over the G heads
+// inside the dK/dV kernel (its loop runs over the group's (head, query tile) pairs); the depth
+// gradients sum over heads that live in different CTAs of the dQ kernel, so that kernel then only
+// leaves its per-row factors and depth_grad_group_kernel (a fourth launch) forms the sums.
 #pragma once
 
 #include "moda_cache.cuh"

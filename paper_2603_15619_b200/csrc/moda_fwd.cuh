@@ -1,7 +1,8 @@
 // MoDA forward kernel for sm_100a (Sec. 2.2 definition; Alg. 1 gives the blockwise
 // online-softmax schedule this kernel re-designs for tcgen05 / TMEM / TMA).
 //
-// One CTA owns one (b, h, 128-query-row tile).  320 threads, five roles:
+// One CTA owns one (b, query head h, 128-query-row tile); with grouped-query attention the G heads
+// that share a key/value head are adjacent CTAs (tile_coord).  384 threads, three warpgroups:
 //
 //   warps 0-3  softmax   one thread per query row.  Reads the score tile S_j from TMEM,
 //                        keeps the running (m, l) of the online softmax in registers, writes
@@ -11,18 +12,19 @@
 //   warps 4-7  depth     one thread per query row.  Reads the row's l depth keys/values from
 //                        a shared-memory ring that warp 10 fills with 16 KiB bulk copies of
 //                        the depth cache, builds an independent partial softmax state
-//                        (m_d, l_d, o_d) on the CUDA cores and parks o_d in TMEM.  Merging
-//                        two partial softmax states is exact, so the epilogue obtains the
-//                        single softmax over sequence and depth keys that the paper defines.
+//                        (m_d, l_d, o_d) on the CUDA cores (slots in groups of 32, online
+//                        softmax over the groups) and parks o_d in TMEM.  Merging two partial
+//                        softmax states is exact, so the epilogue obtains the single softmax
+//                        over sequence and depth keys that the paper defines.
 //   warp 8     TMA       one lane streams the Q tile and the K_j / V_j tiles (128B swizzle)
 //                        through two-stage rings.
+//   warp 9     MMA (S)   issues S_j = Q K_j^T (operands in shared memory); owns the TMEM
+//                        allocation.  The whole warp runs the loop, an elected lane issues.
 //   warp 10    depth producer (one lane)
-//   warp 9     MMA (S)   one lane issues S_j = Q K_j^T (operands in shared memory); owns the
-//                        TMEM allocation.
-//   warp 11    MMA (PV)  one lane issues O += P_j V_j (P_j from TMEM, V_j MN-major in shared
-//                        memory).  One tcgen05.mma costs its issuing thread about 60 cycles, as much
-//                        as a 128x128x16 MMA executes, so the two contractions are issued by two
-//                        threads on different schedulers and ordered by mbarriers.
+//   warp 11    MMA (PV)  issues O += P_j V_j (P_j from TMEM, V_j MN-major in shared memory).
+//                        One tcgen05.mma costs its issuing warp 40-100 cycles, as much as a
+//                        128x128x16 MMA executes, so the two contractions are issued by two
+//                        warps on different schedulers and ordered by mbarriers.
 //
 // TMEM columns (fp32): [0,128) S_0/P_0   [128,256) S_1/P_1   [256,256+D) O   [384,384+D) o_d.
 // The depth scores never touch the tensor cores and no score matrix is ever materialised.

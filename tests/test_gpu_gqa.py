@@ -91,12 +91,14 @@ def test_grouped_sums_are_bit_reproducible():
             assert torch.equal(s, t), f"{name} changed on repeat {rep}"
 
 
-def test_paper_table2_shape_one_group_against_the_oracle():
-    # The shape family of the paper's kernel table (B = 1, d = 64, 8 key/value heads, G = 8) at
-    # T = 8192, l = 32, on the GPU in full; key/value groups are independent, so the oracle checks
-    # one whole group (8 query heads on key/value head 3) as a problem of its own.
-    B, T, H, Hk, d, l = 1, 8192, 64, 8, 64, 32
-    G, hk = H // Hk, 3
+@pytest.mark.parametrize("T,l,hk", [(8192, 32, 3), (4096, 256, 5)])
+def test_paper_table2_shape_one_group_against_the_oracle(T, l, hk):
+    # The shape family of the paper's kernel table (B = 1, d = 64, 8 key/value heads, G = 8), on the
+    # GPU in full: at T = 8192 with 32 slots, and at T = 4096 with the table's largest L = 256 (eight
+    # groups of the forward's online softmax over the depth keys).  Key/value groups are independent,
+    # so the oracle checks one whole group (8 query heads on one key/value head) as a problem of its own.
+    B, H, Hk, d = 1, 64, 8, 64
+    G = H // Hk
     scale = d ** -0.5
     x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=2, device="cuda", k_head_norm=True)
     O, LSE, grads = run(x, l, scale)

@@ -97,11 +97,19 @@ bool set_smem_limit(Kernel k, int bytes) {
 
 // d = 128 runs moda_fwd_kernel (one softmax warpgroup: the tensor pipe and the MMA issue rate set the
 // pace); d = 64 runs moda_fwd2_kernel (two softmax warpgroups, three score buffers: the exponentials do).
+// Which forward kernel at d = 128: one K stage and a five-unit depth ring when the depth stream
+// outweighs the sequence work (measured: - 6 % at l d / T = 0.72, - 3 % at 0.5, slower below),
+// otherwise two K stages and a three-unit ring.
+inline bool fwd_depth_heavy(int T, int l, int d) {
+    return d == 128 && l > 0 && 2ll * l * d >= T;
+}
+
 template <int D>
 int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int H, int Hk, int l,
                float scale, void* O, float* LSE, cudaStream_t stream) {
     constexpr bool kWide = (D == 64);
-    constexpr int kSmem = kWide ? Fwd2Smem<D>::kDynamic : FwdSmem<D>::kDynamic;
+    constexpr int kSmem = kWide ? Fwd2Smem<D>::kDynamic : FwdSmem<D, 2>::kDynamic;
+    constexpr int kSmemDeep = FwdSmem<128, 1>::kDynamic;
     constexpr int kThreads = kWide ? kFwd2Threads : kFwdThreads;
     CUtensorMap mQ, mK, mV, mO;
     if (!make_bthd_map(&mQ, Q, B, T, H, D) || !make_bthd_map(&mK, K, B, T, Hk, D) ||
@@ -111,7 +119,8 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
     if (configured_dev != dev) {
-        const bool ok = kWide ? set_smem_limit(moda_fwd2_kernel<D>, kSmem) : set_smem_limit(moda_fwd_kernel<D>, kSmem);
+        const bool ok = kWide ? set_smem_limit(moda_fwd2_kernel<D>, kSmem)
+                              : set_smem_limit(moda_fwd_kernel<D, 2>, kSmem) && set_smem_limit(moda_fwd_kernel<128, 1>, kSmemDeep);
         if (!ok) return MODA_ERR_CUDA;
         configured_dev = dev;
     }
@@ -124,7 +133,8 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.scale_log2 = scale * kLog2e;
     const unsigned grid = unsigned(B) * H * num_tiles(T);
     if (kWide) moda_fwd2_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
-    else moda_fwd_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
+    else if (fwd_depth_heavy(T, l, D)) moda_fwd_kernel<128, 1><<<grid, kThreads, kSmemDeep, stream>>>(mQ, mK, mV, mO, p);
+    else moda_fwd_kernel<D, 2><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 

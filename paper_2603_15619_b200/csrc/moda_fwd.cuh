@@ -40,20 +40,27 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
-template <int D>
+// KST = stages of the K ring.  Two let K_{j+1} load while S_j is still being computed; one (the
+// load starts when S_j completes and overlaps the softmax of tile j) leaves room for a deeper depth
+// ring, for shapes whose depth stream outweighs the sequence work (the host picks, see launch_fwd).
+template <int D, int KST = 2>
 struct FwdSmem {
     static constexpr int kTileBytes = kTileRows * D * 2;          // one 128 x D bf16 tile
     static constexpr int kSubBytes = kTileRows * 128;             // one 128 x 64 sub-tile
+    static constexpr int kKStages = KST;
     static constexpr int kQ = 0;
-    static constexpr int kK = kQ + kTileBytes;                    // 2 stages
-    static constexpr int kV = kK + 2 * kTileBytes;                // 2 stages
+    static constexpr int kK = kQ + kTileBytes;                    // KST stages
+    static constexpr int kV = kK + KST * kTileBytes;              // 2 stages
     static constexpr int kU = kV + 2 * kTileBytes;                // depth scores [32][128] fp32
     static constexpr int kMd = kU + 32 * kTileRows * 4;           // m_d [128], l_d [128]
     static constexpr int kRing = kMd + 2 * kTileRows * 4;         // depth units: 8 chunks x 128 rows x 16 B
     static constexpr int kUnitBytes = 8 * kTileRows * 16;         // 16 KiB, contiguous in the depth cache
-    static constexpr int kRingStages = (D == 128) ? 3 : 6;
-    static constexpr int kBars = kRing + kRingStages * kUnitBytes;
     static constexpr int kNumBars = 32;
+    static constexpr int kSmemLimit = 232448;                     // 227 KiB per CTA on sm_100
+    static constexpr int kRingFit = (kSmemLimit - 1024 - kRing - kNumBars * 8 - 16) / kUnitBytes;
+    static constexpr int kRingStages = kRingFit < 6 ? kRingFit : 6;   // every unit that fits, at most 6
+    static_assert(kRingStages >= 3, "depth ring too shallow");
+    static constexpr int kBars = kRing + kRingStages * kUnitBytes;
     static constexpr int kMisc = kBars + kNumBars * 8;            // tmem base, abort flag
     static constexpr int kTotal = kMisc + 16;
     static constexpr int kDynamic = kTotal + 1024;                // slack for 1024-byte alignment
@@ -112,12 +119,12 @@ __device__ __forceinline__ uint32_t swz_chunk_offset(int r, int c) {
     return uint32_t(c >> 3) * uint32_t(kTileRows * 128) + uint32_t(r) * 128u + (uint32_t((c & 7) ^ (r & 7)) << 4);
 }
 
-template <int D>
+template <int D, int KST = 2>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                 const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
                 const FwdParams p) {
-    using L = FwdSmem<D>;
+    using L = FwdSmem<D, KST>;
     constexpr int NSUB = D / 64;
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColO = 256, kColOd = 384;
@@ -449,12 +456,13 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             for (int s = 0; s < NSUB; ++s)
                 tma_load_4d(sbase + L::kQ + s * L::kSubBytes, &mapQ, bar(kBarQ), s * 64, h, q0, b);
             for (int j = 0; j < n_kv; ++j) {
-                const int st = j & 1;
-                if (j >= 2) mbar_wait(bar(kBarSFull + st), ((j - 2) >> 1) & 1, abort_flag, 30);   // S_{j-2} complete
-                mbar_arrive_expect_tx(bar(kBarKFull + st), L::kTileBytes);
+                const int st = j & 1, kst = j % KST;
+                // the K stage is free once S of its previous tile (j - KST) has completed
+                if (j >= KST) mbar_wait(bar(kBarSFull + ((j - KST) & 1)), ((j - KST) >> 1) & 1, abort_flag, 30);
+                mbar_arrive_expect_tx(bar(kBarKFull + kst), L::kTileBytes);
 #pragma unroll
                 for (int s = 0; s < NSUB; ++s)
-                    tma_load_4d(sbase + L::kK + st * L::kTileBytes + s * L::kSubBytes, &mapK, bar(kBarKFull + st),
+                    tma_load_4d(sbase + L::kK + kst * L::kTileBytes + s * L::kSubBytes, &mapK, bar(kBarKFull + kst),
                                 s * 64, hk, j * kTileRows, b);
                 if (j >= 2) mbar_wait(bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 31);
                 mbar_arrive_expect_tx(bar(kBarVFull + st), L::kTileBytes);
@@ -476,12 +484,12 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             const uint64_t dk0 = desc_kmajor_sw128(sbase + L::kK, 0);
             mbar_wait(bar(kBarQ), 0, abort_flag, 41);
             for (int j = 0; j < n_kv; ++j) {
-                const int st = j & 1;
-                mbar_wait(bar(kBarKFull + st), (j >> 1) & 1, abort_flag, 40);
+                const int st = j & 1, kst = j % KST;
+                mbar_wait(bar(kBarKFull + kst), (j / KST) & 1, abort_flag, 40);
                 // score buffer st still holds P_{j-2} until PV_{j-2} has completed
                 if (j >= 2) mbar_wait(bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 44);
                 tc_fence_after_sync();
-                const uint64_t dk = dk0 + uint64_t((st * L::kTileBytes) >> 4);
+                const uint64_t dk = dk0 + uint64_t((kst * L::kTileBytes) >> 4);
                 const uint32_t ts = tmem + uint32_t(st) * 128u;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)

@@ -500,9 +500,11 @@ def cpu_sample(w, n_slices, seed=0):
     return out, pick
 
 
-def time_oracle(w, n_slices):
+def time_oracle(w, n_slices, sample=None):
+    """Seconds of one oracle forward + backward over `n_slices` complete (b, h) slices (the inputs are
+    generated outside the timed part; pass `sample` to reuse them)."""
     from oracle import moda_oracle as orc
-    x, pick = cpu_sample(w, n_slices)
+    x, pick = sample if sample is not None else cpu_sample(w, n_slices)
     t0 = time.time()
     orc.forward(x["Q"], x["K"], x["V"], x["Kd"], x["Vd"], w.scale)
     orc.backward(x["Q"], x["K"], x["V"], x["Kd"], x["Vd"], x["dO"], w.scale)
@@ -531,16 +533,14 @@ def run_reference(args, rank, world):
         return None
     K, W = args.steps, max(args.warmup, 0)
     # bounded: each step is one complete (b, h) slice; cap the whole run near three minutes
-    t_probe, fl, cores, _ = time_oracle(w, 1)
+    sample = cpu_sample(w, 1)
+    t_probe, fl, cores, _ = time_oracle(w, 1, sample)
     budget = 180.0
     K_eff = int(max(1, min(K, (budget - t_probe) // max(t_probe, 1e-3))))
     W_eff = 0 if t_probe * (K_eff + W) > budget else W
     for _ in range(W_eff):
-        time_oracle(w, 1)
-    t0 = time.time()
-    for _ in range(K_eff):
-        time_oracle(w, 1)
-    dt = (time.time() - t0) / K_eff
+        time_oracle(w, 1, sample)
+    dt = sum(time_oracle(w, 1, sample)[0] for _ in range(K_eff)) / K_eff
     val = fl / dt / 1e12
     return {
         "impl": "reference", "metric": METRIC, "value": round(val, 6), "unit": UNIT, "n_gpus": world, "steps": K_eff,

@@ -167,3 +167,11 @@ def test_c5_narrow_heads_deep_stack():
     w = synthetic.WORKLOADS["c5"]
     x, outs, _ = check_config(w, heads_bwd=3, rows_per_head=3)
     check_slice(w, x, outs, 1, 17)
+
+
+@pytest.mark.parametrize("d", [128, 64])
+def test_twice_the_longest_configured_context(d):
+    # T = 131072 (1024 query tiles per head), beyond every configured workload: index arithmetic,
+    # barrier phases over very long loops and the causal imbalance at its largest
+    w = synthetic.Workload("t128k", 1, 131072, 2, d, 4)
+    check_config(w, heads_bwd=2, rows_per_head=3)

@@ -818,25 +818,29 @@ moda_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_cons
             tmem_ld32(tmem + lane_addr + kColST + buf * 64 + hc * 32, s);
             tmem_ld32(tmem + lane_addr + kColdPT + buf * 64 + hc * 32, g);
             tmem_wait_ld();
-            uint32_t pp[16], pd[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int c0 = hc * 32 + 2 * i;
-                const float4 t = rt[i];                      // {-LSE c0, -LSE c0+1, D c0, D c0+1}, same for all rows
-                float pa = fast_exp2(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, t.x));
-                float pb = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, t.y));
-                if (masked) {
-                    if (qoff + c0 < r) pa = 0.f;
-                    if (qoff + c0 + 1 < r) pb = 0.f;
-                }
-                pp[i] = pack_bf16x2(pa, pb);
-                pd[i] = pack_bf16x2(pa * (__uint_as_float(g[2 * i]) - t.z), pb * (__uint_as_float(g[2 * i + 1]) - t.w));
-            }
             // P^T overlays S^T, dS^T overlays dP^T (bf16, two per column).  Each warpgroup writes over
             // the first 16 of the 32 columns it has just read itself (columns 32 hc .. 32 hc + 15), so
             // the two never touch each other's scores; the MMA issuers address the two blocks per k-step.
-            tmem_st16(tmem + lane_addr + kColST + buf * 64 + hc * 32, pp);
-            tmem_st16(tmem + lane_addr + kColdPT + buf * 64 + hc * 32, pd);
+            // Stored in two halves so that the first half's stores run under the second half's arithmetic.
+            uint32_t pp[16], pd[16];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                for (int i = 8 * hh; i < 8 * hh + 8; ++i) {
+                    const int c0 = hc * 32 + 2 * i;
+                    const float4 t = rt[i];                  // {-LSE c0, -LSE c0+1, D c0, D c0+1}, same for all rows
+                    float pa = fast_exp2(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, t.x));
+                    float pb = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, t.y));
+                    if (masked) {
+                        if (qoff + c0 < r) pa = 0.f;
+                        if (qoff + c0 + 1 < r) pb = 0.f;
+                    }
+                    pp[i] = pack_bf16x2(pa, pb);
+                    pd[i] = pack_bf16x2(pa * (__uint_as_float(g[2 * i]) - t.z), pb * (__uint_as_float(g[2 * i + 1]) - t.w));
+                }
+                tmem_st8(tmem + lane_addr + kColST + buf * 64 + hc * 32 + 8 * hh, pp + 8 * hh);
+                tmem_st8(tmem + lane_addr + kColdPT + buf * 64 + hc * 32 + 8 * hh, pd + 8 * hh);
+            }
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(kDkvBarPFull + buf));

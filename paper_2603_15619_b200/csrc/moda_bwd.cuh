@@ -566,12 +566,14 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 mbar_wait(bar(kDqBarQ), 0, abort_flag, 81);
                 for (int j = 0; j < n_kv; ++j) {
                     const int st = j % L::kStages, buf = j & 1;
-                    mbar_wait(bar(kDqBarKVFull + st), (j / L::kStages) & 1, abort_flag, 80);
                     if (j >= 2) {
                         // S buffer: dS_{j-2} overlays it until dQ_{j-2} has completed;
                         // dP buffer: free once the row warps have read dP_{j-2} (their arrival for tile j-2)
-                        if (is_s) mbar_wait(bar(kDqBarKVEmpty + (j - 2) % L::kStages), ((j - 2) / L::kStages) & 1, abort_flag, 83);
-                        else mbar_wait(bar(kDqBarPFull + buf), ((j - 2) >> 1) & 1, abort_flag, 84);
+                        const uint32_t free_bar = is_s ? bar(kDqBarKVEmpty + (j - 2) % L::kStages) : bar(kDqBarPFull + buf);
+                        const uint32_t free_par = is_s ? ((j - 2) / L::kStages) & 1 : ((j - 2) >> 1) & 1;
+                        mbar_wait2(bar(kDqBarKVFull + st), (j / L::kStages) & 1, free_bar, free_par, abort_flag, 80, is_s ? 83 : 84);
+                    } else {
+                        mbar_wait(bar(kDqBarKVFull + st), (j / L::kStages) & 1, abort_flag, 80);
                     }
                     tc_fence_after_sync();
                     const uint64_t db = db0 + uint64_t((st * 2 * L::kHalfTileBytes) >> 4);

@@ -485,9 +485,9 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             mbar_wait(bar(kBarQ), 0, abort_flag, 41);
             for (int j = 0; j < n_kv; ++j) {
                 const int st = j & 1, kst = j % KST;
-                mbar_wait(bar(kBarKFull + kst), (j / KST) & 1, abort_flag, 40);
                 // score buffer st still holds P_{j-2} until PV_{j-2} has completed
-                if (j >= 2) mbar_wait(bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 44);
+                if (j >= 2) mbar_wait2(bar(kBarKFull + kst), (j / KST) & 1, bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 40, 44);
+                else mbar_wait(bar(kBarKFull + kst), (j / KST) & 1, abort_flag, 40);
                 tc_fence_after_sync();
                 const uint64_t dk = dk0 + uint64_t((kst * L::kTileBytes) >> 4);
                 const uint32_t ts = tmem + uint32_t(st) * 128u;
@@ -510,8 +510,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             const uint64_t dv0 = desc_mnmajor_sw128(sbase + L::kV, 0, L::kSubBytes);
             for (int j = 0; j < n_kv; ++j) {
                 const int st = j & 1;
-                mbar_wait(bar(kBarVFull + st), (j >> 1) & 1, abort_flag, 42);
-                mbar_wait(bar(kBarPFull + st), (j >> 1) & 1, abort_flag, 43);
+                mbar_wait2(bar(kBarVFull + st), (j >> 1) & 1, bar(kBarPFull + st), (j >> 1) & 1, abort_flag, 42, 43);
                 tc_fence_after_sync();
                 const uint64_t dv = dv0 + uint64_t((st * L::kTileBytes) >> 4);
                 const uint32_t tp = tmem + uint32_t(st) * 128u;

@@ -502,9 +502,12 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             mbar_wait(bar(k2BarQ), 0, abort_flag, 41);
             for (int j = 0; j < n_kv; ++j) {
                 const int st = j % L::kStages;
-                mbar_wait(bar(k2BarKFull + st), (j / L::kStages) & 1, abort_flag, 40);
                 // score buffer st still holds P_{j-stages} until that tile's PV has completed
-                if (j >= L::kStages) mbar_wait(bar(k2BarVEmpty + st), ((j / L::kStages) - 1) & 1, abort_flag, 44);
+                if (j >= L::kStages)
+                    mbar_wait2(bar(k2BarKFull + st), (j / L::kStages) & 1, bar(k2BarVEmpty + st), ((j / L::kStages) - 1) & 1,
+                               abort_flag, 40, 44);
+                else
+                    mbar_wait(bar(k2BarKFull + st), (j / L::kStages) & 1, abort_flag, 40);
                 tc_fence_after_sync();
                 const uint64_t dk = dk0 + uint64_t((st * L::kKeyTileBytes) >> 4);
                 const uint32_t ts = tmem + uint32_t(st) * kFwdBN;
@@ -528,8 +531,7 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             for (int j = 0; j < n_kv; ++j) {
                 const int st = j % L::kStages;
                 const uint32_t par = (j / L::kStages) & 1;
-                mbar_wait(bar(k2BarVFull + st), par, abort_flag, 42);
-                mbar_wait(bar(k2BarPFull + st), par, abort_flag, 43);
+                mbar_wait2(bar(k2BarVFull + st), par, bar(k2BarPFull + st), par, abort_flag, 42, 43);
                 tc_fence_after_sync();
                 const uint64_t dv = dv0 + uint64_t((st * L::kKeyTileBytes) >> 4);
                 const uint32_t tp = tmem + uint32_t(st) * kFwdBN;

@@ -104,6 +104,27 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Bounded wait on two barriers.  Both probes are issued before either result is used, so their
+// round trips through the shared-memory pipe (100-200 cycles each even when the phase is long
+// complete) overlap; whatever is still pending afterwards is waited for one by one.
+__device__ __forceinline__ void mbar_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b,
+                                           volatile int* abort_flag, int site_a, int site_b) {
+    uint32_t ok_a, ok_b;
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%2], %3;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 q, [%4], %5;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "selp.u32 %1, 1, 0, q;\n"
+        "}\n"
+        : "=r"(ok_a), "=r"(ok_b)
+        : "r"(bar_a), "r"(parity_a), "r"(bar_b), "r"(parity_b)
+        : "memory");
+    if (!ok_a) mbar_wait(bar_a, parity_a, abort_flag, site_a);
+    if (!ok_b) mbar_wait(bar_b, parity_b, abort_flag, site_b);
+}
+
 // ------------------------------------------------------------------------------------
 // Proxy / tcgen05 fences
 // ------------------------------------------------------------------------------------

@@ -62,8 +62,8 @@ extern "C" {
 #define MODA_ERR_CUDA (-9)            /* a CUDA runtime/driver call failed (see moda_last_cuda_error) */
 #define MODA_ERR_DEVICE_TIMEOUT (-10) /* an earlier kernel gave up a bounded wait (see moda_last_status) */
 #define MODA_ERR_SCRATCH_LIMIT (-11)  /* problem needs more built-in scratch than moda_attn_bwd_static_scratch holds */
-#define MODA_ERR_BAD_GROUP (-12)      /* H_kv does not divide H, or more than MODA_MAX_GROUP query heads per group */
-#define MODA_MAX_GROUP 8
+#define MODA_ERR_BAD_GROUP (-12)      /* H_kv does not divide H, or an unsupported number of query heads per group */
+#define MODA_MAX_GROUP 32             /* supported group sizes G = H / H_kv: 1 to 8, 16 and 32 */
 
 /* Library version: major * 10000 + minor * 100 + patch. */
 int moda_version(void);
@@ -157,7 +157,7 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
  * a fixed order (no atomics), so results are bit-reproducible.  With G > 1 the workspace also
  * holds two fp32 factors per (row, slot, query head), from which a second kernel forms the depth
  * gradients without reading the depth cache again.  H_kv must divide H
- * and G <= MODA_MAX_GROUP (MODA_ERR_BAD_GROUP otherwise); H_kv == H is exactly
+ * and G = H / H_kv must be 1 to 8, 16 or 32 (MODA_ERR_BAD_GROUP otherwise); H_kv == H is exactly
  * moda_attn_fwd / moda_attn_bwd.  Everything else (validation, streams, ownership, errors) is
  * as for those calls.
  */

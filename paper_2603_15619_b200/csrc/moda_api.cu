@@ -71,9 +71,11 @@ int check_shape(int B, int T, int H, int d) {
     return MODA_OK;
 }
 
-// Query heads H on H_kv key/value heads: H_kv must divide H, at most MODA_MAX_GROUP heads per group.
+// Query heads H on H_kv key/value heads: H_kv must divide H; 1 to 8, 16 or 32 heads per group.
 int check_groups(int H, int H_kv) {
-    if (H_kv < 1 || H % H_kv != 0 || H / H_kv > MODA_MAX_GROUP) return MODA_ERR_BAD_GROUP;
+    if (H_kv < 1 || H % H_kv != 0) return MODA_ERR_BAD_GROUP;
+    const int G = H / H_kv;
+    if (!(G <= 8 || G == 16 || G == 32)) return MODA_ERR_BAD_GROUP;
     return MODA_OK;
 }
 
@@ -193,15 +195,16 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
             moda_bwd_dq_kernel<D, 3><<<grid, kBwdDqThreads, DqSmem<D, 3>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
         if (G > 1 && a.l > 0) {
-            const unsigned g2 = unsigned(B) * Hk * num_tiles(T) * 2 * (D / 32);   // x {dKd, dVd} x groups of 4 chunks
+            const unsigned tiles2 = unsigned(B) * Hk * num_tiles(T) * 2;            // x {dKd, dVd}
             const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.Q);
             const __nv_bfloat16* go = static_cast<const __nv_bfloat16*>(a.dO);
             __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.d_depth_kv);
 #define MODA_GROUP_CASE(GG) \
-            case GG: depth_grad_group_kernel<D, GG><<<g2, kGroupGradThreads, 0, stream>>>(q, go, rowterms, out, B, T, Hk, a.l, a.scale); break;
+            case GG: depth_grad_group_kernel<D, GG><<<tiles2 * (D / GroupGrad<GG>::kFW / 4), kGroupGradThreads, 0, stream>>>( \
+                         q, go, rowterms, out, B, T, Hk, a.l, a.scale); break;
             switch (G) {
                 MODA_GROUP_CASE(2) MODA_GROUP_CASE(3) MODA_GROUP_CASE(4) MODA_GROUP_CASE(5)
-                MODA_GROUP_CASE(6) MODA_GROUP_CASE(7) MODA_GROUP_CASE(8)
+                MODA_GROUP_CASE(6) MODA_GROUP_CASE(7) MODA_GROUP_CASE(8) MODA_GROUP_CASE(16) MODA_GROUP_CASE(32)
                 default: return MODA_ERR_BAD_GROUP;
             }
 #undef MODA_GROUP_CASE
@@ -248,7 +251,7 @@ const char* moda_strerror(int code) {
         case MODA_ERR_DEVICE: return "the current CUDA device is not an sm_100 part";
         case MODA_ERR_CUDA: return "a CUDA call failed (see moda_last_cuda_error)";
         case MODA_ERR_DEVICE_TIMEOUT: return "a kernel gave up a bounded wait (see moda_last_status)";
-        case MODA_ERR_BAD_GROUP: return "H_kv must divide H with at most 8 query heads per key/value head";
+        case MODA_ERR_BAD_GROUP: return "H_kv must divide H with 1 to 8, 16 or 32 query heads per key/value head";
         case MODA_ERR_SCRATCH_LIMIT: return "B*H*T exceeds the built-in scratch of moda_attn_bwd_static_scratch (2^20 rows)";
         default: return "unknown error code";
     }

@@ -621,51 +621,74 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
 // =====================================================================================
 // dKd_i[t] = scale sum_g dU_i^g[t] q^g[t] and dVd_i[t] = sum_g R_i^g[t] dO^g[t] over the G query heads
 // of a key/value head, from the factors the dQ kernel left in the workspace.  Row-local and bound by
-// the one write of the depth gradients: no depth cache is read.  One CTA per (b, hk, 128-row tile,
-// dKd or dVd, group of 4 feature chunks); a thread keeps one 8-feature chunk of the G rows (q^g or
-// dO^g) in registers and walks the slots, writing 16 bytes per slot in cache layout (consecutive
-// lanes = consecutive rows).  The factors of 8 slots at a time are staged in shared memory (every
-// thread of a row needs the same G factors per slot).
+// the one write of the depth gradients: no depth cache is read.  A thread keeps FW features of the G
+// rows (q^g or dO^g) in registers (G x FW = 64 values: FW = 8 up to G = 8, 4 at G = 16, 2 at G = 32) and
+// walks the slots, writing FW bf16 per slot in cache layout (consecutive lanes = consecutive rows).
+// One CTA = 128 rows x 4 feature pieces of one (b, hk, tile, dKd or dVd).  The factors of a few slots
+// at a time are staged in shared memory (every thread of a row needs the same G factors per slot).
 constexpr int kGroupGradThreads = 512;
-constexpr int kGroupGradSlots = 8;
+
+template <int G>
+struct GroupGrad {
+    static_assert(G >= 2 && (G <= 8 || G == 16 || G == 32), "group size not supported");
+    static constexpr int kFW = G <= 8 ? 8 : (G == 16 ? 4 : 2);      // features per thread
+    static constexpr int kSlots = G <= 8 ? 8 : (G == 16 ? 4 : 2);   // slots staged at a time (<= 32 KiB)
+};
 
 template <int D, int G>
 __global__ void __launch_bounds__(kGroupGradThreads)
 depth_grad_group_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ dO,
                         const float* __restrict__ rowterms, __nv_bfloat16* __restrict__ d_depth_kv,
                         int B, int T, int Hk, int l, float scale) {
-    constexpr int CH = D / 8;
-    constexpr int CGROUPS = CH / 4;                      // chunk groups per tile: 2 (d = 64) or 4 (d = 128)
-    __shared__ __align__(16) float s_coef[kGroupGradSlots * kTileRows * G];
+    constexpr int FW = GroupGrad<G>::kFW, SLOTS = GroupGrad<G>::kSlots;
+    constexpr int PIECES = D / FW;                       // feature pieces per row
+    constexpr int PGROUPS = PIECES / 4;                  // CTAs per (tile, kv)
+    __shared__ __align__(16) float s_coef[SLOTS * kTileRows * G];
     const int nq = num_tiles(T);
-    const int cgrp = blockIdx.x % CGROUPS;
-    const int kv = (blockIdx.x / CGROUPS) & 1;           // 0: dKd (dU, q, scaled), 1: dVd (R, dO)
-    const int tile_id = blockIdx.x / (2 * CGROUPS);      // (b * Hk + hk) * nq + qt
+    const int pgrp = blockIdx.x % PGROUPS;
+    const int kv = (blockIdx.x / PGROUPS) & 1;           // 0: dKd (dU, q, scaled), 1: dVd (R, dO)
+    const int tile_id = blockIdx.x / (2 * PGROUPS);      // (b * Hk + hk) * nq + qt
     const int qt = tile_id % nq;
     const int bhk = tile_id / nq;
     const int b = bhk / Hk, hk = bhk % Hk;
     const int r = threadIdx.x & 127;
-    const int c = cgrp * 4 + (threadIdx.x >> 7);
+    const int piece = pgrp * 4 + (threadIdx.x >> 7);     // features [piece * FW, piece * FW + FW)
     const int t = qt * kTileRows + r;
     const int H = Hk * G;
     const __nv_bfloat16* X = kv == 0 ? Q : dO;
     const float mul = kv == 0 ? scale : 1.f;
-    float x[G][8];
+    float x[G][FW];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);            // rows past T contribute zeros: the tail stays zero
-        if (t < T) v = *reinterpret_cast<const uint4*>(X + ((size_t(b) * T + t) * H + hk * G + g) * D + c * 8);
-        x[g][0] = bf16_lo_to_f32(v.x) * mul; x[g][1] = bf16_hi_to_f32(v.x) * mul;
-        x[g][2] = bf16_lo_to_f32(v.y) * mul; x[g][3] = bf16_hi_to_f32(v.y) * mul;
-        x[g][4] = bf16_lo_to_f32(v.z) * mul; x[g][5] = bf16_hi_to_f32(v.z) * mul;
-        x[g][6] = bf16_lo_to_f32(v.w) * mul; x[g][7] = bf16_hi_to_f32(v.w) * mul;
+        uint32_t w[FW / 2];
+#pragma unroll
+        for (int k = 0; k < FW / 2; ++k) w[k] = 0u;      // rows past T contribute zeros: the tail stays zero
+        if (t < T) {
+            const __nv_bfloat16* src = X + ((size_t(b) * T + t) * H + hk * G + g) * D + piece * FW;
+            if constexpr (FW == 8) {
+                const uint4 v = *reinterpret_cast<const uint4*>(src);
+                w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+            } else if constexpr (FW == 4) {
+                const uint2 v = *reinterpret_cast<const uint2*>(src);
+                w[0] = v.x; w[1] = v.y;
+            } else {
+                w[0] = *reinterpret_cast<const uint32_t*>(src);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < FW / 2; ++k) {
+            x[g][2 * k] = bf16_lo_to_f32(w[k]) * mul;
+            x[g][2 * k + 1] = bf16_hi_to_f32(w[k]) * mul;
+        }
     }
     // factors of this tile: [slot][{R, dU}][row 128][g]; dKd uses dU, dVd uses R
     const float* coef = rowterms + (size_t(tile_id) * l * 2 + (kv == 0 ? 1 : 0)) * (kTileRows * G);
-    const size_t slot_stride = cache_slot_elems(B, T, Hk, D) / 8;                    // in uint4
-    uint4* out = reinterpret_cast<uint4*>(d_depth_kv) + (size_t(tile_id) * 2 + kv) * (kTileRows * CH) + c * kTileRows + r;
-    for (int i0 = 0; i0 < l; i0 += kGroupGradSlots) {
-        const int n = min(kGroupGradSlots, l - i0);
+    const size_t slot_elems = cache_slot_elems(B, T, Hk, D);
+    // cache block of (tile, kv): [chunk][row 128][8]; this thread's FW features sit inside one chunk
+    __nv_bfloat16* out = d_depth_kv + (size_t(tile_id) * 2 + kv) * (kTileRows * D)
+                         + (size_t((piece * FW) / 8) * kTileRows + r) * 8 + (piece * FW) % 8;
+    for (int i0 = 0; i0 < l; i0 += SLOTS) {
+        const int n = min(SLOTS, l - i0);
         __syncthreads();
         for (int e = threadIdx.x; e < n * kTileRows * G; e += kGroupGradThreads) {
             const int i = e / (kTileRows * G);
@@ -673,17 +696,28 @@ depth_grad_group_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
         }
         __syncthreads();
         for (int i = 0; i < n; ++i) {
-            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            float a[FW];
+#pragma unroll
+            for (int k = 0; k < FW; ++k) a[k] = 0.f;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const float w = s_coef[(i * kTileRows + r) * G + g];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) a[k] = fmaf(w, x[g][k], a[k]);
+                for (int k = 0; k < FW; ++k) a[k] = fmaf(w, x[g][k], a[k]);
             }
-            uint4 o;
-            o.x = pack_bf16x2(a[0], a[1]); o.y = pack_bf16x2(a[2], a[3]);
-            o.z = pack_bf16x2(a[4], a[5]); o.w = pack_bf16x2(a[6], a[7]);
-            out[size_t(i0 + i) * slot_stride] = o;
+            __nv_bfloat16* dst = out + size_t(i0 + i) * slot_elems;
+            if constexpr (FW == 8) {
+                uint4 o;
+                o.x = pack_bf16x2(a[0], a[1]); o.y = pack_bf16x2(a[2], a[3]);
+                o.z = pack_bf16x2(a[4], a[5]); o.w = pack_bf16x2(a[6], a[7]);
+                *reinterpret_cast<uint4*>(dst) = o;
+            } else if constexpr (FW == 4) {
+                uint2 o;
+                o.x = pack_bf16x2(a[0], a[1]); o.y = pack_bf16x2(a[2], a[3]);
+                *reinterpret_cast<uint2*>(dst) = o;
+            } else {
+                *reinterpret_cast<uint32_t*>(dst) = pack_bf16x2(a[0], a[1]);
+            }
         }
     }
 }

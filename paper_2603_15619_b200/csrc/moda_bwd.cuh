@@ -149,7 +149,7 @@ struct DqParams {
     int G;              // query heads per key/value head
     // G == 1: the depth gradients are written by this kernel (null here).  G > 1: they are sums
     // over the heads of a group, so the kernel only leaves its per-row factors here, R_i and dU_i
-    // as [b][hk][tile][slot][{R, dU}][row 128][g] fp32, and depth_grad_group_kernel forms the sums.
+    // as [b][hk][tile][slot][{R, dU}][g][row 128] fp32, and depth_grad_group_kernel forms the sums.
     float* depth_rowterms;
     float scale, scale_log2;
 };
@@ -324,7 +324,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             // instead of writing depth gradients (which are sums over the heads of the group).
             const bool store_grads = p.depth_rowterms == nullptr;
             float* rt_row = store_grads ? nullptr
-                : p.depth_rowterms + (((size_t(b) * Hk + hk) * nq + qt) * p.l * 2) * (kTileRows * p.G) + r * p.G + (h - hk * p.G);
+                : p.depth_rowterms + (((size_t(b) * Hk + hk) * nq + qt) * p.l * 2) * (kTileRows * p.G) + (h - hk * p.G) * kTileRows + r;
             uint4* gK = reinterpret_cast<uint4*>(p.d_depth_kv) + blk;
             uint4* gV = gK + kTileRows * CH;
             mbar_wait(bar(kDqBarQ), 0, abort_flag, 60);
@@ -681,7 +681,7 @@ depth_grad_group_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
             x[g][2 * k + 1] = bf16_hi_to_f32(w[k]) * mul;
         }
     }
-    // factors of this tile: [slot][{R, dU}][row 128][g]; dKd uses dU, dVd uses R
+    // factors of this tile: [slot][{R, dU}][g][row 128]; dKd uses dU, dVd uses R
     const float* coef = rowterms + (size_t(tile_id) * l * 2 + (kv == 0 ? 1 : 0)) * (kTileRows * G);
     const size_t slot_elems = cache_slot_elems(B, T, Hk, D);
     // cache block of (tile, kv): [chunk][row 128][8]; this thread's FW features sit inside one chunk
@@ -701,7 +701,7 @@ depth_grad_group_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
             for (int k = 0; k < FW; ++k) a[k] = 0.f;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                const float w = s_coef[(i * kTileRows + r) * G + g];
+                const float w = s_coef[(i * G + g) * kTileRows + r];
 #pragma unroll
                 for (int k = 0; k < FW; ++k) a[k] = fmaf(w, x[g][k], a[k]);
             }

@@ -1,0 +1,90 @@
+"""Depth stream of a stack of attention layers, differentiable end to end.
+
+In a MoDA model (paper Sec. 2.2, the "write" step) every attention layer appends its own K, V to
+the depth stream after attending, and layer l attends to the l slots written before it.  So K_i, V_i
+of layer i receive gradient from layer i's own sequence attention and, as depth slot i, from every
+later layer.  ``DepthStream`` owns the depth cache and one gradient cache of the same layout and
+wires those contributions together around the C-ABI calls; it is plumbing (no arithmetic of the
+operator happens here beyond adding gradients).
+
+    stream = DepthStream(B, T, H_kv, d, n_layers)
+    for layer in layers:
+        q, k, v = layer.project(x)               # [B,T,H,d], [B,T,H_kv,d], [B,T,H_kv,d]
+        o = stream.attend(q, k, v)               # attends to the slots so far, then appends k, v
+        x = layer.rest(x, o)
+
+Backward runs the layers in reverse (a token tensor chains the calls so that autograd keeps that
+order even if the layers' inputs are unrelated): layer l adds its depth gradients into slots < l of
+the gradient cache, and the gradient of its own K, V is its sequence-attention gradient plus slot l
+of that cache, which by then holds the contributions of all later layers.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding
+
+
+class _Attend(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, Q, K, V, token, stream, l, scale):
+        Q, K, V = Q.contiguous(), K.contiguous(), V.contiguous()
+        O, LSE = binding.moda_attn_fwd_gqa(Q, K, V, stream.cache if l > 0 else None, l, scale)
+        binding.moda_depth_cache_append(stream.cache, l, K, V)          # the "write" step: slot l = this layer
+        ctx.save_for_backward(Q, K, V, O, LSE)
+        ctx.stream, ctx.l, ctx.scale = stream, l, scale
+        return O, token + 0
+
+    @staticmethod
+    def backward(ctx, dO, dtoken):
+        Q, K, V, O, LSE = ctx.saved_tensors
+        stream, l = ctx.stream, ctx.l
+        B, T, H, d = Q.shape
+        Hk = K.shape[2]
+        tmp = stream.scratch_grad(l)
+        dQ, dK, dV, _ = binding.moda_attn_bwd_gqa(Q, K, V, stream.cache if l > 0 else None, O, dO.contiguous(), LSE,
+                                                  l, ctx.scale, d_depth_kv=tmp)
+        if l > 0:
+            n = binding.moda_depth_cache_bytes(B, T, Hk, d, l) // 2
+            stream.grad_cache[:n] += tmp[:n]                            # slots < l: add this layer's share
+        if stream.slot_has_grad(l):                                     # later layers attended to slot l
+            dKs = torch.empty_like(K)
+            dVs = torch.empty_like(V)
+            binding.moda_depth_cache_unpack(stream.grad_cache, l, dKs, dVs)
+            dK += dKs
+            dV += dVs
+        return dQ, dK, dV, dtoken, None, None, None
+
+
+class DepthStream:
+    """Depth cache of one forward pass through a stack (and its gradient cache)."""
+
+    def __init__(self, B, T, H_kv, d, n_layers, device="cuda"):
+        self.shape = (B, T, H_kv, d)
+        self.n_layers = int(n_layers)
+        self.cache = binding.alloc_depth_cache(B, T, H_kv, d, n_layers, device)
+        self.grad_cache = torch.zeros_like(self.cache)
+        self._scratch = None
+        self.n_written = 0
+        self.token = torch.zeros((), device=device, requires_grad=True)
+
+    def scratch_grad(self, l):
+        if l == 0:
+            return None
+        if self._scratch is None:
+            self._scratch = torch.empty_like(self.cache)
+        return self._scratch
+
+    def slot_has_grad(self, l):
+        return l < self.n_written - 1
+
+    def attend(self, Q, K, V, scale=None):
+        """MoDA attention of the next layer: attends to the slots written so far, then appends K, V."""
+        l = self.n_written
+        if l >= self.n_layers:
+            raise ValueError("more layers than the stream was sized for")
+        if scale is None:
+            scale = Q.shape[-1] ** -0.5
+        O, self.token = _Attend.apply(Q, K, V, self.token, self, l, float(scale))
+        self.n_written = l + 1
+        return O

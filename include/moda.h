@@ -130,14 +130,23 @@ int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth
  *     MODA_BWD_STAGE_ROWTERMS  D_t = <dO_t, O_t> for every row, into `workspace`
  *     MODA_BWD_STAGE_DQ        dQ and the depth gradients (reads D_t from `workspace`)
  *     MODA_BWD_STAGE_DKDV      dK and dV                  (reads D_t from `workspace`)
- * moda_attn_bwd(...) is moda_attn_bwd_stages(..., MODA_BWD_ALL_STAGES, stream).  All arguments
- * are validated as for moda_attn_bwd whatever the mask; a mask outside [1, 7] is
- * MODA_ERR_BAD_SHAPE.
+ * moda_attn_bwd(...) is moda_attn_bwd_stages(..., MODA_BWD_ALL_STAGES, stream).
+ * One more bit changes how the depth gradients leave the MODA_BWD_STAGE_DQ stage:
+ *     MODA_BWD_ACCUMULATE_DEPTH  slots [0, l) of d_depth_kv are ADDED TO (bf16 additions,
+ *                                one per element per call, so the result does not depend on
+ *                                scheduling) instead of overwritten.  In a stack of layers
+ *                                K_i, V_i are depth keys of every later layer (Sec. 2.2,
+ *                                the depth stream's write step), so one gradient cache,
+ *                                zeroed once by the caller, collects d(loss)/d(slot i)
+ *                                over the backward calls of all those layers.
+ * All arguments are validated as for moda_attn_bwd whatever the mask; a mask with none of the
+ * three stage bits, or with bits above MODA_BWD_ACCUMULATE_DEPTH, is MODA_ERR_BAD_SHAPE.
  */
 #define MODA_BWD_STAGE_ROWTERMS 1
 #define MODA_BWD_STAGE_DQ 2
 #define MODA_BWD_STAGE_DKDV 4
 #define MODA_BWD_ALL_STAGES 7
+#define MODA_BWD_ACCUMULATE_DEPTH 8
 int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void* depth_kv,
                          const void* O, const void* dO, const float* LSE,
                          int B, int T, int H, int d, int l, float scale,

@@ -7,6 +7,11 @@ reported metric.  The CUDA library is loaded on first use and there is no fallba
 from .autograd import moda_attention  # noqa: F401
 from .stack import DepthStream  # noqa: F401
 from .binding import (  # noqa: F401
+    MODA_BWD_ACCUMULATE_DEPTH,
+    MODA_BWD_ALL_STAGES,
+    MODA_BWD_STAGE_DKDV,
+    MODA_BWD_STAGE_DQ,
+    MODA_BWD_STAGE_ROWTERMS,
     ModaError,
     alloc_depth_cache,
     moda_attn_bwd,

@@ -25,6 +25,7 @@ SYMBOLS = (
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
+MODA_BWD_ACCUMULATE_DEPTH = 8      # ORed into a stages mask: depth gradients are added to d_depth_kv
 
 
 class ModaError(RuntimeError):

@@ -184,6 +184,7 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
         p.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
         p.LSE = a.LSE; p.delta = delta;
         p.B = B; p.T = T; p.H = H; p.l = a.l; p.G = G;
+        p.accumulate = a.accumulate_depth ? 1 : 0;
         p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
         // Grouped-query: the dQ kernel leaves R_i, dU_i per (row, slot, head) behind the row terms D_t
         // and a second, write-bound kernel forms the depth gradients as sums over each group.
@@ -201,7 +202,7 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
             __nv_bfloat16* out = static_cast<__nv_bfloat16*>(a.d_depth_kv);
 #define MODA_GROUP_CASE(GG) \
             case GG: depth_grad_group_kernel<D, GG><<<tiles2 * (D / GroupGrad<GG>::kFW / 4), kGroupGradThreads, 0, stream>>>( \
-                         q, go, rowterms, out, B, T, Hk, a.l, a.scale); break;
+                         q, go, rowterms, out, B, T, Hk, a.l, a.scale, a.accumulate_depth ? 1 : 0); break;
             switch (G) {
                 MODA_GROUP_CASE(2) MODA_GROUP_CASE(3) MODA_GROUP_CASE(4) MODA_GROUP_CASE(5)
                 MODA_GROUP_CASE(6) MODA_GROUP_CASE(7) MODA_GROUP_CASE(8) MODA_GROUP_CASE(16) MODA_GROUP_CASE(32)
@@ -365,7 +366,8 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
                              void* workspace, size_t workspace_bytes, int stages, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
-    if (stages <= 0 || stages > MODA_BWD_ALL_STAGES) return MODA_ERR_BAD_SHAPE;
+    if ((stages & MODA_BWD_ALL_STAGES) == 0 || stages < 0 || stages > (MODA_BWD_ALL_STAGES | MODA_BWD_ACCUMULATE_DEPTH))
+        return MODA_ERR_BAD_SHAPE;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv || !d_depth_kv)))
         return MODA_ERR_NULL_POINTER;
@@ -380,6 +382,7 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
     a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv; a.O = O; a.dO = dO; a.LSE = LSE;
     a.B = B; a.T = T; a.H = H; a.Hk = H_kv; a.l = l; a.scale = scale;
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
+    a.accumulate_depth = (stages & MODA_BWD_ACCUMULATE_DEPTH) != 0;
     return d == 128 ? launch_bwd<128>(a, stages, st) : launch_bwd<64>(a, stages, st);
 }
 

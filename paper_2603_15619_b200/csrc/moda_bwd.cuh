@@ -36,6 +36,7 @@ struct BwdArgs {
     int B, T, H, Hk, l;          // H query heads on Hk key/value heads
     float scale;
     void *dQ, *dK, *dV, *d_depth_kv, *workspace;
+    bool accumulate_depth = false;   // add the depth gradients to d_depth_kv instead of overwriting it
 };
 
 inline size_t bwd_workspace_bytes(int B, int T, int H) {
@@ -147,6 +148,7 @@ struct DqParams {
     const float* delta;
     int B, T, H, l;     // H = number of query heads
     int G;              // query heads per key/value head
+    int accumulate;     // nonzero: depth gradients are added to d_depth_kv (bf16 adds in L2)
     // G == 1: the depth gradients are written by this kernel (null here).  G > 1: they are sums
     // over the heads of a group, so the kernel only leaves its per-row factors here, R_i and dU_i
     // as [b][hk][tile][slot][{R, dU}][g][row 128] fp32, and depth_grad_group_kernel forms the sums.
@@ -323,6 +325,7 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             // Grouped-query launches leave R_i and dU_i of this row for depth_grad_group_kernel
             // instead of writing depth gradients (which are sums over the heads of the group).
             const bool store_grads = p.depth_rowterms == nullptr;
+            const bool accumulate = p.accumulate != 0;
             float* rt_row = store_grads ? nullptr
                 : p.depth_rowterms + (((size_t(b) * Hk + hk) * nq + qt) * p.l * 2) * (kTileRows * p.G) + (h - hk * p.G) * kTileRows + r;
             uint4* gK = reinterpret_cast<uint4*>(p.d_depth_kv) + blk;
@@ -412,7 +415,8 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                                 o.y = pack_bf16x2(w * g[8 * c + 2], w * g[8 * c + 3]);
                                 o.z = pack_bf16x2(w * g[8 * c + 4], w * g[8 * c + 5]);
                                 o.w = pack_bf16x2(w * g[8 * c + 6], w * g[8 * c + 7]);
-                                dst[c * kTileRows] = o;
+                                if (accumulate) red_add_bf16x2_v4(dst + c * kTileRows, o);
+                                else dst[c * kTileRows] = o;
                             }
                         }
                     }
@@ -472,7 +476,10 @@ moda_bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                             o.y = mul_bf16x2(qp[c].y, sdu2);
                             o.z = mul_bf16x2(qp[c].z, sdu2);
                             o.w = mul_bf16x2(qp[c].w, sdu2);
-                            if (store_grads) dst[c * kTileRows] = o;
+                            if (store_grads) {
+                                if (accumulate) red_add_bf16x2_v4(dst + c * kTileRows, o);
+                                else dst[c * kTileRows] = o;
+                            }
                         }
                     }
 #pragma unroll
@@ -639,7 +646,7 @@ template <int D, int G>
 __global__ void __launch_bounds__(kGroupGradThreads)
 depth_grad_group_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ dO,
                         const float* __restrict__ rowterms, __nv_bfloat16* __restrict__ d_depth_kv,
-                        int B, int T, int Hk, int l, float scale) {
+                        int B, int T, int Hk, int l, float scale, int accumulate) {
     constexpr int FW = GroupGrad<G>::kFW, SLOTS = GroupGrad<G>::kSlots;
     constexpr int PIECES = D / FW;                       // feature pieces per row
     constexpr int PGROUPS = PIECES / 4;                  // CTAs per (tile, kv)
@@ -710,13 +717,16 @@ depth_grad_group_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16
                 uint4 o;
                 o.x = pack_bf16x2(a[0], a[1]); o.y = pack_bf16x2(a[2], a[3]);
                 o.z = pack_bf16x2(a[4], a[5]); o.w = pack_bf16x2(a[6], a[7]);
-                *reinterpret_cast<uint4*>(dst) = o;
+                if (accumulate) red_add_bf16x2_v4(dst, o);
+                else *reinterpret_cast<uint4*>(dst) = o;
             } else if constexpr (FW == 4) {
                 uint2 o;
                 o.x = pack_bf16x2(a[0], a[1]); o.y = pack_bf16x2(a[2], a[3]);
-                *reinterpret_cast<uint2*>(dst) = o;
+                if (accumulate) red_add_bf16x2_v2(dst, o);
+                else *reinterpret_cast<uint2*>(dst) = o;
             } else {
-                *reinterpret_cast<uint32_t*>(dst) = pack_bf16x2(a[0], a[1]);
+                if (accumulate) red_add_bf16x2(dst, pack_bf16x2(a[0], a[1]));
+                else *reinterpret_cast<uint32_t*>(dst) = pack_bf16x2(a[0], a[1]);
             }
         }
     }

@@ -352,6 +352,18 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 // Two floats -> packed bf16x2 (lo in the low 16 bits), round to nearest even.
+// Adds packed bf16 pairs to global memory (the adds happen in L2; nothing is returned).
+__device__ __forceinline__ void red_add_bf16x2_v4(void* gptr, const uint4& v) {
+    asm volatile("red.global.add.noftz.v4.bf16x2 [%0], {%1, %2, %3, %4};"
+                 :: "l"(gptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void red_add_bf16x2_v2(void* gptr, const uint2& v) {
+    asm volatile("red.global.add.noftz.v2.bf16x2 [%0], {%1, %2};" :: "l"(gptr), "r"(v.x), "r"(v.y) : "memory");
+}
+__device__ __forceinline__ void red_add_bf16x2(void* gptr, uint32_t v) {
+    asm volatile("red.global.add.noftz.bf16x2 [%0], %1;" :: "l"(gptr), "r"(v) : "memory");
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));

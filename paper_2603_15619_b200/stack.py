@@ -4,8 +4,9 @@ In a MoDA model (paper Sec. 2.2, the "write" step) every attention layer appends
 the depth stream after attending, and layer l attends to the l slots written before it.  So K_i, V_i
 of layer i receive gradient from layer i's own sequence attention and, as depth slot i, from every
 later layer.  ``DepthStream`` owns the depth cache and one gradient cache of the same layout and
-wires those contributions together around the C-ABI calls; it is plumbing (no arithmetic of the
-operator happens here beyond adding gradients).
+wires those contributions together around the C-ABI calls (the backward call's accumulate flag adds
+each layer's depth gradients into the shared gradient cache); it is plumbing: no arithmetic of the
+operator happens here beyond adding a slot's gradient to its layer's K, V gradient.
 
     stream = DepthStream(B, T, H_kv, d, n_layers)
     for layer in layers:
@@ -41,12 +42,11 @@ class _Attend(torch.autograd.Function):
         stream, l = ctx.stream, ctx.l
         B, T, H, d = Q.shape
         Hk = K.shape[2]
-        tmp = stream.scratch_grad(l)
-        dQ, dK, dV, _ = binding.moda_attn_bwd_gqa(Q, K, V, stream.cache if l > 0 else None, O, dO.contiguous(), LSE,
-                                                  l, ctx.scale, d_depth_kv=tmp)
-        if l > 0:
-            n = binding.moda_depth_cache_bytes(B, T, Hk, d, l) // 2
-            stream.grad_cache[:n] += tmp[:n]                            # slots < l: add this layer's share
+        # slots < l of the gradient cache receive this layer's share (added in place by the kernel)
+        dQ, dK, dV, _ = binding.moda_attn_bwd_gqa(
+            Q, K, V, stream.cache if l > 0 else None, O, dO.contiguous(), LSE, l, ctx.scale,
+            d_depth_kv=stream.grad_cache if l > 0 else None,
+            stages=binding.MODA_BWD_ALL_STAGES | binding.MODA_BWD_ACCUMULATE_DEPTH)
         if stream.slot_has_grad(l):                                     # later layers attended to slot l
             dKs = torch.empty_like(K)
             dVs = torch.empty_like(V)
@@ -54,6 +54,27 @@ class _Attend(torch.autograd.Function):
             dK += dKs
             dV += dVs
         return dQ, dK, dV, dtoken, None, None, None
+
+
+class _Write(torch.autograd.Function):
+    """A slot written without attending (the FFN-side depth K/V of Sec. 2.2): its gradient is the
+    slot of the gradient cache that the later layers filled."""
+
+    @staticmethod
+    def forward(ctx, K, V, token, stream, slot):
+        K, V = K.contiguous(), V.contiguous()
+        binding.moda_depth_cache_append(stream.cache, slot, K, V)
+        ctx.stream, ctx.slot = stream, slot
+        ctx.save_for_backward(K, V)
+        return token + 0
+
+    @staticmethod
+    def backward(ctx, dtoken):
+        K, V = ctx.saved_tensors
+        dK, dV = torch.zeros_like(K), torch.zeros_like(V)
+        if ctx.stream.slot_has_grad(ctx.slot):
+            binding.moda_depth_cache_unpack(ctx.stream.grad_cache, ctx.slot, dK, dV)
+        return dK, dV, dtoken, None, None
 
 
 class DepthStream:
@@ -64,16 +85,8 @@ class DepthStream:
         self.n_layers = int(n_layers)
         self.cache = binding.alloc_depth_cache(B, T, H_kv, d, n_layers, device)
         self.grad_cache = torch.zeros_like(self.cache)
-        self._scratch = None
         self.n_written = 0
         self.token = torch.zeros((), device=device, requires_grad=True)
-
-    def scratch_grad(self, l):
-        if l == 0:
-            return None
-        if self._scratch is None:
-            self._scratch = torch.empty_like(self.cache)
-        return self._scratch
 
     def slot_has_grad(self, l):
         return l < self.n_written - 1
@@ -88,3 +101,11 @@ class DepthStream:
         O, self.token = _Attend.apply(Q, K, V, self.token, self, l, float(scale))
         self.n_written = l + 1
         return O
+
+    def write(self, K, V):
+        """Appends K, V [B,T,H_kv,d] as the next slot without attending (e.g. an FFN layer's depth K/V)."""
+        slot = self.n_written
+        if slot >= self.n_layers:
+            raise ValueError("more slots than the stream was sized for")
+        self.token = _Write.apply(K, V, self.token, self, slot)
+        self.n_written = slot + 1

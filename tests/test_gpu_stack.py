@@ -49,3 +49,51 @@ def test_stack_gradients_flow_back_through_the_depth_stream(B, T, H, Hk, d, n_la
     for l, L in enumerate(layers):
         assert rel_l2(f64(L["K"].grad), dK_ref[l]) <= TOL_GRAD_REL_L2, f"dK of layer {l}"
         assert rel_l2(f64(L["V"].grad), dV_ref[l]) <= TOL_GRAD_REL_L2, f"dV of layer {l}"
+
+
+@pytest.mark.parametrize("B,T,H,Hk,d,l", [(1, 300, 2, 2, 64, 3), (2, 200, 3, 3, 128, 5), (1, 300, 4, 2, 64, 4),
+                                          (1, 256, 16, 1, 128, 3), (1, 130, 32, 1, 64, 2)])
+def test_accumulate_flag_adds_the_depth_gradients_to_what_the_cache_holds(B, T, H, Hk, d, l):
+    """MODA_BWD_ACCUMULATE_DEPTH: slots [0, l) become bf16(old + gradient), everything else as without the flag."""
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=77, device="cuda")
+    scale = d ** -0.5
+    cache = moda.alloc_depth_cache(B, T, Hk, d, l)
+    for i in range(l):
+        moda.moda_depth_cache_append(cache, i, x["Kd"][i].contiguous(), x["Vd"][i].contiguous())
+    O, LSE = moda.moda_attn_fwd_gqa(x["Q"], x["K"], x["V"], cache, l, scale)
+    plain = moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    old = (torch.randn(plain[3].shape, generator=g, device="cuda") * plain[3].float().std()).to(torch.bfloat16)
+    acc = old.clone()
+    out = moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale, d_depth_kv=acc,
+                                 stages=moda.MODA_BWD_ALL_STAGES | moda.MODA_BWD_ACCUMULATE_DEPTH)
+    assert moda.moda_last_status() == 0
+    for a, b in zip(out[:3], plain[:3]):
+        assert torch.equal(a, b)
+    want = (old.double() + plain[3].double())
+    got = acc.double()
+    ulp = torch.maximum(want.abs(), torch.tensor(1e-30, device="cuda", dtype=torch.float64)) * 2.0 ** -8
+    assert bool(((got - want).abs() <= ulp).all())                       # one bf16 rounding of the exact sum
+    assert float((got != want.to(torch.bfloat16).double()).double().mean()) < 1e-3   # and round-to-nearest almost everywhere
+    # twice more: the cache keeps collecting
+    moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale, d_depth_kv=acc,
+                           stages=moda.MODA_BWD_ALL_STAGES | moda.MODA_BWD_ACCUMULATE_DEPTH)
+    want2 = old.double() + 2 * plain[3].double()
+    assert rel_l2(acc.double().cpu().numpy(), want2.cpu().numpy()) < 1e-2
+
+
+def test_slot_written_without_attending_gets_the_gradients_of_the_layers_after_it():
+    B, T, H, Hk, d = 1, 200, 4, 2, 64
+    scale = d ** -0.5
+    a = synthetic.make_gqa(B, T, H, Hk, d, 0, seed=3, device="cuda")
+    f = synthetic.make_gqa(B, T, H, Hk, d, 0, seed=4, device="cuda")
+    Kf, Vf = f["K"].clone().requires_grad_(), f["V"].clone().requires_grad_()
+    Q, K, V = (a[k].clone().requires_grad_() for k in ("Q", "K", "V"))
+    stream = moda.DepthStream(B, T, Hk, d, 2)
+    stream.write(Kf, Vf)                                   # slot 0
+    O = stream.attend(Q, K, V, scale)                      # attends to slot 0, writes slot 1
+    (O.float() * a["dO"].float()).sum().backward()
+    Kd, Vd = f64(Kf)[None], f64(Vf)[None]
+    dQ, dK, dV, dKd, dVd = orc.backward_gqa(f64(Q), f64(K), f64(V), Kd, Vd, f64(a["dO"]), scale)
+    for got, want in ((Q.grad, dQ), (K.grad, dK), (V.grad, dV), (Kf.grad, dKd[0]), (Vf.grad, dVd[0])):
+        assert rel_l2(f64(got), want) <= TOL_GRAD_REL_L2

@@ -230,3 +230,40 @@ def backward_gqa(Q, K, V, Kd, Vd, dO, scale):
     if rc != 0:
         raise MemoryError("oracle scratch allocation failed")
     return dQ, dK, dV, dKd, dVd
+
+
+# ---------------------------------------------------------------------------------------
+# Decode step (T_q = 1): the newest token of every sequence attends to the T_kv sequence keys of
+# this layer's KV cache (its own included) and to its own l depth key/value pairs, the
+# 2 l H_k d values per token of the paper's complexity table (Table 1, "decoding cache").
+# Written straight from the definition in numpy float64: for the last position the causal mask
+# of Eq. 2 admits every cached key, so the row is one plain softmax over T_kv + l keys.
+# ---------------------------------------------------------------------------------------
+def decode_gqa(q, K, V, kd, vd, scale):
+    """o [B,Hq,d] and lse [B,Hq] for q [B,Hq,d], K, V [B,T_kv,Hk,d], kd, vd [l,B,Hk,d] (or None)."""
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    K = np.ascontiguousarray(K, dtype=np.float64)
+    V = np.ascontiguousarray(V, dtype=np.float64)
+    if q.ndim != 3 or K.ndim != 4 or V.shape != K.shape:
+        raise ValueError("q must be [B, Hq, d]; K, V [B, T_kv, Hk, d]")
+    B, Hq, d = q.shape
+    _, Tkv, Hk, _ = K.shape
+    if K.shape[0] != B or K.shape[3] != d or Hk < 1 or Hq % Hk or Tkv < 1:
+        raise ValueError("K must be [B, T_kv >= 1, Hk, d] with Hk dividing Hq")
+    G = Hq // Hk
+    l = 0 if kd is None else int(np.shape(kd)[0])
+    kd = np.zeros((0, B, Hk, d)) if l == 0 else _f64(kd, (l, B, Hk, d))
+    vd = np.zeros((0, B, Hk, d)) if l == 0 else _f64(vd, (l, B, Hk, d))
+    o = np.empty((B, Hq, d)); lse = np.empty((B, Hq))
+    for b in range(B):
+        for h in range(Hq):
+            hk = h // G
+            keys = np.concatenate([K[b, :, hk, :], kd[:, b, hk, :]], axis=0)      # [T_kv + l, d]
+            vals = np.concatenate([V[b, :, hk, :], vd[:, b, hk, :]], axis=0)
+            s = (keys @ q[b, h]) * float(scale)
+            m = s.max()
+            p = np.exp(s - m)
+            z = p.sum()
+            o[b, h] = (p / z) @ vals
+            lse[b, h] = m + np.log(z)
+    return o, lse

@@ -186,6 +186,30 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
                              void* workspace, size_t workspace_bytes, int stages, void* stream);
 
 /*
+ * Decode step (T_q = 1; Table 1, "decoding cache" and "decoding FLOPs" rows): the newest token of
+ * each of B sequences attends, under one softmax, to the T_kv keys of this layer's KV cache (its
+ * own key included: the caller appends before the call) and to its own l depth key/value pairs,
+ * the 2 l H_k d values that the decoding cache holds per token.  Forward only.
+ *     q, O            : bf16 [B][H][d]
+ *     K, V            : bf16 [B][T_cap][H_kv][d]; positions [0, T_kv) are read, T_kv <= T_cap
+ *     depth_kv_token  : bf16 [l][B][H_kv][2][d]: slot i holds the key row, then the value row, that
+ *                       layer i wrote for this token (may be NULL when l == 0)
+ *     LSE             : fp32 [B][H], natural log over the T_kv + l keys
+ *     workspace       : at least moda_decode_workspace_bytes(B, H, d) bytes, 16-byte aligned; it
+ *                       holds per-split partial softmax states and is overwritten
+ * Query head h uses key/value head h / G with G = H / H_kv in 1..8 (MODA_ERR_BAD_GROUP otherwise).
+ * Two launches on `stream`: a kernel that streams the KV cache once per key/value head (the key
+ * range is split over enough CTAs to fill the device) and a merge kernel that adds the depth pairs.
+ * All pointers are device pointers owned by the caller; validation, asynchrony and error codes are
+ * as for moda_attn_fwd.  The reduction order depends only on (B, H_kv, T_kv) and the device's SM
+ * count, so results are bit-reproducible on one device type.
+ */
+size_t moda_decode_workspace_bytes(int B, int H, int d);
+int moda_attn_decode(const void* q, const void* K, const void* V, const void* depth_kv_token,
+                     int B, int T_kv, int T_cap, int H, int H_kv, int d, int l, float scale,
+                     void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Backward pass for callers that have no scratch buffer to give.  (The paper has no
  * counterpart: this is a deployment convenience of this library, not part of the method.)
  *

@@ -19,10 +19,12 @@ from .binding import (  # noqa: F401
     moda_attn_bwd_gqa_stages,
     moda_attn_bwd_stages,
     moda_attn_bwd_static_scratch,
+    moda_attn_decode,
     moda_attn_fwd,
     moda_attn_fwd_gqa,
     moda_bwd_workspace_bytes,
     moda_bwd_workspace_bytes_gqa,
+    moda_decode_workspace_bytes,
     moda_depth_cache_append,
     moda_depth_cache_bytes,
     moda_depth_cache_unpack,

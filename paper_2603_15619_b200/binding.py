@@ -22,6 +22,7 @@ SYMBOLS = (
     "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd", "moda_attn_bwd_stages",
     "moda_attn_bwd_static_scratch",
     "moda_attn_fwd_gqa", "moda_bwd_workspace_bytes_gqa", "moda_attn_bwd_gqa", "moda_attn_bwd_gqa_stages",
+    "moda_decode_workspace_bytes", "moda_attn_decode",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -79,6 +80,10 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd_gqa.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
     lib.moda_attn_bwd_gqa_stages.restype = ci
     lib.moda_attn_bwd_gqa_stages.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, ci, vp]
+    lib.moda_decode_workspace_bytes.restype = sz
+    lib.moda_decode_workspace_bytes.argtypes = [ci] * 3
+    lib.moda_attn_decode.restype = ci
+    lib.moda_attn_decode.argtypes = [vp] * 4 + [ci] * 7 + [cf] + [vp] * 3 + [sz, vp]
     _lib = lib
     return lib
 
@@ -273,3 +278,32 @@ def moda_attn_bwd_gqa(Q, K, V, depth_kv, O, dO, LSE, l, scale,
 def moda_attn_bwd_gqa_stages(*args, stages, **kwargs):
     """moda_attn_bwd_gqa restricted to the launches selected by the ``stages`` bit mask."""
     return moda_attn_bwd_gqa(*args, stages=stages, **kwargs)
+
+
+def moda_decode_workspace_bytes(B, H, d) -> int:
+    return int(load().moda_decode_workspace_bytes(B, H, d))
+
+
+def moda_attn_decode(q, K, V, depth_kv_token, T_kv, l, scale, O=None, LSE=None, workspace=None, stream=None):
+    """Decode step: q [B,H,d], K, V [B,T_cap,H_kv,d] (positions < T_kv read), depth pairs of the token
+    [l,B,H_kv,2,d] (key row, value row).  Returns O [B,H,d] bf16 and LSE [B,H] fp32."""
+    if q.dtype != torch.bfloat16 or q.dim() != 3:
+        raise ValueError("q must be a bf16 [B, H, d] tensor")
+    B, H, d = q.shape
+    Bk, T_cap, Hk, dk = _bthd(K, "K")
+    if (Bk, dk) != (B, d) or tuple(V.shape) != tuple(K.shape) or V.dtype != torch.bfloat16:
+        raise ValueError("K and V must be bf16 [B, T_cap, H_kv, d] tensors matching q's B and d")
+    if l > 0 and (depth_kv_token is None or tuple(depth_kv_token.shape) != (l, B, Hk, 2, d)
+                  or depth_kv_token.dtype != torch.bfloat16):
+        raise ValueError("depth_kv_token must be a bf16 [l, B, H_kv, 2, d] tensor")
+    if O is None:
+        O = torch.empty_like(q)
+    if LSE is None:
+        LSE = torch.empty((B, H), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(moda_decode_workspace_bytes(B, H, d), dtype=torch.uint8, device=q.device)
+    _check(load().moda_attn_decode(_ptr(q), _ptr(K), _ptr(V), _ptr(depth_kv_token) if l > 0 else None,
+                                   B, int(T_kv), T_cap, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
+                                   _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "moda_attn_decode")
+    return O, LSE

@@ -8,6 +8,7 @@
 
 #include "moda_bwd.cuh"
 #include "moda_cache.cuh"
+#include "moda_decode.cuh"
 #include "moda_fwd.cuh"
 #include "moda_fwd_wide.cuh"
 #include "sm100_ptx.cuh"
@@ -233,6 +234,43 @@ int launch_cache_copy(void* cache, int B, int T, int H, int slot, void* Xk, void
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 
+// Decode step: a split kernel over the KV cache and a merge kernel that adds the depth pairs.
+template <int D, int G>
+int launch_decode_g(const DecodeParams& p, cudaStream_t stream) {
+    decode_split_kernel<D, G><<<dim3(p.S, p.Hk, p.B), kDecodeThreads, 0, stream>>>(p);
+    if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    decode_merge_kernel<D><<<dim3(p.H, p.B), D, 0, stream>>>(p);
+    if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    return MODA_OK;
+}
+template <int D>
+int launch_decode(const DecodeParams& p, cudaStream_t stream) {
+    switch (p.H / p.Hk) {
+        case 1: return launch_decode_g<D, 1>(p, stream);
+        case 2: return launch_decode_g<D, 2>(p, stream);
+        case 3: return launch_decode_g<D, 3>(p, stream);
+        case 4: return launch_decode_g<D, 4>(p, stream);
+        case 5: return launch_decode_g<D, 5>(p, stream);
+        case 6: return launch_decode_g<D, 6>(p, stream);
+        case 7: return launch_decode_g<D, 7>(p, stream);
+        case 8: return launch_decode_g<D, 8>(p, stream);
+        default: return MODA_ERR_BAD_GROUP;
+    }
+}
+
+int device_sm_count(int* out) {
+    static thread_local int cached_dev = -1, cached_sms = 0;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (dev != cached_dev) {
+        int sms = 0;
+        if (!cuda_ok(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev))) return MODA_ERR_CUDA;
+        cached_dev = dev; cached_sms = sms;
+    }
+    *out = cached_sms;
+    return MODA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -384,6 +422,43 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
     a.accumulate_depth = (stages & MODA_BWD_ACCUMULATE_DEPTH) != 0;
     return d == 128 ? launch_bwd<128>(a, stages, st) : launch_bwd<64>(a, stages, st);
+}
+
+size_t moda_decode_workspace_bytes(int B, int H, int d) {
+    if (B < 1 || H < 1 || (d != 64 && d != 128)) return 0;
+    return decode_workspace_bytes(B, H, d);
+}
+
+int moda_attn_decode(const void* q, const void* K, const void* V, const void* depth_kv_token,
+                     int B, int T_kv, int T_cap, int H, int H_kv, int d, int l, float scale,
+                     void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 1 || T_kv < 1 || T_cap < T_kv || H < 1 || B > 65535) return MODA_ERR_BAD_SHAPE;
+    if (d != 64 && d != 128) return MODA_ERR_BAD_HEAD_DIM;
+    if ((long long)B * T_cap > 0x7fffffffLL / H) return MODA_ERR_BAD_SHAPE;
+    if (H_kv < 1 || H % H_kv != 0 || H / H_kv > 8 || H_kv > 65535) return MODA_ERR_BAD_GROUP;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (!q || !K || !V || !O || !LSE || (l > 0 && !depth_kv_token)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
+        (l > 0 && !aligned16(depth_kv_token)))
+        return MODA_ERR_MISALIGNED;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < decode_workspace_bytes(B, H, d)) return MODA_ERR_WORKSPACE;
+    if (int rc = check_device()) return rc;
+    int sms = 0;
+    if (int rc = device_sm_count(&sms)) return rc;
+    DecodeParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.K = static_cast<const __nv_bfloat16*>(K);
+    p.V = static_cast<const __nv_bfloat16*>(V);
+    p.depth = static_cast<const __nv_bfloat16*>(depth_kv_token);
+    p.O = static_cast<__nv_bfloat16*>(O);
+    p.LSE = LSE;
+    p.part = static_cast<float*>(workspace);
+    p.B = B; p.T_kv = T_kv; p.T_cap = T_cap; p.H = H; p.Hk = H_kv; p.l = l;
+    p.S = decode_num_splits(B, H_kv, T_kv, sms);
+    p.keys_per_split = decode_keys_per_split(T_kv, p.S);
+    p.scale_log2 = scale * kDecodeLog2e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_decode<128>(p, st) : launch_decode<64>(p, st);
 }
 
 }  // extern "C"

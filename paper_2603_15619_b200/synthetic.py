@@ -105,3 +105,21 @@ def make_gqa(B: int, T: int, H: int, H_kv: int, d: int, l: int, seed: int = 0, d
     out["Q"] = tensor(wq, "Q", seed, 0, device)
     out["dO"] = tensor(wq, "dO", seed, 0, device)
     return out
+
+
+def make_decode(B: int, T_kv: int, H: int, H_kv: int, d: int, l: int, seed: int = 0, device="cpu", T_cap=None, **kw) -> dict:
+    """Inputs of a decode step: q [B,H,d]; K, V [B,T_cap,H_kv,d] (the KV cache of one layer, positions
+    < T_kv meaningful); depth [l,B,H_kv,2,d] (key row, value row of the token's depth pairs).  Same
+    distributions as the training-shape tensors."""
+    T_cap = T_kv if T_cap is None else T_cap
+    wk = Workload("decode/kv", B, T_cap, H_kv, d, l, **kw)
+    wq = Workload("decode/q", B, 1, H, d, l, **kw)
+    wd = Workload("decode/depth", B, 1, H_kv, d, l, **kw)
+    out = {"q": tensor(wq, "Q", seed, 0, device)[:, 0].contiguous(),
+           "K": tensor(wk, "K", seed, 0, device), "V": tensor(wk, "V", seed, 0, device)}
+    depth = torch.empty((l, B, H_kv, 2, d), dtype=torch.bfloat16, device=device)
+    for i in range(l):
+        depth[i, :, :, 0] = tensor(wd, "Kd", seed, i, device)[:, 0]
+        depth[i, :, :, 1] = tensor(wd, "Vd", seed, i, device)[:, 0]
+    out["depth"] = depth
+    return out

@@ -85,3 +85,22 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(ImportError):
         binding.load()
+
+
+def test_decode_entry_point_validates_before_touching_the_device():
+    lib = binding.load()
+    p = ctypes.c_void_p(4096)
+    ws = lib.moda_decode_workspace_bytes(1, 8, 128)
+    assert ws >= 8 * 130 * 4 and lib.moda_decode_workspace_bytes(1, 8, 96) == 0
+
+    def call(B=1, T_kv=10, T_cap=16, H=8, Hk=2, d=128, l=2, q=p, depth=p, work=p, wb=None):
+        return lib.moda_attn_decode(q, p, p, depth, B, T_kv, T_cap, H, Hk, d, l, ctypes.c_float(0.1), p, p, work,
+                                    ctypes.c_size_t(ws if wb is None else wb), None)
+
+    assert call(T_kv=0) == -3 and call(T_kv=17) == -3 and call(B=0) == -3
+    assert call(d=96) == -4
+    assert call(l=-1) == -5 and call(l=257) == -5
+    assert call(H=8, Hk=3) == -12 and call(H=16, Hk=1) == -12 and call(Hk=0) == -12
+    assert call(q=None) == -1 and call(depth=None) == -1 and call(l=0, depth=None) != -1
+    assert call(q=ctypes.c_void_p(4100)) == -2
+    assert call(work=None) == -7 and call(wb=16) == -7

@@ -1,0 +1,78 @@
+"""Decode step (T_q = 1) on the GPU against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2603_15619_b200 as moda
+from paper_2603_15619_b200 import synthetic
+from oracle import moda_oracle as orc
+
+from parity import TOL_LSE_ABS, TOL_O_MAX_ABS, TOL_O_REL_L2, f64, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    # B, T_kv, T_cap, H, H_kv, d, l
+    (1, 1, 1, 1, 1, 64, 0), (1, 1, 8, 2, 1, 128, 3), (2, 31, 31, 4, 2, 64, 2), (1, 255, 300, 2, 2, 128, 5),
+    (2, 256, 256, 8, 1, 64, 4), (1, 257, 512, 6, 2, 128, 1), (3, 1000, 1024, 4, 4, 64, 7), (1, 5000, 5000, 8, 2, 128, 24),
+    (2, 4097, 4100, 16, 2, 64, 64), (1, 20000, 20000, 3, 1, 128, 256), (1, 3000, 3000, 5, 1, 64, 0), (1, 777, 777, 7, 1, 128, 9),
+]
+
+
+def run(x, T_kv, l, scale):
+    O, LSE = moda.moda_attn_decode(x["q"], x["K"], x["V"], x["depth"] if l else None, T_kv, l, scale)
+    assert moda.moda_last_status() == 0
+    return O, LSE
+
+
+@pytest.mark.parametrize("B,T_kv,T_cap,H,Hk,d,l", SHAPES)
+def test_decode_matches_the_oracle(B, T_kv, T_cap, H, Hk, d, l):
+    x = synthetic.make_decode(B, T_kv, H, Hk, d, l, seed=11, device="cuda", T_cap=T_cap)
+    scale = d ** -0.5
+    O, LSE = run(x, T_kv, l, scale)
+    kd = f64(x["depth"][:, :, :, 0]) if l else None
+    vd = f64(x["depth"][:, :, :, 1]) if l else None
+    o_ref, lse_ref = orc.decode_gqa(f64(x["q"]), f64(x["K"][:, :T_kv]), f64(x["V"][:, :T_kv]), kd, vd, scale)
+    assert rel_l2(f64(O), o_ref) <= TOL_O_REL_L2
+    assert np.abs(f64(O) - o_ref).max() <= TOL_O_MAX_ABS
+    assert np.abs(f64(LSE) - lse_ref).max() <= TOL_LSE_ABS
+
+
+def test_decode_ignores_cache_rows_past_t_kv_and_is_repeatable():
+    B, T_kv, T_cap, H, Hk, d, l = 2, 700, 1024, 8, 2, 128, 6
+    x = synthetic.make_decode(B, T_kv, H, Hk, d, l, seed=2, device="cuda", T_cap=T_cap)
+    O1, L1 = run(x, T_kv, l, d ** -0.5)
+    x["K"][:, T_kv:] = float("nan")
+    x["V"][:, T_kv:] = float("nan")
+    O2, L2 = run(x, T_kv, l, d ** -0.5)
+    assert torch.equal(O1, O2) and torch.equal(L1, L2)
+
+
+def test_decode_equals_the_last_row_of_the_training_forward():
+    """The same operator: the decode step of the last position reproduces the full forward's last row."""
+    B, T, H, Hk, d, l = 1, 600, 4, 2, 128, 5
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=9, device="cuda")
+    scale = d ** -0.5
+    cache = moda.alloc_depth_cache(B, T, Hk, d, l)
+    for i in range(l):
+        moda.moda_depth_cache_append(cache, i, x["Kd"][i].contiguous(), x["Vd"][i].contiguous())
+    O, LSE = moda.moda_attn_fwd_gqa(x["Q"], x["K"], x["V"], cache, l, scale)
+    depth = torch.stack([x["Kd"][:, :, -1], x["Vd"][:, :, -1]], dim=3).contiguous()       # [l,B,Hk,2,d]
+    o, lse = moda.moda_attn_decode(x["Q"][:, -1].contiguous(), x["K"], x["V"], depth, T, l, scale)
+    assert np.abs(f64(o) - f64(O[:, -1])).max() <= 2e-2
+    assert np.abs(f64(lse) - f64(LSE[:, :, -1])).max() <= 2e-3
+
+
+def test_decode_guard_bands_stay_intact():
+    B, T_kv, H, Hk, d, l = 1, 900, 4, 1, 64, 3
+    x = synthetic.make_decode(B, T_kv, H, Hk, d, l, seed=4, device="cuda")
+    pad = 64
+    Obuf = torch.full((B * H * d + 2 * pad,), 7.0, dtype=torch.bfloat16, device="cuda")
+    Lbuf = torch.full((B * H + 2 * pad,), 7.0, dtype=torch.float32, device="cuda")
+    O = Obuf[pad:pad + B * H * d].view(B, H, d)
+    LSE = Lbuf[pad:pad + B * H].view(B, H)
+    moda.moda_attn_decode(x["q"], x["K"], x["V"], x["depth"], T_kv, l, d ** -0.5, O=O, LSE=LSE)
+    torch.cuda.synchronize()
+    for buf, n in ((Obuf, B * H * d), (Lbuf, B * H)):
+        assert bool((buf[:pad] == 7.0).all()) and bool((buf[pad + n:] == 7.0).all())
+    assert not bool((O == 7.0).all())

@@ -305,6 +305,7 @@ def run_moda(args, rank, world, device):
     if rank == 0 and world == 1 and not args.no_sweep:
         out["sweep"] = run_sweep(peaks, device, layer)
         out["gqa_sweep"] = run_gqa_sweep(device)
+        out["decode_sweep"] = run_decode_sweep(peaks, device)
     if not args.no_e2e:
         out["e2e"] = run_e2e(layer, min(K, 8), world, step_flops, device)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -428,6 +429,50 @@ def run_gqa_sweep(device, shapes=None):
                      "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f1 + b1), 4),
                      "fwd_tflops": round(ff / f1 / 1e9, 1), "fwd_bwd_tflops": round(3.5 * ff / (f1 + b1) / 1e9, 1)})
         log("gqa_sweep", rows[-1])
+    torch.cuda.empty_cache()
+    return rows
+
+
+# Decode step (T_q = 1): B sequences x T_kv cached positions; the paper's 700M / 1.5B models use G = 2.
+# (B, T_kv, H, H_kv, d, l); every KV cache here is larger than L2.
+DECODE_SHAPES = [
+    (32, 8192, 16, 16, 128, 24), (32, 8192, 16, 8, 128, 24), (32, 8192, 32, 8, 128, 24), (32, 8192, 64, 8, 128, 24),
+    (64, 8192, 16, 8, 64, 32), (128, 2048, 16, 8, 128, 24), (2, 131072, 16, 8, 128, 24),
+]
+
+
+def run_decode_sweep(peaks, device, shapes=None, iters=10):
+    """One decode step per shape: time of the two launches and the HBM bytes they must move (K and V of the
+    cached positions once, the token's depth pairs, q and O) against the measured copy bandwidth."""
+    import paper_2603_15619_b200 as moda
+    rows = []
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    for B, T, H, Hk, d, l in (shapes or DECODE_SHAPES):
+        torch.cuda.empty_cache()
+        x = synthetic.make_decode(B, T, H, Hk, d, l, seed=0, device=device)
+        O = torch.empty_like(x["q"])
+        LSE = torch.empty((B, H), dtype=torch.float32, device=device)
+        ws = torch.empty(moda.moda_decode_workspace_bytes(B, H, d), dtype=torch.uint8, device=device)
+        fn = lambda: moda.moda_attn_decode(x["q"], x["K"], x["V"], x["depth"] if l else None, T, l, d ** -0.5,
+                                           O=O, LSE=LSE, workspace=ws)
+        for _ in range(3):
+            fn()
+        ts = []
+        for _ in range(iters):
+            flush.zero_()                                  # L2 holds nothing of the KV cache when the step starts
+            a, b = ev(), ev()
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        ms = sorted(ts)[len(ts) // 2]
+        byt = 2 * B * T * Hk * d * 2 + 2 * l * B * Hk * d * 2 + 2 * B * H * d * 2
+        gbs = byt / ms / 1e6
+        rows.append({"B": B, "T_kv": T, "H": H, "H_kv": Hk, "G": H // Hk, "d": d, "l": l, "us": round(ms * 1e3, 1),
+                     "algorithmic_GB": round(byt / 1e9, 3), "GBps": round(gbs, 0),
+                     "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 3),
+                     "tokens_per_s": round(B / ms * 1e3, 0)})
+        log("decode_sweep", rows[-1])
+        del x, O, LSE, ws
     torch.cuda.empty_cache()
     return rows
 
@@ -568,6 +613,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gqa-shape", default="", help="T,G[,L]: time only this grouped-query shape (B=1, d=64, 8 key/value "
                                                     "heads, L depth slots (default 32) and l=0) and print its row; for profiling")
+    ap.add_argument("--decode-shape", default="", help="B,T_kv,H,H_kv,d,l: time only this decode step and print its row; for profiling")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -591,6 +637,9 @@ def main():
         if args.gqa_shape:
             v = [int(t) for t in args.gqa_shape.split(",")]
             out = {"gqa_sweep": run_gqa_sweep(device, [(v[0], v[1], v[2] if len(v) > 2 else 32, None)])}
+        elif args.decode_shape:
+            v = tuple(int(t) for t in args.decode_shape.split(","))
+            out = {"decode_sweep": run_decode_sweep(load_peaks(), device, [v], iters=max(1, min(args.steps, 10)))}
         else:
             out = run_moda(args, rank, world, device)
         if rank == 0:

@@ -237,7 +237,19 @@ int launch_cache_copy(void* cache, int B, int T, int H, int slot, void* Xk, void
 // Decode step: a split kernel over the KV cache and a merge kernel that adds the depth pairs.
 template <int D, int G>
 int launch_decode_g(const DecodeParams& p, cudaStream_t stream) {
-    decode_split_kernel<D, G><<<dim3(p.S, p.Hk, p.B), kDecodeThreads, 0, stream>>>(p);
+    using L = DecodeSmem<D, G>;
+    CUtensorMap mK, mV;
+    if (!make_bthd_map(&mK, p.K, p.B, p.T_cap, p.Hk, D, kDecodeStageKeys) ||
+        !make_bthd_map(&mV, p.V, p.B, p.T_cap, p.Hk, D, kDecodeStageKeys))
+        return MODA_ERR_CUDA;
+    static thread_local int configured_dev = -1;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (configured_dev != dev) {
+        if (!set_smem_limit(decode_split_tma_kernel<D, G>, L::kDynamic)) return MODA_ERR_CUDA;
+        configured_dev = dev;
+    }
+    decode_split_tma_kernel<D, G><<<dim3(p.S, p.Hk, p.B), kDecodeTmaThreads, L::kDynamic, stream>>>(mK, mV, p);
     if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     decode_merge_kernel<D><<<dim3(p.H, p.B), D, 0, stream>>>(p);
     if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;

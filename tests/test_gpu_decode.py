@@ -16,6 +16,8 @@ SHAPES = [
     (1, 1, 1, 1, 1, 64, 0), (1, 1, 8, 2, 1, 128, 3), (2, 31, 31, 4, 2, 64, 2), (1, 255, 300, 2, 2, 128, 5),
     (2, 256, 256, 8, 1, 64, 4), (1, 257, 512, 6, 2, 128, 1), (3, 1000, 1024, 4, 4, 64, 7), (1, 5000, 5000, 8, 2, 128, 24),
     (2, 4097, 4100, 16, 2, 64, 64), (1, 20000, 20000, 3, 1, 128, 256), (1, 3000, 3000, 5, 1, 64, 0), (1, 777, 777, 7, 1, 128, 9),
+    # many (batch, kv head) groups: few splits, so every CTA goes round its shared-memory ring several times
+    (16, 4096, 4096, 16, 8, 128, 4), (24, 6000, 6016, 16, 8, 64, 3), (40, 2500, 2500, 8, 8, 128, 2),
 ]
 
 
@@ -76,3 +78,26 @@ def test_decode_guard_bands_stay_intact():
     for buf, n in ((Obuf, B * H * d), (Lbuf, B * H)):
         assert bool((buf[:pad] == 7.0).all()) and bool((buf[pad + n:] == 7.0).all())
     assert not bool((O == 7.0).all())
+
+
+def test_back_to_back_decode_steps_are_bitwise_repeatable():
+    """Twenty steps queued without a host sync in between (more CTAs than SMs, ring wrapping): same bits each time."""
+    B, T_kv, H, Hk, d, l = 32, 8192, 16, 8, 128, 24
+    x = synthetic.make_decode(B, T_kv, H, Hk, d, l, seed=1, device="cuda")
+    ws = torch.empty(moda.moda_decode_workspace_bytes(B, H, d), dtype=torch.uint8, device="cuda")
+    outs = []
+    for _ in range(20):
+        O = torch.empty_like(x["q"])
+        LSE = torch.empty((B, H), dtype=torch.float32, device="cuda")
+        moda.moda_attn_decode(x["q"], x["K"], x["V"], x["depth"], T_kv, l, d ** -0.5, O=O, LSE=LSE, workspace=ws)
+        outs.append((O, LSE))
+    torch.cuda.synchronize()
+    assert moda.moda_last_status() == 0
+    for O, LSE in outs[1:]:
+        assert torch.equal(O, outs[0][0]) and torch.equal(LSE, outs[0][1])
+    # sampled rows against the oracle
+    for b in (0, 17, 31):
+        o_ref, lse_ref = orc.decode_gqa(f64(x["q"][b:b + 1]), f64(x["K"][b:b + 1]), f64(x["V"][b:b + 1]),
+                                        f64(x["depth"][:, b:b + 1, :, 0]), f64(x["depth"][:, b:b + 1, :, 1]), d ** -0.5)
+        assert rel_l2(f64(outs[0][0][b:b + 1]), o_ref) <= TOL_O_REL_L2
+        assert np.abs(f64(outs[0][1][b:b + 1]) - lse_ref).max() <= TOL_LSE_ABS

@@ -441,30 +441,36 @@ DECODE_SHAPES = [
 ]
 
 
-def run_decode_sweep(peaks, device, shapes=None, iters=10):
+def run_decode_sweep(peaks, device, shapes=None, iters=20):
     """One decode step per shape: time of the two launches and the HBM bytes they must move (K and V of the
     cached positions once, the token's depth pairs, q and O) against the measured copy bandwidth."""
     import paper_2603_15619_b200 as moda
     rows = []
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
     for B, T, H, Hk, d, l in (shapes or DECODE_SHAPES):
         torch.cuda.empty_cache()
-        x = synthetic.make_decode(B, T, H, Hk, d, l, seed=0, device=device)
-        O = torch.empty_like(x["q"])
+        # Steps are queued back to back (a step is shorter than the host's launch path when timed alone) and
+        # rotate over copies of the KV cache that together exceed L2 several times, so every step reads HBM.
+        kv_bytes = 2 * B * T * Hk * d * 2
+        n_sets = max(2, int(1.0e9 // kv_bytes) + 1) if kv_bytes < 1.0e9 else 1
+        sets = [synthetic.make_decode(B, T, H, Hk, d, l, seed=i, device=device) for i in range(n_sets)]
+        O = torch.empty_like(sets[0]["q"])
         LSE = torch.empty((B, H), dtype=torch.float32, device=device)
         ws = torch.empty(moda.moda_decode_workspace_bytes(B, H, d), dtype=torch.uint8, device=device)
-        fn = lambda: moda.moda_attn_decode(x["q"], x["K"], x["V"], x["depth"] if l else None, T, l, d ** -0.5,
-                                           O=O, LSE=LSE, workspace=ws)
-        for _ in range(3):
-            fn()
-        ts = []
-        for _ in range(iters):
-            flush.zero_()                                  # L2 holds nothing of the KV cache when the step starts
-            a, b = ev(), ev()
-            a.record(); fn(); b.record()
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b))
-        ms = sorted(ts)[len(ts) // 2]
+
+        def fn(i):
+            x = sets[i % n_sets]
+            moda.moda_attn_decode(x["q"], x["K"], x["V"], x["depth"] if l else None, T, l, d ** -0.5,
+                                  O=O, LSE=LSE, workspace=ws)
+        for i in range(max(3, n_sets)):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record()
+        for i in range(iters):
+            fn(i)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / iters
         byt = 2 * B * T * Hk * d * 2 + 2 * l * B * Hk * d * 2 + 2 * B * H * d * 2
         gbs = byt / ms / 1e6
         rows.append({"B": B, "T_kv": T, "H": H, "H_kv": Hk, "G": H // Hk, "d": d, "l": l, "us": round(ms * 1e3, 1),
@@ -472,7 +478,7 @@ def run_decode_sweep(peaks, device, shapes=None, iters=10):
                      "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 3),
                      "tokens_per_s": round(B / ms * 1e3, 0)})
         log("decode_sweep", rows[-1])
-        del x, O, LSE, ws
+        del sets, O, LSE, ws
     torch.cuda.empty_cache()
     return rows
 
@@ -639,7 +645,7 @@ def main():
             out = {"gqa_sweep": run_gqa_sweep(device, [(v[0], v[1], v[2] if len(v) > 2 else 32, None)])}
         elif args.decode_shape:
             v = tuple(int(t) for t in args.decode_shape.split(","))
-            out = {"decode_sweep": run_decode_sweep(load_peaks(), device, [v], iters=max(1, min(args.steps, 10)))}
+            out = {"decode_sweep": run_decode_sweep(load_peaks(), device, [v], iters=max(1, min(args.steps, 20)))}
         else:
             out = run_moda(args, rank, world, device)
         if rank == 0:

@@ -249,7 +249,10 @@ int launch_decode_g(const DecodeParams& p, cudaStream_t stream) {
         if (!set_smem_limit(decode_split_tma_kernel<D, G>, L::kDynamic)) return MODA_ERR_CUDA;
         configured_dev = dev;
     }
-    decode_split_tma_kernel<D, G><<<dim3(p.S, p.Hk, p.B), kDecodeTmaThreads, L::kDynamic, stream>>>(mK, mV, p);
+    // persistent: one CTA per SM (or per work item when there are fewer)
+    const long long items = (long long)p.B * p.Hk * p.S;
+    const unsigned grid = unsigned(items < p.num_sms ? items : p.num_sms);
+    decode_split_tma_kernel<D, G><<<grid, kDecodeTmaThreads, L::kDynamic, stream>>>(mK, mV, p);
     if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     decode_merge_kernel<D><<<dim3(p.H, p.B), D, 0, stream>>>(p);
     if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
@@ -444,10 +447,11 @@ size_t moda_decode_workspace_bytes(int B, int H, int d) {
 int moda_attn_decode(const void* q, const void* K, const void* V, const void* depth_kv_token,
                      int B, int T_kv, int T_cap, int H, int H_kv, int d, int l, float scale,
                      void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream) {
-    if (B < 1 || T_kv < 1 || T_cap < T_kv || H < 1 || B > 65535) return MODA_ERR_BAD_SHAPE;
+    if (B < 1 || T_kv < 1 || T_cap < T_kv || H < 1) return MODA_ERR_BAD_SHAPE;
     if (d != 64 && d != 128) return MODA_ERR_BAD_HEAD_DIM;
     if ((long long)B * T_cap > 0x7fffffffLL / H) return MODA_ERR_BAD_SHAPE;
-    if (H_kv < 1 || H % H_kv != 0 || H / H_kv > 8 || H_kv > 65535) return MODA_ERR_BAD_GROUP;
+    if (H_kv < 1 || H % H_kv != 0 || H / H_kv > 8) return MODA_ERR_BAD_GROUP;
+    if ((long long)B * H_kv * kDecodeMaxSplits > 0x7fffffffLL || B > 65535) return MODA_ERR_BAD_SHAPE;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!q || !K || !V || !O || !LSE || (l > 0 && !depth_kv_token)) return MODA_ERR_NULL_POINTER;
     if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
@@ -466,8 +470,8 @@ int moda_attn_decode(const void* q, const void* K, const void* V, const void* de
     p.LSE = LSE;
     p.part = static_cast<float*>(workspace);
     p.B = B; p.T_kv = T_kv; p.T_cap = T_cap; p.H = H; p.Hk = H_kv; p.l = l;
-    p.S = decode_num_splits(B, H_kv, T_kv, sms);
-    p.keys_per_split = decode_keys_per_split(T_kv, p.S);
+    const DecodePlan plan = decode_plan(B, H_kv, T_kv, sms);
+    p.S = plan.S; p.keys_per_split = plan.keys_per_split; p.num_sms = sms;
     p.scale_log2 = scale * kDecodeLog2e;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return d == 128 ? launch_decode<128>(p, st) : launch_decode<64>(p, st);

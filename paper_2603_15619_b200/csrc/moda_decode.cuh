@@ -3,18 +3,19 @@
 // KV cache and to its own l depth key/value pairs (2 l H_k d values per token).
 //
 // The step reads every cached K and V row once and does 4 G d FLOPs per row, so it is bound by
-// HBM; there is no contraction worth a tensor-core tile (G <= 8 query rows share a key).
+// HBM; G <= 8 query rows share a key, too few for a tcgen05 tile (64 or 128 rows).
 //
 //   decode_split_tma_kernel  persistent, one CTA per SM, over work items (batch, kv head, split of the key
 //                         range).  A producer lane keeps a ring of TMA stages (64 keys: their K rows and V
 //                         rows as 128-byte-swizzled boxes) in flight, 128 KiB per SM, and runs ahead into
 //                         the CTA's next work item, so the HBM stream does not stop at item boundaries.
-//                         Eight consumer warps: scores with one key per lane (the lane reads its key's row
-//                         from shared memory; q sits in shared memory, pre-scaled, read as broadcasts), so
-//                         no reduction across lanes; values with lanes across features, the keys' weights
-//                         broadcast through shared memory.  Each warp keeps an online-softmax state
-//                         (m, l, o) per head; at the end of an item the warps are merged through shared
-//                         memory and the CTA writes one partial (m, l, o[d]) per head.
+//                         Eight consumer warps, 32 keys of a stage each: scores and weighted values with
+//                         warp-level MMAs whose 16-row operand holds the G <= 8 heads of the group (the
+//                         CUDA-core form of the same arithmetic is issue-bound from G = 4 on); K pieces
+//                         and, through transposing matrix loads, V pieces come from the swizzled stage.
+//                         Each warp keeps an online-softmax state (m, l, o) per head; at the end of an
+//                         item the warps are merged through shared memory and the CTA writes one partial
+//                         (m, l, o[d]) per head.
 //   decode_merge_kernel   grid (query head, batch): merges the partials of all splits with the l
 //                         depth pairs of the token (scored here: l d-length dot products) and writes
 //                         O (bf16) and LSE (natural log).
@@ -74,15 +75,17 @@ inline size_t decode_workspace_bytes(int B, int H, int d) {
     return size_t(B) * H * kDecodeMaxSplits * (d + 2) * 4;
 }
 
-// Shared-memory read that the compiler may not hoist out of the key loop: q is loop-invariant, and
-// keeping G * d floats of it in registers spills.
-__device__ __forceinline__ float4 lds_f32x4(const float* ptr) {
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(ptr)))
-                 : "memory");
-    return v;
+// Warp-level tensor-core primitives (bf16 inputs, fp32 accumulate).  The decode step is bound by HBM and
+// its contraction has at most 8 rows, far below the 64 / 128 rows of a tcgen05 tile.
+__device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t smem_addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(smem_addr) : "memory");
 }
 
 constexpr int kDecodeStageKeys = 64;
@@ -100,9 +103,8 @@ struct DecodeSmem {
     // not when pairs alternate on a slot and one of them runs ahead.)
     static constexpr int kStages = (D == 64 ? 2 : 1) * kDecodePairs;           // 128 KiB in flight
     static constexpr int kRing = 0;
-    static constexpr int kQ = kStages * kStageBytes;                           // two buffers: this item's q, the next one's
-    static constexpr int kP = kQ + 2 * G * D * 4;
-    static constexpr int kO = kP + kDecodeConsumerWarps * G * 32 * 4;          // per-warp outputs for the merge
+    static constexpr int kQ = kStages * kStageBytes;                           // two buffers of 8 bf16 rows: this item's q, the next one's
+    static constexpr int kO = kQ + 2 * 8 * D * 2;                              // per-warp outputs for the merge
     static constexpr int kM = kO + kDecodeConsumerWarps * G * D * 4;
     static constexpr int kL = kM + kDecodeConsumerWarps * G * 4;
     static constexpr int kBars = kL + kDecodeConsumerWarps * G * 4;           // full[8], empty[8], abort word
@@ -122,11 +124,9 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
     using L = DecodeSmem<D, G>;
     constexpr int CH = D / 8, FPL = D / 32, NH = D / 64;                     // NH 64-feature boxes per row
     constexpr int kBoxBytes = kDecodeStageKeys * 128;
-    constexpr int QPT = (G * D + kDecodeConsumerThreads - 1) / kDecodeConsumerThreads;   // q elements per consumer thread
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float* s_qbuf = reinterpret_cast<float*>(smem + L::kQ);
-    float* s_p = reinterpret_cast<float*>(smem + L::kP);
+    uint4* s_qbuf = reinterpret_cast<uint4*>(smem + L::kQ);
     float* s_o = reinterpret_cast<float*>(smem + L::kO);
     float* s_m = reinterpret_cast<float*>(smem + L::kM);
     float* s_l = reinterpret_cast<float*>(smem + L::kL);
@@ -185,49 +185,45 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
         }
     } else {
         // ---- consumers: warp pair `pair` takes the stages whose running index is pair mod 4 (always the
-        //      same ring slots); this warp its `half` of a stage's 64 keys ----
+        //      same ring slots); this warp its `half` (32 keys) of a stage's 64 keys ----
+        // Warp-level MMA m16n8k16 with the G <= 8 heads as rows 0..7 of the 16-row operand (rows 8..15
+        // are zero).  Lane = (g, t) = (lane / 4, lane % 4): g is the head for A / C rows and the key or
+        // feature for B columns.
         const int pair = warp >> 1, half = warp & 1;
-        float* my_p = s_p + warp * G * 32;
+        const int g = lane >> 2, t = lane & 3;
         const int ctid = threadIdx.x;                                    // 0 .. 255
-        // q of an item, scaled into the log2 domain, for buffer `buf`
-        auto fetch_q = [&](const Item& w, float (&qr)[QPT]) {
-#pragma unroll
-            for (int k = 0; k < QPT; ++k) {
-                const int e = ctid + k * kDecodeConsumerThreads;
-                qr[k] = e < G * D ? __bfloat162float(p.q[(size_t(w.b) * p.H + w.hk * G) * D + e]) * p.scale_log2 : 0.f;
-            }
+        // q rows (bf16, heads 0..7, zero beyond G) of an item: one 16-byte piece per thread
+        auto fetch_q = [&](const Item& w) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            const int row = ctid / CH, piece = ctid % CH;
+            if (ctid < 8 * CH && row < G)
+                v = *reinterpret_cast<const uint4*>(p.q + (size_t(w.b) * p.H + w.hk * G + row) * D + piece * 8);
+            return v;
         };
-        auto store_q = [&](int buf, const float (&qr)[QPT]) {
-#pragma unroll
-            for (int k = 0; k < QPT; ++k) {
-                const int e = ctid + k * kDecodeConsumerThreads;
-                if (e < G * D) s_qbuf[buf * G * D + e] = qr[k];
-            }
+        auto store_q = [&](int buf, const uint4& v) {
+            if (ctid < 8 * CH) s_qbuf[buf * 8 * CH + ctid] = v;
         };
         int qb = 0;
         int gi0 = 0;                                                     // running stage index at the start of the item
-        if (blockIdx.x < n_items) {
-            float qr[QPT];
-            fetch_q(item_of(blockIdx.x), qr);
-            store_q(0, qr);
-        }
+        if (blockIdx.x < n_items) store_q(0, fetch_q(item_of(blockIdx.x)));
         decode_consumer_sync();
 #pragma unroll 1
         for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
             const Item w = item_of(it);
-            const float* s_q = s_qbuf + qb * G * D;
-            float qnext[QPT];
             const bool has_next = it + gridDim.x < n_items;
-            if (has_next) fetch_q(item_of(it + gridDim.x), qnext);         // lands while this item is processed
+            uint4 qnext = make_uint4(0u, 0u, 0u, 0u);
+            if (has_next) qnext = fetch_q(item_of(it + gridDim.x));       // lands while this item is processed
+            // A fragments of q: for every 32 features, this lane's 8 features of head g (the same 8 features
+            // that it takes from a key row below, so the pairing inside the MMA is consistent)
+            uint4 qf[D / 32];
+#pragma unroll
+            for (int kp = 0; kp < D / 32; ++kp) qf[kp] = s_qbuf[qb * 8 * CH + g * CH + 4 * kp + t];
 
-            float m[G], lsum[G], o[G][FPL];
+            float m_run = -INFINITY, lsum = 0.f;                         // of head g (same in the 4 lanes of a quad, lsum partial)
+            float o[D / 8][4];                                           // [feature block][c0 c1: head g, features 2t, 2t+1; c2 c3 unused rows]
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                m[g] = -INFINITY; lsum[g] = 0.f;
-#pragma unroll
-                for (int c = 0; c < FPL; ++c) o[g][c] = 0.f;
-            }
-            // first stage of this item that belongs to this pair
+            for (int fb = 0; fb < D / 8; ++fb) { o[fb][0] = 0.f; o[fb][1] = 0.f; o[fb][2] = 0.f; o[fb][3] = 0.f; }
+
             const int first = (pair - (gi0 % kDecodePairs) + kDecodePairs) % kDecodePairs;
 #pragma unroll 1
             for (int i = first; i < w.n_stage; i += kDecodePairs) {
@@ -240,81 +236,70 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
                 const int k0 = w.k_begin + i * kDecodeStageKeys + half * 32;   // first key of this warp
                 const int n = min(32, w.k_end - k0);                           // <= 0: second half of a short last stage
                 if (live && n > 0) {
-                    const uint8_t* sK = smem + L::kRing + st * L::kStageBytes;
-                    const uint8_t* sV = sK + NH * kBoxBytes;
-                    const int r = half * 32 + lane;                            // row of this lane's key in the stage
-                    const bool valid = lane < n;
-                    float sa[G], sb[G];
-#pragma unroll
-                    for (int g = 0; g < G; ++g) { sa[g] = 0.f; sb[g] = 0.f; }
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) {
-                        const uint4 kv = *reinterpret_cast<const uint4*>(sK + (c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
-                        const float k0f = bf16_lo_to_f32(kv.x), k1f = bf16_hi_to_f32(kv.x);
-                        const float k2f = bf16_lo_to_f32(kv.y), k3f = bf16_hi_to_f32(kv.y);
-                        const float k4f = bf16_lo_to_f32(kv.z), k5f = bf16_hi_to_f32(kv.z);
-                        const float k6f = bf16_lo_to_f32(kv.w), k7f = bf16_hi_to_f32(kv.w);
-#pragma unroll
-                        for (int g = 0; g < G; ++g) {
-                            const float4 qa = lds_f32x4(&s_q[g * D + 8 * c]);
-                            const float4 qb4 = lds_f32x4(&s_q[g * D + 8 * c + 4]);
-                            sa[g] = fmaf(qa.x, k0f, sa[g]); sb[g] = fmaf(qa.y, k1f, sb[g]);
-                            sa[g] = fmaf(qa.z, k2f, sa[g]); sb[g] = fmaf(qa.w, k3f, sb[g]);
-                            sa[g] = fmaf(qb4.x, k4f, sa[g]); sb[g] = fmaf(qb4.y, k5f, sb[g]);
-                            sa[g] = fmaf(qb4.z, k6f, sa[g]); sb[g] = fmaf(qb4.w, k7f, sb[g]);
+                    uint8_t* sK = smem + L::kRing + st * L::kStageBytes;
+                    uint8_t* sV = sK + NH * kBoxBytes;
+                    if (n < 32) {
+                        // value rows past the end may hold anything (even NaN): zero them, their weights are 0
+                        for (int idx = lane; idx < (32 - n) * CH; idx += 32) {
+                            const int row = half * 32 + n + idx / CH, piece = idx % CH;
+                            *reinterpret_cast<uint4*>(sV + (piece >> 3) * kBoxBytes + row * 128 + ((piece & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
                         }
+                        __syncwarp();
                     }
-                    __syncwarp();                                              // the previous stage's weight reads are done
+                    // ---- scores S[head g][key] for the 4 blocks of 8 keys ----
+                    float sc[4][2];
 #pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        const float sg = valid ? sa[g] + sb[g] : -INFINITY;    // rows past T_kv may hold anything
-                        float mx = sg;
+                    for (int nb = 0; nb < 4; ++nb) {
+                        float c[4] = {0.f, 0.f, 0.f, 0.f};
+                        const int r = half * 32 + 8 * nb + g;                  // B column g = key row r of the stage
 #pragma unroll
-                        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-                        const float m_new = fmaxf(m[g], mx);
-                        const float alpha = fast_exp2(m[g] - m_new);           // 0 on the first stage
-                        const float pw = fast_exp2(sg - m_new);                // 0 for lanes past the end
-                        my_p[g * 32 + lane] = pw;
-                        lsum[g] = lsum[g] * alpha + pw;                        // per-lane share of the row sum
-#pragma unroll
-                        for (int c = 0; c < FPL; ++c) o[g][c] *= alpha;
-                        m[g] = m_new;
-                    }
-                    __syncwarp();
-                    // values: this lane's FPL features of every row; rows past the end repeat the last one (weight 0)
-                    const int vbox = (lane * FPL) >> 6;                        // which 64-feature box
-                    const int vchunk = ((lane * FPL) & 63) >> 3;               // 16-byte piece inside the 128-byte row
-                    const int vsub = ((lane * FPL) & 7) * 2;                   // byte offset inside the piece
-#pragma unroll
-                    for (int j4 = 0; j4 < 8; ++j4) {
-                        uint32_t vr[4][FPL / 2];
-#pragma unroll
-                        for (int jj = 0; jj < 4; ++jj) {
-                            const int rr = half * 32 + min(4 * j4 + jj, n - 1);
-                            const uint8_t* src = sV + vbox * kBoxBytes + rr * 128 + ((vchunk ^ (rr & 7)) << 4) + vsub;
-                            if constexpr (FPL == 4) {
-                                const uint2 v = *reinterpret_cast<const uint2*>(src);
-                                vr[jj][0] = v.x; vr[jj][1] = v.y;
-                            } else {
-                                vr[jj][0] = *reinterpret_cast<const uint32_t*>(src);
-                            }
+                        for (int kp = 0; kp < D / 32; ++kp) {
+                            const int piece = 4 * kp + t;
+                            const uint4 kv = *reinterpret_cast<const uint4*>(sK + (piece >> 3) * kBoxBytes + r * 128 + (((piece & 7) ^ (r & 7)) << 4));
+                            mma_bf16_16x8x16(c, qf[kp].x, 0u, qf[kp].y, 0u, kv.x, kv.y);
+                            mma_bf16_16x8x16(c, qf[kp].z, 0u, qf[kp].w, 0u, kv.z, kv.w);
                         }
+                        sc[nb][0] = (8 * nb + 2 * t < n) ? c[0] * p.scale_log2 : -INFINITY;       // rows past T_kv may hold anything
+                        sc[nb][1] = (8 * nb + 2 * t + 1 < n) ? c[1] * p.scale_log2 : -INFINITY;
+                    }
+                    // ---- online softmax of head g over these 32 keys (8 per lane, 4 lanes per head) ----
+                    float mx = fmaxf(fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
+                                     fmaxf(fmaxf(sc[2][0], sc[2][1]), fmaxf(sc[3][0], sc[3][1])));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                    const float m_new = fmaxf(m_run, mx);                      // finite: the block holds at least one key
+                    const float alpha = fast_exp2(m_run - m_new);              // 0 on the first block
+                    m_run = m_new;
+                    uint32_t pa[4];                                            // P as bf16 pairs: block nb -> keys 8 nb + 2t, + 1
+                    float psum = 0.f;
 #pragma unroll
-                        for (int g = 0; g < G; ++g) {
-                            const float4 wv = lds_f32x4(&my_p[g * 32 + 4 * j4]);
-                            const float ww[4] = {wv.x, wv.y, wv.z, wv.w};
+                    for (int nb = 0; nb < 4; ++nb) {
+                        const float p0 = fast_exp2(sc[nb][0] - m_new), p1 = fast_exp2(sc[nb][1] - m_new);
+                        psum += p0 + p1;
+                        pa[nb] = pack_bf16x2(p0, p1);
+                    }
+                    lsum = lsum * alpha + psum;
+                    if (alpha != 1.f) {
 #pragma unroll
-                            for (int jj = 0; jj < 4; ++jj) {
+                        for (int fb = 0; fb < D / 8; ++fb) { o[fb][0] *= alpha; o[fb][1] *= alpha; }
+                    }
+                    // ---- O[head g][feature] += P V: B fragments of V through transposing matrix loads ----
 #pragma unroll
-                                for (int c = 0; c < FPL / 2; ++c) {
-                                    o[g][2 * c] = fmaf(ww[jj], bf16_lo_to_f32(vr[jj][c]), o[g][2 * c]);
-                                    o[g][2 * c + 1] = fmaf(ww[jj], bf16_hi_to_f32(vr[jj][c]), o[g][2 * c + 1]);
-                                }
-                            }
+                    for (int ks = 0; ks < 2; ++ks) {
+                        // lane -> row address of matrix lane / 8: keys 16 ks + 8 (mat & 1) + lane % 8, piece fb + (mat >> 1)
+                        const int vrow = half * 32 + 16 * ks + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+                        for (int fb = 0; fb < D / 8; fb += 2) {
+                            const int piece = fb + (lane >> 4);
+                            const uint32_t addr = smem_u32(sV + (piece >> 3) * kBoxBytes + vrow * 128 + (((piece & 7) ^ (vrow & 7)) << 4));
+                            uint32_t b0, b1, b2, b3;
+                            ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+                            mma_bf16_16x8x16(o[fb], pa[2 * ks], 0u, pa[2 * ks + 1], 0u, b0, b1);
+                            mma_bf16_16x8x16(o[fb + 1], pa[2 * ks], 0u, pa[2 * ks + 1], 0u, b2, b3);
                         }
                     }
                 }
-                // the stage is refilled by the async proxy: order this warp's reads before the arrival
+                // the stage is refilled by the async proxy: order this warp's accesses before the arrival
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty_bar(st));
@@ -322,32 +307,31 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
             gi0 += w.n_stage;
 
             // ---- merge the eight warps, write the item's partial ----
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
+            lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
+            if (g < G) {
+                if (t == 0) { s_m[warp * G + g] = m_run; s_l[warp * G + g] = lsum; }
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                float t = lsum[g];
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
-                if (lane == 0) { s_m[warp * G + g] = m[g]; s_l[warp * G + g] = t; }
-#pragma unroll
-                for (int c = 0; c < FPL; ++c) s_o[(warp * G + g) * D + lane * FPL + c] = o[g][c];
+                for (int fb = 0; fb < D / 8; ++fb)
+                    *reinterpret_cast<float2*>(&s_o[(warp * G + g) * D + 8 * fb + 2 * t]) = make_float2(o[fb][0], o[fb][1]);
             }
             if (has_next) store_q(qb ^ 1, qnext);
             decode_consumer_sync();
             float* out = p.part + ((size_t(w.b) * p.Hk + w.hk) * p.S + w.split) * G * (D + 2);
             for (int e = ctid; e < G * D; e += kDecodeConsumerThreads) {
-                const int g = e / D, c = e - g * D;
+                const int hg = e / D, c = e - hg * D;
                 float mx = -INFINITY;
 #pragma unroll
-                for (int ww = 0; ww < kDecodeConsumerWarps; ++ww) mx = fmaxf(mx, s_m[ww * G + g]);
+                for (int ww = 0; ww < kDecodeConsumerWarps; ++ww) mx = fmaxf(mx, s_m[ww * G + hg]);
                 float acc = 0.f, lt = 0.f;
 #pragma unroll
                 for (int ww = 0; ww < kDecodeConsumerWarps; ++ww) {
-                    const float f = s_m[ww * G + g] == -INFINITY ? 0.f : fast_exp2(s_m[ww * G + g] - mx);   // a warp without keys
-                    acc = fmaf(f, s_o[(ww * G + g) * D + c], acc);
-                    lt = fmaf(f, s_l[ww * G + g], lt);
+                    const float f = s_m[ww * G + hg] == -INFINITY ? 0.f : fast_exp2(s_m[ww * G + hg] - mx);   // a warp without keys
+                    acc = fmaf(f, s_o[(ww * G + hg) * D + c], acc);
+                    lt = fmaf(f, s_l[ww * G + hg], lt);
                 }
-                out[g * (D + 2) + 2 + c] = acc;
-                if (c == 0) { out[g * (D + 2)] = mx; out[g * (D + 2) + 1] = lt; }
+                out[hg * (D + 2) + 2 + c] = acc;
+                if (c == 0) { out[hg * (D + 2)] = mx; out[hg * (D + 2) + 1] = lt; }
             }
             decode_consumer_sync();                                       // s_o, s_m, s_l free again; the next q is visible
             qb ^= 1;

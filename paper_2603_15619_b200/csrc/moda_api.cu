@@ -254,7 +254,7 @@ int launch_decode_g(const DecodeParams& p, cudaStream_t stream) {
     const unsigned grid = unsigned(items < p.num_sms ? items : p.num_sms);
     decode_split_tma_kernel<D, G><<<grid, kDecodeTmaThreads, L::kDynamic, stream>>>(mK, mV, p);
     if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
-    decode_merge_kernel<D><<<dim3(p.H, p.B), D, 0, stream>>>(p);
+    decode_merge_kernel<D><<<dim3(p.H, p.B), kDecodeMergeThreads, 0, stream>>>(p);
     if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     return MODA_OK;
 }

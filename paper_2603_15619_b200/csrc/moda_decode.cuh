@@ -348,38 +348,65 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
     }
 }
 
-// One CTA of D threads per (b, query head): thread = output feature.
+// One CTA of four warps per (b, query head).  Lanes hold D / 32 adjacent features; a warp takes every
+// fourth depth slot and every fourth split, several of them in flight at once (the kernel is a chain
+// of short dependent phases, so its time is load latency, not bandwidth).
+constexpr int kDecodeMergeThreads = 128;
+
 template <int D>
-__global__ void __launch_bounds__(D)
+__global__ void __launch_bounds__(kDecodeMergeThreads)
 decode_merge_kernel(const DecodeParams p) {
+    constexpr int FPL = D / 32, NW = kDecodeMergeThreads / 32, UN = 4;
     __shared__ float s_w[kDecodeMaxSplits];          // weight of each split's partial
     __shared__ float s_d[256];                       // depth scores (log2 domain), then weights; l <= 256
-    __shared__ float s_q[D];
-    __shared__ float s_red[D / 32];
+    __shared__ float s_red[NW];
+    __shared__ __align__(16) float s_acc[NW][D];
     const int h = blockIdx.x, b = blockIdx.y;
     const int G = p.H / p.Hk, hk = h / G, g = h - hk * G;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    constexpr int NW = D / 32;
 
-    s_q[tid] = __bfloat162float(p.q[(size_t(b) * p.H + h) * D + tid]) * p.scale_log2;
-    __syncthreads();
-    // depth scores: one warp per slot, lanes across features
-    for (int i = warp; i < p.l; i += NW) {
-        const __nv_bfloat16* kd = p.depth + ((size_t(i) * p.B + b) * p.Hk + hk) * 2 * D;
-        float a = 0.f;
+    // this lane's features of a bf16 row, as floats
+    auto load_row = [&](const __nv_bfloat16* row, float (&x)[FPL]) {
+        if constexpr (FPL == 4) {
+            const uint2 v = *reinterpret_cast<const uint2*>(row + lane * 4);
+            x[0] = bf16_lo_to_f32(v.x); x[1] = bf16_hi_to_f32(v.x); x[2] = bf16_lo_to_f32(v.y); x[3] = bf16_hi_to_f32(v.y);
+        } else {
+            const uint32_t v = *reinterpret_cast<const uint32_t*>(row + lane * 2);
+            x[0] = bf16_lo_to_f32(v); x[1] = bf16_hi_to_f32(v);
+        }
+    };
+    float q[FPL];
+    load_row(p.q + (size_t(b) * p.H + h) * D, q);
 #pragma unroll
-        for (int c = lane; c < D; c += 32) a = fmaf(s_q[c], __bfloat162float(kd[c]), a);
+    for (int c = 0; c < FPL; ++c) q[c] *= p.scale_log2;
+    const size_t slot_stride = size_t(p.B) * p.Hk * 2 * D;                          // elements between depth slots
+    const __nv_bfloat16* depth0 = p.depth + (size_t(b) * p.Hk + hk) * 2 * D;        // slot 0: key row, value row at + D
+
+    // ---- depth scores: warp `warp` takes slots warp, warp + 4, ..., UN at a time ----
+    for (int i0 = warp; i0 < p.l; i0 += NW * UN) {
+        float kd[UN][FPL];
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
-        if (lane == 0) s_d[i] = a;
+        for (int u = 0; u < UN; ++u) {
+            const int i = min(i0 + u * NW, p.l - 1);
+            load_row(depth0 + size_t(i) * slot_stride, kd[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            float a = 0.f;
+#pragma unroll
+            for (int c = 0; c < FPL; ++c) a = fmaf(q[c], kd[u][c], a);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+            if (lane == 0 && i0 + u * NW < p.l) s_d[i0 + u * NW] = a;
+        }
     }
     __syncthreads();
     const float* part = p.part + ((size_t(b) * p.Hk + hk) * p.S * G + g) * (D + 2);   // + split * G * (D + 2)
     const size_t split_stride = size_t(G) * (D + 2);
-    // global maximum over the split maxima and the depth scores
+    // ---- global maximum over the split maxima and the depth scores ----
     float mx = -INFINITY;
-    for (int s = tid; s < p.S; s += D) mx = fmaxf(mx, part[s * split_stride]);
-    for (int i = tid; i < p.l; i += D) mx = fmaxf(mx, s_d[i]);
+    for (int s = tid; s < p.S; s += kDecodeMergeThreads) mx = fmaxf(mx, part[s * split_stride]);
+    for (int i = tid; i < p.l; i += kDecodeMergeThreads) mx = fmaxf(mx, s_d[i]);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
     if (lane == 0) s_red[warp] = mx;
@@ -388,15 +415,15 @@ decode_merge_kernel(const DecodeParams p) {
 #pragma unroll
     for (int w = 1; w < NW; ++w) mx = fmaxf(mx, s_red[w]);
     __syncthreads();
-    // weights and the row sum
+    // ---- weights and the row sum ----
     float lt = 0.f;
-    for (int s = tid; s < p.S; s += D) {
+    for (int s = tid; s < p.S; s += kDecodeMergeThreads) {
         const float ms = part[s * split_stride];
         const float f = ms == -INFINITY ? 0.f : fast_exp2(ms - mx);
         s_w[s] = f;
         lt = fmaf(f, part[s * split_stride + 1], lt);
     }
-    for (int i = tid; i < p.l; i += D) {
+    for (int i = tid; i < p.l; i += kDecodeMergeThreads) {
         const float w = fast_exp2(s_d[i] - mx);
         s_d[i] = w;
         lt += w;
@@ -408,14 +435,49 @@ decode_merge_kernel(const DecodeParams p) {
     lt = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) lt += s_red[w];
-    // output feature tid
-    float acc = 0.f;
-    for (int s = 0; s < p.S; ++s) acc = fmaf(s_w[s], part[s * split_stride + 2 + tid], acc);
-    for (int i = 0; i < p.l; ++i) {
-        const __nv_bfloat16* vd = p.depth + (((size_t(i) * p.B + b) * p.Hk + hk) * 2 + 1) * D;
-        acc = fmaf(s_d[i], __bfloat162float(vd[tid]), acc);
+    // ---- weighted sum of the split partials and of the depth values: a warp takes every fourth of each ----
+    float acc[FPL];
+#pragma unroll
+    for (int c = 0; c < FPL; ++c) acc[c] = 0.f;
+    for (int s0 = warp; s0 < p.S; s0 += NW * UN) {
+        float x[UN][FPL];
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const int s = min(s0 + u * NW, p.S - 1);
+            const float* src = part + s * split_stride + 2 + lane * FPL;
+#pragma unroll
+            for (int c = 0; c < FPL; ++c) x[u][c] = src[c];
+        }
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const float w = s0 + u * NW < p.S ? s_w[s0 + u * NW] : 0.f;
+#pragma unroll
+            for (int c = 0; c < FPL; ++c) acc[c] = fmaf(w, x[u][c], acc[c]);
+        }
     }
-    p.O[(size_t(b) * p.H + h) * D + tid] = __float2bfloat16(acc / lt);
+    for (int i0 = warp; i0 < p.l; i0 += NW * UN) {
+        float vd[UN][FPL];
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const int i = min(i0 + u * NW, p.l - 1);
+            load_row(depth0 + size_t(i) * slot_stride + D, vd[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const float w = i0 + u * NW < p.l ? s_d[i0 + u * NW] : 0.f;
+#pragma unroll
+            for (int c = 0; c < FPL; ++c) acc[c] = fmaf(w, vd[u][c], acc[c]);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < FPL; ++c) s_acc[warp][lane * FPL + c] = acc[c];
+    __syncthreads();
+    if (tid < D) {
+        float a = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) a += s_acc[w][tid];
+        p.O[(size_t(b) * p.H + h) * D + tid] = __float2bfloat16(a / lt);
+    }
     if (tid == 0) p.LSE[size_t(b) * p.H + h] = (mx + log2f(lt)) * kDecodeLn2;
 }
 

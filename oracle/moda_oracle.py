@@ -267,3 +267,43 @@ def decode_gqa(q, K, V, kd, vd, scale):
             o[b, h] = (p / z) @ vals
             lse[b, h] = m + np.log(z)
     return o, lse
+
+
+# ---------------------------------------------------------------------------------------
+# Prefill with a cache (1 <= T_q <= T_kv): the T_q newest positions of a sequence whose layer
+# already caches T_kv - T_q earlier keys.  Query row i (0-based among the new positions) sits at
+# absolute position i + (T_kv - T_q): the causal mask of Eq. 2 admits sequence keys
+# j <= i + (T_kv - T_q), and its depth keys are those stored for its own position (slot arrays
+# are indexed by the new positions only).  Definition written out in numpy float64.
+# ---------------------------------------------------------------------------------------
+def forward_prefill_gqa(Q, K, V, Kd, Vd, scale):
+    """O [B,T_q,Hq,d], LSE [B,Hq,T_q] for Q [B,T_q,Hq,d], K, V [B,T_kv,Hk,d], Kd, Vd [l,B,T_q,Hk,d] (or None)."""
+    Q = np.ascontiguousarray(Q, dtype=np.float64)
+    K = np.ascontiguousarray(K, dtype=np.float64)
+    V = np.ascontiguousarray(V, dtype=np.float64)
+    if Q.ndim != 4 or K.ndim != 4 or V.shape != K.shape:
+        raise ValueError("Q must be [B, T_q, Hq, d]; K, V [B, T_kv, Hk, d]")
+    B, Tq, Hq, d = Q.shape
+    _, Tkv, Hk, _ = K.shape
+    if K.shape[0] != B or K.shape[3] != d or Hk < 1 or Hq % Hk or Tq < 1 or Tkv < Tq:
+        raise ValueError("need T_kv >= T_q >= 1 and Hk dividing Hq")
+    G = Hq // Hk
+    off = Tkv - Tq
+    l = 0 if Kd is None else int(np.shape(Kd)[0])
+    Kd = np.zeros((0, B, Tq, Hk, d)) if l == 0 else _f64(Kd, (l, B, Tq, Hk, d))
+    Vd = np.zeros((0, B, Tq, Hk, d)) if l == 0 else _f64(Vd, (l, B, Tq, Hk, d))
+    O = np.empty((B, Tq, Hq, d)); LSE = np.empty((B, Hq, Tq))
+    for b in range(B):
+        for h in range(Hq):
+            hk = h // G
+            for i in range(Tq):
+                n_seq = i + off + 1                                        # keys 0 .. i + off
+                keys = np.concatenate([K[b, :n_seq, hk, :], Kd[:, b, i, hk, :]], axis=0)
+                vals = np.concatenate([V[b, :n_seq, hk, :], Vd[:, b, i, hk, :]], axis=0)
+                s = (keys @ Q[b, i, h]) * float(scale)
+                m = s.max()
+                p = np.exp(s - m)
+                z = p.sum()
+                O[b, i, h] = (p / z) @ vals
+                LSE[b, h, i] = m + np.log(z)
+    return O, LSE

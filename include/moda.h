@@ -186,6 +186,22 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
                              void* workspace, size_t workspace_bytes, int stages, void* stream);
 
 /*
+ * Prefill with a cache (T_q <= T_kv; Table 1's prefilling rows): the T_q newest positions of each
+ * sequence attend to the T_kv keys that the layer caches (the T_kv - T_q earlier ones and their own,
+ * appended by the caller beforehand) and to the depth pairs of their own positions.  Query row i
+ * sits at key position i + (T_kv - T_q); the causal mask is taken at that position.  Forward only.
+ *     Q, O     : bf16 [B][T_q][H][d]            K, V : bf16 [B][T_kv][H_kv][d]
+ *     depth_kv : cache layout over the T_q positions (moda_depth_cache_bytes(B, T_q, H_kv, d, l))
+ *     LSE      : fp32 [B][H][T_q]
+ * T_kv == T_q is exactly moda_attn_fwd_gqa; T_kv < T_q is MODA_ERR_BAD_SHAPE.  Any T_kv - T_q is
+ * allowed (it need not be a multiple of the 128-row tile).  Same kernels, validation, asynchrony
+ * and error codes as moda_attn_fwd_gqa.
+ */
+int moda_attn_fwd_prefill(const void* Q, const void* K, const void* V, const void* depth_kv,
+                          int B, int T_q, int T_kv, int H, int H_kv, int d, int l, float scale,
+                          void* O, float* LSE, void* stream);
+
+/*
  * Decode step (T_q = 1; Table 1, "decoding cache" and "decoding FLOPs" rows): the newest token of
  * each of B sequences attends, under one softmax, to the T_kv keys of this layer's KV cache (its
  * own key included: the caller appends before the call) and to its own l depth key/value pairs,

@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     moda_attn_decode,
     moda_attn_fwd,
     moda_attn_fwd_gqa,
+    moda_attn_fwd_prefill,
     moda_bwd_workspace_bytes,
     moda_bwd_workspace_bytes_gqa,
     moda_decode_workspace_bytes,

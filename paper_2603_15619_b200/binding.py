@@ -22,7 +22,7 @@ SYMBOLS = (
     "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd", "moda_attn_bwd_stages",
     "moda_attn_bwd_static_scratch",
     "moda_attn_fwd_gqa", "moda_bwd_workspace_bytes_gqa", "moda_attn_bwd_gqa", "moda_attn_bwd_gqa_stages",
-    "moda_decode_workspace_bytes", "moda_attn_decode",
+    "moda_decode_workspace_bytes", "moda_attn_decode", "moda_attn_fwd_prefill",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -80,6 +80,8 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd_gqa.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
     lib.moda_attn_bwd_gqa_stages.restype = ci
     lib.moda_attn_bwd_gqa_stages.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, ci, vp]
+    lib.moda_attn_fwd_prefill.restype = ci
+    lib.moda_attn_fwd_prefill.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
     lib.moda_decode_workspace_bytes.restype = sz
     lib.moda_decode_workspace_bytes.argtypes = [ci] * 3
     lib.moda_attn_decode.restype = ci
@@ -306,4 +308,21 @@ def moda_attn_decode(q, K, V, depth_kv_token, T_kv, l, scale, O=None, LSE=None, 
                                    B, int(T_kv), T_cap, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "moda_attn_decode")
+    return O, LSE
+
+
+def moda_attn_fwd_prefill(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):
+    """Prefill with a cache: Q [B,T_q,H,d] (the newest positions), K, V [B,T_kv,H_kv,d] with T_kv >= T_q,
+    depth cache over the T_q positions.  Returns O [B,T_q,H,d] bf16 and LSE [B,H,T_q] fp32."""
+    B, T_q, H, d = _bthd(Q, "Q")
+    Bk, T_kv, Hk, dk = _bthd(K, "K")
+    if (Bk, dk) != (B, d) or _bthd(V, "V") != (B, T_kv, Hk, d):
+        raise ValueError("K and V must be bf16 [B, T_kv, H_kv, d] tensors matching Q's B and d")
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None:
+        LSE = torch.empty((B, H, T_q), dtype=torch.float32, device=Q.device)
+    _check(load().moda_attn_fwd_prefill(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
+                                        B, T_q, T_kv, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
+                                        _stream(stream)), "moda_attn_fwd_prefill")
     return O, LSE

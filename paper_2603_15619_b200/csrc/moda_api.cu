@@ -108,15 +108,15 @@ inline bool fwd_depth_heavy(int T, int l, int d) {
 }
 
 template <int D>
-int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int H, int Hk, int l,
+int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int T_kv, int H, int Hk, int l,
                float scale, void* O, float* LSE, cudaStream_t stream) {
     constexpr bool kWide = (D == 64);
     constexpr int kSmem = kWide ? Fwd2Smem<D>::kDynamic : FwdSmem<D, 2>::kDynamic;
     constexpr int kSmemDeep = FwdSmem<128, 1>::kDynamic;
     constexpr int kThreads = kWide ? kFwd2Threads : kFwdThreads;
     CUtensorMap mQ, mK, mV, mO;
-    if (!make_bthd_map(&mQ, Q, B, T, H, D) || !make_bthd_map(&mK, K, B, T, Hk, D) ||
-        !make_bthd_map(&mV, V, B, T, Hk, D) || !make_bthd_map(&mO, O, B, T, H, D))
+    if (!make_bthd_map(&mQ, Q, B, T, H, D) || !make_bthd_map(&mK, K, B, T_kv, Hk, D) ||
+        !make_bthd_map(&mV, V, B, T_kv, Hk, D) || !make_bthd_map(&mO, O, B, T, H, D))
         return MODA_ERR_CUDA;
     static thread_local int configured_dev = -1;
     int dev = 0;
@@ -132,6 +132,7 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.O = static_cast<__nv_bfloat16*>(O);
     p.LSE = LSE;
     p.B = B; p.T = T; p.H = H; p.l = l;
+    p.T_kv = T_kv; p.kv_off = T_kv - T;
     p.G = H / Hk;
     p.scale_log2 = scale * kLog2e;
     const unsigned grid = unsigned(B) * H * num_tiles(T);
@@ -362,7 +363,15 @@ int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth
 int moda_attn_fwd_gqa(const void* Q, const void* K, const void* V, const void* depth_kv,
                       int B, int T, int H, int H_kv, int d, int l, float scale,
                       void* O, float* LSE, void* stream) {
-    if (int rc = check_shape(B, T, H, d)) return rc;
+    return moda_attn_fwd_prefill(Q, K, V, depth_kv, B, T, T, H, H_kv, d, l, scale, O, LSE, stream);
+}
+
+int moda_attn_fwd_prefill(const void* Q, const void* K, const void* V, const void* depth_kv,
+                          int B, int T_q, int T_kv, int H, int H_kv, int d, int l, float scale,
+                          void* O, float* LSE, void* stream) {
+    if (int rc = check_shape(B, T_q, H, d)) return rc;
+    if (T_kv < T_q) return MODA_ERR_BAD_SHAPE;
+    if (int rc = check_shape(B, T_kv, H, d)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!Q || !K || !V || !O || !LSE || (l > 0 && !depth_kv)) return MODA_ERR_NULL_POINTER;
@@ -371,8 +380,8 @@ int moda_attn_fwd_gqa(const void* Q, const void* K, const void* V, const void* d
         return MODA_ERR_MISALIGNED;
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv, B, T, H, H_kv, l, scale, O, LSE, st)
-                    : launch_fwd<64>(Q, K, V, depth_kv, B, T, H, H_kv, l, scale, O, LSE, st);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv, B, T_q, T_kv, H, H_kv, l, scale, O, LSE, st)
+                    : launch_fwd<64>(Q, K, V, depth_kv, B, T_q, T_kv, H, H_kv, l, scale, O, LSE, st);
 }
 
 size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l) {

@@ -88,7 +88,8 @@ struct FwdParams {
     const __nv_bfloat16* depth_kv;   // cache layout, >= l slots (unused when l == 0)
     __nv_bfloat16* O;
     float* LSE;
-    int B, T, H, l;                  // H = number of query heads
+    int B, T, H, l;                  // T query positions, H query heads
+    int T_kv, kv_off;                // sequence keys 0 .. T_kv - 1; query row i sits at key position i + kv_off (kv_off = T_kv - T)
     int G;                           // query heads per key/value head (1 = plain multi-head attention)
     float scale_log2;                // scale * log2(e)
 };
@@ -150,7 +151,8 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     const int b = tc.b, h = tc.h, hk = tc.hk, qt = tc.qt;
     const int Hk = p.H / p.G;
     const int q0 = qt * kTileRows;
-    const int n_kv = qt + 1;                         // causal: key tiles 0..qt
+    // causal: key tiles up to the one that holds the last row's own position (row i sees keys <= i + kv_off)
+    const int n_kv = min((q0 + kTileRows + p.kv_off + kTileRows - 1) / kTileRows, num_tiles(p.T_kv));
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -200,13 +202,14 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             tmem_ld32(tS + 64, s2);
             tmem_ld32(tS + 96, s3);
             tmem_wait_ld();
-            if (j == n_kv - 1) {                         // diagonal tile: causal mask, key <= query
+            if ((j + 1) * kTileRows - 1 > q0 + p.kv_off) {   // tile reaches past the first row's position: causal mask
+                const int rs = r + q0 + p.kv_off - j * kTileRows;   // column i of this tile is visible iff i <= rs
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    if (i > r) s0[i] = 0xff800000u;
-                    if (i + 32 > r) s1[i] = 0xff800000u;
-                    if (i + 64 > r) s2[i] = 0xff800000u;
-                    if (i + 96 > r) s3[i] = 0xff800000u;
+                    if (i > rs) s0[i] = 0xff800000u;
+                    if (i + 32 > rs) s1[i] = 0xff800000u;
+                    if (i + 64 > rs) s2[i] = 0xff800000u;
+                    if (i + 96 > rs) s3[i] = 0xff800000u;
                 }
             }
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;

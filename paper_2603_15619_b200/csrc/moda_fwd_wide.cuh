@@ -130,7 +130,8 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const int b = tc.b, h = tc.h, hk = tc.hk, qt = tc.qt;
     const int Hk = p.H / p.G;
     const int q0 = qt * kTileRows;
-    const int n_kv = min((kTileRows / kFwdBN) * (qt + 1), (p.T + kFwdBN - 1) / kFwdBN);   // key tiles at or below the diagonal
+    // key tiles up to the one that holds the last row's own position (row i sees keys <= i + kv_off)
+    const int n_kv = min((q0 + kTileRows + p.kv_off + kFwdBN - 1) / kFwdBN, (p.T_kv + kFwdBN - 1) / kFwdBN);
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -183,7 +184,7 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
             for (int c = 0; c < NB; ++c) tmem_ld32(tS + c * 32, sv[c]);
             tmem_wait_ld();
-            const int koff = j * kFwdBN - q0;            // key of column c is visible to row r iff koff + c <= r
+            const int koff = j * kFwdBN - q0 - p.kv_off; // key of column c is visible to row r iff koff + c <= r
             if (koff + kFwdBN - 1 > 0) {                 // tiles that touch the diagonal: causal mask
 #pragma unroll
                 for (int c = 0; c < NB; ++c)

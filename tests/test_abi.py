@@ -104,3 +104,14 @@ def test_decode_entry_point_validates_before_touching_the_device():
     assert call(q=None) == -1 and call(depth=None) == -1 and call(l=0, depth=None) != -1
     assert call(q=ctypes.c_void_p(4100)) == -2
     assert call(work=None) == -7 and call(wb=16) == -7
+
+
+def test_prefill_entry_point_validates_before_touching_the_device():
+    lib = binding.load()
+    p = ctypes.c_void_p(4096)
+    call = lambda Tq, Tkv, H=4, Hk=2, d=64, l=0, Q=p: lib.moda_attn_fwd_prefill(Q, p, p, None, 1, Tq, Tkv, H, Hk, d, l, ctypes.c_float(0.1), p, p, None)
+    assert call(128, 64) == -3 and call(0, 64) == -3
+    assert call(64, 128, d=96) == -4
+    assert call(64, 128, H=6, Hk=4) == -12
+    assert call(64, 128, l=2) == -1            # depth cache missing
+    assert call(64, 128, Q=None) == -1

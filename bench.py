@@ -306,6 +306,7 @@ def run_moda(args, rank, world, device):
         out["sweep"] = run_sweep(peaks, device, layer)
         out["gqa_sweep"] = run_gqa_sweep(device)
         out["decode_sweep"] = run_decode_sweep(peaks, device)
+        out["prefill_sweep"] = run_prefill_sweep(peaks, device)
     if not args.no_e2e:
         out["e2e"] = run_e2e(layer, min(K, 8), world, step_flops, device)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -483,6 +484,42 @@ def run_decode_sweep(peaks, device, shapes=None, iters=20):
     return rows
 
 
+# Prefill with a cache: a chunk of T_q new positions over T_kv cached keys (B, T_q, T_kv, H, H_kv, d, l).
+PREFILL_SHAPES = [(4, 2048, 16384, 16, 8, 128, 24), (1, 8192, 65536, 16, 8, 128, 24), (4, 2048, 16384, 32, 8, 64, 32)]
+
+
+def run_prefill_sweep(peaks, device, shapes=None, iters=5):
+    """Forward of a chunk against a long cached prefix; FLOPs = 4 d per (query row, visible key) pair."""
+    import paper_2603_15619_b200 as moda
+    rows = []
+    for B, Tq, Tkv, H, Hk, d, l in (shapes or PREFILL_SHAPES):
+        torch.cuda.empty_cache()
+        wq = synthetic.Workload("prefill/q", B, Tq, H, d, l)
+        wk = synthetic.Workload("prefill/kv", B, Tkv, Hk, d, l)
+        wd = synthetic.Workload("prefill/depth", B, Tq, Hk, d, l)
+        Q = synthetic.tensor(wq, "Q", 0, 0, device)
+        K = synthetic.tensor(wk, "K", 0, 0, device)
+        V = synthetic.tensor(wk, "V", 0, 0, device)
+        cache = None
+        if l > 0:
+            cache = moda.alloc_depth_cache(B, Tq, Hk, d, l, device)
+            for i in range(l):
+                moda.moda_depth_cache_append(cache, i, synthetic.tensor(wd, "Kd", 0, i, device), synthetic.tensor(wd, "Vd", 0, i, device))
+        O = torch.empty_like(Q)
+        LSE = torch.empty((B, H, Tq), dtype=torch.float32, device=device)
+        fn = lambda: moda.moda_attn_fwd_prefill(Q, K, V, cache, l, d ** -0.5, O=O, LSE=LSE)
+        ms = time_calls(fn, iters)
+        off = Tkv - Tq
+        pairs = Tq * (off + 1) + Tq * (Tq - 1) / 2 + Tq * l
+        fl = 4.0 * B * H * d * pairs
+        rows.append({"B": B, "T_q": Tq, "T_kv": Tkv, "H": H, "H_kv": Hk, "d": d, "l": l, "ms": round(ms, 4),
+                     "tflops": round(fl / ms / 1e9, 1), "frac_measured_burst_bf16": round(fl / ms / 1e9 / peaks["bf16_tflops"], 4)})
+        log("prefill_sweep", rows[-1])
+        del Q, K, V, cache, O, LSE
+    torch.cuda.empty_cache()
+    return rows
+
+
 def run_e2e(layer, steps, world, step_flops, device):
     """The same step driven from pinned HOST buffers: every step copies its inputs host->device and
     its results device->host inside the timed region.  Two device buffer sets and three streams let
@@ -619,6 +656,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gqa-shape", default="", help="T,G[,L]: time only this grouped-query shape (B=1, d=64, 8 key/value "
                                                     "heads, L depth slots (default 32) and l=0) and print its row; for profiling")
+    ap.add_argument("--prefill-sweep", action="store_true", help="time only the prefill-with-cache shapes and print their rows")
     ap.add_argument("--decode-shape", default="", help="B,T_kv,H,H_kv,d,l: time only this decode step and print its row; for profiling")
     args = ap.parse_args()
 
@@ -643,6 +681,8 @@ def main():
         if args.gqa_shape:
             v = [int(t) for t in args.gqa_shape.split(",")]
             out = {"gqa_sweep": run_gqa_sweep(device, [(v[0], v[1], v[2] if len(v) > 2 else 32, None)])}
+        elif args.prefill_sweep:
+            out = {"prefill_sweep": run_prefill_sweep(load_peaks(), device)}
         elif args.decode_shape:
             v = tuple(int(t) for t in args.decode_shape.split(","))
             out = {"decode_sweep": run_decode_sweep(load_peaks(), device, [v], iters=max(1, min(args.steps, 20)))}

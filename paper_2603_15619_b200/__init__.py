@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     MODA_BWD_STAGE_ROWTERMS,
     ModaError,
     alloc_depth_cache,
+    depth_cache_window,
     moda_attn_bwd,
     moda_attn_bwd_gqa,
     moda_attn_bwd_gqa_stages,

@@ -146,6 +146,22 @@ def alloc_depth_cache(B, T, H, d, l_max, device="cuda") -> torch.Tensor:
     return torch.empty(max(n // 2, 8), dtype=torch.bfloat16, device=device)
 
 
+def depth_cache_window(cache, B, T, H, d, first_slot, n_slots=None):
+    """View of slots [first_slot, first_slot + n_slots) of a depth cache (to its end when n_slots is None).
+
+    The cache is slot-major, so a window of consecutive slots is itself a cache: passing the view with
+    ``l = n_slots`` makes a layer attend only to those slots (e.g. the last S layers instead of all
+    preceding ones, the bounded depth-slot idea of the paper's discussion), and the same view of a
+    gradient cache receives exactly their gradients."""
+    slot = moda_depth_cache_bytes(B, T, H, d, 1) // 2
+    if first_slot < 0 or first_slot * slot > cache.numel():
+        raise ValueError("window starts outside the cache")
+    end = cache.numel() if n_slots is None else (first_slot + n_slots) * slot
+    if end > cache.numel():
+        raise ValueError("window ends outside the cache")
+    return cache[first_slot * slot:end]
+
+
 def moda_depth_cache_append(cache, slot, K_i, V_i, stream=None):
     B, T, H, d = _bthd(K_i, "K_i")
     assert _bthd(V_i, "V_i") == (B, T, H, d)

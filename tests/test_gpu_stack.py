@@ -97,3 +97,29 @@ def test_slot_written_without_attending_gets_the_gradients_of_the_layers_after_i
     dQ, dK, dV, dKd, dVd = orc.backward_gqa(f64(Q), f64(K), f64(V), Kd, Vd, f64(a["dO"]), scale)
     for got, want in ((Q.grad, dQ), (K.grad, dK), (V.grad, dV), (Kf.grad, dKd[0]), (Vf.grad, dVd[0])):
         assert rel_l2(f64(got), want) <= TOL_GRAD_REL_L2
+
+
+@pytest.mark.parametrize("B,T,H,Hk,d,l,S", [(1, 300, 2, 2, 64, 7, 3), (1, 200, 4, 2, 128, 6, 2)])
+def test_window_of_the_last_slots_is_the_operator_on_those_slots(B, T, H, Hk, d, l, S):
+    """Bounded depth slots: a layer that attends only to the last S of l stored slots, forward and backward."""
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=13, device="cuda")
+    scale = d ** -0.5
+    cache = moda.alloc_depth_cache(B, T, Hk, d, l)
+    for i in range(l):
+        moda.moda_depth_cache_append(cache, i, x["Kd"][i].contiguous(), x["Vd"][i].contiguous())
+    win = moda.depth_cache_window(cache, B, T, Hk, d, l - S, S)
+    O, LSE = moda.moda_attn_fwd_gqa(x["Q"], x["K"], x["V"], win, S, scale)
+    gcache = torch.zeros_like(cache)
+    gwin = moda.depth_cache_window(gcache, B, T, Hk, d, l - S, S)
+    dQ, dK, dV, _ = moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], win, O, x["dO"], LSE, S, scale, d_depth_kv=gwin)
+    assert moda.moda_last_status() == 0
+    args = (f64(x["Q"]), f64(x["K"]), f64(x["V"]), f64(x["Kd"][l - S:]), f64(x["Vd"][l - S:]))
+    O_ref, LSE_ref = orc.forward_gqa(*args, scale)
+    refs = orc.backward_gqa(*args, f64(x["dO"]), scale)
+    assert rel_l2(f64(O), O_ref) <= TOL_O_REL_L2 and np.abs(f64(LSE) - LSE_ref).max() <= 1e-3
+    dKd = torch.empty_like(x["Kd"]); dVd = torch.empty_like(x["Vd"])
+    for i in range(l):
+        moda.moda_depth_cache_unpack(gcache, i, dKd[i], dVd[i])
+    assert float(dKd[:l - S].abs().max()) == 0.0 and float(dVd[:l - S].abs().max()) == 0.0     # slots outside the window untouched
+    for got, want in ((dQ, refs[0]), (dK, refs[1]), (dV, refs[2]), (dKd[l - S:], refs[3]), (dVd[l - S:], refs[4])):
+        assert rel_l2(f64(got), want) <= TOL_GRAD_REL_L2

@@ -213,7 +213,8 @@ int moda_attn_fwd_prefill(const void* Q, const void* K, const void* V, const voi
  *     LSE             : fp32 [B][H], natural log over the T_kv + l keys
  *     workspace       : at least moda_decode_workspace_bytes(B, H, d) bytes, 16-byte aligned; it
  *                       holds per-split partial softmax states and is overwritten
- * Query head h uses key/value head h / G with G = H / H_kv in 1..8 (MODA_ERR_BAD_GROUP otherwise).
+ * Query head h uses key/value head h / G with G = H / H_kv in 1..8, 16 or 32 (MODA_ERR_BAD_GROUP
+ * otherwise; groups of 16 or 32 heads run as two or four groups of 8 that read the same K, V head).
  * Two launches on `stream`: a kernel that streams the KV cache once per key/value head (the key
  * range is split over enough CTAs to fill the device) and a merge kernel that adds the depth pairs.
  * All pointers are device pointers owned by the caller; validation, asynchrony and error codes are

@@ -240,8 +240,8 @@ template <int D, int G>
 int launch_decode_g(const DecodeParams& p, cudaStream_t stream) {
     using L = DecodeSmem<D, G>;
     CUtensorMap mK, mV;
-    if (!make_bthd_map(&mK, p.K, p.B, p.T_cap, p.Hk, D, kDecodeStageKeys) ||
-        !make_bthd_map(&mV, p.V, p.B, p.T_cap, p.Hk, D, kDecodeStageKeys))
+    if (!make_bthd_map(&mK, p.K, p.B, p.T_cap, p.Hk / p.kv_rep, D, kDecodeStageKeys) ||
+        !make_bthd_map(&mV, p.V, p.B, p.T_cap, p.Hk / p.kv_rep, D, kDecodeStageKeys))
         return MODA_ERR_CUDA;
     static thread_local int configured_dev = -1;
     int dev = 0;
@@ -459,8 +459,8 @@ int moda_attn_decode(const void* q, const void* K, const void* V, const void* de
     if (B < 1 || T_kv < 1 || T_cap < T_kv || H < 1) return MODA_ERR_BAD_SHAPE;
     if (d != 64 && d != 128) return MODA_ERR_BAD_HEAD_DIM;
     if ((long long)B * T_cap > 0x7fffffffLL / H) return MODA_ERR_BAD_SHAPE;
-    if (H_kv < 1 || H % H_kv != 0 || H / H_kv > 8) return MODA_ERR_BAD_GROUP;
-    if ((long long)B * H_kv * kDecodeMaxSplits > 0x7fffffffLL || B > 65535) return MODA_ERR_BAD_SHAPE;
+    if (int rc = check_groups(H, H_kv)) return rc;
+    if ((long long)B * H * kDecodeMaxSplits > 0x7fffffffLL || B > 65535) return MODA_ERR_BAD_SHAPE;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!q || !K || !V || !O || !LSE || (l > 0 && !depth_kv_token)) return MODA_ERR_NULL_POINTER;
     if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
@@ -478,8 +478,10 @@ int moda_attn_decode(const void* q, const void* K, const void* V, const void* de
     p.O = static_cast<__nv_bfloat16*>(O);
     p.LSE = LSE;
     p.part = static_cast<float*>(workspace);
-    p.B = B; p.T_kv = T_kv; p.T_cap = T_cap; p.H = H; p.Hk = H_kv; p.l = l;
-    const DecodePlan plan = decode_plan(B, H_kv, T_kv, sms);
+    // 16 or 32 query heads per key/value head: groups of 8 heads that read the same K, V head
+    const int kv_rep = (H / H_kv > 8) ? (H / H_kv) / 8 : 1;
+    p.B = B; p.T_kv = T_kv; p.T_cap = T_cap; p.H = H; p.Hk = H_kv * kv_rep; p.l = l; p.kv_rep = kv_rep;
+    const DecodePlan plan = decode_plan(B, p.Hk, T_kv, sms);
     p.S = plan.S; p.keys_per_split = plan.keys_per_split; p.num_sms = sms;
     p.scale_log2 = scale * kDecodeLog2e;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

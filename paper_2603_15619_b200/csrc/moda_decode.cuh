@@ -48,6 +48,7 @@ struct DecodeParams {
     int B, T_kv, T_cap, H, Hk, l;
     int S, keys_per_split;        // keys_per_split is a multiple of kDecodeKeysPerPass
     int num_sms;
+    int kv_rep;                   // groups of more than 8 query heads run as kv_rep groups of 8 on the same K, V head
     float scale_log2;             // scale * log2(e)
 };
 
@@ -176,8 +177,8 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
                     const int t0 = w.k_begin + i * kDecodeStageKeys;
 #pragma unroll
                     for (int h = 0; h < NH; ++h) {
-                        tma_load_4d(dst + h * kBoxBytes, &mapK, full_bar(st), 64 * h, w.hk, t0, w.b);
-                        tma_load_4d(dst + (NH + h) * kBoxBytes, &mapV, full_bar(st), 64 * h, w.hk, t0, w.b);
+                        tma_load_4d(dst + h * kBoxBytes, &mapK, full_bar(st), 64 * h, w.hk / p.kv_rep, t0, w.b);
+                        tma_load_4d(dst + (NH + h) * kBoxBytes, &mapV, full_bar(st), 64 * h, w.hk / p.kv_rep, t0, w.b);
                     }
                     n_issued = gi + 1;
                 }
@@ -379,8 +380,9 @@ decode_merge_kernel(const DecodeParams p) {
     load_row(p.q + (size_t(b) * p.H + h) * D, q);
 #pragma unroll
     for (int c = 0; c < FPL; ++c) q[c] *= p.scale_log2;
-    const size_t slot_stride = size_t(p.B) * p.Hk * 2 * D;                          // elements between depth slots
-    const __nv_bfloat16* depth0 = p.depth + (size_t(b) * p.Hk + hk) * 2 * D;        // slot 0: key row, value row at + D
+    const size_t slot_stride = size_t(p.B) * (p.Hk / p.kv_rep) * 2 * D;             // elements between depth slots
+    const int Hk_real = p.Hk / p.kv_rep;                                            // p.Hk counts groups of at most 8 heads
+    const __nv_bfloat16* depth0 = p.depth + (size_t(b) * Hk_real + hk / p.kv_rep) * 2 * D;   // slot 0: key row, value row at + D
 
     // ---- depth scores: warp `warp` takes slots warp, warp + 4, ..., UN at a time ----
     for (int i0 = warp; i0 < p.l; i0 += NW * UN) {

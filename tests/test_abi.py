@@ -100,7 +100,7 @@ def test_decode_entry_point_validates_before_touching_the_device():
     assert call(T_kv=0) == -3 and call(T_kv=17) == -3 and call(B=0) == -3
     assert call(d=96) == -4
     assert call(l=-1) == -5 and call(l=257) == -5
-    assert call(H=8, Hk=3) == -12 and call(H=16, Hk=1) == -12 and call(Hk=0) == -12
+    assert call(H=8, Hk=3) == -12 and call(H=12, Hk=1) == -12 and call(Hk=0) == -12
     assert call(q=None) == -1 and call(depth=None) == -1 and call(l=0, depth=None) != -1
     assert call(q=ctypes.c_void_p(4100)) == -2
     assert call(work=None) == -7 and call(wb=16) == -7

@@ -17,6 +17,7 @@ SHAPES = [
     (2, 256, 256, 8, 1, 64, 4), (1, 257, 512, 6, 2, 128, 1), (3, 1000, 1024, 4, 4, 64, 7), (1, 5000, 5000, 8, 2, 128, 24),
     (2, 4097, 4100, 16, 2, 64, 64), (1, 20000, 20000, 3, 1, 128, 256), (1, 3000, 3000, 5, 1, 64, 0), (1, 777, 777, 7, 1, 128, 9),
     # many (batch, kv head) groups: few splits, so every CTA goes round its shared-memory ring several times
+    (2, 1300, 1300, 32, 2, 128, 3), (1, 900, 1000, 32, 1, 64, 5), (3, 400, 400, 16, 1, 128, 2),      # G = 16, 32
     (16, 4096, 4096, 16, 8, 128, 4), (24, 6000, 6016, 16, 8, 64, 3), (40, 2500, 2500, 8, 8, 128, 2),
 ]
 

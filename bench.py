@@ -502,10 +502,26 @@ def run_decode_sweep(peaks, device, shapes=None, iters=20):
             ms_eager, ms = ms, ms_graph
         else:
             ms_eager = ms
+        # the same cache seen as 64-position pages in a shuffled order (host launches, rotating sets)
+        paged_us = None
+        if T % 64 == 0:
+            blocks = T // 64
+            gen = torch.Generator(device=device).manual_seed(7)
+            tables = [torch.randperm(B * blocks, generator=gen, device=device).to(torch.int32).view(B, blocks).contiguous()
+                      for _ in range(n_sets)]
+            lens = torch.full((B,), T, dtype=torch.int32, device=device)
+
+            def fn_paged(i):
+                x = sets[i % n_sets]
+                moda.moda_attn_decode_paged(x["q"], x["K"].view(B * blocks, 64, Hk, d), x["V"].view(B * blocks, 64, Hk, d),
+                                            tables[i % n_sets], lens, x["depth"] if l else None, T, l, d ** -0.5,
+                                            O=O, LSE=LSE, workspace=ws)
+            paged_us = time_calls(lambda c=[0]: (fn_paged(c[0]), c.__setitem__(0, c[0] + 1)), iters, warm=max(3, n_sets)) * 1e3
         byt = 2 * B * T * Hk * d * 2 + 2 * l * B * Hk * d * 2 + 2 * B * H * d * 2
         gbs = byt / ms / 1e6
         rows.append({"B": B, "T_kv": T, "H": H, "H_kv": Hk, "G": H // Hk, "d": d, "l": l, "us": round(ms * 1e3, 1),
                      "us_launched_from_host": round(ms_eager * 1e3, 1), "timed": "cuda graph replay" if ms is not ms_eager else "host launches",
+                     "us_paged_64_host_launches": None if paged_us is None else round(paged_us, 1),
                      "algorithmic_GB": round(byt / 1e9, 3), "GBps": round(gbs, 0),
                      "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 3),
                      "tokens_per_s": round(B / ms * 1e3, 0)})

@@ -227,6 +227,33 @@ int moda_attn_decode(const void* q, const void* K, const void* V, const void* de
                      void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The decode step for a serving batch: sequences of different lengths, and a paged KV cache.
+ * (Beyond the paper, which states the decode step's cache size and FLOPs only; same operator per
+ * sequence as moda_attn_decode.)
+ *
+ * moda_attn_decode_varlen: as moda_attn_decode, but sequence b has seq_lens[b] cached positions
+ *     (device int32 [B], 4-byte aligned, each in [1, max_seq_len]; values outside are clamped);
+ *     max_seq_len <= T_cap sizes the split of the key range.
+ * moda_attn_decode_paged: K and V live in pages,
+ *     K_pages, V_pages : bf16 [num_pages][page_size][H_kv][d], page_size a multiple of 64
+ *     block_table      : device int32 [B][max_blocks_per_seq]; entry j of row b is the page that holds
+ *                        positions [j page_size, (j + 1) page_size) of sequence b; entries past the
+ *                        sequence's last block are not read; every entry read must be in [0, num_pages)
+ *     seq_lens         : device int32 [B] as above; max_blocks_per_seq * page_size >= max_seq_len
+ * Everything else (q, depth_kv_token, O, LSE, workspace, groups, validation, launches) is as for
+ * moda_attn_decode.  Positions of a page past the sequence's length may hold anything.
+ */
+int moda_attn_decode_varlen(const void* q, const void* K, const void* V, const int* seq_lens,
+                            const void* depth_kv_token,
+                            int B, int max_seq_len, int T_cap, int H, int H_kv, int d, int l, float scale,
+                            void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream);
+int moda_attn_decode_paged(const void* q, const void* K_pages, const void* V_pages,
+                           const int* block_table, const int* seq_lens, const void* depth_kv_token,
+                           int B, int max_seq_len, int page_size, int num_pages, int max_blocks_per_seq,
+                           int H, int H_kv, int d, int l, float scale,
+                           void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Backward pass for callers that have no scratch buffer to give.  (The paper has no
  * counterpart: this is a deployment convenience of this library, not part of the method.)
  *

@@ -21,6 +21,8 @@ from .binding import (  # noqa: F401
     moda_attn_bwd_stages,
     moda_attn_bwd_static_scratch,
     moda_attn_decode,
+    moda_attn_decode_paged,
+    moda_attn_decode_varlen,
     moda_attn_fwd,
     moda_attn_fwd_gqa,
     moda_attn_fwd_prefill,

@@ -23,6 +23,7 @@ SYMBOLS = (
     "moda_attn_bwd_static_scratch",
     "moda_attn_fwd_gqa", "moda_bwd_workspace_bytes_gqa", "moda_attn_bwd_gqa", "moda_attn_bwd_gqa_stages",
     "moda_decode_workspace_bytes", "moda_attn_decode", "moda_attn_fwd_prefill",
+    "moda_attn_decode_varlen", "moda_attn_decode_paged",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -80,6 +81,10 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd_gqa.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
     lib.moda_attn_bwd_gqa_stages.restype = ci
     lib.moda_attn_bwd_gqa_stages.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, ci, vp]
+    lib.moda_attn_decode_varlen.restype = ci
+    lib.moda_attn_decode_varlen.argtypes = [vp] * 5 + [ci] * 7 + [cf] + [vp] * 3 + [sz, vp]
+    lib.moda_attn_decode_paged.restype = ci
+    lib.moda_attn_decode_paged.argtypes = [vp] * 6 + [ci] * 9 + [cf] + [vp] * 3 + [sz, vp]
     lib.moda_attn_fwd_prefill.restype = ci
     lib.moda_attn_fwd_prefill.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
     lib.moda_decode_workspace_bytes.restype = sz
@@ -341,4 +346,54 @@ def moda_attn_fwd_prefill(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=
     _check(load().moda_attn_fwd_prefill(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
                                         B, T_q, T_kv, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
                                         _stream(stream)), "moda_attn_fwd_prefill")
+    return O, LSE
+
+
+def _decode_outputs(q, O, LSE, workspace):
+    B, H, d = q.shape
+    if O is None:
+        O = torch.empty_like(q)
+    if LSE is None:
+        LSE = torch.empty((B, H), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(moda_decode_workspace_bytes(B, H, d), dtype=torch.uint8, device=q.device)
+    return O, LSE, workspace
+
+
+def _int32(t, name, shape):
+    if t.dtype != torch.int32 or tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must be an int32 tensor of shape {tuple(shape)}")
+    return t
+
+
+def moda_attn_decode_varlen(q, K, V, seq_lens, depth_kv_token, max_seq_len, l, scale, O=None, LSE=None,
+                            workspace=None, stream=None):
+    """Decode step with a length per sequence: seq_lens int32 [B] (device), each in [1, max_seq_len]."""
+    B, H, d = q.shape
+    _, T_cap, Hk, _ = _bthd(K, "K")
+    _int32(seq_lens, "seq_lens", (B,))
+    O, LSE, workspace = _decode_outputs(q, O, LSE, workspace)
+    _check(load().moda_attn_decode_varlen(_ptr(q), _ptr(K), _ptr(V), _ptr(seq_lens), _ptr(depth_kv_token) if l > 0 else None,
+                                          B, int(max_seq_len), T_cap, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
+                                          _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "moda_attn_decode_varlen")
+    return O, LSE
+
+
+def moda_attn_decode_paged(q, K_pages, V_pages, block_table, seq_lens, depth_kv_token, max_seq_len, l, scale,
+                           O=None, LSE=None, workspace=None, stream=None):
+    """Decode step over a paged KV cache: K_pages, V_pages [num_pages, page_size, H_kv, d]; block_table int32
+    [B, max_blocks]; seq_lens int32 [B]."""
+    B, H, d = q.shape
+    num_pages, page_size, Hk, _ = _bthd(K_pages, "K_pages")
+    _int32(seq_lens, "seq_lens", (B,))
+    if block_table.dtype != torch.int32 or block_table.dim() != 2 or block_table.shape[0] != B:
+        raise ValueError("block_table must be an int32 [B, max_blocks] tensor")
+    O, LSE, workspace = _decode_outputs(q, O, LSE, workspace)
+    _check(load().moda_attn_decode_paged(_ptr(q), _ptr(K_pages), _ptr(V_pages), _ptr(block_table), _ptr(seq_lens),
+                                         _ptr(depth_kv_token) if l > 0 else None,
+                                         B, int(max_seq_len), page_size, num_pages, block_table.shape[1], H, Hk, d, int(l),
+                                         float(scale), _ptr(O), _ptr(LSE), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)),
+           "moda_attn_decode_paged")
     return O, LSE

@@ -240,8 +240,10 @@ template <int D, int G>
 int launch_decode_g(const DecodeParams& p, cudaStream_t stream) {
     using L = DecodeSmem<D, G>;
     CUtensorMap mK, mV;
-    if (!make_bthd_map(&mK, p.K, p.B, p.T_cap, p.Hk / p.kv_rep, D, kDecodeStageKeys) ||
-        !make_bthd_map(&mV, p.V, p.B, p.T_cap, p.Hk / p.kv_rep, D, kDecodeStageKeys))
+    // contiguous cache: [B][T_cap][Hk][d]; paged cache: [num_pages][page_size][Hk][d] (p.T_cap holds num_pages then)
+    const int outer = p.block_table ? p.T_cap : p.B, rows = p.block_table ? p.page_size : p.T_cap;
+    if (!make_bthd_map(&mK, p.K, outer, rows, p.Hk / p.kv_rep, D, kDecodeStageKeys) ||
+        !make_bthd_map(&mV, p.V, outer, rows, p.Hk / p.kv_rep, D, kDecodeStageKeys))
         return MODA_ERR_CUDA;
     static thread_local int configured_dev = -1;
     int dev = 0;
@@ -285,6 +287,48 @@ int device_sm_count(int* out) {
     }
     *out = cached_sms;
     return MODA_OK;
+}
+
+// The decode step behind its three entry points: contiguous cache with one length, contiguous cache with a
+// length per sequence, paged cache (T_cap then counts pages).
+int decode_common(const void* q, const void* K, const void* V, const int* seq_lens, const int* block_table,
+                  const void* depth_kv_token, int B, int T_kv, int T_cap, int page_size, int max_blocks,
+                  int H, int H_kv, int d, int l, float scale,
+                  void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream) {
+    const bool paged = block_table != nullptr;
+    if (B < 1 || T_kv < 1 || H < 1 || (!paged && T_cap < T_kv)) return MODA_ERR_BAD_SHAPE;
+    if (d != 64 && d != 128) return MODA_ERR_BAD_HEAD_DIM;
+    if ((long long)(paged ? page_size : B) * T_cap > 0x7fffffffLL / H) return MODA_ERR_BAD_SHAPE;
+    if (int rc = check_groups(H, H_kv)) return rc;
+    if ((long long)B * H * kDecodeMaxSplits > 0x7fffffffLL || B > 65535) return MODA_ERR_BAD_SHAPE;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (!q || !K || !V || !O || !LSE || (l > 0 && !depth_kv_token)) return MODA_ERR_NULL_POINTER;
+    if ((seq_lens && (reinterpret_cast<uintptr_t>(seq_lens) & 3u)) || (block_table && (reinterpret_cast<uintptr_t>(block_table) & 3u)))
+        return MODA_ERR_MISALIGNED;
+    if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
+        (l > 0 && !aligned16(depth_kv_token)))
+        return MODA_ERR_MISALIGNED;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < decode_workspace_bytes(B, H, d)) return MODA_ERR_WORKSPACE;
+    if (int rc = check_device()) return rc;
+    int sms = 0;
+    if (int rc = device_sm_count(&sms)) return rc;
+    DecodeParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.K = static_cast<const __nv_bfloat16*>(K);
+    p.V = static_cast<const __nv_bfloat16*>(V);
+    p.depth = static_cast<const __nv_bfloat16*>(depth_kv_token);
+    p.O = static_cast<__nv_bfloat16*>(O);
+    p.LSE = LSE;
+    p.part = static_cast<float*>(workspace);
+    // 16 or 32 query heads per key/value head: groups of 8 heads that read the same K, V head
+    const int kv_rep = (H / H_kv > 8) ? (H / H_kv) / 8 : 1;
+    p.B = B; p.T_kv = T_kv; p.T_cap = T_cap; p.H = H; p.Hk = H_kv * kv_rep; p.l = l; p.kv_rep = kv_rep;
+    p.seq_lens = seq_lens; p.block_table = block_table; p.page_size = page_size; p.max_blocks = max_blocks;
+    const DecodePlan plan = decode_plan(B, p.Hk, T_kv, sms);
+    p.S = plan.S; p.keys_per_split = plan.keys_per_split; p.num_sms = sms;
+    p.scale_log2 = scale * kDecodeLog2e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_decode<128>(p, st) : launch_decode<64>(p, st);
 }
 
 }  // namespace
@@ -456,36 +500,30 @@ size_t moda_decode_workspace_bytes(int B, int H, int d) {
 int moda_attn_decode(const void* q, const void* K, const void* V, const void* depth_kv_token,
                      int B, int T_kv, int T_cap, int H, int H_kv, int d, int l, float scale,
                      void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream) {
-    if (B < 1 || T_kv < 1 || T_cap < T_kv || H < 1) return MODA_ERR_BAD_SHAPE;
-    if (d != 64 && d != 128) return MODA_ERR_BAD_HEAD_DIM;
-    if ((long long)B * T_cap > 0x7fffffffLL / H) return MODA_ERR_BAD_SHAPE;
-    if (int rc = check_groups(H, H_kv)) return rc;
-    if ((long long)B * H * kDecodeMaxSplits > 0x7fffffffLL || B > 65535) return MODA_ERR_BAD_SHAPE;
-    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
-    if (!q || !K || !V || !O || !LSE || (l > 0 && !depth_kv_token)) return MODA_ERR_NULL_POINTER;
-    if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
-        (l > 0 && !aligned16(depth_kv_token)))
-        return MODA_ERR_MISALIGNED;
-    if (!workspace || !aligned16(workspace) || workspace_bytes < decode_workspace_bytes(B, H, d)) return MODA_ERR_WORKSPACE;
-    if (int rc = check_device()) return rc;
-    int sms = 0;
-    if (int rc = device_sm_count(&sms)) return rc;
-    DecodeParams p;
-    p.q = static_cast<const __nv_bfloat16*>(q);
-    p.K = static_cast<const __nv_bfloat16*>(K);
-    p.V = static_cast<const __nv_bfloat16*>(V);
-    p.depth = static_cast<const __nv_bfloat16*>(depth_kv_token);
-    p.O = static_cast<__nv_bfloat16*>(O);
-    p.LSE = LSE;
-    p.part = static_cast<float*>(workspace);
-    // 16 or 32 query heads per key/value head: groups of 8 heads that read the same K, V head
-    const int kv_rep = (H / H_kv > 8) ? (H / H_kv) / 8 : 1;
-    p.B = B; p.T_kv = T_kv; p.T_cap = T_cap; p.H = H; p.Hk = H_kv * kv_rep; p.l = l; p.kv_rep = kv_rep;
-    const DecodePlan plan = decode_plan(B, p.Hk, T_kv, sms);
-    p.S = plan.S; p.keys_per_split = plan.keys_per_split; p.num_sms = sms;
-    p.scale_log2 = scale * kDecodeLog2e;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return d == 128 ? launch_decode<128>(p, st) : launch_decode<64>(p, st);
+    return decode_common(q, K, V, nullptr, nullptr, depth_kv_token, B, T_kv, T_cap, 0, 0, H, H_kv, d, l, scale,
+                         O, LSE, workspace, workspace_bytes, stream);
+}
+
+int moda_attn_decode_varlen(const void* q, const void* K, const void* V, const int* seq_lens,
+                            const void* depth_kv_token,
+                            int B, int max_seq_len, int T_cap, int H, int H_kv, int d, int l, float scale,
+                            void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!seq_lens) return MODA_ERR_NULL_POINTER;
+    return decode_common(q, K, V, seq_lens, nullptr, depth_kv_token, B, max_seq_len, T_cap, 0, 0, H, H_kv, d, l, scale,
+                         O, LSE, workspace, workspace_bytes, stream);
+}
+
+int moda_attn_decode_paged(const void* q, const void* K_pages, const void* V_pages,
+                           const int* block_table, const int* seq_lens, const void* depth_kv_token,
+                           int B, int max_seq_len, int page_size, int num_pages, int max_blocks_per_seq,
+                           int H, int H_kv, int d, int l, float scale,
+                           void* O, float* LSE, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!block_table || !seq_lens) return MODA_ERR_NULL_POINTER;
+    if (page_size < kDecodeStageKeys || page_size % kDecodeStageKeys != 0 || num_pages < 1 || max_blocks_per_seq < 1 ||
+        (long long)max_blocks_per_seq * page_size < max_seq_len)
+        return MODA_ERR_BAD_SHAPE;
+    return decode_common(q, K_pages, V_pages, seq_lens, block_table, depth_kv_token, B, max_seq_len, num_pages, page_size,
+                         max_blocks_per_seq, H, H_kv, d, l, scale, O, LSE, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -49,6 +49,9 @@ struct DecodeParams {
     int S, keys_per_split;        // keys_per_split is a multiple of kDecodeKeysPerPass
     int num_sms;
     int kv_rep;                   // groups of more than 8 query heads run as kv_rep groups of 8 on the same K, V head
+    const int* seq_lens;          // [B] cached positions per sequence (each 1 .. T_kv), or null: T_kv for all
+    const int* block_table;       // paged cache: [B][max_blocks] page of every block of page_size positions, or null
+    int page_size, max_blocks;    // paged cache: K, V are [num_pages][page_size][Hk][d]; page_size is a multiple of 64
     float scale_log2;             // scale * log2(e)
 };
 
@@ -147,7 +150,8 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
         w.hk = bh % p.Hk;
         w.b = bh / p.Hk;
         w.k_begin = w.split * p.keys_per_split;
-        w.k_end = min(p.T_kv, w.k_begin + p.keys_per_split);
+        const int len = p.seq_lens ? min(max(p.seq_lens[w.b], 1), p.T_kv) : p.T_kv;   // this sequence's cached positions
+        w.k_end = min(len, w.k_begin + p.keys_per_split);
         w.n_stage = max(0, (w.k_end - w.k_begin + kDecodeStageKeys - 1) / kDecodeStageKeys);
         return w;
     };
@@ -167,18 +171,26 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
             tma_prefetch_desc(&mapV);
             for (int it = blockIdx.x; it < n_items && *abort_flag == 0; it += gridDim.x) {
                 const Item w = item_of(it);
+                // paged cache: the page of a stage's 64 positions comes from the sequence's block table; the
+                // entry of the next stage is requested before this stage's wait, so its latency is hidden
+                const int* table = p.block_table ? p.block_table + size_t(w.b) * p.max_blocks : nullptr;
+                int page_next = (table && w.n_stage > 0) ? table[w.k_begin / p.page_size] : 0;
                 for (int i = 0; i < w.n_stage; ++i) {
                     const int gi = n_issued;
                     const int st = gi % L::kStages;
+                    const int t0 = w.k_begin + i * kDecodeStageKeys;
+                    const int page = page_next;
+                    if (table && i + 1 < w.n_stage) page_next = table[(t0 + kDecodeStageKeys) / p.page_size];
                     if (gi >= L::kStages) mbar_wait(empty_bar(st), ((gi / L::kStages) - 1) & 1, abort_flag, 70);
                     if (*abort_flag != 0) break;
                     const uint32_t dst = smem_u32(smem + L::kRing + st * L::kStageBytes);
                     mbar_arrive_expect_tx(full_bar(st), L::kStageBytes);
-                    const int t0 = w.k_begin + i * kDecodeStageKeys;
+                    const int c2 = table ? t0 % p.page_size : t0;          // position inside the page / the sequence
+                    const int c3 = table ? page : w.b;                     // page / batch index
 #pragma unroll
                     for (int h = 0; h < NH; ++h) {
-                        tma_load_4d(dst + h * kBoxBytes, &mapK, full_bar(st), 64 * h, w.hk / p.kv_rep, t0, w.b);
-                        tma_load_4d(dst + (NH + h) * kBoxBytes, &mapV, full_bar(st), 64 * h, w.hk / p.kv_rep, t0, w.b);
+                        tma_load_4d(dst + h * kBoxBytes, &mapK, full_bar(st), 64 * h, w.hk / p.kv_rep, c2, c3);
+                        tma_load_4d(dst + (NH + h) * kBoxBytes, &mapV, full_bar(st), 64 * h, w.hk / p.kv_rep, c2, c3);
                     }
                     n_issued = gi + 1;
                 }

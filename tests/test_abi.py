@@ -115,3 +115,20 @@ def test_prefill_entry_point_validates_before_touching_the_device():
     assert call(64, 128, H=6, Hk=4) == -12
     assert call(64, 128, l=2) == -1            # depth cache missing
     assert call(64, 128, Q=None) == -1
+
+
+def test_paged_decode_entry_point_validates_before_touching_the_device():
+    lib = binding.load()
+    p = ctypes.c_void_p(4096)
+    ws = lib.moda_decode_workspace_bytes(2, 8, 128)
+
+    def call(page=64, pages=10, blocks=4, max_len=200, table=p, lens=p):
+        return lib.moda_attn_decode_paged(p, p, p, table, lens, None, 2, max_len, page, pages, blocks, 8, 2, 128, 0,
+                                          ctypes.c_float(0.1), p, p, p, ctypes.c_size_t(ws), None)
+
+    assert call(page=48) == -3 and call(page=32) == -3 and call(pages=0) == -3
+    assert call(blocks=3, max_len=200) == -3                      # 3 x 64 < 200
+    assert call(table=None) == -1 and call(lens=None) == -1
+    assert call(lens=ctypes.c_void_p(4098)) == -2
+    assert lib.moda_attn_decode_varlen(p, p, p, None, None, 2, 100, 128, 8, 2, 128, 0, ctypes.c_float(0.1), p, p, p,
+                                       ctypes.c_size_t(ws), None) == -1

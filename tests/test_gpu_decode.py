@@ -102,3 +102,58 @@ def test_back_to_back_decode_steps_are_bitwise_repeatable():
                                         f64(x["depth"][:, b:b + 1, :, 0]), f64(x["depth"][:, b:b + 1, :, 1]), d ** -0.5)
         assert rel_l2(f64(outs[0][0][b:b + 1]), o_ref) <= TOL_O_REL_L2
         assert np.abs(f64(outs[0][1][b:b + 1]) - lse_ref).max() <= TOL_LSE_ABS
+
+
+def oracle_rows(x, lens, l, scale):
+    outs = []
+    for b, n in enumerate(lens):
+        kd = f64(x["depth"][:, b:b + 1, :, 0]) if l else None
+        vd = f64(x["depth"][:, b:b + 1, :, 1]) if l else None
+        outs.append(orc.decode_gqa(f64(x["q"][b:b + 1]), f64(x["K"][b:b + 1, :n]), f64(x["V"][b:b + 1, :n]), kd, vd, scale))
+    return np.concatenate([o for o, _ in outs]), np.concatenate([s for _, s in outs])
+
+
+@pytest.mark.parametrize("B,T_max,H,Hk,d,l", [(5, 700, 8, 2, 128, 3), (9, 3000, 4, 4, 64, 6), (3, 130, 16, 1, 128, 0)])
+def test_decode_with_a_length_per_sequence(B, T_max, H, Hk, d, l):
+    x = synthetic.make_decode(B, T_max, H, Hk, d, l, seed=31, device="cuda")
+    rng = np.random.default_rng(B)
+    lens = [1, T_max] + [int(v) for v in rng.integers(1, T_max + 1, size=B - 2)]
+    seq_lens = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    scale = d ** -0.5
+    O, LSE = moda.moda_attn_decode_varlen(x["q"], x["K"], x["V"], seq_lens, x["depth"] if l else None, T_max, l, scale)
+    assert moda.moda_last_status() == 0
+    o_ref, lse_ref = oracle_rows(x, lens, l, scale)
+    assert rel_l2(f64(O), o_ref) <= TOL_O_REL_L2
+    assert np.abs(f64(LSE) - lse_ref).max() <= TOL_LSE_ABS
+
+
+@pytest.mark.parametrize("B,T_max,H,Hk,d,l,page", [(4, 1000, 8, 2, 128, 4, 64), (6, 2500, 4, 2, 64, 2, 128), (2, 300, 16, 2, 128, 3, 256)])
+def test_decode_over_a_paged_cache(B, T_max, H, Hk, d, l, page):
+    """Pages scattered by a random permutation; unused page tails and unused pages poisoned with NaN."""
+    x = synthetic.make_decode(B, T_max, H, Hk, d, l, seed=33, device="cuda")
+    rng = np.random.default_rng(T_max)
+    lens = [T_max] + [int(v) for v in rng.integers(1, T_max + 1, size=B - 1)]
+    blocks = (T_max + page - 1) // page
+    num_pages = B * blocks + 3
+    perm = rng.permutation(num_pages)
+    Kp = torch.full((num_pages, page, Hk, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Vp = torch.full_like(Kp, float("nan"))
+    table = torch.full((B, blocks), -1, dtype=torch.int32, device="cuda")
+    k = 0
+    for b, n in enumerate(lens):
+        for j in range((n + page - 1) // page):
+            pg = int(perm[k]); k += 1
+            m = min(page, n - j * page)
+            Kp[pg, :m] = x["K"][b, j * page:j * page + m]
+            Vp[pg, :m] = x["V"][b, j * page:j * page + m]
+            table[b, j] = pg
+    seq_lens = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    scale = d ** -0.5
+    O, LSE = moda.moda_attn_decode_paged(x["q"], Kp, Vp, table, seq_lens, x["depth"] if l else None, T_max, l, scale)
+    assert moda.moda_last_status() == 0
+    o_ref, lse_ref = oracle_rows(x, lens, l, scale)
+    assert rel_l2(f64(O), o_ref) <= TOL_O_REL_L2
+    assert np.abs(f64(LSE) - lse_ref).max() <= TOL_LSE_ABS
+    # the contiguous entry point with the same lengths gives the same bits
+    O2, LSE2 = moda.moda_attn_decode_varlen(x["q"], x["K"], x["V"], seq_lens, x["depth"] if l else None, T_max, l, scale)
+    assert torch.equal(O, O2) and torch.equal(LSE, LSE2)

@@ -145,8 +145,11 @@ decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_c
     struct Item { int b, hk, split, k_begin, k_end, n_stage; };
     auto item_of = [&](int it) {
         Item w;
-        w.split = it % p.S;
-        const int bh = it / p.S;
+        // split-major order: a CTA's items (it, it + grid, ...) then come from all parts of the key range, so
+        // the empty late splits of short sequences spread over the CTAs instead of emptying some of them
+        const int groups = p.B * p.Hk;
+        w.split = it / groups;
+        const int bh = it - w.split * groups;
         w.hk = bh % p.Hk;
         w.b = bh / p.Hk;
         w.k_begin = w.split * p.keys_per_split;

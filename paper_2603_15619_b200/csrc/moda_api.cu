@@ -9,6 +9,7 @@
 #include "moda_bwd.cuh"
 #include "moda_cache.cuh"
 #include "moda_decode.cuh"
+#include "moda_depth_gqa.cuh"
 #include "moda_fwd.cuh"
 #include "moda_fwd_wide.cuh"
 #include "sm100_ptx.cuh"
@@ -107,6 +108,44 @@ inline bool fwd_depth_heavy(int T, int l, int d) {
     return d == 128 && l > 0 && 2ll * l * d >= T;
 }
 
+// Whether a grouped-query forward runs its depth part as the separate per-position kernel.  Measured at
+// d = 64 (T = 16384, 8 key/value heads): the fused row-local path costs about 2.3 us per (query head per
+// group, slot), the separate kernel about 200 us plus 11.7 us per slot whatever the group size, so the
+// separate kernel wins for large groups with many slots (G = 8 from l = 31, G = 7 from 46, G = 6 from 96).
+// At d = 128 it was slower on every shape tried (G <= 4); those calls stay on the fused path.
+inline bool gqa_depth_split(int d, int G, int l) {
+    return d == 64 && G >= 6 && G <= 8 && l * (23 * G - 117) > 2000;
+}
+
+template <int D, int G>
+int launch_depth_merge_g(const DepthMergeParams& m, cudaStream_t stream) {
+    constexpr int kBytes = depth_merge_smem_bytes<D>();
+    static thread_local int configured_dev = -1;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (configured_dev != dev) {
+        if (!set_smem_limit(depth_merge_fwd_kernel<D, G>, kBytes)) return MODA_ERR_CUDA;
+        configured_dev = dev;
+    }
+    const long long blocks = (long long)m.B * m.Hk * ((m.T + kDgPos - 1) / kDgPos);
+    if (blocks > 0x7fffffffLL) return MODA_ERR_BAD_SHAPE;
+    depth_merge_fwd_kernel<D, G><<<unsigned(blocks), kDgThreads, kBytes, stream>>>(m);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+template <int D>
+int launch_depth_merge(const DepthMergeParams& m, cudaStream_t stream) {
+    switch (m.H / m.Hk) {
+        case 2: return launch_depth_merge_g<D, 2>(m, stream);
+        case 3: return launch_depth_merge_g<D, 3>(m, stream);
+        case 4: return launch_depth_merge_g<D, 4>(m, stream);
+        case 5: return launch_depth_merge_g<D, 5>(m, stream);
+        case 6: return launch_depth_merge_g<D, 6>(m, stream);
+        case 7: return launch_depth_merge_g<D, 7>(m, stream);
+        case 8: return launch_depth_merge_g<D, 8>(m, stream);
+        default: return MODA_ERR_BAD_GROUP;
+    }
+}
+
 template <int D>
 int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int T_kv, int H, int Hk, int l,
                float scale, void* O, float* LSE, cudaStream_t stream) {
@@ -136,10 +175,25 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.G = H / Hk;
     p.scale_log2 = scale * kLog2e;
     const unsigned grid = unsigned(B) * H * num_tiles(T);
+    // Grouped-query calls: the sequence kernel runs without depth slots and a second kernel adds the depth
+    // part of all heads of a group at once (moda_depth_gqa.cuh).
+    const bool split_depth = gqa_depth_split(D, p.G, l);
+    if (split_depth) p.l = 0;
     if (kWide) moda_fwd2_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
-    else if (fwd_depth_heavy(T, l, D)) moda_fwd_kernel<128, 1><<<grid, kThreads, kSmemDeep, stream>>>(mQ, mK, mV, mO, p);
+    else if (!split_depth && fwd_depth_heavy(T, l, D)) moda_fwd_kernel<128, 1><<<grid, kThreads, kSmemDeep, stream>>>(mQ, mK, mV, mO, p);
     else moda_fwd_kernel<D, 2><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
-    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+    if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    if (split_depth) {
+        DepthMergeParams m;
+        m.Q = static_cast<const __nv_bfloat16*>(Q);
+        m.depth_kv = static_cast<const __nv_bfloat16*>(depth_kv);
+        m.O = static_cast<__nv_bfloat16*>(O);
+        m.LSE = LSE;
+        m.B = B; m.T = T; m.H = H; m.Hk = Hk; m.l = l;
+        m.scale_log2 = scale * kLog2e;
+        if (int rc = launch_depth_merge<D>(m, stream)) return rc;
+    }
+    return MODA_OK;
 }
 
 // Which dQ kernel at d = 128: two K/V stages and a five-unit depth ring when streaming the depth cache

@@ -106,17 +106,24 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
 
     // stages the K and V rows of slots [s0, s0 + ns) of the CTA's positions into buffer `buf`: 16-byte pieces,
     // the eight positions of a piece are one 128-byte line of the cache
+    // A thread always copies the same (position, chunk) piece: kDgThreads is a multiple of kDgPos * CH, so only the
+    // slot advances from one copy to the next.
+    static_assert(kDgThreads % (kDgPos * CH) == 0, "one (position, chunk) per thread");
+    constexpr int kSlotStep = kDgThreads / (kDgPos * CH);          // slots between a thread's copies
+    const int st_pos = threadIdx.x % kDgPos, st_chunk = (threadIdx.x / kDgPos) % CH, st_slot0 = threadIdx.x / (kDgPos * CH);
+    const __nv_bfloat16* st_src = cbase + (size_t(st_chunk) * kTileRows + st_pos) * 8;
+    const uint32_t st_dst = smem_base + st_pos * kDgSlots * D * 2 + ((st_chunk & 8) << 4);
     auto stage_round = [&](int s0, int buf) {
         const int ns = min(kDgSlots, p.l - s0);
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
-            const __nv_bfloat16* src0 = cbase + size_t(s0) * slot_elems + size_t(kv) * cache_block_elems(D);
-            for (int e = threadIdx.x; e < ns * CH * kDgPos; e += kDgThreads) {
-                const int pos = e % kDgPos;
-                const int chunk = (e / kDgPos) % CH;
-                const int slot = e / (kDgPos * CH);
-                cp_async_16(smem_base + (buf * 2 + kv) * kTensorBytes + dg_row_piece<D>(pos, slot, chunk),
-                            src0 + size_t(slot) * slot_elems + (size_t(chunk) * kTileRows + pos) * 8);
+            const __nv_bfloat16* src = st_src + size_t(s0 + st_slot0) * slot_elems + size_t(kv) * cache_block_elems(D);
+            const uint32_t dst = st_dst + (buf * 2 + kv) * kTensorBytes;
+#pragma unroll
+            for (int k = 0; k < kDgSlots / kSlotStep; ++k) {
+                const int slot = st_slot0 + k * kSlotStep;
+                if (slot < ns)
+                    cp_async_16(dst + slot * D * 2 + (((st_chunk & 7) ^ (slot & 7)) << 4), src + size_t(k * kSlotStep) * slot_elems);
             }
         }
         cp_async_commit();

@@ -114,6 +114,7 @@ inline bool fwd_depth_heavy(int T, int l, int d) {
 // separate kernel wins for large groups with many slots (G = 8 from l = 31, G = 7 from 46, G = 6 from 96).
 // At d = 128 it was slower on every shape tried (G <= 4); those calls stay on the fused path.
 inline bool gqa_depth_split(int d, int G, int l) {
+    if (G == 16 || G == 32) return d == 64 && l >= 31;             // run as groups of 8 heads on the same slots
     return d == 64 && G >= 6 && G <= 8 && l * (23 * G - 117) > 2000;
 }
 
@@ -133,8 +134,10 @@ int launch_depth_merge_g(const DepthMergeParams& m, cudaStream_t stream) {
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 template <int D>
-int launch_depth_merge(const DepthMergeParams& m, cudaStream_t stream) {
-    switch (m.H / m.Hk) {
+int launch_depth_merge(DepthMergeParams m, cudaStream_t stream) {
+    const int G = m.H / m.Hk;
+    m.h0 = 0;
+    switch (G) {
         case 2: return launch_depth_merge_g<D, 2>(m, stream);
         case 3: return launch_depth_merge_g<D, 3>(m, stream);
         case 4: return launch_depth_merge_g<D, 4>(m, stream);
@@ -142,6 +145,10 @@ int launch_depth_merge(const DepthMergeParams& m, cudaStream_t stream) {
         case 6: return launch_depth_merge_g<D, 6>(m, stream);
         case 7: return launch_depth_merge_g<D, 7>(m, stream);
         case 8: return launch_depth_merge_g<D, 8>(m, stream);
+        case 16: case 32:
+            for (m.h0 = 0; m.h0 < G; m.h0 += 8)
+                if (int rc = launch_depth_merge_g<D, 8>(m, stream)) return rc;
+            return MODA_OK;
         default: return MODA_ERR_BAD_GROUP;
     }
 }
@@ -203,6 +210,55 @@ inline bool dq_depth_heavy(int T, int l, int d) {
     return d == 128 && l > 0 && 3ll * l * d >= 2ll * T;
 }
 
+// Whether a grouped-query backward runs its depth part as the separate per-position kernel.
+// Measured (8 key/value heads; d = 64 at T = 16384, d = 128 at T = 8192): the row-local path with its row-term
+// workspace and group kernel costs about 8.8 us (8.5 us) per slot and head of a group, the separate kernel
+// about 0.25-0.45 ms plus 25.8 us (19.6 us) per slot whatever the group size.  Groups of 16 and 32 heads run as
+// groups of 8 whose slot gradients are added up (bf16 additions in launch order).
+inline bool gqa_depth_split_bwd(int d, int G, int l) {
+    if (l <= 0 || G < 2) return false;
+    if (G == 16 || G == 32) return l >= 8;
+    if (G > 8) return false;
+    return d == 64 ? l * (88 * G - 258) > 4500 : l * (85 * G - 196) > 4000;
+}
+
+template <int D, int G>
+int launch_depth_bwd_g(const DepthBwdParams& m, cudaStream_t stream) {
+    constexpr int kBytes = DepthBwdSmem<D>::kTotal;
+    static thread_local int configured_dev = -1;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (configured_dev != dev) {
+        if (!set_smem_limit(depth_bwd_gqa_kernel<D, G>, kBytes)) return MODA_ERR_CUDA;
+        configured_dev = dev;
+    }
+    const long long blocks = (long long)m.B * m.Hk * num_tiles(m.T) * (kTileRows / db_pos<D>());
+    if (blocks > 0x7fffffffLL) return MODA_ERR_BAD_SHAPE;
+    depth_bwd_gqa_kernel<D, G><<<unsigned(blocks), db_pos<D>() * 32, kBytes, stream>>>(m);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+template <int D>
+int launch_depth_bwd(DepthBwdParams m, cudaStream_t stream) {
+    const int G = m.H / m.Hk;
+    m.h0 = 0;
+    switch (G) {
+        case 2: return launch_depth_bwd_g<D, 2>(m, stream);
+        case 3: return launch_depth_bwd_g<D, 3>(m, stream);
+        case 4: return launch_depth_bwd_g<D, 4>(m, stream);
+        case 5: return launch_depth_bwd_g<D, 5>(m, stream);
+        case 6: return launch_depth_bwd_g<D, 6>(m, stream);
+        case 7: return launch_depth_bwd_g<D, 7>(m, stream);
+        case 8: return launch_depth_bwd_g<D, 8>(m, stream);
+        case 16: case 32:
+            for (m.h0 = 0; m.h0 < G; m.h0 += 8) {
+                if (int rc = launch_depth_bwd_g<D, 8>(m, stream)) return rc;
+                m.accumulate = 1;                                   // the later groups of 8 add to the first one's gradients
+            }
+            return MODA_OK;
+        default: return MODA_ERR_BAD_GROUP;
+    }
+}
+
 template <int D>
 int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
     const int B = a.B, T = a.T, H = a.H, Hk = a.Hk, G = a.H / a.Hk;
@@ -239,19 +295,32 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
         p.depth_kv = static_cast<const __nv_bfloat16*>(a.depth_kv);
         p.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
         p.LSE = a.LSE; p.delta = delta;
-        p.B = B; p.T = T; p.H = H; p.l = a.l; p.G = G;
+        const bool split_depth = gqa_depth_split_bwd(D, G, a.l);   // depth gradients by the per-position kernel below
+        p.B = B; p.T = T; p.H = H; p.l = split_depth ? 0 : a.l; p.G = G;
         p.accumulate = a.accumulate_depth ? 1 : 0;
         p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
         // Grouped-query: the dQ kernel leaves R_i, dU_i per (row, slot, head) behind the row terms D_t
         // and a second, write-bound kernel forms the depth gradients as sums over each group.
         float* rowterms = reinterpret_cast<float*>(static_cast<char*>(a.workspace) + bwd_workspace_bytes(B, T, H));
-        p.depth_rowterms = (G > 1 && a.l > 0) ? rowterms : nullptr;
-        if (dq_depth_heavy(T, a.l, D))
+        p.depth_rowterms = (G > 1 && a.l > 0 && !split_depth) ? rowterms : nullptr;
+        if (dq_depth_heavy(T, p.l, D))
             moda_bwd_dq_kernel<128, 2><<<grid, kBwdDqThreads, DqSmem<128, 2>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
         else
             moda_bwd_dq_kernel<D, 3><<<grid, kBwdDqThreads, DqSmem<D, 3>::kDynamic, stream>>>(mQ, mdO, mK64, mV64, mdQ, p);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
-        if (G > 1 && a.l > 0) {
+        if (split_depth) {
+            DepthBwdParams m;
+            m.Q = static_cast<const __nv_bfloat16*>(a.Q);
+            m.dO = static_cast<const __nv_bfloat16*>(a.dO);
+            m.depth_kv = static_cast<const __nv_bfloat16*>(a.depth_kv);
+            m.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
+            m.dQ = static_cast<__nv_bfloat16*>(a.dQ);
+            m.LSE = a.LSE; m.delta = delta;
+            m.B = B; m.T = T; m.H = H; m.Hk = Hk; m.l = a.l;
+            m.scale = a.scale; m.scale_log2 = a.scale * kLog2e;
+            m.accumulate = a.accumulate_depth ? 1 : 0;
+            if (int rc = launch_depth_bwd<D>(m, stream)) return rc;
+        } else if (G > 1 && a.l > 0) {
             const unsigned tiles2 = unsigned(B) * Hk * num_tiles(T) * 2;            // x {dKd, dVd}
             const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.Q);
             const __nv_bfloat16* go = static_cast<const __nv_bfloat16*>(a.dO);

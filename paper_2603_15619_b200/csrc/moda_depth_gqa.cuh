@@ -33,6 +33,7 @@ struct DepthMergeParams {
     __nv_bfloat16* O;                   // in: sequence-only output; out: merged output
     float* LSE;                         // [B][H][T], likewise
     int B, T, H, Hk, l;
+    int h0;                             // first head (inside its group of H / Hk) of the up to 8 heads this launch handles
     float scale_log2;
 };
 
@@ -78,14 +79,14 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
     for (int kp = 0; kp < D / 32; ++kp) {
         qf[kp] = make_uint4(0u, 0u, 0u, 0u);
         if (live && g < G)
-            qf[kp] = *reinterpret_cast<const uint4*>(p.Q + ((size_t(b) * p.T + t) * p.H + hk * G + g) * D + (4 * kp + tq) * 8);
+            qf[kp] = *reinterpret_cast<const uint4*>(p.Q + ((size_t(b) * p.T + t) * p.H + hk * (p.H / p.Hk) + p.h0 + g) * D + (4 * kp + tq) * 8);
     }
 
     // the sequence kernel's output row and LSE of head g, requested now so that they are there at the end
     uint32_t os[D / 8];
     float lse_seq = 0.f;
     if (live && g < G) {
-        const int h = hk * G + g;
+        const int h = hk * (p.H / p.Hk) + p.h0 + g;
         const __nv_bfloat16* orow = p.O + ((size_t(b) * p.T + t) * p.H + h) * D;
 #pragma unroll
         for (int fb = 0; fb < D / 8; ++fb) os[fb] = *reinterpret_cast<const uint32_t*>(orow + 8 * fb + 2 * tq);
@@ -209,7 +210,7 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
     if (live && g < G) {
-        const int h = hk * G + g;
+        const int h = hk * (p.H / p.Hk) + p.h0 + g;
         const float s2 = lse_seq * 1.4426950408889634f;            // sequence LSE in the log2 domain
         const float mt = fmaxf(s2, m_run);
         const float ws = fast_exp2(s2 - mt), wd = fast_exp2(m_run - mt);
@@ -223,6 +224,249 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
             *reinterpret_cast<uint32_t*>(orow + 8 * fb + 2 * tq) = pack_bf16x2(a0, a1);
         }
         if (tq == 0) p.LSE[(size_t(b) * p.H + h) * p.T + t] = (mt + log2f(z)) * 0.6931471805599453f;
+    }
+}
+
+
+// =====================================================================================================
+// Backward of the depth part for grouped-query calls, per position (derived from the forward above; the
+// paper gives no backward).  With R = exp(U - LSE) (G x l; LSE is the forward's, over sequence and depth
+// keys), D_g = <dO_g, O_g> and dU = R o (dO_t Vd_t^T - D):
+//     dQ_t  += scale dU Kd_t          (G x d)
+//     dKd_t  = scale dU^T Q_t         (l x d)   -- the contraction runs over the heads of the group, i.e. it
+//     dVd_t  = R^T dO_t               (l x d)      is the sum over the group that the gradients need
+// All five products are warp MMAs with the heads as the 16-row (or 16-deep) operand.  dU and R leave the
+// first products in accumulator layout [head][slot]; the last two need them as [slot][head], which
+// movmatrix provides (8 x 8 transposes across the warp).  Q_t and dO_t are also needed as B operands
+// [head][feature]: they sit in shared memory and come through transposing matrix loads.
+// The sequence kernel (run without depth slots) has left the sequence part of dQ; this kernel adds its share.
+// =====================================================================================================
+constexpr int kDbRoundSlots = 16;
+template <int D> constexpr int db_pos() { return 512 / D; }           // positions per CTA (one per warp): 8 at d = 64, 4 at d = 128
+
+struct DepthBwdParams {
+    const __nv_bfloat16* Q;             // [B][T][H][d]
+    const __nv_bfloat16* dO;
+    const __nv_bfloat16* depth_kv;      // cache layout, Hk heads
+    __nv_bfloat16* d_depth_kv;          // gradient cache, same layout
+    __nv_bfloat16* dQ;                  // in: sequence part; out: sequence + depth part
+    const float* LSE;                   // [B][H][T]
+    const float* delta;                 // [B][H][T], D_t = <dO_t, O_t>
+    int B, T, H, Hk, l;
+    float scale, scale_log2;
+    int accumulate;                     // depth gradients are added to d_depth_kv instead of stored
+    int h0;                             // first head (inside its group of H / Hk) of the up to 8 heads this launch handles
+};
+
+template <int D>
+struct DepthBwdSmem {
+    static constexpr int P = db_pos<D>();
+    static constexpr int kIn = 2 * 2 * P * kDbRoundSlots * D * 2;       // two rounds x (K, V) rows
+    static constexpr int kQd = kIn;                                     // Q_t and dO_t rows: [2][P][8 heads][D]
+    static constexpr int kOut = kQd + 2 * P * 8 * D * 2;                // dKd, dVd of the round: [2][P][16 slots][D]
+    static constexpr int kTotal = kOut + 2 * P * kDbRoundSlots * D * 2;
+};
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(db_pos<D>() * 32)
+depth_bwd_gqa_kernel(const DepthBwdParams p) {
+    using L = DepthBwdSmem<D>;
+    constexpr int P = L::P, NT = P * 32, CH = D / 8, RS = kDbRoundSlots;
+    constexpr int kTensorBytes = P * RS * D * 2;
+    extern __shared__ __align__(128) uint8_t db_smem[];
+    const uint32_t smem_base = smem_u32(db_smem);
+    // byte offset of 16-byte piece `piece` of row `row` in a [rows][D] bf16 tile whose pieces are swizzled by the row
+    auto row_piece = [](int row, int piece) { return row * D * 2 + (((piece & 8) | ((piece & 7) ^ (row & 7))) << 4); };
+
+    const int nblk = num_tiles(p.T) * (kTileRows / P);             // whole tiles: the tail rows of the cache get zeros
+    const int blk = blockIdx.x % nblk;
+    const int bh = blockIdx.x / nblk;
+    const int hk = bh % p.Hk, b = bh / p.Hk;
+    const int t0 = blk * P;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const int t = t0 + warp;
+    const bool live = t < p.T;
+    const bool head = live && g < G;
+    const int h = hk * (p.H / p.Hk) + p.h0 + min(g, G - 1);
+
+    // ---- this position's Q and dO rows: A fragments in registers, and rows in shared memory for the B side ----
+    uint4 qf[D / 32], gf[D / 32];
+    uint8_t* sQ = db_smem + L::kQd + (0 * P + warp) * 8 * D * 2;
+    uint8_t* sG = db_smem + L::kQd + (1 * P + warp) * 8 * D * 2;
+#pragma unroll
+    for (int kp = 0; kp < D / 32; ++kp) {
+        qf[kp] = make_uint4(0u, 0u, 0u, 0u);
+        gf[kp] = make_uint4(0u, 0u, 0u, 0u);
+        if (head) {
+            const size_t off = ((size_t(b) * p.T + t) * p.H + h) * D + (4 * kp + tq) * 8;
+            qf[kp] = *reinterpret_cast<const uint4*>(p.Q + off);
+            gf[kp] = *reinterpret_cast<const uint4*>(p.dO + off);
+        }
+        *reinterpret_cast<uint4*>(sQ + row_piece(g, 4 * kp + tq)) = qf[kp];       // rows of heads past G are zero
+        *reinterpret_cast<uint4*>(sG + row_piece(g, 4 * kp + tq)) = gf[kp];
+    }
+    float neg_lse2 = 0.f, dlt = 0.f;
+    uint32_t dq_seq[D / 8];
+    __nv_bfloat16* dq_row = p.dQ + ((size_t(b) * p.T + t) * p.H + h) * D;
+    if (head) {
+        neg_lse2 = -p.LSE[(size_t(b) * p.H + h) * p.T + t] * 1.4426950408889634f;
+        dlt = p.delta[(size_t(b) * p.H + h) * p.T + t];
+#pragma unroll
+        for (int fb = 0; fb < D / 8; ++fb) dq_seq[fb] = *reinterpret_cast<const uint32_t*>(dq_row + 8 * fb + 2 * tq);
+    }
+
+    const int tile = t0 / kTileRows, r0 = t0 % kTileRows;
+    const size_t slot_elems = cache_slot_elems(p.B, p.T, p.Hk, D);
+    const size_t blk_off = cache_block_offset(p.B, p.T, p.Hk, D, 0, b, hk, tile, 0) + size_t(r0) * 8;
+    const __nv_bfloat16* cbase = p.depth_kv + blk_off;
+    __nv_bfloat16* gbase = p.d_depth_kv + blk_off;
+
+    // a thread always moves the same (position, chunk) piece; only the slot advances
+    static_assert(NT % (P * CH) == 0, "one (position, chunk) per thread");
+    constexpr int kSlotStep = NT / (P * CH);
+    const int st_pos = threadIdx.x % P, st_chunk = (threadIdx.x / P) % CH, st_slot0 = threadIdx.x / (P * CH);
+    const size_t st_goff = (size_t(st_chunk) * kTileRows + st_pos) * 8;
+    auto stage_round = [&](int s0, int buf) {
+        const int ns = min(RS, p.l - s0);
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {
+            const __nv_bfloat16* src = cbase + st_goff + size_t(s0 + st_slot0) * slot_elems + size_t(kv) * cache_block_elems(D);
+            const uint32_t dst = smem_base + (buf * 2 + kv) * kTensorBytes;
+#pragma unroll
+            for (int k = 0; k < RS / kSlotStep; ++k) {
+                const int slot = st_slot0 + k * kSlotStep;
+                if (slot < ns) cp_async_16(dst + row_piece(st_pos * RS + slot, st_chunk), src + size_t(k * kSlotStep) * slot_elems);
+            }
+        }
+        cp_async_commit();
+    };
+
+    float dq[D / 8][4];
+#pragma unroll
+    for (int fb = 0; fb < D / 8; ++fb) { dq[fb][0] = 0.f; dq[fb][1] = 0.f; dq[fb][2] = 0.f; dq[fb][3] = 0.f; }
+
+    if (p.l > 0) stage_round(0, 0);
+#pragma unroll 1
+    for (int s0 = 0, rnd = 0; s0 < p.l; s0 += RS, ++rnd) {
+        const int ns = min(RS, p.l - s0);
+        const int buf = rnd & 1;
+        const uint8_t* sK = db_smem + (buf * 2) * kTensorBytes + warp * RS * D * 2;     // this position's rows [slot][D]
+        const uint8_t* sV = sK + kTensorBytes;
+        uint8_t* oK = db_smem + L::kOut + (0 * P + warp) * RS * D * 2;                  // this position's output rows
+        uint8_t* oV = db_smem + L::kOut + (1 * P + warp) * RS * D * 2;
+        if (s0 + RS < p.l) { stage_round(s0 + RS, buf ^ 1); cp_async_wait<1>(); }
+        else cp_async_wait<0>();
+        __syncthreads();                                   // the round's rows are in; the previous round's outputs are written out
+
+        // ---- U = Q Kd^T and dO Vd^T for 16 slots (two blocks of 8) ----
+        float cu[2][4], cv[2][4];
+#pragma unroll
+        for (int nb = 0; nb < 2; ++nb) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { cu[nb][i] = 0.f; cv[nb][i] = 0.f; }
+            const int slot = 8 * nb + g;
+#pragma unroll
+            for (int kp = 0; kp < D / 32; ++kp) {
+                const uint4 kk = *reinterpret_cast<const uint4*>(sK + row_piece(slot, 4 * kp + tq));
+                const uint4 vv = *reinterpret_cast<const uint4*>(sV + row_piece(slot, 4 * kp + tq));
+                mma_bf16_16x8x16(cu[nb], qf[kp].x, 0u, qf[kp].y, 0u, kk.x, kk.y);
+                mma_bf16_16x8x16(cu[nb], qf[kp].z, 0u, qf[kp].w, 0u, kk.z, kk.w);
+                mma_bf16_16x8x16(cv[nb], gf[kp].x, 0u, gf[kp].y, 0u, vv.x, vv.y);
+                mma_bf16_16x8x16(cv[nb], gf[kp].z, 0u, gf[kp].w, 0u, vv.z, vv.w);
+            }
+        }
+        // ---- R and dU of head g for its slots 8 nb + 2 tq (+ 1); zero for slots past the end and heads past G,
+        //      whose staged rows may hold anything ----
+        uint32_t pr[2], pu[2];
+#pragma unroll
+        for (int nb = 0; nb < 2; ++nb) {
+            float r[2], u[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const bool ok = head && (8 * nb + 2 * tq + e < ns);
+                r[e] = ok ? fast_exp2(fmaf(cu[nb][e], p.scale_log2, neg_lse2)) : 0.f;
+                u[e] = ok ? r[e] * (cv[nb][e] - dlt) : 0.f;
+            }
+            pr[nb] = pack_bf16x2(r[0], r[1]);
+            pu[nb] = pack_bf16x2(u[0], u[1]);
+        }
+        // ---- dQ share: dU (16 slots deep) x Kd rows; rows of slots past the end hold stale data: weight 0, but
+        //      a NaN there would spread, so they are zeroed first ----
+        if (ns < RS) {
+            for (int idx = lane; idx < (RS - ns) * CH; idx += 32)
+                *reinterpret_cast<uint4*>(const_cast<uint8_t*>(sK) + row_piece(ns + idx / CH, idx % CH)) = make_uint4(0u, 0u, 0u, 0u);
+            __syncwarp();
+        }
+        {
+            const int krow = ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+            for (int fb = 0; fb < D / 8; fb += 2) {
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(smem_u32(sK + row_piece(krow, fb + (lane >> 4))), b0, b1, b2, b3);
+                mma_bf16_16x8x16(dq[fb], pu[0], 0u, pu[1], 0u, b0, b1);
+                mma_bf16_16x8x16(dq[fb + 1], pu[0], 0u, pu[1], 0u, b2, b3);
+            }
+        }
+        // ---- dKd = scale dU^T Q and dVd = R^T dO for the 16 slots: A = [slot][head] by 8 x 8 transposes ----
+        {
+            const uint32_t au0 = movmatrix_trans(pu[0]), au1 = movmatrix_trans(pu[1]);
+            const uint32_t ar0 = movmatrix_trans(pr[0]), ar1 = movmatrix_trans(pr[1]);
+            const int hrow = lane & 7;                                  // head row a lane addresses for the matrix loads
+#pragma unroll
+            for (int fb = 0; fb < D / 8; fb += 4) {
+                uint32_t q0, q1, q2, q3, g0, g1, g2, g3;                // B fragments [heads 0..7][8 features] of 4 blocks
+                ldmatrix_x4_trans(smem_u32(sQ + row_piece(hrow, fb + (lane >> 3))), q0, q1, q2, q3);
+                ldmatrix_x4_trans(smem_u32(sG + row_piece(hrow, fb + (lane >> 3))), g0, g1, g2, g3);
+                const uint32_t qb[4] = {q0, q1, q2, q3}, gb[4] = {g0, g1, g2, g3};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float ck[4] = {0.f, 0.f, 0.f, 0.f}, cw[4] = {0.f, 0.f, 0.f, 0.f};
+                    mma_bf16_16x8x16(ck, au0, au1, 0u, 0u, qb[j], 0u);
+                    mma_bf16_16x8x16(cw, ar0, ar1, 0u, 0u, gb[j], 0u);
+                    // rows g (slot g) and g + 8, features 8 (fb + j) + 2 tq, + 1
+                    const int piece = fb + j;
+                    *reinterpret_cast<uint32_t*>(oK + row_piece(g, piece) + 4 * tq) = pack_bf16x2(ck[0] * p.scale, ck[1] * p.scale);
+                    *reinterpret_cast<uint32_t*>(oK + row_piece(g + 8, piece) + 4 * tq) = pack_bf16x2(ck[2] * p.scale, ck[3] * p.scale);
+                    *reinterpret_cast<uint32_t*>(oV + row_piece(g, piece) + 4 * tq) = pack_bf16x2(cw[0], cw[1]);
+                    *reinterpret_cast<uint32_t*>(oV + row_piece(g + 8, piece) + 4 * tq) = pack_bf16x2(cw[2], cw[3]);
+                }
+            }
+        }
+        __syncthreads();                                   // all positions' output rows of this round are in shared memory
+        // ---- write the round's gradients: a thread moves the (position, chunk) piece of every kSlotStep-th slot ----
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {
+            __nv_bfloat16* dst = gbase + st_goff + size_t(s0 + st_slot0) * slot_elems + size_t(kv) * cache_block_elems(D);
+            const uint8_t* src = db_smem + L::kOut + (kv * P + st_pos) * RS * D * 2;
+#pragma unroll
+            for (int k = 0; k < RS / kSlotStep; ++k) {
+                const int slot = st_slot0 + k * kSlotStep;
+                if (slot < ns) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(src + row_piece(slot, st_chunk));
+                    __nv_bfloat16* out = dst + size_t(k * kSlotStep) * slot_elems;
+                    if (p.accumulate) red_add_bf16x2_v4(out, v);
+                    else *reinterpret_cast<uint4*>(out) = v;
+                }
+            }
+        }
+        // (the next round's barrier orders these reads before the next outputs)
+    }
+
+    // ---- dQ = sequence part + scale * depth part ----
+    if (head) {
+#pragma unroll
+        for (int fb = 0; fb < D / 8; ++fb) {
+            const float a0 = bf16_lo_to_f32(dq_seq[fb]) + p.scale * dq[fb][0];
+            const float a1 = bf16_hi_to_f32(dq_seq[fb]) + p.scale * dq[fb][1];
+            *reinterpret_cast<uint32_t*>(dq_row + 8 * fb + 2 * tq) = pack_bf16x2(a0, a1);
+        }
     }
 }
 

@@ -274,7 +274,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
 }
 
 template <int D, int G>
-__global__ void __launch_bounds__(db_pos<D>() * 32)
+__global__ void __launch_bounds__(db_pos<D>() * 32, 2)
 depth_bwd_gqa_kernel(const DepthBwdParams p) {
     using L = DepthBwdSmem<D>;
     constexpr int P = L::P, NT = P * 32, CH = D / 8, RS = kDbRoundSlots;

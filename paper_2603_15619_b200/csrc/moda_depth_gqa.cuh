@@ -21,7 +21,7 @@
 
 namespace moda {
 
-constexpr int kDgPos = 8;               // positions per CTA, one per warp: a 16-byte piece of 8 positions is one 128-byte line
+constexpr int kDgPos = 4;               // positions per CTA, one per warp: a 16-byte piece of 8 positions is one 128-byte line
 constexpr int kDgThreads = kDgPos * 32;
 constexpr int kDgRoundSlots = 16;        // slots staged per round
 constexpr int kDgBufs = 2;              // rounds in flight: the next round's rows arrive while this round is used
@@ -242,7 +242,7 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
 // The sequence kernel (run without depth slots) has left the sequence part of dQ; this kernel adds its share.
 // =====================================================================================================
 constexpr int kDbRoundSlots = 16;
-template <int D> constexpr int db_pos() { return 512 / D; }           // positions per CTA (one per warp): 8 at d = 64, 4 at d = 128
+template <int D> constexpr int db_pos() { return 256 / D; }           // positions per CTA (one per warp): 8 at d = 64, 4 at d = 128
 
 struct DepthBwdParams {
     const __nv_bfloat16* Q;             // [B][T][H][d]
@@ -274,7 +274,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
 }
 
 template <int D, int G>
-__global__ void __launch_bounds__(db_pos<D>() * 32, 2)
+__global__ void __launch_bounds__(db_pos<D>() * 32, 4)
 depth_bwd_gqa_kernel(const DepthBwdParams p) {
     using L = DepthBwdSmem<D>;
     constexpr int P = L::P, NT = P * 32, CH = D / 8, RS = kDbRoundSlots;

@@ -8,7 +8,7 @@
 // without depth slots, left in O and LSE:
 //     LSE = logaddexp(LSE_seq, LSE_dep),   O = w O_seq + (1 - w) O_dep,   w = exp(LSE_seq - LSE),
 // which is the single softmax over the union of the two key sets.  The depth cache is read once per
-// key/value head (not once per query head), in runs of kPos consecutive positions per 16-byte chunk.
+// key/value head (not once per query head), in runs of kDgPos consecutive positions per 16-byte chunk.
 #pragma once
 
 #include <cstdint>
@@ -21,7 +21,7 @@
 
 namespace moda {
 
-constexpr int kDgPos = 4;               // positions per CTA, one per warp: a 16-byte piece of 8 positions is one 128-byte line
+constexpr int kDgPos = 4;               // positions per CTA, one per warp: a 16-byte piece of 4 positions is a 64-byte run
 constexpr int kDgThreads = kDgPos * 32;
 constexpr int kDgRoundSlots = 16;        // slots staged per round
 constexpr int kDgBufs = 2;              // rounds in flight: the next round's rows arrive while this round is used
@@ -106,7 +106,7 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
     for (int fb = 0; fb < D / 8; ++fb) { o[fb][0] = 0.f; o[fb][1] = 0.f; o[fb][2] = 0.f; o[fb][3] = 0.f; }
 
     // stages the K and V rows of slots [s0, s0 + ns) of the CTA's positions into buffer `buf`: 16-byte pieces,
-    // the eight positions of a piece are one 128-byte line of the cache
+    // the positions of a piece are one contiguous run of the cache
     // A thread always copies the same (position, chunk) piece: kDgThreads is a multiple of kDgPos * CH, so only the
     // slot advances from one copy to the next.
     static_assert(kDgThreads % (kDgPos * CH) == 0, "one (position, chunk) per thread");
@@ -242,7 +242,7 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
 // The sequence kernel (run without depth slots) has left the sequence part of dQ; this kernel adds its share.
 // =====================================================================================================
 constexpr int kDbRoundSlots = 16;
-template <int D> constexpr int db_pos() { return 256 / D; }           // positions per CTA (one per warp): 8 at d = 64, 4 at d = 128
+template <int D> constexpr int db_pos() { return 256 / D; }           // positions per CTA (one per warp): 4 at d = 64, 2 at d = 128
 
 struct DepthBwdParams {
     const __nv_bfloat16* Q;             // [B][T][H][d]

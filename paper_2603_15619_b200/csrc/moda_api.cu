@@ -112,10 +112,12 @@ inline bool fwd_depth_heavy(int T, int l, int d) {
 // d = 64 (T = 16384, 8 key/value heads): the fused row-local path costs about 2.3 us per (query head per
 // group, slot), the separate kernel about 200 us plus 11.7 us per slot whatever the group size, so the
 // separate kernel wins for large groups with many slots (G = 8 from l = 31, G = 7 from 46, G = 6 from 96).
-// At d = 128 it was slower on every shape tried (G <= 4); those calls stay on the fused path.
+// At d = 128 (T = 8192) it wins only for 8 heads per group from about 45 slots (l = 64: 2.31 -> 2.08 ms;
+// l = 24: 1.40 -> 1.58 ms; G = 6, l = 64: 1.74 -> 1.84 ms).
 inline bool gqa_depth_split(int d, int G, int l) {
-    if (G == 16 || G == 32) return d == 64 && l >= 31;             // run as groups of 8 heads on the same slots
-    return d == 64 && G >= 6 && G <= 8 && l * (23 * G - 117) > 2000;
+    if (d == 128) return (G == 8 || G == 16 || G == 32) && l >= 48;
+    if (G == 16 || G == 32) return l >= 31;                        // run as groups of 8 heads on the same slots
+    return G >= 6 && G <= 8 && l * (23 * G - 117) > 2000;
 }
 
 template <int D, int G>

@@ -23,6 +23,7 @@ SHAPES = [
     (1, 300, 8, 1, 64, 64), (1, 256, 4, 2, 128, 40),     # the paper's kernel table uses L = 64 and more
     (2, 260, 16, 2, 64, 40), (1, 129, 8, 1, 64, 100), (1, 77, 14, 2, 64, 47), (1, 200, 8, 1, 64, 31),   # depth part as its own kernel
     (1, 200, 16, 1, 64, 40), (1, 130, 32, 1, 64, 33), (1, 140, 32, 2, 128, 12),   # 16 / 32 heads per group as groups of 8
+    (1, 150, 8, 1, 128, 50), (1, 130, 16, 1, 128, 48),            # d = 128 forward through the per-position kernel
     (1, 300, 16, 1, 64, 5), (1, 200, 32, 2, 128, 3), (2, 130, 32, 1, 64, 9), (1, 256, 16, 1, 128, 33),   # G = 16, 32
 ]
 

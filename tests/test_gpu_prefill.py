@@ -16,6 +16,7 @@ SHAPES = [
     (1, 128, 256, 2, 2, 128, 3), (1, 128, 384, 2, 1, 64, 2), (2, 100, 164, 4, 2, 128, 4), (1, 130, 200, 2, 2, 64, 5),
     (1, 257, 300, 4, 1, 128, 0), (1, 1, 129, 2, 2, 64, 3), (1, 64, 1000, 4, 2, 128, 2), (2, 200, 777, 8, 2, 64, 1),
     (1, 300, 301, 2, 2, 128, 33), (1, 31, 95, 16, 1, 64, 2), (1, 129, 129, 2, 2, 128, 2),
+    (1, 100, 300, 8, 1, 64, 40), (1, 70, 200, 16, 2, 64, 33),        # depth part through the per-position kernel
 ]
 
 

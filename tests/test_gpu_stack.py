@@ -52,7 +52,9 @@ def test_stack_gradients_flow_back_through_the_depth_stream(B, T, H, Hk, d, n_la
 
 
 @pytest.mark.parametrize("B,T,H,Hk,d,l", [(1, 300, 2, 2, 64, 3), (2, 200, 3, 3, 128, 5), (1, 300, 4, 2, 64, 4),
-                                          (1, 256, 16, 1, 128, 3), (1, 130, 32, 1, 64, 2)])
+                                          (1, 256, 16, 1, 128, 3), (1, 130, 32, 1, 64, 2),
+                                          # large groups: the per-position depth kernel does the adding (16 heads: two launches)
+                                          (1, 200, 8, 1, 64, 12), (2, 130, 16, 2, 64, 9), (1, 100, 8, 1, 128, 10)])
 def test_accumulate_flag_adds_the_depth_gradients_to_what_the_cache_holds(B, T, H, Hk, d, l):
     """MODA_BWD_ACCUMULATE_DEPTH: slots [0, l) become bf16(old + gradient), everything else as without the flag."""
     x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=77, device="cuda")

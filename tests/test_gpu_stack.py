@@ -54,7 +54,7 @@ def test_stack_gradients_flow_back_through_the_depth_stream(B, T, H, Hk, d, n_la
 @pytest.mark.parametrize("B,T,H,Hk,d,l", [(1, 300, 2, 2, 64, 3), (2, 200, 3, 3, 128, 5), (1, 300, 4, 2, 64, 4),
                                           (1, 256, 16, 1, 128, 3), (1, 130, 32, 1, 64, 2),
                                           # large groups: the per-position depth kernel does the adding (16 heads: two launches)
-                                          (1, 200, 8, 1, 64, 12), (2, 130, 16, 2, 64, 9), (1, 100, 8, 1, 128, 10)])
+                                          (1, 200, 8, 1, 64, 12), (2, 130, 16, 1, 64, 9), (1, 100, 8, 1, 128, 10)])
 def test_accumulate_flag_adds_the_depth_gradients_to_what_the_cache_holds(B, T, H, Hk, d, l):
     """MODA_BWD_ACCUMULATE_DEPTH: slots [0, l) become bf16(old + gradient), everything else as without the flag."""
     x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=77, device="cuda")
@@ -74,9 +74,15 @@ def test_accumulate_flag_adds_the_depth_gradients_to_what_the_cache_holds(B, T, 
         assert torch.equal(a, b)
     want = (old.double() + plain[3].double())
     got = acc.double()
-    ulp = torch.maximum(want.abs(), torch.tensor(1e-30, device="cuda", dtype=torch.float64)) * 2.0 ** -8
-    assert bool(((got - want).abs() <= ulp).all())                       # one bf16 rounding of the exact sum
-    assert float((got != want.to(torch.bfloat16).double()).double().mean()) < 1e-3   # and round-to-nearest almost everywhere
+    if H // Hk <= 8:
+        ulp = torch.maximum(want.abs(), torch.tensor(1e-30, device="cuda", dtype=torch.float64)) * 2.0 ** -8
+        assert bool(((got - want).abs() <= ulp).all())                       # one bf16 rounding of the exact sum
+        assert float((got != want.to(torch.bfloat16).double()).double().mean()) < 1e-3   # and round-to-nearest almost everywhere
+    else:
+        # 16 / 32 heads per group: the groups of 8 add their shares one after the other (a rounding each),
+        # while the plain call rounds the sum of the shares once
+        # (the shares of the groups may be larger than their sum, so the bound is on the whole tensor)
+        assert rel_l2(got.cpu().numpy(), want.cpu().numpy()) < 5e-3
     # twice more: the cache keeps collecting
     moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale, d_depth_kv=acc,
                            stages=moda.MODA_BWD_ALL_STAGES | moda.MODA_BWD_ACCUMULATE_DEPTH)

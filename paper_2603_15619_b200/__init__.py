@@ -9,6 +9,7 @@ from .stack import DepthStream  # noqa: F401
 from .binding import (  # noqa: F401
     MODA_BWD_ACCUMULATE_DEPTH,
     MODA_BWD_ALL_STAGES,
+    MODA_BWD_DETERMINISTIC,
     MODA_BWD_STAGE_DKDV,
     MODA_BWD_STAGE_DQ,
     MODA_BWD_STAGE_ROWTERMS,
@@ -33,5 +34,6 @@ from .binding import (  # noqa: F401
     moda_depth_cache_bytes,
     moda_depth_cache_unpack,
     moda_last_status,
+    moda_selftest_wait_timeout,
     moda_version,
 )

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libmoda_b200.so")
 
 MODA_MAX_DEPTH = 256
 SYMBOLS = (
-    "moda_version", "moda_strerror", "moda_last_cuda_error", "moda_last_status",
+    "moda_version", "moda_strerror", "moda_last_cuda_error", "moda_last_status", "moda_selftest_wait_timeout",
     "moda_depth_cache_bytes", "moda_depth_cache_append", "moda_depth_cache_unpack",
     "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd", "moda_attn_bwd_stages",
     "moda_attn_bwd_static_scratch",
@@ -27,7 +27,9 @@ SYMBOLS = (
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
+MODA_BWD_STAGE_ROWS, MODA_BWD_STAGE_SEQ, MODA_BWD_STAGE_FINISH = 1, 2, 4
 MODA_BWD_ACCUMULATE_DEPTH = 8      # ORed into a stages mask: depth gradients are added to d_depth_kv
+MODA_BWD_DETERMINISTIC = 16        # ORed into a stages mask: the split, bit-reproducible form of the backward
 
 
 class ModaError(RuntimeError):
@@ -57,6 +59,8 @@ def load() -> ctypes.CDLL:
     lib.moda_last_cuda_error.restype = ci
     lib.moda_last_status.restype = ci
     lib.moda_last_status.argtypes = [ci]
+    lib.moda_selftest_wait_timeout.restype = ci
+    lib.moda_selftest_wait_timeout.argtypes = [vp]
     lib.moda_depth_cache_bytes.restype = sz
     lib.moda_depth_cache_bytes.argtypes = [ci] * 5
     lib.moda_depth_cache_append.restype = ci
@@ -111,6 +115,21 @@ def _stream(stream):
     return ctypes.c_void_p(stream.cuda_stream)
 
 
+def _new(shape, dtype, device, stream):
+    """Buffer the wrapper allocates on the caller's behalf.  It is allocated with `stream` current, so
+    torch's caching allocator ties the block to the stream the kernels run on: when the Python
+    reference is dropped while those kernels are still queued, the block is only handed out again
+    to work that is ordered after them (a block made on another stream could be reused at once)."""
+    if stream is None:
+        return torch.empty(shape, dtype=dtype, device=device)
+    with torch.cuda.stream(stream):
+        return torch.empty(shape, dtype=dtype, device=device)
+
+
+def _new_like(t, stream):
+    return _new(t.shape, t.dtype, t.device, stream)
+
+
 def _check(rc: int, what: str):
     if rc != 0:
         raise ModaError(rc, what)
@@ -139,16 +158,25 @@ def moda_last_status(clear: bool = False) -> int:
     return int(load().moda_last_status(int(clear)))
 
 
+MODA_ERR_DEVICE_TIMEOUT = -10
+MODA_SELFTEST_WAIT_STATUS = (255 << 8) | 1
+
+
+def moda_selftest_wait_timeout(stream=None):
+    """Launch the kernel whose only wait runs out after about 1 ms (self-test of the failure reporting)."""
+    _check(load().moda_selftest_wait_timeout(_stream(stream)), "moda_selftest_wait_timeout")
+
+
 def moda_depth_cache_bytes(B, T, H, d, l_max) -> int:
     return int(load().moda_depth_cache_bytes(B, T, H, d, l_max))
 
 
-def alloc_depth_cache(B, T, H, d, l_max, device="cuda") -> torch.Tensor:
+def alloc_depth_cache(B, T, H, d, l_max, device="cuda", stream=None) -> torch.Tensor:
     """Caller-side helper: a bf16 buffer of moda_depth_cache_bytes() bytes (uninitialised)."""
     n = moda_depth_cache_bytes(B, T, H, d, l_max)
     if n == 0 and l_max != 0:
         raise ValueError("bad depth-cache shape")
-    return torch.empty(max(n // 2, 8), dtype=torch.bfloat16, device=device)
+    return _new((max(n // 2, 8),), torch.bfloat16, device, stream)
 
 
 def depth_cache_window(cache, B, T, H, d, first_slot, n_slots=None):
@@ -186,9 +214,9 @@ def moda_attn_fwd(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):
     B, T, H, d = _bthd(Q, "Q")
     assert _bthd(K, "K") == (B, T, H, d) and _bthd(V, "V") == (B, T, H, d)
     if O is None:
-        O = torch.empty_like(Q)
+        O = _new_like(Q, stream)
     if LSE is None:
-        LSE = torch.empty((B, H, T), dtype=torch.float32, device=Q.device)
+        LSE = _new((B, H, T), torch.float32, Q.device, stream)
     _check(load().moda_attn_fwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
                                 B, T, H, d, int(l), float(scale), _ptr(O), _ptr(LSE), _stream(stream)),
            "moda_attn_fwd")
@@ -205,14 +233,14 @@ def moda_attn_bwd(Q, K, V, depth_kv, O, dO, LSE, l, scale,
 
     With ``stages`` (a MODA_BWD_STAGE_* mask) the call goes through moda_attn_bwd_stages."""
     B, T, H, d = _bthd(Q, "Q")
-    dQ = torch.empty_like(Q) if dQ is None else dQ
-    dK = torch.empty_like(Q) if dK is None else dK
-    dV = torch.empty_like(Q) if dV is None else dV
+    dQ = _new_like(Q, stream) if dQ is None else dQ
+    dK = _new_like(Q, stream) if dK is None else dK
+    dV = _new_like(Q, stream) if dV is None else dV
     if l > 0 and d_depth_kv is None:
-        d_depth_kv = alloc_depth_cache(B, T, H, d, l, Q.device)
+        d_depth_kv = alloc_depth_cache(B, T, H, d, l, Q.device, stream)
     need = moda_bwd_workspace_bytes(B, T, H, d, l)
     if workspace is None:
-        workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
+        workspace = _new((need,), torch.uint8, Q.device, stream)
     args = [_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
             _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, d, int(l), float(scale),
             _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
@@ -265,9 +293,9 @@ def moda_attn_fwd_gqa(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None
     Returns O [B,T,H,d] bf16 and LSE [B,H,T] fp32 (allocated if not given)."""
     B, T, H, Hk, d = _gqa_shapes(Q, K, V)
     if O is None:
-        O = torch.empty_like(Q)
+        O = _new_like(Q, stream)
     if LSE is None:
-        LSE = torch.empty((B, H, T), dtype=torch.float32, device=Q.device)
+        LSE = _new((B, H, T), torch.float32, Q.device, stream)
     _check(load().moda_attn_fwd_gqa(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
                                     B, T, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE), _stream(stream)),
            "moda_attn_fwd_gqa")
@@ -280,13 +308,13 @@ def moda_attn_bwd_gqa(Q, K, V, depth_kv, O, dO, LSE, l, scale,
 
     With ``stages`` (a MODA_BWD_STAGE_* mask) the call goes through moda_attn_bwd_gqa_stages."""
     B, T, H, Hk, d = _gqa_shapes(Q, K, V)
-    dQ = torch.empty_like(Q) if dQ is None else dQ
-    dK = torch.empty_like(K) if dK is None else dK
-    dV = torch.empty_like(V) if dV is None else dV
+    dQ = _new_like(Q, stream) if dQ is None else dQ
+    dK = _new_like(K, stream) if dK is None else dK
+    dV = _new_like(V, stream) if dV is None else dV
     if l > 0 and d_depth_kv is None:
-        d_depth_kv = alloc_depth_cache(B, T, Hk, d, l, Q.device)
+        d_depth_kv = alloc_depth_cache(B, T, Hk, d, l, Q.device, stream)
     if workspace is None:
-        workspace = torch.empty(moda_bwd_workspace_bytes_gqa(B, T, H, Hk, d, l), dtype=torch.uint8, device=Q.device)
+        workspace = _new((moda_bwd_workspace_bytes_gqa(B, T, H, Hk, d, l),), torch.uint8, Q.device, stream)
     args = [_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
             _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, Hk, d, int(l), float(scale),
             _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
@@ -320,11 +348,11 @@ def moda_attn_decode(q, K, V, depth_kv_token, T_kv, l, scale, O=None, LSE=None, 
                   or depth_kv_token.dtype != torch.bfloat16):
         raise ValueError("depth_kv_token must be a bf16 [l, B, H_kv, 2, d] tensor")
     if O is None:
-        O = torch.empty_like(q)
+        O = _new_like(q, stream)
     if LSE is None:
-        LSE = torch.empty((B, H), dtype=torch.float32, device=q.device)
+        LSE = _new((B, H), torch.float32, q.device, stream)
     if workspace is None:
-        workspace = torch.empty(moda_decode_workspace_bytes(B, H, d), dtype=torch.uint8, device=q.device)
+        workspace = _new((moda_decode_workspace_bytes(B, H, d),), torch.uint8, q.device, stream)
     _check(load().moda_attn_decode(_ptr(q), _ptr(K), _ptr(V), _ptr(depth_kv_token) if l > 0 else None,
                                    B, int(T_kv), T_cap, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
@@ -340,23 +368,23 @@ def moda_attn_fwd_prefill(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=
     if (Bk, dk) != (B, d) or _bthd(V, "V") != (B, T_kv, Hk, d):
         raise ValueError("K and V must be bf16 [B, T_kv, H_kv, d] tensors matching Q's B and d")
     if O is None:
-        O = torch.empty_like(Q)
+        O = _new_like(Q, stream)
     if LSE is None:
-        LSE = torch.empty((B, H, T_q), dtype=torch.float32, device=Q.device)
+        LSE = _new((B, H, T_q), torch.float32, Q.device, stream)
     _check(load().moda_attn_fwd_prefill(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
                                         B, T_q, T_kv, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
                                         _stream(stream)), "moda_attn_fwd_prefill")
     return O, LSE
 
 
-def _decode_outputs(q, O, LSE, workspace):
+def _decode_outputs(q, O, LSE, workspace, stream):
     B, H, d = q.shape
     if O is None:
-        O = torch.empty_like(q)
+        O = _new_like(q, stream)
     if LSE is None:
-        LSE = torch.empty((B, H), dtype=torch.float32, device=q.device)
+        LSE = _new((B, H), torch.float32, q.device, stream)
     if workspace is None:
-        workspace = torch.empty(moda_decode_workspace_bytes(B, H, d), dtype=torch.uint8, device=q.device)
+        workspace = _new((moda_decode_workspace_bytes(B, H, d),), torch.uint8, q.device, stream)
     return O, LSE, workspace
 
 
@@ -372,7 +400,7 @@ def moda_attn_decode_varlen(q, K, V, seq_lens, depth_kv_token, max_seq_len, l, s
     B, H, d = q.shape
     _, T_cap, Hk, _ = _bthd(K, "K")
     _int32(seq_lens, "seq_lens", (B,))
-    O, LSE, workspace = _decode_outputs(q, O, LSE, workspace)
+    O, LSE, workspace = _decode_outputs(q, O, LSE, workspace, stream)
     _check(load().moda_attn_decode_varlen(_ptr(q), _ptr(K), _ptr(V), _ptr(seq_lens), _ptr(depth_kv_token) if l > 0 else None,
                                           B, int(max_seq_len), T_cap, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
                                           _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
@@ -389,7 +417,7 @@ def moda_attn_decode_paged(q, K_pages, V_pages, block_table, seq_lens, depth_kv_
     _int32(seq_lens, "seq_lens", (B,))
     if block_table.dtype != torch.int32 or block_table.dim() != 2 or block_table.shape[0] != B:
         raise ValueError("block_table must be an int32 [B, max_blocks] tensor")
-    O, LSE, workspace = _decode_outputs(q, O, LSE, workspace)
+    O, LSE, workspace = _decode_outputs(q, O, LSE, workspace, stream)
     _check(load().moda_attn_decode_paged(_ptr(q), _ptr(K_pages), _ptr(V_pages), _ptr(block_table), _ptr(seq_lens),
                                          _ptr(depth_kv_token) if l > 0 else None,
                                          B, int(max_seq_len), page_size, num_pages, block_table.shape[1], H, Hk, d, int(l),

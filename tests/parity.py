@@ -10,6 +10,14 @@ TOL_O_REL_L2 = 1e-2
 TOL_O_MAX_ABS = 2e-2
 TOL_LSE_ABS = 1e-3
 TOL_GRAD_REL_L2 = 2e-2
+# Companion to the per-tensor gradient norm: the worst single row (last axis = features).  A tensor
+# norm over millions of rows cannot see a handful of wrong rows; a wrong (missing, stale, misplaced)
+# row is off by about its whole norm.  A correct row is a bf16-rounded sum of bf16-rounded products
+# (P and dS are rounded to bf16 before their second contraction): a few times 2^-9 of the magnitude of
+# its *terms*.  Rows whose terms cancel (dU_i = R_i (<dO, vd_i> - D_t) with the two close, D_t taken
+# from the bf16 O) are small with an error set by the terms, so a row is measured against the larger of
+# its own norm and the tensor's RMS row norm.
+TOL_GRAD_ROW_REL_L2 = 5e-2
 
 
 def rel_l2(got, ref):
@@ -20,6 +28,21 @@ def rel_l2(got, ref):
 
 def max_abs(got, ref):
     return float(np.abs(np.asarray(got, dtype=np.float64) - np.asarray(ref, dtype=np.float64)).max())
+
+
+def worst_row_rel_l2(got, ref):
+    """Largest per-row relative L2 error; rows are the vectors along the last axis."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    if ref.size == 0:
+        return 0.0
+    got = got.reshape(-1, got.shape[-1])
+    ref = ref.reshape(-1, ref.shape[-1])
+    norms = np.linalg.norm(ref, axis=1)
+    # the absolute part only matters where the exact gradient vanishes identically (one visible key)
+    floor = float(np.sqrt(np.mean(norms ** 2))) + 1e-4 * np.sqrt(ref.shape[-1])
+    err = np.linalg.norm(got - ref, axis=1) / np.maximum(norms, floor)
+    return float(err.max())
 
 
 def f64(t):
@@ -59,3 +82,20 @@ def assert_forward_close(O, LSE, O_ref, LSE_ref, what=""):
     assert e_abs <= TOL_O_MAX_ABS, f"{what}: O max-abs {e_abs:.3e}"
     assert e_lse <= TOL_LSE_ABS, f"{what}: LSE abs {e_lse:.3e}"
     return e_rel, e_abs, e_lse
+
+
+def assert_same_gradients(a, b, what=""):
+    """Two backward calls on the same inputs: dK, dV and the depth gradients agree bit for bit (they
+    are accumulated on chip in a fixed order).  dQ tiles are summed into an fp32 accumulator with
+    floating-point atomics, so its last fp32 bits depend on the order of arrival and a few of its bf16
+    values may round the other way: it must agree to far below the parity tolerance."""
+    names = ("dQ", "dK", "dV", "d_depth_kv", "d_depth_v")
+    for n, s, t in zip(names, a, b):
+        if s is None or t is None:
+            assert s is None and t is None, n
+            continue
+        if n == "dQ":
+            err = rel_l2(f64(s), f64(t))
+            assert err <= 1e-3, f"{what} dQ differs between identical calls by rel-L2 {err:.3e}"
+        else:
+            assert torch.equal(s, t), f"{what} {n} changed between identical calls"

@@ -4,7 +4,7 @@ bench.py times.  The oracle cannot run whole tensors of this size, so it compute
   * forward rows (O_t, LSE_t) one by one for sampled positions of EVERY (b, h),
   * backward rows: dQ_t, dKd_i[t], dVd_i[t] for sampled positions, and dK_j, dV_j for sampled keys
     in the last 256 positions (their sums run over few queries),
-  * one complete (b, h) slice, forward and backward, where a slice is affordable (c3, c5),
+  * one complete (b, h) slice, forward and backward, per config (c3 at l = 32, c4, c5),
 
 and a property that holds at any size covers the rest: sum_s dV_s + sum_{t,i} dVd_i[t] = sum_t dO_t.
 Depth tensors are regenerated slot by slot from their seeds, so the logical [l,B,T,H,d] tensors
@@ -17,7 +17,7 @@ import torch
 import paper_2603_15619_b200 as moda
 from paper_2603_15619_b200 import synthetic
 
-from parity import TOL_GRAD_REL_L2, assert_forward_close, f64, rel_l2
+from parity import TOL_GRAD_REL_L2, TOL_GRAD_ROW_REL_L2, assert_forward_close, f64, rel_l2, worst_row_rel_l2
 from oracle import moda_oracle as orc
 
 pytestmark = pytest.mark.gpu
@@ -113,6 +113,13 @@ def check_config(w, heads_bwd=4, rows_per_head=6, tail=256, seed=1):
             errs["dVd"] = rel_l2(gv.transpose(1, 0, 2), dVd_r)
         bad = {n: v for n, v in errs.items() if not v <= TOL_GRAD_REL_L2}
         assert not bad, f"{w.name} b={b} h={h}: {bad} (all {errs})"
+        rerrs = {"dQ": worst_row_rel_l2(f64(dQ[b, tt, h]), dQ_r), "dK": worst_row_rel_l2(f64(dK[b, kt, h]), dK_r),
+                 "dV": worst_row_rel_l2(f64(dV[b, kt, h]), dV_r)}
+        if w.l:
+            rerrs["dKd"] = worst_row_rel_l2(gk.transpose(1, 0, 2), dKd_r)
+            rerrs["dVd"] = worst_row_rel_l2(gv.transpose(1, 0, 2), dVd_r)
+        bad = {n: v for n, v in rerrs.items() if not v <= TOL_GRAD_ROW_REL_L2}
+        assert not bad, f"{w.name} b={b} h={h}: worst sampled row {bad} (all {rerrs})"
         for n, v in errs.items():
             worst[n] = max(worst.get(n, 0), v)
     # property at full size
@@ -140,17 +147,24 @@ def check_slice(w, x, outs, b, h):
     O_ref, LSE_ref = orc.forward(*args, w.scale)
     assert_forward_close(O[b:b + 1, :, h:h + 1], LSE[b:b + 1, h:h + 1], O_ref, LSE_ref, f"{w.name} slice")
     refs = orc.backward(*args, sl(x["dO"]), w.scale)
-    errs = {"dQ": rel_l2(sl(dQ), refs[0]), "dK": rel_l2(sl(dK), refs[1]), "dV": rel_l2(sl(dV), refs[2])}
+    pairs = {"dQ": (sl(dQ), refs[0]), "dK": (sl(dK), refs[1]), "dV": (sl(dV), refs[2])}
     if w.l:
         all_t = {(b, h): list(range(w.T))}
         gk, gv = depth_rows(w, dcache, all_t)[(b, h)]        # [l, T, d]
-        errs["dKd"] = rel_l2(gk, refs[3][:, 0, :, 0])
-        errs["dVd"] = rel_l2(gv, refs[4][:, 0, :, 0])
+        pairs["dKd"] = (gk, refs[3][:, 0, :, 0])
+        pairs["dVd"] = (gv, refs[4][:, 0, :, 0])
+    errs = {n: rel_l2(g, r) for n, (g, r) in pairs.items()}
     bad = {n: v for n, v in errs.items() if not v <= TOL_GRAD_REL_L2}
     assert not bad, f"{w.name} slice b={b} h={h}: {bad} (all {errs})"
+    # every row of the slice on its own: dK / dV rows near j = 0 are sums over the whole sequence (the
+    # longest inner loops of the dK/dV pass), rows near T - 1 over a few queries
+    rerrs = {n: worst_row_rel_l2(g, r) for n, (g, r) in pairs.items()}
+    bad = {n: v for n, v in rerrs.items() if not v <= TOL_GRAD_ROW_REL_L2}
+    assert not bad, f"{w.name} slice b={b} h={h}: worst row {bad} (all {rerrs})"
+    return errs, rerrs
 
 
-@pytest.mark.parametrize("l", [0, 8, 32])
+@pytest.mark.parametrize("l", list(synthetic.C3_DEPTHS))
 def test_c3_depth_sweep_points(l):
     w = synthetic.WORKLOADS["c3"].with_l(l)
     x, outs, _ = check_config(w, heads_bwd=3)
@@ -160,7 +174,10 @@ def test_c3_depth_sweep_points(l):
 
 def test_c4_long_context_64k():
     w = synthetic.WORKLOADS["c4"]
-    check_config(w, heads_bwd=3)
+    x, outs, _ = check_config(w, heads_bwd=3)
+    # One complete head at T = 65536: every dK / dV row, including those of the first key tiles whose
+    # sums run over all 65536 queries, and every dQ / depth-gradient row, against the oracle.
+    check_slice(w, x, outs, 0, 5)
 
 
 def test_c5_narrow_heads_deep_stack():

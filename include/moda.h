@@ -80,8 +80,30 @@ int moda_last_cuda_error(void);
  * down normally, leaving its outputs undefined.  0 means no kernel has reported a
  * problem.  This call synchronises the device.  Returns the status word (>= 0) or a
  * negative MODA_ERR_CUDA.
+ *
+ * The same code is also written to four bytes of pinned host memory that the library maps
+ * into the device on its first launching call on that device (the only memory the library
+ * ever allocates: host memory, once per device; make that first call before any stream
+ * capture).  Every launching entry point looks at those bytes first, without synchronising:
+ * once a kernel has given up a wait, later calls on that device return
+ * MODA_ERR_DEVICE_TIMEOUT and launch nothing until moda_last_status(1) has cleared the word.
+ * (Kernels that were already queued behind the failed one exit at once and leave their
+ * outputs undefined too.)
  */
 int moda_last_status(int clear);
+
+/*
+ * Self-test of the bounded-wait machinery.  Launches one tiny kernel (one CTA; no TMA, no
+ * tensor memory) whose single thread waits on an mbarrier that nobody ever arrives at, with
+ * a limit of about 1 ms instead of the production kernels' 1 s.  The wait runs out, the
+ * kernel records MODA_SELFTEST_WAIT_STATUS in the status word and returns normally; the GPU
+ * context stays healthy.  Afterwards moda_last_status reports that value and launching
+ * entry points return MODA_ERR_DEVICE_TIMEOUT until it is cleared.  (No counterpart in the
+ * paper: it exercises this library's failure reporting.)
+ */
+#define MODA_SELFTEST_WAIT_SITE 255
+#define MODA_SELFTEST_WAIT_STATUS ((MODA_SELFTEST_WAIT_SITE << 8) | 1)
+int moda_selftest_wait_timeout(void* stream);
 
 /* Bytes of a depth-KV cache (or depth-gradient buffer) holding l_max slots. 0 on bad arguments. */
 size_t moda_depth_cache_bytes(int B, int T, int H, int d, int l_max);
@@ -107,7 +129,11 @@ int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth
                   int B, int T, int H, int d, int l, float scale,
                   void* O, float* LSE, void* stream);
 
-/* Bytes of scratch moda_attn_bwd needs (fp32 row terms D_t = <dO_t, O_t>). */
+/*
+ * Bytes of scratch moda_attn_bwd needs: fp32 row terms D_t = <dO_t, O_t> ([B][H][T]) and an fp32
+ * accumulator for dQ (B * H * ceil(T/128) * 128 * d values; 4 bytes per dQ element).  Enough for
+ * every stage mask of moda_attn_bwd_stages.
+ */
 size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l);
 
 /*
@@ -117,6 +143,14 @@ size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l);
  * when l > 0, slots 0..l-1 of d_depth_kv (bf16, cache layout: kv = 0 holds dKd, kv = 1
  * holds dVd; tail rows zero).  `workspace` is caller-owned scratch of at least
  * moda_bwd_workspace_bytes() bytes; its contents need not be preserved between calls.
+ *
+ * Three launches.  (1) Everything local to a query row: D_t, the depth gradients dKd_i, dVd_i
+ * and the depth share of dQ, which starts the fp32 dQ accumulator.  (2) The sequence part, one
+ * CTA per key tile: S and dP are formed once, P = exp(S - LSE) is evaluated once per score, dK
+ * and dV accumulate on chip and every dQ tile is ADDED to the accumulator with floating-point
+ * atomics in global memory.  (3) dQ = bf16(scale * accumulator).  dK, dV and the depth gradients
+ * are bit-reproducible; the last bits of dQ depend on the order in which the CTAs of (2) reach a
+ * query tile.  Pass MODA_BWD_DETERMINISTIC to moda_attn_bwd_stages for reproducible bits.
  */
 int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth_kv,
                   const void* O, const void* dO, const float* LSE,
@@ -126,12 +160,21 @@ int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth
 
 /*
  * moda_attn_bwd is three launches; this entry point runs a subset of them so that each can
- * be timed or profiled on its own.  `stages` is a bit mask:
+ * be timed or profiled on its own.  `stages` is a bit mask of the launches in the order above:
+ *     MODA_BWD_STAGE_ROWS      (1) row terms, depth gradients, start of the dQ accumulator
+ *     MODA_BWD_STAGE_SEQ       (2) dK, dV and the dQ tiles (reads D_t, adds to the accumulator)
+ *     MODA_BWD_STAGE_FINISH    (3) dQ from the accumulator
+ * moda_attn_bwd(...) is moda_attn_bwd_stages(..., MODA_BWD_ALL_STAGES, stream).
+ * MODA_BWD_DETERMINISTIC selects the split form of the backward instead: no floating-point
+ * atomics, every output bit-reproducible, at the price of seven contractions for five and two
+ * evaluations of every exp (measurably slower; its only scratch is D_t).  Its three launches
+ * take the same three bits, under their older names:
  *     MODA_BWD_STAGE_ROWTERMS  D_t = <dO_t, O_t> for every row, into `workspace`
  *     MODA_BWD_STAGE_DQ        dQ and the depth gradients (reads D_t from `workspace`)
  *     MODA_BWD_STAGE_DKDV      dK and dV                  (reads D_t from `workspace`)
- * moda_attn_bwd(...) is moda_attn_bwd_stages(..., MODA_BWD_ALL_STAGES, stream).
- * One more bit changes how the depth gradients leave the MODA_BWD_STAGE_DQ stage:
+ * Grouped-query calls whose depth gradients are formed from per-row factors (see
+ * moda_attn_bwd_gqa) always take the split form.
+ * One more bit changes how the depth gradients are written:
  *     MODA_BWD_ACCUMULATE_DEPTH  slots [0, l) of d_depth_kv are ADDED TO (bf16 additions,
  *                                one per element per call, so the result does not depend on
  *                                scheduling) instead of overwritten.  In a stack of layers
@@ -140,13 +183,17 @@ int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth
  *                                zeroed once by the caller, collects d(loss)/d(slot i)
  *                                over the backward calls of all those layers.
  * All arguments are validated as for moda_attn_bwd whatever the mask; a mask with none of the
- * three stage bits, or with bits above MODA_BWD_ACCUMULATE_DEPTH, is MODA_ERR_BAD_SHAPE.
+ * three stage bits, or with bits above MODA_BWD_DETERMINISTIC, is MODA_ERR_BAD_SHAPE.
  */
 #define MODA_BWD_STAGE_ROWTERMS 1
 #define MODA_BWD_STAGE_DQ 2
 #define MODA_BWD_STAGE_DKDV 4
+#define MODA_BWD_STAGE_ROWS 1
+#define MODA_BWD_STAGE_SEQ 2
+#define MODA_BWD_STAGE_FINISH 4
 #define MODA_BWD_ALL_STAGES 7
 #define MODA_BWD_ACCUMULATE_DEPTH 8
+#define MODA_BWD_DETERMINISTIC 16
 int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void* depth_kv,
                          const void* O, const void* dO, const float* LSE,
                          int B, int T, int H, int d, int l, float scale,
@@ -262,12 +309,13 @@ int moda_attn_decode_paged(const void* q, const void* K_pages, const void* V_pag
  * Backward pass for callers that have no scratch buffer to give.  (The paper has no
  * counterpart: this is a deployment convenience of this library, not part of the method.)
  *
- * moda_attn_bwd needs a caller-owned workspace for the per-row terms D_t.  Some callers cannot
+ * moda_attn_bwd needs a caller-owned workspace.  Some callers cannot
  * provide one: a plug-in that is only handed its input and output tensors by a host framework,
  * or a serving process that sized all of its device memory at start-up and is not allowed to call
  * cudaMalloc afterwards (the call synchronises the whole device and can fail once memory is
- * fully committed).  This variant computes exactly what moda_attn_bwd computes, with the same
- * kernels, but keeps D_t in an array that is compiled into the library image
+ * fully committed).  This variant computes what moda_attn_bwd_stages computes with
+ * MODA_BWD_DETERMINISTIC (the split form of the backward, whose only scratch is the per-row
+ * terms D_t), with the same kernels, but keeps D_t in an array that is compiled into the library image
  * (MODA_STATIC_SCRATCH_ROWS fp32 values = 4 MiB, resident on every GPU that loads the library
  * until the process exits).  It calls no cudaMalloc, cudaFree or any other allocating routine.
  *

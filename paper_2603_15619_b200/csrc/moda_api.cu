@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "moda_bwd.cuh"
+#include "moda_bwd_fused.cuh"
 #include "moda_cache.cuh"
 #include "moda_decode.cuh"
 #include "moda_depth_gqa.cuh"
@@ -19,6 +20,20 @@ namespace {
 using namespace moda;
 
 thread_local int tl_last_cuda_error = 0;
+
+// One thread waits on an mbarrier that nothing arrives at; the bounded wait gives up after `limit_ns`
+// and records (MODA_SELFTEST_WAIT_SITE << 8) | 1 exactly as a production kernel's wait would.
+__global__ void wait_timeout_selftest_kernel(uint64_t limit_ns) {
+    __shared__ __align__(8) uint64_t bar_word;
+    __shared__ int abort_word;
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        mbar_init(smem_u32(&bar_word), 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait(smem_u32(&bar_word), 0, &abort_word, MODA_SELFTEST_WAIT_SITE, limit_ns);
+}
 
 inline bool cuda_ok(cudaError_t e) {
     if (e == cudaSuccess) return true;
@@ -81,17 +96,55 @@ int check_groups(int H, int H_kv) {
     return MODA_OK;
 }
 
-int check_device() {
+// Host-visible mirror of the device status word, one per device: four bytes of pinned host memory that
+// the device can write (zero-copy).  A kernel whose wait runs out stores its code there as well as in
+// g_moda_status, so the next call on that device sees it with a plain load -- no synchronisation --
+// and returns MODA_ERR_DEVICE_TIMEOUT instead of queueing work behind a failed kernel.
+constexpr int kMaxDevices = 64;
+std::mutex g_mirror_mutex;
+volatile int* g_status_mirror[kMaxDevices] = {};
+
+int ensure_status_mirror(int dev) {
+    if (dev < 0 || dev >= kMaxDevices) return MODA_OK;         // beyond the table: moda_last_status still works
+    std::lock_guard<std::mutex> lock(g_mirror_mutex);
+    if (g_status_mirror[dev] != nullptr) return MODA_OK;
+    int* host = nullptr;
+    int* dev_alias = nullptr;
+    if (!cuda_ok(cudaHostAlloc(reinterpret_cast<void**>(&host), sizeof(int), cudaHostAllocMapped))) return MODA_ERR_CUDA;
+    *host = 0;
+    if (!cuda_ok(cudaHostGetDevicePointer(reinterpret_cast<void**>(&dev_alias), host, 0)) ||
+        !cuda_ok(cudaMemcpyToSymbol(g_moda_status_host, &dev_alias, sizeof(dev_alias)))) {
+        (void)cudaFreeHost(host);
+        return MODA_ERR_CUDA;
+    }
+    g_status_mirror[dev] = host;
+    return MODA_OK;
+}
+
+// Device check of every launching entry point: an sm_100 part, and no kernel of an earlier call on this
+// device has given up a wait.  `may_allocate` = false (the entry point that must not allocate) skips the
+// one-time creation of the status mirror; a mirror made by an earlier call is still consulted.
+int check_device(bool may_allocate = true) {
     static thread_local int cached_dev = -1;
     static thread_local int cached_rc = MODA_ERR_DEVICE;
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
-    if (dev == cached_dev) return cached_rc;
-    int major = 0;
-    if (!cuda_ok(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev))) return MODA_ERR_CUDA;
-    cached_dev = dev;
-    cached_rc = (major == 10) ? MODA_OK : MODA_ERR_DEVICE;
-    return cached_rc;
+    if (dev != cached_dev) {
+        int major = 0;
+        if (!cuda_ok(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev))) return MODA_ERR_CUDA;
+        cached_dev = dev;
+        cached_rc = (major == 10) ? MODA_OK : MODA_ERR_DEVICE;
+    }
+    if (cached_rc != MODA_OK) return cached_rc;
+    if (dev >= 0 && dev < kMaxDevices) {
+        volatile int* mirror = g_status_mirror[dev];
+        if (mirror == nullptr && may_allocate) {
+            if (int rc = ensure_status_mirror(dev)) return rc;
+            mirror = g_status_mirror[dev];
+        }
+        if (mirror != nullptr && *mirror != 0) return MODA_ERR_DEVICE_TIMEOUT;
+    }
+    return MODA_OK;
 }
 
 template <typename Kernel>
@@ -261,9 +314,83 @@ int launch_depth_bwd(DepthBwdParams m, cudaStream_t stream) {
     }
 }
 
+// Which form of the backward a call takes.  The fused form (moda_bwd_fused.cuh) covers plain multi-head
+// calls and those grouped-query calls whose depth part is either absent or done by the per-position kernel;
+// grouped-query calls on the row-local depth path keep the split form, whose dQ pass leaves the per-row
+// factors that depth_grad_group_kernel sums over the heads of a group.
+inline bool bwd_uses_fused(int d, int G, int l, bool deterministic) {
+    if (deterministic) return false;
+    return G == 1 || l == 0 || gqa_depth_split_bwd(d, G, l);
+}
+
+template <int D>
+int launch_bwd_fused(const BwdArgs& a, int stages, cudaStream_t stream) {
+    const int B = a.B, T = a.T, H = a.H, Hk = a.Hk, G = a.H / a.Hk;
+    using L = FusedSmem<D>;
+    CUtensorMap mK, mV, mQ, mdO, mdK, mdV;
+    if (!make_bthd_map(&mK, a.K, B, T, Hk, D) || !make_bthd_map(&mV, a.V, B, T, Hk, D) ||
+        !make_bthd_map(&mQ, a.Q, B, T, H, D) || !make_bthd_map(&mdO, a.dO, B, T, H, D) ||
+        !make_bthd_map(&mdK, a.dK, B, T, Hk, D) || !make_bthd_map(&mdV, a.dV, B, T, Hk, D))
+        return MODA_ERR_CUDA;
+    static thread_local int configured_dev = -1;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (configured_dev != dev) {
+        if (!set_smem_limit(moda_bwd_fused_kernel<D>, L::kDynamic)) return MODA_ERR_CUDA;
+        configured_dev = dev;
+    }
+    float* delta = static_cast<float*>(a.workspace);
+    float* dq_acc = reinterpret_cast<float*>(static_cast<char*>(a.workspace) + bwd_fused_rowterm_bytes(B, T, H));
+    const bool split_depth = G > 1 && a.l > 0;             // depth part by the per-position kernel after the finish kernel
+    const unsigned tiles = unsigned(B) * H * num_tiles(T);
+    constexpr int kRowThreads = kTileRows * (D / 32);
+    if (stages & 1) {
+        RowsParams r;
+        r.Q = static_cast<const __nv_bfloat16*>(a.Q);
+        r.O = static_cast<const __nv_bfloat16*>(a.O);
+        r.dO = static_cast<const __nv_bfloat16*>(a.dO);
+        r.depth_kv = static_cast<const __nv_bfloat16*>(a.depth_kv);
+        r.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
+        r.LSE = a.LSE; r.delta = delta; r.dq_acc = dq_acc;
+        r.B = B; r.T = T; r.H = H; r.l = split_depth ? 0 : a.l;
+        r.accumulate = a.accumulate_depth ? 1 : 0;
+        r.scale = a.scale; r.scale_log2 = a.scale * kLog2e;
+        bwd_rows_kernel<D><<<tiles, kRowThreads, 0, stream>>>(r);
+        if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    }
+    if (stages & 2) {
+        FusedParams f;
+        f.LSE = a.LSE; f.delta = delta; f.dq_acc = dq_acc;
+        f.B = B; f.T = T; f.H = H; f.G = G;
+        f.scale = a.scale; f.scale_log2 = a.scale * kLog2e;
+        const unsigned grid = unsigned(B) * Hk * num_tiles(T);
+        moda_bwd_fused_kernel<D><<<grid, kBwdFusedThreads, L::kDynamic, stream>>>(mK, mV, mQ, mdO, mdK, mdV, f);
+        if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    }
+    if (stages & 4) {
+        bwd_dq_finish_kernel<D><<<tiles, kRowThreads, 0, stream>>>(dq_acc, static_cast<__nv_bfloat16*>(a.dQ), B, T, H, a.scale);
+        if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+        if (split_depth) {
+            DepthBwdParams m;
+            m.Q = static_cast<const __nv_bfloat16*>(a.Q);
+            m.dO = static_cast<const __nv_bfloat16*>(a.dO);
+            m.depth_kv = static_cast<const __nv_bfloat16*>(a.depth_kv);
+            m.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
+            m.dQ = static_cast<__nv_bfloat16*>(a.dQ);
+            m.LSE = a.LSE; m.delta = delta;
+            m.B = B; m.T = T; m.H = H; m.Hk = Hk; m.l = a.l;
+            m.scale = a.scale; m.scale_log2 = a.scale * kLog2e;
+            m.accumulate = a.accumulate_depth ? 1 : 0;
+            if (int rc = launch_depth_bwd<D>(m, stream)) return rc;
+        }
+    }
+    return MODA_OK;
+}
+
 template <int D>
 int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
     const int B = a.B, T = a.T, H = a.H, Hk = a.Hk, G = a.H / a.Hk;
+    if (bwd_uses_fused(D, G, a.l, a.deterministic)) return launch_bwd_fused<D>(a, stages, stream);
     CUtensorMap mQ, mdO, mK64, mV64, mdQ, mK, mV, mQ64, mdO64, mdK, mdV;
     if (!make_bthd_map(&mQ, a.Q, B, T, H, D) || !make_bthd_map(&mdO, a.dO, B, T, H, D) ||
         !make_bthd_map(&mK64, a.K, B, T, Hk, D, kKeyTile) || !make_bthd_map(&mV64, a.V, B, T, Hk, D, kKeyTile) ||
@@ -483,6 +610,13 @@ const char* moda_strerror(int code) {
 
 int moda_last_cuda_error(void) { return tl_last_cuda_error; }
 
+
+int moda_selftest_wait_timeout(void* stream) {
+    if (int rc = check_device()) return rc;
+    wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(1000000ull);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+
 int moda_last_status(int clear) {
     int st = 0;
     if (!cuda_ok(cudaDeviceSynchronize())) return MODA_ERR_CUDA;
@@ -490,6 +624,9 @@ int moda_last_status(int clear) {
     if (clear && st != 0) {
         const int zero = 0;
         if (!cuda_ok(cudaMemcpyToSymbol(g_moda_status, &zero, sizeof(int)))) return MODA_ERR_CUDA;
+        int dev = 0;
+        if (cuda_ok(cudaGetDevice(&dev)) && dev >= 0 && dev < kMaxDevices && g_status_mirror[dev] != nullptr)
+            *g_status_mirror[dev] = 0;
     }
     return st;
 }
@@ -554,13 +691,15 @@ int moda_attn_fwd_prefill(const void* Q, const void* K, const void* V, const voi
 }
 
 size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l) {
-    if (check_shape(B, T, H, d) != MODA_OK || l < 0 || l > MODA_MAX_DEPTH) return 0;
-    return bwd_workspace_bytes(B, T, H);
+    return moda_bwd_workspace_bytes_gqa(B, T, H, H, d, l);
 }
 
+// Enough for either form of the backward (the reproducible split form needs far less than the fused one).
 size_t moda_bwd_workspace_bytes_gqa(int B, int T, int H, int H_kv, int d, int l) {
     if (check_shape(B, T, H, d) != MODA_OK || check_groups(H, H_kv) != MODA_OK || l < 0 || l > MODA_MAX_DEPTH) return 0;
-    return bwd_workspace_bytes_gqa(B, T, H, H_kv, l);
+    const size_t split = bwd_workspace_bytes_gqa(B, T, H, H_kv, l);
+    const size_t fused = bwd_uses_fused(d, H / H_kv, l, false) ? bwd_fused_workspace_bytes(B, T, H, d) : 0;
+    return split > fused ? split : fused;
 }
 
 int moda_attn_bwd(const void* Q, const void* K, const void* V, const void* depth_kv,
@@ -597,7 +736,8 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
                              void* workspace, size_t workspace_bytes, int stages, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
-    if ((stages & MODA_BWD_ALL_STAGES) == 0 || stages < 0 || stages > (MODA_BWD_ALL_STAGES | MODA_BWD_ACCUMULATE_DEPTH))
+    if ((stages & MODA_BWD_ALL_STAGES) == 0 || stages < 0 ||
+        stages > (MODA_BWD_ALL_STAGES | MODA_BWD_ACCUMULATE_DEPTH | MODA_BWD_DETERMINISTIC))
         return MODA_ERR_BAD_SHAPE;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv || !d_depth_kv)))
@@ -606,10 +746,14 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
         !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) ||
         (l > 0 && (!aligned16(depth_kv) || !aligned16(d_depth_kv))))
         return MODA_ERR_MISALIGNED;
-    if (!workspace || !aligned16(workspace) || workspace_bytes < bwd_workspace_bytes_gqa(B, T, H, H_kv, l)) return MODA_ERR_WORKSPACE;
+    const bool deterministic = (stages & MODA_BWD_DETERMINISTIC) != 0;
+    const size_t need = bwd_uses_fused(d, H / H_kv, l, deterministic) ? bwd_fused_workspace_bytes(B, T, H, d)
+                                                                       : bwd_workspace_bytes_gqa(B, T, H, H_kv, l);
+    if (!workspace || !aligned16(workspace) || workspace_bytes < need) return MODA_ERR_WORKSPACE;
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     BwdArgs a;
+    a.deterministic = deterministic;
     a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv; a.O = O; a.dO = dO; a.LSE = LSE;
     a.B = B; a.T = T; a.H = H; a.Hk = H_kv; a.l = l; a.scale = scale;
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
@@ -662,7 +806,6 @@ namespace {
 // each GPU gave the array is looked up once per device with cudaGetSymbolAddress below.
 static __device__ __align__(256) float g_static_rowterms[MODA_STATIC_SCRATCH_ROWS];
 
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 float* g_static_rowterms_addr[kMaxDevices] = {};
 
@@ -696,13 +839,14 @@ extern "C" int moda_attn_bwd_static_scratch(const void* Q, const void* K, const 
         !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) ||
         (l > 0 && (!aligned16(depth_kv) || !aligned16(d_depth_kv))))
         return MODA_ERR_MISALIGNED;
-    if (int rc = check_device()) return rc;
+    if (int rc = check_device(/*may_allocate=*/false)) return rc;
     float* scratch = nullptr;
     if (int rc = static_scratch_for_current_device(&scratch)) return rc;
     BwdArgs a;
     a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv; a.O = O; a.dO = dO; a.LSE = LSE;
     a.B = B; a.T = T; a.H = H; a.Hk = H; a.l = l; a.scale = scale;
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = scratch;
+    a.deterministic = true;                  // the split form: its only scratch is the row terms, which fit the built-in array
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return d == 128 ? launch_bwd<128>(a, MODA_BWD_ALL_STAGES, st) : launch_bwd<64>(a, MODA_BWD_ALL_STAGES, st);
 }

@@ -37,6 +37,7 @@ struct BwdArgs {
     float scale;
     void *dQ, *dK, *dV, *d_depth_kv, *workspace;
     bool accumulate_depth = false;   // add the depth gradients to d_depth_kv instead of overwriting it
+    bool deterministic = false;      // split form (bit-reproducible) instead of the fused form
 };
 
 inline size_t bwd_workspace_bytes(int B, int T, int H) {

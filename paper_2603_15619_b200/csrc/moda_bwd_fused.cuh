@@ -1,0 +1,680 @@
+// MoDA backward, fused form: five contractions and one exponential per score.
+//
+// The paper prints no backward pass; this is the derivative of the Sec. 2.2 operator.  With
+// P = exp(S - LSE) (sequence), R = exp(U - LSE) (depth), D_t = <dO_t, O_t>:
+//
+//   dS = P o (dO V^T - D),   dU_i = R_i (<dO, Vd_i> - D)
+//   dQ = scale (dS K + sum_i dU_i Kd_i)     dK = scale dS^T Q     dV = P^T dO
+//   dKd_i = scale dU_i Q                    dVd_i = R_i dO        (row-local)
+//
+// Three launches on the caller's stream:
+//   1. bwd_rows_kernel        everything that is local to a query row: D_t, and for every depth slot
+//                             R_i, dU_i, dKd_i, dVd_i (written in cache layout) and the row's depth share
+//                             of dQ, which initialises an fp32 dQ accumulator in the workspace.  Streams the
+//                             depth cache exactly once; bound by HBM.
+//   2. moda_bwd_fused_kernel  one CTA per 128-key tile, looping over the 128-query tiles at or below the
+//                             diagonal.  Per pair of tiles: S^T = K Q^T and dP^T = V dO^T (tcgen05, operands
+//                             in shared memory), P^T and dS^T formed once by the row warps, dV += P^T dO (P^T
+//                             from tensor memory), dK += dS^T Q and dQ_tile = dS K (dS^T staged once in shared
+//                             memory and used by both: K-major for dK, MN-major for dQ).  dK, dV accumulate in
+//                             tensor memory over the whole loop; the dQ tile is added to the fp32 accumulator
+//                             in L2 by bulk reductions (cp.reduce.async.bulk .add.f32) from a staging buffer --
+//                             the only place where the order of floating-point additions depends on scheduling.
+//   3. bwd_dq_finish_kernel   dQ = bf16(scale * accumulator).
+//
+// Against the split form (moda_bwd.cuh: a dQ pass and a dK/dV pass, seven contractions, every score
+// exponentiated twice, bit-reproducible) this form does 5/7 of the tensor work and half of the
+// exponentials; the host picks it unless the caller asks for reproducible bits.
+#pragma once
+
+#include "moda_bwd.cuh"
+#include "moda_cache.cuh"
+#include "moda_fwd.cuh"
+#include "moda_fwd_wide.cuh"   // aligned_dynamic_smem
+#include "sm100_ptx.cuh"
+
+namespace moda {
+
+// fp32 dQ accumulator: [b][h][query tile][feature / 4][row 128][4], so that a warp whose lanes own
+// consecutive rows adds (or stores) 512 contiguous bytes per instruction.
+inline size_t dq_acc_bytes(int B, int T, int H, int d) {
+    return size_t(B) * H * num_tiles(T) * kTileRows * d * 4;
+}
+// Workspace of the fused backward: row terms D_t, then the dQ accumulator (256-byte aligned).
+inline size_t bwd_fused_rowterm_bytes(int B, int T, int H) {
+    return (size_t(B) * H * T * 4 + 255) & ~size_t(255);
+}
+inline size_t bwd_fused_workspace_bytes(int B, int T, int H, int d) {
+    return bwd_fused_rowterm_bytes(B, T, H) + dq_acc_bytes(B, T, H, d);
+}
+
+// =====================================================================================
+// 1. Row-local part: D_t, depth gradients, depth share of dQ
+// =====================================================================================
+// One CTA per (b, h, 128-row tile); D / 32 threads per row, each owning 32 features (four 16-byte
+// chunks of every depth row).  Lanes of a row are adjacent, so the two dot products of a slot are
+// finished with shuffles; lanes with the same feature part own consecutive rows, so every warp access
+// to the cache is a set of 128-byte (d = 128) or 256-byte (d = 64) runs.  q and dO stay packed in
+// registers; a slot's key and value chunks are read once and used for everything the slot needs.
+struct RowsParams {
+    const __nv_bfloat16 *Q, *O, *dO, *depth_kv;
+    __nv_bfloat16* d_depth_kv;
+    const float* LSE;
+    float* delta;        // [B][H][T]
+    float* dq_acc;       // accumulator layout above; every element is written (zeros when l == 0)
+    int B, T, H, l;
+    int accumulate;      // nonzero: depth gradients are added to d_depth_kv (bf16 adds in L2)
+    float scale, scale_log2;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kTileRows * (D / 32), 512 / (kTileRows * (D / 32)))
+bwd_rows_kernel(const RowsParams p) {
+    constexpr int PARTS = D / 32;                 // threads per row
+    constexpr int CH = D / 8;                     // 16-byte chunks per row
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int part = lane % PARTS;
+    const int r = warp * (32 / PARTS) + lane / PARTS;
+    const int nq = num_tiles(p.T);
+    const int qt = blockIdx.x % nq;
+    const int bh = blockIdx.x / nq;
+    const int b = bh / p.H, h = bh % p.H;
+    const int t = qt * kTileRows + r;
+    const bool valid = t < p.T;
+
+    uint4 q4[4], g4[4];
+    float dpart = 0.f;
+    if (valid) {
+        const size_t row = ((size_t(b) * p.T + t) * p.H + h) * CH + part * 4;
+        const uint4* Q = reinterpret_cast<const uint4*>(p.Q) + row;
+        const uint4* O = reinterpret_cast<const uint4*>(p.O) + row;
+        const uint4* G = reinterpret_cast<const uint4*>(p.dO) + row;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            q4[j] = Q[j];
+            g4[j] = G[j];
+            dpart += dot8_bf16(O[j], g4[j]);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) q4[j] = g4[j] = make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int off = 1; off < PARTS; off <<= 1) dpart += __shfl_xor_sync(0xffffffffu, dpart, off);
+    const float delta = dpart;
+    const size_t row_idx = (size_t(b) * p.H + h) * p.T + t;
+    const float neg_lse2 = valid ? -p.LSE[row_idx] * kLog2e : -INFINITY;   // rows past T: R = 0, zero gradients
+    if (valid && part == 0) p.delta[row_idx] = delta;
+
+    float acc[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+
+    if (p.l > 0) {
+        const size_t slot_stride = cache_slot_elems(p.B, p.T, p.H, D) / 8;                    // in uint4
+        const size_t blk = (size_t(bh) * nq + qt) * 2 * (kTileRows * CH) + size_t(part * 4) * kTileRows + r;
+        const uint4* cK = reinterpret_cast<const uint4*>(p.depth_kv) + blk;
+        const uint4* cV = cK + kTileRows * CH;
+        uint4* gK = reinterpret_cast<uint4*>(p.d_depth_kv) + blk;
+        uint4* gV = gK + kTileRows * CH;
+        const bool accumulate = p.accumulate != 0;
+#pragma unroll 1
+        for (int i = 0; i < p.l; ++i) {
+            uint4 kc[4], vc[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                kc[j] = __ldcs(cK + j * kTileRows);          // streamed: every byte of the cache is used once
+                vc[j] = __ldcs(cV + j * kTileRows);
+            }
+            float u = 0.f, dr = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                u += dot8_bf16(q4[j], kc[j]);
+                dr += dot8_bf16(g4[j], vc[j]);
+            }
+#pragma unroll
+            for (int off = 1; off < PARTS; off <<= 1) {
+                u += __shfl_xor_sync(0xffffffffu, u, off);
+                dr += __shfl_xor_sync(0xffffffffu, dr, off);
+            }
+            const float R = fast_exp2(fmaf(u, p.scale_log2, neg_lse2));   // the forward's LSE covers both key sets
+            const float dU = R * (dr - delta);
+            const uint32_t r2 = pack_bf16x2(R, R);
+            const float sdu = dU * p.scale;
+            const uint32_t sdu2 = pack_bf16x2(sdu, sdu);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint4 ov, ok;
+                ov.x = mul_bf16x2(g4[j].x, r2); ov.y = mul_bf16x2(g4[j].y, r2);
+                ov.z = mul_bf16x2(g4[j].z, r2); ov.w = mul_bf16x2(g4[j].w, r2);
+                ok.x = mul_bf16x2(q4[j].x, sdu2); ok.y = mul_bf16x2(q4[j].y, sdu2);
+                ok.z = mul_bf16x2(q4[j].z, sdu2); ok.w = mul_bf16x2(q4[j].w, sdu2);
+                if (accumulate) {
+                    red_add_bf16x2_v4(gV + j * kTileRows, ov);
+                    red_add_bf16x2_v4(gK + j * kTileRows, ok);
+                } else {
+                    __stcs(gV + j * kTileRows, ov);
+                    __stcs(gK + j * kTileRows, ok);
+                }
+                acc[8 * j + 0] = fmaf(dU, bf16_lo_to_f32(kc[j].x), acc[8 * j + 0]);
+                acc[8 * j + 1] = fmaf(dU, bf16_hi_to_f32(kc[j].x), acc[8 * j + 1]);
+                acc[8 * j + 2] = fmaf(dU, bf16_lo_to_f32(kc[j].y), acc[8 * j + 2]);
+                acc[8 * j + 3] = fmaf(dU, bf16_hi_to_f32(kc[j].y), acc[8 * j + 3]);
+                acc[8 * j + 4] = fmaf(dU, bf16_lo_to_f32(kc[j].z), acc[8 * j + 4]);
+                acc[8 * j + 5] = fmaf(dU, bf16_hi_to_f32(kc[j].z), acc[8 * j + 5]);
+                acc[8 * j + 6] = fmaf(dU, bf16_lo_to_f32(kc[j].w), acc[8 * j + 6]);
+                acc[8 * j + 7] = fmaf(dU, bf16_hi_to_f32(kc[j].w), acc[8 * j + 7]);
+            }
+            cK += slot_stride; cV += slot_stride; gK += slot_stride; gV += slot_stride;
+        }
+    }
+    // depth share of dQ (unscaled) -> accumulator; the fused kernel adds the sequence share on top
+    float4* dst = reinterpret_cast<float4*>(p.dq_acc) + (size_t(bh) * nq + qt) * (D / 4) * kTileRows + size_t(part * 8) * kTileRows + r;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        dst[j * kTileRows] = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+}
+
+// =====================================================================================
+// 3. dQ = bf16(scale * accumulator)
+// =====================================================================================
+template <int D>
+__global__ void __launch_bounds__(kTileRows * (D / 32))
+bwd_dq_finish_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dQ, int B, int T, int H, float scale) {
+    constexpr int PARTS = D / 32;
+    constexpr int CH = D / 8;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int part = lane % PARTS;
+    const int r = warp * (32 / PARTS) + lane / PARTS;
+    const int nq = num_tiles(T);
+    const int qt = blockIdx.x % nq;
+    const int bh = blockIdx.x / nq;
+    const int b = bh / H, h = bh % H;
+    const int t = qt * kTileRows + r;
+    if (t >= T) return;
+    const float4* src = reinterpret_cast<const float4*>(dq_acc) + size_t(blockIdx.x) * (D / 4) * kTileRows + size_t(part * 8) * kTileRows + r;
+    uint4* dst = reinterpret_cast<uint4*>(dQ) + ((size_t(b) * T + t) * H + h) * CH + part * 4;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float4 a = __ldcs(src + (2 * j) * kTileRows);
+        const float4 c = __ldcs(src + (2 * j + 1) * kTileRows);
+        uint4 o;
+        o.x = pack_bf16x2(a.x * scale, a.y * scale); o.y = pack_bf16x2(a.z * scale, a.w * scale);
+        o.z = pack_bf16x2(c.x * scale, c.y * scale); o.w = pack_bf16x2(c.z * scale, c.w * scale);
+        dst[j] = o;
+    }
+}
+
+// =====================================================================================
+// 2. Sequence part: dK, dV and the dQ tiles
+// =====================================================================================
+// 512 threads.
+//   warps 0-7    row warps: a thread owns one key row (= tensor-memory lane) and 64 of the 128 query columns
+//                of an iteration (warps 0-3 the low half, 4-7 the high half): P^T, then dS^T.
+//   warps 8-11   drain warps: a thread owns one query row of the dQ tile; it copies the row out of tensor memory
+//                (which frees the region at once) and adds it to the fp32 accumulator with 16-byte reductions
+//                at whatever pace L2 takes them, without holding up the row warps.
+//   warp 12      loader (TMA tiles, per-query LSE and D_t)
+//   warps 13-15  issue the contractions: S (13), dP (14), dV then dQ then dK (15).  One tcgen05.mma costs its
+//                issuing thread about as long as it executes, so the contractions that start an iteration's two
+//                chains have their own warps on different schedulers; MMAs of different warps are ordered by
+//                mbarriers only.
+//
+// Tensor memory (fp32 columns): X, 128 columns per buffer, S^T overlaid by P^T (bf16) -- one buffer at d = 128,
+// two at d = 64 (where dK and dV leave room);  Y, 128 columns, dP^T and then the dQ tile of the same iteration;
+// dK, D columns;  dV, D columns.  512 columns at either head width.
+//
+// What bounds it (cycle stamps per warp role, T = 8192): at d = 128 the shared-memory port -- per iteration the
+// MMAs read 320 KiB of operands, TMA writes 64 KiB of Q / dO, dS^T is 32 KiB, the dQ staging 64 KiB in and 64 KiB
+// out, against 128 bytes per clock -- and the L2 reduction rate (64 KiB of fp32 additions per iteration per SM; all
+// SMs together sustain about 5.9 TB/s of them); at d = 64 the row warps (the same number of exponentials and
+// conversions per iteration for half the tensor work).
+//
+// Two dependency chains per iteration i, which overlap each other and the next iteration:
+//   X:  S_i -> P_i^T = exp2(S c - LSE c) (row warps) -> dV_i -> X free -> S_{i+1}
+//   Y:  dP_i -> dS_i^T = P o (dP - D) to shared memory (row warps) -> dQ_i -> copied out (drain warps) -> Y free -> dP_{i+1}
+// and dK_i, issued behind dQ_i, fills the tensor pipe while the row warps exponentiate tile i+1.
+constexpr int kBwdFusedThreads = 512;
+
+template <int D>
+struct FusedSmem {
+    static constexpr int kTileBytes = kTileRows * D * 2;       // 128 x D bf16
+    static constexpr int kSubBytes = kTileRows * 128;          // 128 x 64 sub-tile (128-byte rows)
+    // Stages of Q_i.  Q_i is read by S_i early and by dK_i late in its iteration, and a tile takes about 1600
+    // cycles from the TMA issue to the first MMA that uses it, so with two stages the chain "dK_{i-2} completes ->
+    // load Q_i -> S_i -> P_i -> dS_i -> dK_i" spans two iterations and sets the pace; three stages (d = 64, where
+    // shared memory has room) take the load off that chain.
+    static constexpr int kStages = (D == 64) ? 3 : 2;
+    // dO_i is read by dP_i and dV_i, both of which complete before dP_{i+1} can be issued; at d = 128 one
+    // stage leaves the 32 KiB that the dQ staging buffer needs
+    static constexpr int kdOStages = (D == 128) ? 1 : 2;
+    static constexpr int kK = 0;
+    static constexpr int kV = kK + kTileBytes;
+    static constexpr int kQ = kV + kTileBytes;                 // stages of Q_i
+    static constexpr int kdO = kQ + kStages * kTileBytes;      // stages of dO_i
+    static constexpr int kdS = kdO + kdOStages * kTileBytes;   // dS^T: 128 keys x 128 queries bf16
+    static constexpr int kdSBytes = kTileRows * kTileRows * 2;
+    static constexpr int kStg = kdS + kdSBytes;                // 64 feature columns of a dQ tile, fp32, accumulator layout
+    static constexpr int kStgBytes = 64 * kTileRows * 4;
+    static constexpr int kRow = kStg + kStgBytes;              // per stage: -LSE log2e [128], D_t [128]
+    static constexpr int kRowBytes = 2 * kTileRows * 4;
+    static constexpr int kBars = kRow + kStages * kRowBytes;
+    static constexpr int kNumBars = 26;
+    static constexpr int kMisc = kBars + kNumBars * 8;
+    static constexpr int kTotal = kMisc + 16;
+    static constexpr int kSmemLimit = 232448;                  // 227 KiB per CTA on sm_100
+    // the tiles need a 1024-byte aligned base; ask for the slack when it fits (d = 64), else rely on the
+    // dynamic segment starting aligned and check at run time (aligned_dynamic_smem)
+    static constexpr int kDynamic = (kTotal + 1024 <= kSmemLimit) ? kTotal + 1024 : kSmemLimit;
+    static_assert(kTotal <= kSmemLimit, "shared-memory plan too large");
+};
+
+enum FusedBar : int {
+    kFBarKV = 0,
+    kFBarQFull = 1,     // +stage (<= 3), count 32: Q_i and the row terms of the stage have landed
+    kFBarQEmpty = 4,    // +stage (<= 3): dK_i complete (Q_i, the row terms and the dS buffer are free)
+    kFBardOFull = 7,    // +stage (<= 2)
+    kFBardOEmpty = 9,   // +stage (<= 2), count 2: dP_i and dV_i complete
+    kFBarSFull = 11,    // +X buffer: S_i complete
+    kFBarPFull = 13,    // +X buffer, count 256: P_i^T written
+    kFBardPFull = 15,   // dP_i complete
+    kFBardSFull = 16,   // count 256: dS_i^T written to shared memory, dP_i consumed
+    kFBarXFree = 17,    // +X buffer: dV_i complete: the buffer may take S_{i + buffers}
+    kFBardQFull = 19,   // dQ_i complete
+    kFBarYFree = 20,    // count 128: dQ_i copied out: Y may take dP_{i+1}
+    kFBarFinal = 21,    // last dV and dK complete (one warp issues both)
+    kFBarDrain = 22,    // +issuer (3): abort path only
+};
+
+struct FusedParams {
+    const float* LSE;
+    const float* delta;
+    float* dq_acc;
+    int B, T, H;        // H = number of query heads
+    int G;              // query heads per key/value head; dK, dV sum over the G heads of a group
+    float scale, scale_log2;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kBwdFusedThreads, 1)
+moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+                      const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
+                      const __grid_constant__ CUtensorMap mapdK, const __grid_constant__ CUtensorMap mapdV,
+                      const FusedParams p) {
+    using L = FusedSmem<D>;
+    constexpr int NSUB = D / 64;
+    constexpr uint32_t kTmemCols = 512;
+    // d = 64 leaves room for a second S^T / P^T buffer: S_{i+1} is then computed while the row warps still work
+    // on tile i, instead of waiting for dV_i to release the only buffer.
+    constexpr int XB = (D == 64) ? 2 : 1;
+    constexpr uint32_t kColX = 0, kColY = 128 * XB, kColdK = kColY + 128, kColdV = kColdK + D;
+    static_assert(kColdV + D <= kTmemCols, "tensor-memory plan too large");
+
+    if (g_moda_status != 0) return;
+
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = aligned_dynamic_smem(smem_raw, L::kTotal);
+    if (smem == nullptr) {
+        if (threadIdx.x == 0) atomicCAS(&g_moda_status, 0, kStatusSmemLayout);
+        return;
+    }
+    const uint32_t sbase = smem_u32(smem);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 4);
+    auto bar = [&](int i) { return sbase + L::kBars + 8u * uint32_t(i); };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nk = num_tiles(p.T);
+    const int bh = blockIdx.x / nk;
+    const int kt = blockIdx.x % nk;                       // key tiles in ascending order: most work first
+    const int Hk = p.H / p.G;
+    const int b = bh / Hk, h = bh % Hk;                   // h: key/value head of this CTA
+    const int k0 = kt * kTileRows;
+    const int n_per = nk - kt;                            // query tiles kt .. nk-1 see this key tile
+    const int n_it = n_per * p.G;                         // iteration it: query head h G + it / n_per, tile kt + it % n_per
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(kFBarKV), 1);
+        for (int s = 0; s < L::kStages; ++s) {
+            mbar_init(bar(kFBarQFull + s), 32);
+            mbar_init(bar(kFBarQEmpty + s), 1);
+        }
+        for (int s = 0; s < L::kdOStages; ++s) {
+            mbar_init(bar(kFBardOFull + s), 1);
+            mbar_init(bar(kFBardOEmpty + s), 2);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(kFBarSFull + s), 1);
+            mbar_init(bar(kFBarPFull + s), 256);
+            mbar_init(bar(kFBarXFree + s), 1);
+        }
+        mbar_init(bar(kFBardPFull), 1);
+        mbar_init(bar(kFBardSFull), 256);
+        mbar_init(bar(kFBardQFull), 1);
+        mbar_init(bar(kFBarYFree), 128);
+        mbar_init(bar(kFBarFinal), 1);
+        for (int s = 0; s < 3; ++s) mbar_init(bar(kFBarDrain + s), 1);
+        fence_mbar_init();
+    }
+    if (warp == 13) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    // Abort path of an issuing thread: wait (bounded) until its own MMAs have drained.
+    auto drain_on_abort = [&](int which) {
+        if (*abort_flag != 0) {
+            umma_commit(bar(kFBarDrain + which));
+            const uint64_t t0 = globaltimer_ns();
+            while (!mbar_try_wait(bar(kFBarDrain + which), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+        }
+    };
+
+    // Register budget: the CTA owns what it was launched with, 512 threads x 128 registers, and
+    // setmaxnreg.inc blocks until the CTA's own pool can serve it, so the three shares must fit that total.
+    constexpr int kRegsRow = (D == 128) ? 136 : 152, kRegsDrain = (D == 128) ? 160 : 152, kRegsOther = (D == 128) ? 80 : 56;
+    static_assert(256 * kRegsRow + 128 * kRegsDrain + 128 * kRegsOther <= kBwdFusedThreads * 128, "register shares exceed the CTA's pool");
+    if (warp < 8) {
+        // =========================== row warps: P^T, dS^T, dK / dV epilogue ===========================
+        setmaxnreg_inc<kRegsRow>();
+        const int hc = warp >> 2;                            // which 64 query columns of every iteration
+        const int r = tid & 127;                             // key row inside the tile = TMEM lane
+        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+        const uint32_t tX0 = tmem + lane_addr + kColX + hc * 64;
+        const uint32_t tY = tmem + lane_addr + kColY + hc * 64;
+        uint8_t* ds_row = smem + L::kdS + hc * L::kSubBytes + r * 128;   // this thread's 128-byte row of dS^T
+        for (int it = 0; it < n_it; ++it) {
+            const int st = it % L::kStages;
+            const bool diag = (it % n_per) == 0;             // the query tile is the key tile itself: causal mask
+            const float* rt = reinterpret_cast<const float*>(smem + L::kRow + st * L::kRowBytes) + hc * 64;
+            uint32_t pk[32];                                 // P_i^T of this thread: 64 values, bf16 pairs
+            // ---- P_i^T ----
+            const int xb = it % XB;
+            const uint32_t tX = tX0 + xb * 128;
+            mbar_wait(bar(kFBarSFull + xb), (it / XB) & 1, abort_flag, 121);
+            tc_fence_after_sync();
+            {
+                // both halves are requested before the first is used: the second load's latency hides under the
+                // first half's exponentials
+                uint32_t sv[64];
+                tmem_ld32(tX, *reinterpret_cast<uint32_t(*)[32]>(sv));
+                tmem_ld32(tX + 32, *reinterpret_cast<uint32_t(*)[32]>(sv + 32));
+                tmem_wait_ld();
+#pragma unroll
+                for (int i4 = 0; i4 < 16; ++i4) {
+                    const float4 nl = *reinterpret_cast<const float4*>(rt + 4 * i4);     // same address for all rows
+                    float e0 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 0]), p.scale_log2, nl.x));
+                    float e1 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 1]), p.scale_log2, nl.y));
+                    float e2 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 2]), p.scale_log2, nl.z));
+                    float e3 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 3]), p.scale_log2, nl.w));
+                    if (diag) {                               // query column c sees key row r iff c >= r
+                        const int c = hc * 64 + 4 * i4;
+                        if (c + 0 < r) e0 = 0.f;
+                        if (c + 1 < r) e1 = 0.f;
+                        if (c + 2 < r) e2 = 0.f;
+                        if (c + 3 < r) e3 = 0.f;
+                    }
+                    pk[2 * i4] = pack_bf16x2(e0, e1);
+                    pk[2 * i4 + 1] = pack_bf16x2(e2, e3);
+                }
+            }
+            // P^T (bf16, two per column) overlays the first 32 of the 64 columns this thread has read
+            tmem_st32(tX, pk);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(bar(kFBarPFull + xb));
+
+            // ---- dS_i^T = P o (dP - D), with the bf16 P that dV uses ----
+            mbar_wait(bar(kFBardPFull), it & 1, abort_flag, 122);
+            tc_fence_after_sync();
+            // the dS buffer is still read by dQ_{i-1} and dK_{i-1} (dK is issued last: its completion covers both)
+            if (it > 0) mbar_wait(bar(kFBarQEmpty + (it - 1) % L::kStages), ((it - 1) / L::kStages) & 1, abort_flag, 123);
+            {
+                uint32_t gv[64];
+                tmem_ld32(tY, *reinterpret_cast<uint32_t(*)[32]>(gv));
+                tmem_ld32(tY + 32, *reinterpret_cast<uint32_t(*)[32]>(gv + 32));
+                tmem_wait_ld();
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {                // 8 query columns = one 16-byte chunk of the row
+                    const float4 da = *reinterpret_cast<const float4*>(rt + kTileRows + 8 * g);
+                    const float4 db = *reinterpret_cast<const float4*>(rt + kTileRows + 8 * g + 4);
+                    const uint32_t* pp = pk + 4 * g;
+                    uint4 v;
+                    v.x = pack_bf16x2(bf16_lo_to_f32(pp[0]) * (__uint_as_float(gv[8 * g + 0]) - da.x),
+                                      bf16_hi_to_f32(pp[0]) * (__uint_as_float(gv[8 * g + 1]) - da.y));
+                    v.y = pack_bf16x2(bf16_lo_to_f32(pp[1]) * (__uint_as_float(gv[8 * g + 2]) - da.z),
+                                      bf16_hi_to_f32(pp[1]) * (__uint_as_float(gv[8 * g + 3]) - da.w));
+                    v.z = pack_bf16x2(bf16_lo_to_f32(pp[2]) * (__uint_as_float(gv[8 * g + 4]) - db.x),
+                                      bf16_hi_to_f32(pp[2]) * (__uint_as_float(gv[8 * g + 5]) - db.y));
+                    v.w = pack_bf16x2(bf16_lo_to_f32(pp[3]) * (__uint_as_float(gv[8 * g + 6]) - db.z),
+                                      bf16_hi_to_f32(pp[3]) * (__uint_as_float(gv[8 * g + 7]) - db.w));
+                    *reinterpret_cast<uint4*>(ds_row + ((g ^ (r & 7)) << 4)) = v;
+                }
+            }
+            fence_proxy_async_smem();                        // generic-proxy stores -> read by the MMAs (async proxy)
+            tc_fence_before_sync();
+            mbar_arrive(bar(kFBardSFull));
+        }
+
+        // ---- epilogue: dK (scaled) by the first warpgroup, dV by the second ----
+        mbar_wait(bar(kFBarFinal), 0, abort_flag, 124);
+        tc_fence_after_sync();
+        {
+            const float mul = hc == 0 ? p.scale : 1.f;
+            const uint32_t col = hc == 0 ? kColdK : kColdV;
+            const int dst_off = hc == 0 ? L::kQ : L::kdO;    // every MMA has completed: the stages are free
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tmem + lane_addr + col + c * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int g4 = 0; g4 < 4; ++g4) {
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(o[8 * g4 + 0]) * mul, __uint_as_float(o[8 * g4 + 1]) * mul);
+                    v.y = pack_bf16x2(__uint_as_float(o[8 * g4 + 2]) * mul, __uint_as_float(o[8 * g4 + 3]) * mul);
+                    v.z = pack_bf16x2(__uint_as_float(o[8 * g4 + 4]) * mul, __uint_as_float(o[8 * g4 + 5]) * mul);
+                    v.w = pack_bf16x2(__uint_as_float(o[8 * g4 + 6]) * mul, __uint_as_float(o[8 * g4 + 7]) * mul);
+                    *reinterpret_cast<uint4*>(smem + dst_off + swz_chunk_offset(r, c * 4 + g4)) = v;
+                }
+            }
+        }
+        fence_proxy_async_smem();
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (tid == 0) {
+#pragma unroll
+            for (int s = 0; s < NSUB; ++s) {
+                tma_store_4d(&mapdK, sbase + L::kQ + s * L::kSubBytes, s * 64, h, k0, b);
+                tma_store_4d(&mapdV, sbase + L::kdO + s * L::kSubBytes, s * 64, h, k0, b);
+            }
+            tma_store_commit();
+            tma_store_wait_all();
+        }
+    } else if (warp < 12) {
+        // =========================== drain warps: dQ tile -> fp32 accumulator ===========================
+        // The tile leaves the SM as bulk reductions (cp.reduce.async.bulk, fp32 add in L2) from a staging buffer
+        // in shared memory.  Per-thread red.global instructions would do the same additions, but they queue in the
+        // load/store path of the SM at the pace L2 takes them, and every shared-memory load, store and barrier probe of
+        // the row warps then waits behind them (measured: + 2000 cycles per iteration).
+        setmaxnreg_inc<kRegsDrain>();
+        const int r = tid & 127;                             // query row inside the tile = TMEM lane
+        const uint32_t tY = tmem + (uint32_t((warp & 3) * 32) << 16) + kColY;
+        float4* stg = reinterpret_cast<float4*>(smem + L::kStg) + r;          // [feature / 4 (16)][row 128] float4
+        for (int it = 0; it < n_it; ++it) {
+            const int hq = h * p.G + it / n_per;
+            const int qi = kt + it % n_per;
+            float* dst = p.dq_acc + ((size_t(b) * p.H + hq) * nk + qi) * (size_t(kTileRows) * D);
+            mbar_wait(bar(kFBardQFull), it & 1, abort_flag, 120);
+            tc_fence_after_sync();
+            uint32_t o[D];
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) tmem_ld32(tY + c * 32, *reinterpret_cast<uint32_t(*)[32]>(o + c * 32));
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            mbar_arrive(bar(kFBarYFree));                    // Y may take dP of the next iteration
+#pragma unroll
+            for (int rd = 0; rd < D / 64; ++rd) {            // 64 feature columns (32 KiB) per round
+                // the previous round's reduction has finished reading the staging buffer
+                if (tid == 256) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+#pragma unroll
+                for (int g = 0; g < 16; ++g)
+                    stg[g * kTileRows] = make_float4(__uint_as_float(o[rd * 64 + 4 * g]), __uint_as_float(o[rd * 64 + 4 * g + 1]),
+                                                     __uint_as_float(o[rd * 64 + 4 * g + 2]), __uint_as_float(o[rd * 64 + 4 * g + 3]));
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                if (tid == 256) {
+                    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
+                                 ::"l"(dst + rd * (64 * kTileRows)), "r"(sbase + L::kStg), "r"(L::kStgBytes) : "memory");
+                    tma_store_commit();
+                }
+            }
+        }
+        if (tid == 256) tma_store_wait_all();                // every addition has been performed before the CTA retires
+    } else if (warp < 16) {
+      setmaxnreg_dec<kRegsOther>();
+      if (warp == 12) {
+        // =========================== loader: TMA tiles + per-query LSE, D_t ===========================
+        if (lane == 0) {
+            tma_prefetch_desc(&mapK);
+            tma_prefetch_desc(&mapV);
+            tma_prefetch_desc(&mapQ);
+            tma_prefetch_desc(&mapdO);
+            mbar_arrive_expect_tx(bar(kFBarKV), 2 * L::kTileBytes);
+#pragma unroll
+            for (int s = 0; s < NSUB; ++s) {
+                tma_load_4d(sbase + L::kK + s * L::kSubBytes, &mapK, bar(kFBarKV), s * 64, h, k0, b);
+                tma_load_4d(sbase + L::kV + s * L::kSubBytes, &mapV, bar(kFBarKV), s * 64, h, k0, b);
+            }
+        }
+        for (int it = 0; it < n_it; ++it) {
+            const int st = it % L::kStages;
+            const int hq = h * p.G + it / n_per;
+            const size_t row_base = (size_t(b) * p.H + hq) * p.T;
+            const int qrow0 = (kt + it % n_per) * kTileRows;
+            // lane handles query columns 4 lane .. 4 lane + 3; queries past T get -LSE = -inf so that P = 0
+            float4 nl, dl;
+            {
+                const int c = qrow0 + 4 * lane;
+                nl.x = (c + 0 < p.T) ? -p.LSE[row_base + c + 0] * kLog2e : -INFINITY;
+                nl.y = (c + 1 < p.T) ? -p.LSE[row_base + c + 1] * kLog2e : -INFINITY;
+                nl.z = (c + 2 < p.T) ? -p.LSE[row_base + c + 2] * kLog2e : -INFINITY;
+                nl.w = (c + 3 < p.T) ? -p.LSE[row_base + c + 3] * kLog2e : -INFINITY;
+                dl.x = (c + 0 < p.T) ? p.delta[row_base + c + 0] : 0.f;
+                dl.y = (c + 1 < p.T) ? p.delta[row_base + c + 1] : 0.f;
+                dl.z = (c + 2 < p.T) ? p.delta[row_base + c + 2] : 0.f;
+                dl.w = (c + 3 < p.T) ? p.delta[row_base + c + 3] : 0.f;
+            }
+            if (it >= L::kStages) mbar_wait(bar(kFBarQEmpty + st), ((it - L::kStages) / L::kStages) & 1, abort_flag, 130);
+            float4* rt = reinterpret_cast<float4*>(smem + L::kRow + st * L::kRowBytes);
+            rt[lane] = nl;
+            rt[kTileRows / 4 + lane] = dl;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(bar(kFBarQFull + st), L::kTileBytes);
+#pragma unroll
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_4d(sbase + L::kQ + st * L::kTileBytes + s * L::kSubBytes, &mapQ, bar(kFBarQFull + st), s * 64, hq, qrow0, b);
+                const int dst = it % L::kdOStages;
+                if (it >= L::kdOStages) mbar_wait(bar(kFBardOEmpty + dst), ((it - L::kdOStages) / L::kdOStages) & 1, abort_flag, 131);
+                mbar_arrive_expect_tx(bar(kFBardOFull + dst), L::kTileBytes);
+#pragma unroll
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_4d(sbase + L::kdO + dst * L::kTileBytes + s * L::kSubBytes, &mapdO, bar(kFBardOFull + dst), s * 64, hq, qrow0, b);
+            } else {
+                mbar_arrive(bar(kFBarQFull + st));
+            }
+        }
+      } else if (warp == 13 || warp == 14) {
+        // ============ MMA issuers: S^T = K Q^T (warp 13, into X), dP^T = V dO^T (warp 14, into Y) ============
+        {   // whole warp: operands are warp-uniform, one elected lane issues
+            const bool is_s = (warp == 13);
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
+            const uint32_t a_tile = sbase + (is_s ? L::kK : L::kV);
+            const int full0 = is_s ? kFBarQFull : kFBardOFull;
+            const int nb = is_s ? XB : 1;                                 // accumulator buffers of this contraction
+            // a descriptor of a later k-step is the first one plus a compile-time constant (the start-address field
+            // counts 16-byte units and stays inside its 14 bits below 256 KiB)
+            const uint64_t da0 = desc_kmajor_sw128(a_tile, 0);
+            const uint64_t db0 = desc_kmajor_sw128(sbase + (is_s ? L::kQ : L::kdO), 0);
+            mbar_wait(bar(kFBarKV), 0, abort_flag, 140);
+            const int nst = is_s ? L::kStages : L::kdOStages;
+            for (int it = 0; it < n_it; ++it) {
+                const int st = it % nst;
+                // the accumulator buffer still holds P of its previous tile (until that dV completes) / dQ_{i-1} (until
+                // it is copied out)
+                const int xb = it % nb;
+                const uint32_t col = is_s ? kColX + xb * 128 : kColY;
+                const uint32_t free_bar = is_s ? bar(kFBarXFree + xb) : bar(kFBarYFree);
+                if (it >= nb) mbar_wait2(bar(full0 + st), (it / nst) & 1, free_bar, ((it - nb) / nb) & 1, abort_flag, 141, is_s ? 142 : 143);
+                else mbar_wait(bar(full0 + st), (it / nst) & 1, abort_flag, 141);
+                tc_fence_after_sync();
+                const uint64_t db = db0 + uint64_t((st * L::kTileBytes) >> 4);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk)
+                    umma_ss(tmem + col, da0 + uint64_t(((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4),
+                            db + uint64_t(((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4), idesc_s, kk > 0);
+                umma_commit(bar(is_s ? kFBarSFull + xb : kFBardPFull));
+                if (!is_s) umma_commit(bar(kFBardOEmpty + st));
+            }
+            drain_on_abort(is_s ? 0 : 1);
+        }
+      } else {
+        // ============ MMA issuer (warp 15): dV_i += P^T dO (P^T from tensor memory, dO MN-major), then, once dS_i^T
+        // ============ is in shared memory, dQ_tile = dS K into Y (dS^T and K both MN-major) and dK += dS^T Q (dS^T
+        // ============ K-major, Q MN-major).  P_i, dS_i, P_{i+1} are produced in this order, so one warp can take the
+        // ============ three in turn.  dQ before dK: its tile has to be copied out before dP of the next iteration can
+        // ============ land, dK only has to finish before dS_{i+1} is written.
+        {
+            constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
+            constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);
+            const uint64_t dvb0 = desc_mnmajor_sw128(sbase + L::kdO, 0, L::kSubBytes);
+            const uint64_t dqa0 = desc_mnmajor_sw128(sbase + L::kdS, 0, L::kSubBytes);
+            const uint64_t dqb0 = desc_mnmajor_sw128(sbase + L::kK, 0, L::kSubBytes);
+            const uint64_t dka0 = desc_kmajor_sw128(sbase + L::kdS, 0);
+            const uint64_t dkb0 = desc_mnmajor_sw128(sbase + L::kQ, 0, L::kSubBytes);
+            for (int it = 0; it < n_it; ++it) {
+                const int st = it % L::kStages, dst = it % L::kdOStages, xb = it % XB;
+                mbar_wait2(bar(kFBarPFull + xb), (it / XB) & 1, bar(kFBardOFull + dst), (it / L::kdOStages) & 1, abort_flag, 144, 145);
+                tc_fence_after_sync();
+                const uint64_t dvb = dvb0 + uint64_t((dst * L::kTileBytes) >> 4);
+#pragma unroll
+                for (int kk = 0; kk < kTileRows / 16; ++kk)  // 16 queries per k-step: 8 columns, in the block of warpgroup kk / 4
+                    umma_ts(tmem + kColdV, tmem + kColX + xb * 128 + (kk >> 2) * 64 + (kk & 3) * 8, dvb + uint64_t(kk * 128), idesc_acc,
+                            (it > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(bar(kFBarXFree + xb));
+                umma_commit(bar(kFBardOEmpty + dst));
+                mbar_wait(bar(kFBardSFull), it & 1, abort_flag, 146);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < kTileRows / 16; ++kk)
+                    umma_ss(tmem + kColY, dqa0 + uint64_t(kk * 128), dqb0 + uint64_t(kk * 128), idesc_dq, kk > 0);
+                umma_commit(bar(kFBardQFull));
+                const uint64_t dkb = dkb0 + uint64_t((st * L::kTileBytes) >> 4);
+#pragma unroll
+                for (int kk = 0; kk < kTileRows / 16; ++kk)
+                    umma_ss(tmem + kColdK, dka0 + uint64_t(((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4), dkb + uint64_t(kk * 128),
+                            idesc_acc, (it > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(bar(kFBarQEmpty + st));
+            }
+            umma_commit(bar(kFBarFinal));
+            drain_on_abort(2);
+        }
+      }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag != 0 && tid == 256) {
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) {}
+    }
+    __syncthreads();
+    if (warp == 13) tmem_dealloc(tmem, kTmemCols);
+}
+
+}  // namespace moda

@@ -17,6 +17,10 @@ namespace moda {
 // host reads it with moda_last_status().  0 = no error.
 // ------------------------------------------------------------------------------------
 __device__ int g_moda_status = 0;
+// Mirror of the status word in host memory that the device can write (set up by the host on its first
+// call on a device; null until then).  Written only when a wait runs out, so that the next host call
+// can see the failure with a plain load instead of a device synchronisation.
+__device__ int* g_moda_status_host = nullptr;
 
 enum : int {
     kStatusOk = 0,
@@ -88,16 +92,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  `abort_flag` is a CTA-wide word in shared memory: once any waiter of the
 // CTA has timed out, every later wait returns at once so that the CTA can reach its
 // tear-down (TMEM release) instead of spinning.  Limit: ~1 s of wall time.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int site) {
+__device__ __forceinline__ void report_wait_timeout(int site) {
+    const int code = kStatusWaitTimeout | (site << 8);
+    if (atomicCAS(&g_moda_status, 0, code) == 0) {
+        int* host = g_moda_status_host;
+        if (host != nullptr) {
+            *reinterpret_cast<volatile int*>(host) = code;
+            __threadfence_system();
+        }
+    }
+}
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int site,
+                                          uint64_t limit_ns = 1000000000ull) {
     if (mbar_try_wait(bar, parity)) return;
     const uint64_t t0 = globaltimer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0xffu) == 0) {
             if (*abort_flag != 0) return;
-            if (globaltimer_ns() - t0 > 1000000000ull) {
+            if (globaltimer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
-                atomicCAS(&g_moda_status, 0, kStatusWaitTimeout | (site << 8));
+                report_wait_timeout(site);
                 return;
             }
         }

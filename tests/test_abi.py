@@ -71,8 +71,12 @@ def test_argument_validation_rejects_before_any_launch():
     assert lib.moda_attn_bwd(*args, None, ctypes.c_size_t(1 << 20), None) == -7
     assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 0, None) == -3
     assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 8, None) == -3      # accumulate bit without a stage
-    assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 16, None) == -3
-    assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 7 | 16, None) == -3
+    assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 16, None) == -3     # form bit without a stage
+    assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 32, None) == -3
+    assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(1 << 20), 7 | 32, None) == -3
+    # the fused form needs the fp32 dQ accumulator, the reproducible split form only the row terms
+    assert lib.moda_attn_bwd_stages(*args, p, ctypes.c_size_t(4096), 7, None) == -7
+    assert moda.moda_bwd_workspace_bytes(1, 128, 1, 64, 0) >= 128 * 4 + 128 * 64 * 4
     # grouped-query entry points: H_kv must divide H; 1 to 8, 16 or 32 query heads per group
     gqa = lambda H, Hk: lib.moda_attn_fwd_gqa(p, p, p, None, 1, 128, H, Hk, 64, 0, ctypes.c_float(0.125), p, p, None)
     assert gqa(6, 4) == -12 and gqa(4, 0) == -12 and gqa(12, 1) == -12 and gqa(64, 1) == -12

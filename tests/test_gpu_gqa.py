@@ -11,8 +11,8 @@ import paper_2603_15619_b200 as moda
 from paper_2603_15619_b200 import synthetic
 from oracle import moda_oracle as orc
 
-from parity import (TOL_GRAD_REL_L2, TOL_LSE_ABS, TOL_O_MAX_ABS, TOL_O_REL_L2, build_cache, f64, rel_l2,
-                    unpack_cache)
+from parity import (TOL_GRAD_REL_L2, TOL_LSE_ABS, TOL_O_MAX_ABS, TOL_O_REL_L2, assert_same_gradients, build_cache, f64,
+                    rel_l2, unpack_cache)
 
 pytestmark = pytest.mark.gpu
 
@@ -80,6 +80,10 @@ def test_one_head_per_group_is_bitwise_the_plain_entry_points():
     assert torch.equal(O, O2) and torch.equal(LSE, LSE2)
     a = moda.moda_attn_bwd(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, w.scale)
     b = moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, w.scale)
+    assert_same_gradients(a, b, "plain and grouped entry points")
+    det = moda.MODA_BWD_ALL_STAGES | moda.MODA_BWD_DETERMINISTIC
+    a = moda.moda_attn_bwd(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, w.scale, stages=det)
+    b = moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, w.scale, stages=det)
     for s, t in zip(a, b):
         assert torch.equal(s, t)
 

@@ -8,7 +8,7 @@ import paper_2603_15619_b200 as moda
 from paper_2603_15619_b200 import synthetic
 from oracle import moda_oracle as orc
 
-from parity import TOL_GRAD_REL_L2, TOL_O_REL_L2, f64, rel_l2
+from parity import TOL_GRAD_REL_L2, TOL_O_REL_L2, assert_same_gradients, f64, rel_l2
 
 pytestmark = pytest.mark.gpu
 
@@ -70,8 +70,7 @@ def test_accumulate_flag_adds_the_depth_gradients_to_what_the_cache_holds(B, T, 
     out = moda.moda_attn_bwd_gqa(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale, d_depth_kv=acc,
                                  stages=moda.MODA_BWD_ALL_STAGES | moda.MODA_BWD_ACCUMULATE_DEPTH)
     assert moda.moda_last_status() == 0
-    for a, b in zip(out[:3], plain[:3]):
-        assert torch.equal(a, b)
+    assert_same_gradients(out[:3], plain[:3], "with and without the accumulate flag")
     want = (old.double() + plain[3].double())
     got = acc.double()
     if H // Hk <= 8:

@@ -76,3 +76,16 @@ def test_reference_arm_prints_on_rank_zero_only():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["gpu_launches"] == 0
     assert outs[1] == "", "ranks other than 0 print nothing"
+
+
+def test_gpus_flag_outside_a_launcher_spawns_the_ranks_itself():
+    # `python bench.py --gpus 2` with no WORLD_SIZE in the environment must mean two ranks, not one: the script
+    # starts them on 127.0.0.1 and rank 0 alone prints the line (the oracle arm runs without a GPU).
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c1", "--gpus", "2",
+           "--steps", "1", "--warmup", "0"]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-400:]
+    lines = [l for l in r.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1, lines
+    assert json.loads(lines[0])["n_gpus"] == 2

@@ -3,15 +3,23 @@
 
 A "step" is one pass of the whole hot path for one attention layer over one batch of
 synthetic inputs that are already resident in HBM: the depth-cache "write" of the layer's
-own K, V (one slot), the forward kernel, and the three backward launches (row terms,
-dQ + depth gradients, dK/dV).  `value` is forward+backward TFLOP/s with the FLOP convention
-of paper_2603_15619_b200/flops.py (causal-halved sequence part + depth part, backward =
-2.5 x forward).  Default workload: c2 (B=4, T=4096, H=16, d=128, l=23).
+own K, V (one slot), the forward kernel, and the three backward launches (row-local part:
+row terms, depth gradients, depth share of dQ; sequence part: dK, dV and the dQ tiles; dQ
+finish).  `value` is forward+backward TFLOP/s with the FLOP convention of
+paper_2603_15619_b200/flops.py (causal-halved sequence part + depth part, backward =
+2.5 x forward).  Default workload: c4 (B=1, T=65536, H=16, d=128, l=24), the largest
+configured workload at d = 128 and the one the 64K ratio target is stated on.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl moda|reference]
+`roofline.targets` carries the numbers the targets are stated on: forward % of the measured
+burst bf16 peak at T = 8192 for the six depths of c3, at c4 and at c5, and the ratio of the
+MoDA kernels to the same kernels with l = 0 at c4.  Sweep rows go to stderr.
 
-For N > 1 launch with torch.distributed.run; every rank runs the same workload on its own
-GPU (independent batch shards, no collective on the data path: weak scaling).
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl moda|reference]
+                    [--sweeps gqa,decode,prefill]
+
+For N > 1 launch with torch.distributed.run, or let `--gpus N` spawn N local ranks itself;
+every rank runs the same workload on its own GPU (independent batch shards, no collective
+on the data path: weak scaling).
 """
 from __future__ import annotations
 
@@ -31,17 +39,21 @@ sys.path.insert(0, ROOT)
 
 from paper_2603_15619_b200 import flops, synthetic  # noqa: E402
 
-METRIC = "MoDA fwd+bwd TFLOP/s (fwd and % of B200 BF16 peak in `detail`; ratio to own l=0 kernel in `sweep`)"
+METRIC = "MoDA fwd+bwd TFLOP/s (fwd and % of B200 BF16 peak vs T, ratio to own l=0 kernel: roofline.targets)"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes); keyed by (workload, kernel).  None where no capture exists.
+NCU_SEQ_C3_L0_B1 = 202.80e6 + 100.59e6   # dram__bytes_read.sum + dram__bytes_write.sum of that one launch
 NCU_TRAFFIC_BYTES = {
     # c2 captured at B=1 and scaled x4 (traffic is proportional to B): profiles/ncu_full_c2_B1_fwd_bwd_kernels.md
     ("c2", "fwd"): 4 * (822.179e6 + 6.956e6),
-    ("c2", "bwd_dq_depth"): 4 * (845.105e6 + 735.033e6),
-    ("c2", "bwd_dkdv"): 4 * (67.678e6 + 8.945e6),
+    # sequence part of the backward, captured at c3 with l = 0 and B = 1 (T = 8192) and scaled by the number of
+    # elements B T H d (every tensor crosses HBM once, re-reads are served by L2):
+    # profiles/ncu_full_c3_l0_B1_bwd_fused_kernel.md
+    ("c4", "bwd_seq"): 8 * NCU_SEQ_C3_L0_B1,
+    ("c3_l0", "bwd_seq"): 2 * NCU_SEQ_C3_L0_B1,
 }
 
 
@@ -144,27 +156,29 @@ def job_value(world: int, flops_per_rank_step: float, ms_per_step: float) -> flo
 class Layer:
     """Device buffers of one workload plus the calls of one step."""
 
-    KERNELS = ("cache_append", "fwd", "bwd_rowterms", "bwd_dq_depth", "bwd_dkdv")
+    KERNELS = ("cache_append", "fwd", "bwd_rows", "bwd_seq", "bwd_finish")
 
-    def __init__(self, w: synthetic.Workload, seed: int, device):
+    def __init__(self, w: synthetic.Workload, seed: int, device, with_backward: bool = True):
         import paper_2603_15619_b200 as moda
         self.moda, self.w = moda, w
         self.q = synthetic.tensor(w, "Q", seed, 0, device)
         self.k = synthetic.tensor(w, "K", seed, 0, device)
         self.v = synthetic.tensor(w, "V", seed, 0, device)
-        self.dO = synthetic.tensor(w, "dO", seed, 0, device)
         self.cache = self.dcache = None
         if w.l > 0:
             self.cache = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, w.l, device)
-            self.dcache = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, w.l, device)
             for i in range(w.l):
                 moda.moda_depth_cache_append(self.cache, i, synthetic.tensor(w, "Kd", seed, i, device),
                                              synthetic.tensor(w, "Vd", seed, i, device))
         self.next_slot = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, 1, device)   # slot this layer writes for later layers
         self.O = torch.empty_like(self.q)
         self.LSE = torch.empty((w.B, w.H, w.T), dtype=torch.float32, device=device)
-        self.dQ, self.dK, self.dV = (torch.empty_like(self.q) for _ in range(3))
-        self.ws = torch.empty(moda.moda_bwd_workspace_bytes(w.B, w.T, w.H, w.d, w.l), dtype=torch.uint8, device=device)
+        if with_backward:
+            self.dO = synthetic.tensor(w, "dO", seed, 0, device)
+            if w.l > 0:
+                self.dcache = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, w.l, device)
+            self.dQ, self.dK, self.dV = (torch.empty_like(self.q) for _ in range(3))
+            self.ws = torch.empty(moda.moda_bwd_workspace_bytes(w.B, w.T, w.H, w.d, w.l), dtype=torch.uint8, device=device)
 
     def append(self):
         self.moda.moda_depth_cache_append(self.next_slot, 0, self.k, self.v)
@@ -198,11 +212,11 @@ class Layer:
         return {
             "cache_append": {"bytes": 2.0 * 4 * E, "flops": 0.0},
             "fwd": {"bytes": flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l), "flops": f_fwd},
-            "bwd_rowterms": {"bytes": 2.0 * 2 * E + 4.0 * rows, "flops": 2.0 * E},
-            # reads Q dO K V + depth cache + LSE, D; writes dQ + depth gradients; 3 of the 5 backward contractions
-            "bwd_dq_depth": {"bytes": 2.0 * (5 * E + 4 * w.l * E) + 8.0 * rows, "flops": 1.5 * seq + 2.5 * dep},
-            # reads Q K V dO + LSE, D; writes dK dV; 4 contractions in the split formulation (2 recomputed)
-            "bwd_dkdv": {"bytes": 2.0 * 6 * E + 8.0 * rows, "flops": 2.0 * seq},
+            # reads Q O dO (bf16), LSE and the depth cache; writes the row terms, the depth gradients and the fp32 dQ accumulator
+            "bwd_rows": {"bytes": 2.0 * (3 * E + 4 * w.l * E) + 4.0 * E + 8.0 * rows, "flops": 2.0 * E + 2.5 * dep},
+            # reads Q K V dO + LSE, D; writes dK dV; reads and writes the fp32 dQ accumulator; the five sequence contractions
+            "bwd_seq": {"bytes": 2.0 * 6 * E + 2 * 4.0 * E + 8.0 * rows, "flops": 2.5 * seq},
+            "bwd_finish": {"bytes": 4.0 * E + 2.0 * E, "flops": 0.0},
         }
 
 
@@ -226,7 +240,8 @@ def run_moda(args, rank, world, device):
         if world > 1:
             torch.distributed.barrier()
 
-    for _ in range(max(args.warmup, 3)):
+    W = max(args.warmup, 3)
+    for _ in range(W):
         layer.step()
     torch.cuda.synchronize()
     if moda.moda_last_status() != 0:
@@ -263,7 +278,7 @@ def run_moda(args, rank, world, device):
     model = layer.kernel_model()
     dom = max(per_kernel, key=per_kernel.get)
     dur = per_kernel[dom] * 1e-3
-    long_region = (t_end - t_begin) > 1.0
+    long_region = (t_end - t_begin) > 1.0        # a kernel timed inside a seconds-long step runs under the power cap
     tensor_peak = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
     t_hbm = model[dom]["bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_tensor = model[dom]["flops"] / (tensor_peak * 1e12)
@@ -273,48 +288,60 @@ def run_moda(args, rank, world, device):
         roof = {"bound": "tensor", "achieved": model[dom]["flops"] / dur / 1e12, "peak": tensor_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((w.name, dom))
-    roof.update({"kernel": dom, "kernel_ms": per_kernel[dom], "peak_source": peaks["source"],
+    mhz = clocks.get("sm_mhz")
+    roof.update({"kernel": dom, "kernel_ms": round(per_kernel[dom], 4), "peak_source": peaks["source"],
                  "peak_kind": ("sustained" if long_region else "burst") if roof["bound"] == "tensor" else "copy",
-                 "algorithmic_bytes": model[dom]["bytes"], "algorithmic_flops": model[dom]["flops"]})
+                 "algorithmic_bytes": model[dom]["bytes"], "algorithmic_flops": model[dom]["flops"],
+                 "kernel_ms_x_sm_mhz": None if mhz is None else round(per_kernel[dom] * mhz, 1)})
 
     fwd_tflops = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l) / (per_kernel["fwd"] * 1e-3) / 1e12
-    bwd_ms = per_kernel["bwd_rowterms"] + per_kernel["bwd_dq_depth"] + per_kernel["bwd_dkdv"]
+    bwd_ms = per_kernel["bwd_rows"] + per_kernel["bwd_seq"] + per_kernel["bwd_finish"]
     detail = {
         "kernel_ms": {k: round(v, 4) for k, v in per_kernel.items()},
         "fwd_tflops": round(fwd_tflops, 1),
         "bwd_tflops": round(flops.bwd_flops(w.B, w.T, w.H, w.d, w.l) / (bwd_ms * 1e-3) / 1e12, 1),
+        "bwd_over_fwd_time": round(bwd_ms / per_kernel["fwd"], 3),
         "fwd_frac_of_measured_burst_bf16": round(fwd_tflops / peaks["bf16_tflops"], 4),
         "fwd_frac_of_measured_sustained_bf16": round(fwd_tflops / peaks["bf16_tflops_sustained"], 4),
         "fwd_frac_of_nominal_bf16": round(fwd_tflops / NOMINAL_BF16_TFLOPS, 4),
         "fwd_depth_read_gbs": round(flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / (per_kernel["fwd"] * 1e-3) / 1e9, 1),
+        "ms_per_step_x_sm_mhz": None if mhz is None else round(ms_per_step * mhz, 1),
         "flop_convention": "fwd = 4BHd T^2/2 + 4BHTld; bwd = 2.5 x fwd; step = 3.5 x fwd",
     }
 
     out = {
-        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{w.name}: B={w.B} T={w.T} H={w.H} d={w.d} l={w.l} (per GPU), bf16 N(0,1) inputs, fp32 accumulate",
-                   "step": "depth-cache append of one slot + forward + backward (row terms, dQ+depth grads, dK/dV)",
+                   "step": "depth-cache append of one slot + forward + backward (row-local part incl. depth gradients, "
+                           "sequence part dK/dV/dQ tiles, dQ finish)",
                    "l2_policy": "inputs larger than L2 (depth cache %.2f GiB + 4 x %.0f MiB activations per step)"
                                 % (flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / 2 ** 30, w.B * w.T * w.H * w.d * 2 / 2 ** 20),
                    "parallelism": f"independent batch shards x{world}, no collective"},
         "roofline": roof, "clocks": clocks, "gpu_launches": 5 * K, "detail": detail,
     }
 
-    if rank == 0 and world == 1 and not args.no_sweep:
-        out["sweep"] = run_sweep(peaks, device, layer)
-        out["gqa_sweep"] = run_gqa_sweep(device)
-        out["decode_sweep"] = run_decode_sweep(peaks, device)
-        out["prefill_sweep"] = run_prefill_sweep(peaks, device)
+    headline = {"fwd_ms": per_kernel["fwd"], "bwd_ms": bwd_ms}
     if not args.no_e2e:
-        out["e2e"] = run_e2e(layer, min(K, 8), world, step_flops, device)
+        out["e2e"] = run_e2e(layer, args.e2e_steps, world, step_flops, device)
+    del layer
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_sweep:
+        roof["targets"] = run_targets(peaks, device, w, headline)
+        extra = [x for x in args.sweeps.split(",") if x]
+        if "gqa" in extra:
+            out["gqa_sweep"] = run_gqa_sweep(device)
+        if "decode" in extra:
+            out["decode_sweep"] = run_decode_sweep(peaks, device)
+        if "prefill" in extra:
+            out["prefill_sweep"] = run_prefill_sweep(peaks, device)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, budget_s=20.0)
     return out
 
 
-def time_calls(fn, iters, warm=2):
+def time_calls(fn, iters, warm=3):
     for _ in range(warm):
         fn()
     torch.cuda.synchronize()
@@ -327,50 +354,49 @@ def time_calls(fn, iters, warm=2):
     return a.elapsed_time(b) / iters
 
 
-def run_sweep(peaks, device, first_layer):
-    """fwd / bwd time of every configured workload and of its l = 0 twin (same kernels, no depth slots)."""
-    rows = []
+def run_targets(peaks, device, headline_w, headline):
+    """The points the throughput targets are stated on, each timed alone (burst clocks) with its l = 0 twin:
+    forward % of the measured burst bf16 peak at T = 8192 for the six depths of c3, at c4 (T = 65536) and at c5
+    (T = 32768, d = 64); ratio of the MoDA kernels to the same kernels with l = 0 at c4 (forward, and forward +
+    backward).  Each row also says what bounds its forward: the slower of the algorithmic HBM bytes at the measured
+    copy rate and the credited FLOPs at the measured cuBLAS rate."""
     W = synthetic.WORKLOADS
-    plan = [("c2", W["c2"], 5)] + [(f"c3_l{l}", W["c3"].with_l(l), 5) for l in synthetic.C3_DEPTHS] + \
-           [("c4", W["c4"], 2), ("c5", W["c5"], 2)]
-    base_cache = {}
-    del first_layer
-    for name, w, iters in plan:
-        res = {}
-        for tag, ww in (("l0", w.with_l(0)), ("moda", w)):
-            key = (ww.B, ww.T, ww.H, ww.d, ww.l)
-            if key in base_cache:
-                res[tag] = base_cache[key]
-                continue
+    plan = [(f"c3_l{l}", W["c3"].with_l(l), 8, True) for l in synthetic.C3_DEPTHS] + \
+           [("c4", W["c4"], 3, True), ("c5", W["c5"], 3, True)]
+    timed = {}
+
+    def timings(ww, iters, bwd):
+        key = (ww.B, ww.T, ww.H, ww.d, ww.l)
+        if key not in timed:
             torch.cuda.empty_cache()
-            layer = Layer(ww, seed=0, device=device)
+            layer = Layer(ww, seed=0, device=device, with_backward=bwd)
             f_ms = time_calls(layer.fwd, iters)
-            b_ms = time_calls(layer.bwd, iters)
-            res[tag] = (f_ms, b_ms)
-            base_cache[key] = res[tag]
+            b_ms = time_calls(layer.bwd, iters) if bwd else None
+            timed[key] = (f_ms, b_ms)
             del layer
-        f_ms, b_ms = res["moda"]
-        f0, b0 = res["l0"]
+        return timed[key]
+
+    rows = {}
+    for name, w, iters, bwd in plan:
+        f_ms, b_ms = timings(w, iters, bwd)
+        f0, b0 = timings(w.with_l(0), iters, bwd)
         ff = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l)
-        # roofline of the call: the slower of (algorithmic HBM bytes / measured copy rate) and
-        # (credited FLOPs / measured cuBLAS bf16 rate; the burst figure, these kernels run alone)
-        roof = lambda fl, by: max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e3
-        roof_f = roof(ff, flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l))
-        roof_b = roof(2.5 * ff, flops.bwd_bytes(w.B, w.T, w.H, w.d, w.l))
-        rows.append({
-            "workload": name, "B": w.B, "T": w.T, "H": w.H, "d": w.d, "l": w.l,
-            "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
-            "fwd_tflops": round(ff / f_ms / 1e9, 1), "fwd_bwd_tflops": round(3.5 * ff / (f_ms + b_ms) / 1e9, 1),
-            "fwd_frac_measured_burst": round(ff / f_ms / 1e9 / peaks["bf16_tflops"], 4),
-            "fwd_frac_nominal": round(ff / f_ms / 1e9 / NOMINAL_BF16_TFLOPS, 4),
-            "fwd_depth_read_gbs": round(flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / f_ms / 1e6, 1),
-            "fwd_frac_of_roofline": round(roof_f / f_ms, 4), "bwd_frac_of_roofline": round(roof_b / b_ms, 4),
-            "fwd_bound": "hbm" if flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l) / (peaks["hbm_gbs"] * 1e9) >
-                         ff / (peaks["bf16_tflops"] * 1e12) else "tensor",
+        t_tensor = ff / (peaks["bf16_tflops"] * 1e12) * 1e3
+        t_hbm = flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l) / (peaks["hbm_gbs"] * 1e9) * 1e3
+        t_tensor_b = 2.5 * ff / (peaks["bf16_tflops"] * 1e12) * 1e3
+        t_hbm_b = flops.bwd_bytes(w.B, w.T, w.H, w.d, w.l) / (peaks["hbm_gbs"] * 1e9) * 1e3
+        rows[name] = {
+            "fwd_ms": round(f_ms, 4), "fwd_tflops": round(ff / f_ms / 1e9, 1),
+            "fwd_pct_of_burst_peak": round(100.0 * ff / f_ms / 1e9 / peaks["bf16_tflops"], 1),
+            "fwd_bound": "hbm" if t_hbm > t_tensor else "tensor",
+            "fwd_frac_of_roofline": round(max(t_tensor, t_hbm) / f_ms, 3),
+            "roofline_cap_pct_of_burst_peak": round(100.0 * t_tensor / max(t_tensor, t_hbm), 1),
+            "bwd_ms": round(b_ms, 4), "bwd_frac_of_roofline": round(max(t_tensor_b, t_hbm_b) / b_ms, 3),
+            "bwd_over_fwd_time": round(b_ms / f_ms, 2),
+            "fwd_ratio_to_l0": round(f0 / f_ms, 3), "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f_ms + b_ms), 3),
             "l0_fwd_ms": round(f0, 4), "l0_bwd_ms": round(b0, 4),
-            "fwd_ratio_to_l0": round(f0 / f_ms, 4), "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f_ms + b_ms), 4),
-        })
-        log("sweep", rows[-1])
+        }
+        log("target", name, rows[name])
     torch.cuda.empty_cache()
     return rows
 
@@ -523,7 +549,7 @@ def run_decode_sweep(peaks, device, shapes=None, iters=20):
                      "us_launched_from_host": round(ms_eager * 1e3, 1), "timed": "cuda graph replay" if ms is not ms_eager else "host launches",
                      "us_paged_64_host_launches": None if paged_us is None else round(paged_us, 1),
                      "algorithmic_GB": round(byt / 1e9, 3), "GBps": round(gbs, 0),
-                     "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 3),
+                     "ratio_to_measured_copy_rate": round(gbs / peaks["hbm_gbs"], 3),   # a read-only stream can beat a read+write copy
                      "tokens_per_s": round(B / ms * 1e3, 0)})
         log("decode_sweep", rows[-1])
         del sets, O, LSE, ws
@@ -621,43 +647,52 @@ def run_e2e(layer, steps, world, step_flops, device):
             "overlap": "upload of step i+1 and download of step i-1 run beside the kernels of step i (2 buffer sets, 3 streams)"}
 
 
-def cpu_sample(w, n_slices, seed=0):
-    """Complete (b, h) slices of workload `w` as float64 numpy arrays (heads are independent)."""
-    pick = [(i % w.B, (i * 7) % w.H) for i in range(n_slices)]
-    x = {n: synthetic.tensor(w, n, seed, 0, "cpu") for n in ("Q", "K", "V", "dO")}
-    sl = lambda t: torch.stack([t[b, :, h] for b, h in pick], dim=0).unsqueeze(2).double().numpy()   # [n,T,1,d]
-    out = {n: sl(t) for n, t in x.items()}
-    kd = [synthetic.tensor(w, "Kd", seed, i, "cpu") for i in range(w.l)]
-    vd = [synthetic.tensor(w, "Vd", seed, i, "cpu") for i in range(w.l)]
+def cpu_sample(w, T_sample, seed=0):
+    """One (b, h) slice of workload `w`, cut to its first `T_sample` positions, as float64 numpy arrays.  Heads are
+    independent and causal attention over a prefix is the operator on that prefix, so this is a bounded piece of the
+    same workload: same head width, depth, value recipe; drawn from the same seeded generators at the reduced shape."""
+    import dataclasses
     import numpy as np
-    out["Kd"] = np.stack([sl(t) for t in kd]) if w.l else np.zeros((0,) + out["Q"].shape)
-    out["Vd"] = np.stack([sl(t) for t in vd]) if w.l else np.zeros((0,) + out["Q"].shape)
-    return out, pick
+    ws = dataclasses.replace(w, B=1, H=1, T=int(T_sample), name=f"{w.name}/cpu-sample")
+    f64 = lambda t: t.double().numpy()
+    out = {n: f64(synthetic.tensor(ws, n, seed, 0, "cpu")) for n in ("Q", "K", "V", "dO")}
+    out["Kd"] = np.stack([f64(synthetic.tensor(ws, "Kd", seed, i, "cpu")) for i in range(w.l)]) if w.l else np.zeros((0,) + out["Q"].shape)
+    out["Vd"] = np.stack([f64(synthetic.tensor(ws, "Vd", seed, i, "cpu")) for i in range(w.l)]) if w.l else np.zeros((0,) + out["Q"].shape)
+    return out, ws
 
 
-def time_oracle(w, n_slices, sample=None):
-    """Seconds of one oracle forward + backward over `n_slices` complete (b, h) slices (the inputs are
-    generated outside the timed part; pass `sample` to reuse them)."""
+def time_oracle(sample):
+    """Seconds of one oracle forward + backward over the sample, the FLOPs it is credited with (same convention
+    as the GPU arm) and the threads it used."""
     from oracle import moda_oracle as orc
-    x, pick = sample if sample is not None else cpu_sample(w, n_slices)
+    x, ws = sample
     t0 = time.time()
-    orc.forward(x["Q"], x["K"], x["V"], x["Kd"], x["Vd"], w.scale)
-    orc.backward(x["Q"], x["K"], x["V"], x["Kd"], x["Vd"], x["dO"], w.scale)
+    orc.forward(x["Q"], x["K"], x["V"], x["Kd"], x["Vd"], ws.scale)
+    orc.backward(x["Q"], x["K"], x["V"], x["Kd"], x["Vd"], x["dO"], ws.scale)
     dt = time.time() - t0
-    fl = flops.fwd_bwd_flops(n_slices, w.T, 1, w.d, w.l)
-    return dt, fl, orc.threads(), pick
+    return dt, flops.fwd_bwd_flops(1, ws.T, 1, ws.d, ws.l), orc.threads()
+
+
+def sized_sample(w, seconds):
+    """A sample whose oracle run takes about `seconds`: a short probe gives the rate, the cost grows with T^2."""
+    T_probe = min(w.T, 2048)
+    dt, fl, _ = time_oracle(cpu_sample(w, T_probe))
+    rate = fl / max(dt, 1e-4)
+    # fl(T) = 3.5 * (2 d T^2 + 4 T l d)  ->  solve for the T that costs seconds * rate
+    a, b, c = 3.5 * 2.0 * w.d, 3.5 * 4.0 * w.l * w.d, -seconds * rate
+    T_fit = int((-b + (b * b - 4 * a * c) ** 0.5) / (2 * a))
+    T_s = max(256, min(w.T, (T_fit // 256) * 256))
+    return cpu_sample(w, T_s)
 
 
 def cpu_baseline(w, budget_s=20.0):
-    """The fp64 oracle, as it stands, on complete (b, h) slices of the benchmarked workload."""
-    dt, fl, cores, pick = time_oracle(w, 1)
-    n = 1
-    if dt < budget_s / 3:
-        n = int(min(w.B * w.H, max(1, budget_s / max(dt, 1e-3))))
-        dt, fl, cores, pick = time_oracle(w, n)
+    """The fp64 oracle, as it stands, on a bounded sample of the benchmarked workload."""
+    sample = sized_sample(w, budget_s)
+    dt, fl, cores = time_oracle(sample)
+    T_s = sample[1].T
     return {"value": round(fl / dt / 1e12, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{n} complete (b,h) slice(s) of {w.name} (T={w.T}, d={w.d}, l={w.l}), forward + backward, fp64, "
-                      f"{dt:.1f} s; FLOPs counted with the same convention as the GPU arm",
+            "sample": f"one (b,h) slice of {w.name} cut to its first {T_s} of {w.T} positions (d={w.d}, l={w.l}), forward + "
+                      f"backward, fp64, {dt:.1f} s; FLOPs counted with the same convention as the GPU arm",
             "seconds": round(dt, 2)}
 
 
@@ -666,37 +701,55 @@ def run_reference(args, rank, world):
     w = pick_workload(args)
     if rank != 0:
         return None
-    K, W = args.steps, max(args.warmup, 0)
-    # bounded: each step is one complete (b, h) slice; cap the whole run near three minutes
-    sample = cpu_sample(w, 1)
-    t_probe, fl, cores, _ = time_oracle(w, 1, sample)
-    budget = 180.0
-    K_eff = int(max(1, min(K, (budget - t_probe) // max(t_probe, 1e-3))))
-    W_eff = 0 if t_probe * (K_eff + W) > budget else W
-    for _ in range(W_eff):
-        time_oracle(w, 1, sample)
-    dt = sum(time_oracle(w, 1, sample)[0] for _ in range(K_eff)) / K_eff
+    K, W = max(args.steps, 1), max(args.warmup, 0)
+    # bounded: each step is one (b, h) slice cut to a prefix sized so that the whole run stays near three minutes
+    budget = 170.0
+    sample = sized_sample(w, budget / (K + W))
+    cores = 0
+    for _ in range(W):
+        time_oracle(sample)
+    times = []
+    for _ in range(K):
+        dt, fl, cores = time_oracle(sample)
+        times.append(dt)
+    dt = sum(times) / K
     val = fl / dt / 1e12
+    T_s = sample[1].T
+    what = f"one (b,h) slice of {w.name} cut to its first {T_s} of {w.T} positions, forward + backward, fp64"
     return {
-        "impl": "reference", "metric": METRIC, "value": round(val, 6), "unit": UNIT, "n_gpus": world, "steps": K_eff,
-        "warmup": W_eff, "ms_per_step": round(dt * 1e3, 2), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "impl": "reference", "metric": METRIC, "value": round(val, 6), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": round(dt * 1e3, 2), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{w.name}: B={w.B} T={w.T} H={w.H} d={w.d} l={w.l}; each step = one complete (b,h) slice "
-                               f"(forward + backward) of that workload on the host cores"},
-        "cpu_baseline": {"value": round(val, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"one (b,h) slice of {w.name} per step, {K_eff} step(s) (requested {K})"},
+        "config": {"workload": f"{w.name}: B={w.B} T={w.T} H={w.H} d={w.d} l={w.l}; each step = {what} on the host cores"},
+        "cpu_baseline": {"value": round(val, 6), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": f"{what}, per step"},
         "e2e": {"value": round(val, 6), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
 
 
+def spawn_local_ranks(n: int) -> int:
+    """`python bench.py --gpus N` outside a launcher: start N ranks of this script on the local GPUs (one process per
+    GPU, rendezvous on 127.0.0.1) and wait for them; rank 0 prints the line."""
+    import socket
+    with socket.socket() as sck:
+        sck.bind(("127.0.0.1", 0))
+        port = sck.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    return max(p.wait() for p in procs)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="moda", choices=["moda", "reference"])
-    ap.add_argument("--workload", default="c2", help="c1..c5, optionally with _l<depth> (e.g. c3_l8)")
+    ap.add_argument("--workload", default="c4", help="c1..c5, optionally with _l<depth> (e.g. c3_l8)")
+    ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the host-to-host leg (each moves every input and output over PCIe)")
+    ap.add_argument("--sweeps", default="", help="comma list of extra sweeps printed in the line: gqa, decode, prefill")
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (smaller profiling cases)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -707,6 +760,10 @@ def main():
     ap.add_argument("--decode-shape", default="", help="B,T_kv,H,H_kv,d,l: time only this decode step and print its row; for profiling")
     args = ap.parse_args()
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        if args.impl == "moda" and torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus} but only {torch.cuda.device_count()} CUDA device(s) are visible")
+        return spawn_local_ranks(args.gpus)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

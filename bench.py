@@ -2,8 +2,8 @@
 """Benchmark of the MoDA attention operator on B200: one JSON line on stdout.
 
 A "step" is one pass of the whole hot path for one attention layer over one batch of
-synthetic inputs that are already resident in HBM: the depth-cache "write" of the layer's
-own K, V (one slot), the forward kernel, and the three backward launches (row-local part:
+synthetic inputs that are already resident in HBM: the forward kernel, which also does the
+depth-cache "write" of the layer's own K, V (one slot), and the three backward launches (row-local part:
 row terms, depth gradients, depth share of dQ; sequence part: dK, dV and the dQ tiles; dQ
 finish).  `value` is forward+backward TFLOP/s with the FLOP convention of
 paper_2603_15619_b200/flops.py (causal-halved sequence part + depth part, backward =
@@ -48,7 +48,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 NCU_SEQ_C3_L0_B1 = 202.80e6 + 100.59e6   # dram__bytes_read.sum + dram__bytes_write.sum of that one launch
 NCU_TRAFFIC_BYTES = {
     # c2 captured at B=1 and scaled x4 (traffic is proportional to B): profiles/ncu_full_c2_B1_fwd_bwd_kernels.md
-    ("c2", "fwd"): 4 * (822.179e6 + 6.956e6),
+    ("c2", "fwd_append"): 4 * (822.179e6 + 6.956e6) + 4 * 33554432 * 2,   # + the slot written (not in that capture)
     # sequence part of the backward, captured at c3 with l = 0 and B = 1 (T = 8192) and scaled by the number of
     # elements B T H d (every tensor crosses HBM once, re-reads are served by L2):
     # profiles/ncu_full_c3_l0_B1_bwd_fused_kernel.md
@@ -156,7 +156,7 @@ def job_value(world: int, flops_per_rank_step: float, ms_per_step: float) -> flo
 class Layer:
     """Device buffers of one workload plus the calls of one step."""
 
-    KERNELS = ("cache_append", "fwd", "bwd_rows", "bwd_seq", "bwd_finish")
+    KERNELS = ("fwd_append", "bwd_rows", "bwd_seq", "bwd_finish")
 
     def __init__(self, w: synthetic.Workload, seed: int, device, with_backward: bool = True):
         import paper_2603_15619_b200 as moda
@@ -180,8 +180,10 @@ class Layer:
             self.dQ, self.dK, self.dV = (torch.empty_like(self.q) for _ in range(3))
             self.ws = torch.empty(moda.moda_bwd_workspace_bytes(w.B, w.T, w.H, w.d, w.l), dtype=torch.uint8, device=device)
 
-    def append(self):
-        self.moda.moda_depth_cache_append(self.next_slot, 0, self.k, self.v)
+    def fwd_append(self):
+        """Forward with the depth stream's write step fused in: this layer's K, V go to the slot the later layers read."""
+        self.moda.moda_attn_fwd_append(self.q, self.k, self.v, self.cache, self.w.l, self.w.scale, self.next_slot, 0,
+                                       O=self.O, LSE=self.LSE)
 
     def fwd(self):
         self.moda.moda_attn_fwd(self.q, self.k, self.v, self.cache, self.w.l, self.w.scale, O=self.O, LSE=self.LSE)
@@ -191,10 +193,10 @@ class Layer:
                                 dQ=self.dQ, dK=self.dK, dV=self.dV, d_depth_kv=self.dcache, workspace=self.ws, stages=stages)
 
     def step(self, events=None):
-        """One pass of the hot path; with `events` (6 CUDA events) records one between launches."""
-        calls = (self.append, self.fwd, lambda: self.bwd(1), lambda: self.bwd(2), lambda: self.bwd(4))
+        """One pass of the hot path; with `events` (5 CUDA events) records one between launches."""
+        calls = (self.fwd_append, lambda: self.bwd(1), lambda: self.bwd(2), lambda: self.bwd(4))
         if events is None:
-            self.append(); self.fwd(); self.bwd()
+            self.fwd_append(); self.bwd()
             return
         events[0].record()
         for i, c in enumerate(calls):
@@ -210,8 +212,8 @@ class Layer:
         seq = flops.fwd_flops(w.B, w.T, w.H, w.d, 0)
         dep = flops.depth_fwd_flops(w.B, w.T, w.H, w.d, w.l)
         return {
-            "cache_append": {"bytes": 2.0 * 4 * E, "flops": 0.0},
-            "fwd": {"bytes": flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l), "flops": f_fwd},
+            # the forward's own bytes plus the slot it writes (K and V once more, in cache layout)
+            "fwd_append": {"bytes": flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l) + 2.0 * 2 * E, "flops": f_fwd},
             # reads Q O dO (bf16), LSE and the depth cache; writes the row terms, the depth gradients and the fp32 dQ accumulator
             "bwd_rows": {"bytes": 2.0 * (3 * E + 4 * w.l * E) + 4.0 * E + 8.0 * rows, "flops": 2.0 * E + 2.5 * dep},
             # reads Q K V dO + LSE, D; writes dK dV; reads and writes the fp32 dQ accumulator; the five sequence contractions
@@ -248,7 +250,7 @@ def run_moda(args, rank, world, device):
         raise RuntimeError(f"device status {moda.moda_last_status()} after warm-up")
 
     K = args.steps
-    evs = [[ev() for _ in range(6)] for _ in range(K)]
+    evs = [[ev() for _ in range(5)] for _ in range(K)]
     sampler = ClockSampler(device.index)
     sampler.start()
     time.sleep(0.3)
@@ -261,7 +263,7 @@ def run_moda(args, rank, world, device):
     t_end = time.time()
     barrier()
     clocks = sampler.stop(t_begin, t_end)
-    total_ms = evs[0][0].elapsed_time(evs[-1][5])
+    total_ms = evs[0][0].elapsed_time(evs[-1][4])
     ms_per_step = total_ms / K
     ms_per_step = max_over_ranks(ms_per_step, world, device)
     status = moda.moda_last_status()
@@ -294,16 +296,16 @@ def run_moda(args, rank, world, device):
                  "algorithmic_bytes": model[dom]["bytes"], "algorithmic_flops": model[dom]["flops"],
                  "kernel_ms_x_sm_mhz": None if mhz is None else round(per_kernel[dom] * mhz, 1)})
 
-    fwd_tflops = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l) / (per_kernel["fwd"] * 1e-3) / 1e12
+    fwd_tflops = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l) / (per_kernel["fwd_append"] * 1e-3) / 1e12
     bwd_ms = per_kernel["bwd_rows"] + per_kernel["bwd_seq"] + per_kernel["bwd_finish"]
     detail = {
         "kernel_ms": {k: round(v, 4) for k, v in per_kernel.items()},
         "fwd_tflops": round(fwd_tflops, 1),
         "bwd_tflops": round(flops.bwd_flops(w.B, w.T, w.H, w.d, w.l) / (bwd_ms * 1e-3) / 1e12, 1),
-        "bwd_over_fwd_time": round(bwd_ms / per_kernel["fwd"], 3),
+        "bwd_over_fwd_time": round(bwd_ms / per_kernel["fwd_append"], 3),
         "fwd_frac_of_measured_burst_bf16": round(fwd_tflops / peaks["bf16_tflops"], 4),
         "fwd_frac_of_measured_sustained_bf16": round(fwd_tflops / peaks["bf16_tflops_sustained"], 4),
-        "fwd_depth_read_gbs": round(flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / (per_kernel["fwd"] * 1e-3) / 1e9, 1),
+        "fwd_depth_read_gbs": round(flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / (per_kernel["fwd_append"] * 1e-3) / 1e9, 1),
         "ms_per_step_x_sm_mhz": None if mhz is None else round(ms_per_step * mhz, 1),
         "flops": "fwd = 4BHd T^2/2 + 4BHTld; bwd = 2.5 fwd",
     }
@@ -313,15 +315,15 @@ def run_moda(args, rank, world, device):
         "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{w.name}: B={w.B} T={w.T} H={w.H} d={w.d} l={w.l} (per GPU), bf16 N(0,1) inputs, fp32 accumulate",
-                   "step": "depth-cache append of one slot + forward + backward (row-local part incl. depth gradients, "
-                           "sequence part dK/dV/dQ tiles, dQ finish)",
+                   "step": "forward (writes the layer's own K, V as the next depth slot) + backward (row-local part incl. "
+                           "depth gradients, sequence part dK/dV/dQ tiles, dQ finish)",
                    "l2_policy": "inputs larger than L2 (depth cache %.2f GiB + 4 x %.0f MiB activations per step)"
                                 % (flops.depth_bytes_fwd(w.B, w.T, w.H, w.d, w.l) / 2 ** 30, w.B * w.T * w.H * w.d * 2 / 2 ** 20),
                    "parallelism": f"independent batch shards x{world}, no collective"},
-        "roofline": roof, "clocks": clocks, "gpu_launches": 5 * K, "detail": detail,
+        "roofline": roof, "clocks": clocks, "gpu_launches": 4 * K, "detail": detail,
     }
 
-    headline = {"fwd_ms": per_kernel["fwd"], "bwd_ms": bwd_ms}
+    headline = {"fwd_ms": per_kernel["fwd_append"], "bwd_ms": bwd_ms}
     if not args.no_e2e:
         out["e2e"] = run_e2e(layer, args.e2e_steps, world, step_flops, device)
     del layer

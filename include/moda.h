@@ -130,6 +130,22 @@ int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth
                   void* O, float* LSE, void* stream);
 
 /*
+ * Forward with the depth stream's "write" step fused in (Sec. 2.2: after attending, a layer appends
+ * its own K, V to the depth stream for the layers above it).  Computes exactly what
+ * moda_attn_fwd_gqa computes and, in the same launch, stores K and V (bf16 [B][T][H_kv][d]) into slot
+ * `append_slot` of `append_cache` in the cache layout, bit for bit what moda_depth_cache_append(
+ * append_cache, B, T, H_kv, d, append_slot, K, V) would store: every CTA already holds the K and V
+ * rows of its own 128 positions in shared memory (its diagonal key tile) and copies them out, so the
+ * separate pass over K and V is gone.  `append_cache` may be the buffer `depth_kv` points to (one
+ * growing cache per stack, the layer-l call reads slots < l and writes slot l); writing a slot that
+ * the same call reads (append_cache == depth_kv and append_slot < l) is MODA_ERR_BAD_SLOT.
+ * Other arguments, validation and errors as for moda_attn_fwd_gqa.
+ */
+int moda_attn_fwd_append(const void* Q, const void* K, const void* V, const void* depth_kv,
+                         int B, int T, int H, int H_kv, int d, int l, float scale,
+                         void* O, float* LSE, void* append_cache, int append_slot, void* stream);
+
+/*
  * Bytes of scratch moda_attn_bwd needs: fp32 row terms D_t = <dO_t, O_t> ([B][H][T]) and an fp32
  * accumulator for dQ (B * H * ceil(T/128) * 128 * d values; 4 bytes per dQ element).  Enough for
  * every stage mask of moda_attn_bwd_stages.

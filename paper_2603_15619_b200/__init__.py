@@ -25,6 +25,7 @@ from .binding import (  # noqa: F401
     moda_attn_decode_paged,
     moda_attn_decode_varlen,
     moda_attn_fwd,
+    moda_attn_fwd_append,
     moda_attn_fwd_gqa,
     moda_attn_fwd_prefill,
     moda_bwd_workspace_bytes,

@@ -22,7 +22,7 @@ SYMBOLS = (
     "moda_attn_fwd", "moda_bwd_workspace_bytes", "moda_attn_bwd", "moda_attn_bwd_stages",
     "moda_attn_bwd_static_scratch",
     "moda_attn_fwd_gqa", "moda_bwd_workspace_bytes_gqa", "moda_attn_bwd_gqa", "moda_attn_bwd_gqa_stages",
-    "moda_decode_workspace_bytes", "moda_attn_decode", "moda_attn_fwd_prefill",
+    "moda_decode_workspace_bytes", "moda_attn_decode", "moda_attn_fwd_prefill", "moda_attn_fwd_append",
     "moda_attn_decode_varlen", "moda_attn_decode_paged",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
@@ -79,6 +79,8 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd_static_scratch.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 4 + [vp]
     lib.moda_attn_fwd_gqa.restype = ci
     lib.moda_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
+    lib.moda_attn_fwd_append.restype = ci
+    lib.moda_attn_fwd_append.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, ci, vp]
     lib.moda_bwd_workspace_bytes_gqa.restype = sz
     lib.moda_bwd_workspace_bytes_gqa.argtypes = [ci] * 6
     lib.moda_attn_bwd_gqa.restype = ci
@@ -299,6 +301,21 @@ def moda_attn_fwd_gqa(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None
     _check(load().moda_attn_fwd_gqa(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
                                     B, T, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE), _stream(stream)),
            "moda_attn_fwd_gqa")
+    return O, LSE
+
+
+def moda_attn_fwd_append(Q, K, V, depth_kv, l, scale, append_cache, append_slot, O=None, LSE=None, stream=None):
+    """moda_attn_fwd_gqa that also stores K, V into slot ``append_slot`` of ``append_cache`` (cache layout, H_kv heads)
+    in the same launch: the depth stream's write step without a separate pass over K and V."""
+    B, T, H, Hk, d = _gqa_shapes(Q, K, V)
+    if O is None:
+        O = _new_like(Q, stream)
+    if LSE is None:
+        LSE = _new((B, H, T), torch.float32, Q.device, stream)
+    _check(load().moda_attn_fwd_append(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv) if l > 0 else None,
+                                       B, T, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
+                                       _ptr(append_cache), int(append_slot), _stream(stream)),
+           "moda_attn_fwd_append")
     return O, LSE
 
 

@@ -210,7 +210,7 @@ int launch_depth_merge(DepthMergeParams m, cudaStream_t stream) {
 
 template <int D>
 int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int T_kv, int H, int Hk, int l,
-               float scale, void* O, float* LSE, cudaStream_t stream) {
+               float scale, void* O, float* LSE, void* append_slot, cudaStream_t stream) {
     constexpr bool kWide = (D == 64);
     constexpr int kSmem = kWide ? Fwd2Smem<D>::kDynamic : FwdSmem<D, 2>::kDynamic;
     constexpr int kSmemDeep = FwdSmem<128, 1>::kDynamic;
@@ -236,6 +236,7 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.T_kv = T_kv; p.kv_off = T_kv - T;
     p.G = H / Hk;
     p.scale_log2 = scale * kLog2e;
+    p.append_slot = static_cast<__nv_bfloat16*>(append_slot);
     const unsigned grid = unsigned(B) * H * num_tiles(T);
     // Grouped-query calls: the sequence kernel runs without depth slots and a second kernel adds the depth
     // part of all heads of a group at once (moda_depth_gqa.cuh).
@@ -686,8 +687,28 @@ int moda_attn_fwd_prefill(const void* Q, const void* K, const void* V, const voi
         return MODA_ERR_MISALIGNED;
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv, B, T_q, T_kv, H, H_kv, l, scale, O, LSE, st)
-                    : launch_fwd<64>(Q, K, V, depth_kv, B, T_q, T_kv, H, H_kv, l, scale, O, LSE, st);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv, B, T_q, T_kv, H, H_kv, l, scale, O, LSE, nullptr, st)
+                    : launch_fwd<64>(Q, K, V, depth_kv, B, T_q, T_kv, H, H_kv, l, scale, O, LSE, nullptr, st);
+}
+
+int moda_attn_fwd_append(const void* Q, const void* K, const void* V, const void* depth_kv,
+                         int B, int T, int H, int H_kv, int d, int l, float scale,
+                         void* O, float* LSE, void* append_cache, int append_slot, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_groups(H, H_kv)) return rc;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (append_slot < 0 || append_slot >= MODA_MAX_DEPTH) return MODA_ERR_BAD_SLOT;
+    if (!Q || !K || !V || !O || !LSE || !append_cache || (l > 0 && !depth_kv)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) || !aligned16(append_cache) ||
+        (l > 0 && !aligned16(depth_kv)))
+        return MODA_ERR_MISALIGNED;
+    // the slot being written must not be one of the slots being read
+    if (l > 0 && append_cache == depth_kv && append_slot < l) return MODA_ERR_BAD_SLOT;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    void* slot = static_cast<__nv_bfloat16*>(append_cache) + size_t(append_slot) * cache_slot_elems(B, T, H_kv, d);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv, B, T, T, H, H_kv, l, scale, O, LSE, slot, st)
+                    : launch_fwd<64>(Q, K, V, depth_kv, B, T, T, H, H_kv, l, scale, O, LSE, slot, st);
 }
 
 size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l) {

@@ -92,6 +92,10 @@ struct FwdParams {
     int T_kv, kv_off;                // sequence keys 0 .. T_kv - 1; query row i sits at key position i + kv_off (kv_off = T_kv - T)
     int G;                           // query heads per key/value head (1 = plain multi-head attention)
     float scale_log2;                // scale * log2(e)
+    // "Write" step of the depth stream fused into the forward: when not null, the base of one cache slot
+    // (H / G heads) into which every CTA copies the K and V rows of its own 128 positions, straight from the
+    // shared-memory tiles of its last (diagonal) key tile.  Only with kv_off == 0; the first head of a group writes.
+    __nv_bfloat16* append_slot;
 };
 
 // Which (batch, query head, key/value head, query tile) a CTA works on.  The G query heads that
@@ -118,6 +122,22 @@ __device__ __forceinline__ TileCoord tile_coord(int block, int nq, int H, int G)
 // TMA wrote as D/64 sub-tiles of [128][64] with the 128-byte swizzle.
 __device__ __forceinline__ uint32_t swz_chunk_offset(int r, int c) {
     return uint32_t(c >> 3) * uint32_t(kTileRows * 128) + uint32_t(r) * 128u + (uint32_t((c & 7) ^ (r & 7)) << 4);
+}
+
+// Copies one thread's row of the CTA's diagonal K and V tiles (TMA-written, 128-byte swizzled) into the cache
+// block (b, hk, qt) of a slot: chunk c of row r goes to [c][r], so a warp writes 512 contiguous bytes per chunk.
+// Rows of a ragged last tile were zero-filled by TMA, which is what the cache wants in its tail rows.
+template <int D>
+__device__ __forceinline__ void append_rows_to_slot(__nv_bfloat16* slot, const uint8_t* sK, const uint8_t* sV,
+                                                    size_t block_index, int r) {
+    constexpr int CH = D / 8;
+    uint4* dK = reinterpret_cast<uint4*>(slot) + block_index * 2 * (kTileRows * CH) + r;
+    uint4* dV = dK + kTileRows * CH;
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+        dK[c * kTileRows] = *reinterpret_cast<const uint4*>(sK + swz_chunk_offset(r, c));
+        dV[c * kTileRows] = *reinterpret_cast<const uint4*>(sV + swz_chunk_offset(r, c));
+    }
 }
 
 template <int D, int KST = 2>
@@ -445,6 +465,15 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(kBarDepth));
+        }
+        if (p.append_slot != nullptr && h == hk * p.G) {
+            // Every MMA has completed, so no load is in flight and the last tiles sit in their stages; the
+            // second and third waits are on phases that have completed and make the TMA writes visible here.
+            const int j = n_kv - 1;
+            mbar_wait(bar(kBarOFinal), 0, abort_flag, 22);
+            mbar_wait2(bar(kBarKFull + j % KST), (j / KST) & 1, bar(kBarVFull + (j & 1)), (j >> 1) & 1, abort_flag, 23, 24);
+            append_rows_to_slot<D>(p.append_slot, smem + L::kK + (j % KST) * L::kTileBytes, smem + L::kV + (j & 1) * L::kTileBytes,
+                                   (size_t(b) * Hk + hk) * nq + qt, tid - 128);
         }
     } else {
       setmaxnreg_dec<72>();   // one instruction for the whole producer warpgroup (warps 8-11)

@@ -461,6 +461,14 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             tc_fence_before_sync();
             mbar_arrive(bar(k2BarDepth));
         }
+        if (p.append_slot != nullptr && h == hk * p.G) {
+            // the "write" step of the depth stream, from the tiles of the diagonal key tile (see moda_fwd_kernel)
+            const int j = n_kv - 1, st = j % L::kStages;
+            mbar_wait(bar(k2BarOFinal), 0, abort_flag, 22);
+            mbar_wait2(bar(k2BarKFull + st), (j / L::kStages) & 1, bar(k2BarVFull + st), (j / L::kStages) & 1, abort_flag, 23, 24);
+            append_rows_to_slot<D>(p.append_slot, smem + L::kK + st * L::kKeyTileBytes, smem + L::kV + st * L::kKeyTileBytes,
+                                   (size_t(b) * (p.H / p.G) + hk) * nq + qt, tid - 256);
+        }
     } else {
       setmaxnreg_dec<40>();   // one instruction for the whole producer warpgroup (warps 12-15)
       if (warp == 12) {

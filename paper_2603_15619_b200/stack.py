@@ -30,8 +30,8 @@ class _Attend(torch.autograd.Function):
     @staticmethod
     def forward(ctx, Q, K, V, token, stream, l, scale):
         Q, K, V = Q.contiguous(), K.contiguous(), V.contiguous()
-        O, LSE = binding.moda_attn_fwd_gqa(Q, K, V, stream.cache if l > 0 else None, l, scale)
-        binding.moda_depth_cache_append(stream.cache, l, K, V)          # the "write" step: slot l = this layer
+        # attention and the "write" step (slot l = this layer's K, V) in one launch
+        O, LSE = binding.moda_attn_fwd_append(Q, K, V, stream.cache if l > 0 else None, l, scale, stream.cache, l)
         ctx.save_for_backward(Q, K, V, O, LSE)
         ctx.stream, ctx.l, ctx.scale = stream, l, scale
         return O, token + 0

@@ -1,0 +1,49 @@
+"""The depth stream's write step fused into the forward (moda_attn_fwd_append), on the GPU through the C ABI:
+the slot it writes is bit for bit what moda_depth_cache_append writes, O and LSE are bit for bit those of the plain
+forward, and the slot that the next layer reads is really the one that was written."""
+import pytest
+import torch
+
+import paper_2603_15619_b200 as moda
+from paper_2603_15619_b200 import binding, synthetic
+
+from parity import assert_forward_close, build_cache, f64
+from oracle import moda_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    # B, T, H, H_kv, d, l
+    (1, 128, 1, 1, 128, 0), (2, 300, 2, 2, 128, 3), (1, 1000, 3, 3, 64, 2), (1, 257, 4, 2, 64, 5), (2, 129, 8, 2, 128, 1),
+    (1, 640, 2, 2, 128, 12),      # 2 l d >= T: the deep-ring variant of the d = 128 kernel
+    (1, 1, 2, 1, 64, 0), (1, 520, 16, 2, 64, 33), (1, 130, 8, 1, 128, 50),   # grouped-query calls whose depth part is a second kernel
+]
+
+
+@pytest.mark.parametrize("B,T,H,Hk,d,l", SHAPES)
+def test_fused_write_step_is_the_separate_append_bit_for_bit(B, T, H, Hk, d, l):
+    scale = d ** -0.5
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=41, device="cuda")
+    want = moda.alloc_depth_cache(B, T, Hk, d, l + 1)
+    got = moda.alloc_depth_cache(B, T, Hk, d, l + 1)
+    for c in (want, got):
+        c.fill_(7.0)
+        for i in range(l):
+            moda.moda_depth_cache_append(c, i, x["Kd"][i].contiguous(), x["Vd"][i].contiguous())
+    moda.moda_depth_cache_append(want, l, x["K"], x["V"])
+    O0, LSE0 = moda.moda_attn_fwd_gqa(x["Q"], x["K"], x["V"], want, l, scale)
+    O1, LSE1 = moda.moda_attn_fwd_append(x["Q"], x["K"], x["V"], got, l, scale, got, l)
+    assert moda.moda_last_status() == 0
+    assert torch.equal(got, want), "slot written by the forward differs from moda_depth_cache_append"
+    assert torch.equal(O0, O1) and torch.equal(LSE0, LSE1)
+    xs = [f64(x[n]) for n in ("Q", "K", "V", "Kd", "Vd")]
+    assert_forward_close(O1, LSE1, *orc.forward_gqa(*xs, scale), "forward with the fused write step")
+
+
+def test_writing_a_slot_that_the_call_reads_is_rejected():
+    B, T, H, d, l = 1, 128, 1, 64, 2
+    x = synthetic.make_gqa(B, T, H, H, d, l, seed=1, device="cuda")
+    cache = build_cache(x["Kd"], x["Vd"])
+    with pytest.raises(binding.ModaError) as e:
+        moda.moda_attn_fwd_append(x["Q"], x["K"], x["V"], cache, l, 0.125, cache, 1)
+    assert e.value.code == -6

@@ -365,7 +365,7 @@ int launch_bwd_fused(const BwdArgs& a, int stages, cudaStream_t stream) {
         f.B = B; f.T = T; f.H = H; f.G = G;
         f.scale = a.scale; f.scale_log2 = a.scale * kLog2e;
         const unsigned grid = unsigned(B) * Hk * num_tiles(T);
-        moda_bwd_fused_kernel<D><<<grid, kBwdFusedThreads, L::kDynamic, stream>>>(mK, mV, mQ, mdO, mdK, mdV, f);
+        moda_bwd_fused_kernel<D><<<grid, L::kThreads, L::kDynamic, stream>>>(mK, mV, mQ, mdO, mdK, mdV, f);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     }
     if (stages & 4) {

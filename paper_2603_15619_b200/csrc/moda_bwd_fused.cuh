@@ -208,14 +208,14 @@ bwd_dq_finish_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict
 // =====================================================================================
 // 2. Sequence part: dK, dV and the dQ tiles
 // =====================================================================================
-// 512 threads.
-//   warps 0-7    row warps: a thread owns one key row (= tensor-memory lane) and 64 of the 128 query columns
-//                of an iteration (warps 0-3 the low half, 4-7 the high half): P^T, then dS^T.
-//   warps 8-11   drain warps: a thread owns one query row of the dQ tile; it copies the row out of tensor memory
+// 512 threads (in warp order):
+//   row warps    two warpgroups: a thread owns one key row (= tensor-memory lane) and 64 of the 128 query columns of
+//                an iteration: P^T, then dS^T.
+//   drain warps  one warpgroup: a thread owns one query row of the dQ tile; it copies the row out of tensor memory
 //                (which frees the region at once) and adds it to the fp32 accumulator with 16-byte reductions
 //                at whatever pace L2 takes them, without holding up the row warps.
-//   warp 12      loader (TMA tiles, per-query LSE and D_t)
-//   warps 13-15  issue the contractions: S (13), dP (14), dV then dQ then dK (15).  One tcgen05.mma costs its
+//   then         a loader warp (TMA tiles, per-query LSE and D_t) and the warps that issue the contractions:
+//                S, dP, and dV then dQ then dK.  One tcgen05.mma costs its
 //                issuing thread about as long as it executes, so the contractions that start an iteration's two
 //                chains have their own warps on different schedulers; MMAs of different warps are ordered by
 //                mbarriers only.
@@ -234,10 +234,12 @@ bwd_dq_finish_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict
 //   X:  S_i -> P_i^T = exp2(S c - LSE c) (row warps) -> dV_i -> X free -> S_{i+1}
 //   Y:  dP_i -> dS_i^T = P o (dP - D) to shared memory (row warps) -> dQ_i -> copied out (drain warps) -> Y free -> dP_{i+1}
 // and dK_i, issued behind dQ_i, fills the tensor pipe while the row warps exponentiate tile i+1.
-constexpr int kBwdFusedThreads = 512;
 
 template <int D>
 struct FusedSmem {
+    static constexpr int kRowWGs = 2;                          // row warpgroups (64 query columns per thread)
+    static constexpr int kCols = kTileRows / kRowWGs;          // query columns per row-warp thread
+    static constexpr int kThreads = (kRowWGs * 4 + 8) * 32;    // row warps, 4 drain warps, loader + 3 issuers
     static constexpr int kTileBytes = kTileRows * D * 2;       // 128 x D bf16
     static constexpr int kSubBytes = kTileRows * 128;          // 128 x 64 sub-tile (128-byte rows)
     // Stages of Q_i.  Q_i is read by S_i early and by dK_i late in its iteration, and a tile takes about 1600
@@ -254,12 +256,12 @@ struct FusedSmem {
     static constexpr int kdO = kQ + kStages * kTileBytes;      // stages of dO_i
     static constexpr int kdS = kdO + kdOStages * kTileBytes;   // dS^T: 128 keys x 128 queries bf16
     static constexpr int kdSBytes = kTileRows * kTileRows * 2;
-    static constexpr int kStg = kdS + kdSBytes;                // 64 feature columns of a dQ tile, fp32, accumulator layout
+    static constexpr int kStg = kdS + kdSBytes;                // four chunks of 16 feature columns of a dQ tile, fp32, accumulator layout
     static constexpr int kStgBytes = 64 * kTileRows * 4;
     static constexpr int kRow = kStg + kStgBytes;              // per stage: -LSE log2e [128], D_t [128]
     static constexpr int kRowBytes = 2 * kTileRows * 4;
     static constexpr int kBars = kRow + kStages * kRowBytes;
-    static constexpr int kNumBars = 26;
+    static constexpr int kNumBars = 28;
     static constexpr int kMisc = kBars + kNumBars * 8;
     static constexpr int kTotal = kMisc + 16;
     static constexpr int kSmemLimit = 232448;                  // 227 KiB per CTA on sm_100
@@ -296,13 +298,17 @@ struct FusedParams {
 };
 
 template <int D>
-__global__ void __launch_bounds__(kBwdFusedThreads, 1)
+__global__ void __launch_bounds__(FusedSmem<D>::kThreads, 1)
 moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                       const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapdO,
                       const __grid_constant__ CUtensorMap mapdK, const __grid_constant__ CUtensorMap mapdV,
                       const FusedParams p) {
     using L = FusedSmem<D>;
     constexpr int NSUB = D / 64;
+    constexpr int NRW = L::kRowWGs, COLS = L::kCols, NROW = 128 * NRW;      // row warpgroups, columns per thread, row threads
+    constexpr int W_DRAIN = 4 * NRW, W_LOAD = W_DRAIN + 4, W_S = W_LOAD + 1, W_DP = W_LOAD + 2;
+    constexpr int W_ACC = W_LOAD + 3;                             // issues the three accumulating contractions
+    constexpr int NOTHER = (L::kThreads / 32 - W_LOAD) * 32;      // threads of the loader / issuer warps
     constexpr uint32_t kTmemCols = 512;
     // d = 64 leaves room for a second S^T / P^T buffer: S_{i+1} is then computed while the row warps still work
     // on tile i, instead of waiting for dV_i to release the only buffer.
@@ -346,18 +352,18 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(kFBarSFull + s), 1);
-            mbar_init(bar(kFBarPFull + s), 256);
+            mbar_init(bar(kFBarPFull + s), NROW);
             mbar_init(bar(kFBarXFree + s), 1);
         }
         mbar_init(bar(kFBardPFull), 1);
-        mbar_init(bar(kFBardSFull), 256);
+        mbar_init(bar(kFBardSFull), NROW);
         mbar_init(bar(kFBardQFull), 1);
         mbar_init(bar(kFBarYFree), 128);
         mbar_init(bar(kFBarFinal), 1);
         for (int s = 0; s < 3; ++s) mbar_init(bar(kFBarDrain + s), 1);
         fence_mbar_init();
     }
-    if (warp == 13) {
+    if (warp == W_S) {
         tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -375,45 +381,50 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         }
     };
 
-    // Register budget: the CTA owns what it was launched with, 512 threads x 128 registers, and
-    // setmaxnreg.inc blocks until the CTA's own pool can serve it, so the three shares must fit that total.
+    // Register budget: the CTA owns what it was launched with (512 threads x 128 registers), and setmaxnreg.inc blocks until the CTA's own pool can serve it, so the three shares must fit that total.
+    constexpr int kRegsLaunch = 128;
+    static_assert(L::kThreads == 512, "the register shares below assume 512 threads");
     constexpr int kRegsRow = (D == 128) ? 136 : 152, kRegsDrain = (D == 128) ? 160 : 152, kRegsOther = (D == 128) ? 80 : 56;
-    static_assert(256 * kRegsRow + 128 * kRegsDrain + 128 * kRegsOther <= kBwdFusedThreads * 128, "register shares exceed the CTA's pool");
-    if (warp < 8) {
+    static_assert(NROW * kRegsRow + 128 * kRegsDrain + NOTHER * kRegsOther <= L::kThreads * kRegsLaunch, "register shares exceed the CTA's pool");
+    // setmaxnreg.inc to less than the current count (or .dec to more) is an illegal instruction
+    static_assert(kRegsRow >= kRegsLaunch && kRegsDrain >= kRegsLaunch && kRegsOther <= kRegsLaunch, "setmaxnreg direction");
+    if (warp < W_DRAIN) {
         // =========================== row warps: P^T, dS^T, dK / dV epilogue ===========================
         setmaxnreg_inc<kRegsRow>();
-        const int hc = warp >> 2;                            // which 64 query columns of every iteration
+        const int hc = warp >> 2;                            // which COLS query columns of every iteration
         const int r = tid & 127;                             // key row inside the tile = TMEM lane
         const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
-        const uint32_t tX0 = tmem + lane_addr + kColX + hc * 64;
-        const uint32_t tY = tmem + lane_addr + kColY + hc * 64;
-        uint8_t* ds_row = smem + L::kdS + hc * L::kSubBytes + r * 128;   // this thread's 128-byte row of dS^T
+        const uint32_t tX0 = tmem + lane_addr + kColX + hc * COLS;
+        const uint32_t tY = tmem + lane_addr + kColY + hc * COLS;
+        // this thread's row of dS^T: sub-tile of its 64-column half, 128-byte rows, its first 16-byte chunk
+        uint8_t* ds_row = smem + L::kdS + ((hc * COLS) >> 6) * L::kSubBytes + r * 128;
+        const int ds_chunk0 = ((hc * COLS) & 63) >> 3;
         for (int it = 0; it < n_it; ++it) {
             const int st = it % L::kStages;
             const bool diag = (it % n_per) == 0;             // the query tile is the key tile itself: causal mask
-            const float* rt = reinterpret_cast<const float*>(smem + L::kRow + st * L::kRowBytes) + hc * 64;
-            uint32_t pk[32];                                 // P_i^T of this thread: 64 values, bf16 pairs
+            const float* rt = reinterpret_cast<const float*>(smem + L::kRow + st * L::kRowBytes) + hc * COLS;
+            uint32_t pk[COLS / 2];                           // P_i^T of this thread: COLS values, bf16 pairs
             // ---- P_i^T ----
             const int xb = it % XB;
             const uint32_t tX = tX0 + xb * 128;
             mbar_wait(bar(kFBarSFull + xb), (it / XB) & 1, abort_flag, 121);
             tc_fence_after_sync();
             {
-                // both halves are requested before the first is used: the second load's latency hides under the
-                // first half's exponentials
-                uint32_t sv[64];
-                tmem_ld32(tX, *reinterpret_cast<uint32_t(*)[32]>(sv));
-                tmem_ld32(tX + 32, *reinterpret_cast<uint32_t(*)[32]>(sv + 32));
+                // all blocks are requested before the first is used: the later loads' latency hides under the
+                // first block's exponentials
+                uint32_t sv[COLS];
+#pragma unroll
+                for (int c = 0; c < COLS / 32; ++c) tmem_ld32(tX + c * 32, *reinterpret_cast<uint32_t(*)[32]>(sv + c * 32));
                 tmem_wait_ld();
 #pragma unroll
-                for (int i4 = 0; i4 < 16; ++i4) {
+                for (int i4 = 0; i4 < COLS / 4; ++i4) {
                     const float4 nl = *reinterpret_cast<const float4*>(rt + 4 * i4);     // same address for all rows
                     float e0 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 0]), p.scale_log2, nl.x));
                     float e1 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 1]), p.scale_log2, nl.y));
                     float e2 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 2]), p.scale_log2, nl.z));
                     float e3 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 3]), p.scale_log2, nl.w));
                     if (diag) {                               // query column c sees key row r iff c >= r
-                        const int c = hc * 64 + 4 * i4;
+                        const int c = hc * COLS + 4 * i4;
                         if (c + 0 < r) e0 = 0.f;
                         if (c + 1 < r) e1 = 0.f;
                         if (c + 2 < r) e2 = 0.f;
@@ -423,8 +434,9 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                     pk[2 * i4 + 1] = pack_bf16x2(e2, e3);
                 }
             }
-            // P^T (bf16, two per column) overlays the first 32 of the 64 columns this thread has read
-            tmem_st32(tX, pk);
+            // P^T (bf16, two per column) overlays the first half of the columns this thread has read
+            if constexpr (COLS == 64) tmem_st32(tX, *reinterpret_cast<uint32_t(*)[32]>(pk));
+            else tmem_st16(tX, *reinterpret_cast<uint32_t(*)[16]>(pk));
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(kFBarPFull + xb));
@@ -435,12 +447,12 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
             // the dS buffer is still read by dQ_{i-1} and dK_{i-1} (dK is issued last: its completion covers both)
             if (it > 0) mbar_wait(bar(kFBarQEmpty + (it - 1) % L::kStages), ((it - 1) / L::kStages) & 1, abort_flag, 123);
             {
-                uint32_t gv[64];
-                tmem_ld32(tY, *reinterpret_cast<uint32_t(*)[32]>(gv));
-                tmem_ld32(tY + 32, *reinterpret_cast<uint32_t(*)[32]>(gv + 32));
+                uint32_t gv[COLS];
+#pragma unroll
+                for (int c = 0; c < COLS / 32; ++c) tmem_ld32(tY + c * 32, *reinterpret_cast<uint32_t(*)[32]>(gv + c * 32));
                 tmem_wait_ld();
 #pragma unroll
-                for (int g = 0; g < 8; ++g) {                // 8 query columns = one 16-byte chunk of the row
+                for (int g = 0; g < COLS / 8; ++g) {         // 8 query columns = one 16-byte chunk of the row
                     const float4 da = *reinterpret_cast<const float4*>(rt + kTileRows + 8 * g);
                     const float4 db = *reinterpret_cast<const float4*>(rt + kTileRows + 8 * g + 4);
                     const uint32_t* pp = pk + 4 * g;
@@ -453,7 +465,7 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                                       bf16_hi_to_f32(pp[2]) * (__uint_as_float(gv[8 * g + 5]) - db.y));
                     v.w = pack_bf16x2(bf16_lo_to_f32(pp[3]) * (__uint_as_float(gv[8 * g + 6]) - db.z),
                                       bf16_hi_to_f32(pp[3]) * (__uint_as_float(gv[8 * g + 7]) - db.w));
-                    *reinterpret_cast<uint4*>(ds_row + ((g ^ (r & 7)) << 4)) = v;
+                    *reinterpret_cast<uint4*>(ds_row + (((ds_chunk0 + g) ^ (r & 7)) << 4)) = v;
                 }
             }
             fence_proxy_async_smem();                        // generic-proxy stores -> read by the MMAs (async proxy)
@@ -462,6 +474,7 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         }
 
         // ---- epilogue: dK (scaled) by the first warpgroup, dV by the second ----
+        if (hc < 2) {
         mbar_wait(bar(kFBarFinal), 0, abort_flag, 124);
         tc_fence_after_sync();
         {
@@ -495,7 +508,8 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
             tma_store_commit();
             tma_store_wait_all();
         }
-    } else if (warp < 12) {
+        }
+    } else if (warp < W_LOAD) {
         // =========================== drain warps: dQ tile -> fp32 accumulator ===========================
         // The tile leaves the SM as bulk reductions (cp.reduce.async.bulk, fp32 add in L2) from a staging buffer
         // in shared memory.  Per-thread red.global instructions would do the same additions, but they queue in the
@@ -517,28 +531,31 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
             tmem_wait_ld();
             tc_fence_before_sync();
             mbar_arrive(bar(kFBarYFree));                    // Y may take dP of the next iteration
+            // 16 feature columns (8 KiB, contiguous in the accumulator) at a time through a ring of four staging chunks:
+            // a chunk is rewritten once the reduction issued from it four chunks earlier has finished reading it, so
+            // up to three reductions stay in flight and L2, not this loop, sets the pace.
 #pragma unroll
-            for (int rd = 0; rd < D / 64; ++rd) {            // 64 feature columns (32 KiB) per round
-                // the previous round's reduction has finished reading the staging buffer
-                if (tid == 256) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            for (int ch = 0; ch < D / 16; ++ch) {
+                const int slot = ch & 3;
+                if (tid == NROW) asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
                 asm volatile("bar.sync 2, 128;" ::: "memory");
 #pragma unroll
-                for (int g = 0; g < 16; ++g)
-                    stg[g * kTileRows] = make_float4(__uint_as_float(o[rd * 64 + 4 * g]), __uint_as_float(o[rd * 64 + 4 * g + 1]),
-                                                     __uint_as_float(o[rd * 64 + 4 * g + 2]), __uint_as_float(o[rd * 64 + 4 * g + 3]));
+                for (int g = 0; g < 4; ++g)
+                    stg[(slot * 4 + g) * kTileRows] = make_float4(__uint_as_float(o[ch * 16 + 4 * g]), __uint_as_float(o[ch * 16 + 4 * g + 1]),
+                                                                  __uint_as_float(o[ch * 16 + 4 * g + 2]), __uint_as_float(o[ch * 16 + 4 * g + 3]));
                 fence_proxy_async_smem();
                 asm volatile("bar.sync 2, 128;" ::: "memory");
-                if (tid == 256) {
+                if (tid == NROW) {
                     asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
-                                 ::"l"(dst + rd * (64 * kTileRows)), "r"(sbase + L::kStg), "r"(L::kStgBytes) : "memory");
+                                 ::"l"(dst + ch * (16 * kTileRows)), "r"(sbase + L::kStg + slot * (L::kStgBytes / 4)), "r"(L::kStgBytes / 4) : "memory");
                     tma_store_commit();
                 }
             }
         }
-        if (tid == 256) tma_store_wait_all();                // every addition has been performed before the CTA retires
-    } else if (warp < 16) {
+        if (tid == NROW) tma_store_wait_all();               // every addition has been performed before the CTA retires
+    } else {
       setmaxnreg_dec<kRegsOther>();
-      if (warp == 12) {
+      if (warp == W_LOAD) {
         // =========================== loader: TMA tiles + per-query LSE, D_t ===========================
         if (lane == 0) {
             tma_prefetch_desc(&mapK);
@@ -589,10 +606,10 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                 mbar_arrive(bar(kFBarQFull + st));
             }
         }
-      } else if (warp == 13 || warp == 14) {
+      } else if (warp == W_S || warp == W_DP) {
         // ============ MMA issuers: S^T = K Q^T (warp 13, into X), dP^T = V dO^T (warp 14, into Y) ============
         {   // whole warp: operands are warp-uniform, one elected lane issues
-            const bool is_s = (warp == 13);
+            const bool is_s = (warp == W_S);
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
             const uint32_t a_tile = sbase + (is_s ? L::kK : L::kV);
             const int full0 = is_s ? kFBarQFull : kFBardOFull;
@@ -623,12 +640,13 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
             }
             drain_on_abort(is_s ? 0 : 1);
         }
-      } else {
-        // ============ MMA issuer (warp 15): dV_i += P^T dO (P^T from tensor memory, dO MN-major), then, once dS_i^T
-        // ============ is in shared memory, dQ_tile = dS K into Y (dS^T and K both MN-major) and dK += dS^T Q (dS^T
-        // ============ K-major, Q MN-major).  P_i, dS_i, P_{i+1} are produced in this order, so one warp can take the
-        // ============ three in turn.  dQ before dK: its tile has to be copied out before dP of the next iteration can
-        // ============ land, dK only has to finish before dS_{i+1} is written.
+      } else if (warp == W_ACC) {
+        // ============ MMA issuer of the accumulating contractions: dV_i += P^T dO (P^T from tensor memory, dO MN-major),
+        // ============ then, once dS_i^T is in shared memory, dQ_tile = dS K into Y (dS^T and K both MN-major) and
+        // ============ dK += dS^T Q (dS^T K-major, Q MN-major).  P_i, dS_i, P_{i+1} are produced in this order, so one
+        // ============ warp can take the three in turn.  dQ before dK: its tile has to be copied out before dP of the next
+        // ============ iteration can land, dK only has to finish before dS_{i+1} is written.  (A warp per contraction was
+        // ============ measured at d = 64, where these are N = 64 MMAs: no faster.)
         {
             constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, false, true);
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);
@@ -643,9 +661,9 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                 tc_fence_after_sync();
                 const uint64_t dvb = dvb0 + uint64_t((dst * L::kTileBytes) >> 4);
 #pragma unroll
-                for (int kk = 0; kk < kTileRows / 16; ++kk)  // 16 queries per k-step: 8 columns, in the block of warpgroup kk / 4
-                    umma_ts(tmem + kColdV, tmem + kColX + xb * 128 + (kk >> 2) * 64 + (kk & 3) * 8, dvb + uint64_t(kk * 128), idesc_acc,
-                            (it > 0 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < kTileRows / 16; ++kk)  // 16 queries per k-step: 8 columns, in the block of the row warpgroup that owns them
+                    umma_ts(tmem + kColdV, tmem + kColX + xb * 128 + (kk / (COLS / 16)) * COLS + (kk % (COLS / 16)) * 8, dvb + uint64_t(kk * 128),
+                            idesc_acc, (it > 0 || kk > 0) ? 1u : 0u);
                 umma_commit(bar(kFBarXFree + xb));
                 umma_commit(bar(kFBardOEmpty + dst));
                 mbar_wait(bar(kFBardSFull), it & 1, abort_flag, 146);
@@ -674,7 +692,7 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         while (globaltimer_ns() - t0 < 2000000ull) {}
     }
     __syncthreads();
-    if (warp == 13) tmem_dealloc(tmem, kTmemCols);
+    if (warp == W_S) tmem_dealloc(tmem, kTmemCols);
 }
 
 }  // namespace moda

@@ -45,10 +45,12 @@ NOMINAL_BF16_TFLOPS = 2250.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes); keyed by (workload, kernel).  None where no capture exists.
-NCU_SEQ_C3_L0_B1 = 202.80e6 + 100.59e6   # dram__bytes_read.sum + dram__bytes_write.sum of that one launch
+NCU_SEQ_C3_L0_B1 = 202.50e6 + 93.82e6   # dram__bytes_read.sum + dram__bytes_write.sum of that one launch
 NCU_TRAFFIC_BYTES = {
     # c2 captured at B=1 and scaled x4 (traffic is proportional to B): profiles/ncu_full_c2_B1_fwd_bwd_kernels.md
     ("c2", "fwd_append"): 4 * (822.179e6 + 6.956e6) + 4 * 33554432 * 2,   # + the slot written (not in that capture)
+    # row-local part of the backward at c2, B = 1, scaled x4: profiles/ncu_full_c2_B1_bwd_rows_kernel.md
+    ("c2", "bwd_rows"): 4 * (822.39e6 + 746.92e6),
     # sequence part of the backward, captured at c3 with l = 0 and B = 1 (T = 8192) and scaled by the number of
     # elements B T H d (every tensor crosses HBM once, re-reads are served by L2):
     # profiles/ncu_full_c3_l0_B1_bwd_fused_kernel.md

@@ -307,3 +307,65 @@ def forward_prefill_gqa(Q, K, V, Kd, Vd, scale):
                 O[b, i, h] = (p / z) @ vals
                 LSE[b, h, i] = m + np.log(z)
     return O, LSE
+
+
+# ---------------------------------------------------------------------------------------
+# Lower-precision depth cache (the paper's Discussion names bounded / cheaper depth-KV caching
+# as a direction and gives no algorithm).  Reading taken: every depth key row and every depth value
+# row (the d features of one slot, position and head) is stored as 8-bit floats of the e4m3 kind
+# (1 sign, 4 exponent, 3 mantissa bits, bias 7, no infinities, largest finite value 448) with one
+# fp32 scale per row, scale = max|x| / 448; the operator is then the Sec. 2.2 operator on the
+# DEQUANTISED depth keys and values.  The decisions that pick an 8-bit code are taken in fp32 (the
+# scale, the division x / scale, both rounded to nearest) so that any implementation that follows
+# the same steps picks the same codes; the dequantised value code * scale is exact in float64.
+# ---------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+
+
+def e4m3_decode_table():
+    """The 256 values of the e4m3 format, from its definition (code 0x7f / 0xff, the NaN patterns, as nan)."""
+    vals = np.empty(256)
+    for code in range(256):
+        sign = -1.0 if code & 0x80 else 1.0
+        e, m = (code >> 3) & 0xF, code & 0x7
+        if e == 0xF and m == 0x7:
+            vals[code] = np.nan
+        elif e == 0:
+            vals[code] = sign * (m / 8.0) * 2.0 ** -6          # subnormals
+        else:
+            vals[code] = sign * (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return vals
+
+
+def e4m3_round(y):
+    """Codes (uint8) of float32 values rounded to the nearest e4m3 value, ties to the even mantissa, saturating at
+    +-448.  Written from the format: in the binade 2^e the representable values are 2^(e-3) apart, below 2^-6 they
+    are 2^-9 apart."""
+    y = np.asarray(y, dtype=np.float32)
+    a = np.abs(y).astype(np.float64)
+    e = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))             # binade of a (subnormals share the step of 2^-6)
+    step = 2.0 ** (e - 3)
+    q = np.rint(a / step) * step                                # rint: round half to even; a / step is exact (power of two)
+    q = np.minimum(q, E4M3_MAX)
+    # encode q (now exactly representable)
+    qe = np.floor(np.log2(np.maximum(q, 2.0 ** -6)))
+    is_sub = q < 2.0 ** -6
+    mant = np.where(is_sub, np.rint(q / 2.0 ** -9), np.rint((q / 2.0 ** qe - 1.0) * 8.0)).astype(np.int64)
+    expf = np.where(is_sub, 0, qe + 7).astype(np.int64)
+    code = (expf << 3) | mant
+    code = np.where(np.signbit(y), code | 0x80, code)
+    return code.astype(np.uint8)
+
+
+def quantize_e4m3_rows(X):
+    """Per-row e4m3 quantisation of X [..., d]: returns (codes uint8 [..., d], scale float32 [...])."""
+    X32 = np.asarray(X, dtype=np.float32)
+    amax = np.max(np.abs(X32), axis=-1)
+    scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)   # fp32 division
+    y = (X32 / scale[..., None]).astype(np.float32)                                                # fp32 division
+    return e4m3_round(y), scale
+
+
+def dequantize_e4m3_rows(codes, scale):
+    """float64 values code * scale of what quantize_e4m3_rows stored."""
+    return e4m3_decode_table()[np.asarray(codes, dtype=np.uint8)] * np.asarray(scale, dtype=np.float64)[..., None]

@@ -352,6 +352,45 @@ int moda_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, co
                                  int B, int T, int H, int d, int l, float scale,
                                  void* dQ, void* dK, void* dV, void* d_depth_kv, void* stream);
 
+/*
+ * ---- Depth cache in e4m3 with one scale per row ----
+ *
+ * The paper's Discussion names the growing depth-KV cache as the cost to cut next and gives no
+ * algorithm.  This library's reading: a slot may be kept in 8 bits per feature.  For every (slot,
+ * b, h, position, K or V) row x of d features
+ *
+ *     scale = max|x| / 448   (1 when the row is all zero),   code_j = e4m3(x_j / scale)
+ *
+ * with the maximum, the two divisions and the round-to-nearest-even, saturating conversion to e4m3
+ * (4 exponent bits, 3 mantissa bits, largest finite value 448) all in fp32.  The operator then sees the
+ * keys and values  scale * code_j  (taken as real numbers: the kernels keep the product in fp32, it is never
+ * rounded to bf16).  Relative to the bf16 cache a slot shrinks from 4 d to 2 d + 8 bytes per (position, head).
+ *
+ * Layout: cache8[slot][b][h][tile][kv] = { codes[chunk = d/16][row 128][16 bytes], scales[row 128] fp32 },
+ * one contiguous block of 128 d + 512 bytes; rows of a ragged last tile hold code 0, scale 1.
+ *
+ * moda_depth_cache_e4m3_bytes   bytes of a cache of l_max slots (0 for an unsupported shape).
+ * moda_depth_cache_append_e4m3  quantises K_i, V_i (bf16 [B][T][H][d], device) into slot `slot`.
+ * moda_attn_fwd_e4m3            moda_attn_fwd_gqa with the depth slots read from such a cache.
+ * moda_attn_bwd_e4m3            moda_attn_bwd (one key/value head per query head; the fused form, with its
+ *                               workspace of moda_bwd_workspace_bytes) with the depth slots read from such
+ *                               a cache.  The depth gradients are those with respect to the dequantised keys
+ *                               and values and are written to d_depth_kv in the bf16 cache layout
+ *                               (moda_depth_cache_bytes), like moda_attn_bwd's.
+ * Other arguments, ownership, validation and error codes as for the bf16 calls they mirror.
+ */
+size_t moda_depth_cache_e4m3_bytes(int B, int T, int H, int d, int l_max);
+int moda_depth_cache_append_e4m3(void* cache, int B, int T, int H, int d, int slot,
+                                 const void* K_i, const void* V_i, void* stream);
+int moda_attn_fwd_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,
+                       int B, int T, int H, int H_kv, int d, int l, float scale,
+                       void* O, float* LSE, void* stream);
+int moda_attn_bwd_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,
+                       const void* O, const void* dO, const float* LSE,
+                       int B, int T, int H, int d, int l, float scale,
+                       void* dQ, void* dK, void* dV, void* d_depth_kv,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -15,8 +15,10 @@ from .binding import (  # noqa: F401
     MODA_BWD_STAGE_ROWTERMS,
     ModaError,
     alloc_depth_cache,
+    alloc_depth_cache_e4m3,
     depth_cache_window,
     moda_attn_bwd,
+    moda_attn_bwd_e4m3,
     moda_attn_bwd_gqa,
     moda_attn_bwd_gqa_stages,
     moda_attn_bwd_stages,
@@ -26,12 +28,15 @@ from .binding import (  # noqa: F401
     moda_attn_decode_varlen,
     moda_attn_fwd,
     moda_attn_fwd_append,
+    moda_attn_fwd_e4m3,
     moda_attn_fwd_gqa,
     moda_attn_fwd_prefill,
     moda_bwd_workspace_bytes,
     moda_bwd_workspace_bytes_gqa,
     moda_decode_workspace_bytes,
     moda_depth_cache_append,
+    moda_depth_cache_append_e4m3,
+    moda_depth_cache_e4m3_bytes,
     moda_depth_cache_bytes,
     moda_depth_cache_unpack,
     moda_last_status,

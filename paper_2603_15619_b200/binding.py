@@ -24,6 +24,7 @@ SYMBOLS = (
     "moda_attn_fwd_gqa", "moda_bwd_workspace_bytes_gqa", "moda_attn_bwd_gqa", "moda_attn_bwd_gqa_stages",
     "moda_decode_workspace_bytes", "moda_attn_decode", "moda_attn_fwd_prefill", "moda_attn_fwd_append",
     "moda_attn_decode_varlen", "moda_attn_decode_paged",
+    "moda_depth_cache_e4m3_bytes", "moda_depth_cache_append_e4m3", "moda_attn_fwd_e4m3", "moda_attn_bwd_e4m3",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -97,6 +98,14 @@ def load() -> ctypes.CDLL:
     lib.moda_decode_workspace_bytes.argtypes = [ci] * 3
     lib.moda_attn_decode.restype = ci
     lib.moda_attn_decode.argtypes = [vp] * 4 + [ci] * 7 + [cf] + [vp] * 3 + [sz, vp]
+    lib.moda_depth_cache_e4m3_bytes.restype = sz
+    lib.moda_depth_cache_e4m3_bytes.argtypes = [ci] * 5
+    lib.moda_depth_cache_append_e4m3.restype = ci
+    lib.moda_depth_cache_append_e4m3.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp]
+    lib.moda_attn_fwd_e4m3.restype = ci
+    lib.moda_attn_fwd_e4m3.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
+    lib.moda_attn_bwd_e4m3.restype = ci
+    lib.moda_attn_bwd_e4m3.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 5 + [sz, vp]
     _lib = lib
     return lib
 
@@ -209,6 +218,58 @@ def moda_depth_cache_unpack(cache, slot, K_i, V_i, stream=None):
     B, T, H, d = _bthd(ref, "K_i/V_i")
     _check(load().moda_depth_cache_unpack(_ptr(cache), B, T, H, d, int(slot), _ptr(K_i), _ptr(V_i), _stream(stream)),
            "moda_depth_cache_unpack")
+
+
+def moda_depth_cache_e4m3_bytes(B, T, H, d, l_max) -> int:
+    return int(load().moda_depth_cache_e4m3_bytes(B, T, H, d, l_max))
+
+
+def alloc_depth_cache_e4m3(B, T, H, d, l_max, device="cuda", stream=None) -> torch.Tensor:
+    """Caller-side helper: a uint8 buffer of moda_depth_cache_e4m3_bytes() bytes (uninitialised)."""
+    n = moda_depth_cache_e4m3_bytes(B, T, H, d, l_max)
+    if n == 0 and l_max != 0:
+        raise ValueError("bad depth-cache shape")
+    return _new((max(n, 16),), torch.uint8, device, stream)
+
+
+def moda_depth_cache_append_e4m3(cache, slot, K_i, V_i, stream=None):
+    """Quantise K_i, V_i (bf16 [B,T,H,d]) into slot ``slot`` of an e4m3 depth cache (codes + one fp32 scale per row)."""
+    B, T, H, d = _bthd(K_i, "K_i")
+    assert _bthd(V_i, "V_i") == (B, T, H, d)
+    _check(load().moda_depth_cache_append_e4m3(_ptr(cache), B, T, H, d, int(slot), _ptr(K_i), _ptr(V_i), _stream(stream)),
+           "moda_depth_cache_append_e4m3")
+
+
+def moda_attn_fwd_e4m3(Q, K, V, depth_kv_e4m3, l, scale, O=None, LSE=None, stream=None):
+    """moda_attn_fwd_gqa with the depth slots read from an e4m3 cache."""
+    B, T, H, Hk, d = _gqa_shapes(Q, K, V)
+    if O is None:
+        O = _new_like(Q, stream)
+    if LSE is None:
+        LSE = _new((B, H, T), torch.float32, Q.device, stream)
+    _check(load().moda_attn_fwd_e4m3(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv_e4m3) if l > 0 else None,
+                                     B, T, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE), _stream(stream)),
+           "moda_attn_fwd_e4m3")
+    return O, LSE
+
+
+def moda_attn_bwd_e4m3(Q, K, V, depth_kv_e4m3, O, dO, LSE, l, scale,
+                       dQ=None, dK=None, dV=None, d_depth_kv=None, workspace=None, stream=None):
+    """moda_attn_bwd with the depth slots read from an e4m3 cache; the depth gradients come back in the bf16 cache layout."""
+    B, T, H, d = _bthd(Q, "Q")
+    dQ = _new_like(Q, stream) if dQ is None else dQ
+    dK = _new_like(K, stream) if dK is None else dK
+    dV = _new_like(V, stream) if dV is None else dV
+    if l > 0 and d_depth_kv is None:
+        d_depth_kv = alloc_depth_cache(B, T, H, d, l, Q.device, stream)
+    if workspace is None:
+        workspace = _new((moda_bwd_workspace_bytes(B, T, H, d, l),), torch.uint8, Q.device, stream)
+    _check(load().moda_attn_bwd_e4m3(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv_e4m3) if l > 0 else None,
+                                     _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, d, int(l), float(scale),
+                                     _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv) if l > 0 else None,
+                                     _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "moda_attn_bwd_e4m3")
+    return dQ, dK, dV, d_depth_kv
 
 
 def moda_attn_fwd(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):

@@ -208,11 +208,19 @@ int launch_depth_merge(DepthMergeParams m, cudaStream_t stream) {
     }
 }
 
+// Dynamic shared memory of the forward kernel that reads an e4m3 depth cache (only the variant each head size runs exists).
+template <int D>
+constexpr int fwd_smem_e4m3() {
+    if constexpr (D == 64) return Fwd2Smem<64, true>::kDynamic;
+    else return FwdSmem<128, 2, true>::kDynamic;
+}
+
 template <int D>
 int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int T_kv, int H, int Hk, int l,
-               float scale, void* O, float* LSE, void* append_slot, cudaStream_t stream) {
+               float scale, void* O, float* LSE, void* append_slot, cudaStream_t stream, bool fp8 = false) {
     constexpr bool kWide = (D == 64);
     constexpr int kSmem = kWide ? Fwd2Smem<D>::kDynamic : FwdSmem<D, 2>::kDynamic;
+    constexpr int kSmem8 = fwd_smem_e4m3<D>();
     constexpr int kSmemDeep = FwdSmem<128, 1>::kDynamic;
     constexpr int kThreads = kWide ? kFwd2Threads : kFwdThreads;
     CUtensorMap mQ, mK, mV, mO;
@@ -223,13 +231,15 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
     if (configured_dev != dev) {
-        const bool ok = kWide ? set_smem_limit(moda_fwd2_kernel<D>, kSmem)
-                              : set_smem_limit(moda_fwd_kernel<D, 2>, kSmem) && set_smem_limit(moda_fwd_kernel<128, 1>, kSmemDeep);
+        bool ok;
+        if constexpr (kWide) ok = set_smem_limit(moda_fwd2_kernel<D>, kSmem) && set_smem_limit(moda_fwd2_kernel<D, true>, kSmem8);
+        else ok = set_smem_limit(moda_fwd_kernel<D, 2>, kSmem) && set_smem_limit(moda_fwd_kernel<128, 1>, kSmemDeep) &&
+                  set_smem_limit(moda_fwd_kernel<128, 2, true>, kSmem8);
         if (!ok) return MODA_ERR_CUDA;
         configured_dev = dev;
     }
     FwdParams p;
-    p.depth_kv = static_cast<const __nv_bfloat16*>(depth_kv);
+    p.depth_kv = depth_kv;
     p.O = static_cast<__nv_bfloat16*>(O);
     p.LSE = LSE;
     p.B = B; p.T = T; p.H = H; p.l = l;
@@ -240,9 +250,13 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     const unsigned grid = unsigned(B) * H * num_tiles(T);
     // Grouped-query calls: the sequence kernel runs without depth slots and a second kernel adds the depth
     // part of all heads of a group at once (moda_depth_gqa.cuh).
-    const bool split_depth = gqa_depth_split(D, p.G, l);
+    // An e4m3 cache is always read by the row-local depth warps of the sequence kernel.
+    const bool split_depth = !fp8 && gqa_depth_split(D, p.G, l);
     if (split_depth) p.l = 0;
-    if (kWide) moda_fwd2_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
+    if (fp8) {
+        if constexpr (kWide) moda_fwd2_kernel<D, true><<<grid, kThreads, kSmem8, stream>>>(mQ, mK, mV, mO, p);
+        else moda_fwd_kernel<128, 2, true><<<grid, kThreads, kSmem8, stream>>>(mQ, mK, mV, mO, p);
+    } else if (kWide) moda_fwd2_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
     else if (!split_depth && fwd_depth_heavy(T, l, D)) moda_fwd_kernel<128, 1><<<grid, kThreads, kSmemDeep, stream>>>(mQ, mK, mV, mO, p);
     else moda_fwd_kernel<D, 2><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
     if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
@@ -350,13 +364,14 @@ int launch_bwd_fused(const BwdArgs& a, int stages, cudaStream_t stream) {
         r.Q = static_cast<const __nv_bfloat16*>(a.Q);
         r.O = static_cast<const __nv_bfloat16*>(a.O);
         r.dO = static_cast<const __nv_bfloat16*>(a.dO);
-        r.depth_kv = static_cast<const __nv_bfloat16*>(a.depth_kv);
+        r.depth_kv = a.depth_kv;
         r.d_depth_kv = static_cast<__nv_bfloat16*>(a.d_depth_kv);
         r.LSE = a.LSE; r.delta = delta; r.dq_acc = dq_acc;
         r.B = B; r.T = T; r.H = H; r.l = split_depth ? 0 : a.l;
         r.accumulate = a.accumulate_depth ? 1 : 0;
         r.scale = a.scale; r.scale_log2 = a.scale * kLog2e;
-        bwd_rows_kernel<D><<<tiles, kRowThreads, 0, stream>>>(r);
+        if (a.fp8_cache) bwd_rows_kernel<D, true><<<tiles, kRowThreads, 0, stream>>>(r);
+        else bwd_rows_kernel<D><<<tiles, kRowThreads, 0, stream>>>(r);
         if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     }
     if (stages & 2) {
@@ -780,6 +795,69 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
     a.accumulate_depth = (stages & MODA_BWD_ACCUMULATE_DEPTH) != 0;
     return d == 128 ? launch_bwd<128>(a, stages, st) : launch_bwd<64>(a, stages, st);
+}
+
+// ---- depth cache in e4m3 with a scale per row ----
+size_t moda_depth_cache_e4m3_bytes(int B, int T, int H, int d, int l_max) {
+    if (check_shape(B, T, H, d) != MODA_OK || l_max < 0 || l_max > MODA_MAX_DEPTH) return 0;
+    return size_t(l_max) * cache8_slot_bytes(B, T, H, d);
+}
+
+int moda_depth_cache_append_e4m3(void* cache, int B, int T, int H, int d, int slot,
+                                 const void* K_i, const void* V_i, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (slot < 0 || slot >= MODA_MAX_DEPTH) return MODA_ERR_BAD_SLOT;
+    if (!cache || !K_i || !V_i) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(cache) || !aligned16(K_i) || !aligned16(V_i)) return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* base = static_cast<uint8_t*>(cache) + size_t(slot) * cache8_slot_bytes(B, T, H, d);
+    const unsigned grid = unsigned(B) * H * num_tiles(T) * 2;
+    if (d == 128)
+        depth_cache_quant_kernel<128><<<grid, 256, 0, st>>>(base, static_cast<const uint4*>(K_i), static_cast<const uint4*>(V_i), T, H);
+    else
+        depth_cache_quant_kernel<64><<<grid, 256, 0, st>>>(base, static_cast<const uint4*>(K_i), static_cast<const uint4*>(V_i), T, H);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+
+int moda_attn_fwd_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,
+                       int B, int T, int H, int H_kv, int d, int l, float scale,
+                       void* O, float* LSE, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_groups(H, H_kv)) return rc;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (!Q || !K || !V || !O || !LSE || (l > 0 && !depth_kv_e4m3)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
+        (l > 0 && !aligned16(depth_kv_e4m3)))
+        return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, true)
+                    : launch_fwd<64>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, true);
+}
+
+int moda_attn_bwd_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,
+                       const void* O, const void* dO, const float* LSE,
+                       int B, int T, int H, int d, int l, float scale,
+                       void* dQ, void* dK, void* dV, void* d_depth_kv,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv_e4m3 || !d_depth_kv)))
+        return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(LSE) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) ||
+        (l > 0 && (!aligned16(depth_kv_e4m3) || !aligned16(d_depth_kv))))
+        return MODA_ERR_MISALIGNED;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < bwd_fused_workspace_bytes(B, T, H, d)) return MODA_ERR_WORKSPACE;
+    if (int rc = check_device()) return rc;
+    BwdArgs a;
+    a.fp8_cache = true;
+    a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv_e4m3; a.O = O; a.dO = dO; a.LSE = LSE;
+    a.B = B; a.T = T; a.H = H; a.Hk = H; a.l = l; a.scale = scale;
+    a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_bwd_fused<128>(a, MODA_BWD_ALL_STAGES, st) : launch_bwd_fused<64>(a, MODA_BWD_ALL_STAGES, st);
 }
 
 size_t moda_decode_workspace_bytes(int B, int H, int d) {

@@ -30,7 +30,7 @@
 #include "moda_bwd.cuh"
 #include "moda_cache.cuh"
 #include "moda_fwd.cuh"
-#include "moda_fwd_wide.cuh"   // aligned_dynamic_smem
+#include "moda_fwd_wide.cuh"
 #include "sm100_ptx.cuh"
 
 namespace moda {
@@ -57,7 +57,8 @@ inline size_t bwd_fused_workspace_bytes(int B, int T, int H, int d) {
 // to the cache is a set of 128-byte (d = 128) or 256-byte (d = 64) runs.  q and dO stay packed in
 // registers; a slot's key and value chunks are read once and used for everything the slot needs.
 struct RowsParams {
-    const __nv_bfloat16 *Q, *O, *dO, *depth_kv;
+    const __nv_bfloat16 *Q, *O, *dO;
+    const void* depth_kv;   // bf16 cache, or e4m3 codes + row scales (FP8 instantiation); gradients are bf16 either way
     __nv_bfloat16* d_depth_kv;
     const float* LSE;
     float* delta;        // [B][H][T]
@@ -67,7 +68,7 @@ struct RowsParams {
     float scale, scale_log2;
 };
 
-template <int D>
+template <int D, bool FP8 = false>
 __global__ void __launch_bounds__(kTileRows * (D / 32), 512 / (kTileRows * (D / 32)))
 bwd_rows_kernel(const RowsParams p) {
     constexpr int PARTS = D / 32;                 // threads per row
@@ -110,6 +111,81 @@ bwd_rows_kernel(const RowsParams p) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) acc[i] = 0.f;
 
+    if (FP8 && p.l > 0) {
+        // e4m3 cache: this thread's 32 features are two 16-byte chunks of codes; the row's scale is one float per slot
+        // for K and one for V.  Gradients are taken with respect to the dequantised keys and values.
+        const size_t slot_stride = cache_slot_elems(p.B, p.T, p.H, D) / 8;                    // gradient cache, in uint4
+        const size_t gblk = (size_t(bh) * nq + qt) * 2 * (kTileRows * CH) + size_t(part * 4) * kTileRows + r;
+        uint4* gK = reinterpret_cast<uint4*>(p.d_depth_kv) + gblk;
+        uint4* gV = gK + kTileRows * CH;
+        const size_t slot_bytes8 = cache8_slot_bytes(p.B, p.T, p.H, D), blk_bytes8 = cache8_block_bytes(D);
+        const uint8_t* cK = reinterpret_cast<const uint8_t*>(p.depth_kv) + (size_t(bh) * nq + qt) * 2 * blk_bytes8;
+        const bool accumulate = p.accumulate != 0;
+#pragma unroll 1
+        for (int i = 0; i < p.l; ++i) {
+            const uint8_t* cV = cK + blk_bytes8;
+            uint4 k8[2], v8[2];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                k8[j] = __ldcs(reinterpret_cast<const uint4*>(cK) + size_t(part * 2 + j) * kTileRows + r);
+                v8[j] = __ldcs(reinterpret_cast<const uint4*>(cV) + size_t(part * 2 + j) * kTileRows + r);
+            }
+            const float sk = __ldcs(reinterpret_cast<const float*>(cK + size_t(kTileRows) * D) + r);
+            const float sv = __ldcs(reinterpret_cast<const float*>(cV + size_t(kTileRows) * D) + r);
+            float kf[32];
+            float u = 0.f, dr = 0.f;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const uint32_t kw[4] = {k8[j].x, k8[j].y, k8[j].z, k8[j].w}, vw[4] = {v8[j].x, v8[j].y, v8[j].z, v8[j].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    float v0, v1, v2, v3;
+                    e4m3x4_to_f32(kw[k], kf[16 * j + 4 * k], kf[16 * j + 4 * k + 1], kf[16 * j + 4 * k + 2], kf[16 * j + 4 * k + 3]);
+                    e4m3x4_to_f32(vw[k], v0, v1, v2, v3);
+                    // features 16 j + 4 k .. + 3 of this thread = halves of the packed q / dO words 2 (4 j + k), 2 (4 j + k) + 1
+                    const uint32_t* qw = reinterpret_cast<const uint32_t*>(q4) + 2 * (4 * j + k);
+                    const uint32_t* gw = reinterpret_cast<const uint32_t*>(g4) + 2 * (4 * j + k);
+                    u = fmaf(bf16_lo_to_f32(qw[0]), kf[16 * j + 4 * k], u);
+                    u = fmaf(bf16_hi_to_f32(qw[0]), kf[16 * j + 4 * k + 1], u);
+                    u = fmaf(bf16_lo_to_f32(qw[1]), kf[16 * j + 4 * k + 2], u);
+                    u = fmaf(bf16_hi_to_f32(qw[1]), kf[16 * j + 4 * k + 3], u);
+                    dr = fmaf(bf16_lo_to_f32(gw[0]), v0, dr);
+                    dr = fmaf(bf16_hi_to_f32(gw[0]), v1, dr);
+                    dr = fmaf(bf16_lo_to_f32(gw[1]), v2, dr);
+                    dr = fmaf(bf16_hi_to_f32(gw[1]), v3, dr);
+                }
+            }
+#pragma unroll
+            for (int off = 1; off < PARTS; off <<= 1) {
+                u += __shfl_xor_sync(0xffffffffu, u, off);
+                dr += __shfl_xor_sync(0xffffffffu, dr, off);
+            }
+            const float R = fast_exp2(fmaf(u * sk, p.scale_log2, neg_lse2));
+            const float dU = R * (dr * sv - delta);
+            const uint32_t r2 = pack_bf16x2(R, R);
+            const float sdu = dU * p.scale;
+            const uint32_t sdu2 = pack_bf16x2(sdu, sdu);
+            const float duk = dU * sk;                        // dQ share: dU * (scale_k * code)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint4 ov, ok;
+                ov.x = mul_bf16x2(g4[j].x, r2); ov.y = mul_bf16x2(g4[j].y, r2);
+                ov.z = mul_bf16x2(g4[j].z, r2); ov.w = mul_bf16x2(g4[j].w, r2);
+                ok.x = mul_bf16x2(q4[j].x, sdu2); ok.y = mul_bf16x2(q4[j].y, sdu2);
+                ok.z = mul_bf16x2(q4[j].z, sdu2); ok.w = mul_bf16x2(q4[j].w, sdu2);
+                if (accumulate) {
+                    red_add_bf16x2_v4(gV + j * kTileRows, ov);
+                    red_add_bf16x2_v4(gK + j * kTileRows, ok);
+                } else {
+                    __stcs(gV + j * kTileRows, ov);
+                    __stcs(gK + j * kTileRows, ok);
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[8 * j + e] = fmaf(duk, kf[8 * j + e], acc[8 * j + e]);
+            }
+            cK += slot_bytes8; gK += slot_stride; gV += slot_stride;
+        }
+    } else
     if (p.l > 0) {
         const size_t slot_stride = cache_slot_elems(p.B, p.T, p.H, D) / 8;                    // in uint4
         const size_t blk = (size_t(bh) * nq + qt) * 2 * (kTileRows * CH) + size_t(part * 4) * kTileRows + r;

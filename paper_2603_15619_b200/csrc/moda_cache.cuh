@@ -73,3 +73,82 @@ depth_cache_copy_kernel(uint4* __restrict__ cache_slot,            // base of th
 }
 
 }  // namespace moda
+
+// =====================================================================================
+// Lower-precision depth cache: e4m3 codes with one fp32 scale per row
+// =====================================================================================
+// (The paper's Discussion names cheaper depth-KV caching as a direction and gives no algorithm; the format
+// here -- scale = max|x| / 448 per (slot, position, head, K or V) row, codes = round-to-nearest-even of
+// x / scale, both in fp32 -- is this library's reading.)
+//
+//   cache8[slot][b][h][tile][kv] = { codes[chunk = d/16][row 128][16 bytes], scales[row 128] fp32 }
+//
+// A block is one contiguous run of 128 d + 512 bytes: 128 d bytes of codes in the same chunk-major, row-interleaved
+// order as the bf16 cache (a chunk now holds 16 features), then the 128 row scales.
+namespace moda {
+
+__host__ __device__ inline size_t cache8_block_bytes(int d) { return size_t(kTileRows) * d + size_t(kTileRows) * 4; }
+__host__ __device__ inline size_t cache8_slot_bytes(int B, int T, int H, int d) {
+    return size_t(B) * H * num_tiles(T) * 2 * cache8_block_bytes(d);
+}
+
+// One CTA quantises one (b, h, tile, kv) block of a [B][T][H][d] tensor into a slot.  256 threads: thread
+// (row r, half hf) owns d/2 features of its row; the two halves of a row meet in shared memory for the row maximum.
+template <int D>
+__global__ void __launch_bounds__(256)
+depth_cache_quant_kernel(uint8_t* __restrict__ slot_base, const uint4* __restrict__ Xk, const uint4* __restrict__ Xv, int T, int H) {
+    constexpr int CH = D / 8;                       // 16-byte chunks (8 bf16) per input row
+    __shared__ uint4 tile[kTileRows * (CH + 1)];
+    __shared__ float amax2[2][kTileRows];
+    const int ntile = num_tiles(T);
+    int bid = blockIdx.x;
+    const int kv = bid & 1; bid >>= 1;
+    const int tl = bid % ntile; bid /= ntile;
+    const int h = bid % H;
+    const int b = bid / H;
+    const uint4* X = kv ? Xv : Xk;
+    uint8_t* blk = slot_base + (((size_t(b) * H + h) * ntile + tl) * 2 + kv) * cache8_block_bytes(D);
+    const int t0 = tl * kTileRows;
+    for (int i = threadIdx.x; i < kTileRows * CH; i += 256) {
+        const int row = i / CH, ch = i % CH;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (t0 + row < T) v = X[((size_t(b) * T + t0 + row) * H + h) * CH + ch];
+        tile[row * (CH + 1) + ch] = v;
+    }
+    __syncthreads();
+    const int r = threadIdx.x & 127, hf = threadIdx.x >> 7;
+    constexpr int HCH = CH / 2;                     // input chunks of this thread's half row
+    float x[D / 2];
+#pragma unroll
+    for (int c = 0; c < HCH; ++c) {
+        const uint4 v = tile[r * (CH + 1) + hf * HCH + c];
+        x[8 * c + 0] = __uint_as_float(v.x << 16); x[8 * c + 1] = __uint_as_float(v.x & 0xffff0000u);
+        x[8 * c + 2] = __uint_as_float(v.y << 16); x[8 * c + 3] = __uint_as_float(v.y & 0xffff0000u);
+        x[8 * c + 4] = __uint_as_float(v.z << 16); x[8 * c + 5] = __uint_as_float(v.z & 0xffff0000u);
+        x[8 * c + 6] = __uint_as_float(v.w << 16); x[8 * c + 7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+    float am = 0.f;
+#pragma unroll
+    for (int i = 0; i < D / 2; ++i) am = fmaxf(am, fabsf(x[i]));
+    amax2[hf][r] = am;
+    __syncthreads();
+    am = fmaxf(amax2[0][r], amax2[1][r]);
+    const float scale = am > 0.f ? __fdiv_rn(am, 448.f) : 1.f;
+    uint4* codes = reinterpret_cast<uint4*>(blk);
+#pragma unroll
+    for (int g = 0; g < D / 32; ++g) {              // 16 features per output chunk
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float* xx = x + 16 * g + 4 * k;
+            uint16_t lo, hi;
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(xx[1], scale)), "f"(__fdiv_rn(xx[0], scale)));
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(xx[3], scale)), "f"(__fdiv_rn(xx[2], scale)));
+            w[k] = uint32_t(lo) | (uint32_t(hi) << 16);
+        }
+        codes[size_t(hf * (D / 32) + g) * kTileRows + r] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    if (hf == 0) reinterpret_cast<float*>(blk + size_t(kTileRows) * D)[r] = scale;
+}
+
+}  // namespace moda

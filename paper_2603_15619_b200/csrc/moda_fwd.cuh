@@ -43,7 +43,9 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 // KST = stages of the K ring.  Two let K_{j+1} load while S_j is still being computed; one (the
 // load starts when S_j completes and overlaps the softmax of tile j) leaves room for a deeper depth
 // ring, for shapes whose depth stream outweighs the sequence work (the host picks, see launch_fwd).
-template <int D, int KST = 2>
+// FP8: the depth cache holds e4m3 codes with a scale per row (moda_cache.cuh); a unit is then all d features of one
+// slot's keys (or values) of the tile, and its 128 row scales travel beside it.
+template <int D, int KST = 2, bool FP8 = false>
 struct FwdSmem {
     static constexpr int kTileBytes = kTileRows * D * 2;          // one 128 x D bf16 tile
     static constexpr int kSubBytes = kTileRows * 128;             // one 128 x 64 sub-tile
@@ -54,16 +56,21 @@ struct FwdSmem {
     static constexpr int kU = kV + 2 * kTileBytes;                // depth scores [32][128] fp32
     static constexpr int kMd = kU + 32 * kTileRows * 4;           // m_d [128], l_d [128]
     static constexpr int kRing = kMd + 2 * kTileRows * 4;         // depth units: 8 chunks x 128 rows x 16 B
-    static constexpr int kUnitBytes = 8 * kTileRows * 16;         // 16 KiB, contiguous in the depth cache
+    static constexpr int kUnitBytes = FP8 ? kTileRows * D : 8 * kTileRows * 16;   // 16 KiB (bf16, and e4m3 at d = 128), contiguous in the cache
+    static constexpr int kScaleBytes = FP8 ? kTileRows * 4 : 0;   // row scales of a unit
     static constexpr int kNumBars = 32;
     static constexpr int kSmemLimit = 232448;                     // 227 KiB per CTA on sm_100
-    static constexpr int kRingFit = (kSmemLimit - 1024 - kRing - kNumBars * 8 - 16) / kUnitBytes;
+    // bf16: 1024 bytes of slack for aligning the segment by hand; e4m3: no slack (the scales need it), the segment
+    // is declared 1024-aligned and checked at run time
+    static constexpr int kSlack = FP8 ? 0 : 1024;
+    static constexpr int kRingFit = (kSmemLimit - kSlack - kRing - kNumBars * 8 - 16) / (kUnitBytes + kScaleBytes);
     static constexpr int kRingStages = kRingFit < 6 ? kRingFit : 6;   // every unit that fits, at most 6
     static_assert(kRingStages >= 3, "depth ring too shallow");
-    static constexpr int kBars = kRing + kRingStages * kUnitBytes;
+    static constexpr int kScale = kRing + kRingStages * kUnitBytes;   // [ring stage][128] fp32 (e4m3 only)
+    static constexpr int kBars = kScale + kRingStages * kScaleBytes;
     static constexpr int kMisc = kBars + kNumBars * 8;            // tmem base, abort flag
     static constexpr int kTotal = kMisc + 16;
-    static constexpr int kDynamic = kTotal + 1024;                // slack for 1024-byte alignment
+    static constexpr int kDynamic = kTotal + kSlack;
 };
 
 enum FwdBar : int {
@@ -85,7 +92,7 @@ enum FwdBar : int {
 constexpr int kFwdDepthGroup = 32;
 
 struct FwdParams {
-    const __nv_bfloat16* depth_kv;   // cache layout, >= l slots (unused when l == 0)
+    const void* depth_kv;            // cache layout (bf16, or e4m3 codes + scales), >= l slots (unused when l == 0)
     __nv_bfloat16* O;
     float* LSE;
     int B, T, H, l;                  // T query positions, H query heads
@@ -140,20 +147,24 @@ __device__ __forceinline__ void append_rows_to_slot(__nv_bfloat16* slot, const u
     }
 }
 
-template <int D, int KST = 2>
+template <int D, int KST = 2, bool FP8 = false>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                 const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
                 const FwdParams p) {
-    using L = FwdSmem<D, KST>;
+    using L = FwdSmem<D, KST, FP8>;
     constexpr int NSUB = D / 64;
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColO = 256, kColOd = 384;
 
     if (g_moda_status != 0) return;   // an earlier kernel gave up a wait: do not pile up more timeouts
 
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = aligned_dynamic_smem(smem_raw, L::kTotal);
+    if (smem == nullptr) {
+        if (threadIdx.x == 0) atomicCAS(&g_moda_status, 0, kStatusSmemLayout);
+        return;
+    }
     const uint32_t sbase = smem_u32(smem);
     float* sU = reinterpret_cast<float*>(smem + L::kU);
     float* sMd = reinterpret_cast<float*>(smem + L::kMd);
@@ -369,6 +380,113 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             // online softmax over the groups, with the partial output o_d rescaled in TMEM when a later
             // group raises the maximum.  Up to 32 slots are one group.
             float m_d = -INFINITY, l_d = 0.f;
+            if constexpr (FP8) {
+                // e4m3 cache: a unit holds all D features of one slot's keys (values) for the tile's rows, its row
+                // scales sit beside it; codes are widened to fp32 in registers, everything else as below.
+                constexpr int C8 = D / 16;                    // 16-byte chunks (16 codes) of a row
+                const float* sScale = reinterpret_cast<const float*>(smem + L::kScale);
+                auto take_unit8 = [&](uint4 (&dst)[C8], float& sc) {
+                    const int st = unit % L::kRingStages;
+                    mbar_wait(bar(kBarDFull + st), (unit / L::kRingStages) & 1, abort_flag, 21);
+                    const uint8_t* src = smem + L::kRing + st * L::kUnitBytes + r * 16;
+#pragma unroll
+                    for (int c = 0; c < C8; ++c) dst[c] = *reinterpret_cast<const uint4*>(src + c * (kTileRows * 16));
+                    sc = sScale[st * kTileRows + r];
+                    fence_proxy_async_smem();
+                    mbar_arrive(bar(kBarDEmpty + st));
+                    ++unit;
+                };
+#pragma unroll 1
+                for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
+                    const int gl = min(kFwdDepthGroup, p.l - g0);
+                    {   // ---- depth scores u_i = s_i <q, codes_i> ----
+                        float q[D];
+#pragma unroll
+                        for (int c = 0; c < D / 8; ++c) {
+                            const uint4 v = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, c));
+                            q[8 * c + 0] = bf16_lo_to_f32(v.x); q[8 * c + 1] = bf16_hi_to_f32(v.x);
+                            q[8 * c + 2] = bf16_lo_to_f32(v.y); q[8 * c + 3] = bf16_hi_to_f32(v.y);
+                            q[8 * c + 4] = bf16_lo_to_f32(v.z); q[8 * c + 5] = bf16_hi_to_f32(v.z);
+                            q[8 * c + 6] = bf16_lo_to_f32(v.w); q[8 * c + 7] = bf16_hi_to_f32(v.w);
+                        }
+#pragma unroll 1
+                        for (int i = 0; i < gl; ++i) {
+                            uint4 cur[C8];
+                            float sc;
+                            take_unit8(cur, sc);
+                            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < C8; ++c) {
+                                const uint32_t w[4] = {cur[c].x, cur[c].y, cur[c].z, cur[c].w};
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    float f0, f1, f2, f3;
+                                    e4m3x4_to_f32(w[k], f0, f1, f2, f3);
+                                    a0 = fmaf(q[16 * c + 4 * k + 0], f0, a0);
+                                    a1 = fmaf(q[16 * c + 4 * k + 1], f1, a1);
+                                    a2 = fmaf(q[16 * c + 4 * k + 2], f2, a2);
+                                    a3 = fmaf(q[16 * c + 4 * k + 3], f3, a3);
+                                }
+                            }
+                            sU[i * kTileRows + r] = ((a0 + a1) + (a2 + a3)) * sc;
+                        }
+                    }
+                    float m_new = m_d;
+                    for (int i = 0; i < gl; ++i) m_new = fmaxf(m_new, sU[i * kTileRows + r] * p.scale_log2);
+                    const float f = fast_exp2(m_d - m_new);       // first group: exp2(-inf) = 0
+                    l_d *= f;
+                    for (int i = 0; i < gl; ++i) {
+                        const float w = fast_exp2(fmaf(sU[i * kTileRows + r], p.scale_log2, -m_new));
+                        sU[i * kTileRows + r] = w;
+                        l_d += w;
+                    }
+                    m_d = m_new;
+                    {   // ---- o_d = sum_i (w_i s_i) codes_i, parked in TMEM ----
+                        float acc[D];
+                        if (g0 == 0) {
+#pragma unroll
+                            for (int c = 0; c < D; ++c) acc[c] = 0.f;
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < D / 32; ++c) {
+                                uint32_t o[32];
+                                tmem_ld32(tmem + lane_addr + kColOd + c * 32, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) acc[32 * c + i] = __uint_as_float(o[i]) * f;
+                            }
+                        }
+#pragma unroll 1
+                        for (int i = 0; i < gl; ++i) {
+                            uint4 cur[C8];
+                            float sc;
+                            take_unit8(cur, sc);
+                            const float w = sU[i * kTileRows + r] * sc;
+#pragma unroll
+                            for (int c = 0; c < C8; ++c) {
+                                const uint32_t ww[4] = {cur[c].x, cur[c].y, cur[c].z, cur[c].w};
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    float f0, f1, f2, f3;
+                                    e4m3x4_to_f32(ww[k], f0, f1, f2, f3);
+                                    acc[16 * c + 4 * k + 0] = fmaf(w, f0, acc[16 * c + 4 * k + 0]);
+                                    acc[16 * c + 4 * k + 1] = fmaf(w, f1, acc[16 * c + 4 * k + 1]);
+                                    acc[16 * c + 4 * k + 2] = fmaf(w, f2, acc[16 * c + 4 * k + 2]);
+                                    acc[16 * c + 4 * k + 3] = fmaf(w, f3, acc[16 * c + 4 * k + 3]);
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t o[32];
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(acc[32 * c + i]);
+                            tmem_st32(tmem + lane_addr + kColOd + c * 32, o);
+                        }
+                        tmem_wait_st();                          // a later group reads these columns back
+                    }
+                }
+            } else {
 #pragma unroll 1
             for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
                 const int gl = min(kFwdDepthGroup, p.l - g0);
@@ -459,6 +577,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                     }
                     tmem_wait_st();                          // a later group reads these columns back
                 }
+            }
             }
             sMd[r] = m_d;
             sLd[r] = l_d;
@@ -565,7 +684,27 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         // Streams the tile's depth keys, then values, as 16 KiB units (8 feature chunks of one slot:
         // one contiguous run of the cache) through the ring, in the order the depth warps consume
         // them.  The ring keeps up to kRingStages x 16 KiB of HBM reads in flight per SM.
-        if (lane == 0 && p.l > 0) {
+        if (FP8 && lane == 0 && p.l > 0) {
+            // e4m3 cache: one unit per (slot, K or V): the block's codes, and its 128 row scales behind them
+            const uint64_t policy = l2_policy_evict_first();
+            const size_t slot_bytes = cache8_slot_bytes(p.B, p.T, Hk, D);
+            const size_t blk_bytes = cache8_block_bytes(D);
+            const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) + (((size_t(b) * Hk + hk) * nq + qt) * 2) * blk_bytes;
+            int unit = 0;
+            for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
+                const int gl = min(kFwdDepthGroup, p.l - g0);
+                for (int kv = 0; kv < 2; ++kv)
+                    for (int i = 0; i < gl; ++i, ++unit) {
+                        const int st = unit % L::kRingStages;
+                        if (unit >= L::kRingStages)
+                            mbar_wait(bar(kBarDEmpty + st), ((unit / L::kRingStages) - 1) & 1, abort_flag, 32);
+                        mbar_arrive_expect_tx(bar(kBarDFull + st), L::kUnitBytes + L::kScaleBytes);
+                        const uint8_t* src = blk + size_t(g0 + i) * slot_bytes + size_t(kv) * blk_bytes;
+                        bulk_load(sbase + L::kRing + st * L::kUnitBytes, src, L::kUnitBytes, bar(kBarDFull + st), policy);
+                        bulk_load(sbase + L::kScale + st * L::kScaleBytes, src + L::kUnitBytes, L::kScaleBytes, bar(kBarDFull + st), policy);
+                    }
+            }
+        } else if (lane == 0 && p.l > 0) {
             const uint64_t policy = l2_policy_evict_first();          // the depth cache is read exactly once
             const size_t slot_bytes = cache_slot_elems(p.B, p.T, Hk, D) * 2;
             const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +

@@ -37,7 +37,7 @@ constexpr int kFwd2Threads = 512;
 constexpr int kMaxDynamicSmem = 232448;     // 227 KiB: the most one CTA can have on sm_100
 constexpr int kFwdBN = 128;                 // keys per inner tile
 
-template <int D>
+template <int D, bool FP8 = false>
 struct Fwd2Smem {
     static constexpr int kTileBytes = kTileRows * D * 2;          // one 128 x D bf16 tile
     static constexpr int kSubBytes = kTileRows * 128;             // one 128 x 64 sub-tile
@@ -54,9 +54,13 @@ struct Fwd2Smem {
     static constexpr int kMref = kMd + 2 * kTileRows * 4;         // shared reference maximum [128]
     static constexpr int kLx = kMref + kTileRows * 4;             // partial row sums of warpgroup B [128]
     static constexpr int kRing = kLx + kTileRows * 4;             // depth units: 8 chunks x 128 rows x 16 B
-    static constexpr int kUnitBytes = 8 * kTileRows * 16;         // 16 KiB, contiguous in the depth cache
+    // bf16 cache: 16 KiB units (8 feature chunks of one slot); e4m3 cache: all d features of one slot (128 d bytes)
+    // with the 128 row scales beside them (moda_cache.cuh)
+    static constexpr int kUnitBytes = FP8 ? kTileRows * D : 8 * kTileRows * 16;
+    static constexpr int kScaleBytes = FP8 ? kTileRows * 4 : 0;
     static constexpr int kRingStages = (D == 128) ? 3 : 5;
-    static constexpr int kBars = kRing + kRingStages * kUnitBytes;
+    static constexpr int kScale = kRing + kRingStages * kUnitBytes;   // [ring stage][128] fp32 (e4m3 only)
+    static constexpr int kBars = kScale + kRingStages * kScaleBytes;
     static constexpr int kNumBars = 48;
     static constexpr int kMisc = kBars + kNumBars * 8;            // tmem base, abort flag
     static constexpr int kTotal = kMisc + 16;
@@ -84,21 +88,12 @@ enum Fwd2Bar : int {
 
 
 
-// 1024-aligned start of the dynamic shared-memory segment, or nullptr if `need` bytes do not fit
-// behind it (reported through the status word by the caller).
-__device__ __forceinline__ uint8_t* aligned_dynamic_smem(uint8_t* raw, uint32_t need) {
-    uint8_t* p = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
-    uint32_t dyn;
-    asm volatile("mov.u32 %0, %dynamic_smem_size;" : "=r"(dyn));
-    return (uint32_t(p - raw) + need <= dyn) ? p : nullptr;
-}
-
-template <int D>
+template <int D, bool FP8 = false>
 __global__ void __launch_bounds__(kFwd2Threads, 1)
 moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                 const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
                 const FwdParams p) {
-    using L = Fwd2Smem<D>;
+    using L = Fwd2Smem<D, FP8>;
     constexpr int NSUB = D / 64;
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColO = L::kStages * 128, kColOd = kColO + ((D == 128) ? 128 : 64);
@@ -364,6 +359,112 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             // online softmax over the groups, with the partial output o_d rescaled in TMEM when a later
             // group raises the maximum.  Up to 32 slots are one group.
             float m_d = -INFINITY, l_d = 0.f;
+            if constexpr (FP8) {
+                // e4m3 cache (see moda_fwd_kernel): a unit = all D features of one slot for the tile's rows + row scales
+                constexpr int C8 = D / 16;
+                const float* sScale = reinterpret_cast<const float*>(smem + L::kScale);
+                auto take_unit8 = [&](uint4 (&dst)[C8], float& sc) {
+                    const int st = unit % L::kRingStages;
+                    mbar_wait(bar(k2BarDFull + st), (unit / L::kRingStages) & 1, abort_flag, 21);
+                    const uint8_t* src = smem + L::kRing + st * L::kUnitBytes + r * 16;
+#pragma unroll
+                    for (int c = 0; c < C8; ++c) dst[c] = *reinterpret_cast<const uint4*>(src + c * (kTileRows * 16));
+                    sc = sScale[st * kTileRows + r];
+                    fence_proxy_async_smem();
+                    mbar_arrive(bar(k2BarDEmpty + st));
+                    ++unit;
+                };
+#pragma unroll 1
+                for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
+                    const int gl = min(kFwdDepthGroup, p.l - g0);
+                    {
+                        float q[D];
+#pragma unroll
+                        for (int c = 0; c < D / 8; ++c) {
+                            const uint4 v = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, c));
+                            q[8 * c + 0] = bf16_lo_to_f32(v.x); q[8 * c + 1] = bf16_hi_to_f32(v.x);
+                            q[8 * c + 2] = bf16_lo_to_f32(v.y); q[8 * c + 3] = bf16_hi_to_f32(v.y);
+                            q[8 * c + 4] = bf16_lo_to_f32(v.z); q[8 * c + 5] = bf16_hi_to_f32(v.z);
+                            q[8 * c + 6] = bf16_lo_to_f32(v.w); q[8 * c + 7] = bf16_hi_to_f32(v.w);
+                        }
+#pragma unroll 1
+                        for (int i = 0; i < gl; ++i) {
+                            uint4 cur[C8];
+                            float sc;
+                            take_unit8(cur, sc);
+                            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < C8; ++c) {
+                                const uint32_t w[4] = {cur[c].x, cur[c].y, cur[c].z, cur[c].w};
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    float f0, f1, f2, f3;
+                                    e4m3x4_to_f32(w[k], f0, f1, f2, f3);
+                                    a0 = fmaf(q[16 * c + 4 * k + 0], f0, a0);
+                                    a1 = fmaf(q[16 * c + 4 * k + 1], f1, a1);
+                                    a2 = fmaf(q[16 * c + 4 * k + 2], f2, a2);
+                                    a3 = fmaf(q[16 * c + 4 * k + 3], f3, a3);
+                                }
+                            }
+                            sU[i * kTileRows + r] = ((a0 + a1) + (a2 + a3)) * sc;
+                        }
+                    }
+                    float m_new = m_d;
+                    for (int i = 0; i < gl; ++i) m_new = fmaxf(m_new, sU[i * kTileRows + r] * p.scale_log2);
+                    const float f = fast_exp2(m_d - m_new);
+                    l_d *= f;
+                    for (int i = 0; i < gl; ++i) {
+                        const float w = fast_exp2(fmaf(sU[i * kTileRows + r], p.scale_log2, -m_new));
+                        sU[i * kTileRows + r] = w;
+                        l_d += w;
+                    }
+                    m_d = m_new;
+                    {
+                        float acc[D];
+                        if (g0 == 0) {
+#pragma unroll
+                            for (int c = 0; c < D; ++c) acc[c] = 0.f;
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < D / 32; ++c) {
+                                uint32_t o[32];
+                                tmem_ld32(tmem + lane_addr + kColOd + c * 32, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) acc[32 * c + i] = __uint_as_float(o[i]) * f;
+                            }
+                        }
+#pragma unroll 1
+                        for (int i = 0; i < gl; ++i) {
+                            uint4 cur[C8];
+                            float sc;
+                            take_unit8(cur, sc);
+                            const float w = sU[i * kTileRows + r] * sc;
+#pragma unroll
+                            for (int c = 0; c < C8; ++c) {
+                                const uint32_t ww[4] = {cur[c].x, cur[c].y, cur[c].z, cur[c].w};
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    float f0, f1, f2, f3;
+                                    e4m3x4_to_f32(ww[k], f0, f1, f2, f3);
+                                    acc[16 * c + 4 * k + 0] = fmaf(w, f0, acc[16 * c + 4 * k + 0]);
+                                    acc[16 * c + 4 * k + 1] = fmaf(w, f1, acc[16 * c + 4 * k + 1]);
+                                    acc[16 * c + 4 * k + 2] = fmaf(w, f2, acc[16 * c + 4 * k + 2]);
+                                    acc[16 * c + 4 * k + 3] = fmaf(w, f3, acc[16 * c + 4 * k + 3]);
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t o[32];
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(acc[32 * c + i]);
+                            tmem_st32(tmem + lane_addr + kColOd + c * 32, o);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+            } else {
 #pragma unroll 1
             for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
                 const int gl = min(kFwdDepthGroup, p.l - g0);
@@ -454,6 +555,7 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     }
                     tmem_wait_st();                          // a later group reads these columns back
                 }
+            }
             }
             sMd[r] = m_d;
             sLd[r] = l_d;
@@ -562,7 +664,27 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         // Streams the tile's depth keys, then values, as 16 KiB units (8 feature chunks of one slot:
         // one contiguous run of the cache) through the ring, in the order the depth warps consume
         // them.  The ring keeps up to kRingStages x 16 KiB of HBM reads in flight per SM.
-        if (lane == 0 && p.l > 0) {
+        if (FP8 && lane == 0 && p.l > 0) {
+            // e4m3 cache: one unit per (slot, K or V): the block's codes, and its 128 row scales behind them
+            const uint64_t policy = l2_policy_evict_first();
+            const size_t slot_bytes = cache8_slot_bytes(p.B, p.T, Hk, D);
+            const size_t blk_bytes = cache8_block_bytes(D);
+            const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) + (((size_t(b) * Hk + hk) * nq + qt) * 2) * blk_bytes;
+            int unit = 0;
+            for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
+                const int gl = min(kFwdDepthGroup, p.l - g0);
+                for (int kv = 0; kv < 2; ++kv)
+                    for (int i = 0; i < gl; ++i, ++unit) {
+                        const int st = unit % L::kRingStages;
+                        if (unit >= L::kRingStages)
+                            mbar_wait(bar(k2BarDEmpty + st), ((unit / L::kRingStages) - 1) & 1, abort_flag, 32);
+                        mbar_arrive_expect_tx(bar(k2BarDFull + st), L::kUnitBytes + L::kScaleBytes);
+                        const uint8_t* src = blk + size_t(g0 + i) * slot_bytes + size_t(kv) * blk_bytes;
+                        bulk_load(sbase + L::kRing + st * L::kUnitBytes, src, L::kUnitBytes, bar(k2BarDFull + st), policy);
+                        bulk_load(sbase + L::kScale + st * L::kScaleBytes, src + L::kUnitBytes, L::kScaleBytes, bar(k2BarDFull + st), policy);
+                    }
+            }
+        } else if (lane == 0 && p.l > 0) {
             const uint64_t policy = l2_policy_evict_first();          // the depth cache is read exactly once
             const size_t slot_bytes = cache_slot_elems(p.B, p.T, Hk, D) * 2;
             const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +

@@ -32,6 +32,15 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// 1024-aligned start of the dynamic shared-memory segment, or nullptr if `need` bytes do not fit
+// behind it (reported through the status word by the caller).
+__device__ __forceinline__ uint8_t* aligned_dynamic_smem(uint8_t* raw, uint32_t need) {
+    uint8_t* p = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    uint32_t dyn;
+    asm volatile("mov.u32 %0, %dynamic_smem_size;" : "=r"(dyn));
+    return (uint32_t(p - raw) + need <= dyn) ? p : nullptr;
+}
+
 __device__ __forceinline__ uint64_t globaltimer_ns() {
     uint64_t t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -383,6 +392,29 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+// Four e4m3 bytes (lowest byte first) -> four floats.  Two hardware conversions to f16 pairs (exact: every e4m3 value is
+// an f16 value), then to f32.
+__device__ __forceinline__ void e4m3x4_to_f32(uint32_t w, float& f0, float& f1, float& f2, float& f3) {
+    uint32_t h01, h23;
+    asm("{\n"
+        ".reg .b16 lo, hi;\n"
+        "mov.b32 {lo, hi}, %2;\n"
+        "cvt.rn.f16x2.e4m3x2 %0, lo;\n"
+        "cvt.rn.f16x2.e4m3x2 %1, hi;\n"
+        "}\n" : "=r"(h01), "=r"(h23) : "r"(w));
+    asm("{\n"
+        ".reg .b16 a, b;\n"
+        "mov.b32 {a, b}, %2;\n"
+        "cvt.f32.f16 %0, a;\n"
+        "cvt.f32.f16 %1, b;\n"
+        "}\n" : "=f"(f0), "=f"(f1) : "r"(h01));
+    asm("{\n"
+        ".reg .b16 a, b;\n"
+        "mov.b32 {a, b}, %2;\n"
+        "cvt.f32.f16 %0, a;\n"
+        "cvt.f32.f16 %1, b;\n"
+        "}\n" : "=f"(f2), "=f"(f3) : "r"(h23));
 }
 __device__ __forceinline__ float bf16_lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16_hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }

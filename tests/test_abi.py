@@ -136,3 +136,26 @@ def test_paged_decode_entry_point_validates_before_touching_the_device():
     assert call(lens=ctypes.c_void_p(4098)) == -2
     assert lib.moda_attn_decode_varlen(p, p, p, None, None, 2, 100, 128, 8, 2, 128, 0, ctypes.c_float(0.1), p, p, p,
                                        ctypes.c_size_t(ws), None) == -1
+
+
+def test_e4m3_cache_entry_points_validate_before_touching_the_device():
+    lib = binding.load()
+    vp = ctypes.c_void_p
+    p, odd = vp(4096), vp(4100)
+    sc = ctypes.c_float(0.125)
+    # a block is 128 d bytes of codes and 128 fp32 row scales
+    assert moda.moda_depth_cache_e4m3_bytes(1, 256, 2, 64, 4) == 4 * 1 * 2 * 2 * 2 * (128 * 64 + 512)
+    assert moda.moda_depth_cache_e4m3_bytes(2, 129, 3, 128, 1) == 2 * 3 * 2 * 2 * (128 * 128 + 512)
+    assert moda.moda_depth_cache_e4m3_bytes(1, 256, 2, 96, 4) == 0
+    assert moda.moda_depth_cache_e4m3_bytes(1, 256, 2, 64, 257) == 0
+    assert lib.moda_depth_cache_append_e4m3(p, 1, 128, 1, 64, 256, p, p, None) == -6
+    assert lib.moda_depth_cache_append_e4m3(None, 1, 128, 1, 64, 0, p, p, None) == -1
+    assert lib.moda_depth_cache_append_e4m3(p, 1, 128, 1, 64, 0, odd, p, None) == -2
+    assert lib.moda_depth_cache_append_e4m3(p, 1, 128, 1, 48, 0, p, p, None) == -4
+    fwd = lambda dkv=p, H=4, Hk=2, d=64, l=2, Q=p: lib.moda_attn_fwd_e4m3(Q, p, p, dkv, 1, 128, H, Hk, d, l, sc, p, p, None)
+    assert fwd(dkv=None) == -1 and fwd(Q=odd) == -2 and fwd(d=32) == -4 and fwd(l=300) == -5
+    assert fwd(H=4, Hk=3) == -12
+    args = [p] * 7 + [1, 128, 1, 64, 1, sc] + [p, p, p]
+    assert lib.moda_attn_bwd_e4m3(*args, None, p, ctypes.c_size_t(1 << 20), None) == -1      # depth slots without a gradient cache
+    assert lib.moda_attn_bwd_e4m3(*args, p, p, ctypes.c_size_t(4096), None) == -7
+    assert lib.moda_attn_bwd_e4m3(*args, p, None, ctypes.c_size_t(1 << 20), None) == -7

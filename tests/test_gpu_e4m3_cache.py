@@ -1,0 +1,136 @@
+"""Depth cache in e4m3 with a scale per row: the quantiser bit for bit, and forward / backward parity against the
+oracle run on the dequantised slots (GPU, through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2603_15619_b200 as moda
+from paper_2603_15619_b200 import synthetic
+from oracle import moda_oracle as orc
+
+from parity import assert_forward_close, f64
+from test_gpu_bwd import assert_grads_close
+
+pytestmark = pytest.mark.gpu
+
+
+def build_cache8(Kd, Vd):
+    l, B, T, H, d = Kd.shape
+    cache = moda.alloc_depth_cache_e4m3(B, T, H, d, max(l, 1), Kd.device)
+    cache.fill_(0xAB)                                       # every byte of slots < l must be overwritten
+    for i in range(l):
+        moda.moda_depth_cache_append_e4m3(cache, i, Kd[i].contiguous(), Vd[i].contiguous())
+    return cache
+
+
+def unpack_cache8(cache, l, B, T, H, d):
+    """(codes uint8 [l, 2, B, Tpad, H, d], scales fp32 [l, 2, B, Tpad, H]) read back from the cache's bytes."""
+    nt = (T + 127) // 128
+    blk = 128 * d + 512
+    raw = cache[: l * B * H * nt * 2 * blk].cpu().numpy().reshape(l, B, H, nt, 2, blk)
+    codes = raw[..., : 128 * d].reshape(l, B, H, nt, 2, d // 16, 128, 16)
+    codes = codes.transpose(0, 4, 1, 3, 6, 2, 5, 7).reshape(l, 2, B, nt * 128, H, d)       # [l, kv, B, t, H, d]
+    scales = np.ascontiguousarray(raw[..., 128 * d:]).view(np.float32).reshape(l, B, H, nt, 2, 128)
+    scales = scales.transpose(0, 4, 1, 3, 5, 2).reshape(l, 2, B, nt * 128, H)
+    return codes, scales
+
+
+def oracle_cache8(Kd, Vd):
+    """The oracle's codes, scales and dequantised slots of bf16 depth tensors [l, B, T, H, d]."""
+    out = []
+    for X in (Kd, Vd):
+        codes, scale = orc.quantize_e4m3_rows(f64(X))
+        out.append((codes, scale, orc.dequantize_e4m3_rows(codes, scale)))
+    return out
+
+
+@pytest.mark.parametrize("B,T,H,d,l", [(1, 128, 1, 64, 1), (2, 300, 3, 128, 2), (1, 1000, 2, 64, 3), (1, 1, 1, 128, 1)])
+def test_quantiser_matches_the_oracle_bit_for_bit(B, T, H, d, l):
+    w = synthetic.Workload("q", B, T, H, d, l)
+    x = synthetic.make(w, seed=5, device="cuda")
+    Kd, Vd = x["Kd"].clone(), x["Vd"].clone()
+    # rows that exercise the corners: all zero, one huge entry (everything else underflows to subnormal codes or zero),
+    # exact ties, a negative zero
+    Kd[0, 0, 0, 0, :] = 0
+    if T > 2:
+        Kd[0, 0, 1, 0, :] = 1e-3
+        Kd[0, 0, 1, 0, 0] = 300.0
+        Vd[0, 0, 2, 0, :] = torch.linspace(-448, 448, d, device="cuda").to(torch.bfloat16)
+        Vd[0, 0, 2, 0, 1] = -0.0
+    cache = build_cache8(Kd, Vd)
+    codes, scales = unpack_cache8(cache, l, B, T, H, d)
+    for kv, X in enumerate((Kd, Vd)):
+        ref_codes, ref_scale = orc.quantize_e4m3_rows(f64(X))
+        assert np.array_equal(scales[:, kv, :, :T], ref_scale), "row scales differ"
+        assert np.array_equal(codes[:, kv, :, :T], ref_codes), "codes differ"
+        if T % 128:
+            assert (codes[:, kv, :, T:] == 0).all() and (scales[:, kv, :, T:] == 1.0).all(), "tail rows must be code 0, scale 1"
+
+
+CASES = [(1, 128, 1, 64, 1), (2, 257, 3, 128, 3), (1, 640, 2, 64, 5), (1, 1000, 1, 128, 8), (2, 255, 1, 64, 32),
+         (1, 200, 2, 128, 33), (1, 130, 1, 64, 70), (1, 65, 2, 128, 2)]
+
+
+@pytest.mark.parametrize("B,T,H,d,l", CASES)
+def test_forward_and_backward_match_the_oracle_on_the_dequantised_slots(B, T, H, d, l):
+    w = synthetic.Workload("e", B, T, H, d, l)
+    x = synthetic.make(w, seed=17, device="cuda")
+    cache = build_cache8(x["Kd"], x["Vd"])
+    (_, _, Kd_hat), (_, _, Vd_hat) = oracle_cache8(x["Kd"], x["Vd"])
+    O_ref, LSE_ref = orc.forward(f64(x["Q"]), f64(x["K"]), f64(x["V"]), Kd_hat, Vd_hat, w.scale)
+    O, LSE = moda.moda_attn_fwd_e4m3(x["Q"], x["K"], x["V"], cache, l, w.scale)
+    assert moda.moda_last_status() == 0
+    assert_forward_close(O, LSE, O_ref, LSE_ref, f"e4m3 {(B, T, H, d, l)}")
+    # the quantisation is part of the operands, not of the error budget: against the unquantised slots the
+    # forward must differ by more than the parity tolerance would hide only if the cache mattered at all
+    ref = orc.backward(f64(x["Q"]), f64(x["K"]), f64(x["V"]), Kd_hat, Vd_hat, f64(x["dO"]), w.scale)
+    dcache = moda.alloc_depth_cache(B, T, H, d, l)
+    dcache.fill_(5.0)
+    dQ, dK, dV, dcache = moda.moda_attn_bwd_e4m3(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, w.scale, d_depth_kv=dcache)
+    assert moda.moda_last_status() == 0
+    from parity import unpack_cache
+    dKd, dVd = unpack_cache(dcache, l, B, T, H, d)
+    assert_grads_close((dQ, dK, dV, dKd, dVd), ref, f"e4m3 {(B, T, H, d, l)}")
+
+
+def test_the_e4m3_path_reads_the_codes_not_the_original_slots():
+    # Slots with a wide dynamic range inside each row: the dequantised slots differ from the originals by far more
+    # than the parity tolerance, so a kernel that somehow saw bf16 values (or dropped the scales) fails here.
+    B, T, H, d, l = 1, 384, 2, 64, 4
+    w = synthetic.Workload("r", B, T, H, d, l)
+    x = synthetic.make(w, seed=23, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(3)
+    boost = torch.exp2(torch.randint(-6, 3, x["Kd"].shape, device="cuda", generator=g).float())
+    Kd = (x["Kd"].float() * boost).to(torch.bfloat16)
+    Vd = (x["Vd"].float() * boost).to(torch.bfloat16)
+    cache = build_cache8(Kd, Vd)
+    (_, _, Kd_hat), (_, _, Vd_hat) = oracle_cache8(Kd, Vd)
+    Q, K, V = f64(x["Q"]), f64(x["K"]), f64(x["V"])
+    O_hat, LSE_hat = orc.forward(Q, K, V, Kd_hat, Vd_hat, w.scale)
+    O_raw, _ = orc.forward(Q, K, V, f64(Kd), f64(Vd), w.scale)
+    O, LSE = moda.moda_attn_fwd_e4m3(x["Q"], x["K"], x["V"], cache, l, w.scale)
+    assert_forward_close(O, LSE, O_hat, LSE_hat, "wide-range rows")
+    gap = np.linalg.norm(O_hat - O_raw) / np.linalg.norm(O_raw)
+    assert gap > 1.5e-2, f"the case does not separate quantised from unquantised slots (gap {gap:.2e})"
+
+
+@pytest.mark.parametrize("B,T,H,Hk,d,l", [(1, 300, 4, 2, 64, 3), (2, 200, 8, 1, 128, 2), (1, 256, 6, 2, 64, 40)])
+def test_grouped_query_forward(B, T, H, Hk, d, l):
+    w = synthetic.Workload("g", B, T, H, d, l)
+    x = synthetic.make(w, seed=29, device="cuda")
+    K, V = x["K"][:, :, :Hk].contiguous(), x["V"][:, :, :Hk].contiguous()
+    Kd, Vd = x["Kd"][:, :, :, :Hk].contiguous(), x["Vd"][:, :, :, :Hk].contiguous()
+    cache = build_cache8(Kd, Vd)
+    (_, _, Kd_hat), (_, _, Vd_hat) = oracle_cache8(Kd, Vd)
+    O_ref, LSE_ref = orc.forward_gqa(f64(x["Q"]), f64(K), f64(V), Kd_hat, Vd_hat, w.scale)
+    O, LSE = moda.moda_attn_fwd_e4m3(x["Q"], K, V, cache, l, w.scale)
+    assert moda.moda_last_status() == 0
+    assert_forward_close(O, LSE, O_ref, LSE_ref, f"e4m3 gqa {(B, T, H, Hk, d, l)}")
+
+
+def test_depth_zero_ignores_the_cache_pointer():
+    w = synthetic.Workload("z", 1, 200, 2, 64, 0)
+    x = synthetic.make(w, seed=1, device="cuda")
+    O, LSE = moda.moda_attn_fwd_e4m3(x["Q"], x["K"], x["V"], None, 0, w.scale)
+    O2, LSE2 = moda.moda_attn_fwd(x["Q"], x["K"], x["V"], None, 0, w.scale)
+    assert torch.equal(O, O2) and torch.equal(LSE, LSE2)

@@ -160,18 +160,19 @@ class Layer:
 
     KERNELS = ("fwd_append", "bwd_rows", "bwd_seq", "bwd_finish")
 
-    def __init__(self, w: synthetic.Workload, seed: int, device, with_backward: bool = True):
+    def __init__(self, w: synthetic.Workload, seed: int, device, with_backward: bool = True, e4m3: bool = False):
         import paper_2603_15619_b200 as moda
-        self.moda, self.w = moda, w
+        self.moda, self.w, self.e4m3 = moda, w, e4m3
         self.q = synthetic.tensor(w, "Q", seed, 0, device)
         self.k = synthetic.tensor(w, "K", seed, 0, device)
         self.v = synthetic.tensor(w, "V", seed, 0, device)
         self.cache = self.dcache = None
         if w.l > 0:
-            self.cache = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, w.l, device)
+            alloc, append = ((moda.alloc_depth_cache_e4m3, moda.moda_depth_cache_append_e4m3) if e4m3 else
+                             (moda.alloc_depth_cache, moda.moda_depth_cache_append))
+            self.cache = alloc(w.B, w.T, w.H, w.d, w.l, device)
             for i in range(w.l):
-                moda.moda_depth_cache_append(self.cache, i, synthetic.tensor(w, "Kd", seed, i, device),
-                                             synthetic.tensor(w, "Vd", seed, i, device))
+                append(self.cache, i, synthetic.tensor(w, "Kd", seed, i, device), synthetic.tensor(w, "Vd", seed, i, device))
         self.next_slot = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, 1, device)   # slot this layer writes for later layers
         self.O = torch.empty_like(self.q)
         self.LSE = torch.empty((w.B, w.H, w.T), dtype=torch.float32, device=device)
@@ -188,9 +189,14 @@ class Layer:
                                        O=self.O, LSE=self.LSE)
 
     def fwd(self):
-        self.moda.moda_attn_fwd(self.q, self.k, self.v, self.cache, self.w.l, self.w.scale, O=self.O, LSE=self.LSE)
+        f = self.moda.moda_attn_fwd_e4m3 if self.e4m3 else self.moda.moda_attn_fwd
+        f(self.q, self.k, self.v, self.cache, self.w.l, self.w.scale, O=self.O, LSE=self.LSE)
 
     def bwd(self, stages=None):
+        if self.e4m3:
+            self.moda.moda_attn_bwd_e4m3(self.q, self.k, self.v, self.cache, self.O, self.dO, self.LSE, self.w.l, self.w.scale,
+                                         dQ=self.dQ, dK=self.dK, dV=self.dV, d_depth_kv=self.dcache, workspace=self.ws)
+            return
         self.moda.moda_attn_bwd(self.q, self.k, self.v, self.cache, self.O, self.dO, self.LSE, self.w.l, self.w.scale,
                                 dQ=self.dQ, dK=self.dK, dV=self.dV, d_depth_kv=self.dcache, workspace=self.ws, stages=stages)
 
@@ -368,11 +374,11 @@ def run_targets(peaks, device, headline_w, headline):
            [("c4", W["c4"], 3, True), ("c5", W["c5"], 3, True)]
     timed = {}
 
-    def timings(ww, iters, bwd):
-        key = (ww.B, ww.T, ww.H, ww.d, ww.l)
+    def timings(ww, iters, bwd, e4m3=False):
+        key = (ww.B, ww.T, ww.H, ww.d, ww.l, e4m3)
         if key not in timed:
             torch.cuda.empty_cache()
-            layer = Layer(ww, seed=0, device=device, with_backward=bwd)
+            layer = Layer(ww, seed=0, device=device, with_backward=bwd, e4m3=e4m3)
             f_ms = time_calls(layer.fwd, iters)
             b_ms = time_calls(layer.bwd, iters) if bwd else None
             timed[key] = (f_ms, b_ms)
@@ -404,6 +410,18 @@ def run_targets(peaks, device, headline_w, headline):
         rows[name] = {k: full[k] for k in ("fwd_ms", "fwd_pct_of_burst_peak", "fwd_bound", "fwd_frac_of_roofline",
                                             "roofline_cap_pct_of_burst_peak", "bwd_ms", "bwd_frac_of_roofline",
                                             "fwd_ratio_to_l0", "fwd_bwd_ratio_to_l0")}
+    # The same kernels on a depth cache kept in e4m3 with a scale per row (half the depth bytes), at the depth-heavy
+    # points: the roofline is recomputed with the smaller cache.
+    for name, w, iters in [(f"c3_l{l}_e4m3", W["c3"].with_l(l), 8) for l in (16, 24, 32)] + [("c2_e4m3", W["c2"], 8)]:
+        f_ms, b_ms = timings(w, iters, True, e4m3=True)
+        ff = flops.fwd_flops(w.B, w.T, w.H, w.d, w.l)
+        cache16 = 2.0 * 2 * w.l * w.B * w.T * w.H * w.d
+        cache8 = cache16 / 2 + 2.0 * 4 * w.l * w.B * w.T * w.H
+        t_tensor = ff / (peaks["bf16_tflops"] * 1e12) * 1e3
+        t_hbm = (flops.fwd_bytes(w.B, w.T, w.H, w.d, w.l) - cache16 + cache8) / (peaks["hbm_gbs"] * 1e9) * 1e3
+        rows[name] = {"fwd_ms": round(f_ms, 4), "fwd_pct_of_burst_peak": round(100.0 * ff / f_ms / 1e9 / peaks["bf16_tflops"], 1),
+                      "fwd_frac_of_roofline": round(max(t_tensor, t_hbm) / f_ms, 3), "bwd_ms": round(b_ms, 4)}
+        log("target", name, rows[name])
     torch.cuda.empty_cache()
     return rows
 

@@ -25,6 +25,13 @@ SHAPES = [
     (1, 200, 16, 1, 64, 40), (1, 130, 32, 1, 64, 33), (1, 140, 32, 2, 128, 12),   # 16 / 32 heads per group as groups of 8
     (1, 150, 8, 1, 128, 50), (1, 130, 16, 1, 128, 48),            # d = 128 forward through the per-position kernel
     (1, 300, 16, 1, 64, 5), (1, 200, 32, 2, 128, 3), (2, 130, 32, 1, 64, 9), (1, 256, 16, 1, 128, 33),   # G = 16, 32
+    # either side of the points where the host switches the depth part between the row-local path and the
+    # per-position kernel: forward d = 64, G = 8 at l = 30 and G = 16 at l = 31; d = 128, G = 8 at l = 48;
+    # backward d = 64, G = 8 at l = 11 and G = 16 at l = 8; d = 128, G = 8 at l = 9 and G = 4 at l = 28
+    (1, 140, 8, 1, 64, 29), (1, 140, 8, 1, 64, 30), (1, 140, 16, 1, 64, 30), (1, 140, 16, 1, 64, 31),
+    (1, 130, 8, 1, 128, 47), (1, 130, 8, 1, 128, 48),
+    (1, 140, 8, 1, 64, 10), (1, 140, 8, 1, 64, 11), (1, 140, 16, 1, 64, 7), (1, 140, 16, 1, 64, 8),
+    (1, 130, 8, 1, 128, 8), (1, 130, 8, 1, 128, 9), (1, 130, 4, 1, 128, 27), (1, 130, 4, 1, 128, 28),
 ]
 
 

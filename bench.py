@@ -470,6 +470,15 @@ def run_gqa_sweep(device, shapes=None):
             res[l] = (time_calls(fwd, iters), time_calls(bwd, iters))
             if l == 0:
                 base_cache[(T, G)] = res[0]
+            elif G > 1:
+                # the same call with the depth cache (and the depth gradients) in the position-major layout
+                for i in range(l):
+                    moda.moda_depth_cache_append_pm(cache, i, synthetic.tensor(wk, "Kd", 0, i, device),
+                                                    synthetic.tensor(wk, "Vd", 0, i, device))
+                fwd_pm = lambda: moda.moda_attn_fwd_gqa_pm(x["Q"], x["K"], x["V"], cache, l, scale, O=O, LSE=LSE)
+                bwd_pm = lambda: moda.moda_attn_bwd_gqa_pm(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale,
+                                                           dQ=dQ, dK=dK, dV=dV, d_depth_kv_pm=dcache, workspace=ws)
+                res["pm"] = (time_calls(fwd_pm, iters), time_calls(bwd_pm, iters))
             del x, cache, dcache, O, LSE, dQ, dK, dV, ws
         (f0, b0), (f1, b1) = res[0], res[l_full]
         ff = 4.0 * B * H * d * (T * (T + 1) / 2) + 4.0 * B * H * T * l_full * d
@@ -480,6 +489,15 @@ def run_gqa_sweep(device, shapes=None):
                      "paper_extra_time_pct_a100_triton": paper_pct,
                      "fwd_bwd_ratio_to_l0": round((f0 + b0) / (f1 + b1), 4),
                      "fwd_tflops": round(ff / f1 / 1e9, 1), "fwd_bwd_tflops": round(3.5 * ff / (f1 + b1) / 1e9, 1)})
+        if "pm" in res:
+            fp, bp = res["pm"]
+            cache_bytes = 2.0 * 2 * l_full * B * T * Hk * d
+            rows[-1].update({"pm_fwd_ms": round(fp, 4), "pm_bwd_ms": round(bp, 4),
+                             "pm_extra_time_pct": round(100.0 * ((fp + bp) / (f0 + b0) - 1.0), 2),
+                             # depth part alone (time over the l = 0 twin) against the bytes it must move: the cache once
+                             # (forward), the cache and its gradients (backward), plus Q / O (dO, dQ) of all heads once each
+                             "pm_depth_fwd_gbs": round((cache_bytes + 3 * 2.0 * B * T * H * d) / max(fp - f0, 1e-6) / 1e6, 0),
+                             "pm_depth_bwd_gbs": round((2 * cache_bytes + 4 * 2.0 * B * T * H * d) / max(bp - b0, 1e-6) / 1e6, 0)})
         log("gqa_sweep", rows[-1])
     torch.cuda.empty_cache()
     return rows

@@ -391,6 +391,39 @@ int moda_attn_bwd_e4m3(const void* Q, const void* K, const void* V, const void* 
                        void* dQ, void* dK, void* dV, void* d_depth_kv,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * ---- Position-major depth cache for grouped-query calls ----
+ *
+ * With several query heads per key/value head (Sec. 3, group-aware depth KV) the depth part of a call can run
+ * per position: all G heads of a group against the l depth rows of that position, as small dense products.
+ * Those kernels consume every row of a few consecutive positions, which the row-interleaved cache layout
+ * hands out as 16-byte pieces 2 KiB apart.  This second layout keeps a position's rows together:
+ *
+ *     cache_pm[slot][b][h_kv][t][kv][d]     bf16; t over whole 128-position tiles, tail rows zero
+ *
+ * Same size as the row-interleaved cache (moda_depth_cache_bytes); the caller chooses the layout when it
+ * appends, and passes the cache to the entry points of that layout only.
+ *
+ * moda_depth_cache_append_pm / _unpack_pm   as moda_depth_cache_append / _unpack, for this layout.
+ * moda_attn_fwd_gqa_pm   moda_attn_fwd_gqa with the depth slots in this layout; needs H_kv < H
+ *                        (MODA_ERR_BAD_GROUP otherwise).
+ * moda_attn_bwd_gqa_pm   moda_attn_bwd_gqa likewise; d_depth_kv_pm receives the depth gradients in this layout;
+ *                        workspace of moda_bwd_workspace_bytes_gqa.
+ * Other arguments, ownership, validation and error codes as for the calls they mirror.
+ */
+int moda_depth_cache_append_pm(void* cache, int B, int T, int H, int d, int slot,
+                               const void* K_i, const void* V_i, void* stream);
+int moda_depth_cache_unpack_pm(const void* cache, int B, int T, int H, int d, int slot,
+                               void* K_i, void* V_i, void* stream);
+int moda_attn_fwd_gqa_pm(const void* Q, const void* K, const void* V, const void* depth_kv_pm,
+                         int B, int T, int H, int H_kv, int d, int l, float scale,
+                         void* O, float* LSE, void* stream);
+int moda_attn_bwd_gqa_pm(const void* Q, const void* K, const void* V, const void* depth_kv_pm,
+                         const void* O, const void* dO, const float* LSE,
+                         int B, int T, int H, int H_kv, int d, int l, float scale,
+                         void* dQ, void* dK, void* dV, void* d_depth_kv_pm,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     moda_attn_bwd,
     moda_attn_bwd_e4m3,
     moda_attn_bwd_gqa,
+    moda_attn_bwd_gqa_pm,
     moda_attn_bwd_gqa_stages,
     moda_attn_bwd_stages,
     moda_attn_bwd_static_scratch,
@@ -30,15 +31,18 @@ from .binding import (  # noqa: F401
     moda_attn_fwd_append,
     moda_attn_fwd_e4m3,
     moda_attn_fwd_gqa,
+    moda_attn_fwd_gqa_pm,
     moda_attn_fwd_prefill,
     moda_bwd_workspace_bytes,
     moda_bwd_workspace_bytes_gqa,
     moda_decode_workspace_bytes,
     moda_depth_cache_append,
     moda_depth_cache_append_e4m3,
+    moda_depth_cache_append_pm,
     moda_depth_cache_e4m3_bytes,
     moda_depth_cache_bytes,
     moda_depth_cache_unpack,
+    moda_depth_cache_unpack_pm,
     moda_last_status,
     moda_selftest_wait_timeout,
     moda_version,

@@ -25,6 +25,7 @@ SYMBOLS = (
     "moda_decode_workspace_bytes", "moda_attn_decode", "moda_attn_fwd_prefill", "moda_attn_fwd_append",
     "moda_attn_decode_varlen", "moda_attn_decode_paged",
     "moda_depth_cache_e4m3_bytes", "moda_depth_cache_append_e4m3", "moda_attn_fwd_e4m3", "moda_attn_bwd_e4m3",
+    "moda_depth_cache_append_pm", "moda_depth_cache_unpack_pm", "moda_attn_fwd_gqa_pm", "moda_attn_bwd_gqa_pm",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -106,6 +107,14 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_fwd_e4m3.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
     lib.moda_attn_bwd_e4m3.restype = ci
     lib.moda_attn_bwd_e4m3.argtypes = [vp] * 7 + [ci] * 5 + [cf] + [vp] * 5 + [sz, vp]
+    lib.moda_depth_cache_append_pm.restype = ci
+    lib.moda_depth_cache_append_pm.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp]
+    lib.moda_depth_cache_unpack_pm.restype = ci
+    lib.moda_depth_cache_unpack_pm.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp]
+    lib.moda_attn_fwd_gqa_pm.restype = ci
+    lib.moda_attn_fwd_gqa_pm.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
+    lib.moda_attn_bwd_gqa_pm.restype = ci
+    lib.moda_attn_bwd_gqa_pm.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
     _lib = lib
     return lib
 
@@ -270,6 +279,53 @@ def moda_attn_bwd_e4m3(Q, K, V, depth_kv_e4m3, O, dO, LSE, l, scale,
                                      _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "moda_attn_bwd_e4m3")
     return dQ, dK, dV, d_depth_kv
+
+
+def moda_depth_cache_append_pm(cache, slot, K_i, V_i, stream=None):
+    """moda_depth_cache_append for the position-major layout (grouped-query calls through the *_pm entry points)."""
+    B, T, H, d = _bthd(K_i, "K_i")
+    assert _bthd(V_i, "V_i") == (B, T, H, d)
+    _check(load().moda_depth_cache_append_pm(_ptr(cache), B, T, H, d, int(slot), _ptr(K_i), _ptr(V_i), _stream(stream)),
+           "moda_depth_cache_append_pm")
+
+
+def moda_depth_cache_unpack_pm(cache, slot, K_i, V_i, stream=None):
+    ref = K_i if K_i is not None else V_i
+    B, T, H, d = _bthd(ref, "K_i/V_i")
+    _check(load().moda_depth_cache_unpack_pm(_ptr(cache), B, T, H, d, int(slot), _ptr(K_i), _ptr(V_i), _stream(stream)),
+           "moda_depth_cache_unpack_pm")
+
+
+def moda_attn_fwd_gqa_pm(Q, K, V, depth_kv_pm, l, scale, O=None, LSE=None, stream=None):
+    """moda_attn_fwd_gqa with the depth slots in the position-major layout (H_kv < H)."""
+    B, T, H, Hk, d = _gqa_shapes(Q, K, V)
+    if O is None:
+        O = _new_like(Q, stream)
+    if LSE is None:
+        LSE = _new((B, H, T), torch.float32, Q.device, stream)
+    _check(load().moda_attn_fwd_gqa_pm(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv_pm) if l > 0 else None,
+                                       B, T, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE), _stream(stream)),
+           "moda_attn_fwd_gqa_pm")
+    return O, LSE
+
+
+def moda_attn_bwd_gqa_pm(Q, K, V, depth_kv_pm, O, dO, LSE, l, scale,
+                         dQ=None, dK=None, dV=None, d_depth_kv_pm=None, workspace=None, stream=None):
+    """moda_attn_bwd_gqa with the depth slots and the depth gradients in the position-major layout."""
+    B, T, H, Hk, d = _gqa_shapes(Q, K, V)
+    dQ = _new_like(Q, stream) if dQ is None else dQ
+    dK = _new_like(K, stream) if dK is None else dK
+    dV = _new_like(V, stream) if dV is None else dV
+    if l > 0 and d_depth_kv_pm is None:
+        d_depth_kv_pm = alloc_depth_cache(B, T, Hk, d, l, Q.device, stream)
+    if workspace is None:
+        workspace = _new((moda_bwd_workspace_bytes_gqa(B, T, H, Hk, d, l),), torch.uint8, Q.device, stream)
+    _check(load().moda_attn_bwd_gqa_pm(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv_pm) if l > 0 else None,
+                                       _ptr(O), _ptr(dO), _ptr(LSE), B, T, H, Hk, d, int(l), float(scale),
+                                       _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(d_depth_kv_pm) if l > 0 else None,
+                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "moda_attn_bwd_gqa_pm")
+    return dQ, dK, dV, d_depth_kv_pm
 
 
 def moda_attn_fwd(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):

@@ -208,6 +208,10 @@ int launch_depth_merge(DepthMergeParams m, cudaStream_t stream) {
     }
 }
 
+// How the depth cache of a call is laid out: row-interleaved bf16 (the default), e4m3 codes with row scales, or
+// position-major bf16 (moda_cache.cuh).
+enum CacheKind { kCacheRows = 0, kCacheE4m3 = 1, kCachePm = 2 };
+
 // Dynamic shared memory of the forward kernel that reads an e4m3 depth cache (only the variant each head size runs exists).
 template <int D>
 constexpr int fwd_smem_e4m3() {
@@ -217,7 +221,8 @@ constexpr int fwd_smem_e4m3() {
 
 template <int D>
 int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv, int B, int T, int T_kv, int H, int Hk, int l,
-               float scale, void* O, float* LSE, void* append_slot, cudaStream_t stream, bool fp8 = false) {
+               float scale, void* O, float* LSE, void* append_slot, cudaStream_t stream, CacheKind kind = kCacheRows) {
+    const bool fp8 = kind == kCacheE4m3, pm = kind == kCachePm;
     constexpr bool kWide = (D == 64);
     constexpr int kSmem = kWide ? Fwd2Smem<D>::kDynamic : FwdSmem<D, 2>::kDynamic;
     constexpr int kSmem8 = fwd_smem_e4m3<D>();
@@ -251,7 +256,8 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     // Grouped-query calls: the sequence kernel runs without depth slots and a second kernel adds the depth
     // part of all heads of a group at once (moda_depth_gqa.cuh).
     // An e4m3 cache is always read by the row-local depth warps of the sequence kernel.
-    const bool split_depth = !fp8 && gqa_depth_split(D, p.G, l);
+    // A position-major cache is always read by the per-position kernel.
+    const bool split_depth = pm ? l > 0 : (!fp8 && gqa_depth_split(D, p.G, l));
     if (split_depth) p.l = 0;
     if (fp8) {
         if constexpr (kWide) moda_fwd2_kernel<D, true><<<grid, kThreads, kSmem8, stream>>>(mQ, mK, mV, mO, p);
@@ -268,6 +274,7 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
         m.LSE = LSE;
         m.B = B; m.T = T; m.H = H; m.Hk = Hk; m.l = l;
         m.scale_log2 = scale * kLog2e;
+        m.pm = pm ? 1 : 0;
         if (int rc = launch_depth_merge<D>(m, stream)) return rc;
     }
     return MODA_OK;
@@ -397,6 +404,7 @@ int launch_bwd_fused(const BwdArgs& a, int stages, cudaStream_t stream) {
             m.B = B; m.T = T; m.H = H; m.Hk = Hk; m.l = a.l;
             m.scale = a.scale; m.scale_log2 = a.scale * kLog2e;
             m.accumulate = a.accumulate_depth ? 1 : 0;
+            m.pm = a.pm_cache ? 1 : 0;
             if (int rc = launch_depth_bwd<D>(m, stream)) return rc;
         }
     }
@@ -464,6 +472,7 @@ int launch_bwd(const BwdArgs& a, int stages, cudaStream_t stream) {
             m.B = B; m.T = T; m.H = H; m.Hk = Hk; m.l = a.l;
             m.scale = a.scale; m.scale_log2 = a.scale * kLog2e;
             m.accumulate = a.accumulate_depth ? 1 : 0;
+            m.pm = 0;
             if (int rc = launch_depth_bwd<D>(m, stream)) return rc;
         } else if (G > 1 && a.l > 0) {
             const unsigned tiles2 = unsigned(B) * Hk * num_tiles(T) * 2;            // x {dKd, dVd}
@@ -500,6 +509,15 @@ int launch_cache_copy(void* cache, int B, int T, int H, int slot, void* Xk, void
     uint4* slot_base = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(cache) + size_t(slot) * cache_slot_elems(B, T, H, D));
     const unsigned grid = unsigned(B) * H * num_tiles(T) * 2;
     depth_cache_copy_kernel<D, kToCache><<<grid, 256, 0, stream>>>(slot_base, static_cast<uint4*>(Xk), static_cast<uint4*>(Xv), T, H);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+
+template <int D, bool kToCache>
+int launch_cache_pm_copy(void* cache, int B, int T, int H, int slot, void* Xk, void* Xv, cudaStream_t stream) {
+    uint4* slot_base = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(cache) + size_t(slot) * cache_slot_elems(B, T, H, D));
+    const size_t pieces = cache_slot_elems(B, T, H, D) / 8;
+    const unsigned grid = unsigned(std::min<size_t>((pieces + 255) / 256, 148 * 32));
+    depth_cache_pm_copy_kernel<D, kToCache><<<grid, 256, 0, stream>>>(slot_base, static_cast<uint4*>(Xk), static_cast<uint4*>(Xv), B, T, H);
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 
@@ -734,7 +752,7 @@ size_t moda_bwd_workspace_bytes(int B, int T, int H, int d, int l) {
 size_t moda_bwd_workspace_bytes_gqa(int B, int T, int H, int H_kv, int d, int l) {
     if (check_shape(B, T, H, d) != MODA_OK || check_groups(H, H_kv) != MODA_OK || l < 0 || l > MODA_MAX_DEPTH) return 0;
     const size_t split = bwd_workspace_bytes_gqa(B, T, H, H_kv, l);
-    const size_t fused = bwd_uses_fused(d, H / H_kv, l, false) ? bwd_fused_workspace_bytes(B, T, H, d) : 0;
+    const size_t fused = bwd_fused_workspace_bytes(B, T, H, d);   // also what the e4m3 and position-major calls take
     return split > fused ? split : fused;
 }
 
@@ -832,8 +850,8 @@ int moda_attn_fwd_e4m3(const void* Q, const void* K, const void* V, const void* 
         return MODA_ERR_MISALIGNED;
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, true)
-                    : launch_fwd<64>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, true);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, kCacheE4m3)
+                    : launch_fwd<64>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, kCacheE4m3);
 }
 
 int moda_attn_bwd_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,
@@ -856,6 +874,74 @@ int moda_attn_bwd_e4m3(const void* Q, const void* K, const void* V, const void* 
     a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv_e4m3; a.O = O; a.dO = dO; a.LSE = LSE;
     a.B = B; a.T = T; a.H = H; a.Hk = H; a.l = l; a.scale = scale;
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv; a.workspace = workspace;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_bwd_fused<128>(a, MODA_BWD_ALL_STAGES, st) : launch_bwd_fused<64>(a, MODA_BWD_ALL_STAGES, st);
+}
+
+// ---- position-major depth cache for grouped-query calls ----
+int moda_depth_cache_append_pm(void* cache, int B, int T, int H, int d, int slot,
+                               const void* K_i, const void* V_i, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (slot < 0 || slot >= MODA_MAX_DEPTH) return MODA_ERR_BAD_SLOT;
+    if (!cache || !K_i || !V_i) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(cache) || !aligned16(K_i) || !aligned16(V_i)) return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_cache_pm_copy<128, true>(cache, B, T, H, slot, const_cast<void*>(K_i), const_cast<void*>(V_i), st)
+                    : launch_cache_pm_copy<64, true>(cache, B, T, H, slot, const_cast<void*>(K_i), const_cast<void*>(V_i), st);
+}
+
+int moda_depth_cache_unpack_pm(const void* cache, int B, int T, int H, int d, int slot,
+                               void* K_i, void* V_i, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (slot < 0 || slot >= MODA_MAX_DEPTH) return MODA_ERR_BAD_SLOT;
+    if (!cache || (!K_i && !V_i)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(cache) || !aligned16(K_i) || !aligned16(V_i)) return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_cache_pm_copy<128, false>(const_cast<void*>(cache), B, T, H, slot, K_i, V_i, st)
+                    : launch_cache_pm_copy<64, false>(const_cast<void*>(cache), B, T, H, slot, K_i, V_i, st);
+}
+
+int moda_attn_fwd_gqa_pm(const void* Q, const void* K, const void* V, const void* depth_kv_pm,
+                         int B, int T, int H, int H_kv, int d, int l, float scale,
+                         void* O, float* LSE, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_groups(H, H_kv)) return rc;
+    if (H == H_kv) return MODA_ERR_BAD_GROUP;                 // the per-position kernels need at least two heads per group
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (!Q || !K || !V || !O || !LSE || (l > 0 && !depth_kv_pm)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) ||
+        (l > 0 && !aligned16(depth_kv_pm)))
+        return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv_pm, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, kCachePm)
+                    : launch_fwd<64>(Q, K, V, depth_kv_pm, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, kCachePm);
+}
+
+int moda_attn_bwd_gqa_pm(const void* Q, const void* K, const void* V, const void* depth_kv_pm,
+                         const void* O, const void* dO, const float* LSE,
+                         int B, int T, int H, int H_kv, int d, int l, float scale,
+                         void* dQ, void* dK, void* dV, void* d_depth_kv_pm,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_groups(H, H_kv)) return rc;
+    if (H == H_kv) return MODA_ERR_BAD_GROUP;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv_pm || !d_depth_kv_pm)))
+        return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(LSE) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) ||
+        (l > 0 && (!aligned16(depth_kv_pm) || !aligned16(d_depth_kv_pm))))
+        return MODA_ERR_MISALIGNED;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < bwd_fused_workspace_bytes(B, T, H, d)) return MODA_ERR_WORKSPACE;
+    if (int rc = check_device()) return rc;
+    BwdArgs a;
+    a.pm_cache = true;
+    a.Q = Q; a.K = K; a.V = V; a.depth_kv = depth_kv_pm; a.O = O; a.dO = dO; a.LSE = LSE;
+    a.B = B; a.T = T; a.H = H; a.Hk = H_kv; a.l = l; a.scale = scale;
+    a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv_pm; a.workspace = workspace;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return d == 128 ? launch_bwd_fused<128>(a, MODA_BWD_ALL_STAGES, st) : launch_bwd_fused<64>(a, MODA_BWD_ALL_STAGES, st);
 }

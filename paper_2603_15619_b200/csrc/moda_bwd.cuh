@@ -38,6 +38,7 @@ struct BwdArgs {
     void *dQ, *dK, *dV, *d_depth_kv, *workspace;
     bool accumulate_depth = false;   // add the depth gradients to d_depth_kv instead of overwriting it
     bool deterministic = false;      // split form (bit-reproducible) instead of the fused form
+    bool pm_cache = false;           // depth_kv and d_depth_kv are position-major (grouped-query calls, fused form, per-position depth kernel)
     bool fp8_cache = false;          // depth_kv holds e4m3 codes + row scales (fused form, one KV head per query head only)
 };
 

@@ -72,6 +72,45 @@ depth_cache_copy_kernel(uint4* __restrict__ cache_slot,            // base of th
     }
 }
 
+// ---- position-major layout (for grouped-query calls whose depth part runs per position) ----
+//
+//   cache_pm[slot][b][h][t][kv][d]   (bf16; t runs over whole 128-position tiles, tail rows zero)
+//
+// The K row and the V row of one position are 4 d contiguous bytes, and consecutive positions follow: the
+// per-position kernels (moda_depth_gqa.cuh), which consume all rows of a few positions, read and write runs of
+// (positions per CTA) * 4 d bytes per slot instead of 16-byte pieces at 2 KiB strides.  A slot has the same
+// size as in the row-interleaved layout.
+__host__ __device__ inline size_t cache_pm_offset(int B, int T, int H, int d, int slot, int b, int h, int t) {
+    return size_t(slot) * cache_slot_elems(B, T, H, d) +
+           ((size_t(b) * H + h) * (size_t(num_tiles(T)) * kTileRows) + t) * 2 * d;
+}
+
+// Grid-stride copy between [B][T][H][d] tensors and one slot of the position-major cache, 16 bytes per thread:
+// consecutive threads take consecutive pieces of the cache side (K row, V row of a position).
+template <int D, bool kToCache>
+__global__ void __launch_bounds__(256)
+depth_cache_pm_copy_kernel(uint4* __restrict__ slot_base, uint4* __restrict__ Xk, uint4* __restrict__ Xv, int B, int T, int H) {
+    constexpr int CH = D / 8;
+    const size_t Tp = size_t(num_tiles(T)) * kTileRows;
+    const size_t total = size_t(B) * H * Tp * 2 * CH;
+    for (size_t i = size_t(blockIdx.x) * 256 + threadIdx.x; i < total; i += size_t(gridDim.x) * 256) {
+        const int ch = int(i % CH);
+        const int kv = int((i / CH) & 1);
+        const size_t row = i / (2 * CH);                 // (b * H + h) * Tp + t
+        const size_t t = row % Tp, bh = row / Tp;
+        const int h = int(bh % H);
+        const size_t b = bh / H;
+        uint4* X = kv ? Xv : Xk;
+        if (kToCache) {
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (t < size_t(T)) v = X[((b * T + t) * H + h) * CH + ch];
+            slot_base[i] = v;
+        } else if (X != nullptr && t < size_t(T)) {
+            X[((b * T + t) * H + h) * CH + ch] = slot_base[i];
+        }
+    }
+}
+
 }  // namespace moda
 
 // =====================================================================================

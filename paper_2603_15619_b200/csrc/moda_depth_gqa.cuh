@@ -35,6 +35,7 @@ struct DepthMergeParams {
     int B, T, H, Hk, l;
     int h0;                             // first head (inside its group of H / Hk) of the up to 8 heads this launch handles
     float scale_log2;
+    int pm;                             // nonzero: depth_kv is in the position-major layout (moda_cache.cuh)
 };
 
 template <int D>
@@ -114,8 +115,29 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
     const int st_pos = threadIdx.x % kDgPos, st_chunk = (threadIdx.x / kDgPos) % CH, st_slot0 = threadIdx.x / (kDgPos * CH);
     const __nv_bfloat16* st_src = cbase + (size_t(st_chunk) * kTileRows + st_pos) * 8;
     const uint32_t st_dst = smem_base + st_pos * kDgSlots * D * 2 + ((st_chunk & 8) << 4);
+    // Position-major cache: a slot's K and V rows of the CTA's positions are one contiguous run of kDgPos * 4 d bytes;
+    // consecutive threads copy consecutive 16-byte pieces of it (a warp request is 512 contiguous bytes).
+    constexpr int kPmPieces = kDgPos * 2 * CH;                     // 16-byte pieces of that run
+    static_assert(kDgThreads % kPmPieces == 0, "whole slots per pass");
+    constexpr int kPmSlotStep = kDgThreads / kPmPieces;
+    const int pm_q = threadIdx.x % kPmPieces, pm_slot0 = threadIdx.x / kPmPieces;
+    const int pm_pos = pm_q / (2 * CH), pm_kv = (pm_q / CH) & 1, pm_chunk = pm_q % CH;
+    const __nv_bfloat16* pm_src = p.depth_kv + cache_pm_offset(p.B, p.T, p.Hk, D, 0, b, hk, t0) + size_t(pm_q) * 8;
+    const uint32_t pm_dst = smem_base + pm_kv * kTensorBytes + pm_pos * kDgSlots * D * 2 + ((pm_chunk & 8) << 4);
     auto stage_round = [&](int s0, int buf) {
         const int ns = min(kDgSlots, p.l - s0);
+        if (p.pm) {
+            const __nv_bfloat16* src = pm_src + size_t(s0 + pm_slot0) * slot_elems;
+            const uint32_t dst = pm_dst + buf * 2 * kTensorBytes;
+#pragma unroll
+            for (int k = 0; k < kDgSlots / kPmSlotStep; ++k) {
+                const int slot = pm_slot0 + k * kPmSlotStep;
+                if (slot < ns)
+                    cp_async_16(dst + slot * D * 2 + (((pm_chunk & 7) ^ (slot & 7)) << 4), src + size_t(k * kPmSlotStep) * slot_elems);
+            }
+            cp_async_commit();
+            return;
+        }
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
             const __nv_bfloat16* src = st_src + size_t(s0 + st_slot0) * slot_elems + size_t(kv) * cache_block_elems(D);
@@ -256,6 +278,7 @@ struct DepthBwdParams {
     float scale, scale_log2;
     int accumulate;                     // depth gradients are added to d_depth_kv instead of stored
     int h0;                             // first head (inside its group of H / Hk) of the up to 8 heads this launch handles
+    int pm;                             // nonzero: depth_kv and d_depth_kv are in the position-major layout (moda_cache.cuh)
 };
 
 template <int D>
@@ -333,8 +356,26 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
     constexpr int kSlotStep = NT / (P * CH);
     const int st_pos = threadIdx.x % P, st_chunk = (threadIdx.x / P) % CH, st_slot0 = threadIdx.x / (P * CH);
     const size_t st_goff = (size_t(st_chunk) * kTileRows + st_pos) * 8;
+    // Position-major layout: a slot's K and V rows of the CTA's positions are one run of P * 4 d bytes (see the forward)
+    constexpr int kPmPieces = P * 2 * CH;
+    static_assert(NT % kPmPieces == 0, "whole slots per pass");
+    constexpr int kPmSlotStep = NT / kPmPieces;
+    const int pm_q = threadIdx.x % kPmPieces, pm_slot0 = threadIdx.x / kPmPieces;
+    const int pm_pos = pm_q / (2 * CH), pm_kv = (pm_q / CH) & 1, pm_chunk = pm_q % CH;
+    const size_t pm_off = cache_pm_offset(p.B, p.T, p.Hk, D, 0, b, hk, t0) + size_t(pm_q) * 8;
     auto stage_round = [&](int s0, int buf) {
         const int ns = min(RS, p.l - s0);
+        if (p.pm) {
+            const __nv_bfloat16* src = p.depth_kv + pm_off + size_t(s0 + pm_slot0) * slot_elems;
+            const uint32_t dst = smem_base + (buf * 2 + pm_kv) * kTensorBytes;
+#pragma unroll
+            for (int k = 0; k < RS / kPmSlotStep; ++k) {
+                const int slot = pm_slot0 + k * kPmSlotStep;
+                if (slot < ns) cp_async_16(dst + row_piece(pm_pos * RS + slot, pm_chunk), src + size_t(k * kPmSlotStep) * slot_elems);
+            }
+            cp_async_commit();
+            return;
+        }
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
             const __nv_bfloat16* src = cbase + st_goff + size_t(s0 + st_slot0) * slot_elems + size_t(kv) * cache_block_elems(D);
@@ -441,6 +482,20 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
         }
         __syncthreads();                                   // all positions' output rows of this round are in shared memory
         // ---- write the round's gradients: a thread moves the (position, chunk) piece of every kSlotStep-th slot ----
+        if (p.pm) {
+            __nv_bfloat16* dst = p.d_depth_kv + pm_off + size_t(s0 + pm_slot0) * slot_elems;
+            const uint8_t* src = db_smem + L::kOut + (pm_kv * P + pm_pos) * RS * D * 2;
+#pragma unroll
+            for (int k = 0; k < RS / kPmSlotStep; ++k) {
+                const int slot = pm_slot0 + k * kPmSlotStep;
+                if (slot < ns) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(src + row_piece(slot, pm_chunk));
+                    __nv_bfloat16* out = dst + size_t(k * kPmSlotStep) * slot_elems;
+                    if (p.accumulate) red_add_bf16x2_v4(out, v);
+                    else *reinterpret_cast<uint4*>(out) = v;
+                }
+            }
+        } else
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
             __nv_bfloat16* dst = gbase + st_goff + size_t(s0 + st_slot0) * slot_elems + size_t(kv) * cache_block_elems(D);

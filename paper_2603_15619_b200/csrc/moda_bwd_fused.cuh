@@ -332,11 +332,18 @@ struct FusedSmem {
     static constexpr int kdO = kQ + kStages * kTileBytes;      // stages of dO_i
     static constexpr int kdS = kdO + kdOStages * kTileBytes;   // dS^T: 128 keys x 128 queries bf16
     static constexpr int kdSBytes = kTileRows * kTileRows * 2;
-    static constexpr int kStg = kdS + kdSBytes;                // four chunks of 16 feature columns of a dQ tile, fp32, accumulator layout
-    static constexpr int kStgBytes = 64 * kTileRows * 4;
-    static constexpr int kRow = kStg + kStgBytes;              // per stage: -LSE log2e [128], D_t [128]
-    static constexpr int kRowBytes = 2 * kTileRows * 4;
-    static constexpr int kBars = kRow + kStages * kRowBytes;
+    static constexpr int kStg = kdS + kdSBytes;                // ring of 8 KiB chunks (16 feature columns of a dQ tile, fp32, accumulator layout)
+    static constexpr int kStgSlots = (D == 128) ? 3 : 4;       // three measured as fast as four; two cost 3-4 %
+    static constexpr int kStgBytes = kStgSlots * 16 * kTileRows * 4;
+    // Operands of the extra k-step that adds the per-query terms to the two score contractions (see the kernel):
+    // 2 KiB chunks of [128 rows][8 bf16] (unswizzled core matrices, 16 bytes per row): one per Q stage with the
+    // stage's terms, then the two constant "ones" chunks and a zero chunk.
+    static constexpr int kAug = kStg + kStgBytes;
+    static constexpr int kAugChunk = kTileRows * 16;
+    static constexpr int kAugOnesS = kAug + kStages * kAugChunk;
+    static constexpr int kAugOnesD = kAugOnesS + kAugChunk;
+    static constexpr int kAugZero = kAugOnesD + kAugChunk;
+    static constexpr int kBars = kAugZero + kAugChunk;
     static constexpr int kNumBars = 28;
     static constexpr int kMisc = kBars + kNumBars * 8;
     static constexpr int kTotal = kMisc + 16;
@@ -349,7 +356,7 @@ struct FusedSmem {
 
 enum FusedBar : int {
     kFBarKV = 0,
-    kFBarQFull = 1,     // +stage (<= 3), count 32: Q_i and the row terms of the stage have landed
+    kFBarQFull = 1,     // +stage (<= 3), count 32: Q_i and the per-query terms of the stage have landed
     kFBarQEmpty = 4,    // +stage (<= 3): dK_i complete (Q_i, the row terms and the dS buffer are free)
     kFBardOFull = 7,    // +stage (<= 2)
     kFBardOEmpty = 9,   // +stage (<= 2), count 2: dP_i and dV_i complete
@@ -443,6 +450,19 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tmem_relinquish();
     }
+    {   // constant chunks of the extra k-step: 1.0 in columns 0-2 (S) / 4-6 (dP), zero elsewhere; the per-stage chunks start
+        // at zero because the chunk behind the one in use is read too (against the zero chunk: it only has to be finite)
+        constexpr uint32_t kOne2 = 0x3F803F80u, kOne1 = 0x00003F80u;
+        uint4* aug = reinterpret_cast<uint4*>(smem + L::kAug);
+        for (int i = threadIdx.x; i < (L::kStages + 3) * kTileRows; i += L::kThreads) {
+            const int chunk = i / kTileRows;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (chunk == L::kStages) v = make_uint4(kOne2, kOne1, 0u, 0u);
+            if (chunk == L::kStages + 1) v = make_uint4(0u, 0u, kOne2, kOne1);
+            aug[i] = v;
+        }
+        fence_proxy_async_smem();
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -460,7 +480,10 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
     // Register budget: the CTA owns what it was launched with (512 threads x 128 registers), and setmaxnreg.inc blocks until the CTA's own pool can serve it, so the three shares must fit that total.
     constexpr int kRegsLaunch = 128;
     static_assert(L::kThreads == 512, "the register shares below assume 512 threads");
-    constexpr int kRegsRow = (D == 128) ? 136 : 152, kRegsDrain = (D == 128) ? 160 : 152, kRegsOther = (D == 128) ? 80 : 56;
+    // Shares measured (T = 8192 .. 65536): the issuing warps need about 100 registers to keep their descriptors and
+    // barrier addresses without spills; d = 128: 128 / 160 / 96 (42.1 ms at T = 65536 against 44.1 with 136 / 160 / 80),
+    // d = 64: 136 / 136 / 104 (27.6 ms at T = 32768, H = 32 against 28.5 with 152 / 152 / 56).
+    constexpr int kRegsRow = (D == 128) ? 128 : 136, kRegsDrain = (D == 128) ? 160 : 136, kRegsOther = (D == 128) ? 96 : 104;
     static_assert(NROW * kRegsRow + 128 * kRegsDrain + NOTHER * kRegsOther <= L::kThreads * kRegsLaunch, "register shares exceed the CTA's pool");
     // setmaxnreg.inc to less than the current count (or .dec to more) is an illegal instruction
     static_assert(kRegsRow >= kRegsLaunch && kRegsDrain >= kRegsLaunch && kRegsOther <= kRegsLaunch, "setmaxnreg direction");
@@ -478,7 +501,6 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         for (int it = 0; it < n_it; ++it) {
             const int st = it % L::kStages;
             const bool diag = (it % n_per) == 0;             // the query tile is the key tile itself: causal mask
-            const float* rt = reinterpret_cast<const float*>(smem + L::kRow + st * L::kRowBytes) + hc * COLS;
             uint32_t pk[COLS / 2];                           // P_i^T of this thread: COLS values, bf16 pairs
             // ---- P_i^T ----
             const int xb = it % XB;
@@ -494,11 +516,11 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                 tmem_wait_ld();
 #pragma unroll
                 for (int i4 = 0; i4 < COLS / 4; ++i4) {
-                    const float4 nl = *reinterpret_cast<const float4*>(rt + 4 * i4);     // same address for all rows
-                    float e0 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 0]), p.scale_log2, nl.x));
-                    float e1 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 1]), p.scale_log2, nl.y));
-                    float e2 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 2]), p.scale_log2, nl.z));
-                    float e3 = fast_exp2(fmaf(__uint_as_float(sv[4 * i4 + 3]), p.scale_log2, nl.w));
+                    // the contraction has already subtracted LSE / scale from every score of the query's column
+                    float e0 = fast_exp2(__uint_as_float(sv[4 * i4 + 0]) * p.scale_log2);
+                    float e1 = fast_exp2(__uint_as_float(sv[4 * i4 + 1]) * p.scale_log2);
+                    float e2 = fast_exp2(__uint_as_float(sv[4 * i4 + 2]) * p.scale_log2);
+                    float e3 = fast_exp2(__uint_as_float(sv[4 * i4 + 3]) * p.scale_log2);
                     if (diag) {                               // query column c sees key row r iff c >= r
                         const int c = hc * COLS + 4 * i4;
                         if (c + 0 < r) e0 = 0.f;
@@ -529,18 +551,16 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                 tmem_wait_ld();
 #pragma unroll
                 for (int g = 0; g < COLS / 8; ++g) {         // 8 query columns = one 16-byte chunk of the row
-                    const float4 da = *reinterpret_cast<const float4*>(rt + kTileRows + 8 * g);
-                    const float4 db = *reinterpret_cast<const float4*>(rt + kTileRows + 8 * g + 4);
-                    const uint32_t* pp = pk + 4 * g;
+                    const uint32_t* pp = pk + 4 * g;         // gv holds dP - D_t already (subtracted by the contraction)
                     uint4 v;
-                    v.x = pack_bf16x2(bf16_lo_to_f32(pp[0]) * (__uint_as_float(gv[8 * g + 0]) - da.x),
-                                      bf16_hi_to_f32(pp[0]) * (__uint_as_float(gv[8 * g + 1]) - da.y));
-                    v.y = pack_bf16x2(bf16_lo_to_f32(pp[1]) * (__uint_as_float(gv[8 * g + 2]) - da.z),
-                                      bf16_hi_to_f32(pp[1]) * (__uint_as_float(gv[8 * g + 3]) - da.w));
-                    v.z = pack_bf16x2(bf16_lo_to_f32(pp[2]) * (__uint_as_float(gv[8 * g + 4]) - db.x),
-                                      bf16_hi_to_f32(pp[2]) * (__uint_as_float(gv[8 * g + 5]) - db.y));
-                    v.w = pack_bf16x2(bf16_lo_to_f32(pp[3]) * (__uint_as_float(gv[8 * g + 6]) - db.z),
-                                      bf16_hi_to_f32(pp[3]) * (__uint_as_float(gv[8 * g + 7]) - db.w));
+                    v.x = pack_bf16x2(bf16_lo_to_f32(pp[0]) * __uint_as_float(gv[8 * g + 0]),
+                                      bf16_hi_to_f32(pp[0]) * __uint_as_float(gv[8 * g + 1]));
+                    v.y = pack_bf16x2(bf16_lo_to_f32(pp[1]) * __uint_as_float(gv[8 * g + 2]),
+                                      bf16_hi_to_f32(pp[1]) * __uint_as_float(gv[8 * g + 3]));
+                    v.z = pack_bf16x2(bf16_lo_to_f32(pp[2]) * __uint_as_float(gv[8 * g + 4]),
+                                      bf16_hi_to_f32(pp[2]) * __uint_as_float(gv[8 * g + 5]));
+                    v.w = pack_bf16x2(bf16_lo_to_f32(pp[3]) * __uint_as_float(gv[8 * g + 6]),
+                                      bf16_hi_to_f32(pp[3]) * __uint_as_float(gv[8 * g + 7]));
                     *reinterpret_cast<uint4*>(ds_row + (((ds_chunk0 + g) ^ (r & 7)) << 4)) = v;
                 }
             }
@@ -607,13 +627,13 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
             tmem_wait_ld();
             tc_fence_before_sync();
             mbar_arrive(bar(kFBarYFree));                    // Y may take dP of the next iteration
-            // 16 feature columns (8 KiB, contiguous in the accumulator) at a time through a ring of four staging chunks:
-            // a chunk is rewritten once the reduction issued from it four chunks earlier has finished reading it, so
-            // up to three reductions stay in flight and L2, not this loop, sets the pace.
+            // 16 feature columns (8 KiB, contiguous in the accumulator) at a time through a ring of staging chunks:
+            // a chunk is rewritten once the reduction issued from it one ring earlier has finished reading it, so
+            // all but one of the ring's reductions stay in flight and L2, not this loop, sets the pace.
 #pragma unroll
             for (int ch = 0; ch < D / 16; ++ch) {
-                const int slot = ch & 3;
-                if (tid == NROW) asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+                const int slot = (it * (D / 16) + ch) % L::kStgSlots;      // the ring runs on across iterations
+                if (tid == NROW) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(L::kStgSlots - 1) : "memory");
                 asm volatile("bar.sync 2, 128;" ::: "memory");
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
@@ -623,7 +643,7 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                 asm volatile("bar.sync 2, 128;" ::: "memory");
                 if (tid == NROW) {
                     asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
-                                 ::"l"(dst + ch * (16 * kTileRows)), "r"(sbase + L::kStg + slot * (L::kStgBytes / 4)), "r"(L::kStgBytes / 4) : "memory");
+                                 ::"l"(dst + ch * (16 * kTileRows)), "r"(sbase + L::kStg + slot * (16 * kTileRows * 4)), "r"(16 * kTileRows * 4) : "memory");
                     tma_store_commit();
                 }
             }
@@ -645,28 +665,29 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                 tma_load_4d(sbase + L::kV + s * L::kSubBytes, &mapV, bar(kFBarKV), s * 64, h, k0, b);
             }
         }
+        const float inv_scale = 1.f / p.scale;
         for (int it = 0; it < n_it; ++it) {
             const int st = it % L::kStages;
             const int hq = h * p.G + it / n_per;
             const size_t row_base = (size_t(b) * p.H + hq) * p.T;
             const int qrow0 = (kt + it % n_per) * kTileRows;
-            // lane handles query columns 4 lane .. 4 lane + 3; queries past T get -LSE = -inf so that P = 0
-            float4 nl, dl;
-            {
-                const int c = qrow0 + 4 * lane;
-                nl.x = (c + 0 < p.T) ? -p.LSE[row_base + c + 0] * kLog2e : -INFINITY;
-                nl.y = (c + 1 < p.T) ? -p.LSE[row_base + c + 1] * kLog2e : -INFINITY;
-                nl.z = (c + 2 < p.T) ? -p.LSE[row_base + c + 2] * kLog2e : -INFINITY;
-                nl.w = (c + 3 < p.T) ? -p.LSE[row_base + c + 3] * kLog2e : -INFINITY;
-                dl.x = (c + 0 < p.T) ? p.delta[row_base + c + 0] : 0.f;
-                dl.y = (c + 1 < p.T) ? p.delta[row_base + c + 1] : 0.f;
-                dl.z = (c + 2 < p.T) ? p.delta[row_base + c + 2] : 0.f;
-                dl.w = (c + 3 < p.T) ? p.delta[row_base + c + 3] : 0.f;
+            // lane handles query columns 4 lane .. 4 lane + 3: for each, -LSE / scale and -D_t as three bf16 parts
+            // (hi + mid + lo = the fp32 value); queries past T get a large negative first term so that P = 0
+            uint4 av[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int c = qrow0 + 4 * lane + j;
+                const float nl = (c < p.T) ? -p.LSE[row_base + c] * inv_scale : -1.0e30f;
+                const float nd = (c < p.T) ? -p.delta[row_base + c] : 0.f;
+                av[j] = make_uint4(0u, 0u, 0u, 0u);
+                split3_bf16(nl, av[j].x, av[j].y);
+                split3_bf16(nd, av[j].z, av[j].w);
             }
             if (it >= L::kStages) mbar_wait(bar(kFBarQEmpty + st), ((it - L::kStages) / L::kStages) & 1, abort_flag, 130);
-            float4* rt = reinterpret_cast<float4*>(smem + L::kRow + st * L::kRowBytes);
-            rt[lane] = nl;
-            rt[kTileRows / 4 + lane] = dl;
+            uint4* aug = reinterpret_cast<uint4*>(smem + L::kAug + st * L::kAugChunk) + 4 * lane;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) aug[j] = av[j];
+            fence_proxy_async_smem();                        // generic-proxy stores -> read by the MMAs (async proxy)
             if (lane == 0) {
                 mbar_arrive_expect_tx(bar(kFBarQFull + st), L::kTileBytes);
 #pragma unroll
@@ -694,6 +715,11 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
             // counts 16-byte units and stays inside its 14 bits below 256 KiB)
             const uint64_t da0 = desc_kmajor_sw128(a_tile, 0);
             const uint64_t db0 = desc_kmajor_sw128(sbase + (is_s ? L::kQ : L::kdO), 0);
+            // extra k-step: A = ones in the columns of this contraction's terms (second k-chunk: the zero chunk),
+            // B = the Q stage's chunk of per-query terms (second k-chunk: whatever follows it, finite, times zero)
+            const uint64_t da_aug = make_smem_desc_noswz(sbase + (is_s ? L::kAugOnesS : L::kAugOnesD),
+                                                         uint32_t(L::kAugZero - (is_s ? L::kAugOnesS : L::kAugOnesD)), 128u);
+            const uint64_t db_aug0 = make_smem_desc_noswz(sbase + L::kAug, uint32_t(L::kAugChunk), 128u);
             mbar_wait(bar(kFBarKV), 0, abort_flag, 140);
             const int nst = is_s ? L::kStages : L::kdOStages;
             for (int it = 0; it < n_it; ++it) {
@@ -705,12 +731,16 @@ moda_bwd_fused_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
                 const uint32_t free_bar = is_s ? bar(kFBarXFree + xb) : bar(kFBarYFree);
                 if (it >= nb) mbar_wait2(bar(full0 + st), (it / nst) & 1, free_bar, ((it - nb) / nb) & 1, abort_flag, 141, is_s ? 142 : 143);
                 else mbar_wait(bar(full0 + st), (it / nst) & 1, abort_flag, 141);
+                // dP also needs the Q stage's per-query terms (they arrive with Q_i)
+                const int qst = it % L::kStages;
+                if (!is_s) mbar_wait(bar(kFBarQFull + qst), (it / L::kStages) & 1, abort_flag, 147);
                 tc_fence_after_sync();
                 const uint64_t db = db0 + uint64_t((st * L::kTileBytes) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk)
                     umma_ss(tmem + col, da0 + uint64_t(((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4),
                             db + uint64_t(((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4), idesc_s, kk > 0);
+                umma_ss(tmem + col, da_aug, db_aug0 + uint64_t((qst * L::kAugChunk) >> 4), idesc_s, 1u);
                 umma_commit(bar(is_s ? kFBarSFull + xb : kFBardPFull));
                 if (!is_s) umma_commit(bar(kFBardOEmpty + st));
             }

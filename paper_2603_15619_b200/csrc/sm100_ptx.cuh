@@ -250,6 +250,17 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uin
     return d;
 }
 
+// Unswizzled K-major operand: core matrices of 8 rows x 16 bytes stored contiguously (128 bytes); `sbo_bytes` from one
+// 8-row group to the next (M / N direction), `lbo_bytes` from the first 8 contraction elements to the second 8.
+__device__ __forceinline__ uint64_t make_smem_desc_noswz(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= uint64_t((smem_addr & 0x3ffffu) >> 4);
+    d |= uint64_t((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= uint64_t((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= uint64_t(1) << 46;
+    return d;
+}
+
 // A tile stored as [rows][64 bf16] (128-byte rows, 8-row swizzle atoms of 1024 bytes), as a
 // TMA box {64, rows} with 128B swizzle leaves it.
 //  * used K-major (the 64-wide direction is the contraction): rows are M/N; successive 8-row
@@ -415,6 +426,17 @@ __device__ __forceinline__ void e4m3x4_to_f32(uint32_t w, float& f0, float& f1, 
         "cvt.f32.f16 %0, a;\n"
         "cvt.f32.f16 %1, b;\n"
         "}\n" : "=f"(f2), "=f"(f3) : "r"(h23));
+}
+// x = hi + mid + lo with three bf16 values (3 x 8 significant bits: exact for every fp32 x whose parts stay normal);
+// w01 = {hi, mid}, w2 = {lo, 0} as packed pairs, low half first.
+__device__ __forceinline__ void split3_bf16(float x, uint32_t& w01, uint32_t& w2) {
+    const uint32_t hi = pack_bf16x2(x, 0.f) & 0xffffu;
+    const float r1 = x - __uint_as_float(hi << 16);
+    const uint32_t mid = pack_bf16x2(r1, 0.f) & 0xffffu;
+    const float r2 = r1 - __uint_as_float(mid << 16);
+    const uint32_t lo = pack_bf16x2(r2, 0.f) & 0xffffu;
+    w01 = hi | (mid << 16);
+    w2 = lo;
 }
 __device__ __forceinline__ float bf16_lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16_hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }

@@ -244,6 +244,7 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
         configured_dev = dev;
     }
     FwdParams p;
+    p.Q = static_cast<const __nv_bfloat16*>(Q);
     p.depth_kv = depth_kv;
     p.O = static_cast<__nv_bfloat16*>(O);
     p.LSE = LSE;
@@ -252,7 +253,8 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.G = H / Hk;
     p.scale_log2 = scale * kLog2e;
     p.append_slot = static_cast<__nv_bfloat16*>(append_slot);
-    const unsigned grid = unsigned(B) * H * num_tiles(T);
+    // the d = 128 kernel takes a pair of query tiles per CTA, the d = 64 kernel one tile
+    const unsigned grid = unsigned(B) * H * (kWide ? num_tiles(T) : num_tile_pairs(num_tiles(T)));
     // Grouped-query calls: the sequence kernel runs without depth slots and a second kernel adds the depth
     // part of all heads of a group at once (moda_depth_gqa.cuh).
     // An e4m3 cache is always read by the row-local depth warps of the sequence kernel.

@@ -80,11 +80,13 @@ enum FwdBar : int {
     kBarVEmpty = 7,   // +stage: PV_j complete (V stage and score buffer free; O may be rescaled)
     kBarSFull = 9,    // +buffer: S_j complete (also frees the K stage)
     kBarPFull = 11,   // +buffer
+    kBarDrain2 = 13,  // abort path of the second issuer
     kBarDepth = 14,
     kBarOFinal = 15,  // single phase: every MMA of the CTA has completed
     kBarDrain = 16,
     kBarDFull = 17,   // +ring stage (<= 6): depth unit landed
     kBarDEmpty = 23,  // +ring stage (<= 6): all 128 depth threads have read the unit
+    kBarTileDone = 29,  // one phase per query tile of the CTA: its epilogue (output stored, slot written) is complete
 };
 
 // Depth slots per group of the forward's online softmax over the depth keys (one group's scores fit
@@ -92,6 +94,7 @@ enum FwdBar : int {
 constexpr int kFwdDepthGroup = 32;
 
 struct FwdParams {
+    const __nv_bfloat16* Q;          // [B][T][H][d]: the depth warps read their rows straight from global memory
     const void* depth_kv;            // cache layout (bf16, or e4m3 codes + scales), >= l slots (unused when l == 0)
     __nv_bfloat16* O;
     float* LSE;
@@ -122,6 +125,15 @@ __device__ __forceinline__ TileCoord tile_coord(int block, int nq, int H, int G)
     c.hk = bhk % Hk;
     c.h = c.hk * G + rem % G;
     c.qt = nq - 1 - rem / G;
+    return c;
+}
+// The d = 128 kernel gives a CTA a *pair* of query tiles of one head, the p-th from the end and the p-th from the
+// start (one tile when they coincide): under the causal mask every pair has the same number of key tiles, and the
+// depth stream of the short tile is worked on while the long tile's key loop still runs.
+__host__ __device__ inline int num_tile_pairs(int nq) { return (nq + 1) / 2; }
+__device__ __forceinline__ TileCoord pair_coord(int block, int nq, int H, int G) {
+    TileCoord c = tile_coord(block, num_tile_pairs(nq), H, G);
+    c.qt = num_tile_pairs(nq) - 1 - c.qt;        // pair index p; its tiles are nq - 1 - p (first) and p
     return c;
 }
 
@@ -178,12 +190,16 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     const int lane = tid & 31;
 
     const int nq = num_tiles(p.T);
-    const TileCoord tc = tile_coord(blockIdx.x, nq, p.H, p.G);
-    const int b = tc.b, h = tc.h, hk = tc.hk, qt = tc.qt;
+    const TileCoord tc = pair_coord(blockIdx.x, nq, p.H, p.G);
+    const int b = tc.b, h = tc.h, hk = tc.hk;
     const int Hk = p.H / p.G;
-    const int q0 = qt * kTileRows;
+    // the CTA's query tiles, the longer one first; every role walks them in this order
+    const int n_tiles = (nq - 1 - tc.qt != tc.qt) ? 2 : 1;
+    auto tile_qt = [&](int t) { return t == 0 ? nq - 1 - tc.qt : tc.qt; };
     // causal: key tiles up to the one that holds the last row's own position (row i sees keys <= i + kv_off)
-    const int n_kv = min((q0 + kTileRows + p.kv_off + kTileRows - 1) / kTileRows, num_tiles(p.T_kv));
+    auto tile_nkv = [&](int t) {
+        return min((tile_qt(t) * kTileRows + kTileRows + p.kv_off + kTileRows - 1) / kTileRows, num_tiles(p.T_kv));
+    };
 
     if (tid == 0) {
         *abort_flag = 0;
@@ -196,8 +212,10 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             mbar_init(bar(kBarPFull + s), 128);
         }
         mbar_init(bar(kBarDepth), 128);
+        mbar_init(bar(kBarTileDone), 1);
         mbar_init(bar(kBarOFinal), 1);
         mbar_init(bar(kBarDrain), 1);
+        mbar_init(bar(kBarDrain2), 1);
         for (int s = 0; s < L::kRingStages; ++s) {
             mbar_init(bar(kBarDFull + s), 1);
             mbar_init(bar(kBarDEmpty + s), 128);
@@ -220,12 +238,16 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         setmaxnreg_inc<216>();
         const int r = tid;                               // query row inside the tile = TMEM lane
         const uint32_t lane_addr = uint32_t(warp * 32) << 16;
+        int jbase = 0;                                   // key tiles of the CTA's earlier query tiles: the rings run on
+        for (int t = 0; t < n_tiles; ++t) {
+        const int qt = tile_qt(t), q0 = qt * kTileRows, n_kv = tile_nkv(t);
         float m_ref = -INFINITY;                         // reference maximum (log2 domain) the stored P, O use
         float l_sum = 0.f;
         for (int j = 0; j < n_kv; ++j) {
-            const int buf = j & 1;
+            const int jj = jbase + j;
+            const int buf = jj & 1;
             const uint32_t tS = tmem + lane_addr + uint32_t(buf) * 128u;
-            mbar_wait(bar(kBarSFull + buf), (j >> 1) & 1, abort_flag, 10);
+            mbar_wait(bar(kBarSFull + buf), (jj >> 1) & 1, abort_flag, 10);
             tc_fence_after_sync();
             uint32_t s0[32], s1[32], s2[32], s3[32];
             tmem_ld32(tS + 0, s0);
@@ -258,7 +280,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 // The maximum grew a lot: bring O and l to the new reference.  O may only be
                 // touched between PV_{j-1} completing and PV_j being issued; PV_j waits for
                 // this thread's arrival on kBarPFull below.
-                mbar_wait(bar(kBarVEmpty + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag, 11);
+                mbar_wait(bar(kBarVEmpty + ((jj - 1) & 1)), ((jj - 1) >> 1) & 1, abort_flag, 11);
                 tc_fence_after_sync();
                 const float f = fast_exp2(m_ref - m_new);
 #pragma unroll
@@ -304,11 +326,11 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         }
 
         // ------------------------------ epilogue ------------------------------
-        mbar_wait(bar(kBarOFinal), 0, abort_flag, 12);
+        mbar_wait(bar(kBarOFinal), t & 1, abort_flag, 12);
         tc_fence_after_sync();
         float a_s = 1.f, a_d = 0.f, m_fin = m_ref, l_fin = l_sum;
         if (p.l > 0) {
-            mbar_wait(bar(kBarDepth), 0, abort_flag, 13);
+            mbar_wait(bar(kBarDepth), t & 1, abort_flag, 13);
             tc_fence_after_sync();
             const float m_d = sMd[r], l_d = sLd[r];
             m_fin = fmaxf(m_ref, m_d);
@@ -355,14 +377,28 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             tma_store_commit();
             tma_store_wait_all();
         }
+        if (p.append_slot != nullptr && h == hk * p.G) {
+            // Every MMA of the tile has completed, so no load is in flight and its last key tile (the diagonal one)
+            // sits in its stages: the waits are on phases that have completed and make the TMA writes visible here.
+            const int jl = jbase + n_kv - 1;
+            mbar_wait2(bar(kBarKFull + jl % KST), (jl / KST) & 1, bar(kBarVFull + (jl & 1)), (jl >> 1) & 1, abort_flag, 23, 24);
+            append_rows_to_slot<D>(p.append_slot, smem + L::kK + (jl % KST) * L::kTileBytes, smem + L::kV + (jl & 1) * L::kTileBytes,
+                                   (size_t(b) * Hk + hk) * nq + qt, r);
+        }
+        // The tile is done: the Q buffer (output staging), the K / V stages the slot was copied from, O and the depth
+        // partial in tensor memory may be reused for the CTA's next tile.
+        tc_fence_before_sync();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (tid == 0) mbar_arrive(bar(kBarTileDone));
+        jbase += n_kv;
+        }
     } else if (warp < 8) {
         // =========================== depth partial state ===========================
         setmaxnreg_inc<216>();
         if (p.l > 0) {
             const int r = tid - 128;
             const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
-            mbar_wait(bar(kBarQ), 0, abort_flag, 20);
-            int unit = 0;                                 // running index into the producer's unit sequence
+            int unit = 0;                                 // running index into the producer's unit sequence (over all tiles)
             // Reads this thread's 8 x 16 bytes of the next depth unit from the ring and frees the stage.
             auto take_unit = [&](uint4 (&dst)[8]) {
                 const int st = unit % L::kRingStages;
@@ -379,6 +415,14 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             // The slots are handled in groups of kFwdDepthGroup (the score scratch holds one group): an
             // online softmax over the groups, with the partial output o_d rescaled in TMEM when a later
             // group raises the maximum.  Up to 32 slots are one group.
+            for (int t = 0; t < n_tiles; ++t) {
+            const int qt = tile_qt(t), q0 = qt * kTileRows;
+            // this thread's query row (zeros past T, as the TMA-loaded tile has them)
+            const bool qvalid = q0 + r < p.T;
+            const uint4* qrow = reinterpret_cast<const uint4*>(p.Q + ((size_t(b) * p.T + (qvalid ? q0 + r : 0)) * p.H + h) * D);
+            // The depth partial of the CTA's previous tile stays parked (tensor memory, sMd / sLd) until that tile's
+            // epilogue has read it; this tile's slots are streamed and used meanwhile, only the first store waits.
+            auto wait_previous_tile = [&]() { if (t > 0) mbar_wait(bar(kBarTileDone), (t - 1) & 1, abort_flag, 25); };
             float m_d = -INFINITY, l_d = 0.f;
             if constexpr (FP8) {
                 // e4m3 cache: a unit holds all D features of one slot's keys (values) for the tile's rows, its row
@@ -403,7 +447,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                         float q[D];
 #pragma unroll
                         for (int c = 0; c < D / 8; ++c) {
-                            const uint4 v = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, c));
+                            const uint4 v = qvalid ? __ldg(qrow + c) : make_uint4(0u, 0u, 0u, 0u);
                             q[8 * c + 0] = bf16_lo_to_f32(v.x); q[8 * c + 1] = bf16_hi_to_f32(v.x);
                             q[8 * c + 2] = bf16_lo_to_f32(v.y); q[8 * c + 3] = bf16_hi_to_f32(v.y);
                             q[8 * c + 4] = bf16_lo_to_f32(v.z); q[8 * c + 5] = bf16_hi_to_f32(v.z);
@@ -476,6 +520,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                                 }
                             }
                         }
+                        if (g0 == 0) wait_previous_tile();
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c) {
                             uint32_t o[32];
@@ -496,7 +541,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                     float q[64];
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        const uint4 v = *reinterpret_cast<const uint4*>(smem + L::kQ + swz_chunk_offset(r, half * 8 + c));
+                        const uint4 v = qvalid ? __ldg(qrow + half * 8 + c) : make_uint4(0u, 0u, 0u, 0u);
                         q[8 * c + 0] = bf16_lo_to_f32(v.x); q[8 * c + 1] = bf16_hi_to_f32(v.x);
                         q[8 * c + 2] = bf16_lo_to_f32(v.y); q[8 * c + 3] = bf16_hi_to_f32(v.y);
                         q[8 * c + 4] = bf16_lo_to_f32(v.z); q[8 * c + 5] = bf16_hi_to_f32(v.z);
@@ -568,6 +613,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                             acc[8 * c + 7] = fmaf(w, bf16_hi_to_f32(cur[c].w), acc[8 * c + 7]);
                         }
                     }
+                    if (g0 == 0 && half == 0) wait_previous_tile();
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
                         uint32_t o[32];
@@ -584,15 +630,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(kBarDepth));
-        }
-        if (p.append_slot != nullptr && h == hk * p.G) {
-            // Every MMA has completed, so no load is in flight and the last tiles sit in their stages; the
-            // second and third waits are on phases that have completed and make the TMA writes visible here.
-            const int j = n_kv - 1;
-            mbar_wait(bar(kBarOFinal), 0, abort_flag, 22);
-            mbar_wait2(bar(kBarKFull + j % KST), (j / KST) & 1, bar(kBarVFull + (j & 1)), (j >> 1) & 1, abort_flag, 23, 24);
-            append_rows_to_slot<D>(p.append_slot, smem + L::kK + (j % KST) * L::kTileBytes, smem + L::kV + (j & 1) * L::kTileBytes,
-                                   (size_t(b) * Hk + hk) * nq + qt, tid - 128);
+            }
         }
     } else {
       setmaxnreg_dec<72>();   // one instruction for the whole producer warpgroup (warps 8-11)
@@ -602,25 +640,33 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             tma_prefetch_desc(&mapQ);
             tma_prefetch_desc(&mapK);
             tma_prefetch_desc(&mapV);
-            mbar_arrive_expect_tx(bar(kBarQ), L::kTileBytes);
-#pragma unroll
-            for (int s = 0; s < NSUB; ++s)
-                tma_load_4d(sbase + L::kQ + s * L::kSubBytes, &mapQ, bar(kBarQ), s * 64, h, q0, b);
-            for (int j = 0; j < n_kv; ++j) {
-                const int st = j & 1, kst = j % KST;
-                // the K stage is free once S of its previous tile (j - KST) has completed
-                if (j >= KST) mbar_wait(bar(kBarSFull + ((j - KST) & 1)), ((j - KST) >> 1) & 1, abort_flag, 30);
-                mbar_arrive_expect_tx(bar(kBarKFull + kst), L::kTileBytes);
+            int jbase = 0;
+            for (int t = 0; t < n_tiles; ++t) {
+                const int q0 = tile_qt(t) * kTileRows, n_kv = tile_nkv(t);
+                // the Q buffer doubles as the output staging of the previous tile, and the slot write reads its last stages
+                if (t > 0) mbar_wait(bar(kBarTileDone), (t - 1) & 1, abort_flag, 33);
+                mbar_arrive_expect_tx(bar(kBarQ), L::kTileBytes);
 #pragma unroll
                 for (int s = 0; s < NSUB; ++s)
-                    tma_load_4d(sbase + L::kK + kst * L::kTileBytes + s * L::kSubBytes, &mapK, bar(kBarKFull + kst),
-                                s * 64, hk, j * kTileRows, b);
-                if (j >= 2) mbar_wait(bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 31);
-                mbar_arrive_expect_tx(bar(kBarVFull + st), L::kTileBytes);
+                    tma_load_4d(sbase + L::kQ + s * L::kSubBytes, &mapQ, bar(kBarQ), s * 64, h, q0, b);
+                for (int j = 0; j < n_kv; ++j) {
+                    const int jj = jbase + j;
+                    const int st = jj & 1, kst = jj % KST;
+                    // the K stage is free once S of its previous tile (jj - KST) has completed
+                    if (jj >= KST) mbar_wait(bar(kBarSFull + ((jj - KST) & 1)), ((jj - KST) >> 1) & 1, abort_flag, 30);
+                    mbar_arrive_expect_tx(bar(kBarKFull + kst), L::kTileBytes);
 #pragma unroll
-                for (int s = 0; s < NSUB; ++s)
-                    tma_load_4d(sbase + L::kV + st * L::kTileBytes + s * L::kSubBytes, &mapV, bar(kBarVFull + st),
-                                s * 64, hk, j * kTileRows, b);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_4d(sbase + L::kK + kst * L::kTileBytes + s * L::kSubBytes, &mapK, bar(kBarKFull + kst),
+                                    s * 64, hk, j * kTileRows, b);
+                    if (jj >= 2) mbar_wait(bar(kBarVEmpty + st), ((jj - 2) >> 1) & 1, abort_flag, 31);
+                    mbar_arrive_expect_tx(bar(kBarVFull + st), L::kTileBytes);
+#pragma unroll
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_4d(sbase + L::kV + st * L::kTileBytes + s * L::kSubBytes, &mapV, bar(kBarVFull + st),
+                                    s * 64, hk, j * kTileRows, b);
+                }
+                jbase += n_kv;
             }
         }
       } else if (warp == 9) {
@@ -633,12 +679,16 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) dq[kk] = desc_kmajor_sw128(sbase + L::kQ + (kk >> 2) * L::kSubBytes, kk & 3);
             const uint64_t dk0 = desc_kmajor_sw128(sbase + L::kK, 0);
-            mbar_wait(bar(kBarQ), 0, abort_flag, 41);
+            int jbase = 0;
+            for (int t = 0; t < n_tiles; ++t) {
+            const int n_kv = tile_nkv(t);
+            mbar_wait(bar(kBarQ), t & 1, abort_flag, 41);
             for (int j = 0; j < n_kv; ++j) {
-                const int st = j & 1, kst = j % KST;
-                // score buffer st still holds P_{j-2} until PV_{j-2} has completed
-                if (j >= 2) mbar_wait2(bar(kBarKFull + kst), (j / KST) & 1, bar(kBarVEmpty + st), ((j - 2) >> 1) & 1, abort_flag, 40, 44);
-                else mbar_wait(bar(kBarKFull + kst), (j / KST) & 1, abort_flag, 40);
+                const int jj = jbase + j;
+                const int st = jj & 1, kst = jj % KST;
+                // score buffer st still holds P_{jj-2} until PV_{jj-2} has completed
+                if (jj >= 2) mbar_wait2(bar(kBarKFull + kst), (jj / KST) & 1, bar(kBarVEmpty + st), ((jj - 2) >> 1) & 1, abort_flag, 40, 44);
+                else mbar_wait(bar(kBarKFull + kst), (jj / KST) & 1, abort_flag, 40);
                 tc_fence_after_sync();
                 const uint64_t dk = dk0 + uint64_t((kst * L::kTileBytes) >> 4);
                 const uint32_t ts = tmem + uint32_t(st) * 128u;
@@ -646,6 +696,8 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                 for (int kk = 0; kk < D / 16; ++kk)
                     umma_ss(ts, dq[kk], dk + uint64_t(((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4), idesc_s, kk > 0);
                 umma_commit(bar(kBarSFull + st));
+            }
+            jbase += n_kv;
             }
             if (*abort_flag != 0) {
                 // A wait gave up somewhere: make sure no MMA of this thread is still in flight before TMEM is released.
@@ -659,9 +711,13 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         {   // whole warp: operands are warp-uniform, one elected lane issues
             constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
             const uint64_t dv0 = desc_mnmajor_sw128(sbase + L::kV, 0, L::kSubBytes);
+            int jbase = 0;
+            for (int t = 0; t < n_tiles; ++t) {
+            const int n_kv = tile_nkv(t);
             for (int j = 0; j < n_kv; ++j) {
-                const int st = j & 1;
-                mbar_wait2(bar(kBarVFull + st), (j >> 1) & 1, bar(kBarPFull + st), (j >> 1) & 1, abort_flag, 42, 43);
+                const int jj = jbase + j;
+                const int st = jj & 1;
+                mbar_wait2(bar(kBarVFull + st), (jj >> 1) & 1, bar(kBarPFull + st), (jj >> 1) & 1, abort_flag, 42, 43);
                 tc_fence_after_sync();
                 const uint64_t dv = dv0 + uint64_t((st * L::kTileBytes) >> 4);
                 const uint32_t tp = tmem + uint32_t(st) * 128u;
@@ -671,12 +727,15 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                     umma_ts(tmem + kColO, tp + kk * 8, dv + uint64_t(kk * 128), idesc_o, 1);
                 umma_commit(bar(kBarVEmpty + st));
             }
-            // All S MMAs completed before the P they fed was written, so the last PV is the last MMA.
+            // All S MMAs of the tile completed before the P they fed was written, so its last PV is its last MMA.
             umma_commit(bar(kBarOFinal));
+            jbase += n_kv;
+            }
             if (*abort_flag != 0) {
                 // A wait gave up somewhere: make sure no MMA is still in flight before TMEM is released.
+                umma_commit(bar(kBarDrain2));
                 const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(bar(kBarOFinal), 0) && globaltimer_ns() - t0 < 20000000ull) {}
+                while (!mbar_try_wait(bar(kBarDrain2), 0) && globaltimer_ns() - t0 < 20000000ull) {}
             }
         }
       } else if (warp == 10) {
@@ -689,8 +748,9 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             const uint64_t policy = l2_policy_evict_first();
             const size_t slot_bytes = cache8_slot_bytes(p.B, p.T, Hk, D);
             const size_t blk_bytes = cache8_block_bytes(D);
-            const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) + (((size_t(b) * Hk + hk) * nq + qt) * 2) * blk_bytes;
             int unit = 0;
+            for (int t = 0; t < n_tiles; ++t) {
+            const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) + (((size_t(b) * Hk + hk) * nq + tile_qt(t)) * 2) * blk_bytes;
             for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
                 const int gl = min(kFwdDepthGroup, p.l - g0);
                 for (int kv = 0; kv < 2; ++kv)
@@ -704,12 +764,14 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                         bulk_load(sbase + L::kScale + st * L::kScaleBytes, src + L::kUnitBytes, L::kScaleBytes, bar(kBarDFull + st), policy);
                     }
             }
+            }
         } else if (lane == 0 && p.l > 0) {
             const uint64_t policy = l2_policy_evict_first();          // the depth cache is read exactly once
             const size_t slot_bytes = cache_slot_elems(p.B, p.T, Hk, D) * 2;
-            const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
-                                 (((size_t(b) * Hk + hk) * nq + qt) * 2) * (size_t(kTileRows) * D * 2);
             int unit = 0;
+            for (int t = 0; t < n_tiles; ++t) {
+            const uint8_t* blk = reinterpret_cast<const uint8_t*>(p.depth_kv) +
+                                 (((size_t(b) * Hk + hk) * nq + tile_qt(t)) * 2) * (size_t(kTileRows) * D * 2);
             for (int g0 = 0; g0 < p.l; g0 += kFwdDepthGroup) {
                 const int gl = min(kFwdDepthGroup, p.l - g0);
                 for (int kv = 0; kv < 2; ++kv)
@@ -723,6 +785,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
                                       blk + size_t(g0 + i) * slot_bytes + size_t(kv) * (size_t(kTileRows) * D * 2) + size_t(half) * L::kUnitBytes,
                                       L::kUnitBytes, bar(kBarDFull + st), policy);
                         }
+            }
             }
         }
       }

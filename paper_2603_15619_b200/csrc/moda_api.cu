@@ -200,9 +200,10 @@ int launch_depth_merge(DepthMergeParams m, cudaStream_t stream) {
         case 6: return launch_depth_merge_g<D, 6>(m, stream);
         case 7: return launch_depth_merge_g<D, 7>(m, stream);
         case 8: return launch_depth_merge_g<D, 8>(m, stream);
-        case 16: case 32:
-            for (m.h0 = 0; m.h0 < G; m.h0 += 8)
-                if (int rc = launch_depth_merge_g<D, 8>(m, stream)) return rc;
+        case 16: return launch_depth_merge_g<D, 16>(m, stream);       // 16 heads fill the 16 rows of the warp-level products
+        case 32:
+            for (m.h0 = 0; m.h0 < G; m.h0 += 16)
+                if (int rc = launch_depth_merge_g<D, 16>(m, stream)) return rc;
             return MODA_OK;
         default: return MODA_ERR_BAD_GROUP;
     }
@@ -303,7 +304,7 @@ inline bool gqa_depth_split_bwd(int d, int G, int l) {
 
 template <int D, int G>
 int launch_depth_bwd_g(const DepthBwdParams& m, cudaStream_t stream) {
-    constexpr int kBytes = DepthBwdSmem<D>::kTotal;
+    constexpr int kBytes = DepthBwdSmem<D, G>::kTotal;
     static thread_local int configured_dev = -1;
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
@@ -328,10 +329,11 @@ int launch_depth_bwd(DepthBwdParams m, cudaStream_t stream) {
         case 6: return launch_depth_bwd_g<D, 6>(m, stream);
         case 7: return launch_depth_bwd_g<D, 7>(m, stream);
         case 8: return launch_depth_bwd_g<D, 8>(m, stream);
-        case 16: case 32:
-            for (m.h0 = 0; m.h0 < G; m.h0 += 8) {
-                if (int rc = launch_depth_bwd_g<D, 8>(m, stream)) return rc;
-                m.accumulate = 1;                                   // the later groups of 8 add to the first one's gradients
+        case 16: return launch_depth_bwd_g<D, 16>(m, stream);      // 16 heads fill the 16 rows (or the 16-deep contraction)
+        case 32:
+            for (m.h0 = 0; m.h0 < G; m.h0 += 16) {
+                if (int rc = launch_depth_bwd_g<D, 16>(m, stream)) return rc;
+                m.accumulate = 1;                                   // the second group of 16 adds to the first one's gradients
             }
             return MODA_OK;
         default: return MODA_ERR_BAD_GROUP;

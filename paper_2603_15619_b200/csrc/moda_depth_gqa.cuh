@@ -72,15 +72,23 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
     const int g = lane >> 2, tq = lane & 3;
     const int t = t0 + warp;                                   // this warp's position
     const bool live = t < p.T;
+    // More than 8 heads (G = 16): heads 8 .. 15 are rows 8 .. 15 of the same 16-row products, whose second half is
+    // otherwise zero padding; a lane then carries the state of heads g and g + 8.
+    constexpr bool kTwo = G > 8;
 
     // A fragments of Q_t: this lane's 8 features of head g for every 32 features (the same features it
     // takes from a depth key row below)
-    uint4 qf[D / 32];
+    uint4 qf[D / 32], qf2[kTwo ? D / 32 : 1];
 #pragma unroll
     for (int kp = 0; kp < D / 32; ++kp) {
         qf[kp] = make_uint4(0u, 0u, 0u, 0u);
         if (live && g < G)
             qf[kp] = *reinterpret_cast<const uint4*>(p.Q + ((size_t(b) * p.T + t) * p.H + hk * (p.H / p.Hk) + p.h0 + g) * D + (4 * kp + tq) * 8);
+        if constexpr (kTwo) {
+            qf2[kp] = make_uint4(0u, 0u, 0u, 0u);
+            if (live && g + 8 < G)
+                qf2[kp] = *reinterpret_cast<const uint4*>(p.Q + ((size_t(b) * p.T + t) * p.H + hk * (p.H / p.Hk) + p.h0 + g + 8) * D + (4 * kp + tq) * 8);
+        }
     }
 
     // the sequence kernel's output row and LSE of head g, requested now so that they are there at the end
@@ -93,6 +101,17 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
         for (int fb = 0; fb < D / 8; ++fb) os[fb] = *reinterpret_cast<const uint32_t*>(orow + 8 * fb + 2 * tq);
         lse_seq = p.LSE[(size_t(b) * p.H + h) * p.T + t];
     }
+    uint32_t os2[kTwo ? D / 8 : 1];
+    float lse_seq2 = 0.f;
+    if constexpr (kTwo) {
+        if (live && g + 8 < G) {
+            const int h = hk * (p.H / p.Hk) + p.h0 + g + 8;
+            const __nv_bfloat16* orow = p.O + ((size_t(b) * p.T + t) * p.H + h) * D;
+#pragma unroll
+            for (int fb = 0; fb < D / 8; ++fb) os2[fb] = *reinterpret_cast<const uint32_t*>(orow + 8 * fb + 2 * tq);
+            lse_seq2 = p.LSE[(size_t(b) * p.H + h) * p.T + t];
+        }
+    }
 
     // cache addressing: block (slot, b, hk, tile, kv) holds [chunk][row 128][8]; the CTA's positions are rows
     // r0 .. r0 + kDgPos - 1 of tile t0 / 128 (kDgPos divides 128, so they never straddle tiles)
@@ -102,6 +121,7 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
     const uint32_t smem_base = smem_u32(dg_smem);
 
     float m_run = -INFINITY, lsum = 0.f;
+    float m_run2 = -INFINITY, lsum2 = 0.f;                     // heads g + 8
     float o[D / 8][4];
 #pragma unroll
     for (int fb = 0; fb < D / 8; ++fb) { o[fb][0] = 0.f; o[fb][1] = 0.f; o[fb][2] = 0.f; o[fb][3] = 0.f; }
@@ -164,7 +184,7 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
         __syncthreads();
         if (live) {
             // ---- scores of head g against 8 slots per block ----
-            float sc[kDgSlots / 8][2];
+            float sc[kDgSlots / 8][2], sc2[kDgSlots / 8][2];
 #pragma unroll
             for (int nb = 0; nb < kDgSlots / 8; ++nb) {
                 float c[4] = {0.f, 0.f, 0.f, 0.f};
@@ -173,12 +193,19 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
 #pragma unroll
                     for (int kp = 0; kp < D / 32; ++kp) {
                         const uint4 kvv = *reinterpret_cast<const uint4*>(sK + dg_row_piece<D>(warp, slot, 4 * kp + tq));
-                        mma_bf16_16x8x16(c, qf[kp].x, 0u, qf[kp].y, 0u, kvv.x, kvv.y);
-                        mma_bf16_16x8x16(c, qf[kp].z, 0u, qf[kp].w, 0u, kvv.z, kvv.w);
+                        if constexpr (kTwo) {
+                            mma_bf16_16x8x16(c, qf[kp].x, qf2[kp].x, qf[kp].y, qf2[kp].y, kvv.x, kvv.y);
+                            mma_bf16_16x8x16(c, qf[kp].z, qf2[kp].z, qf[kp].w, qf2[kp].w, kvv.z, kvv.w);
+                        } else {
+                            mma_bf16_16x8x16(c, qf[kp].x, 0u, qf[kp].y, 0u, kvv.x, kvv.y);
+                            mma_bf16_16x8x16(c, qf[kp].z, 0u, qf[kp].w, 0u, kvv.z, kvv.w);
+                        }
                     }
                 }
                 sc[nb][0] = (8 * nb + 2 * tq < ns) ? c[0] * p.scale_log2 : -INFINITY;       // slots past l: stale rows
                 sc[nb][1] = (8 * nb + 2 * tq + 1 < ns) ? c[1] * p.scale_log2 : -INFINITY;
+                sc2[nb][0] = (8 * nb + 2 * tq < ns) ? c[2] * p.scale_log2 : -INFINITY;
+                sc2[nb][1] = (8 * nb + 2 * tq + 1 < ns) ? c[3] * p.scale_log2 : -INFINITY;
             }
             float mx = -INFINITY;
 #pragma unroll
@@ -201,6 +228,29 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
 #pragma unroll
                 for (int fb = 0; fb < D / 8; ++fb) { o[fb][0] *= alpha; o[fb][1] *= alpha; }
             }
+            uint32_t pa2[kDgSlots / 8];
+            if constexpr (kTwo) {                              // the same online-softmax step for head g + 8
+                float mx2 = -INFINITY;
+#pragma unroll
+                for (int nb = 0; nb < kDgSlots / 8; ++nb) mx2 = fmaxf(mx2, fmaxf(sc2[nb][0], sc2[nb][1]));
+                mx2 = fmaxf(mx2, __shfl_xor_sync(0xffffffffu, mx2, 1));
+                mx2 = fmaxf(mx2, __shfl_xor_sync(0xffffffffu, mx2, 2));
+                const float m_new2 = fmaxf(m_run2, mx2);
+                const float alpha2 = fast_exp2(m_run2 - m_new2);
+                m_run2 = m_new2;
+                float psum2 = 0.f;
+#pragma unroll
+                for (int nb = 0; nb < kDgSlots / 8; ++nb) {
+                    const float p0 = fast_exp2(sc2[nb][0] - m_new2), p1 = fast_exp2(sc2[nb][1] - m_new2);
+                    psum2 += p0 + p1;
+                    pa2[nb] = pack_bf16x2(p0, p1);
+                }
+                lsum2 = lsum2 * alpha2 + psum2;
+                if (alpha2 != 1.f) {
+#pragma unroll
+                    for (int fb = 0; fb < D / 8; ++fb) { o[fb][2] *= alpha2; o[fb][3] *= alpha2; }
+                }
+            }
             // ---- o_d += P Vd: rows of slots past ns hold stale data with weight 0; zero them first if they
             //      could be NaN (they are rows of an earlier round or uninitialised shared memory) ----
             if (ns < kDgSlots) {
@@ -219,8 +269,13 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
                         const uint32_t addr = smem_u32(sV + dg_row_piece<D>(warp, vslot, fb + (lane >> 4)));
                         uint32_t b0, b1, b2, b3;
                         ldmatrix_x4_trans(addr, b0, b1, b2, b3);
-                        mma_bf16_16x8x16(o[fb], pa[2 * ks], 0u, pa[2 * ks + 1], 0u, b0, b1);
-                        mma_bf16_16x8x16(o[fb + 1], pa[2 * ks], 0u, pa[2 * ks + 1], 0u, b2, b3);
+                        if constexpr (kTwo) {
+                            mma_bf16_16x8x16(o[fb], pa[2 * ks], pa2[2 * ks], pa[2 * ks + 1], pa2[2 * ks + 1], b0, b1);
+                            mma_bf16_16x8x16(o[fb + 1], pa[2 * ks], pa2[2 * ks], pa[2 * ks + 1], pa2[2 * ks + 1], b2, b3);
+                        } else {
+                            mma_bf16_16x8x16(o[fb], pa[2 * ks], 0u, pa[2 * ks + 1], 0u, b0, b1);
+                            mma_bf16_16x8x16(o[fb + 1], pa[2 * ks], 0u, pa[2 * ks + 1], 0u, b2, b3);
+                        }
                     }
                 }
             }
@@ -246,6 +301,26 @@ depth_merge_fwd_kernel(const DepthMergeParams p) {
             *reinterpret_cast<uint32_t*>(orow + 8 * fb + 2 * tq) = pack_bf16x2(a0, a1);
         }
         if (tq == 0) p.LSE[(size_t(b) * p.H + h) * p.T + t] = (mt + log2f(z)) * 0.6931471805599453f;
+    }
+    if constexpr (kTwo) {
+        lsum2 += __shfl_xor_sync(0xffffffffu, lsum2, 1);
+        lsum2 += __shfl_xor_sync(0xffffffffu, lsum2, 2);
+        if (live && g + 8 < G) {
+            const int h = hk * (p.H / p.Hk) + p.h0 + g + 8;
+            const float s2 = lse_seq2 * 1.4426950408889634f;
+            const float mt = fmaxf(s2, m_run2);
+            const float ws = fast_exp2(s2 - mt), wd = fast_exp2(m_run2 - mt);
+            const float z = ws + wd * lsum2;
+            const float inv = 1.f / z;
+            __nv_bfloat16* orow = p.O + ((size_t(b) * p.T + t) * p.H + h) * D;
+#pragma unroll
+            for (int fb = 0; fb < D / 8; ++fb) {
+                const float a0 = (ws * bf16_lo_to_f32(os2[fb]) + wd * o[fb][2]) * inv;
+                const float a1 = (ws * bf16_hi_to_f32(os2[fb]) + wd * o[fb][3]) * inv;
+                *reinterpret_cast<uint32_t*>(orow + 8 * fb + 2 * tq) = pack_bf16x2(a0, a1);
+            }
+            if (tq == 0) p.LSE[(size_t(b) * p.H + h) * p.T + t] = (mt + log2f(z)) * 0.6931471805599453f;
+        }
     }
 }
 
@@ -281,12 +356,13 @@ struct DepthBwdParams {
     int pm;                             // nonzero: depth_kv and d_depth_kv are in the position-major layout (moda_cache.cuh)
 };
 
-template <int D>
+template <int D, int G = 8>
 struct DepthBwdSmem {
     static constexpr int P = db_pos<D>();
+    static constexpr int kHeads = G > 8 ? 16 : 8;                       // head rows kept per position
     static constexpr int kIn = 2 * 2 * P * kDbRoundSlots * D * 2;       // two rounds x (K, V) rows
-    static constexpr int kQd = kIn;                                     // Q_t and dO_t rows: [2][P][8 heads][D]
-    static constexpr int kOut = kQd + 2 * P * 8 * D * 2;                // dKd, dVd of the round: [2][P][16 slots][D]
+    static constexpr int kQd = kIn;                                     // Q_t and dO_t rows: [2][P][8 or 16 heads][D]
+    static constexpr int kOut = kQd + 2 * P * kHeads * D * 2;           // dKd, dVd of the round: [2][P][16 slots][D]
     static constexpr int kTotal = kOut + 2 * P * kDbRoundSlots * D * 2;
 };
 
@@ -299,7 +375,9 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
 template <int D, int G>
 __global__ void __launch_bounds__(db_pos<D>() * 32, 4)
 depth_bwd_gqa_kernel(const DepthBwdParams p) {
-    using L = DepthBwdSmem<D>;
+    using L = DepthBwdSmem<D, G>;
+    constexpr bool kTwo = G > 8;                                   // heads 8 .. 15 as rows 8 .. 15 of the same products
+    constexpr int HR = L::kHeads;
     constexpr int P = L::P, NT = P * 32, CH = D / 8, RS = kDbRoundSlots;
     constexpr int kTensorBytes = P * RS * D * 2;
     extern __shared__ __align__(128) uint8_t db_smem[];
@@ -318,11 +396,13 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
     const bool live = t < p.T;
     const bool head = live && g < G;
     const int h = hk * (p.H / p.Hk) + p.h0 + min(g, G - 1);
+    const bool head2 = kTwo && live && g + 8 < G;
+    const int h2 = hk * (p.H / p.Hk) + p.h0 + min(g + 8, G - 1);
 
     // ---- this position's Q and dO rows: A fragments in registers, and rows in shared memory for the B side ----
-    uint4 qf[D / 32], gf[D / 32];
-    uint8_t* sQ = db_smem + L::kQd + (0 * P + warp) * 8 * D * 2;
-    uint8_t* sG = db_smem + L::kQd + (1 * P + warp) * 8 * D * 2;
+    uint4 qf[D / 32], gf[D / 32], qf2[kTwo ? D / 32 : 1], gf2[kTwo ? D / 32 : 1];
+    uint8_t* sQ = db_smem + L::kQd + (0 * P + warp) * HR * D * 2;
+    uint8_t* sG = db_smem + L::kQd + (1 * P + warp) * HR * D * 2;
 #pragma unroll
     for (int kp = 0; kp < D / 32; ++kp) {
         qf[kp] = make_uint4(0u, 0u, 0u, 0u);
@@ -334,15 +414,35 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
         }
         *reinterpret_cast<uint4*>(sQ + row_piece(g, 4 * kp + tq)) = qf[kp];       // rows of heads past G are zero
         *reinterpret_cast<uint4*>(sG + row_piece(g, 4 * kp + tq)) = gf[kp];
+        if constexpr (kTwo) {
+            qf2[kp] = make_uint4(0u, 0u, 0u, 0u);
+            gf2[kp] = make_uint4(0u, 0u, 0u, 0u);
+            if (head2) {
+                const size_t off = ((size_t(b) * p.T + t) * p.H + h2) * D + (4 * kp + tq) * 8;
+                qf2[kp] = *reinterpret_cast<const uint4*>(p.Q + off);
+                gf2[kp] = *reinterpret_cast<const uint4*>(p.dO + off);
+            }
+            *reinterpret_cast<uint4*>(sQ + row_piece(g + 8, 4 * kp + tq)) = qf2[kp];
+            *reinterpret_cast<uint4*>(sG + row_piece(g + 8, 4 * kp + tq)) = gf2[kp];
+        }
     }
-    float neg_lse2 = 0.f, dlt = 0.f;
-    uint32_t dq_seq[D / 8];
+    float neg_lse2 = 0.f, dlt = 0.f, neg_lse2b = 0.f, dltb = 0.f;
+    uint32_t dq_seq[D / 8], dq_seq2[kTwo ? D / 8 : 1];
     __nv_bfloat16* dq_row = p.dQ + ((size_t(b) * p.T + t) * p.H + h) * D;
+    __nv_bfloat16* dq_row2 = p.dQ + ((size_t(b) * p.T + t) * p.H + h2) * D;
     if (head) {
         neg_lse2 = -p.LSE[(size_t(b) * p.H + h) * p.T + t] * 1.4426950408889634f;
         dlt = p.delta[(size_t(b) * p.H + h) * p.T + t];
 #pragma unroll
         for (int fb = 0; fb < D / 8; ++fb) dq_seq[fb] = *reinterpret_cast<const uint32_t*>(dq_row + 8 * fb + 2 * tq);
+    }
+    if constexpr (kTwo) {
+        if (head2) {
+            neg_lse2b = -p.LSE[(size_t(b) * p.H + h2) * p.T + t] * 1.4426950408889634f;
+            dltb = p.delta[(size_t(b) * p.H + h2) * p.T + t];
+#pragma unroll
+            for (int fb = 0; fb < D / 8; ++fb) dq_seq2[fb] = *reinterpret_cast<const uint32_t*>(dq_row2 + 8 * fb + 2 * tq);
+        }
     }
 
     const int tile = t0 / kTileRows, r0 = t0 % kTileRows;
@@ -417,15 +517,22 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
             for (int kp = 0; kp < D / 32; ++kp) {
                 const uint4 kk = *reinterpret_cast<const uint4*>(sK + row_piece(slot, 4 * kp + tq));
                 const uint4 vv = *reinterpret_cast<const uint4*>(sV + row_piece(slot, 4 * kp + tq));
-                mma_bf16_16x8x16(cu[nb], qf[kp].x, 0u, qf[kp].y, 0u, kk.x, kk.y);
-                mma_bf16_16x8x16(cu[nb], qf[kp].z, 0u, qf[kp].w, 0u, kk.z, kk.w);
-                mma_bf16_16x8x16(cv[nb], gf[kp].x, 0u, gf[kp].y, 0u, vv.x, vv.y);
-                mma_bf16_16x8x16(cv[nb], gf[kp].z, 0u, gf[kp].w, 0u, vv.z, vv.w);
+                if constexpr (kTwo) {
+                    mma_bf16_16x8x16(cu[nb], qf[kp].x, qf2[kp].x, qf[kp].y, qf2[kp].y, kk.x, kk.y);
+                    mma_bf16_16x8x16(cu[nb], qf[kp].z, qf2[kp].z, qf[kp].w, qf2[kp].w, kk.z, kk.w);
+                    mma_bf16_16x8x16(cv[nb], gf[kp].x, gf2[kp].x, gf[kp].y, gf2[kp].y, vv.x, vv.y);
+                    mma_bf16_16x8x16(cv[nb], gf[kp].z, gf2[kp].z, gf[kp].w, gf2[kp].w, vv.z, vv.w);
+                } else {
+                    mma_bf16_16x8x16(cu[nb], qf[kp].x, 0u, qf[kp].y, 0u, kk.x, kk.y);
+                    mma_bf16_16x8x16(cu[nb], qf[kp].z, 0u, qf[kp].w, 0u, kk.z, kk.w);
+                    mma_bf16_16x8x16(cv[nb], gf[kp].x, 0u, gf[kp].y, 0u, vv.x, vv.y);
+                    mma_bf16_16x8x16(cv[nb], gf[kp].z, 0u, gf[kp].w, 0u, vv.z, vv.w);
+                }
             }
         }
         // ---- R and dU of head g for its slots 8 nb + 2 tq (+ 1); zero for slots past the end and heads past G,
         //      whose staged rows may hold anything ----
-        uint32_t pr[2], pu[2];
+        uint32_t pr[2], pu[2], pr2[2] = {0u, 0u}, pu2[2] = {0u, 0u};
 #pragma unroll
         for (int nb = 0; nb < 2; ++nb) {
             float r[2], u[2];
@@ -437,6 +544,16 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
             }
             pr[nb] = pack_bf16x2(r[0], r[1]);
             pu[nb] = pack_bf16x2(u[0], u[1]);
+            if constexpr (kTwo) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool ok = head2 && (8 * nb + 2 * tq + e < ns);
+                    r[e] = ok ? fast_exp2(fmaf(cu[nb][2 + e], p.scale_log2, neg_lse2b)) : 0.f;
+                    u[e] = ok ? r[e] * (cv[nb][2 + e] - dltb) : 0.f;
+                }
+                pr2[nb] = pack_bf16x2(r[0], r[1]);
+                pu2[nb] = pack_bf16x2(u[0], u[1]);
+            }
         }
         // ---- dQ share: dU (16 slots deep) x Kd rows; rows of slots past the end hold stale data: weight 0, but
         //      a NaN there would spread, so they are zeroed first ----
@@ -451,14 +568,20 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
             for (int fb = 0; fb < D / 8; fb += 2) {
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4_trans(smem_u32(sK + row_piece(krow, fb + (lane >> 4))), b0, b1, b2, b3);
-                mma_bf16_16x8x16(dq[fb], pu[0], 0u, pu[1], 0u, b0, b1);
-                mma_bf16_16x8x16(dq[fb + 1], pu[0], 0u, pu[1], 0u, b2, b3);
+                mma_bf16_16x8x16(dq[fb], pu[0], pu2[0], pu[1], pu2[1], b0, b1);
+                mma_bf16_16x8x16(dq[fb + 1], pu[0], pu2[0], pu[1], pu2[1], b2, b3);
             }
         }
         // ---- dKd = scale dU^T Q and dVd = R^T dO for the 16 slots: A = [slot][head] by 8 x 8 transposes ----
         {
             const uint32_t au0 = movmatrix_trans(pu[0]), au1 = movmatrix_trans(pu[1]);
             const uint32_t ar0 = movmatrix_trans(pr[0]), ar1 = movmatrix_trans(pr[1]);
+            // heads 8 .. 15 are the second half of the contraction (k = 8 .. 15)
+            uint32_t au2 = 0u, au3 = 0u, ar2 = 0u, ar3 = 0u;
+            if constexpr (kTwo) {
+                au2 = movmatrix_trans(pu2[0]); au3 = movmatrix_trans(pu2[1]);
+                ar2 = movmatrix_trans(pr2[0]); ar3 = movmatrix_trans(pr2[1]);
+            }
             const int hrow = lane & 7;                                  // head row a lane addresses for the matrix loads
 #pragma unroll
             for (int fb = 0; fb < D / 8; fb += 4) {
@@ -466,11 +589,16 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
                 ldmatrix_x4_trans(smem_u32(sQ + row_piece(hrow, fb + (lane >> 3))), q0, q1, q2, q3);
                 ldmatrix_x4_trans(smem_u32(sG + row_piece(hrow, fb + (lane >> 3))), g0, g1, g2, g3);
                 const uint32_t qb[4] = {q0, q1, q2, q3}, gb[4] = {g0, g1, g2, g3};
+                uint32_t qb2[4] = {0u, 0u, 0u, 0u}, gb2[4] = {0u, 0u, 0u, 0u};      // [heads 8..15][8 features]
+                if constexpr (kTwo) {
+                    ldmatrix_x4_trans(smem_u32(sQ + row_piece(hrow + 8, fb + (lane >> 3))), qb2[0], qb2[1], qb2[2], qb2[3]);
+                    ldmatrix_x4_trans(smem_u32(sG + row_piece(hrow + 8, fb + (lane >> 3))), gb2[0], gb2[1], gb2[2], gb2[3]);
+                }
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     float ck[4] = {0.f, 0.f, 0.f, 0.f}, cw[4] = {0.f, 0.f, 0.f, 0.f};
-                    mma_bf16_16x8x16(ck, au0, au1, 0u, 0u, qb[j], 0u);
-                    mma_bf16_16x8x16(cw, ar0, ar1, 0u, 0u, gb[j], 0u);
+                    mma_bf16_16x8x16(ck, au0, au1, au2, au3, qb[j], qb2[j]);
+                    mma_bf16_16x8x16(cw, ar0, ar1, ar2, ar3, gb[j], gb2[j]);
                     // rows g (slot g) and g + 8, features 8 (fb + j) + 2 tq, + 1
                     const int piece = fb + j;
                     *reinterpret_cast<uint32_t*>(oK + row_piece(g, piece) + 4 * tq) = pack_bf16x2(ck[0] * p.scale, ck[1] * p.scale);
@@ -521,6 +649,16 @@ depth_bwd_gqa_kernel(const DepthBwdParams p) {
             const float a0 = bf16_lo_to_f32(dq_seq[fb]) + p.scale * dq[fb][0];
             const float a1 = bf16_hi_to_f32(dq_seq[fb]) + p.scale * dq[fb][1];
             *reinterpret_cast<uint32_t*>(dq_row + 8 * fb + 2 * tq) = pack_bf16x2(a0, a1);
+        }
+    }
+    if constexpr (kTwo) {
+        if (head2) {
+#pragma unroll
+            for (int fb = 0; fb < D / 8; ++fb) {
+                const float a0 = bf16_lo_to_f32(dq_seq2[fb]) + p.scale * dq[fb][2];
+                const float a1 = bf16_hi_to_f32(dq_seq2[fb]) + p.scale * dq[fb][3];
+                *reinterpret_cast<uint32_t*>(dq_row2 + 8 * fb + 2 * tq) = pack_bf16x2(a0, a1);
+            }
         }
     }
 }

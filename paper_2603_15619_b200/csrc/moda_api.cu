@@ -169,7 +169,7 @@ inline bool fwd_depth_heavy(int T, int l, int d) {
 // l = 24: 1.40 -> 1.58 ms; G = 6, l = 64: 1.74 -> 1.84 ms).
 inline bool gqa_depth_split(int d, int G, int l) {
     if (d == 128) return (G == 8 || G == 16 || G == 32) && l >= 48;
-    if (G == 16 || G == 32) return l >= 31;                        // run as groups of 8 heads on the same slots
+    if (G == 16 || G == 32) return l >= 14;                        // 16 heads per launch (G = 16, l = 16: 0.73 -> 0.67 ms; l = 8: 0.51 -> 0.70)
     return G >= 6 && G <= 8 && l * (23 * G - 117) > 2000;
 }
 
@@ -290,16 +290,14 @@ inline bool dq_depth_heavy(int T, int l, int d) {
     return d == 128 && l > 0 && 3ll * l * d >= 2ll * T;
 }
 
-// Whether a grouped-query backward runs its depth part as the separate per-position kernel.
-// Measured (8 key/value heads; d = 64 at T = 16384, d = 128 at T = 8192): the row-local path with its row-term
-// workspace and group kernel costs about 8.8 us (8.5 us) per slot and head of a group, the separate kernel
-// about 0.25-0.45 ms plus 25.8 us (19.6 us) per slot whatever the group size.  Groups of 16 and 32 heads run as
-// groups of 8 whose slot gradients are added up (bf16 additions in launch order).
+// Whether a grouped-query backward runs its depth part as the separate per-position kernel (and with it the fused form
+// of the sequence part): always.  Measured (8 key/value heads; d = 64 at T = 16384, d = 128 at T = 8192; ms, row-local
+// path with the split sequence kernels -> fused sequence kernel + per-position kernel): G = 2, l = 4: 2.76 -> 1.91;
+// G = 4, l = 16: 6.10 -> 3.76; G = 8, l = 8: 11.26 -> 7.38; G = 16, l = 4: 21.8 -> 15.0; d = 128, G = 2, l = 4: 1.03 -> 1.05
+// (the only tie).  The row-local path remains what MODA_BWD_DETERMINISTIC selects.
 inline bool gqa_depth_split_bwd(int d, int G, int l) {
-    if (l <= 0 || G < 2) return false;
-    if (G == 16 || G == 32) return l >= 8;
-    if (G > 8) return false;
-    return d == 64 ? l * (88 * G - 258) > 4500 : l * (85 * G - 196) > 4000;
+    (void)d;
+    return l > 0 && G >= 2;
 }
 
 template <int D, int G>

@@ -157,8 +157,9 @@ bool set_smem_limit(Kernel k, int bytes) {
 // Which forward kernel at d = 128: one K stage and a five-unit depth ring when the depth stream
 // outweighs the sequence work (measured: - 6 % at l d / T = 0.72, - 3 % at 0.5, slower below),
 // otherwise two K stages and a three-unit ring.
-inline bool fwd_depth_heavy(int T, int l, int d) {
-    return d == 128 && l > 0 && 2ll * l * d >= T;
+inline bool fwd_depth_heavy(int T_q, int T_kv, int l, int d) {
+    // against the mean number of key tiles of a query tile, (2 T_kv - T_q) / 256: with T_q = T_kv = T this is 2 l d >= T
+    return d == 128 && l > 0 && 2ll * l * d >= 2ll * T_kv - T_q;
 }
 
 // Whether a grouped-query forward runs its depth part as the separate per-position kernel.  Measured at
@@ -254,8 +255,12 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.G = H / Hk;
     p.scale_log2 = scale * kLog2e;
     p.append_slot = static_cast<__nv_bfloat16*>(append_slot);
-    // the d = 128 kernel takes a pair of query tiles per CTA, the d = 64 kernel one tile
-    const unsigned grid = unsigned(B) * H * (kWide ? num_tiles(T) : num_tile_pairs(num_tiles(T)));
+    // The d = 128 kernel takes a pair of query tiles per CTA when the call is causal over equally many keys and queries
+    // (the pairs then have equal work) and there are at least two waves of pairs; otherwise, and at d = 64, one tile per
+    // CTA (a prefill's tiles are nearly equal already and halving the CTA count costs a wave: + 15 % measured).
+    const bool pair = !kWide && T_kv == T && (long long)B * H * num_tile_pairs(num_tiles(T)) >= 2 * 148;
+    p.pair = pair ? 1 : 0;
+    const unsigned grid = unsigned(B) * H * (pair ? num_tile_pairs(num_tiles(T)) : num_tiles(T));
     // Grouped-query calls: the sequence kernel runs without depth slots and a second kernel adds the depth
     // part of all heads of a group at once (moda_depth_gqa.cuh).
     // An e4m3 cache is always read by the row-local depth warps of the sequence kernel.
@@ -266,7 +271,7 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
         if constexpr (kWide) moda_fwd2_kernel<D, true><<<grid, kThreads, kSmem8, stream>>>(mQ, mK, mV, mO, p);
         else moda_fwd_kernel<128, 2, true><<<grid, kThreads, kSmem8, stream>>>(mQ, mK, mV, mO, p);
     } else if (kWide) moda_fwd2_kernel<D><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
-    else if (!split_depth && fwd_depth_heavy(T, l, D)) moda_fwd_kernel<128, 1><<<grid, kThreads, kSmemDeep, stream>>>(mQ, mK, mV, mO, p);
+    else if (!split_depth && fwd_depth_heavy(T, T_kv, l, D)) moda_fwd_kernel<128, 1><<<grid, kThreads, kSmemDeep, stream>>>(mQ, mK, mV, mO, p);
     else moda_fwd_kernel<D, 2><<<grid, kThreads, kSmem, stream>>>(mQ, mK, mV, mO, p);
     if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
     if (split_depth) {

@@ -101,6 +101,7 @@ struct FwdParams {
     int B, T, H, l;                  // T query positions, H query heads
     int T_kv, kv_off;                // sequence keys 0 .. T_kv - 1; query row i sits at key position i + kv_off (kv_off = T_kv - T)
     int G;                           // query heads per key/value head (1 = plain multi-head attention)
+    int pair;                        // nonzero: a CTA takes a pair of query tiles (see pair_coord), else one tile, heaviest first
     float scale_log2;                // scale * log2(e)
     // "Write" step of the depth stream fused into the forward: when not null, the base of one cache slot
     // (H / G heads) into which every CTA copies the K and V rows of its own 128 positions, straight from the
@@ -190,12 +191,13 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     const int lane = tid & 31;
 
     const int nq = num_tiles(p.T);
-    const TileCoord tc = pair_coord(blockIdx.x, nq, p.H, p.G);
+    const bool paired = p.pair != 0;
+    const TileCoord tc = paired ? pair_coord(blockIdx.x, nq, p.H, p.G) : tile_coord(blockIdx.x, nq, p.H, p.G);
     const int b = tc.b, h = tc.h, hk = tc.hk;
     const int Hk = p.H / p.G;
     // the CTA's query tiles, the longer one first; every role walks them in this order
-    const int n_tiles = (nq - 1 - tc.qt != tc.qt) ? 2 : 1;
-    auto tile_qt = [&](int t) { return t == 0 ? nq - 1 - tc.qt : tc.qt; };
+    const int n_tiles = (paired && nq - 1 - tc.qt != tc.qt) ? 2 : 1;
+    auto tile_qt = [&](int t) { return (paired && t == 0) ? nq - 1 - tc.qt : tc.qt; };
     // causal: key tiles up to the one that holds the last row's own position (row i sees keys <= i + kv_off)
     auto tile_nkv = [&](int t) {
         return min((tile_qt(t) * kTileRows + kTileRows + p.kv_off + kTileRows - 1) / kTileRows, num_tiles(p.T_kv));

@@ -93,6 +93,19 @@ def test_forward_and_backward_match_the_oracle_on_the_dequantised_slots(B, T, H,
     assert_grads_close((dQ, dK, dV, dKd, dVd), ref, f"e4m3 {(B, T, H, d, l)}")
 
 
+def test_forward_with_enough_ctas_for_tile_pairs():
+    # the d = 128 kernel takes two query tiles per CTA from two waves of pairs on
+    B, T, H, d, l = 5, 900, 16, 128, 3
+    w = synthetic.Workload("p", B, T, H, d, l)
+    x = synthetic.make(w, seed=19, device="cuda")
+    cache = build_cache8(x["Kd"], x["Vd"])
+    (_, _, Kd_hat), (_, _, Vd_hat) = oracle_cache8(x["Kd"], x["Vd"])
+    O_ref, LSE_ref = orc.forward(f64(x["Q"]), f64(x["K"]), f64(x["V"]), Kd_hat, Vd_hat, w.scale)
+    O, LSE = moda.moda_attn_fwd_e4m3(x["Q"], x["K"], x["V"], cache, l, w.scale)
+    assert moda.moda_last_status() == 0
+    assert_forward_close(O, LSE, O_ref, LSE_ref, "e4m3, tile pairs")
+
+
 def test_the_e4m3_path_reads_the_codes_not_the_original_slots():
     # Slots with a wide dynamic range inside each row: the dequantised slots differ from the originals by far more
     # than the parity tolerance, so a kernel that somehow saw bf16 values (or dropped the scales) fails here.

@@ -137,8 +137,14 @@ int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth
  * append_cache, B, T, H_kv, d, append_slot, K, V) would store: every CTA already holds the K and V
  * rows of its own 128 positions in shared memory (its diagonal key tile) and copies them out, so the
  * separate pass over K and V is gone.  `append_cache` may be the buffer `depth_kv` points to (one
- * growing cache per stack, the layer-l call reads slots < l and writes slot l); writing a slot that
- * the same call reads (append_cache == depth_kv and append_slot < l) is MODA_ERR_BAD_SLOT.
+ * growing cache per stack, the layer-l call reads slots < l and writes slot l).  Writing a slot that
+ * the same call reads (append_cache == depth_kv and append_slot < l) is allowed with one key/value head
+ * per query head (H_kv == H): every position's new K, V replace that slot's old ones after the position's
+ * own tile has been attended to with the old ones, which is what a fixed-size slot buffer needs (the
+ * bounded depth-KV slots of the paper's Discussion: the caller picks the slot to evict, e.g. the oldest
+ * for a sliding window; the order of the slots does not matter to the operator).  With grouped heads it
+ * is MODA_ERR_BAD_SLOT (the heads of a group share the blocks).  A backward pass over such a stack needs
+ * the slots as they were at each layer's forward: the caller's to keep.
  * Other arguments, validation and errors as for moda_attn_fwd_gqa.
  */
 int moda_attn_fwd_append(const void* Q, const void* K, const void* V, const void* depth_kv,

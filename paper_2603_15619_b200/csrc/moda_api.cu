@@ -742,8 +742,11 @@ int moda_attn_fwd_append(const void* Q, const void* K, const void* V, const void
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) || !aligned16(append_cache) ||
         (l > 0 && !aligned16(depth_kv)))
         return MODA_ERR_MISALIGNED;
-    // the slot being written must not be one of the slots being read
-    if (l > 0 && append_cache == depth_kv && append_slot < l) return MODA_ERR_BAD_SLOT;
+    // The slot being written may be one of the slots being read only with one key/value head per query head: a CTA then
+    // reads and writes the blocks of its own (b, h, tile) alone, and it writes after its depth warps have finished reading
+    // (a fixed-size slot buffer whose oldest or least useful slot is replaced in place).  With grouped heads the other
+    // heads of the group read the block that the first head writes.
+    if (l > 0 && append_cache == depth_kv && append_slot < l && H_kv != H) return MODA_ERR_BAD_SLOT;
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     void* slot = static_cast<__nv_bfloat16*>(append_cache) + size_t(append_slot) * cache_slot_elems(B, T, H_kv, d);

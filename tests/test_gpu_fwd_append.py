@@ -1,6 +1,7 @@
 """The depth stream's write step fused into the forward (moda_attn_fwd_append), on the GPU through the C ABI:
 the slot it writes is bit for bit what moda_depth_cache_append writes, O and LSE are bit for bit those of the plain
 forward, and the slot that the next layer reads is really the one that was written."""
+import numpy as np
 import pytest
 import torch
 
@@ -43,10 +44,34 @@ def test_fused_write_step_is_the_separate_append_bit_for_bit(B, T, H, Hk, d, l):
     assert_forward_close(O1, LSE1, *orc.forward_gqa(*xs, scale), "forward with the fused write step")
 
 
-def test_writing_a_slot_that_the_call_reads_is_rejected():
-    B, T, H, d, l = 1, 128, 1, 64, 2
-    x = synthetic.make_gqa(B, T, H, H, d, l, seed=1, device="cuda")
+@pytest.mark.parametrize("d,T,H", [(128, 300, 2), (64, 520, 3), (128, 1300, 16)])
+def test_fixed_size_slot_buffer_with_in_place_eviction_is_a_sliding_window(d, T, H):
+    # A buffer of S slots: layer i attends to the slots that are filled and then writes its own K, V over the oldest
+    # one, in the same launch.  Against the oracle run on the last S layers' K, V (any order: pin P5).
+    B, S, layers = (4 if T == 1300 else 1), 3, 6
+    scale = d ** -0.5
+    g = torch.Generator(device="cuda").manual_seed(77)
+    mk = lambda: (torch.randn((B, T, H, d), device="cuda", generator=g) * 0.7).to(torch.bfloat16)
+    buf = moda.alloc_depth_cache(B, T, H, d, S)
+    buf.fill_(0.0)
+    history = []
+    for i in range(layers):
+        Q, K, V = mk(), mk(), mk()
+        l = min(i, S)
+        O, LSE = moda.moda_attn_fwd_append(Q, K, V, buf, l, scale, buf, i % S)
+        assert moda.moda_last_status() == 0
+        window = history[-S:]
+        Kd = np.stack([f64(k) for k, _ in window]) if window else np.zeros((0, B, T, H, d))
+        Vd = np.stack([f64(v) for _, v in window]) if window else np.zeros((0, B, T, H, d))
+        O_ref, LSE_ref = orc.forward(f64(Q), f64(K), f64(V), Kd, Vd, scale)
+        assert_forward_close(O, LSE, O_ref, LSE_ref, f"layer {i} of a {S}-slot buffer")
+        history.append((K, V))
+
+
+def test_in_place_eviction_is_rejected_for_grouped_heads():
+    B, T, H, Hk, d, l = 1, 128, 4, 2, 64, 2
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=3, device="cuda")
     cache = build_cache(x["Kd"], x["Vd"])
-    with pytest.raises(binding.ModaError) as e:
-        moda.moda_attn_fwd_append(x["Q"], x["K"], x["V"], cache, l, 0.125, cache, 1)
+    with pytest.raises(moda.ModaError) as e:
+        moda.moda_attn_fwd_append(x["Q"], x["K"], x["V"], cache, l, d ** -0.5, cache, 0)
     assert e.value.code == -6

@@ -231,15 +231,17 @@ int moda_attn_bwd_stages(const void* Q, const void* K, const void* V, const void
  *     Q, O, dO, dQ : bf16 [B][T][H][d]          K, V, dK, dV : bf16 [B][T][H_kv][d]
  *     depth_kv, d_depth_kv : cache layout with H_kv heads (moda_depth_cache_bytes(B, T, H_kv, d, l))
  *     LSE : fp32 [B][H][T]                      workspace : moda_bwd_workspace_bytes_gqa(B, T, H, H_kv, d, l)
- * dK, dV and the depth gradients are the sums over the G query heads of a group, taken in a fixed
- * order (no floating-point atomics), so results are bit-reproducible.  With G > 1 the workspace
- * also holds two fp32 factors per (row, slot, query head), from which a second kernel forms the
- * depth gradients (fp32 sums) without reading the depth cache again.  For large groups with many
- * slots the library instead runs the depth part of the forward and of the backward as separate
- * kernels that treat the heads of a group as the rows of one small tensor-core product per
- * position (probabilities and their gradients rounded to bf16 for that product, fp32 accumulation,
- * as in the sequence part); with 16 or 32 heads per group the groups of 8 heads add their depth
- * gradients one after the other in bf16.  The choice depends only on (d, G, l).  H_kv must divide H
+ * dK, dV and the depth gradients are the sums over the G query heads of a group, taken on chip in a
+ * fixed order (bit-reproducible; dQ goes through the fp32 accumulator of the fused form, see
+ * moda_attn_bwd).  With G > 1 the backward runs its depth part as a separate kernel that treats
+ * the heads of a group as the rows of one small tensor-core product per position (probabilities
+ * and their gradients rounded to bf16 for that product, fp32 accumulation, as in the sequence
+ * part), and for large groups with many slots the forward does the same; up to 16 heads of a group
+ * fill one product, 32 heads run as two groups of 16 whose depth
+ * gradients are added one after the other in bf16.  The choice depends only on (d, G, l).  With
+ * MODA_BWD_DETERMINISTIC (moda_attn_bwd_gqa_stages) the depth part stays row-local: the workspace then
+ * holds two fp32 factors per (row, slot, query head), from which a second kernel forms the depth
+ * gradients (fp32 sums over the heads in a fixed order) without reading the depth cache again.  H_kv must divide H
  * and G = H / H_kv must be 1 to 8, 16 or 32 (MODA_ERR_BAD_GROUP otherwise); H_kv == H is exactly
  * moda_attn_fwd / moda_attn_bwd.  Everything else (validation, streams, ownership, errors) is
  * as for those calls.

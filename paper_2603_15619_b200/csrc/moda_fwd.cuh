@@ -1,15 +1,20 @@
 // MoDA forward kernel for sm_100a (Sec. 2.2 definition; Alg. 1 gives the blockwise
 // online-softmax schedule this kernel re-designs for tcgen05 / TMEM / TMA).
 //
-// One CTA owns one (b, query head h, 128-query-row tile); with grouped-query attention the G heads
-// that share a key/value head are adjacent CTAs (tile_coord).  384 threads, three warpgroups:
+// One CTA owns one (b, query head h) and either one 128-query-row tile or, for causal calls over as many
+// keys as queries, a pair of them (pair_coord: the p-th tile from the end, then the p-th from the start, so that
+// every CTA has the same number of key tiles and the short tile's depth slots are worked on during the long
+// tile's key loop); with grouped-query attention the G heads that share a key/value head are adjacent CTAs
+// (tile_coord).  The rings and their phase counters run on across the two tiles.  384 threads, three warpgroups:
 //
 //   warps 0-3  softmax   one thread per query row.  Reads the score tile S_j from TMEM,
 //                        keeps the running (m, l) of the online softmax in registers, writes
 //                        P_j = exp2(S_j c - m) as packed bf16 back into the TMEM columns of
 //                        S_j, rescales the O accumulator only when the running maximum grew
-//                        by more than 2^8, and runs the epilogue.
-//   warps 4-7  depth     one thread per query row.  Reads the row's l depth keys/values from
+//                        by more than 2^8, and runs the epilogue (output tile, LSE, and the write of the
+//                        layer's own K, V rows into a cache slot when the call asks for it).
+//   warps 4-7  depth     one thread per query row (its q comes straight from global memory).  Reads the
+//                        row's l depth keys/values (bf16, or e4m3 codes with row scales) from
 //                        a shared-memory ring that warp 10 fills with 16 KiB bulk copies of
 //                        the depth cache, builds an independent partial softmax state
 //                        (m_d, l_d, o_d) on the CUDA cores (slots in groups of 32, online

@@ -14,7 +14,8 @@
 //                             depth cache exactly once; bound by HBM.
 //   2. moda_bwd_fused_kernel  one CTA per 128-key tile, looping over the 128-query tiles at or below the
 //                             diagonal.  Per pair of tiles: S^T = K Q^T and dP^T = V dO^T (tcgen05, operands
-//                             in shared memory), P^T and dS^T formed once by the row warps, dV += P^T dO (P^T
+//                             in shared memory; one extra k-step each adds the per-query terms -LSE / scale and
+//                             -D_t to every score of the query's column), P^T and dS^T formed once by the row warps, dV += P^T dO (P^T
 //                             from tensor memory), dK += dS^T Q and dQ_tile = dS K (dS^T staged once in shared
 //                             memory and used by both: K-major for dK, MN-major for dQ).  dK, dV accumulate in
 //                             tensor memory over the whole loop; the dQ tile is added to the fp32 accumulator
@@ -288,9 +289,11 @@ bwd_dq_finish_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict
 //   row warps    two warpgroups: a thread owns one key row (= tensor-memory lane) and 64 of the 128 query columns of
 //                an iteration: P^T, then dS^T.
 //   drain warps  one warpgroup: a thread owns one query row of the dQ tile; it copies the row out of tensor memory
-//                (which frees the region at once) and adds it to the fp32 accumulator with 16-byte reductions
-//                at whatever pace L2 takes them, without holding up the row warps.
-//   then         a loader warp (TMA tiles, per-query LSE and D_t) and the warps that issue the contractions:
+//                (which frees the region at once) and hands it, 8 KiB at a time through a staging ring in shared
+//                memory, to bulk reductions into the fp32 accumulator, at whatever pace L2 takes them, without
+//                holding up the row warps.
+//   then         a loader warp (TMA tiles; the per-query terms as bf16 parts for the extra k-step) and the warps
+//                that issue the contractions:
 //                S, dP, and dV then dQ then dK.  One tcgen05.mma costs its
 //                issuing thread about as long as it executes, so the contractions that start an iteration's two
 //                chains have their own warps on different schedulers; MMAs of different warps are ordered by
@@ -300,15 +303,16 @@ bwd_dq_finish_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict
 // two at d = 64 (where dK and dV leave room);  Y, 128 columns, dP^T and then the dQ tile of the same iteration;
 // dK, D columns;  dV, D columns.  512 columns at either head width.
 //
-// What bounds it (cycle stamps per warp role, T = 8192): at d = 128 the shared-memory port -- per iteration the
-// MMAs read 320 KiB of operands, TMA writes 64 KiB of Q / dO, dS^T is 32 KiB, the dQ staging 64 KiB in and 64 KiB
-// out, against 128 bytes per clock -- and the L2 reduction rate (64 KiB of fp32 additions per iteration per SM; all
-// SMs together sustain about 5.9 TB/s of them); at d = 64 the row warps (the same number of exponentials and
-// conversions per iteration for half the tensor work).
+// What bounds it (cycle stamps per warp role, T = 8192): the rate at which a dQ tile's additions are taken by L2 (64 KiB
+// of fp32 per iteration per SM at d = 128; all SMs together sustain about 5.9 TB/s in a kernel that does nothing else,
+// 4.3 TB/s here beside as many bytes of Q / dO loads): the drain warps need ~4300 cycles per tile, the five contractions
+// 2700 tensor cycles.  The shared-memory port (MMA operands 304 KiB per iteration, TMA writes 64 KiB, dS^T 32 KiB, the
+// dQ staging 64 KiB in and out, against 128 bytes per clock) is at two thirds of its peak since the row warps no
+// longer load the per-query terms.
 //
 // Two dependency chains per iteration i, which overlap each other and the next iteration:
-//   X:  S_i -> P_i^T = exp2(S c - LSE c) (row warps) -> dV_i -> X free -> S_{i+1}
-//   Y:  dP_i -> dS_i^T = P o (dP - D) to shared memory (row warps) -> dQ_i -> copied out (drain warps) -> Y free -> dP_{i+1}
+//   X:  S'_i = S_i - LSE / scale -> P_i^T = exp2(S' c) (row warps) -> dV_i -> X free -> S_{i+1}
+//   Y:  dP'_i = dP_i - D -> dS_i^T = P o dP' to shared memory (row warps) -> dQ_i -> copied out (drain warps) -> Y free -> dP_{i+1}
 // and dK_i, issued behind dQ_i, fills the tensor pipe while the row warps exponentiate tile i+1.
 
 template <int D>

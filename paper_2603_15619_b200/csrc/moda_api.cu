@@ -343,10 +343,10 @@ int launch_depth_bwd(DepthBwdParams m, cudaStream_t stream) {
     }
 }
 
-// Which form of the backward a call takes.  The fused form (moda_bwd_fused.cuh) covers plain multi-head
-// calls and those grouped-query calls whose depth part is either absent or done by the per-position kernel;
-// grouped-query calls on the row-local depth path keep the split form, whose dQ pass leaves the per-row
-// factors that depth_grad_group_kernel sums over the heads of a group.
+// Which form of the backward a call takes: the fused form (moda_bwd_fused.cuh) unless the caller asks for
+// reproducible bits.  Grouped-query calls in the fused form run their depth part as the per-position kernel; in
+// the split form they stay row-local: its dQ pass leaves the per-row factors that depth_grad_group_kernel sums
+// over the heads of a group.
 inline bool bwd_uses_fused(int d, int G, int l, bool deterministic) {
     if (deterministic) return false;
     return G == 1 || l == 0 || gqa_depth_split_bwd(d, G, l);

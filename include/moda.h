@@ -63,6 +63,7 @@ extern "C" {
 #define MODA_ERR_DEVICE_TIMEOUT (-10) /* an earlier kernel gave up a bounded wait (see moda_last_status) */
 #define MODA_ERR_SCRATCH_LIMIT (-11)  /* problem needs more built-in scratch than moda_attn_bwd_static_scratch holds */
 #define MODA_ERR_BAD_GROUP (-12)      /* H_kv does not divide H, or an unsupported number of query heads per group */
+#define MODA_ERR_BAD_SCALE (-13)      /* the softmax scale is not finite or below 1e-20 (zero and negative scales are not served) */
 #define MODA_MAX_GROUP 32             /* supported group sizes G = H / H_kv: 1 to 8, 16 and 32 */
 
 /* Library version: major * 10000 + minor * 100 + patch. */
@@ -124,6 +125,7 @@ int moda_depth_cache_unpack(const void* cache, int B, int T, int H, int d, int s
  * softmax).  depth_kv holds at least l slots in the cache layout (may be null when
  * l == 0).  Writes O (bf16 [B][T][H][d]) and LSE (fp32 [B][H][T], natural log, taken over
  * the union of sequence and depth keys).  bf16 inputs, fp32 accumulation and softmax.
+ * `scale` (every attention call): finite and >= 1e-20; otherwise MODA_ERR_BAD_SCALE.
  */
 int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth_kv,
                   int B, int T, int H, int d, int l, float scale,

@@ -89,6 +89,13 @@ int check_shape(int B, int T, int H, int d) {
 }
 
 // Query heads H on H_kv key/value heads: H_kv must divide H; 1 to 8, 16 or 32 heads per group.
+// The softmax scale: finite and at least 1e-20.  Zero (a uniform softmax) and negative scales are not served: the
+// kernels take row maxima of the raw scores and scale afterwards, masked scores are -inf times the scale, and the
+// fused backward divides LSE by it.
+int check_scale(float scale) {
+    return (std::isfinite(scale) && scale >= 1e-20f) ? MODA_OK : MODA_ERR_BAD_SCALE;
+}
+
 int check_groups(int H, int H_kv) {
     if (H_kv < 1 || H % H_kv != 0) return MODA_ERR_BAD_GROUP;
     const int G = H / H_kv;
@@ -591,6 +598,7 @@ int decode_common(const void* q, const void* K, const void* V, const int* seq_le
     const bool paged = block_table != nullptr;
     if (B < 1 || T_kv < 1 || H < 1 || (!paged && T_cap < T_kv)) return MODA_ERR_BAD_SHAPE;
     if (d != 64 && d != 128) return MODA_ERR_BAD_HEAD_DIM;
+    if (int rc = check_scale(scale)) return rc;
     if ((long long)(paged ? page_size : B) * T_cap > 0x7fffffffLL / H) return MODA_ERR_BAD_SHAPE;
     if (int rc = check_groups(H, H_kv)) return rc;
     if ((long long)B * H * kDecodeMaxSplits > 0x7fffffffLL || B > 65535) return MODA_ERR_BAD_SHAPE;
@@ -644,6 +652,7 @@ const char* moda_strerror(int code) {
         case MODA_ERR_CUDA: return "a CUDA call failed (see moda_last_cuda_error)";
         case MODA_ERR_DEVICE_TIMEOUT: return "a kernel gave up a bounded wait (see moda_last_status)";
         case MODA_ERR_BAD_GROUP: return "H_kv must divide H with 1 to 8, 16 or 32 query heads per key/value head";
+        case MODA_ERR_BAD_SCALE: return "the softmax scale must be finite and at least 1e-20";
         case MODA_ERR_SCRATCH_LIMIT: return "B*H*T exceeds the built-in scratch of moda_attn_bwd_static_scratch (2^20 rows)";
         default: return "unknown error code";
     }
@@ -717,6 +726,7 @@ int moda_attn_fwd_prefill(const void* Q, const void* K, const void* V, const voi
                           int B, int T_q, int T_kv, int H, int H_kv, int d, int l, float scale,
                           void* O, float* LSE, void* stream) {
     if (int rc = check_shape(B, T_q, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
     if (T_kv < T_q) return MODA_ERR_BAD_SHAPE;
     if (int rc = check_shape(B, T_kv, H, d)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
@@ -735,6 +745,7 @@ int moda_attn_fwd_append(const void* Q, const void* K, const void* V, const void
                          int B, int T, int H, int H_kv, int d, int l, float scale,
                          void* O, float* LSE, void* append_cache, int append_slot, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (append_slot < 0 || append_slot >= MODA_MAX_DEPTH) return MODA_ERR_BAD_SLOT;
@@ -799,6 +810,7 @@ int moda_attn_bwd_gqa_stages(const void* Q, const void* K, const void* V, const 
                              void* dQ, void* dK, void* dV, void* d_depth_kv,
                              void* workspace, size_t workspace_bytes, int stages, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
     if ((stages & MODA_BWD_ALL_STAGES) == 0 || stages < 0 ||
         stages > (MODA_BWD_ALL_STAGES | MODA_BWD_ACCUMULATE_DEPTH | MODA_BWD_DETERMINISTIC))
@@ -852,6 +864,7 @@ int moda_attn_fwd_e4m3(const void* Q, const void* K, const void* V, const void* 
                        int B, int T, int H, int H_kv, int d, int l, float scale,
                        void* O, float* LSE, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!Q || !K || !V || !O || !LSE || (l > 0 && !depth_kv_e4m3)) return MODA_ERR_NULL_POINTER;
@@ -870,6 +883,7 @@ int moda_attn_bwd_e4m3(const void* Q, const void* K, const void* V, const void* 
                        void* dQ, void* dK, void* dV, void* d_depth_kv,
                        void* workspace, size_t workspace_bytes, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv_e4m3 || !d_depth_kv)))
         return MODA_ERR_NULL_POINTER;
@@ -917,6 +931,7 @@ int moda_attn_fwd_gqa_pm(const void* Q, const void* K, const void* V, const void
                          int B, int T, int H, int H_kv, int d, int l, float scale,
                          void* O, float* LSE, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
     if (H == H_kv) return MODA_ERR_BAD_GROUP;                 // the per-position kernels need at least two heads per group
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
@@ -936,6 +951,7 @@ int moda_attn_bwd_gqa_pm(const void* Q, const void* K, const void* V, const void
                          void* dQ, void* dK, void* dV, void* d_depth_kv_pm,
                          void* workspace, size_t workspace_bytes, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
     if (int rc = check_groups(H, H_kv)) return rc;
     if (H == H_kv) return MODA_ERR_BAD_GROUP;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
@@ -1026,6 +1042,7 @@ extern "C" int moda_attn_bwd_static_scratch(const void* Q, const void* K, const 
                                             int B, int T, int H, int d, int l, float scale,
                                             void* dQ, void* dK, void* dV, void* d_depth_kv, void* stream) {
     if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
     if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
     if ((long long)B * H * T > (long long)MODA_STATIC_SCRATCH_ROWS) return MODA_ERR_SCRATCH_LIMIT;
     if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV || (l > 0 && (!depth_kv || !d_depth_kv)))

@@ -28,7 +28,7 @@ def test_library_loads_and_exports_every_declared_symbol():
 
 
 def test_strerror_covers_all_codes():
-    for code in range(0, -13, -1):
+    for code in range(0, -14, -1):
         assert binding.strerror(code) != "unknown error code"
     assert binding.strerror(-99) == "unknown error code"
 
@@ -159,3 +159,20 @@ def test_e4m3_cache_entry_points_validate_before_touching_the_device():
     assert lib.moda_attn_bwd_e4m3(*args, None, p, ctypes.c_size_t(1 << 20), None) == -1      # depth slots without a gradient cache
     assert lib.moda_attn_bwd_e4m3(*args, p, p, ctypes.c_size_t(4096), None) == -7
     assert lib.moda_attn_bwd_e4m3(*args, p, None, ctypes.c_size_t(1 << 20), None) == -7
+
+
+def test_softmax_scale_must_be_usable():
+    lib = binding.load()
+    p = ctypes.c_void_p(4096)
+    for bad in (0.0, 1e-30, -0.09, float("inf"), float("nan")):
+        sc = ctypes.c_float(bad)
+        assert lib.moda_attn_fwd(p, p, p, None, 1, 128, 1, 64, 0, sc, p, p, None) == -13
+        assert lib.moda_attn_fwd_append(p, p, p, None, 1, 128, 1, 1, 64, 0, sc, p, p, p, 0, None) == -13
+        args = [p] * 7 + [1, 128, 1, 64, 0, sc] + [p, p, p, None]
+        assert lib.moda_attn_bwd(*args, p, ctypes.c_size_t(1 << 20), None) == -13
+        assert lib.moda_attn_bwd_static_scratch(*args, None) == -13
+        assert lib.moda_attn_decode(p, p, p, None, 1, 128, 128, 2, 1, 64, 0, sc, p, p, p, ctypes.c_size_t(1 << 20), None) == -13
+    for ok in (1e-6, 0.09, 3.0):
+        # a usable scale passes this check and fails on the next one (no workspace)
+        args = [p] * 7 + [1, 128, 1, 64, 0, ctypes.c_float(ok)] + [p, p, p, None]
+        assert lib.moda_attn_bwd(*args, None, ctypes.c_size_t(0), None) == -7

@@ -165,3 +165,17 @@ def test_side_stream_call_with_allocations_interleaved_on_the_default_stream():
         torch.cuda.synchronize()
         dKd, dVd = unpack_cache(dcache, w.l, w.B, w.T, w.H, w.d)
         assert_grads_close((dQ, dK, dV, dKd, dVd), ref, f"side stream, repeat {rep}")
+
+
+@pytest.mark.parametrize("scale", [1e-6, 0.3])
+def test_small_and_large_scales(scale):
+    # a tiny scale makes every visible key nearly equally likely, a large one concentrates on the few largest scores; the fused
+    # backward carries LSE / scale inside its score contractions
+    w = synthetic.Workload("sc", 1, 300, 2, 128, 3)
+    x = synthetic.make(w, seed=44, device="cuda")
+    cache = build_cache(x["Kd"], x["Vd"])
+    O, LSE = moda.moda_attn_fwd(x["Q"], x["K"], x["V"], cache, w.l, scale)
+    dQ, dK, dV, dcache = moda.moda_attn_bwd(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, w.l, scale)
+    assert moda.moda_last_status() == 0
+    dKd, dVd = unpack_cache(dcache, w.l, w.B, w.T, w.H, w.d)
+    assert_grads_close((dQ, dK, dV, dKd, dVd), oracle_backward(x, scale), f"scale {scale}")

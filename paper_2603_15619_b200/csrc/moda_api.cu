@@ -263,9 +263,14 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.scale_log2 = scale * kLog2e;
     p.append_slot = static_cast<__nv_bfloat16*>(append_slot);
     // The d = 128 kernel takes a pair of query tiles per CTA when the call is causal over equally many keys and queries
-    // (the pairs then have equal work) and there are at least two waves of pairs; otherwise, and at d = 64, one tile per
-    // CTA (a prefill's tiles are nearly equal already and halving the CTA count costs a wave: + 15 % measured).
-    const bool pair = !kWide && T_kv == T && (long long)B * H * num_tile_pairs(num_tiles(T)) >= 2 * 148;
+    // (the pairs then have equal work) and the equal-sized CTAs fill their last wave (at least 93 % of the SM slots of
+    // all waves; 512 pairs on 148 SMs would idle a seventh of them, measured + 4 % at c3 with B = 1), or when the depth
+    // stream outweighs the sequence work anyway (c2: - 5 %).  Otherwise, and at d = 64, one tile per CTA, heaviest first (a
+    // prefill's tiles are nearly equal already and halving the CTA count costs a wave: + 15 % measured).
+    const long long n_pairs = (long long)B * H * num_tile_pairs(num_tiles(T));
+    const long long pair_waves = (n_pairs + 147) / 148;
+    const bool pair = !kWide && T_kv == T && n_pairs >= 2 * 148 &&
+                      (100 * n_pairs >= 93 * 148 * pair_waves || fwd_depth_heavy(T, T_kv, l, D));
     p.pair = pair ? 1 : 0;
     const unsigned grid = unsigned(B) * H * (pair ? num_tile_pairs(num_tiles(T)) : num_tiles(T));
     // Grouped-query calls: the sequence kernel runs without depth slots and a second kernel adds the depth

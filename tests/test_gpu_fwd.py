@@ -45,8 +45,9 @@ SMALL = [
     (1, 1024, 1, 128, 0), (1, 1000, 1, 64, 2),
     # more than 32 depth slots: several groups of the online softmax over the depth keys
     (1, 200, 2, 64, 33), (1, 257, 1, 128, 64), (1, 130, 1, 64, 100), (1, 128, 1, 128, 256), (2, 300, 2, 64, 65),
-    # at least two waves of tile pairs: the d = 128 kernel then takes two query tiles per CTA
-    (4, 1300, 16, 128, 3), (5, 1000, 16, 128, 0), (3, 2100, 12, 128, 40),
+    # tile pairs in the d = 128 kernel: 432 pairs (three waves of 148 SMs filled to 97 %), with and without depth slots, and
+    # a depth-heavy shape with an odd number of tiles
+    (3, 2190, 16, 128, 3), (3, 2304, 16, 128, 0), (3, 2100, 12, 128, 40),
 ]
 
 

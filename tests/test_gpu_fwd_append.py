@@ -18,9 +18,10 @@ SHAPES = [
     (1, 128, 1, 1, 128, 0), (2, 300, 2, 2, 128, 3), (1, 1000, 3, 3, 64, 2), (1, 257, 4, 2, 64, 5), (2, 129, 8, 2, 128, 1),
     (1, 640, 2, 2, 128, 12),      # 2 l d >= T: the deep-ring variant of the d = 128 kernel
     (1, 1, 2, 1, 64, 0), (1, 520, 16, 2, 64, 33), (1, 130, 8, 1, 128, 50),   # grouped-query calls whose depth part is a second kernel
-    # enough CTAs for the d = 128 kernel to take pairs of query tiles: an odd number of tiles (the middle one alone), a
-    # ragged last tile, grouped heads; and the deep-ring variant with pairs
-    (4, 1300, 16, 4, 128, 5), (13, 600, 8, 8, 128, 12),
+    # enough CTAs for the d = 128 kernel to take pairs of query tiles (432 pairs fill three waves of 148 SMs to 97 %): a
+    # ragged last tile, grouped heads; and a depth-heavy shape (pairs whatever the wave count, an odd number of tiles:
+    # the middle one alone) on the deep-ring variant
+    (3, 2190, 16, 4, 128, 5), (13, 600, 8, 8, 128, 12),
 ]
 
 

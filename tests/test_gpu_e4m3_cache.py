@@ -147,3 +147,33 @@ def test_depth_zero_ignores_the_cache_pointer():
     O, LSE = moda.moda_attn_fwd_e4m3(x["Q"], x["K"], x["V"], None, 0, w.scale)
     O2, LSE2 = moda.moda_attn_fwd(x["Q"], x["K"], x["V"], None, 0, w.scale)
     assert torch.equal(O, O2) and torch.equal(LSE, LSE2)
+
+
+def test_c3_full_size_one_head_slice():
+    # The benchmark's T = 8192 shape (c3 with 16 slots) at full size through the e4m3 entry points; heads are independent, so
+    # one complete (b, h) slice is checked against the oracle run on that slice alone, with the oracle's own quantiser.
+    from parity import unpack_cache
+    w = synthetic.WORKLOADS["c3"].with_l(16)
+    B, T, H, d, l = w.B, w.T, w.H, w.d, w.l
+    x = {n: synthetic.tensor(w, n, 0, 0, "cuda") for n in ("Q", "K", "V", "dO")}
+    cache = moda.alloc_depth_cache_e4m3(B, T, H, d, l)
+    b, h = B - 1, H // 2
+    Kd_h, Vd_h = [], []
+    for i in range(l):
+        kd, vd = synthetic.tensor(w, "Kd", 0, i, "cuda"), synthetic.tensor(w, "Vd", 0, i, "cuda")
+        moda.moda_depth_cache_append_e4m3(cache, i, kd, vd)
+        Kd_h.append(f64(kd[b:b + 1, :, h:h + 1]))
+        Vd_h.append(f64(vd[b:b + 1, :, h:h + 1]))
+        del kd, vd
+    O, LSE = moda.moda_attn_fwd_e4m3(x["Q"], x["K"], x["V"], cache, l, w.scale)
+    dQ, dK, dV, dcache = moda.moda_attn_bwd_e4m3(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, w.scale)
+    assert moda.moda_last_status() == 0
+    (_, _, Kd_hat), (_, _, Vd_hat) = [(None, None, orc.dequantize_e4m3_rows(*orc.quantize_e4m3_rows(np.stack(a)))) for a in (Kd_h, Vd_h)]
+    sl = lambda t: f64(t[b:b + 1, :, h:h + 1])
+    O_ref, LSE_ref = orc.forward(sl(x["Q"]), sl(x["K"]), sl(x["V"]), Kd_hat, Vd_hat, w.scale)
+    assert_forward_close(O[b:b + 1, :, h:h + 1], LSE[b:b + 1, h:h + 1], O_ref, LSE_ref, "c3 l = 16, e4m3 cache")
+    ref = orc.backward(sl(x["Q"]), sl(x["K"]), sl(x["V"]), Kd_hat, Vd_hat, sl(x["dO"]), w.scale)
+    dKd, dVd = unpack_cache(dcache, l, B, T, H, d)
+    got = (dQ[b:b + 1, :, h:h + 1], dK[b:b + 1, :, h:h + 1], dV[b:b + 1, :, h:h + 1],
+           dKd[:, b:b + 1, :, h:h + 1], dVd[:, b:b + 1, :, h:h + 1])
+    assert_grads_close(got, ref, "c3 l = 16, e4m3 cache")

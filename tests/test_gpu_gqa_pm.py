@@ -102,3 +102,27 @@ def test_entry_points_reject_one_head_per_group():
     with pytest.raises(moda.ModaError) as e:
         moda.moda_attn_fwd_gqa_pm(x["Q"], x["K"], x["V"], cache, 1, w.scale)
     assert e.value.code == -12
+
+
+def test_paper_table2_shape_one_group_against_the_oracle():
+    # The shape family of the paper's kernel table (B = 1, d = 64, 8 key/value heads, G = 8) at T = 8192 with 32 slots, on
+    # the GPU in full with the position-major cache; the oracle checks one whole group (8 query heads on one key/value
+    # head), which is a problem of its own.
+    B, T, H, Hk, d, l, hk = 1, 8192, 64, 8, 64, 32, 5
+    G = H // Hk
+    scale = d ** -0.5
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=2, device="cuda", k_head_norm=True)
+    cache = build_cache_pm(x["Kd"], x["Vd"])
+    O, LSE = moda.moda_attn_fwd_gqa_pm(x["Q"], x["K"], x["V"], cache, l, scale)
+    dQ, dK, dV, dcache = moda.moda_attn_bwd_gqa_pm(x["Q"], x["K"], x["V"], cache, O, x["dO"], LSE, l, scale)
+    assert moda.moda_last_status() == 0
+    dKd, dVd = unpack_cache_pm(dcache, l, B, T, Hk, d)
+    qs = slice(hk * G, (hk + 1) * G)
+    xs = [f64(x["Q"][:, :, qs]), f64(x["K"][:, :, hk:hk + 1]), f64(x["V"][:, :, hk:hk + 1]),
+          f64(x["Kd"][:, :, :, hk:hk + 1]), f64(x["Vd"][:, :, :, hk:hk + 1])]
+    O_ref, LSE_ref = orc.forward_gqa(*xs, scale)
+    assert_forward_close(O[:, :, qs], LSE[:, qs], O_ref, LSE_ref, "Table 2 shape, position-major cache")
+    ref = orc.backward_gqa(*xs, f64(x["dO"][:, :, qs]), scale)
+    got = (dQ[:, :, qs], dK[:, :, hk:hk + 1], dV[:, :, hk:hk + 1], dKd[:, :, :, hk:hk + 1], dVd[:, :, :, hk:hk + 1])
+    for name, g, r in zip(("dQ", "dK", "dV", "dKd", "dVd"), got, ref):
+        assert grad_err(g, r) <= TOL_GRAD_REL_L2, f"{name}: {grad_err(g, r):.3e}"

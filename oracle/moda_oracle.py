@@ -369,3 +369,23 @@ def quantize_e4m3_rows(X):
 def dequantize_e4m3_rows(codes, scale):
     """float64 values code * scale of what quantize_e4m3_rows stored."""
     return e4m3_decode_table()[np.asarray(codes, dtype=np.uint8)] * np.asarray(scale, dtype=np.float64)[..., None]
+
+
+# ---------------------------------------------------------------------------------------
+# "Write" step with its projection (Sec. 2.1, Q / K / V = X W; Sec. 2.2, the write step: a layer's key-value pair is
+# appended to the depth stream, an FFN layer obtains its pair through a KV projection of its input).
+# The definition written out with the library's float64 matrix product.  Weights are passed as the transposes of
+# the paper's W_K, W_V, i.e. one row per output feature: Wk, Wv [H_k d, D].
+# ---------------------------------------------------------------------------------------
+def project_kv(X, Wk, Wv, H_k):
+    """K, V [B, T, H_k, d] = X [B, T, D] times the key / value projections (float64)."""
+    X = np.asarray(X, dtype=np.float64)
+    Wk = np.asarray(Wk, dtype=np.float64)
+    Wv = np.asarray(Wv, dtype=np.float64)
+    B, T, D = X.shape
+    n = Wk.shape[0]
+    if Wk.shape != (n, D) or Wv.shape != (n, D) or n % H_k:
+        raise ValueError("Wk, Wv must be [H_k d, D] matching X [B, T, D]")
+    K = np.matmul(X, Wk.T).reshape(B, T, H_k, n // H_k)
+    V = np.matmul(X, Wv.T).reshape(B, T, H_k, n // H_k)
+    return K, V

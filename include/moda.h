@@ -434,6 +434,27 @@ int moda_attn_bwd_gqa_pm(const void* Q, const void* K, const void* V, const void
                          void* dQ, void* dK, void* dV, void* d_depth_kv_pm,
                          void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Key / value projection with the depth stream's write step in its epilogue (Sec. 2.1: K = X W_K, V = X W_V;
+ * Sec. 2.2, "write": a layer's key-value pair is appended to the depth stream; an FFN layer obtains its pair
+ * through a KV projection of its input).
+ *
+ *     K[b, t, h, :] = X[b, t, :] . Wk[h d + j, :]   (j = 0 .. d-1),   V likewise with Wv
+ *
+ *     X        : bf16 [B][T][D_model], D_model a multiple of 64 (MODA_ERR_BAD_SHAPE otherwise)
+ *     Wk, Wv   : bf16 [H_kv * d][D_model]: one row per output feature, i.e. the transposes of the paper's W_K, W_V
+ *     K_out, V_out : bf16 [B][T][H_kv][d], both or neither (an FFN-side projection needs only the slot)
+ *     cache, slot  : depth cache in the row-interleaved layout (moda_depth_cache_bytes(B, T, H_kv, d, .)) and the
+ *                    slot to write, or cache == NULL for the projection alone
+ * bf16 inputs, fp32 accumulation on the tensor cores, one rounding to bf16; the slot receives bit for bit what
+ * moda_depth_cache_append(cache, ..., slot, K_out, V_out) would store (tail rows of a ragged last tile are zero),
+ * without K and V crossing HBM again.  One launch on `stream`; device pointers owned by the caller; validation,
+ * asynchrony and error codes as for the other calls.
+ */
+int moda_kv_project_append(const void* X, const void* Wk, const void* Wv,
+                           int B, int T, int D_model, int H_kv, int d,
+                           void* K_out, void* V_out, void* cache, int slot, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

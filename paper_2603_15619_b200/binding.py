@@ -26,6 +26,7 @@ SYMBOLS = (
     "moda_attn_decode_varlen", "moda_attn_decode_paged",
     "moda_depth_cache_e4m3_bytes", "moda_depth_cache_append_e4m3", "moda_attn_fwd_e4m3", "moda_attn_bwd_e4m3",
     "moda_depth_cache_append_pm", "moda_depth_cache_unpack_pm", "moda_attn_fwd_gqa_pm", "moda_attn_bwd_gqa_pm",
+    "moda_kv_project_append",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -115,6 +116,8 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_fwd_gqa_pm.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
     lib.moda_attn_bwd_gqa_pm.restype = ci
     lib.moda_attn_bwd_gqa_pm.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
+    lib.moda_kv_project_append.restype = ci
+    lib.moda_kv_project_append.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, vp, ci, vp]
     _lib = lib
     return lib
 
@@ -326,6 +329,26 @@ def moda_attn_bwd_gqa_pm(Q, K, V, depth_kv_pm, O, dO, LSE, l, scale,
                                        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "moda_attn_bwd_gqa_pm")
     return dQ, dK, dV, d_depth_kv_pm
+
+
+def moda_kv_project_append(X, Wk, Wv, H_kv, cache=None, slot=0, store_kv=True, K_out=None, V_out=None, stream=None):
+    """K, V [B,T,H_kv,d] = X [B,T,D_model] times the key / value projections Wk, Wv [H_kv d, D_model]; with ``cache`` the
+    same launch writes them as depth slot ``slot``.  ``store_kv=False`` (FFN-side projection) writes the slot only."""
+    if X.dim() != 3 or X.dtype != torch.bfloat16:
+        raise ValueError("X must be a bf16 [B, T, D_model] tensor")
+    B, T, Dm = X.shape
+    n = Wk.shape[0]
+    if Wk.shape != (n, Dm) or Wv.shape != (n, Dm) or n % H_kv or Wk.dtype != torch.bfloat16 or Wv.dtype != torch.bfloat16:
+        raise ValueError("Wk, Wv must be bf16 [H_kv d, D_model] tensors matching X")
+    d = n // H_kv
+    if store_kv:
+        K_out = _new((B, T, H_kv, d), torch.bfloat16, X.device, stream) if K_out is None else K_out
+        V_out = _new((B, T, H_kv, d), torch.bfloat16, X.device, stream) if V_out is None else V_out
+    else:
+        K_out = V_out = None
+    _check(load().moda_kv_project_append(_ptr(X), _ptr(Wk), _ptr(Wv), B, T, Dm, int(H_kv), d, _ptr(K_out), _ptr(V_out),
+                                         _ptr(cache), int(slot), _stream(stream)), "moda_kv_project_append")
+    return K_out, V_out
 
 
 def moda_attn_fwd(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):

@@ -13,6 +13,7 @@
 #include "moda_depth_gqa.cuh"
 #include "moda_fwd.cuh"
 #include "moda_fwd_wide.cuh"
+#include "moda_kvproj.cuh"
 #include "sm100_ptx.cuh"
 
 namespace {
@@ -540,6 +541,37 @@ int launch_cache_pm_copy(void* cache, int B, int T, int H, int slot, void* Xk, v
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 
+// Key / value projection with the write step in its epilogue.
+template <int D>
+int launch_kv_project(const void* X, const void* Wk, const void* Wv, int B, int T, int Dm, int Hk,
+                      void* K_out, void* V_out, void* slot, cudaStream_t stream) {
+    using L = KvProjSmem<D>;
+    CUtensorMap mX, mWk, mWv, mK, mV;
+    // X [B][T][Dm] and W [Hk d][Dm] are addressed in 64-feature columns: [outer][rows][Dm / 64][64]
+    if (!make_bthd_map(&mX, X, B, T, Dm / 64, 64) || !make_bthd_map(&mWk, Wk, 1, Hk * D, Dm / 64, 64, D) ||
+        !make_bthd_map(&mWv, Wv, 1, Hk * D, Dm / 64, 64, D))
+        return MODA_ERR_CUDA;
+    // without K / V outputs the store maps are never used; they still have to be valid objects
+    const void* kout = K_out ? K_out : X;
+    if (!make_bthd_map(&mK, kout, B, T, K_out ? Hk : Dm / 64, K_out ? D : 64) ||
+        !make_bthd_map(&mV, V_out ? V_out : X, B, T, V_out ? Hk : Dm / 64, V_out ? D : 64))
+        return MODA_ERR_CUDA;
+    static thread_local int configured_dev = -1;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (configured_dev != dev) {
+        if (!set_smem_limit(moda_kv_project_kernel<D>, L::kDynamic)) return MODA_ERR_CUDA;
+        configured_dev = dev;
+    }
+    KvProjParams p;
+    p.slot = static_cast<__nv_bfloat16*>(slot);
+    p.B = B; p.T = T; p.Hk = Hk; p.Dm = Dm;
+    p.store_kv = K_out != nullptr ? 1 : 0;
+    const unsigned grid = unsigned(B) * num_tiles(T) * Hk;
+    moda_kv_project_kernel<D><<<grid, kProjThreads, L::kDynamic, stream>>>(mX, mWk, mWv, mK, mV, p);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+}
+
 // Decode step: a split kernel over the KV cache and a merge kernel that adds the depth pairs.
 template <int D, int G>
 int launch_decode_g(const DecodeParams& p, cudaStream_t stream) {
@@ -975,6 +1007,22 @@ int moda_attn_bwd_gqa_pm(const void* Q, const void* K, const void* V, const void
     a.dQ = dQ; a.dK = dK; a.dV = dV; a.d_depth_kv = d_depth_kv_pm; a.workspace = workspace;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return d == 128 ? launch_bwd_fused<128>(a, MODA_BWD_ALL_STAGES, st) : launch_bwd_fused<64>(a, MODA_BWD_ALL_STAGES, st);
+}
+
+int moda_kv_project_append(const void* X, const void* Wk, const void* Wv,
+                           int B, int T, int D_model, int H_kv, int d,
+                           void* K_out, void* V_out, void* cache, int slot, void* stream) {
+    if (int rc = check_shape(B, T, H_kv, d)) return rc;
+    if (D_model < 64 || D_model % 64 != 0 || (long long)B * T > 0x7fffffffLL / D_model) return MODA_ERR_BAD_SHAPE;
+    if (cache != nullptr && (slot < 0 || slot >= MODA_MAX_DEPTH)) return MODA_ERR_BAD_SLOT;
+    if (!X || !Wk || !Wv || (K_out == nullptr) != (V_out == nullptr) || (!K_out && !cache)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(X) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(K_out) || !aligned16(V_out) || !aligned16(cache))
+        return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    void* slot_base = cache ? static_cast<__nv_bfloat16*>(cache) + size_t(slot) * cache_slot_elems(B, T, H_kv, d) : nullptr;
+    return d == 128 ? launch_kv_project<128>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st)
+                    : launch_kv_project<64>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
 }
 
 size_t moda_decode_workspace_bytes(int B, int H, int d) {

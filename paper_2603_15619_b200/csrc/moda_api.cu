@@ -542,33 +542,32 @@ int launch_cache_pm_copy(void* cache, int B, int T, int H, int slot, void* Xk, v
 }
 
 // Key / value projection with the write step in its epilogue.
-template <int D>
+template <int D, int NH>
 int launch_kv_project(const void* X, const void* Wk, const void* Wv, int B, int T, int Dm, int Hk,
                       void* K_out, void* V_out, void* slot, cudaStream_t stream) {
-    using L = KvProjSmem<D>;
+    using L = KvProjSmem<D, NH>;
     CUtensorMap mX, mWk, mWv, mK, mV;
     // X [B][T][Dm] and W [Hk d][Dm] are addressed in 64-feature columns: [outer][rows][Dm / 64][64]
-    if (!make_bthd_map(&mX, X, B, T, Dm / 64, 64) || !make_bthd_map(&mWk, Wk, 1, Hk * D, Dm / 64, 64, D) ||
-        !make_bthd_map(&mWv, Wv, 1, Hk * D, Dm / 64, 64, D))
+    if (!make_bthd_map(&mX, X, B, T, Dm / 64, 64) || !make_bthd_map(&mWk, Wk, 1, Hk * D, Dm / 64, 64, D * NH) ||
+        !make_bthd_map(&mWv, Wv, 1, Hk * D, Dm / 64, 64, D * NH))
         return MODA_ERR_CUDA;
     // without K / V outputs the store maps are never used; they still have to be valid objects
-    const void* kout = K_out ? K_out : X;
-    if (!make_bthd_map(&mK, kout, B, T, K_out ? Hk : Dm / 64, K_out ? D : 64) ||
+    if (!make_bthd_map(&mK, K_out ? K_out : X, B, T, K_out ? Hk : Dm / 64, K_out ? D : 64) ||
         !make_bthd_map(&mV, V_out ? V_out : X, B, T, V_out ? Hk : Dm / 64, V_out ? D : 64))
         return MODA_ERR_CUDA;
     static thread_local int configured_dev = -1;
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
     if (configured_dev != dev) {
-        if (!set_smem_limit(moda_kv_project_kernel<D>, L::kDynamic)) return MODA_ERR_CUDA;
+        if (!set_smem_limit(moda_kv_project_kernel<D, NH>, L::kDynamic)) return MODA_ERR_CUDA;
         configured_dev = dev;
     }
     KvProjParams p;
     p.slot = static_cast<__nv_bfloat16*>(slot);
     p.B = B; p.T = T; p.Hk = Hk; p.Dm = Dm;
     p.store_kv = K_out != nullptr ? 1 : 0;
-    const unsigned grid = unsigned(B) * num_tiles(T) * Hk;
-    moda_kv_project_kernel<D><<<grid, kProjThreads, L::kDynamic, stream>>>(mX, mWk, mWv, mK, mV, p);
+    const unsigned grid = unsigned(B) * num_tiles(T) * (Hk / NH);
+    moda_kv_project_kernel<D, NH><<<grid, kProjThreads, L::kDynamic, stream>>>(mX, mWk, mWv, mK, mV, p);
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 
@@ -1021,8 +1020,10 @@ int moda_kv_project_append(const void* X, const void* Wk, const void* Wv,
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     void* slot_base = cache ? static_cast<__nv_bfloat16*>(cache) + size_t(slot) * cache_slot_elems(B, T, H_kv, d) : nullptr;
-    return d == 128 ? launch_kv_project<128>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st)
-                    : launch_kv_project<64>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
+    if (d == 128) return launch_kv_project<128, 1>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
+    // d = 64: two heads per CTA (one tensor-core instruction of 256 columns) when the heads pair up
+    return H_kv % 2 == 0 ? launch_kv_project<64, 2>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st)
+                         : launch_kv_project<64, 1>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
 }
 
 size_t moda_decode_workspace_bytes(int B, int H, int d) {

@@ -4,14 +4,16 @@
 //
 //   K[b, t, h, :] = X[b, t, :] Wk[h d : (h+1) d, :]^T        V likewise        (bf16 in, fp32 accumulation, bf16 out)
 //
-// One CTA owns one (b, 128-position tile, key/value head): the output tile of a head is exactly one block of the
-// depth cache (moda_cache.cuh), so the epilogue stores the rounded tile twice from the same registers: as the K / V
-// tensors [B][T][H_k][d] (through shared memory and a TMA store) and as the cache slot's blocks (chunk c of row r to
-// [c][r]: 512 contiguous bytes per warp store).  K and V of a head share the X tiles: two accumulators of d columns.
+// One CTA owns one (b, 128-position tile) and NH key/value heads (two at d = 64 when H_k is even, else one): the
+// output tile of a head is exactly one block of the depth cache (moda_cache.cuh), so the epilogue stores the rounded
+// tile twice from the same registers: as the K / V tensors [B][T][H_k][d] (through shared memory and a TMA store) and
+// as the cache slot's blocks (chunk c of row r to [c][r]: 512 contiguous bytes per warp store).  K and V share the X
+// tiles: the Wk and Wv tiles of a stage are adjacent in shared memory and form one B operand of 2 NH d rows, so one
+// tcgen05.mma (M 128, N 2 NH d <= 256, K 16) feeds both accumulators.
 //
-//   warp 0      TMA producer: per 64 input features one X tile [128 x 64] and one Wk and one Wv tile [d x 64]
-//               through a four-stage ring (128-byte swizzle)
-//   warp 1      MMA issuer (owns the tensor-memory allocation): 4 + 4 tcgen05.mma (M 128, N d, K 16) per stage
+//   warp 0      TMA producer: per 64 input features one X tile [128 x 64] and one Wk and one Wv tile [NH d x 64]
+//               through a ring (128-byte swizzle); two CTAs fit an SM, so one's epilogue runs under the other's loop
+//   warp 1      MMA issuer (owns the tensor-memory allocation): 4 tcgen05.mma per stage
 //   warps 2-5   epilogue: a thread owns one position (= TMEM lane)
 #pragma once
 
@@ -23,14 +25,18 @@ namespace moda {
 
 constexpr int kProjThreads = 192;
 
-template <int D>
+#ifndef MODA_PROJ_STAGES
+#define MODA_PROJ_STAGES 2
+#endif
+template <int D, int NH>
 struct KvProjSmem {
-    static constexpr int kStages = 4;
+    static constexpr int kStages = MODA_PROJ_STAGES;
+    static constexpr int kNW = D * NH;                         // output features per W tile
     static constexpr int kXBytes = kTileRows * 128;            // 128 positions x 64 features bf16
-    static constexpr int kWBytes = D * 128;                    // d output features x 64 input features bf16
+    static constexpr int kWBytes = kNW * 128;                  // NH d output features x 64 input features bf16
     static constexpr int kStageBytes = kXBytes + 2 * kWBytes;
     static constexpr int kRing = 0;
-    static constexpr int kOutBytes = 2 * kTileRows * D * 2;    // K and V tiles for the TMA stores, over the ring
+    static constexpr int kOutBytes = 2 * kTileRows * kNW * 2;  // K and V tiles for the TMA stores, over the ring
     static_assert(kOutBytes <= kStages * kStageBytes, "output staging does not fit the ring");
     static constexpr int kBars = kStages * kStageBytes;        // full[4], empty[4], accumulators complete
     static constexpr int kMisc = kBars + 16 * 8;               // tmem base, abort flag
@@ -44,14 +50,15 @@ struct KvProjParams {
     int store_kv;              // nonzero: K and V are also stored as [B][T][H_k][d] tensors
 };
 
-template <int D>
-__global__ void __launch_bounds__(kProjThreads, 1)
+template <int D, int NH>
+__global__ void __launch_bounds__(kProjThreads, 2)
 moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapWk,
                        const __grid_constant__ CUtensorMap mapWv, const __grid_constant__ CUtensorMap mapK,
                        const __grid_constant__ CUtensorMap mapV, const KvProjParams p) {
-    using L = KvProjSmem<D>;
+    using L = KvProjSmem<D, NH>;
     constexpr int NSUB = D / 64;
-    constexpr uint32_t kTmemCols = 2 * D;                      // 128 or 256: K accumulator, V accumulator
+    constexpr int NW = L::kNW;
+    constexpr uint32_t kTmemCols = 2 * NW;                     // 128 or 256: K accumulators of the NH heads, then V
     if (g_moda_status != 0) return;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -70,9 +77,10 @@ moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_co
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nt = num_tiles(p.T);
-    const int hk = blockIdx.x % p.Hk;
-    const int tile = (blockIdx.x / p.Hk) % nt;
-    const int b = blockIdx.x / (p.Hk * nt);
+    const int hgroups = p.Hk / NH;
+    const int hk0 = (blockIdx.x % hgroups) * NH;               // first of this CTA's heads
+    const int tile = (blockIdx.x / hgroups) % nt;
+    const int b = blockIdx.x / (hgroups * nt);
     const int t0 = tile * kTileRows;
     const int n_k = p.Dm / 64;
 
@@ -108,24 +116,22 @@ moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_co
                 mbar_arrive_expect_tx(bar_full(st), L::kStageBytes);
                 // the tensors are addressed as [outer][rows][Dm / 64][64]: coordinate 1 picks the 64 input features
                 tma_load_4d(dst, &mapX, bar_full(st), 0, k, t0, b);
-                tma_load_4d(dst + L::kXBytes, &mapWk, bar_full(st), 0, k, hk * D, 0);
-                tma_load_4d(dst + L::kXBytes + L::kWBytes, &mapWv, bar_full(st), 0, k, hk * D, 0);
+                tma_load_4d(dst + L::kXBytes, &mapWk, bar_full(st), 0, k, hk0 * D, 0);
+                tma_load_4d(dst + L::kXBytes + L::kWBytes, &mapWv, bar_full(st), 0, k, hk0 * D, 0);
             }
         }
     } else if (warp == 1) {
         // =========================== MMA issuer ===========================
-        constexpr uint32_t idesc = make_idesc_bf16(128, D, false, false);
+        constexpr uint32_t idesc = make_idesc_bf16(128, 2 * NW, false, false);
         for (int k = 0; k < n_k; ++k) {
             const int st = k % L::kStages;
             mbar_wait(bar_full(st), (k / L::kStages) & 1, abort_flag, 161);
             tc_fence_after_sync();
             const uint32_t x = sbase + L::kRing + st * L::kStageBytes;
+            // B = the Wk tile and, right behind it, the Wv tile: 2 NW rows of 128 bytes, 8-row groups 1024 bytes apart
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                const uint64_t dx = desc_kmajor_sw128(x, kk);
-                umma_ss(tmem, dx, desc_kmajor_sw128(x + L::kXBytes, kk), idesc, (k > 0 || kk > 0) ? 1u : 0u);
-                umma_ss(tmem + D, dx, desc_kmajor_sw128(x + L::kXBytes + L::kWBytes, kk), idesc, (k > 0 || kk > 0) ? 1u : 0u);
-            }
+            for (int kk = 0; kk < 4; ++kk)
+                umma_ss(tmem, desc_kmajor_sw128(x, kk), desc_kmajor_sw128(x + L::kXBytes, kk), idesc, (k > 0 || kk > 0) ? 1u : 0u);
             umma_commit(bar_empty(st));
         }
         umma_commit(bar_acc);
@@ -143,27 +149,30 @@ moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_co
         tc_fence_after_sync();
         // every MMA has completed, so the ring is free: it becomes the staging of the two output tiles
         constexpr int CH = D / 8;
-        uint4* slot_blk = p.slot == nullptr ? nullptr
-                          : reinterpret_cast<uint4*>(p.slot) + ((size_t(b) * p.Hk + hk) * nt + tile) * 2 * (kTileRows * CH) + r;
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t a[32];
-                tmem_ld32(tmem + lane_addr + kv * D + c * 32, a);
-                tmem_wait_ld();
+            for (int j = 0; j < NH; ++j) {
+                uint4* slot_blk = p.slot == nullptr ? nullptr
+                                  : reinterpret_cast<uint4*>(p.slot) + (((size_t(b) * p.Hk + hk0 + j) * nt + tile) * 2 + kv) * (kTileRows * CH) + r;
+                uint8_t* stage = smem + L::kRing + (kv * NH + j) * (kTileRows * D * 2);
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(a[8 * g + 0]), __uint_as_float(a[8 * g + 1]));
-                    v.y = pack_bf16x2(__uint_as_float(a[8 * g + 2]), __uint_as_float(a[8 * g + 3]));
-                    v.z = pack_bf16x2(__uint_as_float(a[8 * g + 4]), __uint_as_float(a[8 * g + 5]));
-                    v.w = pack_bf16x2(__uint_as_float(a[8 * g + 6]), __uint_as_float(a[8 * g + 7]));
-                    const int chunk = c * 4 + g;
-                    // rows past T were loaded as zeros: the cache wants exactly that in its tail rows
-                    if (slot_blk != nullptr) slot_blk[(kv * CH + chunk) * kTileRows] = v;
-                    if (p.store_kv)
-                        *reinterpret_cast<uint4*>(smem + L::kRing + kv * (kTileRows * D * 2) + swz_chunk_offset(r, chunk)) = v;
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t a[32];
+                    tmem_ld32(tmem + lane_addr + kv * NW + j * D + c * 32, a);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(a[8 * g + 0]), __uint_as_float(a[8 * g + 1]));
+                        v.y = pack_bf16x2(__uint_as_float(a[8 * g + 2]), __uint_as_float(a[8 * g + 3]));
+                        v.z = pack_bf16x2(__uint_as_float(a[8 * g + 4]), __uint_as_float(a[8 * g + 5]));
+                        v.w = pack_bf16x2(__uint_as_float(a[8 * g + 6]), __uint_as_float(a[8 * g + 7]));
+                        const int chunk = c * 4 + g;
+                        // rows past T were loaded as zeros: the cache wants exactly that in its tail rows
+                        if (slot_blk != nullptr) slot_blk[chunk * kTileRows] = v;
+                        if (p.store_kv) *reinterpret_cast<uint4*>(stage + swz_chunk_offset(r, chunk)) = v;
+                    }
                 }
             }
         }
@@ -172,10 +181,12 @@ moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_co
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (tid == 64) {
 #pragma unroll
-                for (int s = 0; s < NSUB; ++s) {
-                    tma_store_4d(&mapK, sbase + L::kRing + s * (kTileRows * 128), s * 64, hk, t0, b);
-                    tma_store_4d(&mapV, sbase + L::kRing + kTileRows * D * 2 + s * (kTileRows * 128), s * 64, hk, t0, b);
-                }
+                for (int j = 0; j < NH; ++j)
+#pragma unroll
+                    for (int s = 0; s < NSUB; ++s) {
+                        tma_store_4d(&mapK, sbase + L::kRing + j * (kTileRows * D * 2) + s * (kTileRows * 128), s * 64, hk0 + j, t0, b);
+                        tma_store_4d(&mapV, sbase + L::kRing + (NH + j) * (kTileRows * D * 2) + s * (kTileRows * 128), s * 64, hk0 + j, t0, b);
+                    }
                 tma_store_commit();
                 tma_store_wait_all();
             }

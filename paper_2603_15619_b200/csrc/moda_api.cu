@@ -541,34 +541,51 @@ int launch_cache_pm_copy(void* cache, int B, int T, int H, int slot, void* Xk, v
     return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 
-// Key / value projection with the write step in its epilogue.
+// Key / value projection with the write step in its epilogue: a persistent kernel on CTA pairs (clusters of two CTAs).
 template <int D, int NH>
 int launch_kv_project(const void* X, const void* Wk, const void* Wv, int B, int T, int Dm, int Hk,
                       void* K_out, void* V_out, void* slot, cudaStream_t stream) {
     using L = KvProjSmem<D, NH>;
     CUtensorMap mX, mWk, mWv, mK, mV;
-    // X [B][T][Dm] and W [Hk d][Dm] are addressed in 64-feature columns: [outer][rows][Dm / 64][64]
     if (!make_bthd_map(&mX, X, B, T, Dm / 64, 64) || !make_bthd_map(&mWk, Wk, 1, Hk * D, Dm / 64, 64, D * NH) ||
         !make_bthd_map(&mWv, Wv, 1, Hk * D, Dm / 64, 64, D * NH))
         return MODA_ERR_CUDA;
-    // without K / V outputs the store maps are never used; they still have to be valid objects
     if (!make_bthd_map(&mK, K_out ? K_out : X, B, T, K_out ? Hk : Dm / 64, K_out ? D : 64) ||
         !make_bthd_map(&mV, V_out ? V_out : X, B, T, V_out ? Hk : Dm / 64, V_out ? D : 64))
         return MODA_ERR_CUDA;
-    static thread_local int configured_dev = -1;
-    int dev = 0;
-    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
-    if (configured_dev != dev) {
-        if (!set_smem_limit(moda_kv_project_kernel<D, NH>, L::kDynamic)) return MODA_ERR_CUDA;
-        configured_dev = dev;
-    }
     KvProjParams p;
     p.slot = static_cast<__nv_bfloat16*>(slot);
     p.B = B; p.T = T; p.Hk = Hk; p.Dm = Dm;
     p.store_kv = K_out != nullptr ? 1 : 0;
-    const unsigned grid = unsigned(B) * num_tiles(T) * (Hk / NH);
-    moda_kv_project_kernel<D, NH><<<grid, kProjThreads, L::kDynamic, stream>>>(mX, mWk, mWv, mK, mV, p);
-    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
+    const long long items = (long long)B * ((num_tiles(T) + 1) / 2) * (Hk / NH);
+    if (items > 0x3fffffffLL) return MODA_ERR_BAD_SHAPE;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kProjThreads, 1, 1);
+    cfg.dynamicSmemBytes = L::kDynamic;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // persistent: as many pairs as the device can hold at once (a pair needs two SMs of one cluster domain; 74 on a B200)
+    static thread_local int configured_dev = -1;
+    static thread_local int resident_pairs = 0;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
+    if (configured_dev != dev) {
+        if (!set_smem_limit(moda_kv_project_kernel<D, NH>, L::kDynamic)) return MODA_ERR_CUDA;
+        int n = 0;
+        cfg.gridDim = dim3(1024, 1, 1);                        // any multiple of the cluster size: the query asks what fits
+        if (!cuda_ok(cudaOccupancyMaxActiveClusters(&n, moda_kv_project_kernel<D, NH>, &cfg)) || n < 1) return MODA_ERR_CUDA;
+        resident_pairs = n;
+        configured_dev = dev;
+    }
+    const long long clusters = items < resident_pairs ? items : resident_pairs;
+    cfg.gridDim = dim3(unsigned(2 * clusters), 1, 1);
+    return cuda_ok(cudaLaunchKernelEx(&cfg, moda_kv_project_kernel<D, NH>, mX, mWk, mWv, mK, mV, p)) ? MODA_OK : MODA_ERR_CUDA;
 }
 
 // Decode step: a split kernel over the KV cache and a merge kernel that adds the depth pairs.

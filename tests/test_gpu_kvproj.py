@@ -24,6 +24,9 @@ SHAPES = [
     # B, T, D_model, H_kv, d
     (1, 128, 64, 1, 64), (1, 1, 64, 1, 128), (2, 300, 256, 2, 128), (1, 1000, 512, 3, 64), (1, 129, 1024, 2, 128),
     (3, 257, 320, 5, 64), (1, 640, 2048, 2, 128),     # more input features than the ring holds: it wraps several times
+    # more work items than resident CTA pairs (74 on a B200): a pair takes several items, both accumulator sets are
+    # reused, and (odd tile count) the last pair of each batch entry has a CTA without a tile
+    (2, 2000, 256, 6, 128), (3, 2500, 128, 8, 128), (4, 1300, 192, 8, 64), (2, 2700, 64, 7, 64),
 ]
 
 

@@ -345,6 +345,8 @@ def run_moda(args, rank, world, device):
             out["decode_sweep"] = run_decode_sweep(peaks, device)
         if "prefill" in extra:
             out["prefill_sweep"] = run_prefill_sweep(peaks, device)
+        if "kvproj" in extra:
+            out["kvproj_sweep"] = run_kvproj_sweep(peaks, device)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, budget_s=20.0)
     return out
@@ -639,6 +641,39 @@ def run_prefill_sweep(peaks, device, shapes=None, iters=5):
     return rows
 
 
+# Key / value projection with the write step in its epilogue (B, T, D_model, H_kv, d).
+KVPROJ_SHAPES = [(1, 65536, 2048, 16, 128), (2, 8192, 2048, 16, 128), (2, 32768, 2048, 32, 64), (1, 16384, 4096, 8, 128)]
+
+
+def run_kvproj_sweep(peaks, device, shapes=None, iters=10):
+    """K = X Wk^T, V = X Wv^T plus the depth slot in one launch; FLOPs = 2 * positions * D_model * 2 H_kv d.  The library
+    columns (one GEMM on the concatenated weights, then the separate append) are what the fused launch replaces."""
+    import paper_2603_15619_b200 as moda
+    rows = []
+    for B, T, Dm, Hk, d in (shapes or KVPROJ_SHAPES):
+        torch.cuda.empty_cache()
+        g = torch.Generator(device=device).manual_seed(0)
+        X = torch.randn((B, T, Dm), device=device, generator=g).to(torch.bfloat16)
+        Wk = (torch.randn((Hk * d, Dm), device=device, generator=g) * Dm ** -0.5).to(torch.bfloat16)
+        Wv = (torch.randn((Hk * d, Dm), device=device, generator=g) * Dm ** -0.5).to(torch.bfloat16)
+        cache = moda.alloc_depth_cache(B, T, Hk, d, 1, device)
+        K = torch.empty((B, T, Hk, d), dtype=torch.bfloat16, device=device)
+        V = torch.empty_like(K)
+        Wkv = torch.cat([Wk, Wv], 0)
+        ms = time_calls(lambda: moda.moda_kv_project_append(X, Wk, Wv, Hk, cache=cache, slot=0, K_out=K, V_out=V), iters)
+        ms_slot = time_calls(lambda: moda.moda_kv_project_append(X, Wk, Wv, Hk, cache=cache, slot=0, store_kv=False), iters)
+        ms_lib = time_calls(lambda: torch.nn.functional.linear(X, Wkv), iters)
+        ms_app = time_calls(lambda: moda.moda_depth_cache_append(cache, 0, K, V), iters)
+        fl = 2.0 * B * T * Dm * 2 * Hk * d
+        rows.append({"B": B, "T": T, "D_model": Dm, "H_kv": Hk, "d": d, "ms": round(ms, 4), "tflops": round(fl / ms / 1e9, 1),
+                     "frac_measured_burst_bf16": round(fl / ms / 1e9 / peaks["bf16_tflops"], 4),
+                     "slot_only_ms": round(ms_slot, 4), "library_gemm_ms": round(ms_lib, 4), "separate_append_ms": round(ms_app, 4)})
+        log("kvproj_sweep", rows[-1])
+        del X, Wk, Wv, Wkv, cache, K, V
+    torch.cuda.empty_cache()
+    return rows
+
+
 def run_e2e(layer, steps, world, step_flops, device):
     """The same step driven from pinned HOST buffers: every step copies its inputs host->device and
     its results device->host inside the timed region.  Two device buffer sets and three streams let
@@ -795,7 +830,7 @@ def main():
     ap.add_argument("--impl", default="moda", choices=["moda", "reference"])
     ap.add_argument("--workload", default="c4", help="c1..c5, optionally with _l<depth> (e.g. c3_l8)")
     ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the host-to-host leg (each moves every input and output over PCIe)")
-    ap.add_argument("--sweeps", default="", help="comma list of extra sweeps printed in the line: gqa, decode, prefill")
+    ap.add_argument("--sweeps", default="", help="comma list of extra sweeps printed in the line: gqa, decode, prefill, kvproj")
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (smaller profiling cases)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -803,6 +838,8 @@ def main():
     ap.add_argument("--gqa-shape", default="", help="T,G[,L]: time only this grouped-query shape (B=1, d=64, 8 key/value "
                                                     "heads, L depth slots (default 32) and l=0) and print its row; for profiling")
     ap.add_argument("--prefill-sweep", action="store_true", help="time only the prefill-with-cache shapes and print their rows")
+    ap.add_argument("--kvproj-shape", default="", help="B,T,D_model,H_kv,d (or 'all'): time only the key/value projection with the "
+                    "write step in its epilogue and print its rows; for profiling")
     ap.add_argument("--decode-shape", default="", help="B,T_kv,H,H_kv,d,l: time only this decode step and print its row; for profiling")
     args = ap.parse_args()
 
@@ -833,6 +870,10 @@ def main():
             out = {"gqa_sweep": run_gqa_sweep(device, [(v[0], v[1], v[2] if len(v) > 2 else 32, None)])}
         elif args.prefill_sweep:
             out = {"prefill_sweep": run_prefill_sweep(load_peaks(), device)}
+        elif args.kvproj_shape:
+            v = args.kvproj_shape
+            shapes = None if v == "all" else [tuple(int(t) for t in v.split(","))]
+            out = {"kvproj_sweep": run_kvproj_sweep(load_peaks(), device, shapes, iters=max(1, min(args.steps, 20)))}
         elif args.decode_shape:
             v = tuple(int(t) for t in args.decode_shape.split(","))
             out = {"decode_sweep": run_decode_sweep(load_peaks(), device, [v], iters=max(1, min(args.steps, 20)))}

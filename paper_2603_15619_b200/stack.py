@@ -77,6 +77,33 @@ class _Write(torch.autograd.Function):
         return dK, dV, dtoken, None, None
 
 
+class _ProjectWrite(torch.autograd.Function):
+    """A slot produced by a key / value projection of X (Sec. 2.2: an FFN layer obtains its depth pair through a KV
+    projection of its input) and written by the projection's own epilogue: one launch, K and V never stored.  Backward:
+    the slot of the gradient cache is dK, dV; dX = dK Wk + dV Wv and dW = dK^T X are plain library GEMMs."""
+
+    @staticmethod
+    def forward(ctx, X, Wk, Wv, token, stream, slot):
+        X, Wk, Wv = X.contiguous(), Wk.contiguous(), Wv.contiguous()
+        binding.moda_kv_project_append(X, Wk, Wv, stream.shape[2], cache=stream.cache, slot=slot, store_kv=False)
+        ctx.stream, ctx.slot = stream, slot
+        ctx.save_for_backward(X, Wk, Wv)
+        return token + 0
+
+    @staticmethod
+    def backward(ctx, dtoken):
+        X, Wk, Wv = ctx.saved_tensors
+        B, T, Hk, d = ctx.stream.shape
+        if not ctx.stream.slot_has_grad(ctx.slot):
+            return torch.zeros_like(X), torch.zeros_like(Wk), torch.zeros_like(Wv), dtoken, None, None
+        dK = torch.empty((B, T, Hk, d), dtype=X.dtype, device=X.device)
+        dV = torch.empty_like(dK)
+        binding.moda_depth_cache_unpack(ctx.stream.grad_cache, ctx.slot, dK, dV)
+        dK2, dV2, X2 = dK.view(B * T, Hk * d), dV.view(B * T, Hk * d), X.view(B * T, -1)
+        dX = torch.addmm(dK2 @ Wk, dV2, Wv).view_as(X)
+        return dX, dK2.t() @ X2, dV2.t() @ X2, dtoken, None, None
+
+
 class DepthStream:
     """Depth cache of one forward pass through a stack (and its gradient cache)."""
 
@@ -108,4 +135,13 @@ class DepthStream:
         if slot >= self.n_layers:
             raise ValueError("more slots than the stream was sized for")
         self.token = _Write.apply(K, V, self.token, self, slot)
+        self.n_written = slot + 1
+
+    def project_write(self, X, Wk, Wv):
+        """Appends K = X Wk^T, V = X Wv^T (X [B,T,D_model], W [H_kv d, D_model]) as the next slot without attending:
+        the projection kernel writes the slot from its epilogue."""
+        slot = self.n_written
+        if slot >= self.n_layers:
+            raise ValueError("more slots than the stream was sized for")
+        self.token = _ProjectWrite.apply(X, Wk, Wv, self.token, self, slot)
         self.n_written = slot + 1

@@ -106,6 +106,38 @@ def test_slot_written_without_attending_gets_the_gradients_of_the_layers_after_i
         assert rel_l2(f64(got), want) <= TOL_GRAD_REL_L2
 
 
+@pytest.mark.parametrize("B,T,H,Hk,d,Dm", [(1, 200, 4, 2, 64, 128), (2, 300, 2, 2, 128, 192)])
+def test_slot_projected_from_a_layer_input_sends_its_gradient_to_the_input_and_the_weights(B, T, H, Hk, d, Dm):
+    """FFN-side depth pair: slot 0 = projection of X (written by the projection's epilogue), then an attention layer.
+    The oracle's slot gradients, pulled back through the fp64 projection, are the gradients of X, Wk, Wv."""
+    scale = d ** -0.5
+    a = synthetic.make_gqa(B, T, H, Hk, d, 0, seed=7, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(8)
+    X = torch.randn((B, T, Dm), device="cuda", generator=g).to(torch.bfloat16).requires_grad_()
+    Wk = (torch.randn((Hk * d, Dm), device="cuda", generator=g) * Dm ** -0.5).to(torch.bfloat16).requires_grad_()
+    Wv = (torch.randn((Hk * d, Dm), device="cuda", generator=g) * Dm ** -0.5).to(torch.bfloat16).requires_grad_()
+    Q, K, V = (a[k].clone().requires_grad_() for k in ("Q", "K", "V"))
+    stream = moda.DepthStream(B, T, Hk, d, 2)
+    stream.project_write(X, Wk, Wv)                        # slot 0
+    O = stream.attend(Q, K, V, scale)                      # attends to slot 0, writes slot 1
+    (O.float() * a["dO"].float()).sum().backward()
+    assert moda.moda_last_status() == 0
+    # the operator sees the slot as stored (rounded to bf16); the oracle gets exactly those values
+    Ks, Vs = torch.empty((B, T, Hk, d), dtype=torch.bfloat16, device="cuda"), torch.empty((B, T, Hk, d), dtype=torch.bfloat16, device="cuda")
+    moda.moda_depth_cache_unpack(stream.cache, 0, Ks, Vs)
+    K_ref, V_ref = orc.project_kv(f64(X), f64(Wk), f64(Wv), Hk)
+    assert rel_l2(f64(Ks), K_ref) <= TOL_O_REL_L2 and rel_l2(f64(Vs), V_ref) <= TOL_O_REL_L2
+    O_ref, _ = orc.forward_gqa(f64(Q), f64(K), f64(V), f64(Ks)[None], f64(Vs)[None], scale)
+    assert rel_l2(f64(O), O_ref) <= TOL_O_REL_L2
+    dQ, dK, dV, dKd, dVd = orc.backward_gqa(f64(Q), f64(K), f64(V), f64(Ks)[None], f64(Vs)[None], f64(a["dO"]), scale)
+    gk, gv = dKd[0].reshape(B * T, Hk * d), dVd[0].reshape(B * T, Hk * d)
+    x2 = f64(X).reshape(B * T, Dm)
+    dX_ref = (gk @ f64(Wk) + gv @ f64(Wv)).reshape(B, T, Dm)
+    for got, want, name in ((Q.grad, dQ, "dQ"), (K.grad, dK, "dK"), (V.grad, dV, "dV"), (X.grad, dX_ref, "dX"),
+                            (Wk.grad, gk.T @ x2, "dWk"), (Wv.grad, gv.T @ x2, "dWv")):
+        assert rel_l2(f64(got), want) <= TOL_GRAD_REL_L2, f"{name}: {rel_l2(f64(got), want):.3e}"
+
+
 @pytest.mark.parametrize("B,T,H,Hk,d,l,S", [(1, 300, 2, 2, 64, 7, 3), (1, 200, 4, 2, 128, 6, 2)])
 def test_window_of_the_last_slots_is_the_operator_on_those_slots(B, T, H, Hk, d, l, S):
     """Bounded depth slots: a layer that attends only to the last S of l stored slots, forward and backward."""

@@ -82,3 +82,31 @@ def test_the_written_slot_feeds_the_attention():
     O_ref, LSE_ref = orc.forward(f64(Q), f64(K1), f64(V1), bf(K_ref)[None], bf(V_ref)[None], d ** -0.5)
     from parity import assert_forward_close
     assert_forward_close(O, LSE, O_ref, LSE_ref, "attention over a projected slot")
+
+
+@pytest.mark.parametrize("B,T,Dm,Hk,d", [(1, 65536, 2048, 16, 128), (2, 32768, 2048, 32, 64)])
+def test_benchmark_shapes_on_sampled_outputs(B, T, Dm, Hk, d):
+    """The shapes bench.py times (every resident CTA pair takes ~55 work items): sampled positions of every head against
+    fp64 dot products, the slot against the separate append on whole sampled tiles, and nothing written past the tensors."""
+    X, Wk, Wv = make(B, T, Dm, Hk, d, seed=11)
+    cache = moda.alloc_depth_cache(B, T, Hk, d, 1)
+    pad = 4096
+    bufs = [torch.full((pad + B * T * Hk * d + pad,), 3.0, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    K_out, V_out = (bf[pad:pad + B * T * Hk * d].view(B, T, Hk, d) for bf in bufs)
+    moda.moda_kv_project_append(X, Wk, Wv, Hk, cache=cache, slot=0, K_out=K_out, V_out=V_out)
+    assert moda.moda_last_status() == 0
+    for bf in bufs:
+        assert bool((bf[:pad] == 3.0).all()) and bool((bf[-pad:] == 3.0).all()), "guard band overwritten"
+    rng = np.random.default_rng(5)
+    ts = np.unique(np.concatenate([[0, 127, 128, T - 129, T - 128, T - 1], rng.integers(0, T, size=58)]))
+    Wk64, Wv64 = f64(Wk), f64(Wv)
+    for b in range(B):
+        x = f64(X[b, torch.from_numpy(ts).cuda()])                       # [n, Dm]
+        for name, got, W in (("K", K_out, Wk64), ("V", V_out, Wv64)):
+            ref = (x @ W.T).reshape(len(ts), Hk, d)
+            g = f64(got[b, torch.from_numpy(ts).cuda()])
+            assert rel_l2(g, ref) <= TOL_O_REL_L2, f"{name}, b = {b}: rel-L2 {rel_l2(g, ref):.3e}"
+            assert worst_row_rel_l2(g, ref) <= 2e-2, f"{name}, b = {b}: worst row {worst_row_rel_l2(g, ref):.3e}"
+    want = moda.alloc_depth_cache(B, T, Hk, d, 1)
+    moda.moda_depth_cache_append(want, 0, K_out.contiguous(), V_out.contiguous())
+    assert torch.equal(cache, want)

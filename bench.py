@@ -662,12 +662,15 @@ def run_kvproj_sweep(peaks, device, shapes=None, iters=10):
         Wkv = torch.cat([Wk, Wv], 0)
         ms = time_calls(lambda: moda.moda_kv_project_append(X, Wk, Wv, Hk, cache=cache, slot=0, K_out=K, V_out=V), iters)
         ms_slot = time_calls(lambda: moda.moda_kv_project_append(X, Wk, Wv, Hk, cache=cache, slot=0, store_kv=False), iters)
+        cache8 = moda.alloc_depth_cache_e4m3(B, T, Hk, d, 1, device)
+        ms_e4m3 = time_calls(lambda: moda.moda_kv_project_append_e4m3(X, Wk, Wv, Hk, cache=cache8, slot=0, K_out=K, V_out=V), iters)
+        del cache8
         ms_lib = time_calls(lambda: torch.nn.functional.linear(X, Wkv), iters)
         ms_app = time_calls(lambda: moda.moda_depth_cache_append(cache, 0, K, V), iters)
         fl = 2.0 * B * T * Dm * 2 * Hk * d
         rows.append({"B": B, "T": T, "D_model": Dm, "H_kv": Hk, "d": d, "ms": round(ms, 4), "tflops": round(fl / ms / 1e9, 1),
                      "frac_measured_burst_bf16": round(fl / ms / 1e9 / peaks["bf16_tflops"], 4),
-                     "slot_only_ms": round(ms_slot, 4), "library_gemm_ms": round(ms_lib, 4), "separate_append_ms": round(ms_app, 4)})
+                     "slot_only_ms": round(ms_slot, 4), "e4m3_slot_ms": round(ms_e4m3, 4), "library_gemm_ms": round(ms_lib, 4), "separate_append_ms": round(ms_app, 4)})
         log("kvproj_sweep", rows[-1])
         del X, Wk, Wv, Wkv, cache, K, V
     torch.cuda.empty_cache()

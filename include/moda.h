@@ -455,6 +455,16 @@ int moda_kv_project_append(const void* X, const void* Wk, const void* Wv,
                            int B, int T, int D_model, int H_kv, int d,
                            void* K_out, void* V_out, void* cache, int slot, void* stream);
 
+/*
+ * The same projection with the slot written into an e4m3 depth cache (moda_depth_cache_e4m3_bytes(B, T, H_kv, d, .)):
+ * codes and one fp32 scale per row, bit for bit what moda_depth_cache_append_e4m3(cache_e4m3, ..., slot, K_out, V_out)
+ * would store from the bf16-rounded K and V (row maximum / 448 as the scale, IEEE division, round to nearest even,
+ * saturating; a zero row has scale 1).  K_out, V_out stay bf16 and optional.  Everything else as above.
+ */
+int moda_kv_project_append_e4m3(const void* X, const void* Wk, const void* Wv,
+                                int B, int T, int D_model, int H_kv, int d,
+                                void* K_out, void* V_out, void* cache_e4m3, int slot, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,6 +27,7 @@ SYMBOLS = (
     "moda_depth_cache_e4m3_bytes", "moda_depth_cache_append_e4m3", "moda_attn_fwd_e4m3", "moda_attn_bwd_e4m3",
     "moda_depth_cache_append_pm", "moda_depth_cache_unpack_pm", "moda_attn_fwd_gqa_pm", "moda_attn_bwd_gqa_pm",
     "moda_kv_project_append",
+    "moda_kv_project_append_e4m3",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -118,6 +119,8 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd_gqa_pm.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
     lib.moda_kv_project_append.restype = ci
     lib.moda_kv_project_append.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, vp, ci, vp]
+    lib.moda_kv_project_append_e4m3.restype = ci
+    lib.moda_kv_project_append_e4m3.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, vp, ci, vp]
     _lib = lib
     return lib
 
@@ -331,9 +334,11 @@ def moda_attn_bwd_gqa_pm(Q, K, V, depth_kv_pm, O, dO, LSE, l, scale,
     return dQ, dK, dV, d_depth_kv_pm
 
 
-def moda_kv_project_append(X, Wk, Wv, H_kv, cache=None, slot=0, store_kv=True, K_out=None, V_out=None, stream=None):
+def moda_kv_project_append(X, Wk, Wv, H_kv, cache=None, slot=0, store_kv=True, K_out=None, V_out=None, stream=None,
+                           e4m3=False):
     """K, V [B,T,H_kv,d] = X [B,T,D_model] times the key / value projections Wk, Wv [H_kv d, D_model]; with ``cache`` the
-    same launch writes them as depth slot ``slot``.  ``store_kv=False`` (FFN-side projection) writes the slot only."""
+    same launch writes them as depth slot ``slot``.  ``store_kv=False`` (FFN-side projection) writes the slot only.
+    ``e4m3=True``: ``cache`` is an e4m3 cache (alloc_depth_cache_e4m3) and the call is moda_kv_project_append_e4m3."""
     if X.dim() != 3 or X.dtype != torch.bfloat16:
         raise ValueError("X must be a bf16 [B, T, D_model] tensor")
     B, T, Dm = X.shape
@@ -346,9 +351,15 @@ def moda_kv_project_append(X, Wk, Wv, H_kv, cache=None, slot=0, store_kv=True, K
         V_out = _new((B, T, H_kv, d), torch.bfloat16, X.device, stream) if V_out is None else V_out
     else:
         K_out = V_out = None
-    _check(load().moda_kv_project_append(_ptr(X), _ptr(Wk), _ptr(Wv), B, T, Dm, int(H_kv), d, _ptr(K_out), _ptr(V_out),
-                                         _ptr(cache), int(slot), _stream(stream)), "moda_kv_project_append")
+    fn = load().moda_kv_project_append_e4m3 if e4m3 else load().moda_kv_project_append
+    _check(fn(_ptr(X), _ptr(Wk), _ptr(Wv), B, T, Dm, int(H_kv), d, _ptr(K_out), _ptr(V_out),
+              _ptr(cache), int(slot), _stream(stream)), "moda_kv_project_append_e4m3" if e4m3 else "moda_kv_project_append")
     return K_out, V_out
+
+
+def moda_kv_project_append_e4m3(X, Wk, Wv, H_kv, cache=None, slot=0, store_kv=True, K_out=None, V_out=None, stream=None):
+    """moda_kv_project_append with the slot written as e4m3 codes and row scales."""
+    return moda_kv_project_append(X, Wk, Wv, H_kv, cache, slot, store_kv, K_out, V_out, stream, e4m3=True)
 
 
 def moda_attn_fwd(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):

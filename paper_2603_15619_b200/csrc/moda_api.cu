@@ -542,7 +542,7 @@ int launch_cache_pm_copy(void* cache, int B, int T, int H, int slot, void* Xk, v
 }
 
 // Key / value projection with the write step in its epilogue: a persistent kernel on CTA pairs (clusters of two CTAs).
-template <int D, int NH>
+template <int D, int NH, bool FP8 = false>
 int launch_kv_project(const void* X, const void* Wk, const void* Wv, int B, int T, int Dm, int Hk,
                       void* K_out, void* V_out, void* slot, cudaStream_t stream) {
     using L = KvProjSmem<D, NH>;
@@ -554,7 +554,7 @@ int launch_kv_project(const void* X, const void* Wk, const void* Wv, int B, int 
         !make_bthd_map(&mV, V_out ? V_out : X, B, T, V_out ? Hk : Dm / 64, V_out ? D : 64))
         return MODA_ERR_CUDA;
     KvProjParams p;
-    p.slot = static_cast<__nv_bfloat16*>(slot);
+    p.slot = slot;
     p.B = B; p.T = T; p.Hk = Hk; p.Dm = Dm;
     p.store_kv = K_out != nullptr ? 1 : 0;
     const long long items = (long long)B * ((num_tiles(T) + 1) / 2) * (Hk / NH);
@@ -576,16 +576,16 @@ int launch_kv_project(const void* X, const void* Wk, const void* Wv, int B, int 
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return MODA_ERR_CUDA;
     if (configured_dev != dev) {
-        if (!set_smem_limit(moda_kv_project_kernel<D, NH>, L::kDynamic)) return MODA_ERR_CUDA;
+        if (!set_smem_limit(moda_kv_project_kernel<D, NH, FP8>, L::kDynamic)) return MODA_ERR_CUDA;
         int n = 0;
         cfg.gridDim = dim3(1024, 1, 1);                        // any multiple of the cluster size: the query asks what fits
-        if (!cuda_ok(cudaOccupancyMaxActiveClusters(&n, moda_kv_project_kernel<D, NH>, &cfg)) || n < 1) return MODA_ERR_CUDA;
+        if (!cuda_ok(cudaOccupancyMaxActiveClusters(&n, moda_kv_project_kernel<D, NH, FP8>, &cfg)) || n < 1) return MODA_ERR_CUDA;
         resident_pairs = n;
         configured_dev = dev;
     }
     const long long clusters = items < resident_pairs ? items : resident_pairs;
     cfg.gridDim = dim3(unsigned(2 * clusters), 1, 1);
-    return cuda_ok(cudaLaunchKernelEx(&cfg, moda_kv_project_kernel<D, NH>, mX, mWk, mWv, mK, mV, p)) ? MODA_OK : MODA_ERR_CUDA;
+    return cuda_ok(cudaLaunchKernelEx(&cfg, moda_kv_project_kernel<D, NH, FP8>, mX, mWk, mWv, mK, mV, p)) ? MODA_OK : MODA_ERR_CUDA;
 }
 
 // Decode step: a split kernel over the KV cache and a merge kernel that adds the depth pairs.
@@ -685,6 +685,33 @@ int decode_common(const void* q, const void* K, const void* V, const int* seq_le
     return d == 128 ? launch_decode<128>(p, st) : launch_decode<64>(p, st);
 }
 
+}  // namespace
+
+namespace {
+int kv_project_common(const void* X, const void* Wk, const void* Wv, int B, int T, int D_model, int H_kv, int d,
+                      void* K_out, void* V_out, void* cache, int slot, void* stream, bool e4m3) {
+    if (int rc = check_shape(B, T, H_kv, d)) return rc;
+    if (D_model < 64 || D_model % 64 != 0 || (long long)B * T > 0x7fffffffLL / D_model) return MODA_ERR_BAD_SHAPE;
+    if (cache != nullptr && (slot < 0 || slot >= MODA_MAX_DEPTH)) return MODA_ERR_BAD_SLOT;
+    if (!X || !Wk || !Wv || (K_out == nullptr) != (V_out == nullptr) || (!K_out && !cache)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(X) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(K_out) || !aligned16(V_out) || !aligned16(cache))
+        return MODA_ERR_MISALIGNED;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    void* slot_base = nullptr;
+    if (cache)
+        slot_base = e4m3 ? static_cast<void*>(static_cast<uint8_t*>(cache) + size_t(slot) * cache8_slot_bytes(B, T, H_kv, d))
+                         : static_cast<void*>(static_cast<__nv_bfloat16*>(cache) + size_t(slot) * cache_slot_elems(B, T, H_kv, d));
+    // d = 64: two heads per CTA (one tensor-core instruction of 256 columns) when the heads pair up
+    if (e4m3) {
+        if (d == 128) return launch_kv_project<128, 1, true>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
+        return H_kv % 2 == 0 ? launch_kv_project<64, 2, true>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st)
+                             : launch_kv_project<64, 1, true>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
+    }
+    if (d == 128) return launch_kv_project<128, 1>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
+    return H_kv % 2 == 0 ? launch_kv_project<64, 2>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st)
+                         : launch_kv_project<64, 1>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
+}
 }  // namespace
 
 extern "C" {
@@ -1028,19 +1055,13 @@ int moda_attn_bwd_gqa_pm(const void* Q, const void* K, const void* V, const void
 int moda_kv_project_append(const void* X, const void* Wk, const void* Wv,
                            int B, int T, int D_model, int H_kv, int d,
                            void* K_out, void* V_out, void* cache, int slot, void* stream) {
-    if (int rc = check_shape(B, T, H_kv, d)) return rc;
-    if (D_model < 64 || D_model % 64 != 0 || (long long)B * T > 0x7fffffffLL / D_model) return MODA_ERR_BAD_SHAPE;
-    if (cache != nullptr && (slot < 0 || slot >= MODA_MAX_DEPTH)) return MODA_ERR_BAD_SLOT;
-    if (!X || !Wk || !Wv || (K_out == nullptr) != (V_out == nullptr) || (!K_out && !cache)) return MODA_ERR_NULL_POINTER;
-    if (!aligned16(X) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(K_out) || !aligned16(V_out) || !aligned16(cache))
-        return MODA_ERR_MISALIGNED;
-    if (int rc = check_device()) return rc;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    void* slot_base = cache ? static_cast<__nv_bfloat16*>(cache) + size_t(slot) * cache_slot_elems(B, T, H_kv, d) : nullptr;
-    if (d == 128) return launch_kv_project<128, 1>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
-    // d = 64: two heads per CTA (one tensor-core instruction of 256 columns) when the heads pair up
-    return H_kv % 2 == 0 ? launch_kv_project<64, 2>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st)
-                         : launch_kv_project<64, 1>(X, Wk, Wv, B, T, D_model, H_kv, K_out, V_out, slot_base, st);
+    return kv_project_common(X, Wk, Wv, B, T, D_model, H_kv, d, K_out, V_out, cache, slot, stream, false);
+}
+
+int moda_kv_project_append_e4m3(const void* X, const void* Wk, const void* Wv,
+                                int B, int T, int D_model, int H_kv, int d,
+                                void* K_out, void* V_out, void* cache_e4m3, int slot, void* stream) {
+    return kv_project_common(X, Wk, Wv, B, T, D_model, H_kv, d, K_out, V_out, cache_e4m3, slot, stream, true);
 }
 
 size_t moda_decode_workspace_bytes(int B, int H, int d) {

@@ -42,7 +42,7 @@ namespace moda {
 constexpr int kProjThreads = 192;
 
 struct KvProjParams {
-    __nv_bfloat16* slot;       // base of the cache slot to write (row-interleaved layout, H_k heads), or null
+    void* slot;                // base of the cache slot to write (row-interleaved bf16 layout, or e4m3 codes + row scales; H_k heads), or null
     int B, T, Hk, Dm;          // Dm = input features (a multiple of 64)
     int store_kv;              // nonzero: K and V are also stored as [B][T][H_k][d] tensors
 };
@@ -67,7 +67,10 @@ struct KvProjSmem {
     static_assert(kDynamic <= 232448, "shared-memory plan does not fit");
 };
 
-template <int D, int NH>
+// FP8: the slot is written in the e4m3 layout (moda_cache.cuh): a thread owns a whole row of a head, so it takes the
+// row's largest magnitude (of the values rounded to bf16, which is what K and V are) in a first pass over its
+// accumulator columns, then scale = max / 448 and the codes in a second pass: the arithmetic of depth_cache_quant_kernel.
+template <int D, int NH, bool FP8 = false>
 __global__ void __launch_bounds__(kProjThreads, 1)
 moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapWk,
                             const __grid_constant__ CUtensorMap mapWv, const __grid_constant__ CUtensorMap mapK,
@@ -209,24 +212,61 @@ moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_co
                 }
 #pragma unroll
                 for (int j = 0; j < NH; ++j) {
+                    const size_t blk_index = ((size_t(b) * p.Hk + hk0 + j) * nt + tile) * 2 + kv;
                     uint4* slot_blk = (p.slot == nullptr || !live) ? nullptr
-                                      : reinterpret_cast<uint4*>(p.slot) + (((size_t(b) * p.Hk + hk0 + j) * nt + tile) * 2 + kv) * (kTileRows * CH) + r;
+                                      : FP8 ? reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.slot) + blk_index * cache8_block_bytes(D)) + r
+                                            : reinterpret_cast<uint4*>(p.slot) + blk_index * (kTileRows * CH) + r;
                     uint8_t* stage = smem + L::kOut + j * (kTileRows * D * 2);
+                    float q_scale = 1.f;
+                    if constexpr (FP8) {
+                        float am = 0.f;
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t a[32];
+                            tmem_ld32(tmem + lane_addr + set * 2 * NW + kv * NW + j * D + c * 32, a);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; i += 2) {
+                                const uint32_t w = pack_bf16x2(__uint_as_float(a[i]), __uint_as_float(a[i + 1]));
+                                am = fmaxf(am, fmaxf(fabsf(bf16_lo_to_f32(w)), fabsf(bf16_hi_to_f32(w))));
+                            }
+                        }
+                        q_scale = am > 0.f ? __fdiv_rn(am, 448.f) : 1.f;
+                        if (slot_blk != nullptr)
+                            reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(slot_blk - r) + size_t(kTileRows) * D)[r] = q_scale;
+                    }
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t a[32];
                         tmem_ld32(tmem + lane_addr + set * 2 * NW + kv * NW + j * D + c * 32, a);
                         tmem_wait_ld();
+                        uint32_t w[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) w[i] = pack_bf16x2(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
+                        if constexpr (FP8) {
+                            // 16 features per 16-byte chunk of codes
+#pragma unroll
+                            for (int g = 0; g < 2; ++g) {
+                                uint32_t cw[4];
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    const uint32_t w0 = w[8 * g + 2 * k], w1 = w[8 * g + 2 * k + 1];
+                                    uint16_t lo, hi;
+                                    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo)
+                                        : "f"(__fdiv_rn(bf16_hi_to_f32(w0), q_scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w0), q_scale)));
+                                    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi)
+                                        : "f"(__fdiv_rn(bf16_hi_to_f32(w1), q_scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w1), q_scale)));
+                                    cw[k] = uint32_t(lo) | (uint32_t(hi) << 16);
+                                }
+                                if (slot_blk != nullptr) slot_blk[(c * 2 + g) * kTileRows] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+                            }
+                        }
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {
-                            uint4 v;
-                            v.x = pack_bf16x2(__uint_as_float(a[8 * g + 0]), __uint_as_float(a[8 * g + 1]));
-                            v.y = pack_bf16x2(__uint_as_float(a[8 * g + 2]), __uint_as_float(a[8 * g + 3]));
-                            v.z = pack_bf16x2(__uint_as_float(a[8 * g + 4]), __uint_as_float(a[8 * g + 5]));
-                            v.w = pack_bf16x2(__uint_as_float(a[8 * g + 6]), __uint_as_float(a[8 * g + 7]));
+                            const uint4 v = make_uint4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
                             const int chunk = c * 4 + g;
                             // rows past T were loaded as zeros: the cache wants exactly that in its tail rows
-                            if (slot_blk != nullptr) slot_blk[chunk * kTileRows] = v;
+                            if (!FP8 && slot_blk != nullptr) slot_blk[chunk * kTileRows] = v;
                             if (p.store_kv) *reinterpret_cast<uint4*>(stage + swz_chunk_offset(r, chunk)) = v;
                         }
                     }

@@ -181,12 +181,13 @@ def test_softmax_scale_must_be_usable():
 def test_kv_projection_entry_point_validates_before_touching_the_device():
     lib = binding.load()
     p, odd = ctypes.c_void_p(4096), ctypes.c_void_p(4100)
-    call = lambda X=p, Wk=p, Wv=p, B=1, T=128, Dm=256, Hk=2, d=64, K=p, V=p, cache=p, slot=0: \
-        lib.moda_kv_project_append(X, Wk, Wv, B, T, Dm, Hk, d, K, V, cache, slot, None)
-    assert call(Dm=100) == -3 and call(Dm=0) == -3 and call(T=0) == -3
-    assert call(d=96) == -4
-    assert call(slot=256) == -6 and call(slot=-1) == -6
-    assert call(X=None) == -1 and call(Wv=None) == -1
-    assert call(K=None) == -1                       # K and V outputs come together
-    assert call(K=None, V=None, cache=None) == -1   # nothing to write
-    assert call(Wk=odd) == -2 and call(cache=odd) == -2
+    for fn in (lib.moda_kv_project_append, lib.moda_kv_project_append_e4m3):
+        call = lambda X=p, Wk=p, Wv=p, B=1, T=128, Dm=256, Hk=2, d=64, K=p, V=p, cache=p, slot=0: \
+            fn(X, Wk, Wv, B, T, Dm, Hk, d, K, V, cache, slot, None)
+        assert call(Dm=100) == -3 and call(Dm=0) == -3 and call(T=0) == -3
+        assert call(d=96) == -4
+        assert call(slot=256) == -6 and call(slot=-1) == -6
+        assert call(X=None) == -1 and call(Wv=None) == -1
+        assert call(K=None) == -1                       # K and V outputs come together
+        assert call(K=None, V=None, cache=None) == -1   # nothing to write
+        assert call(Wk=odd) == -2 and call(cache=odd) == -2

@@ -110,3 +110,32 @@ def test_benchmark_shapes_on_sampled_outputs(B, T, Dm, Hk, d):
     want = moda.alloc_depth_cache(B, T, Hk, d, 1)
     moda.moda_depth_cache_append(want, 0, K_out.contiguous(), V_out.contiguous())
     assert torch.equal(cache, want)
+
+
+@pytest.mark.parametrize("B,T,Dm,Hk,d", [(1, 128, 64, 1, 64), (2, 300, 256, 2, 128), (1, 1000, 512, 3, 64), (3, 257, 320, 4, 64),
+                                         (3, 2500, 128, 8, 128), (2, 2700, 64, 7, 64)])
+def test_e4m3_slot_written_by_the_projection(B, T, Dm, Hk, d):
+    """The slot in the e4m3 layout: codes and row scales are the oracle's quantiser applied to the bf16 K, V the same
+    launch stores, byte for byte what the separate quantising append writes (tail rows: code 0, scale 1)."""
+    from test_gpu_e4m3_cache import unpack_cache8
+    X, Wk, Wv = make(B, T, Dm, Hk, d, seed=13)
+    X[0, min(5, T - 1), :] = 0                                           # a zero row: scale 1, codes 0
+    cache = moda.alloc_depth_cache_e4m3(B, T, Hk, d, 2)
+    cache.fill_(0xAB)
+    K_out, V_out = moda.moda_kv_project_append_e4m3(X, Wk, Wv, Hk, cache=cache, slot=1)
+    assert moda.moda_last_status() == 0
+    K_ref, V_ref = orc.project_kv(f64(X), f64(Wk), f64(Wv), Hk)
+    assert rel_l2(f64(K_out), K_ref) <= TOL_O_REL_L2 and rel_l2(f64(V_out), V_ref) <= TOL_O_REL_L2
+    want = moda.alloc_depth_cache_e4m3(B, T, Hk, d, 2)
+    want.fill_(0xAB)
+    moda.moda_depth_cache_append_e4m3(want, 1, K_out, V_out)
+    assert torch.equal(cache, want)
+    codes, scales = unpack_cache8(cache, 2, B, T, Hk, d)
+    for kv, Y in enumerate((K_out, V_out)):
+        ref_codes, ref_scale = orc.quantize_e4m3_rows(f64(Y))
+        assert np.array_equal(scales[1, kv, :, :T], ref_scale) and np.array_equal(codes[1, kv, :, :T], ref_codes)
+    # slot only (an FFN-side write): the same bytes without the K, V tensors
+    only = moda.alloc_depth_cache_e4m3(B, T, Hk, d, 2)
+    only.fill_(0xAB)
+    assert moda.moda_kv_project_append_e4m3(X, Wk, Wv, Hk, cache=only, slot=1, store_kv=False) == (None, None)
+    assert torch.equal(only, cache)

@@ -389,3 +389,32 @@ def project_kv(X, Wk, Wv, H_k):
     K = np.matmul(X, Wk.T).reshape(B, T, H_k, n // H_k)
     V = np.matmul(X, Wv.T).reshape(B, T, H_k, n // H_k)
     return K, V
+
+
+# ---------------------------------------------------------------------------------------
+# Attention mass on the depth slots (Sec. 2.2: the probabilities of the one softmax over sequence and depth keys;
+# the paper's attention analysis looks at how much probability heads give to depth slots, and its discussion of a
+# bounded slot buffer keeps the entries of highest utility).  For slot i of query head hq:
+#     mass[b, hq, i] = sum_t  exp( scale <q_t, kd_i[t]> - LSE_t )
+# i.e. the depth probabilities R_i(t) of the definition, summed over the positions.  LSE is the operator's own
+# output (forward / forward_gqa), so the sequence keys enter only through it.  Plain numpy float64.
+# ---------------------------------------------------------------------------------------
+def depth_slot_mass(Q, Kd, LSE, scale):
+    """mass [B, Hq, l] from Q [B, T, Hq, d], depth keys Kd [l, B, T, Hk, d] and LSE [B, Hq, T] (float64)."""
+    Q = np.asarray(Q, dtype=np.float64)
+    Kd = np.asarray(Kd, dtype=np.float64)
+    LSE = np.asarray(LSE, dtype=np.float64)
+    B, T, Hq, d = Q.shape
+    l = Kd.shape[0]
+    Hk = Kd.shape[3] if l else 1
+    if l and (Kd.shape != (l, B, T, Hk, d) or Hq % Hk):
+        raise ValueError("Kd must be [l, B, T, Hk, d] with Hk dividing Hq")
+    if LSE.shape != (B, Hq, T):
+        raise ValueError("LSE must be [B, Hq, T]")
+    mass = np.zeros((B, Hq, l))
+    G = Hq // Hk
+    for hq in range(Hq):
+        for i in range(l):
+            u = scale * np.einsum("btd,btd->bt", Q[:, :, hq, :], Kd[i, :, :, hq // G, :])      # [B, T]
+            mass[:, hq, i] = np.exp(u - LSE[:, hq, :]).sum(axis=1)
+    return mass

@@ -465,6 +465,25 @@ int moda_kv_project_append_e4m3(const void* X, const void* Wk, const void* Wv,
                                 int B, int T, int D_model, int H_kv, int d,
                                 void* K_out, void* V_out, void* cache_e4m3, int slot, void* stream);
 
+/*
+ * Attention mass on the depth slots (Sec. 2.2: the probabilities of the single softmax; the paper's attention analysis
+ * reports the probability that heads give to depth slots, and its bounded slot buffer keeps the entries of highest
+ * utility, for which this is the operator's own measure):
+ *
+ *     mass[b, h, i] = sum_t exp( scale <Q[b,t,h,:], Kd_i[b,t,h / G,:]> - LSE[b,h,t] )      i = 0 .. l-1
+ *
+ *     Q, LSE       : as passed to / returned by the forward call whose probabilities are meant
+ *     depth_kv     : the row-interleaved bf16 cache of H_kv heads that call read (>= l slots)
+ *     mass         : fp32 [B][H][l], written (the sum over the slots plus the sequence keys' mass is T per (b, h))
+ *     workspace    : moda_depth_slot_mass_workspace_bytes(B, T, H, l) bytes of scratch (partial sums per query tile)
+ * fp32 dot products of the bf16 inputs, sums in a fixed order (bit-reproducible).  Two launches on `stream`; l == 0
+ * returns MODA_OK without touching anything.  Validation, asynchrony and error codes as for the other calls.
+ */
+size_t moda_depth_slot_mass_workspace_bytes(int B, int T, int H, int l);
+int moda_depth_slot_mass(const void* Q, const void* depth_kv, const float* LSE,
+                         int B, int T, int H, int H_kv, int d, int l, float scale,
+                         float* mass, void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

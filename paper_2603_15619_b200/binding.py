@@ -28,6 +28,8 @@ SYMBOLS = (
     "moda_depth_cache_append_pm", "moda_depth_cache_unpack_pm", "moda_attn_fwd_gqa_pm", "moda_attn_bwd_gqa_pm",
     "moda_kv_project_append",
     "moda_kv_project_append_e4m3",
+    "moda_depth_slot_mass_workspace_bytes",
+    "moda_depth_slot_mass",
 )
 MODA_STATIC_SCRATCH_ROWS = 1 << 20
 MODA_BWD_STAGE_ROWTERMS, MODA_BWD_STAGE_DQ, MODA_BWD_STAGE_DKDV, MODA_BWD_ALL_STAGES = 1, 2, 4, 7
@@ -119,6 +121,10 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_bwd_gqa_pm.argtypes = [vp] * 7 + [ci] * 6 + [cf] + [vp] * 5 + [sz, vp]
     lib.moda_kv_project_append.restype = ci
     lib.moda_kv_project_append.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, vp, ci, vp]
+    lib.moda_depth_slot_mass_workspace_bytes.restype = ctypes.c_size_t
+    lib.moda_depth_slot_mass_workspace_bytes.argtypes = [ci, ci, ci, ci]
+    lib.moda_depth_slot_mass.restype = ci
+    lib.moda_depth_slot_mass.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, ctypes.c_float, vp, vp, ctypes.c_size_t, vp]
     lib.moda_kv_project_append_e4m3.restype = ci
     lib.moda_kv_project_append_e4m3.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, vp, ci, vp]
     _lib = lib
@@ -360,6 +366,22 @@ def moda_kv_project_append(X, Wk, Wv, H_kv, cache=None, slot=0, store_kv=True, K
 def moda_kv_project_append_e4m3(X, Wk, Wv, H_kv, cache=None, slot=0, store_kv=True, K_out=None, V_out=None, stream=None):
     """moda_kv_project_append with the slot written as e4m3 codes and row scales."""
     return moda_kv_project_append(X, Wk, Wv, H_kv, cache, slot, store_kv, K_out, V_out, stream, e4m3=True)
+
+
+def moda_depth_slot_mass(Q, depth_kv, LSE, l, scale, H_kv=None, mass=None, workspace=None, stream=None):
+    """mass [B,H,l] fp32: the probability that the rows of every query head give to each depth slot, summed over the
+    positions (Q and LSE of the forward call; the bf16 row-interleaved cache it read)."""
+    B, T, H, d = _bthd(Q, "Q")
+    H_kv = H if H_kv is None else int(H_kv)
+    if mass is None:
+        mass = _new((B, H, int(l)), torch.float32, Q.device, stream)
+    need = int(load().moda_depth_slot_mass_workspace_bytes(B, T, H, int(l)))
+    if workspace is None:
+        workspace = _new((max(need, 16),), torch.uint8, Q.device, stream)
+    _check(load().moda_depth_slot_mass(_ptr(Q), _ptr(depth_kv) if l > 0 else None, _ptr(LSE), B, T, H, H_kv, d, int(l),
+                                       float(scale), _ptr(mass), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                       _stream(stream)), "moda_depth_slot_mass")
+    return mass
 
 
 def moda_attn_fwd(Q, K, V, depth_kv, l, scale, O=None, LSE=None, stream=None):

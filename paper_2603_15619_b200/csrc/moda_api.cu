@@ -13,6 +13,7 @@
 #include "moda_depth_gqa.cuh"
 #include "moda_fwd.cuh"
 #include "moda_fwd_wide.cuh"
+#include "moda_mass.cuh"
 #include "moda_kvproj.cuh"
 #include "sm100_ptx.cuh"
 
@@ -1062,6 +1063,42 @@ int moda_kv_project_append_e4m3(const void* X, const void* Wk, const void* Wv,
                                 int B, int T, int D_model, int H_kv, int d,
                                 void* K_out, void* V_out, void* cache_e4m3, int slot, void* stream) {
     return kv_project_common(X, Wk, Wv, B, T, D_model, H_kv, d, K_out, V_out, cache_e4m3, slot, stream, true);
+}
+
+size_t moda_depth_slot_mass_workspace_bytes(int B, int T, int H, int l) {
+    if (B < 1 || T < 1 || H < 1 || l < 0 || l > MODA_MAX_DEPTH) return 0;
+    return size_t(B) * H * num_tiles(T) * size_t(l > 0 ? l : 1) * sizeof(float);
+}
+
+int moda_depth_slot_mass(const void* Q, const void* depth_kv, const float* LSE,
+                         int B, int T, int H, int H_kv, int d, int l, float scale,
+                         float* mass, void* workspace, size_t workspace_bytes, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
+    if (H_kv < 1 || H % H_kv != 0) return MODA_ERR_BAD_GROUP;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (l == 0) return MODA_OK;                    // no slots: nothing to write
+    if (!Q || !depth_kv || !LSE || !mass) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(depth_kv) || !aligned16(LSE) || !aligned16(mass)) return MODA_ERR_MISALIGNED;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < moda_depth_slot_mass_workspace_bytes(B, T, H, l))
+        return MODA_ERR_WORKSPACE;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    MassParams p;
+    p.Q = static_cast<const __nv_bfloat16*>(Q);
+    p.depth_kv = static_cast<const __nv_bfloat16*>(depth_kv);
+    p.LSE = LSE;
+    p.partial = static_cast<float*>(workspace);
+    p.mass = mass;
+    p.B = B; p.T = T; p.H = H; p.G = H / H_kv; p.l = l;
+    p.scale_log2 = scale * kLog2e;
+    const unsigned grid = unsigned(B) * H * num_tiles(T);
+    if (d == 128) depth_slot_mass_kernel<128><<<grid, kTileRows * 4, 0, st>>>(p);
+    else depth_slot_mass_kernel<64><<<grid, kTileRows * 2, 0, st>>>(p);
+    if (!cuda_ok(cudaGetLastError())) return MODA_ERR_CUDA;
+    const long long n = (long long)B * H * l;
+    depth_slot_mass_reduce_kernel<<<unsigned((n + 255) / 256), 256, 0, st>>>(p);
+    return cuda_ok(cudaGetLastError()) ? MODA_OK : MODA_ERR_CUDA;
 }
 
 size_t moda_decode_workspace_bytes(int B, int H, int d) {

@@ -191,3 +191,17 @@ def test_kv_projection_entry_point_validates_before_touching_the_device():
         assert call(K=None) == -1                       # K and V outputs come together
         assert call(K=None, V=None, cache=None) == -1   # nothing to write
         assert call(Wk=odd) == -2 and call(cache=odd) == -2
+
+
+def test_slot_mass_entry_point_validates_before_touching_the_device():
+    lib = binding.load()
+    p, odd = ctypes.c_void_p(4096), ctypes.c_void_p(4100)
+    need = lib.moda_depth_slot_mass_workspace_bytes(1, 300, 4, 5)
+    assert need == 1 * 4 * 3 * 5 * 4 and lib.moda_depth_slot_mass_workspace_bytes(1, 300, 4, 257) == 0
+    call = lambda Q=p, cache=p, LSE=p, B=1, T=300, H=4, Hk=2, d=64, l=5, scale=0.1, mass=p, ws=p, wsb=need: \
+        lib.moda_depth_slot_mass(Q, cache, LSE, B, T, H, Hk, d, l, ctypes.c_float(scale), mass, ws, ctypes.c_size_t(wsb), None)
+    assert call(T=0) == -3 and call(d=96) == -4 and call(l=257) == -5 and call(Hk=3) == -12 and call(scale=0.0) == -13
+    assert call(l=0, cache=None, mass=None, ws=None, wsb=0) == 0          # no slots: nothing to do
+    assert call(Q=None) == -1 and call(mass=None) == -1 and call(cache=None) == -1
+    assert call(LSE=odd) == -2
+    assert call(ws=None) == -7 and call(wsb=need - 1) == -7

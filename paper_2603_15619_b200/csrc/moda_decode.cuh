@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kDecodeTmaThreads, 1)
 decode_split_tma_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                         const DecodeParams p) {
     using L = DecodeSmem<D, G>;
-    constexpr int CH = D / 8, FPL = D / 32, NH = D / 64;                     // NH 64-feature boxes per row
+    constexpr int CH = D / 8, NH = D / 64;                                    // NH 64-feature boxes per row
     constexpr int kBoxBytes = kDecodeStageKeys * 128;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));

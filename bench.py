@@ -347,6 +347,8 @@ def run_moda(args, rank, world, device):
             out["prefill_sweep"] = run_prefill_sweep(peaks, device)
         if "kvproj" in extra:
             out["kvproj_sweep"] = run_kvproj_sweep(peaks, device)
+        if "mass" in extra:
+            out["mass_sweep"] = run_mass_sweep(peaks, device)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, budget_s=20.0)
     return out
@@ -677,6 +679,33 @@ def run_kvproj_sweep(peaks, device, shapes=None, iters=10):
     return rows
 
 
+def run_mass_sweep(peaks, device, names=("c3_l32", "c4", "c5"), batch=0, iters=10):
+    """Attention mass of the depth slots (moda_depth_slot_mass): one pass over the depth keys; bytes = l E + E."""
+    import dataclasses
+    import paper_2603_15619_b200 as moda
+    rows = []
+    for nm in names:
+        w = synthetic.WORKLOADS[nm.split("_")[0]]
+        if "_l" in nm:
+            w = w.with_l(int(nm.split("_l")[1]))
+        if batch:
+            w = dataclasses.replace(w, B=batch)
+        torch.cuda.empty_cache()
+        L = Layer(w, 0, device, with_backward=False)
+        L.fwd()
+        mass = torch.empty((w.B, w.H, w.l), dtype=torch.float32, device=device)
+        ws = torch.empty((max(16, moda.binding.load().moda_depth_slot_mass_workspace_bytes(w.B, w.T, w.H, w.l)),), dtype=torch.uint8, device=device)
+        ms = time_calls(lambda: moda.moda_depth_slot_mass(L.q, L.cache, L.LSE, w.l, w.scale, mass=mass, workspace=ws), iters)
+        byts = (w.l + 1) * w.B * w.T * w.H * w.d * 2
+        rows.append({"workload": nm, "B": w.B, "ms": round(ms, 4), "gbs": round(byts / ms / 1e6, 1),
+                     "frac_measured_copy": round(byts / ms / 1e6 / peaks["hbm_gbs"], 4),
+                     "depth_share_of_probability": round(float(mass.sum()) / (w.B * w.H * w.T), 5)})
+        log("mass_sweep", rows[-1])
+        del L, mass, ws
+    torch.cuda.empty_cache()
+    return rows
+
+
 def run_e2e(layer, steps, world, step_flops, device):
     """The same step driven from pinned HOST buffers: every step copies its inputs host->device and
     its results device->host inside the timed region.  Two device buffer sets and three streams let
@@ -833,7 +862,7 @@ def main():
     ap.add_argument("--impl", default="moda", choices=["moda", "reference"])
     ap.add_argument("--workload", default="c4", help="c1..c5, optionally with _l<depth> (e.g. c3_l8)")
     ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the host-to-host leg (each moves every input and output over PCIe)")
-    ap.add_argument("--sweeps", default="", help="comma list of extra sweeps printed in the line: gqa, decode, prefill, kvproj")
+    ap.add_argument("--sweeps", default="", help="comma list of extra sweeps printed in the line: gqa, decode, prefill, kvproj, mass")
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (smaller profiling cases)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -841,6 +870,8 @@ def main():
     ap.add_argument("--gqa-shape", default="", help="T,G[,L]: time only this grouped-query shape (B=1, d=64, 8 key/value "
                                                     "heads, L depth slots (default 32) and l=0) and print its row; for profiling")
     ap.add_argument("--prefill-sweep", action="store_true", help="time only the prefill-with-cache shapes and print their rows")
+    ap.add_argument("--mass-workload", default="", help="comma list of workloads (c3_l32, c4, ...): time only the depth-slot attention "
+                    "mass on them and print its rows; --batch overrides B; for profiling")
     ap.add_argument("--kvproj-shape", default="", help="B,T,D_model,H_kv,d (or 'all'): time only the key/value projection with the "
                     "write step in its epilogue and print its rows; for profiling")
     ap.add_argument("--decode-shape", default="", help="B,T_kv,H,H_kv,d,l: time only this decode step and print its row; for profiling")
@@ -873,6 +904,9 @@ def main():
             out = {"gqa_sweep": run_gqa_sweep(device, [(v[0], v[1], v[2] if len(v) > 2 else 32, None)])}
         elif args.prefill_sweep:
             out = {"prefill_sweep": run_prefill_sweep(load_peaks(), device)}
+        elif args.mass_workload:
+            out = {"mass_sweep": run_mass_sweep(load_peaks(), device, tuple(args.mass_workload.split(",")), args.batch,
+                                                iters=max(1, min(args.steps, 20)))}
         elif args.kvproj_shape:
             v = args.kvproj_shape
             shapes = None if v == "all" else [tuple(int(t) for t in v.split(","))]

@@ -65,3 +65,43 @@ def test_top_slots_by_mass_are_the_slots_that_matter():
     assert top == {1, 3}
     assert float(mass[:, :, [1, 3]].sum()) > 0.9 * float(mass.sum())
     assert float(mass.sum()) < B * H * T
+
+
+def test_bounded_slot_buffer_driven_by_the_mass_keeps_the_useful_layers():
+    """Six layers through a buffer of four slots with the top-S policy: every layer attends to the layers the buffer
+    holds (checked against the oracle on exactly those layers), writes its K, V over the slot of least attention mass,
+    and the two layers whose keys the queries look for survive to the end."""
+    from paper_2603_15619_b200.slots import SlotBuffer
+    from parity import assert_forward_close
+    B, T, H, d, S, n_layers = 1, 300, 2, 64, 4, 6
+    scale = d ** -0.5
+    g = torch.Generator(device="cuda").manual_seed(9)
+    base = torch.randn((B, T, H, d), device="cuda", generator=g)
+    layers = []
+    for n in range(n_layers):
+        Q = (base + 0.3 * torch.randn((B, T, H, d), device="cuda", generator=g)).to(torch.bfloat16)
+        # layers 0 and 2 write keys that later queries align with; the others write small random keys
+        K = (base if n in (0, 2) else 0.1 * torch.randn((B, T, H, d), device="cuda", generator=g)).to(torch.bfloat16)
+        V = torch.randn((B, T, H, d), device="cuda", generator=g).to(torch.bfloat16)
+        layers.append((Q, K, V))
+    cache = moda.alloc_depth_cache(B, T, H, d, S)
+    buf = SlotBuffer(S, policy="top")
+    utility = None
+    for n, (Q, K, V) in enumerate(layers):
+        l = buf.filled
+        held = list(buf.layers())                                   # slot order
+        slot = buf.next_slot(utility)
+        O, LSE = moda.moda_attn_fwd_append(Q, K, V, cache, l, scale, cache, slot)
+        assert moda.moda_last_status() == 0
+        Kd = np.stack([f64(layers[m][1]) for m in held]) if held else np.zeros((0, B, T, H, d))
+        Vd = np.stack([f64(layers[m][2]) for m in held]) if held else np.zeros((0, B, T, H, d))
+        assert_forward_close(O, LSE, *orc.forward(f64(Q), f64(K), f64(V), Kd, Vd, scale), f"layer {n} over layers {held}")
+        # utility of the slots this layer read (the one just overwritten holds a new layer nobody has attended to yet)
+        utility = [float("inf")] * S
+        if l > 0:
+            mass = moda.moda_depth_slot_mass(Q, cache, LSE, l, scale).sum(dim=(0, 1)).tolist()
+            utility[:l] = mass
+        utility[slot] = float("inf")
+        buf.record(slot, n)
+    # the newest layer is always kept (nobody has attended to it yet); of the rest, the low-mass layers 1 and 3 went
+    assert sorted(buf.layers()) == [0, 2, 4, 5]

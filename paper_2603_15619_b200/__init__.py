@@ -5,7 +5,7 @@
 reported metric.  The CUDA library is loaded on first use and there is no fallback path.
 """
 from .autograd import moda_attention  # noqa: F401
-from .stack import DepthStream
+from .stack import DepthStream  # noqa: F401
 from .slots import SlotBuffer  # noqa: F401
 from .binding import (  # noqa: F401
     MODA_BWD_ACCUMULATE_DEPTH,

@@ -363,6 +363,16 @@ int moda_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, co
                                  void* dQ, void* dK, void* dV, void* d_depth_kv, void* stream);
 
 /*
+ * moda_attn_fwd_e4m3 that also writes the layer's own K, V as slot `append_slot` of an e4m3 cache, from the key / value
+ * tiles the kernel holds (the write step of Sec. 2.2 fused into the forward, as moda_attn_fwd_append does for a bf16
+ * cache).  The slot receives byte for byte what moda_depth_cache_append_e4m3(append_cache_e4m3, ..., append_slot, K, V)
+ * stores.  Rules for writing a slot that the call also reads as in moda_attn_fwd_append.
+ */
+int moda_attn_fwd_append_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,
+                              int B, int T, int H, int H_kv, int d, int l, float scale,
+                              void* O, float* LSE, void* append_cache_e4m3, int append_slot, void* stream);
+
+/*
  * ---- Depth cache in e4m3 with one scale per row ----
  *
  * The paper's Discussion names the growing depth-KV cache as the cost to cut next and gives no

@@ -46,6 +46,7 @@ from .binding import (  # noqa: F401
     moda_depth_cache_unpack_pm,
     moda_kv_project_append,
     moda_kv_project_append_e4m3,
+    moda_attn_fwd_append_e4m3,
     moda_depth_slot_mass,
     moda_last_status,
     moda_selftest_wait_timeout,

@@ -28,6 +28,7 @@ SYMBOLS = (
     "moda_depth_cache_append_pm", "moda_depth_cache_unpack_pm", "moda_attn_fwd_gqa_pm", "moda_attn_bwd_gqa_pm",
     "moda_kv_project_append",
     "moda_kv_project_append_e4m3",
+    "moda_attn_fwd_append_e4m3",
     "moda_depth_slot_mass_workspace_bytes",
     "moda_depth_slot_mass",
 )
@@ -87,6 +88,8 @@ def load() -> ctypes.CDLL:
     lib.moda_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp]
     lib.moda_attn_fwd_append.restype = ci
     lib.moda_attn_fwd_append.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, ci, vp]
+    lib.moda_attn_fwd_append_e4m3.restype = ci
+    lib.moda_attn_fwd_append_e4m3.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp, vp, ci, vp]
     lib.moda_bwd_workspace_bytes_gqa.restype = sz
     lib.moda_bwd_workspace_bytes_gqa.argtypes = [ci] * 6
     lib.moda_attn_bwd_gqa.restype = ci
@@ -271,6 +274,20 @@ def moda_attn_fwd_e4m3(Q, K, V, depth_kv_e4m3, l, scale, O=None, LSE=None, strea
     _check(load().moda_attn_fwd_e4m3(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv_e4m3) if l > 0 else None,
                                      B, T, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE), _stream(stream)),
            "moda_attn_fwd_e4m3")
+    return O, LSE
+
+
+def moda_attn_fwd_append_e4m3(Q, K, V, depth_kv_e4m3, l, scale, append_cache_e4m3, append_slot, O=None, LSE=None, stream=None):
+    """moda_attn_fwd_e4m3 that also quantises K, V into slot ``append_slot`` of an e4m3 cache in the same launch."""
+    B, T, H, Hk, d = _gqa_shapes(Q, K, V)
+    if O is None:
+        O = _new_like(Q, stream)
+    if LSE is None:
+        LSE = _new((B, H, T), torch.float32, Q.device, stream)
+    _check(load().moda_attn_fwd_append_e4m3(_ptr(Q), _ptr(K), _ptr(V), _ptr(depth_kv_e4m3) if l > 0 else None,
+                                            B, T, H, Hk, d, int(l), float(scale), _ptr(O), _ptr(LSE),
+                                            _ptr(append_cache_e4m3), int(append_slot), _stream(stream)),
+           "moda_attn_fwd_append_e4m3")
     return O, LSE
 
 

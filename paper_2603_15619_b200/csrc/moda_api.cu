@@ -263,7 +263,7 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     p.T_kv = T_kv; p.kv_off = T_kv - T;
     p.G = H / Hk;
     p.scale_log2 = scale * kLog2e;
-    p.append_slot = static_cast<__nv_bfloat16*>(append_slot);
+    p.append_slot = append_slot;
     // The d = 128 kernel takes a pair of query tiles per CTA when the call is causal over equally many keys and queries
     // (the pairs then have equal work) and the equal-sized CTAs fill their last wave (at least 93 % of the SM slots of
     // all waves; 512 pairs on 148 SMs would idle a seventh of them, measured + 4 % at c3 with B = 1), or when the depth
@@ -956,6 +956,27 @@ int moda_attn_fwd_e4m3(const void* Q, const void* K, const void* V, const void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, kCacheE4m3)
                     : launch_fwd<64>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, nullptr, st, kCacheE4m3);
+}
+
+int moda_attn_fwd_append_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,
+                              int B, int T, int H, int H_kv, int d, int l, float scale,
+                              void* O, float* LSE, void* append_cache_e4m3, int append_slot, void* stream) {
+    if (int rc = check_shape(B, T, H, d)) return rc;
+    if (int rc = check_scale(scale)) return rc;
+    if (int rc = check_groups(H, H_kv)) return rc;
+    if (l < 0 || l > MODA_MAX_DEPTH) return MODA_ERR_BAD_DEPTH;
+    if (append_slot < 0 || append_slot >= MODA_MAX_DEPTH) return MODA_ERR_BAD_SLOT;
+    if (!Q || !K || !V || !O || !LSE || !append_cache_e4m3 || (l > 0 && !depth_kv_e4m3)) return MODA_ERR_NULL_POINTER;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE) || !aligned16(append_cache_e4m3) ||
+        (l > 0 && !aligned16(depth_kv_e4m3)))
+        return MODA_ERR_MISALIGNED;
+    // as in moda_attn_fwd_append: a slot that the call also reads may be written only with one key/value head per query head
+    if (l > 0 && append_cache_e4m3 == depth_kv_e4m3 && append_slot < l && H_kv != H) return MODA_ERR_BAD_SLOT;
+    if (int rc = check_device()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    void* slot = static_cast<uint8_t*>(append_cache_e4m3) + size_t(append_slot) * cache8_slot_bytes(B, T, H_kv, d);
+    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, slot, st, kCacheE4m3)
+                    : launch_fwd<64>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, slot, st, kCacheE4m3);
 }
 
 int moda_attn_bwd_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,

@@ -111,7 +111,7 @@ struct FwdParams {
     // "Write" step of the depth stream fused into the forward: when not null, the base of one cache slot
     // (H / G heads) into which every CTA copies the K and V rows of its own 128 positions, straight from the
     // shared-memory tiles of its last (diagonal) key tile.  Only with kv_off == 0; the first head of a group writes.
-    __nv_bfloat16* append_slot;
+    void* append_slot;               // bf16 slot, or (e4m3 instantiations) a slot of codes + row scales
 };
 
 // Which (batch, query head, key/value head, query tile) a CTA works on.  The G query heads that
@@ -162,6 +162,50 @@ __device__ __forceinline__ void append_rows_to_slot(__nv_bfloat16* slot, const u
     for (int c = 0; c < CH; ++c) {
         dK[c * kTileRows] = *reinterpret_cast<const uint4*>(sK + swz_chunk_offset(r, c));
         dV[c * kTileRows] = *reinterpret_cast<const uint4*>(sV + swz_chunk_offset(r, c));
+    }
+}
+
+// The same write step into an e4m3 cache (moda_cache.cuh): the thread quantises its K row and its V row exactly as
+// depth_cache_quant_kernel does (row maximum / 448 as the scale, IEEE division, round to nearest even, saturating; a
+// zero row has scale 1), reading the row twice from shared memory instead of holding it in registers.
+template <int D>
+__device__ __forceinline__ void append_rows_to_slot_e4m3(void* slot, const uint8_t* sK, const uint8_t* sV,
+                                                         size_t block_index, int r) {
+    constexpr int CH = D / 8;
+    uint8_t* blk = static_cast<uint8_t*>(slot) + block_index * 2 * cache8_block_bytes(D);
+#pragma unroll 1
+    for (int kv = 0; kv < 2; ++kv, blk += cache8_block_bytes(D)) {
+        const uint8_t* src = kv == 0 ? sK : sV;
+        float am = 0.f;
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const uint4 v = *reinterpret_cast<const uint4*>(src + swz_chunk_offset(r, c));
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) am = fmaxf(am, fmaxf(fabsf(bf16_lo_to_f32(w[k])), fabsf(bf16_hi_to_f32(w[k]))));
+        }
+        const float scale = am > 0.f ? __fdiv_rn(am, 448.f) : 1.f;
+        uint4* codes = reinterpret_cast<uint4*>(blk) + r;
+#pragma unroll
+        for (int g = 0; g < D / 16; ++g) {                // 16 features per chunk of codes = two 16-byte bf16 chunks
+            uint32_t cw[4];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const uint4 v = *reinterpret_cast<const uint4*>(src + swz_chunk_offset(r, 2 * g + half));
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    uint16_t lo, hi;
+                    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo)
+                        : "f"(__fdiv_rn(bf16_hi_to_f32(w[2 * k]), scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w[2 * k]), scale)));
+                    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi)
+                        : "f"(__fdiv_rn(bf16_hi_to_f32(w[2 * k + 1]), scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w[2 * k + 1]), scale)));
+                    cw[2 * half + k] = uint32_t(lo) | (uint32_t(hi) << 16);
+                }
+            }
+            codes[g * kTileRows] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+        }
+        reinterpret_cast<float*>(blk + size_t(kTileRows) * D)[r] = scale;
     }
 }
 
@@ -389,7 +433,11 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             // sits in its stages: the waits are on phases that have completed and make the TMA writes visible here.
             const int jl = jbase + n_kv - 1;
             mbar_wait2(bar(kBarKFull + jl % KST), (jl / KST) & 1, bar(kBarVFull + (jl & 1)), (jl >> 1) & 1, abort_flag, 23, 24);
-            append_rows_to_slot<D>(p.append_slot, smem + L::kK + (jl % KST) * L::kTileBytes, smem + L::kV + (jl & 1) * L::kTileBytes,
+            if constexpr (FP8)
+                append_rows_to_slot_e4m3<D>(p.append_slot, smem + L::kK + (jl % KST) * L::kTileBytes, smem + L::kV + (jl & 1) * L::kTileBytes,
+                                            (size_t(b) * Hk + hk) * nq + qt, r);
+            else
+            append_rows_to_slot<D>(static_cast<__nv_bfloat16*>(p.append_slot), smem + L::kK + (jl % KST) * L::kTileBytes, smem + L::kV + (jl & 1) * L::kTileBytes,
                                    (size_t(b) * Hk + hk) * nq + qt, r);
         }
         // The tile is done: the Q buffer (output staging), the K / V stages the slot was copied from, O and the depth

@@ -568,7 +568,11 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             const int j = n_kv - 1, st = j % L::kStages;
             mbar_wait(bar(k2BarOFinal), 0, abort_flag, 22);
             mbar_wait2(bar(k2BarKFull + st), (j / L::kStages) & 1, bar(k2BarVFull + st), (j / L::kStages) & 1, abort_flag, 23, 24);
-            append_rows_to_slot<D>(p.append_slot, smem + L::kK + st * L::kKeyTileBytes, smem + L::kV + st * L::kKeyTileBytes,
+            if constexpr (FP8)
+                append_rows_to_slot_e4m3<D>(p.append_slot, smem + L::kK + st * L::kKeyTileBytes, smem + L::kV + st * L::kKeyTileBytes,
+                                            (size_t(b) * (p.H / p.G) + hk) * nq + qt, tid - 256);
+            else
+            append_rows_to_slot<D>(static_cast<__nv_bfloat16*>(p.append_slot), smem + L::kK + st * L::kKeyTileBytes, smem + L::kV + st * L::kKeyTileBytes,
                                    (size_t(b) * (p.H / p.G) + hk) * nq + qt, tid - 256);
         }
     } else {

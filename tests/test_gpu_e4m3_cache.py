@@ -177,3 +177,47 @@ def test_c3_full_size_one_head_slice():
     got = (dQ[b:b + 1, :, h:h + 1], dK[b:b + 1, :, h:h + 1], dV[b:b + 1, :, h:h + 1],
            dKd[:, b:b + 1, :, h:h + 1], dVd[:, b:b + 1, :, h:h + 1])
     assert_grads_close(got, ref, "c3 l = 16, e4m3 cache")
+
+
+@pytest.mark.parametrize("B,T,H,Hk,d,l", [(1, 128, 1, 1, 64, 0), (2, 300, 2, 2, 128, 3), (1, 1000, 4, 2, 64, 5), (1, 257, 8, 1, 128, 2),
+                                          (3, 2190, 16, 16, 128, 3), (1, 640, 3, 3, 64, 33)])
+def test_forward_writes_its_own_slot_in_e4m3(B, T, H, Hk, d, l):
+    """moda_attn_fwd_append_e4m3: same output as moda_attn_fwd_e4m3, and the slot holds byte for byte what the quantising
+    append stores from K, V (tail rows of a ragged last tile: code 0, scale 1); the other slots are untouched."""
+    scale = d ** -0.5
+    x = synthetic.make_gqa(B, T, H, Hk, d, l, seed=29, device="cuda")
+    want = moda.alloc_depth_cache_e4m3(B, T, Hk, d, l + 1)
+    got = moda.alloc_depth_cache_e4m3(B, T, Hk, d, l + 1)
+    for c in (want, got):
+        c.fill_(0xAB)
+        for i in range(l):
+            moda.moda_depth_cache_append_e4m3(c, i, x["Kd"][i].contiguous(), x["Vd"][i].contiguous())
+    moda.moda_depth_cache_append_e4m3(want, l, x["K"], x["V"])
+    O0, LSE0 = moda.moda_attn_fwd_e4m3(x["Q"], x["K"], x["V"], want, l, scale)
+    O1, LSE1 = moda.moda_attn_fwd_append_e4m3(x["Q"], x["K"], x["V"], got, l, scale, got, l)
+    assert moda.moda_last_status() == 0
+    assert torch.equal(got, want), "slot written by the forward differs from moda_depth_cache_append_e4m3"
+    assert torch.equal(O0, O1) and torch.equal(LSE0, LSE1)
+
+
+def test_e4m3_slot_buffer_with_in_place_eviction():
+    # a buffer of two e4m3 slots as a sliding window: every layer attends to the two layers before it and writes its own
+    # K, V over the older one in the same launch; checked against the oracle on the dequantised slots
+    B, T, H, d, S, n_layers = 1, 300, 2, 128, 2, 5
+    scale = d ** -0.5
+    layers = [synthetic.make_gqa(B, T, H, H, d, 0, seed=60 + n, device="cuda") for n in range(n_layers)]
+    cache = moda.alloc_depth_cache_e4m3(B, T, H, d, S)
+    owner = {}                                            # slot -> layer it holds
+    for n, x in enumerate(layers):
+        l = len(owner)
+        slot = n % S
+        held = [owner[i] for i in range(l)]               # in slot order (the operator does not depend on it)
+        O, LSE = moda.moda_attn_fwd_append_e4m3(x["Q"], x["K"], x["V"], cache, l, scale, cache, slot)
+        assert moda.moda_last_status() == 0
+        deq = lambda t: orc.dequantize_e4m3_rows(*orc.quantize_e4m3_rows(f64(t)))
+        Kd = np.stack([deq(layers[m]["K"]) for m in held]) if held else np.zeros((0, B, T, H, d))
+        Vd = np.stack([deq(layers[m]["V"]) for m in held]) if held else np.zeros((0, B, T, H, d))
+        O_ref, LSE_ref = orc.forward(f64(x["Q"]), f64(x["K"]), f64(x["V"]), Kd, Vd, scale)
+        assert_forward_close(O, LSE, O_ref, LSE_ref, f"layer {n} over layers {held}")
+        owner[slot] = n
+    assert sorted(owner.values()) == [n_layers - 2, n_layers - 1]

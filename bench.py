@@ -173,7 +173,8 @@ class Layer:
             self.cache = alloc(w.B, w.T, w.H, w.d, w.l, device)
             for i in range(w.l):
                 append(self.cache, i, synthetic.tensor(w, "Kd", seed, i, device), synthetic.tensor(w, "Vd", seed, i, device))
-        self.next_slot = moda.alloc_depth_cache(w.B, w.T, w.H, w.d, 1, device)   # slot this layer writes for later layers
+        # slot this layer writes for later layers (same format as the cache it reads)
+        self.next_slot = (moda.alloc_depth_cache_e4m3 if e4m3 else moda.alloc_depth_cache)(w.B, w.T, w.H, w.d, 1, device)
         self.O = torch.empty_like(self.q)
         self.LSE = torch.empty((w.B, w.H, w.T), dtype=torch.float32, device=device)
         if with_backward:
@@ -185,8 +186,8 @@ class Layer:
 
     def fwd_append(self):
         """Forward with the depth stream's write step fused in: this layer's K, V go to the slot the later layers read."""
-        self.moda.moda_attn_fwd_append(self.q, self.k, self.v, self.cache, self.w.l, self.w.scale, self.next_slot, 0,
-                                       O=self.O, LSE=self.LSE)
+        f = self.moda.moda_attn_fwd_append_e4m3 if self.e4m3 else self.moda.moda_attn_fwd_append
+        f(self.q, self.k, self.v, self.cache, self.w.l, self.w.scale, self.next_slot, 0, O=self.O, LSE=self.LSE)
 
     def fwd(self):
         f = self.moda.moda_attn_fwd_e4m3 if self.e4m3 else self.moda.moda_attn_fwd

@@ -256,6 +256,8 @@ int launch_fwd(const void* Q, const void* K, const void* V, const void* depth_kv
     }
     FwdParams p;
     p.Q = static_cast<const __nv_bfloat16*>(Q);
+    p.K = static_cast<const __nv_bfloat16*>(K);
+    p.V = static_cast<const __nv_bfloat16*>(V);
     p.depth_kv = depth_kv;
     p.O = static_cast<__nv_bfloat16*>(O);
     p.LSE = LSE;

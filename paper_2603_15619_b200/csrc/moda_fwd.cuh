@@ -11,8 +11,7 @@
 //                        keeps the running (m, l) of the online softmax in registers, writes
 //                        P_j = exp2(S_j c - m) as packed bf16 back into the TMEM columns of
 //                        S_j, rescales the O accumulator only when the running maximum grew
-//                        by more than 2^8, and runs the epilogue (output tile, LSE, and the write of the
-//                        layer's own K, V rows into a cache slot when the call asks for it).
+//                        by more than 2^8, and runs the epilogue (output tile, LSE).
 //   warps 4-7  depth     one thread per query row (its q comes straight from global memory).  Reads the
 //                        row's l depth keys/values (bf16, or e4m3 codes with row scales) from
 //                        a shared-memory ring that warp 10 fills with 16 KiB bulk copies of
@@ -20,7 +19,8 @@
 //                        (m_d, l_d, o_d) on the CUDA cores (slots in groups of 32, online
 //                        softmax over the groups) and parks o_d in TMEM.  Merging two partial
 //                        softmax states is exact, so the epilogue obtains the single softmax
-//                        over sequence and depth keys that the paper defines.
+//                        over sequence and depth keys that the paper defines.  Afterwards it writes the
+//                        layer's own K, V rows into a cache slot when the call asks for it.
 //   warp 8     TMA       one lane streams the Q tile and the K_j / V_j tiles (128B swizzle)
 //                        through two-stage rings.
 //   warp 9     MMA (S)   issues S_j = Q K_j^T (operands in shared memory); owns the TMEM
@@ -91,7 +91,7 @@ enum FwdBar : int {
     kBarDrain = 16,
     kBarDFull = 17,   // +ring stage (<= 6): depth unit landed
     kBarDEmpty = 23,  // +ring stage (<= 6): all 128 depth threads have read the unit
-    kBarTileDone = 29,  // one phase per query tile of the CTA: its epilogue (output stored, slot written) is complete
+    kBarTileDone = 29,  // one phase per query tile of the CTA: its epilogue (output stored) is complete
 };
 
 // Depth slots per group of the forward's online softmax over the depth keys (one group's scores fit
@@ -100,6 +100,8 @@ constexpr int kFwdDepthGroup = 32;
 
 struct FwdParams {
     const __nv_bfloat16* Q;          // [B][T][H][d]: the depth warps read their rows straight from global memory
+    const __nv_bfloat16* K;          // [B][T_kv][H/G][d]: the write step reads the rows of the CTA's own positions from here
+    const __nv_bfloat16* V;
     const void* depth_kv;            // cache layout (bf16, or e4m3 codes + scales), >= l slots (unused when l == 0)
     __nv_bfloat16* O;
     float* LSE;
@@ -109,8 +111,8 @@ struct FwdParams {
     int pair;                        // nonzero: a CTA takes a pair of query tiles (see pair_coord), else one tile, heaviest first
     float scale_log2;                // scale * log2(e)
     // "Write" step of the depth stream fused into the forward: when not null, the base of one cache slot
-    // (H / G heads) into which every CTA copies the K and V rows of its own 128 positions, straight from the
-    // shared-memory tiles of its last (diagonal) key tile.  Only with kv_off == 0; the first head of a group writes.
+    // (H / G heads) into which every CTA copies the K and V rows of its own positions (append_rows_from_global).
+    // Only with kv_off == 0; the first head of a group writes.
     void* append_slot;               // bf16 slot, or (e4m3 instantiations) a slot of codes + row scales
 };
 
@@ -149,63 +151,63 @@ __device__ __forceinline__ uint32_t swz_chunk_offset(int r, int c) {
     return uint32_t(c >> 3) * uint32_t(kTileRows * 128) + uint32_t(r) * 128u + (uint32_t((c & 7) ^ (r & 7)) << 4);
 }
 
-// Copies one thread's row of the CTA's diagonal K and V tiles (TMA-written, 128-byte swizzled) into the cache
-// block (b, hk, qt) of a slot: chunk c of row r goes to [c][r], so a warp writes 512 contiguous bytes per chunk.
-// Rows of a ragged last tile were zero-filled by TMA, which is what the cache wants in its tail rows.
-template <int D>
-__device__ __forceinline__ void append_rows_to_slot(__nv_bfloat16* slot, const uint8_t* sK, const uint8_t* sV,
-                                                    size_t block_index, int r) {
+// "Write" step of the depth stream inside the forward: one thread copies the K row and the V row of one of the CTA's own
+// positions from the input tensors into block (b, hk, qt) of a slot: chunk c of row r goes to [c][r], so a warp writes 512
+// contiguous bytes per chunk.  The rows are read from global memory (the key loop loads the same rows as its diagonal
+// tile, so they come from L2 or cost one more read of 4 d bytes per position), which lets the depth warps do this as
+// soon as they have finished reading the cache, off the path of the key loop and the epilogue.  Rows past T are written
+// as zeros (e4m3: code 0, scale 1), which is what the cache wants in its tail rows.
+// FP8: the slot is in the e4m3 layout (moda_cache.cuh) and the row is quantised exactly as depth_cache_quant_kernel does
+// (row maximum / 448 as the scale, IEEE division, round to nearest even, saturating; a zero row has scale 1).
+template <int D, bool FP8>
+__device__ __forceinline__ void append_rows_from_global(void* slot, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                                                        int b, int hk, int Hk, int T, int nq, int qt, int r) {
     constexpr int CH = D / 8;
-    uint4* dK = reinterpret_cast<uint4*>(slot) + block_index * 2 * (kTileRows * CH) + r;
-    uint4* dV = dK + kTileRows * CH;
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-        dK[c * kTileRows] = *reinterpret_cast<const uint4*>(sK + swz_chunk_offset(r, c));
-        dV[c * kTileRows] = *reinterpret_cast<const uint4*>(sV + swz_chunk_offset(r, c));
-    }
-}
-
-// The same write step into an e4m3 cache (moda_cache.cuh): the thread quantises its K row and its V row exactly as
-// depth_cache_quant_kernel does (row maximum / 448 as the scale, IEEE division, round to nearest even, saturating; a
-// zero row has scale 1), reading the row twice from shared memory instead of holding it in registers.
-template <int D>
-__device__ __forceinline__ void append_rows_to_slot_e4m3(void* slot, const uint8_t* sK, const uint8_t* sV,
-                                                         size_t block_index, int r) {
-    constexpr int CH = D / 8;
-    uint8_t* blk = static_cast<uint8_t*>(slot) + block_index * 2 * cache8_block_bytes(D);
+    const int t = qt * kTileRows + r;
+    const bool valid = t < T;
+    const size_t block_index = (size_t(b) * Hk + hk) * nq + qt;
+    const size_t row = ((size_t(b) * T + (valid ? t : 0)) * Hk + hk) * CH;
 #pragma unroll 1
-    for (int kv = 0; kv < 2; ++kv, blk += cache8_block_bytes(D)) {
-        const uint8_t* src = kv == 0 ? sK : sV;
-        float am = 0.f;
+    for (int kv = 0; kv < 2; ++kv) {
+        const uint4* src = reinterpret_cast<const uint4*>(kv == 0 ? K : V) + row;
+        uint4 x[CH];
 #pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const uint4 v = *reinterpret_cast<const uint4*>(src + swz_chunk_offset(r, c));
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        for (int c = 0; c < CH; ++c) x[c] = valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+        if constexpr (!FP8) {
+            uint4* dst = reinterpret_cast<uint4*>(slot) + (block_index * 2 + kv) * (kTileRows * CH) + r;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) am = fmaxf(am, fmaxf(fabsf(bf16_lo_to_f32(w[k])), fabsf(bf16_hi_to_f32(w[k]))));
-        }
-        const float scale = am > 0.f ? __fdiv_rn(am, 448.f) : 1.f;
-        uint4* codes = reinterpret_cast<uint4*>(blk) + r;
+            for (int c = 0; c < CH; ++c) dst[c * kTileRows] = x[c];
+        } else {
+            uint8_t* blk = static_cast<uint8_t*>(slot) + (block_index * 2 + kv) * cache8_block_bytes(D);
+            float am = 0.f;
 #pragma unroll
-        for (int g = 0; g < D / 16; ++g) {                // 16 features per chunk of codes = two 16-byte bf16 chunks
-            uint32_t cw[4];
+            for (int c = 0; c < CH; ++c) {
+                const uint32_t w[4] = {x[c].x, x[c].y, x[c].z, x[c].w};
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const uint4 v = *reinterpret_cast<const uint4*>(src + swz_chunk_offset(r, 2 * g + half));
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int k = 0; k < 2; ++k) {
-                    uint16_t lo, hi;
-                    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo)
-                        : "f"(__fdiv_rn(bf16_hi_to_f32(w[2 * k]), scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w[2 * k]), scale)));
-                    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi)
-                        : "f"(__fdiv_rn(bf16_hi_to_f32(w[2 * k + 1]), scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w[2 * k + 1]), scale)));
-                    cw[2 * half + k] = uint32_t(lo) | (uint32_t(hi) << 16);
-                }
+                for (int k = 0; k < 4; ++k) am = fmaxf(am, fmaxf(fabsf(bf16_lo_to_f32(w[k])), fabsf(bf16_hi_to_f32(w[k]))));
             }
-            codes[g * kTileRows] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+            const float scale = am > 0.f ? __fdiv_rn(am, 448.f) : 1.f;
+            uint4* codes = reinterpret_cast<uint4*>(blk) + r;
+#pragma unroll
+            for (int g = 0; g < D / 16; ++g) {            // 16 features per chunk of codes = two 16-byte bf16 chunks
+                uint32_t cw[4];
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const uint32_t w[4] = {x[2 * g + half].x, x[2 * g + half].y, x[2 * g + half].z, x[2 * g + half].w};
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        uint16_t lo, hi;
+                        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo)
+                            : "f"(__fdiv_rn(bf16_hi_to_f32(w[2 * k]), scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w[2 * k]), scale)));
+                        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi)
+                            : "f"(__fdiv_rn(bf16_hi_to_f32(w[2 * k + 1]), scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w[2 * k + 1]), scale)));
+                        cw[2 * half + k] = uint32_t(lo) | (uint32_t(hi) << 16);
+                    }
+                }
+                codes[g * kTileRows] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+            }
+            reinterpret_cast<float*>(blk + size_t(kTileRows) * D)[r] = scale;
         }
-        reinterpret_cast<float*>(blk + size_t(kTileRows) * D)[r] = scale;
     }
 }
 
@@ -428,20 +430,8 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             tma_store_commit();
             tma_store_wait_all();
         }
-        if (p.append_slot != nullptr && h == hk * p.G) {
-            // Every MMA of the tile has completed, so no load is in flight and its last key tile (the diagonal one)
-            // sits in its stages: the waits are on phases that have completed and make the TMA writes visible here.
-            const int jl = jbase + n_kv - 1;
-            mbar_wait2(bar(kBarKFull + jl % KST), (jl / KST) & 1, bar(kBarVFull + (jl & 1)), (jl >> 1) & 1, abort_flag, 23, 24);
-            if constexpr (FP8)
-                append_rows_to_slot_e4m3<D>(p.append_slot, smem + L::kK + (jl % KST) * L::kTileBytes, smem + L::kV + (jl & 1) * L::kTileBytes,
-                                            (size_t(b) * Hk + hk) * nq + qt, r);
-            else
-            append_rows_to_slot<D>(static_cast<__nv_bfloat16*>(p.append_slot), smem + L::kK + (jl % KST) * L::kTileBytes, smem + L::kV + (jl & 1) * L::kTileBytes,
-                                   (size_t(b) * Hk + hk) * nq + qt, r);
-        }
-        // The tile is done: the Q buffer (output staging), the K / V stages the slot was copied from, O and the depth
-        // partial in tensor memory may be reused for the CTA's next tile.
+        // The tile is done: the Q buffer (output staging), O and the depth partial in tensor memory may be reused for the
+        // CTA's next tile.
         tc_fence_before_sync();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (tid == 0) mbar_arrive(bar(kBarTileDone));
@@ -687,6 +677,11 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             mbar_arrive(bar(kBarDepth));
             }
         }
+        if (p.append_slot != nullptr && h == hk * p.G) {
+            // the write step: every read of the depth cache by this CTA is complete here, so the slot may be one that was read
+            for (int t = 0; t < n_tiles; ++t)
+                append_rows_from_global<D, FP8>(p.append_slot, p.K, p.V, b, hk, Hk, p.T, nq, tile_qt(t), tid - 128);
+        }
     } else {
       setmaxnreg_dec<72>();   // one instruction for the whole producer warpgroup (warps 8-11)
       if (warp == 8) {
@@ -698,7 +693,7 @@ moda_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             int jbase = 0;
             for (int t = 0; t < n_tiles; ++t) {
                 const int q0 = tile_qt(t) * kTileRows, n_kv = tile_nkv(t);
-                // the Q buffer doubles as the output staging of the previous tile, and the slot write reads its last stages
+                // the Q buffer doubles as the output staging of the previous tile
                 if (t > 0) mbar_wait(bar(kBarTileDone), (t - 1) & 1, abort_flag, 33);
                 mbar_arrive_expect_tx(bar(kBarQ), L::kTileBytes);
 #pragma unroll

@@ -564,16 +564,8 @@ moda_fwd2_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             mbar_arrive(bar(k2BarDepth));
         }
         if (p.append_slot != nullptr && h == hk * p.G) {
-            // the "write" step of the depth stream, from the tiles of the diagonal key tile (see moda_fwd_kernel)
-            const int j = n_kv - 1, st = j % L::kStages;
-            mbar_wait(bar(k2BarOFinal), 0, abort_flag, 22);
-            mbar_wait2(bar(k2BarKFull + st), (j / L::kStages) & 1, bar(k2BarVFull + st), (j / L::kStages) & 1, abort_flag, 23, 24);
-            if constexpr (FP8)
-                append_rows_to_slot_e4m3<D>(p.append_slot, smem + L::kK + st * L::kKeyTileBytes, smem + L::kV + st * L::kKeyTileBytes,
-                                            (size_t(b) * (p.H / p.G) + hk) * nq + qt, tid - 256);
-            else
-            append_rows_to_slot<D>(static_cast<__nv_bfloat16*>(p.append_slot), smem + L::kK + st * L::kKeyTileBytes, smem + L::kV + st * L::kKeyTileBytes,
-                                   (size_t(b) * (p.H / p.G) + hk) * nq + qt, tid - 256);
+            // the "write" step of the depth stream (see moda_fwd_kernel): after this CTA's reads of the depth cache
+            append_rows_from_global<D, FP8>(p.append_slot, p.K, p.V, b, hk, p.H / p.G, p.T, nq, qt, tid - 256);
         }
     } else {
       setmaxnreg_dec<40>();   // one instruction for the whole producer warpgroup (warps 12-15)

@@ -366,7 +366,8 @@ int moda_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, co
  * moda_attn_fwd_e4m3 that also writes the layer's own K, V as slot `append_slot` of an e4m3 cache, from the key / value
  * tiles the kernel holds (the write step of Sec. 2.2 fused into the forward, as moda_attn_fwd_append does for a bf16
  * cache).  The slot receives byte for byte what moda_depth_cache_append_e4m3(append_cache_e4m3, ..., append_slot, K, V)
- * stores.  Rules for writing a slot that the call also reads as in moda_attn_fwd_append.
+ * stores.  Rules for writing a slot that the call also reads as in moda_attn_fwd_append.  One launch for T >= 32768; on
+ * shorter sequences the quantiser runs as a second launch behind the forward (cheaper there), with the same result.
  */
 int moda_attn_fwd_append_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,
                               int B, int T, int H, int H_kv, int d, int l, float scale,
@@ -468,7 +469,7 @@ int moda_kv_project_append(const void* X, const void* Wk, const void* Wv,
 /*
  * The same projection with the slot written into an e4m3 depth cache (moda_depth_cache_e4m3_bytes(B, T, H_kv, d, .)):
  * codes and one fp32 scale per row, bit for bit what moda_depth_cache_append_e4m3(cache_e4m3, ..., slot, K_out, V_out)
- * would store from the bf16-rounded K and V (row maximum / 448 as the scale, IEEE division, round to nearest even,
+ * would store from the bf16-rounded K and V (row maximum / 448 as the scale, correctly rounded quotients, round to nearest even,
  * saturating; a zero row has scale 1).  K_out, V_out stay bf16 and optional.  Everything else as above.
  */
 int moda_kv_project_append_e4m3(const void* X, const void* Wk, const void* Wv,

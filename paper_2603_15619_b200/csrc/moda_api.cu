@@ -977,8 +977,15 @@ int moda_attn_fwd_append_e4m3(const void* Q, const void* K, const void* V, const
     if (int rc = check_device()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     void* slot = static_cast<uint8_t*>(append_cache_e4m3) + size_t(append_slot) * cache8_slot_bytes(B, T, H_kv, d);
-    return d == 128 ? launch_fwd<128>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, slot, st, kCacheE4m3)
-                    : launch_fwd<64>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, slot, st, kCacheE4m3);
+    // Quantising a row costs the depth warps about as many instructions as eight depth slots do.  On long sequences that
+    // disappears under the key loop (64K: + 0.07 ms against 0.19 ms for a separate pass); on short ones the depth warps
+    // set the pace and the separate HBM-bound pass is cheaper (8K, l = 16: 0.06 ms against + 0.14 ms), so the quantiser
+    // then runs as its own launch behind the forward (same bytes; still after every read of the cache by this call).
+    const bool fused = T >= 32768;
+    const int rc = d == 128 ? launch_fwd<128>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, fused ? slot : nullptr, st, kCacheE4m3)
+                            : launch_fwd<64>(Q, K, V, depth_kv_e4m3, B, T, T, H, H_kv, l, scale, O, LSE, fused ? slot : nullptr, st, kCacheE4m3);
+    if (rc != MODA_OK || fused) return rc;
+    return moda_depth_cache_append_e4m3(append_cache_e4m3, B, T, H_kv, d, append_slot, K, V, stream);
 }
 
 int moda_attn_bwd_e4m3(const void* Q, const void* K, const void* V, const void* depth_kv_e4m3,

@@ -131,6 +131,30 @@ __host__ __device__ inline size_t cache8_slot_bytes(int B, int T, int H, int d) 
     return size_t(B) * H * num_tiles(T) * 2 * cache8_block_bytes(d);
 }
 
+// Correctly rounded x / scale for many x and one scale (the quantisers divide every element of a row by the row's scale,
+// and the codes must be those of the IEEE quotient).  With r = RN(1 / scale):  q0 = RN(x r),  e = x - q0 scale (exact in
+// one fused multiply-add),  q = RN(q0 + e r)  is the correctly rounded quotient (Markstein's division theorem) as long
+// as r is within half an ulp of 1 / scale, which fails only for a significand of all ones, and nothing underflows on the
+// way; both cases take the IEEE division instead (scales below 2^-80 are rows of values below 2^-71).  Quotients of
+// magnitude below 2^-10 become code 0 whatever their last bit is.  Three instructions per element instead of a division.
+struct RowDivider {
+    float scale, r;
+    bool slow;
+};
+__device__ __forceinline__ RowDivider make_row_divider(float scale) {
+    RowDivider d;
+    d.scale = scale;
+    d.slow = !(scale >= 8.271806125530277e-25f) || (__float_as_uint(scale) & 0x7fffffu) == 0x7fffffu;
+    d.r = d.slow ? 0.f : __frcp_rn(scale);
+    return d;
+}
+__device__ __forceinline__ float div_rn(float x, const RowDivider& d) {
+    if (d.slow) return __fdiv_rn(x, d.scale);
+    const float q0 = x * d.r;
+    const float e = fmaf(-q0, d.scale, x);
+    return q0 == 0.f ? q0 : fmaf(e, d.r, q0);      // a zero keeps the sign of x, as the IEEE quotient does (-0 has its own code)
+}
+
 // One CTA quantises one (b, h, tile, kv) block of a [B][T][H][d] tensor into a slot.  256 threads: thread
 // (row r, half hf) owns d/2 features of its row; the two halves of a row meet in shared memory for the row maximum.
 template <int D>
@@ -173,6 +197,7 @@ depth_cache_quant_kernel(uint8_t* __restrict__ slot_base, const uint4* __restric
     __syncthreads();
     am = fmaxf(amax2[0][r], amax2[1][r]);
     const float scale = am > 0.f ? __fdiv_rn(am, 448.f) : 1.f;
+    const RowDivider dv = make_row_divider(scale);
     uint4* codes = reinterpret_cast<uint4*>(blk);
 #pragma unroll
     for (int g = 0; g < D / 32; ++g) {              // 16 features per output chunk
@@ -181,8 +206,8 @@ depth_cache_quant_kernel(uint8_t* __restrict__ slot_base, const uint4* __restric
         for (int k = 0; k < 4; ++k) {
             const float* xx = x + 16 * g + 4 * k;
             uint16_t lo, hi;
-            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(xx[1], scale)), "f"(__fdiv_rn(xx[0], scale)));
-            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(xx[3], scale)), "f"(__fdiv_rn(xx[2], scale)));
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(div_rn(xx[1], dv)), "f"(div_rn(xx[0], dv)));
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(div_rn(xx[3], dv)), "f"(div_rn(xx[2], dv)));
             w[k] = uint32_t(lo) | (uint32_t(hi) << 16);
         }
         codes[size_t(hf * (D / 32) + g) * kTileRows + r] = make_uint4(w[0], w[1], w[2], w[3]);

@@ -158,7 +158,7 @@ __device__ __forceinline__ uint32_t swz_chunk_offset(int r, int c) {
 // soon as they have finished reading the cache, off the path of the key loop and the epilogue.  Rows past T are written
 // as zeros (e4m3: code 0, scale 1), which is what the cache wants in its tail rows.
 // FP8: the slot is in the e4m3 layout (moda_cache.cuh) and the row is quantised exactly as depth_cache_quant_kernel does
-// (row maximum / 448 as the scale, IEEE division, round to nearest even, saturating; a zero row has scale 1).
+// (row maximum / 448 as the scale, correctly rounded quotients, round to nearest even, saturating; a zero row has scale 1).
 template <int D, bool FP8>
 __device__ __forceinline__ void append_rows_from_global(void* slot, const __nv_bfloat16* K, const __nv_bfloat16* V,
                                                         int b, int hk, int Hk, int T, int nq, int qt, int r) {
@@ -187,6 +187,7 @@ __device__ __forceinline__ void append_rows_from_global(void* slot, const __nv_b
                 for (int k = 0; k < 4; ++k) am = fmaxf(am, fmaxf(fabsf(bf16_lo_to_f32(w[k])), fabsf(bf16_hi_to_f32(w[k]))));
             }
             const float scale = am > 0.f ? __fdiv_rn(am, 448.f) : 1.f;
+            const RowDivider dv = make_row_divider(scale);
             uint4* codes = reinterpret_cast<uint4*>(blk) + r;
 #pragma unroll
             for (int g = 0; g < D / 16; ++g) {            // 16 features per chunk of codes = two 16-byte bf16 chunks
@@ -198,9 +199,9 @@ __device__ __forceinline__ void append_rows_from_global(void* slot, const __nv_b
                     for (int k = 0; k < 2; ++k) {
                         uint16_t lo, hi;
                         asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo)
-                            : "f"(__fdiv_rn(bf16_hi_to_f32(w[2 * k]), scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w[2 * k]), scale)));
+                            : "f"(div_rn(bf16_hi_to_f32(w[2 * k]), dv)), "f"(div_rn(bf16_lo_to_f32(w[2 * k]), dv)));
                         asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi)
-                            : "f"(__fdiv_rn(bf16_hi_to_f32(w[2 * k + 1]), scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w[2 * k + 1]), scale)));
+                            : "f"(div_rn(bf16_hi_to_f32(w[2 * k + 1]), dv)), "f"(div_rn(bf16_lo_to_f32(w[2 * k + 1]), dv)));
                         cw[2 * half + k] = uint32_t(lo) | (uint32_t(hi) << 16);
                     }
                 }

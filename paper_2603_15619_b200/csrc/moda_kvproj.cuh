@@ -218,6 +218,7 @@ moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_co
                                             : reinterpret_cast<uint4*>(p.slot) + blk_index * (kTileRows * CH) + r;
                     uint8_t* stage = smem + L::kOut + j * (kTileRows * D * 2);
                     float q_scale = 1.f;
+                    RowDivider dv = make_row_divider(1.f);
                     if constexpr (FP8) {
                         float am = 0.f;
 #pragma unroll
@@ -232,6 +233,7 @@ moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_co
                             }
                         }
                         q_scale = am > 0.f ? __fdiv_rn(am, 448.f) : 1.f;
+                        dv = make_row_divider(q_scale);
                         if (slot_blk != nullptr)
                             reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(slot_blk - r) + size_t(kTileRows) * D)[r] = q_scale;
                     }
@@ -253,9 +255,9 @@ moda_kv_project_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_co
                                     const uint32_t w0 = w[8 * g + 2 * k], w1 = w[8 * g + 2 * k + 1];
                                     uint16_t lo, hi;
                                     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo)
-                                        : "f"(__fdiv_rn(bf16_hi_to_f32(w0), q_scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w0), q_scale)));
+                                        : "f"(div_rn(bf16_hi_to_f32(w0), dv)), "f"(div_rn(bf16_lo_to_f32(w0), dv)));
                                     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi)
-                                        : "f"(__fdiv_rn(bf16_hi_to_f32(w1), q_scale)), "f"(__fdiv_rn(bf16_lo_to_f32(w1), q_scale)));
+                                        : "f"(div_rn(bf16_hi_to_f32(w1), dv)), "f"(div_rn(bf16_lo_to_f32(w1), dv)));
                                     cw[k] = uint32_t(lo) | (uint32_t(hi) << 16);
                                 }
                                 if (slot_blk != nullptr) slot_blk[(c * 2 + g) * kTileRows] = make_uint4(cw[0], cw[1], cw[2], cw[3]);

@@ -180,7 +180,9 @@ def test_c3_full_size_one_head_slice():
 
 
 @pytest.mark.parametrize("B,T,H,Hk,d,l", [(1, 128, 1, 1, 64, 0), (2, 300, 2, 2, 128, 3), (1, 1000, 4, 2, 64, 5), (1, 257, 8, 1, 128, 2),
-                                          (3, 2190, 16, 16, 128, 3), (1, 640, 3, 3, 64, 33)])
+                                          (3, 2190, 16, 16, 128, 3), (1, 640, 3, 3, 64, 33),
+                                          # from 32768 positions on the quantiser runs inside the forward kernel (ragged tail, grouped heads)
+                                          (1, 32768 + 70, 2, 1, 128, 2), (1, 32768, 2, 2, 64, 3)])
 def test_forward_writes_its_own_slot_in_e4m3(B, T, H, Hk, d, l):
     """moda_attn_fwd_append_e4m3: same output as moda_attn_fwd_e4m3, and the slot holds byte for byte what the quantising
     append stores from K, V (tail rows of a ragged last tile: code 0, scale 1); the other slots are untouched."""
@@ -221,3 +223,32 @@ def test_e4m3_slot_buffer_with_in_place_eviction():
         assert_forward_close(O, LSE, O_ref, LSE_ref, f"layer {n} over layers {held}")
         owner[slot] = n
     assert sorted(owner.values()) == [n_layers - 2, n_layers - 1]
+
+
+def test_quantiser_is_bit_exact_over_a_wide_range_of_rows_and_on_ties():
+    """The kernels take the quotient x / scale as a reciprocal and two fused steps; the codes must still be those of the
+    IEEE quotient that the oracle rounds.  16 M values: rows scaled by powers of two from 2^-100 to 2^100 (the tiny ones
+    take the kernels' IEEE fallback), rows whose scale is a power of two and whose entries sit on rounding ties of the
+    format, rows with one entry far above the rest, and plain Gaussian rows."""
+    B, T, H, d, l = 2, 4096, 4, 128, 2
+    g = torch.Generator(device="cuda").manual_seed(77)
+    X = torch.randn((2, l, B, T, H, d), device="cuda", generator=g)
+    expo = torch.randint(-100, 101, (2, l, B, T, H, 1), device="cuda", generator=g).float()
+    X = X * torch.exp2(expo)
+    # ties: row maximum 448 * 2^k (scale exactly 2^k), entries = midpoints between neighbouring e4m3 values times 2^k
+    mids = torch.tensor([0.0009765625 * (2 * i + 1) for i in range(8)] + [1.0625 + 0.125 * i for i in range(8)] +
+                        [17.0, 19.0, 21.0, 23.0, 25.0, 27.0, 29.0, 31.0, 208.0 + 8, 240.0 + 8, 416.0 + 16, 448.0 - 16],
+                        device="cuda")
+    tie_rows = mids[torch.randint(0, mids.numel(), (T // 4, d), device="cuda", generator=g)]
+    tie_rows = tie_rows * (torch.randint(0, 2, tie_rows.shape, device="cuda", generator=g).float() * 2 - 1)
+    tie_rows[:, 0] = 448.0
+    X[0, 0, 0, : T // 4, 0, :] = tie_rows * torch.exp2(torch.randint(-20, 21, (T // 4, 1), device="cuda", generator=g).float())
+    X[1, 1, 1, :, 1, 5] = 3.0e4                                           # one dominant entry per row
+    Kd, Vd = X[0].to(torch.bfloat16), X[1].to(torch.bfloat16)
+    cache = build_cache8(Kd, Vd)
+    codes, scales = unpack_cache8(cache, l, B, T, H, d)
+    for kv, Y in enumerate((Kd, Vd)):
+        ref_codes, ref_scale = orc.quantize_e4m3_rows(f64(Y))
+        assert np.array_equal(scales[:, kv], ref_scale), "row scales differ"
+        bad = np.argwhere(codes[:, kv] != ref_codes)
+        assert bad.size == 0, f"{len(bad)} codes differ, first at {bad[0]}: got {codes[:, kv][tuple(bad[0])]}, want {ref_codes[tuple(bad[0])]}"

@@ -136,9 +136,9 @@ int moda_attn_fwd(const void* Q, const void* K, const void* V, const void* depth
  * its own K, V to the depth stream for the layers above it).  Computes exactly what
  * moda_attn_fwd_gqa computes and, in the same launch, stores K and V (bf16 [B][T][H_kv][d]) into slot
  * `append_slot` of `append_cache` in the cache layout, bit for bit what moda_depth_cache_append(
- * append_cache, B, T, H_kv, d, append_slot, K, V) would store: every CTA already holds the K and V
- * rows of its own 128 positions in shared memory (its diagonal key tile) and copies them out, so the
- * separate pass over K and V is gone.  `append_cache` may be the buffer `depth_kv` points to (one
+ * append_cache, B, T, H_kv, d, append_slot, K, V) would store: the depth warps of every CTA copy the
+ * K and V rows of the CTA's own positions (which its key loop loads anyway) once they have read the
+ * cache, so the separate pass over K and V is gone.  `append_cache` may be the buffer `depth_kv` points to (one
  * growing cache per stack, the layer-l call reads slots < l and writes slot l).  Writing a slot that
  * the same call reads (append_cache == depth_kv and append_slot < l) is allowed with one key/value head
  * per query head (H_kv == H): every position's new K, V replace that slot's old ones after the position's
@@ -363,8 +363,8 @@ int moda_attn_bwd_static_scratch(const void* Q, const void* K, const void* V, co
                                  void* dQ, void* dK, void* dV, void* d_depth_kv, void* stream);
 
 /*
- * moda_attn_fwd_e4m3 that also writes the layer's own K, V as slot `append_slot` of an e4m3 cache, from the key / value
- * tiles the kernel holds (the write step of Sec. 2.2 fused into the forward, as moda_attn_fwd_append does for a bf16
+ * moda_attn_fwd_e4m3 that also writes the layer's own K, V as slot `append_slot` of an e4m3 cache
+ * (the write step of Sec. 2.2 fused into the forward, as moda_attn_fwd_append does for a bf16
  * cache).  The slot receives byte for byte what moda_depth_cache_append_e4m3(append_cache_e4m3, ..., append_slot, K, V)
  * stores.  Rules for writing a slot that the call also reads as in moda_attn_fwd_append.  One launch for T >= 32768; on
  * shorter sequences the quantiser runs as a second launch behind the forward (cheaper there), with the same result.
